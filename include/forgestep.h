@@ -1,0 +1,132 @@
+/* forgestep — C ABI of a single-GPU training step (forward, backward, AdamW) of a
+ * Llama-style dense decoder for NVIDIA B200 (sm_100a).
+ *
+ * The operation is the one the ForgeTrain paper optimises: one microbatch through a
+ * decoder-only transformer with grouped-query attention, SwiGLU feed-forward blocks,
+ * pre-normalisation RMSNorm, RoPE and an untied output head (paper appendix "Model
+ * Architectures"), in bf16 with fp32 master weights and fp32 weight gradients, followed
+ * by the fused clip + Adam + bf16 write-back update (paper appendix on framework-level
+ * optimisation, optimizer-tail listing).
+ *
+ * Conventions
+ *   - "dev" pointers are CUDA device pointers, "host" pointers are ordinary host memory.
+ *   - The caller owns every buffer it passes, including the workspace; the library owns
+ *     only its small host-side handle and allocates no device memory.
+ *   - All device work is enqueued on the stream given at ft_init_model.  A call that
+ *     returns a value to the host synchronises that stream once, at its end.
+ *   - Every function returns an ft_status; ft_last_error gives a message.  Nothing aborts
+ *     the process and no kernel traps: device-side problems (a wait that ran out) set a
+ *     status word that the next synchronising call reports as FT_ETIMEOUT.
+ *   - Parameter tensors are addressed by index (ft_param_info gives name and shape) and
+ *     always use the logical row-major [out, in] layout.  Order: "embed", then per layer
+ *     "layers.{l}.norm1", ".wqkv" (rows: q heads, k heads, v heads), ".wo", ".norm2",
+ *     ".wgu" (rows: gate 0..f-1, then up 0..f-1), ".wd"; then "norm_f", "lm_head".
+ */
+#ifndef FORGESTEP_H_
+#define FORGESTEP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct {
+  int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab;
+  int32_t max_batch, max_seq;     /* ft_train_step requires B <= max_batch, S <= max_seq */
+  float rms_eps, rope_theta;
+  float lr, beta1, beta2, adam_eps, weight_decay; /* decay applies to matrices, not to RMSNorm gains */
+  float max_grad_norm;            /* <= 0: clipping off; else coeff = min(1, max/(norm + 1e-6)) */
+  int32_t recompute;              /* 0: keep every layer's activations; 1: keep layer inputs, rerun the layer forward in backward */
+  int32_t debug_taps;             /* 1: keep the backward intermediates of every layer for ft_get_tap (needs recompute = 0) */
+} ft_config;
+
+typedef struct ft_model ft_model;
+
+typedef enum {
+  FT_OK = 0, FT_EINVAL = 1, FT_ENOMEM = 2, FT_ECUDA = 3, FT_ENONFINITE = 4, FT_ETIMEOUT = 5, FT_ENOTFOUND = 6
+} ft_status;
+
+typedef enum { FT_MASTER_F32 = 0, FT_COMPUTE_BF16 = 1, FT_ADAM_M_F32 = 2, FT_ADAM_V_F32 = 3, FT_GRAD_F32 = 4 } ft_kind;
+
+/* Bytes of device workspace a model of this config needs (0 if the config is invalid). */
+size_t ft_workspace_bytes(const ft_config* cfg);
+
+/* Creates a model inside dev_workspace (256-byte aligned, >= ft_workspace_bytes) on the current CUDA
+ * device.  Masters are drawn from a counter-based N(0, 0.02^2) generator keyed by (seed, tensor index,
+ * element index), gains are 1, Adam moments 0, step 0.  cuda_stream is a cudaStream_t (NULL = default). */
+ft_status ft_init_model(const ft_config* cfg, uint64_t seed, void* dev_workspace, size_t bytes,
+                        void* cuda_stream, ft_model** out);
+
+/* One step: forward, loss, backward, global gradient norm, AdamW (paper: train step of the forged engine).
+ * dev_tokens, dev_labels: int32 [B, S] on the device; labels < 0 do not count in the mean loss.
+ * host_loss / host_gnorm: optional host floats; if either is non-NULL the call synchronises the stream. */
+ft_status ft_train_step(ft_model* m, const int32_t* dev_tokens, const int32_t* dev_labels, int32_t B, int32_t S,
+                        float* host_loss, float* host_gnorm);
+
+/* Same call with HOST token and label arrays: copies them to the device, runs the step, returns the loss. */
+ft_status ft_train_step_host(ft_model* m, const int32_t* host_tokens, const int32_t* host_labels, int32_t B,
+                             int32_t S, float* host_loss, float* host_gnorm);
+
+/* Forward and loss only; no gradients, no update. */
+ft_status ft_forward_loss(ft_model* m, const int32_t* dev_tokens, const int32_t* dev_labels, int32_t B, int32_t S,
+                          float* host_loss);
+
+/* Forward and backward without the update: leaves the fp32 gradients readable through FT_GRAD_F32. */
+ft_status ft_forward_backward(ft_model* m, const int32_t* dev_tokens, const int32_t* dev_labels, int32_t B,
+                              int32_t S, float* host_loss);
+
+/* Gradient norm + AdamW on whatever the FT_GRAD_F32 buffers hold (the optimizer in isolation). */
+ft_status ft_apply_update(ft_model* m, float* host_gnorm);
+
+int32_t ft_num_params(const ft_model* m);
+ft_status ft_param_info(const ft_model* m, int32_t i, const char** name, int32_t* ndim, int64_t shape[2]);
+/* Copies one tensor to / from host memory (bytes must equal the tensor's size in that kind).
+ * Setting FT_MASTER_F32 also rewrites the bf16 compute copy with the rounded master. */
+ft_status ft_get_param(ft_model* m, int32_t i, ft_kind kind, void* host_dst, size_t bytes);
+ft_status ft_set_param(ft_model* m, int32_t i, ft_kind kind, const void* host_src, size_t bytes);
+ft_status ft_get_step(const ft_model* m, int64_t* step);
+ft_status ft_set_step(ft_model* m, int64_t step);
+
+/* Named intermediate of the last step, copied to the host.  Forward taps of layer l: "x_in", "h1", "qkv"
+ * ([T, h_q+2h_kv], q and k already rotated), "attn_lse" (fp32 [B, n_h, S]), "o", "x_mid", "h2", "gu"
+ * ([T, 2f]: gate then up), "a", "x_out"; layer -1: "hF", "ce_lse" (fp32 [T]).  Backward taps (debug_taps = 1):
+ * "d_x_out", "d_a", "d_gu", "d_h2", "d_x_mid", "d_o", "d_qkv", "d_h1", "d_x_in"; layer -1: "d_hF".
+ * *dtype: 0 = bf16, 1 = fp32.  bytes is the capacity of host_dst; *out_bytes the size written. */
+ft_status ft_get_tap(ft_model* m, const char* name, int32_t layer, void* host_dst, size_t bytes,
+                     size_t* out_bytes, int32_t* dtype);
+
+const char* ft_last_error(const ft_model* m);
+/* Number of kernels the library launched since the model was created (for launch accounting). */
+int64_t ft_launch_count(const ft_model* m);
+void ft_destroy(ft_model* m);
+
+/* ---- single kernels, for unit parity tests and kernel timing (device pointers; stream = cudaStream_t) ---- */
+
+/* C[M,N] = sum_k A[m,k] B[n,k] on the tcgen05 tensor cores, fp32 accumulation (the projection, FFN and
+ * head contractions of the paper's FLOP table, forward / data-gradient / weight-gradient forms).
+ * a_mn = 0: A stored row-major [M, lda>=K];  a_mn = 1: A stored row-major [K, lda>=M] (contraction over rows).
+ * b_mn likewise for B ([N, ldb>=K] or [K, ldb>=N]).  out_kind: 0 bf16 store, 1 bf16 store of (resid + acc)
+ * with resid bf16 [M, ldc], 2 fp32 store, 3 fp32 accumulate into C.  M, N, K, lda, ldb, ldc multiples of 8. */
+ft_status ft_k_gemm(const void* dev_A, int32_t a_mn, int64_t lda, const void* dev_B, int32_t b_mn, int64_t ldb,
+                    void* dev_C, int64_t ldc, const void* dev_resid, int32_t out_kind,
+                    int32_t M, int32_t N, int32_t K, int32_t* dev_err, void* stream);
+
+/* Causal attention core forward on a packed qkv buffer bf16 [B*S, (n_h + 2 n_kv) * d] (q heads, k heads,
+ * v heads; q, k already rotated): o bf16 [B*S, n_h*d], lse fp32 [B, n_h, S] (natural log). d in {64, 128}. */
+ft_status ft_k_attention_fwd(const void* dev_qkv, void* dev_o, float* dev_lse, int32_t B, int32_t S,
+                             int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, void* stream);
+
+/* Backward of the same: d_qkv bf16 [B*S, (n_h + 2 n_kv) * d] (d_q, d_k NOT rotated back when
+ * dev_cos/dev_sin are NULL; with fp32 tables [S, d/2] they are rotated by the negative angle before the
+ * single rounding).  dev_delta: fp32 scratch [B, n_h, S]. */
+ft_status ft_k_attention_bwd(const void* dev_qkv, const void* dev_o, const void* dev_do, const float* dev_lse,
+                             float* dev_delta, void* dev_dqkv, const float* dev_cos, const float* dev_sin,
+                             int32_t B, int32_t S, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim,
+                             void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FORGESTEP_H_ */

@@ -1,0 +1,244 @@
+"""ctypes binding of libforgestep.so: argument marshalling only.
+
+Every step of the training path runs inside the CUDA library; PyTorch is used here for
+device memory and the stream.  Loading fails loudly when the library has not been built:
+there is no CPU or PyTorch fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, List, Optional, Tuple
+
+import numpy as np
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libforgestep.so")
+_lib = None
+
+FT_OK, FT_EINVAL, FT_ENOMEM, FT_ECUDA, FT_ENONFINITE, FT_ETIMEOUT, FT_ENOTFOUND = range(7)
+STATUS_NAMES = ["FT_OK", "FT_EINVAL", "FT_ENOMEM", "FT_ECUDA", "FT_ENONFINITE", "FT_ETIMEOUT", "FT_ENOTFOUND"]
+KIND_MASTER, KIND_BF16, KIND_ADAM_M, KIND_ADAM_V, KIND_GRAD = range(5)
+
+
+class FtConfig(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_heads", "n_kv_heads", "head_dim", "d_ffn", "vocab",
+                                          "max_batch", "max_seq")] + \
+               [(n, C.c_float) for n in ("rms_eps", "rope_theta", "lr", "beta1", "beta2", "adam_eps", "weight_decay",
+                                         "max_grad_norm")] + \
+               [("recompute", C.c_int32), ("debug_taps", C.c_int32)]
+
+
+class ForgeStepError(RuntimeError):
+    def __init__(self, status: int, msg: str):
+        super().__init__(f"{STATUS_NAMES[status] if 0 <= status < 7 else status}: {msg}")
+        self.status = status
+
+
+def lib():
+    """The loaded C-ABI library (raises if it has not been built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2609_13645_b200.build`")
+        L = C.CDLL(_LIB_PATH)
+        vp, i32, i64, f32p, i32p = C.c_void_p, C.c_int32, C.c_int64, C.POINTER(C.c_float), C.POINTER(C.c_int32)
+        cfgp = C.POINTER(FtConfig)
+        L.ft_workspace_bytes.restype = C.c_size_t
+        L.ft_workspace_bytes.argtypes = [cfgp]
+        L.ft_init_model.argtypes = [cfgp, C.c_uint64, vp, C.c_size_t, vp, C.POINTER(vp)]
+        L.ft_train_step.argtypes = [vp, vp, vp, i32, i32, f32p, f32p]
+        L.ft_train_step_host.argtypes = [vp, vp, vp, i32, i32, f32p, f32p]
+        L.ft_forward_loss.argtypes = [vp, vp, vp, i32, i32, f32p]
+        L.ft_forward_backward.argtypes = [vp, vp, vp, i32, i32, f32p]
+        L.ft_apply_update.argtypes = [vp, f32p]
+        L.ft_num_params.restype = i32
+        L.ft_num_params.argtypes = [vp]
+        L.ft_param_info.argtypes = [vp, i32, C.POINTER(C.c_char_p), i32p, C.POINTER(i64)]
+        L.ft_get_param.argtypes = [vp, i32, i32, vp, C.c_size_t]
+        L.ft_set_param.argtypes = [vp, i32, i32, vp, C.c_size_t]
+        L.ft_get_step.argtypes = [vp, C.POINTER(i64)]
+        L.ft_set_step.argtypes = [vp, i64]
+        L.ft_get_tap.argtypes = [vp, C.c_char_p, i32, vp, C.c_size_t, C.POINTER(C.c_size_t), i32p]
+        L.ft_last_error.restype = C.c_char_p
+        L.ft_last_error.argtypes = [vp]
+        L.ft_launch_count.restype = i64
+        L.ft_launch_count.argtypes = [vp]
+        L.ft_destroy.restype = None
+        L.ft_destroy.argtypes = [vp]
+        L.ft_k_gemm.argtypes = [vp, i32, i64, vp, i32, i64, vp, i64, vp, i32, i32, i32, i32, vp, vp]
+        L.ft_k_attention_fwd.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp]
+        L.ft_k_attention_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]
+        for name in ("ft_init_model", "ft_train_step", "ft_train_step_host", "ft_forward_loss", "ft_forward_backward",
+                     "ft_apply_update", "ft_param_info", "ft_get_param", "ft_set_param", "ft_get_step", "ft_set_step",
+                     "ft_get_tap", "ft_k_gemm", "ft_k_attention_fwd", "ft_k_attention_bwd"):
+            getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def make_config(n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab, max_batch, max_seq, rms_eps=1e-5,
+                rope_theta=1e4, lr=1e-3, beta1=0.9, beta2=0.95, adam_eps=1e-8, weight_decay=0.1, max_grad_norm=0.0,
+                recompute=0, debug_taps=0) -> FtConfig:
+    return FtConfig(n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab, max_batch, max_seq, rms_eps,
+                    rope_theta, lr, beta1, beta2, adam_eps, weight_decay, max_grad_norm, recompute, debug_taps)
+
+
+def workspace_bytes(cfg: FtConfig) -> int:
+    return int(lib().ft_workspace_bytes(C.byref(cfg)))
+
+
+def _stream_ptr():
+    import torch
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def bf16_bits_to_f32(a: np.ndarray) -> np.ndarray:
+    """uint16 bf16 bit patterns -> float32 values (exact)."""
+    return (a.astype(np.uint32) << 16).view(np.float32)
+
+
+class Model:
+    """A decoder + optimizer state living in one torch-allocated workspace on the current CUDA device."""
+
+    def __init__(self, cfg: FtConfig, seed: int = 1234):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("forgestep needs a CUDA device (sm_100a); there is no CPU path")
+        self.cfg = cfg
+        nbytes = workspace_bytes(cfg)
+        if nbytes == 0:
+            raise ForgeStepError(FT_EINVAL, "invalid config")
+        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        self._h = C.c_void_p()
+        st = lib().ft_init_model(C.byref(cfg), C.c_uint64(seed), C.c_void_p(self.workspace.data_ptr()), nbytes,
+                                 _stream_ptr(), C.byref(self._h))
+        self._check(st)
+        self.params: List[Tuple[str, Tuple[int, ...]]] = []
+        for i in range(lib().ft_num_params(self._h)):
+            name, nd, shp = C.c_char_p(), C.c_int32(), (C.c_int64 * 2)()
+            self._check(lib().ft_param_info(self._h, i, C.byref(name), C.byref(nd), shp))
+            self.params.append((name.value.decode(), (int(shp[0]), int(shp[1])) if nd.value == 2 else (int(shp[0]),)))
+        self.index: Dict[str, int] = {n: i for i, (n, _) in enumerate(self.params)}
+
+    def _check(self, st: int):
+        if st != FT_OK:
+            msg = lib().ft_last_error(self._h).decode() if self._h else "no handle"
+            raise ForgeStepError(st, msg)
+
+    def close(self):
+        if self._h:
+            lib().ft_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- steps (device tensors: int32 [B, S], contiguous) -------------------------------------------
+    def train_step(self, tokens, labels, want_loss: bool = True):
+        B, S = tokens.shape
+        loss, gn = C.c_float(), C.c_float()
+        st = lib().ft_train_step(self._h, C.c_void_p(tokens.data_ptr()), C.c_void_p(labels.data_ptr()), B, S,
+                                 C.byref(loss) if want_loss else None, C.byref(gn) if want_loss else None)
+        self._check(st)
+        return (loss.value, gn.value) if want_loss else None
+
+    def train_step_host(self, tokens: np.ndarray, labels: np.ndarray):
+        """tokens, labels: int32 numpy arrays [B, S] in host memory (copied to the device inside the call)."""
+        B, S = tokens.shape
+        loss, gn = C.c_float(), C.c_float()
+        st = lib().ft_train_step_host(self._h, C.c_void_p(tokens.ctypes.data), C.c_void_p(labels.ctypes.data), B, S,
+                                      C.byref(loss), C.byref(gn))
+        self._check(st)
+        return loss.value, gn.value
+
+    def forward_loss(self, tokens, labels) -> float:
+        B, S = tokens.shape
+        loss = C.c_float()
+        self._check(lib().ft_forward_loss(self._h, C.c_void_p(tokens.data_ptr()), C.c_void_p(labels.data_ptr()), B, S,
+                                          C.byref(loss)))
+        return loss.value
+
+    def forward_backward(self, tokens, labels) -> float:
+        B, S = tokens.shape
+        loss = C.c_float()
+        self._check(lib().ft_forward_backward(self._h, C.c_void_p(tokens.data_ptr()), C.c_void_p(labels.data_ptr()), B,
+                                              S, C.byref(loss)))
+        return loss.value
+
+    def apply_update(self) -> float:
+        gn = C.c_float()
+        self._check(lib().ft_apply_update(self._h, C.byref(gn)))
+        return gn.value
+
+    # ---- state ------------------------------------------------------------------------------------------
+    def get_param(self, name: str, kind: int = KIND_MASTER) -> np.ndarray:
+        i = self.index[name]
+        shape = self.params[i][1]
+        out = np.empty(shape, dtype=np.uint16 if kind == KIND_BF16 else np.float32)
+        self._check(lib().ft_get_param(self._h, i, kind, C.c_void_p(out.ctypes.data), out.nbytes))
+        return bf16_bits_to_f32(out) if kind == KIND_BF16 else out
+
+    def set_param(self, name: str, value: np.ndarray, kind: int = KIND_MASTER):
+        if kind == KIND_BF16:
+            raise ValueError("the bf16 copy is derived from the master; set the master instead")
+        i = self.index[name]
+        v = np.ascontiguousarray(value, dtype=np.float32).reshape(self.params[i][1])
+        self._check(lib().ft_set_param(self._h, i, kind, C.c_void_p(v.ctypes.data), v.nbytes))
+
+    @property
+    def step(self) -> int:
+        s = C.c_int64()
+        self._check(lib().ft_get_step(self._h, C.byref(s)))
+        return s.value
+
+    @step.setter
+    def step(self, v: int):
+        self._check(lib().ft_set_step(self._h, int(v)))
+
+    def get_tap(self, name: str, layer: int = -1) -> np.ndarray:
+        """Named intermediate of the last step as a flat float32 array."""
+        need, dt = C.c_size_t(), C.c_int32()
+        probe = np.empty(1, dtype=np.uint8)
+        st = lib().ft_get_tap(self._h, name.encode(), layer, C.c_void_p(probe.ctypes.data), 0, C.byref(need),
+                              C.byref(dt))
+        if st == FT_ENOTFOUND:
+            self._check(st)
+        buf = np.empty(need.value, dtype=np.uint8)
+        self._check(lib().ft_get_tap(self._h, name.encode(), layer, C.c_void_p(buf.ctypes.data), buf.nbytes,
+                                     C.byref(need), C.byref(dt)))
+        return buf.view(np.float32).copy() if dt.value == 1 else bf16_bits_to_f32(buf.view(np.uint16))
+
+    @property
+    def launch_count(self) -> int:
+        return int(lib().ft_launch_count(self._h))
+
+
+# ---- single kernels (torch device tensors) ---------------------------------------------------------------
+def k_gemm(A, a_mn: int, B, b_mn: int, Cout, out_kind: int, M: int, N: int, K: int, err, resid=None):
+    """C[M,N] = sum_k A[m,k] B[n,k] on device tensors; leading dimensions are the tensors' row strides."""
+    st = lib().ft_k_gemm(C.c_void_p(A.data_ptr()), a_mn, A.stride(0), C.c_void_p(B.data_ptr()), b_mn, B.stride(0),
+                         C.c_void_p(Cout.data_ptr()), Cout.stride(0),
+                         C.c_void_p(resid.data_ptr()) if resid is not None else None, out_kind, M, N, K,
+                         C.c_void_p(err.data_ptr()), _stream_ptr())
+    if st != FT_OK:
+        raise ForgeStepError(st, "ft_k_gemm")
+
+
+def k_attention_fwd(qkv, o, lse, B, S, n_heads, n_kv, d):
+    st = lib().ft_k_attention_fwd(C.c_void_p(qkv.data_ptr()), C.c_void_p(o.data_ptr()), C.c_void_p(lse.data_ptr()), B,
+                                  S, n_heads, n_kv, d, _stream_ptr())
+    if st != FT_OK:
+        raise ForgeStepError(st, "ft_k_attention_fwd")
+
+
+def k_attention_bwd(qkv, o, d_o, lse, delta, dqkv, B, S, n_heads, n_kv, d, cos=None, sin=None):
+    st = lib().ft_k_attention_bwd(C.c_void_p(qkv.data_ptr()), C.c_void_p(o.data_ptr()), C.c_void_p(d_o.data_ptr()),
+                                  C.c_void_p(lse.data_ptr()), C.c_void_p(delta.data_ptr()),
+                                  C.c_void_p(dqkv.data_ptr()), C.c_void_p(cos.data_ptr()) if cos is not None else None,
+                                  C.c_void_p(sin.data_ptr()) if sin is not None else None, B, S, n_heads, n_kv, d,
+                                  _stream_ptr())
+    if st != FT_OK:
+        raise ForgeStepError(st, "ft_k_attention_bwd")

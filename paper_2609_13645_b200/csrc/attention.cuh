@@ -1,0 +1,20 @@
+// Host-side interface of the causal flash-attention kernels.
+#pragma once
+#include <cuda_runtime.h>
+
+#include "common.cuh"
+
+namespace fs {
+
+// qkv bf16 [B*S, (n_h + 2 n_kv) d] packed q heads | k heads | v heads (q, k rotated); o bf16 [B*S, n_h d];
+// lse fp32 [B, n_h, S] in natural log.  d in {64, 128}.  One kernel launch.
+cudaError_t attention_fwd(const bf16* qkv, bf16* o, float* lse, int B, int S, int n_heads, int n_kv, int d,
+                          cudaStream_t st);
+
+// Three kernel launches (delta pre-pass, dQ, dK/dV).  delta: fp32 scratch [B, n_h, S].  dqkv has qkv's layout.
+// cos/sin: fp32 [S, d/2] or both null (then dq, dk are left in the rotated frame).
+cudaError_t attention_bwd(const bf16* qkv, const bf16* o, const bf16* d_o, const float* lse, float* delta, bf16* dqkv,
+                          const float* cos, const float* sin, int B, int S, int n_heads, int n_kv, int d,
+                          cudaStream_t st);
+
+}  // namespace fs

@@ -1,0 +1,600 @@
+// Bandwidth-bound kernels of the train step.  All reductions run in a fixed order (no floating-point
+// atomics), so results are bit-identical from run to run; all global accesses are 16-byte vectors.
+#include "elementwise.cuh"
+
+#include <math.h>
+
+namespace fs {
+namespace {
+
+constexpr int kNormMaxChunks = 16;  // d_model <= 16 * 256
+
+__device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
+  f[0] = bf16_lo(v.x); f[1] = bf16_hi(v.x); f[2] = bf16_lo(v.y); f[3] = bf16_hi(v.y);
+  f[4] = bf16_lo(v.z); f[5] = bf16_hi(v.z); f[6] = bf16_lo(v.w); f[7] = bf16_hi(v.w);
+}
+__device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
+  uint4 o;
+  o.x = pack_bf16(f[0], f[1]); o.y = pack_bf16(f[2], f[3]); o.z = pack_bf16(f[4], f[5]); o.w = pack_bf16(f[6], f[7]);
+  return o;
+}
+
+// ---------------------------------------------------------------- embedding forward
+__global__ void embed_fwd_kernel(const int32_t* __restrict__ tok, const bf16* __restrict__ E, bf16* __restrict__ x,
+                                 long long total_chunks, int chunks_per_row, int h, int vocab) {
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total_chunks;
+       i += (long long)gridDim.x * blockDim.x) {
+    const long long t = i / chunks_per_row;
+    const int c = (int)(i % chunks_per_row) * 8;
+    int id = tok[t];
+    id = id < 0 ? 0 : (id >= vocab ? vocab - 1 : id);
+    *reinterpret_cast<uint4*>(x + t * h + c) = *reinterpret_cast<const uint4*>(E + (long long)id * h + c);
+  }
+}
+
+// ---------------------------------------------------------------- RMSNorm forward: one warp per row
+__global__ void rmsnorm_fwd_kernel(const bf16* __restrict__ x, const bf16* __restrict__ g, bf16* __restrict__ y,
+                                   float* __restrict__ r, int T, int h, float eps) {
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= T) return;
+  const bf16* xr = x + (long long)row * h;
+  float ss = 0.f;
+  for (int c = lane * 8; c < h; c += 256) {
+    float f[8];
+    unpack8(*reinterpret_cast<const uint4*>(xr + c), f);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) ss += f[e] * f[e];
+  }
+  ss = warp_sum(ss);
+  const float rr = 1.0f / sqrtf(ss / (float)h + eps);
+  if (lane == 0) r[row] = rr;
+  bf16* yr = y + (long long)row * h;
+  for (int c = lane * 8; c < h; c += 256) {
+    float f[8], gg[8];
+    unpack8(*reinterpret_cast<const uint4*>(xr + c), f);
+    unpack8(*reinterpret_cast<const uint4*>(g + c), gg);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) f[e] = f[e] * rr * gg[e];
+    *reinterpret_cast<uint4*>(yr + c) = pack8(f);
+  }
+}
+
+// ---------------------------------------------------------------- RMSNorm backward
+// dx_k = r g_k dy_k - x_k r^3 (1/h) sum_j g_j dy_j x_j (+ resid_k);  dg_k = sum_t dy_tk x_tk r_t.
+// One warp per row, rows strided over the grid; each lane keeps the dg of its columns in registers, the 8 warps of a
+// block are then added in warp order, and a second kernel adds the block partials in block order.
+__global__ void __launch_bounds__(256)
+rmsnorm_bwd_kernel(const bf16* __restrict__ dy, const bf16* __restrict__ x, const float* __restrict__ r,
+                   const bf16* __restrict__ g, const bf16* __restrict__ resid, bf16* __restrict__ dx,
+                   float* __restrict__ partial, int T, int h) {
+  extern __shared__ float s_dg[];  // [h]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nch = h >> 8;
+  float dg[kNormMaxChunks][8];
+#pragma unroll
+  for (int i = 0; i < kNormMaxChunks; ++i)
+#pragma unroll
+    for (int e = 0; e < 8; ++e) dg[i][e] = 0.f;
+  const float inv_h = 1.0f / (float)h;
+  for (int row = blockIdx.x * 8 + warp; row < T; row += gridDim.x * 8) {
+    const bf16* dyr = dy + (long long)row * h;
+    const bf16* xr = x + (long long)row * h;
+    const float rr = r[row];
+    float dot = 0.f;
+#pragma unroll
+    for (int i = 0; i < kNormMaxChunks; ++i) {
+      if (i < nch) {
+        const int c = lane * 8 + (i << 8);
+        float a[8], b[8], gg[8];
+        unpack8(*reinterpret_cast<const uint4*>(dyr + c), a);
+        unpack8(*reinterpret_cast<const uint4*>(xr + c), b);
+        unpack8(*reinterpret_cast<const uint4*>(g + c), gg);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) dot += gg[e] * a[e] * b[e];
+      }
+    }
+    dot = warp_sum(dot);
+    const float coef = rr * rr * rr * dot * inv_h;
+#pragma unroll
+    for (int i = 0; i < kNormMaxChunks; ++i) {
+      if (i < nch) {
+        const int c = lane * 8 + (i << 8);
+        float a[8], b[8], gg[8], o[8];
+        unpack8(*reinterpret_cast<const uint4*>(dyr + c), a);
+        unpack8(*reinterpret_cast<const uint4*>(xr + c), b);
+        unpack8(*reinterpret_cast<const uint4*>(g + c), gg);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          o[e] = rr * gg[e] * a[e] - b[e] * coef;
+          dg[i][e] += a[e] * b[e] * rr;
+        }
+        if (resid != nullptr) {
+          float rs[8];
+          unpack8(*reinterpret_cast<const uint4*>(resid + (long long)row * h + c), rs);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) o[e] += rs[e];
+        }
+        *reinterpret_cast<uint4*>(dx + (long long)row * h + c) = pack8(o);
+      }
+    }
+  }
+  for (int w = 0; w < 8; ++w) {
+    if (warp == w) {
+#pragma unroll
+      for (int i = 0; i < kNormMaxChunks; ++i) {
+        if (i < nch) {
+          const int c = lane * 8 + (i << 8);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) s_dg[c + e] = (w == 0 ? 0.f : s_dg[c + e]) + dg[i][e];
+        }
+      }
+    }
+    __syncthreads();
+  }
+  for (int c = threadIdx.x; c < h; c += blockDim.x) partial[(long long)blockIdx.x * h + c] = s_dg[c];
+}
+
+__global__ void colsum_kernel(const float* __restrict__ partial, float* __restrict__ out, int nblk, int h) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= h) return;
+  float s = 0.f;
+  for (int b = 0; b < nblk; ++b) s += partial[(long long)b * h + c];
+  out[c] = s;
+}
+
+// ---------------------------------------------------------------- SwiGLU backward
+__global__ void swiglu_bwd_kernel(const bf16* __restrict__ d_a, const bf16* __restrict__ gu, bf16* __restrict__ d_gu,
+                                  long long total_chunks, int chunks_per_row, int f) {
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total_chunks;
+       i += (long long)gridDim.x * blockDim.x) {
+    const long long t = i / chunks_per_row;
+    const int c = (int)(i % chunks_per_row) * 8;
+    float da[8], G[8], U[8], dG[8], dU[8];
+    unpack8(*reinterpret_cast<const uint4*>(d_a + t * f + c), da);
+    unpack8(*reinterpret_cast<const uint4*>(gu + t * 2 * f + c), G);
+    unpack8(*reinterpret_cast<const uint4*>(gu + t * 2 * f + f + c), U);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const float sg = 1.0f / (1.0f + expf(-G[e]));
+      dU[e] = da[e] * G[e] * sg;
+      dG[e] = da[e] * U[e] * sg * (1.0f + G[e] * (1.0f - sg));
+    }
+    const int phys = ((c >> 4) << 5) + (c & 15);
+    *reinterpret_cast<uint4*>(d_gu + t * 2 * f + phys) = pack8(dG);
+    *reinterpret_cast<uint4*>(d_gu + t * 2 * f + phys + 16) = pack8(dU);
+  }
+}
+
+// ---------------------------------------------------------------- loss
+__global__ void count_labels_kernel(const int32_t* __restrict__ labels, int T, StepScalars* sc) {
+  __shared__ int s[32];
+  int c = 0;
+  for (int i = threadIdx.x; i < T; i += blockDim.x) c += labels[i] >= 0 ? 1 : 0;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+  if ((threadIdx.x & 31) == 0) s[threadIdx.x >> 5] = c;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int tot = 0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += s[w];
+    sc->count = tot;
+    sc->inv_count = 1.0f / (float)(tot > 0 ? tot : 1);
+  }
+}
+
+// one block per row of logits
+__global__ void __launch_bounds__(256)
+cross_entropy_kernel(const float* __restrict__ z, const int32_t* __restrict__ labels, float* __restrict__ lse_out,
+                     float* __restrict__ loss_row, bf16* __restrict__ dz, int V, const StepScalars* __restrict__ sc) {
+  __shared__ float s_m[8], s_s[8];
+  __shared__ float s_lse;
+  const int row = blockIdx.x;
+  const float* zr = z + (long long)row * V;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float m = -INFINITY, s = 0.f;
+  for (int c = threadIdx.x * 4; c < V; c += 1024) {
+    const float4 v = *reinterpret_cast<const float4*>(zr + c);
+    const float m4 = fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w));
+    if (m4 > m) {
+      s *= expf(m - m4);
+      m = m4;
+    }
+    s += expf(v.x - m) + expf(v.y - m) + expf(v.z - m) + expf(v.w - m);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float m2 = __shfl_xor_sync(0xffffffffu, m, o);
+    const float s2 = __shfl_xor_sync(0xffffffffu, s, o);
+    const float mm = fmaxf(m, m2);
+    // symmetric in (m,s) and (m2,s2) up to the commutative add, so both partners get the same bits
+    const float a = (m == -INFINITY) ? 0.f : s * expf(m - mm);
+    const float b = (m2 == -INFINITY) ? 0.f : s2 * expf(m2 - mm);
+    s = (m >= m2) ? a + b : b + a;
+    m = mm;
+  }
+  if (lane == 0) { s_m[warp] = m; s_s[warp] = s; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float mm = s_m[0];
+    for (int w = 1; w < 8; ++w) mm = fmaxf(mm, s_m[w]);
+    float tot = 0.f;
+    for (int w = 0; w < 8; ++w) tot += (s_m[w] == -INFINITY) ? 0.f : s_s[w] * expf(s_m[w] - mm);
+    const float lse = mm + logf(tot);
+    s_lse = lse;
+    lse_out[row] = lse;
+    const int y = labels[row];
+    loss_row[row] = (y >= 0 && y < V) ? lse - zr[y] : 0.f;
+  }
+  __syncthreads();
+  if (dz == nullptr) return;
+  const float lse = s_lse;
+  const int y = labels[row];
+  const bool counted = y >= 0 && y < V;
+  const float w = counted ? sc->inv_count : 0.f;
+  bf16* dr = dz + (long long)row * V;
+  for (int c = threadIdx.x * 4; c < V; c += 1024) {
+    const float4 v = *reinterpret_cast<const float4*>(zr + c);
+    float p0 = expf(v.x - lse), p1 = expf(v.y - lse), p2 = expf(v.z - lse), p3 = expf(v.w - lse);
+    if (y == c) p0 -= 1.f;
+    if (y == c + 1) p1 -= 1.f;
+    if (y == c + 2) p2 -= 1.f;
+    if (y == c + 3) p3 -= 1.f;
+    uint2 o;
+    o.x = pack_bf16(p0 * w, p1 * w);
+    o.y = pack_bf16(p2 * w, p3 * w);
+    *reinterpret_cast<uint2*>(dr + c) = o;
+  }
+}
+
+__global__ void reduce_loss_kernel(const float* __restrict__ loss_row, int T, StepScalars* sc) {
+  __shared__ float s[1024];
+  float a = 0.f;
+  for (int i = threadIdx.x; i < T; i += blockDim.x) a += loss_row[i];
+  s[threadIdx.x] = a;
+  __syncthreads();
+  for (int o = blockDim.x >> 1; o > 0; o >>= 1) {
+    if ((int)threadIdx.x < o) s[threadIdx.x] += s[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const float loss = s[0] * sc->inv_count;
+    sc->loss = loss;
+    sc->nonfinite = isfinite(loss) ? 0 : 1;
+  }
+}
+
+// ---------------------------------------------------------------- embedding backward (sort + ordered segment sums)
+constexpr int kSortChunk = 4096;
+constexpr int kSortThreads = 512;
+
+__global__ void make_keys_kernel(const int32_t* __restrict__ tok, unsigned long long* __restrict__ keys, int T, int n_pad,
+                                 int vocab) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_pad) return;
+  if (i < T) {
+    int id = tok[i];
+    id = id < 0 ? 0 : (id >= vocab ? vocab - 1 : id);
+    keys[i] = ((unsigned long long)(unsigned)id << 32) | (unsigned)i;
+  } else {
+    keys[i] = ~0ull;
+  }
+}
+
+__device__ __forceinline__ void cmp_swap(unsigned long long& a, unsigned long long& b, bool up) {
+  if ((a > b) == up) {
+    const unsigned long long t = a;
+    a = b;
+    b = t;
+  }
+}
+
+// sorts (k_lo == 2) or merges (k_lo == k_hi) one chunk in shared memory: runs the network steps (k, j) for
+// k = k_lo..k_hi and j = min(k/2, chunk/2)..1
+__global__ void __launch_bounds__(kSortThreads)
+bitonic_chunk_kernel(unsigned long long* __restrict__ keys, int k_lo, int k_hi) {
+  __shared__ unsigned long long s[kSortChunk];
+  const int base = blockIdx.x * kSortChunk;
+  for (int i = threadIdx.x; i < kSortChunk; i += kSortThreads) s[i] = keys[base + i];
+  __syncthreads();
+  for (int k = k_lo; k <= k_hi; k <<= 1) {
+    for (int j = min(k >> 1, kSortChunk >> 1); j > 0; j >>= 1) {
+      for (int p = threadIdx.x; p < kSortChunk / 2; p += kSortThreads) {
+        const int i = ((p & ~(j - 1)) << 1) | (p & (j - 1));  // index with bit j clear
+        const bool up = ((base + i) & k) == 0;
+        cmp_swap(s[i], s[i | j], up);
+      }
+      __syncthreads();
+    }
+  }
+  for (int i = threadIdx.x; i < kSortChunk; i += kSortThreads) keys[base + i] = s[i];
+}
+
+__global__ void bitonic_global_kernel(unsigned long long* __restrict__ keys, int n_pad, int k, int j) {
+  const int p = blockIdx.x * blockDim.x + threadIdx.x;
+  if (p >= n_pad / 2) return;
+  const int i = ((p & ~(j - 1)) << 1) | (p & (j - 1));
+  const bool up = (i & k) == 0;
+  unsigned long long a = keys[i], b = keys[i | j];
+  if ((a > b) == up) {
+    keys[i] = b;
+    keys[i | j] = a;
+  }
+}
+
+// block i works only if sorted position i starts a run of equal tokens; its 8 warps take contiguous eighths of the
+// run (position order), and the eight partial rows are added in warp order.
+__global__ void __launch_bounds__(256)
+embed_bwd_kernel(const unsigned long long* __restrict__ keys, const bf16* __restrict__ dx, float* __restrict__ dE, int T,
+                 int h) {
+  __shared__ int s_end;
+  __shared__ float s_part[8][256];
+  const int i = blockIdx.x;
+  const unsigned long long key = keys[i];
+  const unsigned tokid = (unsigned)(key >> 32);
+  if (i > 0 && (unsigned)(keys[i - 1] >> 32) == tokid) return;
+  if (threadIdx.x == 0) {
+    const unsigned long long bound = ((unsigned long long)tokid + 1ull) << 32;  // first key of the next token
+    int lo = i + 1, hi = T;
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if (keys[mid] < bound) lo = mid + 1; else hi = mid;
+    }
+    s_end = lo;
+  }
+  __syncthreads();
+  const int len = s_end - i;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r0 = i + (int)(((long long)len * warp) / 8), r1 = i + (int)(((long long)len * (warp + 1)) / 8);
+  for (int slab = 0; slab < h; slab += 256) {
+    const int c = slab + lane * 8;
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    if (c < h) {
+      for (int rpos = r0; rpos < r1; ++rpos) {
+        const unsigned pos = (unsigned)(keys[rpos] & 0xffffffffull);
+        float f[8];
+        unpack8(*reinterpret_cast<const uint4*>(dx + (long long)pos * h + c), f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] += f[e];
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) s_part[warp][lane * 8 + e] = acc[e];
+    __syncthreads();
+    const int col = slab + threadIdx.x;
+    if (col < h) {
+      float tot = 0.f;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) tot += s_part[w][threadIdx.x];
+      dE[(long long)tokid * h + col] = tot;
+    }
+    __syncthreads();
+  }
+}
+
+// ---------------------------------------------------------------- gradient norm, step scalars, AdamW
+__global__ void __launch_bounds__(256)
+sqnorm_partial_kernel(const float* __restrict__ g, size_t n4, float* __restrict__ partial) {
+  __shared__ float s[8];
+  float a = 0.f;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    const float4 v = reinterpret_cast<const float4*>(g)[i];
+    a += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  a = warp_sum(a);
+  if ((threadIdx.x & 31) == 0) s[threadIdx.x >> 5] = a;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float tot = 0.f;
+    for (int w = 0; w < 8; ++w) tot += s[w];
+    partial[blockIdx.x] = tot;
+  }
+}
+
+__global__ void sqnorm_final_kernel(const float* __restrict__ partial, int nblk, StepScalars* sc, AdamHyper hp) {
+  __shared__ float s[256];
+  float a = 0.f;
+  for (int i = threadIdx.x; i < nblk; i += 256) a += partial[i];
+  s[threadIdx.x] = a;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if ((int)threadIdx.x < o) s[threadIdx.x] += s[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const float gn = sqrtf(fmaxf(s[0], 0.f));
+    sc->gnorm = gn;
+    sc->clip = hp.max_grad_norm > 0.f ? fminf(1.0f, hp.max_grad_norm / (gn + 1e-6f)) : 1.0f;
+  }
+}
+
+__global__ void advance_step_kernel(StepScalars* sc, AdamHyper hp) {
+  const long long t = sc->step + 1;
+  sc->step = t;
+  sc->bc1 = (float)(1.0 - pow((double)hp.beta1, (double)t));
+  sc->bc2 = (float)(1.0 - pow((double)hp.beta2, (double)t));
+}
+
+__global__ void __launch_bounds__(256)
+adamw_kernel(float* __restrict__ p, float* __restrict__ m, float* __restrict__ v, const float* __restrict__ g,
+             bf16* __restrict__ pb, size_t n4, size_t n4_decay, const StepScalars* __restrict__ sc, AdamHyper hp) {
+  const float clip = sc->clip, bc1 = sc->bc1, bc2 = sc->bc2;
+  const float omb1 = 1.0f - hp.beta1, omb2 = 1.0f - hp.beta2;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    const float wd = i < n4_decay ? hp.wd : 0.f;
+    const float4 g4 = reinterpret_cast<const float4*>(g)[i];
+    float4 p4 = reinterpret_cast<float4*>(p)[i];
+    float4 m4 = reinterpret_cast<float4*>(m)[i];
+    float4 v4 = reinterpret_cast<float4*>(v)[i];
+    float gg[4] = {g4.x, g4.y, g4.z, g4.w};
+    float pp[4] = {p4.x, p4.y, p4.z, p4.w};
+    float mm[4] = {m4.x, m4.y, m4.z, m4.w};
+    float vv[4] = {v4.x, v4.y, v4.z, v4.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float ge = gg[e] * clip;
+      mm[e] = hp.beta1 * mm[e] + omb1 * ge;
+      vv[e] = hp.beta2 * vv[e] + omb2 * ge * ge;
+      const float mhat = mm[e] / bc1;
+      const float vhat = vv[e] / bc2;
+      const float upd = mhat / (sqrtf(vhat) + hp.eps) + wd * pp[e];
+      pp[e] = pp[e] - hp.lr * upd;
+    }
+    reinterpret_cast<float4*>(p)[i] = make_float4(pp[0], pp[1], pp[2], pp[3]);
+    reinterpret_cast<float4*>(m)[i] = make_float4(mm[0], mm[1], mm[2], mm[3]);
+    reinterpret_cast<float4*>(v)[i] = make_float4(vv[0], vv[1], vv[2], vv[3]);
+    uint2 o;
+    o.x = pack_bf16(pp[0], pp[1]);
+    o.y = pack_bf16(pp[2], pp[3]);
+    reinterpret_cast<uint2*>(pb)[i] = o;
+  }
+}
+
+// ---------------------------------------------------------------- initialisation
+__device__ __forceinline__ unsigned long long splitmix64(unsigned long long z) {
+  z += 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+__global__ void init_normal_kernel(float* __restrict__ p, size_t n, unsigned long long seed, unsigned long long tensor_id,
+                                   float stddev) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    const unsigned long long k = seed ^ ((tensor_id + 1ull) * 0xD1B54A32D192ED03ull) ^ ((unsigned long long)i * 0x8CB92BA72F3D8DD7ull);
+    const unsigned long long r = splitmix64(k);
+    const double u1 = ((double)(r >> 40) + 1.0) / 16777216.0;
+    const double u2 = (double)((r >> 16) & 0xFFFFFFull) / 16777216.0;
+    const double z = sqrt(-2.0 * log(u1)) * cos(6.283185307179586476925286766559 * u2);
+    p[i] = (float)(z * (double)stddev);
+  }
+}
+
+__global__ void fill_kernel(float* __restrict__ p, size_t n, float v) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) p[i] = v;
+}
+
+__global__ void cast_bf16_kernel(const float* __restrict__ src, bf16* __restrict__ dst, size_t n) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    dst[i] = __float2bfloat16_rn(src[i]);
+}
+
+inline int grid_for(size_t work_items, int threads, int max_blocks = 148 * 16) {
+  size_t b = (work_items + threads - 1) / threads;
+  if (b < 1) b = 1;
+  if (b > (size_t)max_blocks) b = max_blocks;
+  return (int)b;
+}
+inline int ok(int launches) { return cudaGetLastError() == cudaSuccess ? launches : -1; }
+
+}  // namespace
+
+int elementwise_blocks_for_norm(int T) {
+  const int need = (T + 7) / 8;
+  return need < 296 ? need : 296;
+}
+
+size_t sort_pad(size_t n) {
+  size_t p = kSortChunk;
+  while (p < n) p <<= 1;
+  return p;
+}
+
+int embed_fwd(const int32_t* tok, const bf16* E, bf16* x, int T, int h, int vocab, cudaStream_t st) {
+  const long long total = (long long)T * (h / 8);
+  embed_fwd_kernel<<<grid_for(total, 256), 256, 0, st>>>(tok, E, x, total, h / 8, h, vocab);
+  return ok(1);
+}
+
+int rmsnorm_fwd(const bf16* x, const bf16* g, bf16* y, float* r, int T, int h, float eps, cudaStream_t st) {
+  rmsnorm_fwd_kernel<<<(T + 7) / 8, 256, 0, st>>>(x, g, y, r, T, h, eps);
+  return ok(1);
+}
+
+int rmsnorm_bwd(const bf16* dy, const bf16* x, const float* r, const bf16* g, const bf16* resid, bf16* dx, float* dg,
+                float* partial, int T, int h, cudaStream_t st) {
+  if ((h & 255) || h > 256 * kNormMaxChunks) return -1;
+  const int nblk = elementwise_blocks_for_norm(T);
+  rmsnorm_bwd_kernel<<<nblk, 256, h * sizeof(float), st>>>(dy, x, r, g, resid, dx, partial, T, h);
+  colsum_kernel<<<(h + 255) / 256, 256, 0, st>>>(partial, dg, nblk, h);
+  return ok(2);
+}
+
+int swiglu_bwd(const bf16* d_a, const bf16* gu, bf16* d_gu, int T, int f, cudaStream_t st) {
+  const long long total = (long long)T * (f / 8);
+  swiglu_bwd_kernel<<<grid_for(total, 256), 256, 0, st>>>(d_a, gu, d_gu, total, f / 8, f);
+  return ok(1);
+}
+
+int count_labels(const int32_t* labels, int T, StepScalars* sc, cudaStream_t st) {
+  count_labels_kernel<<<1, 1024, 0, st>>>(labels, T, sc);
+  return ok(1);
+}
+
+int cross_entropy_rows(const float* z, const int32_t* labels, float* lse, float* loss_row, bf16* dz, int rows, int V,
+                       const StepScalars* sc, cudaStream_t st) {
+  cross_entropy_kernel<<<rows, 256, 0, st>>>(z, labels, lse, loss_row, dz, V, sc);
+  return ok(1);
+}
+
+int reduce_loss(const float* loss_row, int T, StepScalars* sc, cudaStream_t st) {
+  reduce_loss_kernel<<<1, 1024, 0, st>>>(loss_row, T, sc);
+  return ok(1);
+}
+
+int embed_bwd(const int32_t* tok, const bf16* dx, float* dE, unsigned long long* keys, int T, int h, int vocab,
+              cudaStream_t st) {
+  const int n_pad = (int)sort_pad((size_t)T);
+  int launches = 0;
+  make_keys_kernel<<<(n_pad + 255) / 256, 256, 0, st>>>(tok, keys, T, n_pad, vocab);
+  ++launches;
+  const int nchunks = n_pad / kSortChunk;
+  bitonic_chunk_kernel<<<nchunks, kSortThreads, 0, st>>>(keys, 2, kSortChunk);
+  ++launches;
+  for (int k = kSortChunk * 2; k <= n_pad; k <<= 1) {
+    for (int j = k >> 1; j >= kSortChunk; j >>= 1) {
+      bitonic_global_kernel<<<(n_pad / 2 + 255) / 256, 256, 0, st>>>(keys, n_pad, k, j);
+      ++launches;
+    }
+    bitonic_chunk_kernel<<<nchunks, kSortThreads, 0, st>>>(keys, k, k);
+    ++launches;
+  }
+  if (cudaMemsetAsync(dE, 0, (size_t)vocab * h * sizeof(float), st) != cudaSuccess) return -1;
+  embed_bwd_kernel<<<T, 256, 0, st>>>(keys, dx, dE, T, h);
+  ++launches;
+  return ok(launches);
+}
+
+int grad_norm_and_clip(const float* g, size_t n, float* partial, StepScalars* sc, AdamHyper hp, cudaStream_t st) {
+  sqnorm_partial_kernel<<<kSqnormBlocks, 256, 0, st>>>(g, n / 4, partial);
+  sqnorm_final_kernel<<<1, 256, 0, st>>>(partial, kSqnormBlocks, sc, hp);
+  return ok(2);
+}
+
+int advance_step(StepScalars* sc, AdamHyper hp, cudaStream_t st) {
+  advance_step_kernel<<<1, 1, 0, st>>>(sc, hp);
+  return ok(1);
+}
+
+int adamw(float* p, float* m, float* v, const float* g, bf16* pb, size_t n, size_t n_decay, const StepScalars* sc,
+          AdamHyper hp, cudaStream_t st) {
+  adamw_kernel<<<148 * 8, 256, 0, st>>>(p, m, v, g, pb, n / 4, n_decay / 4, sc, hp);
+  return ok(1);
+}
+
+int init_normal(float* p, size_t n, uint64_t seed, int tensor_id, float stddev, cudaStream_t st) {
+  init_normal_kernel<<<grid_for(n, 256), 256, 0, st>>>(p, n, seed, (unsigned long long)tensor_id, stddev);
+  return ok(1);
+}
+
+int fill_f32(float* p, size_t n, float v, cudaStream_t st) {
+  fill_kernel<<<grid_for(n, 256), 256, 0, st>>>(p, n, v);
+  return ok(1);
+}
+
+int cast_bf16(const float* src, bf16* dst, size_t n, cudaStream_t st) {
+  cast_bf16_kernel<<<grid_for(n, 256), 256, 0, st>>>(src, dst, n);
+  return ok(1);
+}
+
+}  // namespace fs

@@ -1,0 +1,58 @@
+// Host-side interface of the bandwidth-bound kernels: embedding, RMSNorm, SwiGLU backward, cross-entropy,
+// deterministic embedding backward, gradient norm, AdamW, initialisation.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "common.cuh"
+
+namespace fs {
+
+// Device-resident per-step scalars (nothing here is read by the host inside a step).
+struct StepScalars {
+  long long step;     // optimizer step counter t
+  float bc1, bc2;     // 1 - beta1^t, 1 - beta2^t
+  float clip;         // gradient clip coefficient
+  float gnorm;        // global gradient norm of the last step
+  float loss;         // mean loss of the last step
+  float inv_count;    // 1 / number of counted labels
+  int count;          // number of labels >= 0
+  int nonfinite;      // 1 if the last loss was not finite
+  int err;            // device status word (ERR_*)
+  int pad[5];
+};
+
+struct AdamHyper {
+  float lr, beta1, beta2, eps, wd, max_grad_norm;
+};
+
+int elementwise_blocks_for_norm(int T);            // grid of rmsnorm_bwd (also rows of its partial buffer)
+constexpr int kSqnormBlocks = 1184;               // partial sums of the gradient norm
+size_t sort_pad(size_t n);                         // padded key count of the embedding-backward sort
+
+// each returns the number of kernels it launched, or a negative value after a CUDA launch error
+int embed_fwd(const int32_t* tok, const bf16* E, bf16* x, int T, int h, int vocab, cudaStream_t st);
+int rmsnorm_fwd(const bf16* x, const bf16* g, bf16* y, float* r, int T, int h, float eps, cudaStream_t st);
+// dx = R(resid + rmsnorm_bwd(dy)) (resid may be null); dg = column sums (fp32, fixed order) via `partial`.
+int rmsnorm_bwd(const bf16* dy, const bf16* x, const float* r, const bf16* g, const bf16* resid, bf16* dx, float* dg,
+                float* partial, int T, int h, cudaStream_t st);
+// d_gu (physical 16/16 interleave of gate and up columns) from d_a and the saved gate|up activations.
+int swiglu_bwd(const bf16* d_a, const bf16* gu, bf16* d_gu, int T, int f, cudaStream_t st);
+int count_labels(const int32_t* labels, int T, StepScalars* sc, cudaStream_t st);
+// per row: lse, loss contribution, and (if dz != null) dz = R((softmax(z) - onehot) * inv_count), zero for ignored rows
+int cross_entropy_rows(const float* z, const int32_t* labels, float* lse, float* loss_row, bf16* dz, int rows, int V,
+                       const StepScalars* sc, cudaStream_t st);
+int reduce_loss(const float* loss_row, int T, StepScalars* sc, cudaStream_t st);
+// dE[v,:] = sum over positions with token v (fp32, position order); keys: scratch of sort_pad(T) uint64
+int embed_bwd(const int32_t* tok, const bf16* dx, float* dE, unsigned long long* keys, int T, int h, int vocab,
+              cudaStream_t st);
+int grad_norm_and_clip(const float* g, size_t n, float* partial, StepScalars* sc, AdamHyper hp, cudaStream_t st);
+int advance_step(StepScalars* sc, AdamHyper hp, cudaStream_t st);
+// fused clip + Adam + decoupled decay + bf16 write-back over a flat arena; elements >= n_decay get no decay
+int adamw(float* p, float* m, float* v, const float* g, bf16* pb, size_t n, size_t n_decay, const StepScalars* sc,
+          AdamHyper hp, cudaStream_t st);
+int init_normal(float* p, size_t n, uint64_t seed, int tensor_id, float std, cudaStream_t st);
+int fill_f32(float* p, size_t n, float v, cudaStream_t st);
+int cast_bf16(const float* src, bf16* dst, size_t n, cudaStream_t st);
+
+}  // namespace fs

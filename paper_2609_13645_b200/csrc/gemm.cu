@@ -1,0 +1,423 @@
+// bf16 GEMM family on the 5th-generation tensor cores (tcgen05.mma, accumulators in TMEM, operands staged in
+// shared memory by TMA with the 128-byte swizzle).  One persistent, warp-specialised kernel:
+//   warp 0      : TMA producer (one elected thread)
+//   warp 1      : TMEM allocator + MMA issuer (one elected thread)
+//   warps 2..5  : epilogue, one TMEM lane quarter each; the accumulator is double-buffered in TMEM so the
+//                 epilogue of tile i overlaps the main loop of tile i+1.
+// Computes C[M,N] = sum_k A[m,k] B[n,k] for the three operand layouts a training step needs
+// (forward: both k-contiguous; data gradient: B mn-contiguous; weight gradient: both mn-contiguous, i.e. the
+// contraction runs over the rows of the stored activations) without materialising any transpose.
+#include "gemm.cuh"
+
+#include <cuda.h>
+
+#include <mutex>
+
+namespace fs {
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 64;  // 64 bf16 = 128 bytes = one swizzle row
+constexpr int A_BYTES = BM * BK * 2;
+constexpr int CHUNK_BYTES = 64 * BK * 2;  // one 64 x 64 box of an mn-major operand
+constexpr int GEMM_THREADS = 192;
+
+template <int BN>
+struct Cfg {
+  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int STAGES = (BN == 256) ? 4 : 6;
+  static constexpr int TMEM_COLS = 2 * BN;
+  static constexpr int BAR_BYTES = 256;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024;  // + slack to align to 1024
+};
+
+struct GemmDev {
+  void* C;
+  const bf16* resid;
+  bf16* gu;
+  const float* rope_cos;
+  const float* rope_sin;
+  int* err;
+  long long ldc;
+  int M, N, K;
+  int epi;
+  int seq, head_dim, rope_cols, d_ffn;
+};
+
+__device__ __forceinline__ void store8_bf16(bf16* dst, const float* v) {
+  uint4 o;
+  o.x = pack_bf16(v[0], v[1]);
+  o.y = pack_bf16(v[2], v[3]);
+  o.z = pack_bf16(v[4], v[5]);
+  o.w = pack_bf16(v[6], v[7]);
+  *reinterpret_cast<uint4*>(dst) = o;
+}
+
+template <int BN, bool A_MN, bool B_MN>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmDev p) {
+  using C = Cfg<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::STAGES * C::STAGE_BYTES);
+  const uint32_t bar0 = smem_u32(bars);
+  // barrier slots: [0,S) full, [S,2S) empty, 2S+{0,1} accumulator full, 2S+{2,3} accumulator empty
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (C::STAGES + s); };
+  auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * C::STAGES + b); };
+  auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * C::STAGES + 2 + b); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * C::STAGES + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(tfull_bar(b), 1);
+      mbar_init(tempty_bar(b), 4);
+    }
+    *abort_flag = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tmA);
+    tma_prefetch_desc(&tmB);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_slot), C::TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int tiles_m = (p.M + BM - 1) / BM;
+  const int tiles_n = (p.N + BN - 1) / BN;
+  const int ntiles = tiles_m * tiles_n;
+  const int kblocks = (p.K + BK - 1) / BK;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+        const int m0 = (t % tiles_m) * BM;
+        const int n0 = (t / tiles_m) * BN;
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.err)) { ok = false; break; }
+          const uint32_t fb = full_bar(stage);
+          mbar_expect_tx(fb, C::STAGE_BYTES);
+          const uint32_t a_dst = smem_u32(smem + stage * C::STAGE_BYTES);
+          const uint32_t b_dst = a_dst + A_BYTES;
+          if constexpr (!A_MN) {
+            tma_load_2d(a_dst, &tmA, fb, kb * BK, m0);
+          } else {
+#pragma unroll
+            for (int j = 0; j < BM / 64; ++j) tma_load_2d(a_dst + j * CHUNK_BYTES, &tmA, fb, m0 + 64 * j, kb * BK);
+          }
+          if constexpr (!B_MN) {
+            tma_load_2d(b_dst, &tmB, fb, kb * BK, n0);
+          } else {
+#pragma unroll
+            for (int j = 0; j < BN / 64; ++j) tma_load_2d(b_dst + j * CHUNK_BYTES, &tmB, fb, n0 + 64 * j, kb * BK);
+          }
+          if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // instruction descriptor: fp32 accumulate, bf16 A and B, majors, N/8, M/16
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) | ((B_MN ? 1u : 0u) << 16) |
+                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.err)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.err)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(smem + stage * C::STAGE_BYTES);
+          const uint32_t b_addr = a_addr + A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            const uint64_t adesc = A_MN ? umma_desc_sw128(a_addr + k * 2048, CHUNK_BYTES, 1024)
+                                        : umma_desc_sw128(a_addr + k * 32, 0, 1024);
+            const uint64_t bdesc = B_MN ? umma_desc_sw128(b_addr + k * 2048, CHUNK_BYTES, 1024)
+                                        : umma_desc_sw128(b_addr + k * 32, 0, 1024);
+            umma_bf16(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          umma_commit(empty_bar(stage));
+          if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit(tfull_bar(acc));
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+  } else {
+    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    for (int t = blockIdx.x; t < ntiles; t += gridDim.x) {
+      const int m0 = (t % tiles_m) * BM;
+      const int n0 = (t / tiles_m) * BN;
+      bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.err);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const int row = m0 + q * 32 + lane;
+      const bool row_ok = row < p.M;
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
+      uint32_t r[32];
+      if (p.epi == EPI_ROPE) {
+        const int d = p.head_dim;
+        const int half = d >> 1;
+        const int pos = row_ok ? (row % p.seq) : 0;
+        bf16* crow = reinterpret_cast<bf16*>(p.C) + (long long)row * p.ldc;
+        for (int hc = 0; hc < BN; hc += d) {
+          const int g0 = n0 + hc;
+          if (g0 >= p.N) break;
+          if (g0 >= p.rope_cols) {
+            for (int c = 0; c < d; c += 32) {
+              tmem_ld32(taddr + hc + c, r);
+              tmem_ld_wait();
+              if (row_ok) {
+                float v[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) store8_bf16(crow + g0 + c + j, v + j);
+              }
+            }
+          } else {
+            uint32_t r2[32];
+            for (int i0 = 0; i0 < half; i0 += 32) {
+              tmem_ld32(taddr + hc + i0, r);
+              tmem_ld32(taddr + hc + i0 + half, r2);
+              tmem_ld_wait();
+              if (row_ok) {
+                const float* cs = p.rope_cos + (long long)pos * half + i0;
+                const float* sn = p.rope_sin + (long long)pos * half + i0;
+                float lo[32], hi[32];
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) {
+                  const float4 c4 = *reinterpret_cast<const float4*>(cs + j);
+                  const float4 s4 = *reinterpret_cast<const float4*>(sn + j);
+                  const float cc[4] = {c4.x, c4.y, c4.z, c4.w};
+                  const float ss[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+                  for (int u = 0; u < 4; ++u) {
+                    const float x1 = __uint_as_float(r[j + u]);
+                    const float x2 = __uint_as_float(r2[j + u]);
+                    lo[j + u] = x1 * cc[u] - x2 * ss[u];
+                    hi[j + u] = x2 * cc[u] + x1 * ss[u];
+                  }
+                }
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) {
+                  store8_bf16(crow + g0 + i0 + j, lo + j);
+                  store8_bf16(crow + g0 + i0 + half + j, hi + j);
+                }
+              }
+            }
+          }
+        }
+      } else if (p.epi == EPI_SWIGLU) {
+        // physical columns alternate 16 gate / 16 up of the same 16 logical ffn columns
+        const int f = p.d_ffn;
+        bf16* arow = reinterpret_cast<bf16*>(p.C) + (long long)row * p.ldc;
+        bf16* gurow = p.gu + (long long)row * (2LL * f);
+        for (int c = 0; c < BN; c += 32) {
+          const int gc = n0 + c;
+          if (gc >= p.N) break;
+          tmem_ld32(taddr + c, r);
+          tmem_ld_wait();
+          if (row_ok) {
+            const int lc = gc >> 1;  // logical ffn column of this 16-wide group
+            float g[16], u[16], a[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              g[j] = round_bf16(__uint_as_float(r[j]));
+              u[j] = round_bf16(__uint_as_float(r[16 + j]));
+              a[j] = g[j] / (1.0f + __expf(-g[j])) * u[j];
+            }
+            store8_bf16(gurow + lc, g);
+            store8_bf16(gurow + lc + 8, g + 8);
+            store8_bf16(gurow + f + lc, u);
+            store8_bf16(gurow + f + lc + 8, u + 8);
+            store8_bf16(arow + lc, a);
+            store8_bf16(arow + lc + 8, a + 8);
+          }
+        }
+      } else {
+        for (int c = 0; c < BN; c += 32) {
+          const int gc = n0 + c;
+          if (gc >= p.N) break;
+          tmem_ld32(taddr + c, r);
+          tmem_ld_wait();
+          if (row_ok) {
+            float v[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+            if (p.epi == EPI_BF16 || p.epi == EPI_BF16_RESID) {
+              bf16* crow = reinterpret_cast<bf16*>(p.C) + (long long)row * p.ldc + gc;
+              const bf16* rrow = p.resid + (long long)row * p.ldc + gc;
+#pragma unroll
+              for (int j = 0; j < 32; j += 8) {
+                if (gc + j < p.N) {
+                  if (p.epi == EPI_BF16_RESID) {
+                    const uint4 x = *reinterpret_cast<const uint4*>(rrow + j);
+                    v[j + 0] += bf16_lo(x.x); v[j + 1] += bf16_hi(x.x);
+                    v[j + 2] += bf16_lo(x.y); v[j + 3] += bf16_hi(x.y);
+                    v[j + 4] += bf16_lo(x.z); v[j + 5] += bf16_hi(x.z);
+                    v[j + 6] += bf16_lo(x.w); v[j + 7] += bf16_hi(x.w);
+                  }
+                  store8_bf16(crow + j, v + j);
+                }
+              }
+            } else {
+              float* crow = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + gc;
+#pragma unroll
+              for (int j = 0; j < 32; j += 4) {
+                if (gc + j < p.N) {
+                  float4 o = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                  if (p.epi == EPI_F32_ACC) {
+                    const float4 x = *reinterpret_cast<const float4*>(crow + j);
+                    o.x += x.x; o.y += x.y; o.z += x.z; o.w += x.w;
+                  }
+                  *reinterpret_cast<float4*>(crow + j) = o;
+                }
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1u;
+    }
+  }
+
+  // teardown: everyone meets here, also after a wait that ran out
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag != 0) {
+    // give copies and MMAs still in flight time to land before shared memory and TMEM are released
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000LL) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, C::TMEM_COLS);
+  }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+// 2-D bf16 tensor map over a row-major matrix [rows, row_stride] of which `cols` columns are valid;
+// box = 64 columns x box_rows rows, 128-byte swizzle, zero fill outside.
+bool make_tmap(CUtensorMap* tm, const bf16* base, uint64_t cols, uint64_t rows, uint64_t row_stride, uint32_t box_rows) {
+  EncodeTiledFn enc = get_encode_fn();
+  if (!enc) return false;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {row_stride * sizeof(bf16)};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<bf16*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 148;
+  }
+  return n;
+}
+
+template <int BN, bool A_MN, bool B_MN>
+cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
+  using C = Cfg<BN>;
+  static bool attr_set = false;
+  auto kern = gemm_tc_kernel<BN, A_MN, B_MN>;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  CUtensorMap tmA, tmB;
+  bool ok = A_MN ? make_tmap(&tmA, a.A, a.M, a.K, a.lda, 64) : make_tmap(&tmA, a.A, a.K, a.M, a.lda, BM);
+  ok = ok && (B_MN ? make_tmap(&tmB, a.B, a.N, a.K, a.ldb, 64) : make_tmap(&tmB, a.B, a.K, a.N, a.ldb, BN));
+  if (!ok) return cudaErrorInvalidValue;
+  GemmDev p;
+  p.C = a.C; p.resid = a.resid; p.gu = a.gu; p.rope_cos = a.rope_cos; p.rope_sin = a.rope_sin; p.err = a.err;
+  p.ldc = a.ldc; p.M = a.M; p.N = a.N; p.K = a.K; p.epi = a.epi;
+  p.seq = a.seq; p.head_dim = a.head_dim; p.rope_cols = a.rope_cols; p.d_ffn = a.d_ffn;
+  const int tiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN);
+  const int grid = tiles < sm_count() ? tiles : sm_count();
+  kern<<<grid, GEMM_THREADS, C::SMEM_BYTES, stream>>>(tmA, tmB, p);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream) {
+  if (a.M <= 0 || a.N <= 0 || a.K <= 0 || !a.A || !a.B || !a.C || !a.err) return cudaErrorInvalidValue;
+  if ((a.N & 7) || (a.lda & 7) || (a.ldb & 7) || (a.ldc & 3)) return cudaErrorInvalidValue;
+  if ((a.a_mn ? a.M : a.K) & 7) return cudaErrorInvalidValue;
+  if ((a.b_mn ? a.N : a.K) & 7) return cudaErrorInvalidValue;
+  if ((reinterpret_cast<uintptr_t>(a.A) | reinterpret_cast<uintptr_t>(a.B) | reinterpret_cast<uintptr_t>(a.C)) & 15)
+    return cudaErrorInvalidValue;
+  if (a.epi == EPI_BF16_RESID && !a.resid) return cudaErrorInvalidValue;
+  if (a.epi == EPI_ROPE && (!a.rope_cos || !a.rope_sin || (a.head_dim != 64 && a.head_dim != 128) || a.seq <= 0 ||
+                            a.rope_cols % a.head_dim || a.N % a.head_dim))
+    return cudaErrorInvalidValue;
+  if (a.epi == EPI_SWIGLU && (!a.gu || a.d_ffn <= 0 || a.d_ffn % 16 || a.N != 2 * a.d_ffn)) return cudaErrorInvalidValue;
+  const int tiles256 = ((a.M + BM - 1) / BM) * ((a.N + 255) / 256);
+  const bool wide = tiles256 >= sm_count();
+  if (!a.a_mn && !a.b_mn) return wide ? launch_variant<256, false, false>(a, stream) : launch_variant<128, false, false>(a, stream);
+  if (!a.a_mn && a.b_mn) return wide ? launch_variant<256, false, true>(a, stream) : launch_variant<128, false, true>(a, stream);
+  if (a.a_mn && a.b_mn) return wide ? launch_variant<256, true, true>(a, stream) : launch_variant<128, true, true>(a, stream);
+  return cudaErrorInvalidValue;  // (mn-major A with k-major B) is not needed by the train step
+}
+
+}  // namespace fs

@@ -1,0 +1,723 @@
+// The train-step schedule and the C ABI.  A model is a carve-up of the caller's workspace plus a fixed launch
+// order: there is no autograd graph and no host synchronisation inside a step; optimizer scalars live in device
+// memory and are advanced by a kernel.
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <string>
+#include <vector>
+
+#include "../../include/forgestep.h"
+#include "attention.cuh"
+#include "elementwise.cuh"
+#include "gemm.cuh"
+
+using namespace fs;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct ParamInfo {
+  std::string name;
+  int64_t rows, cols;  // cols == 0 for a gain vector of `rows` elements
+  size_t offset;       // element offset in every arena
+  bool is_wgu;
+  size_t numel() const { return (size_t)rows * (size_t)(cols ? cols : 1); }
+};
+
+struct Carver {
+  uint8_t* base = nullptr;
+  size_t off = 0;
+  template <typename T>
+  T* take(size_t n) {
+    off = align_up(off, kAlign);
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += n * sizeof(T);
+    return p;
+  }
+};
+
+struct LayerActs {
+  bf16 *h1, *qkv, *o, *x_mid, *h2, *gu, *a;
+  float *lse, *r1, *r2;
+};
+
+struct LayerTaps {  // debug copies of one layer's backward intermediates
+  bf16 *d_x_out, *d_a, *d_gu, *d_h2, *d_x_mid, *d_o, *d_qkv, *d_h1, *d_x_in;
+};
+
+}  // namespace
+
+struct ft_model {
+  ft_config cfg;
+  cudaStream_t stream = nullptr;
+  std::string err;
+  int64_t launches = 0;
+  int h, hq, hkv, nqkv, f, V, L, d, maxT;
+  int n_slots;
+  int ce_chunk;
+
+  std::vector<ParamInfo> params;
+  size_t arena = 0, n_decay = 0;
+  float *master, *adam_m, *adam_v, *grad;
+  bf16* pbf;
+  float *rope_cos, *rope_sin;
+  StepScalars* sc;
+  int32_t *tok_dev, *lab_dev;
+  std::vector<bf16*> x;  // x[l] = input of layer l, x[L] = output of the last layer
+  std::vector<LayerActs> acts;
+  std::vector<LayerTaps> taps;
+  float *rF, *ce_lse, *loss_row;
+  bf16 *hF, *d_hF;
+  bf16 *dxA, *dxB, *d_h, *d_a, *d_gu, *d_o, *d_qkv;
+  float *delta, *norm_partial, *sq_partial, *z;
+  bf16* dz;
+  unsigned long long* keys;
+  int lastB = 0, lastS = 0;
+  bool have_bwd = false;
+
+  const ParamInfo& P(int i) const { return params[i]; }
+  int idx_layer(int l, int k) const { return 1 + l * 6 + k; }  // k: 0 norm1, 1 wqkv, 2 wo, 3 norm2, 4 wgu, 5 wd
+  bf16* wb(int i) const { return pbf + params[i].offset; }
+  float* gr(int i) const { return grad + params[i].offset; }
+};
+
+namespace {
+
+bool valid_config(const ft_config* c, std::string* why) {
+  auto bad = [&](const char* m) { if (why) *why = m; return false; };
+  if (!c) return bad("null config");
+  if (c->n_layers < 1 || c->d_model < 1 || c->n_heads < 1 || c->n_kv_heads < 1 || c->d_ffn < 1 || c->vocab < 1)
+    return bad("non-positive dimension");
+  if (c->head_dim != 64 && c->head_dim != 128) return bad("head_dim must be 64 or 128");
+  if (c->n_heads % c->n_kv_heads) return bad("n_heads must be a multiple of n_kv_heads");
+  if (c->d_model % 256 || c->d_model > 4096) return bad("d_model must be a multiple of 256, at most 4096");
+  if (c->d_ffn % 16) return bad("d_ffn must be a multiple of 16");
+  if (c->vocab % 8) return bad("vocab must be a multiple of 8");
+  if (c->max_batch < 1 || c->max_seq < 1) return bad("max_batch and max_seq must be positive");
+  if ((long long)c->max_batch * c->max_seq > (1ll << 24)) return bad("max_batch * max_seq too large");
+  if (c->debug_taps && c->recompute) return bad("debug_taps needs recompute = 0");
+  if (!(c->rms_eps > 0.f) || !(c->rope_theta > 0.f)) return bad("rms_eps and rope_theta must be positive");
+  return true;
+}
+
+int pick_ce_chunk(const ft_config* c) {
+  const long long T = (long long)c->max_batch * c->max_seq;
+  long long rows = 2048;
+  while (rows > 128 && rows * (long long)c->vocab * 6 > (3ll << 30)) rows >>= 1;  // logits + dlogits scratch <= 3 GiB
+  if (rows > T) rows = (T + 7) / 8 * 8;
+  return (int)rows;
+}
+
+// Lays the model out in the workspace.  With base == nullptr it only measures.
+size_t carve(ft_model* m, uint8_t* base) {
+  const ft_config& c = m->cfg;
+  m->h = c.d_model; m->d = c.head_dim; m->hq = c.n_heads * c.head_dim; m->hkv = c.n_kv_heads * c.head_dim;
+  m->nqkv = m->hq + 2 * m->hkv; m->f = c.d_ffn; m->V = c.vocab; m->L = c.n_layers;
+  m->maxT = c.max_batch * c.max_seq;
+  m->n_slots = c.recompute ? 1 : c.n_layers;
+  m->ce_chunk = pick_ce_chunk(&c);
+  const size_t T = (size_t)m->maxT, h = m->h, f = m->f, hq = m->hq, nqkv = m->nqkv, V = m->V;
+
+  // parameter table: matrices first (they get weight decay), gains after
+  m->params.clear();
+  auto add = [&](const std::string& n, int64_t r, int64_t cc, bool wgu) {
+    ParamInfo p; p.name = n; p.rows = r; p.cols = cc; p.offset = 0; p.is_wgu = wgu; m->params.push_back(p);
+  };
+  add("embed", V, h, false);
+  for (int l = 0; l < m->L; ++l) {
+    const std::string p = "layers." + std::to_string(l) + ".";
+    add(p + "norm1", h, 0, false);
+    add(p + "wqkv", nqkv, h, false);
+    add(p + "wo", h, hq, false);
+    add(p + "norm2", h, 0, false);
+    add(p + "wgu", 2 * f, h, true);
+    add(p + "wd", h, f, false);
+  }
+  add("norm_f", h, 0, false);
+  add("lm_head", V, h, false);
+  size_t off = 0;
+  for (auto& p : m->params) if (p.cols) { p.offset = off; off += align_up(p.numel(), 128); }
+  m->n_decay = off;
+  for (auto& p : m->params) if (!p.cols) { p.offset = off; off += align_up(p.numel(), 128); }
+  m->arena = off;
+
+  Carver cv; cv.base = base;
+  m->master = cv.take<float>(m->arena);
+  m->adam_m = cv.take<float>(m->arena);
+  m->adam_v = cv.take<float>(m->arena);
+  m->grad = cv.take<float>(m->arena);
+  m->pbf = cv.take<bf16>(m->arena);
+  m->rope_cos = cv.take<float>((size_t)c.max_seq * (m->d / 2));
+  m->rope_sin = cv.take<float>((size_t)c.max_seq * (m->d / 2));
+  m->sc = cv.take<StepScalars>(1);
+  m->tok_dev = cv.take<int32_t>(T);
+  m->lab_dev = cv.take<int32_t>(T);
+  m->x.assign(m->L + 1, nullptr);
+  for (int l = 0; l <= m->L; ++l) m->x[l] = cv.take<bf16>(T * h);
+  m->acts.assign(m->n_slots, LayerActs());
+  for (auto& a : m->acts) {
+    a.h1 = cv.take<bf16>(T * h); a.qkv = cv.take<bf16>(T * nqkv); a.o = cv.take<bf16>(T * hq);
+    a.x_mid = cv.take<bf16>(T * h); a.h2 = cv.take<bf16>(T * h); a.gu = cv.take<bf16>(T * 2 * f);
+    a.a = cv.take<bf16>(T * f); a.lse = cv.take<float>(T * c.n_heads); a.r1 = cv.take<float>(T);
+    a.r2 = cv.take<float>(T);
+  }
+  m->rF = cv.take<float>(T); m->ce_lse = cv.take<float>(T); m->loss_row = cv.take<float>(T);
+  m->hF = cv.take<bf16>(T * h); m->d_hF = cv.take<bf16>(T * h);
+  m->dxA = cv.take<bf16>(T * h); m->dxB = cv.take<bf16>(T * h); m->d_h = cv.take<bf16>(T * h);
+  m->d_a = cv.take<bf16>(T * f); m->d_gu = cv.take<bf16>(T * 2 * f); m->d_o = cv.take<bf16>(T * hq);
+  m->d_qkv = cv.take<bf16>(T * nqkv);
+  m->delta = cv.take<float>(T * c.n_heads);
+  m->norm_partial = cv.take<float>((size_t)elementwise_blocks_for_norm((int)T) * h);
+  m->sq_partial = cv.take<float>(kSqnormBlocks);
+  m->z = cv.take<float>((size_t)m->ce_chunk * V);
+  m->dz = cv.take<bf16>((size_t)m->ce_chunk * V);
+  m->keys = cv.take<unsigned long long>(sort_pad(T));
+  m->taps.clear();
+  if (c.debug_taps) {
+    m->taps.assign(m->L, LayerTaps());
+    for (auto& t : m->taps) {
+      t.d_x_out = cv.take<bf16>(T * h); t.d_a = cv.take<bf16>(T * f); t.d_gu = cv.take<bf16>(T * 2 * f);
+      t.d_h2 = cv.take<bf16>(T * h); t.d_x_mid = cv.take<bf16>(T * h); t.d_o = cv.take<bf16>(T * hq);
+      t.d_qkv = cv.take<bf16>(T * nqkv); t.d_h1 = cv.take<bf16>(T * h); t.d_x_in = cv.take<bf16>(T * h);
+    }
+  }
+  return align_up(cv.off, kAlign);
+}
+
+ft_status fail(ft_model* m, ft_status s, const std::string& msg) {
+  if (m) m->err = msg;
+  return s;
+}
+ft_status cuda_fail(ft_model* m, cudaError_t e, const char* where) {
+  return fail(m, FT_ECUDA, std::string(where) + ": " + cudaGetErrorString(e));
+}
+
+#define FT_CUDA(call)                                              \
+  do {                                                             \
+    cudaError_t e__ = (call);                                      \
+    if (e__ != cudaSuccess) return cuda_fail(m, e__, #call);       \
+  } while (0)
+#define FT_LAUNCH(call)                                                                     \
+  do {                                                                                      \
+    int n__ = (call);                                                                       \
+    if (n__ < 0) return fail(m, FT_ECUDA, std::string("kernel launch failed: ") + #call);   \
+    m->launches += n__;                                                                     \
+  } while (0)
+#define FT_GEMM(args)                                                                       \
+  do {                                                                                      \
+    cudaError_t e__ = launch_gemm(args, m->stream);                                         \
+    if (e__ != cudaSuccess) return cuda_fail(m, e__, "launch_gemm");                        \
+    m->launches += 1;                                                                       \
+  } while (0)
+
+AdamHyper hyper(const ft_model* m) {
+  AdamHyper hp;
+  hp.lr = m->cfg.lr; hp.beta1 = m->cfg.beta1; hp.beta2 = m->cfg.beta2; hp.eps = m->cfg.adam_eps;
+  hp.wd = m->cfg.weight_decay; hp.max_grad_norm = m->cfg.max_grad_norm;
+  return hp;
+}
+
+GemmArgs gemm_base(ft_model* m) {
+  GemmArgs g;
+  g.err = &m->sc->err;
+  return g;
+}
+
+// forward of layer l from m->x[l] into activation slot `a`, output to m->x[l+1]
+ft_status layer_forward(ft_model* m, int l, LayerActs& a, int B, int S) {
+  const int T = B * S, h = m->h, f = m->f, hq = m->hq, nqkv = m->nqkv;
+  cudaStream_t st = m->stream;
+  FT_LAUNCH(rmsnorm_fwd(m->x[l], m->wb(m->idx_layer(l, 0)), a.h1, a.r1, T, h, m->cfg.rms_eps, st));
+  {
+    GemmArgs g = gemm_base(m);
+    g.A = a.h1; g.lda = h; g.B = m->wb(m->idx_layer(l, 1)); g.ldb = h; g.C = a.qkv; g.ldc = nqkv;
+    g.M = T; g.N = nqkv; g.K = h; g.epi = EPI_ROPE;
+    g.rope_cos = m->rope_cos; g.rope_sin = m->rope_sin; g.seq = S; g.head_dim = m->d; g.rope_cols = hq + m->hkv;
+    FT_GEMM(g);
+  }
+  FT_CUDA(attention_fwd(a.qkv, a.o, a.lse, B, S, m->cfg.n_heads, m->cfg.n_kv_heads, m->d, st));
+  m->launches += 1;
+  {
+    GemmArgs g = gemm_base(m);
+    g.A = a.o; g.lda = hq; g.B = m->wb(m->idx_layer(l, 2)); g.ldb = hq; g.C = a.x_mid; g.ldc = h; g.resid = m->x[l];
+    g.M = T; g.N = h; g.K = hq; g.epi = EPI_BF16_RESID;
+    FT_GEMM(g);
+  }
+  FT_LAUNCH(rmsnorm_fwd(a.x_mid, m->wb(m->idx_layer(l, 3)), a.h2, a.r2, T, h, m->cfg.rms_eps, st));
+  {
+    GemmArgs g = gemm_base(m);
+    g.A = a.h2; g.lda = h; g.B = m->wb(m->idx_layer(l, 4)); g.ldb = h; g.C = a.a; g.ldc = f; g.gu = a.gu; g.d_ffn = f;
+    g.M = T; g.N = 2 * f; g.K = h; g.epi = EPI_SWIGLU;
+    FT_GEMM(g);
+  }
+  {
+    GemmArgs g = gemm_base(m);
+    g.A = a.a; g.lda = f; g.B = m->wb(m->idx_layer(l, 5)); g.ldb = f; g.C = m->x[l + 1]; g.ldc = h; g.resid = a.x_mid;
+    g.M = T; g.N = h; g.K = f; g.epi = EPI_BF16_RESID;
+    FT_GEMM(g);
+  }
+  return FT_OK;
+}
+
+ft_status copy_tap(ft_model* m, bf16* dst, const bf16* src, size_t n) {
+  FT_CUDA(cudaMemcpyAsync(dst, src, n * sizeof(bf16), cudaMemcpyDeviceToDevice, m->stream));
+  return FT_OK;
+}
+
+// data gradient  dX[T, n_in] = dY[T, n_out] W[n_out, n_in]  and weight gradient  dW[n_out, n_in] = dY^T X
+ft_status linear_backward(ft_model* m, const bf16* dY, const bf16* X, int wi, bf16* dX, int T, int n_out, int n_in) {
+  {
+    GemmArgs g = gemm_base(m);
+    g.A = dY; g.lda = n_out; g.B = m->wb(wi); g.b_mn = 1; g.ldb = n_in; g.C = dX; g.ldc = n_in;
+    g.M = T; g.N = n_in; g.K = n_out; g.epi = EPI_BF16;
+    FT_GEMM(g);
+  }
+  {
+    GemmArgs g = gemm_base(m);
+    g.A = dY; g.a_mn = 1; g.lda = n_out; g.B = X; g.b_mn = 1; g.ldb = n_in; g.C = m->gr(wi); g.ldc = n_in;
+    g.M = n_out; g.N = n_in; g.K = T; g.epi = EPI_F32;
+    FT_GEMM(g);
+  }
+  return FT_OK;
+}
+
+ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
+  const int T = B * S, h = m->h, f = m->f, hq = m->hq, nqkv = m->nqkv;
+  cudaStream_t st = m->stream;
+  LayerTaps* tp = m->cfg.debug_taps ? &m->taps[l] : nullptr;
+  // m->dxA holds d_x_out
+  if (tp) { ft_status s = copy_tap(m, tp->d_x_out, m->dxA, (size_t)T * h); if (s) return s; }
+  ft_status s = linear_backward(m, m->dxA, a.a, m->idx_layer(l, 5), m->d_a, T, h, f);
+  if (s) return s;
+  FT_LAUNCH(swiglu_bwd(m->d_a, a.gu, m->d_gu, T, f, st));
+  s = linear_backward(m, m->d_gu, a.h2, m->idx_layer(l, 4), m->d_h, T, 2 * f, h);
+  if (s) return s;
+  if (tp) {
+    if ((s = copy_tap(m, tp->d_a, m->d_a, (size_t)T * f))) return s;
+    if ((s = copy_tap(m, tp->d_gu, m->d_gu, (size_t)T * 2 * f))) return s;
+    if ((s = copy_tap(m, tp->d_h2, m->d_h, (size_t)T * h))) return s;
+  }
+  FT_LAUNCH(rmsnorm_bwd(m->d_h, a.x_mid, a.r2, m->wb(m->idx_layer(l, 3)), m->dxA, m->dxB, m->gr(m->idx_layer(l, 3)),
+                        m->norm_partial, T, h, st));
+  s = linear_backward(m, m->dxB, a.o, m->idx_layer(l, 2), m->d_o, T, h, hq);
+  if (s) return s;
+  FT_CUDA(attention_bwd(a.qkv, a.o, m->d_o, a.lse, m->delta, m->d_qkv, m->rope_cos, m->rope_sin, B, S, m->cfg.n_heads,
+                        m->cfg.n_kv_heads, m->d, st));
+  m->launches += 3;
+  s = linear_backward(m, m->d_qkv, a.h1, m->idx_layer(l, 1), m->d_h, T, nqkv, h);
+  if (s) return s;
+  if (tp) {
+    if ((s = copy_tap(m, tp->d_x_mid, m->dxB, (size_t)T * h))) return s;
+    if ((s = copy_tap(m, tp->d_o, m->d_o, (size_t)T * hq))) return s;
+    if ((s = copy_tap(m, tp->d_qkv, m->d_qkv, (size_t)T * nqkv))) return s;
+    if ((s = copy_tap(m, tp->d_h1, m->d_h, (size_t)T * h))) return s;
+  }
+  FT_LAUNCH(rmsnorm_bwd(m->d_h, m->x[l], a.r1, m->wb(m->idx_layer(l, 0)), m->dxB, m->dxA, m->gr(m->idx_layer(l, 0)),
+                        m->norm_partial, T, h, st));
+  if (tp) { if ((s = copy_tap(m, tp->d_x_in, m->dxA, (size_t)T * h))) return s; }
+  return FT_OK;
+}
+
+// forward (+ backward when with_bwd) of one batch; everything is enqueued, nothing is synchronised
+ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* lab, int B, int S, bool with_bwd) {
+  if (!m || !tok || !lab) return fail(m, FT_EINVAL, "null argument");
+  if (B < 1 || S < 1 || B > m->cfg.max_batch || S > m->cfg.max_seq) return fail(m, FT_EINVAL, "B or S out of range");
+  const int T = B * S, h = m->h, V = m->V, L = m->L;
+  cudaStream_t st = m->stream;
+  m->lastB = B; m->lastS = S; m->have_bwd = false;
+
+  FT_LAUNCH(count_labels(lab, T, m->sc, st));
+  FT_LAUNCH(embed_fwd(tok, m->wb(0), m->x[0], T, h, V, st));
+  for (int l = 0; l < L; ++l) {
+    ft_status s = layer_forward(m, l, m->acts[m->cfg.recompute ? 0 : l], B, S);
+    if (s) return s;
+  }
+  const int i_normf = 1 + 6 * L, i_head = 2 + 6 * L;
+  FT_LAUNCH(rmsnorm_fwd(m->x[L], m->wb(i_normf), m->hF, m->rF, T, h, m->cfg.rms_eps, st));
+
+  // output head + cross-entropy (+ both head gradients) in chunks of rows: the logits of one chunk at a time
+  for (int r0 = 0, chunk = 0; r0 < T; r0 += m->ce_chunk, ++chunk) {
+    const int rows = (T - r0) < m->ce_chunk ? (T - r0) : m->ce_chunk;
+    {
+      GemmArgs g = gemm_base(m);
+      g.A = m->hF + (size_t)r0 * h; g.lda = h; g.B = m->wb(i_head); g.ldb = h; g.C = m->z; g.ldc = V;
+      g.M = rows; g.N = V; g.K = h; g.epi = EPI_F32;
+      FT_GEMM(g);
+    }
+    FT_LAUNCH(cross_entropy_rows(m->z, lab + r0, m->ce_lse + r0, m->loss_row + r0, with_bwd ? m->dz : nullptr, rows, V,
+                                 m->sc, st));
+    if (with_bwd) {
+      {
+        GemmArgs g = gemm_base(m);
+        g.A = m->dz; g.lda = V; g.B = m->wb(i_head); g.b_mn = 1; g.ldb = h; g.C = m->d_hF + (size_t)r0 * h; g.ldc = h;
+        g.M = rows; g.N = h; g.K = V; g.epi = EPI_BF16;
+        FT_GEMM(g);
+      }
+      {
+        GemmArgs g = gemm_base(m);
+        g.A = m->dz; g.a_mn = 1; g.lda = V; g.B = m->hF + (size_t)r0 * h; g.b_mn = 1; g.ldb = h; g.C = m->gr(i_head);
+        g.ldc = h; g.M = V; g.N = h; g.K = rows; g.epi = chunk == 0 ? EPI_F32 : EPI_F32_ACC;
+        FT_GEMM(g);
+      }
+    }
+  }
+  FT_LAUNCH(reduce_loss(m->loss_row, T, m->sc, st));
+  if (!with_bwd) return FT_OK;
+
+  FT_LAUNCH(rmsnorm_bwd(m->d_hF, m->x[L], m->rF, m->wb(i_normf), nullptr, m->dxA, m->gr(i_normf), m->norm_partial, T, h,
+                        st));
+  for (int l = L - 1; l >= 0; --l) {
+    LayerActs& a = m->acts[m->cfg.recompute ? 0 : l];
+    if (m->cfg.recompute) {
+      // rerun the layer's forward from its saved input (same kernels, so the same bits as the first time);
+      // its output lands in x[l+1], which nothing reads any more
+      ft_status s = layer_forward(m, l, a, B, S);
+      if (s) return s;
+    }
+    ft_status s = layer_backward(m, l, a, B, S);
+    if (s) return s;
+  }
+  FT_LAUNCH(embed_bwd(tok, m->dxA, m->gr(0), m->keys, T, h, V, st));
+  m->have_bwd = true;
+  return FT_OK;
+}
+
+ft_status run_update(ft_model* m) {
+  cudaStream_t st = m->stream;
+  const AdamHyper hp = hyper(m);
+  FT_LAUNCH(grad_norm_and_clip(m->grad, m->arena, m->sq_partial, m->sc, hp, st));
+  FT_LAUNCH(advance_step(m->sc, hp, st));
+  FT_LAUNCH(adamw(m->master, m->adam_m, m->adam_v, m->grad, m->pbf, m->arena, m->n_decay, m->sc, hp, st));
+  return FT_OK;
+}
+
+// one synchronisation: reads the scalars back and turns device-side flags into a status
+ft_status finish(ft_model* m, float* host_loss, float* host_gnorm) {
+  StepScalars hs;
+  FT_CUDA(cudaMemcpyAsync(&hs, m->sc, sizeof(hs), cudaMemcpyDeviceToHost, m->stream));
+  FT_CUDA(cudaStreamSynchronize(m->stream));
+  if (host_loss) *host_loss = hs.loss;
+  if (host_gnorm) *host_gnorm = hs.gnorm;
+  if (hs.err != 0) {
+    FT_CUDA(cudaMemsetAsync(&m->sc->err, 0, sizeof(int), m->stream));
+    return fail(m, FT_ETIMEOUT, "a device-side wait ran out of time");
+  }
+  if (hs.nonfinite) return fail(m, FT_ENONFINITE, "loss is not finite");
+  return FT_OK;
+}
+
+// wgu rows: logical (gate 0..f-1, up 0..f-1) <-> physical (16 gate rows, 16 up rows, alternating)
+inline int64_t wgu_phys_row(int64_t r, int64_t f) {
+  const int64_t i = r < f ? r : r - f;
+  return (i / 16) * 32 + (r < f ? 0 : 16) + i % 16;
+}
+
+size_t kind_elem_size(ft_kind k) { return k == FT_COMPUTE_BF16 ? 2 : 4; }
+void* kind_base(ft_model* m, ft_kind k) {
+  switch (k) {
+    case FT_MASTER_F32: return m->master;
+    case FT_COMPUTE_BF16: return m->pbf;
+    case FT_ADAM_M_F32: return m->adam_m;
+    case FT_ADAM_V_F32: return m->adam_v;
+    case FT_GRAD_F32: return m->grad;
+  }
+  return nullptr;
+}
+
+}  // namespace
+
+// =============================================================================== C ABI
+extern "C" {
+
+size_t ft_workspace_bytes(const ft_config* cfg) {
+  if (!valid_config(cfg, nullptr)) return 0;
+  ft_model tmp;
+  tmp.cfg = *cfg;
+  return carve(&tmp, nullptr);
+}
+
+ft_status ft_init_model(const ft_config* cfg, uint64_t seed, void* dev_workspace, size_t bytes, void* cuda_stream,
+                        ft_model** out) {
+  if (!out) return FT_EINVAL;
+  *out = nullptr;
+  std::string why;
+  if (!valid_config(cfg, &why)) return FT_EINVAL;
+  if (!dev_workspace || (reinterpret_cast<uintptr_t>(dev_workspace) & (kAlign - 1))) return FT_EINVAL;
+  ft_model* m = new ft_model();
+  m->cfg = *cfg;
+  m->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const size_t need = carve(m, reinterpret_cast<uint8_t*>(dev_workspace));
+  if (bytes < need) { delete m; return FT_ENOMEM; }
+  *out = m;  // from here on errors are reported through the handle
+  cudaStream_t st = m->stream;
+  int dev = 0, major = 0;
+  FT_CUDA(cudaGetDevice(&dev));
+  FT_CUDA(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+  if (major != 10) return fail(m, FT_ECUDA, "this library needs an sm_100 device");
+
+  FT_CUDA(cudaMemsetAsync(m->adam_m, 0, m->arena * sizeof(float), st));
+  FT_CUDA(cudaMemsetAsync(m->adam_v, 0, m->arena * sizeof(float), st));
+  FT_CUDA(cudaMemsetAsync(m->grad, 0, m->arena * sizeof(float), st));
+  FT_CUDA(cudaMemsetAsync(m->master, 0, m->arena * sizeof(float), st));
+  FT_CUDA(cudaMemsetAsync(m->sc, 0, sizeof(StepScalars), st));
+  for (size_t i = 0; i < m->params.size(); ++i) {
+    const ParamInfo& p = m->params[i];
+    if (p.cols) {
+      // element e of the LOGICAL tensor i gets draw (seed, i, e); wgu is drawn logically, then placed physically
+      if (!p.is_wgu) {
+        FT_LAUNCH(init_normal(m->master + p.offset, p.numel(), seed, (int)i, 0.02f, st));
+      } else {
+        float* tmp = m->grad + p.offset;  // the gradient arena is free at this point
+        FT_LAUNCH(init_normal(tmp, p.numel(), seed, (int)i, 0.02f, st));
+        for (int64_t r0 = 0; r0 < 2 * (int64_t)m->f; r0 += 16) {
+          const int64_t pr = wgu_phys_row(r0, m->f);
+          FT_CUDA(cudaMemcpyAsync(m->master + p.offset + pr * p.cols, tmp + r0 * p.cols, 16 * p.cols * sizeof(float),
+                                  cudaMemcpyDeviceToDevice, st));
+        }
+      }
+    } else {
+      FT_LAUNCH(fill_f32(m->master + p.offset, p.numel(), 1.0f, st));
+    }
+  }
+  FT_CUDA(cudaMemsetAsync(m->grad, 0, m->arena * sizeof(float), st));
+  FT_LAUNCH(cast_bf16(m->master, m->pbf, m->arena, st));
+
+  // RoPE tables: angle(p, i) = p * theta^(-2i/d), evaluated in double on the host, stored as fp32
+  {
+    const int half = m->d / 2;
+    std::vector<float> cs((size_t)cfg->max_seq * half), sn((size_t)cfg->max_seq * half);
+    for (int i = 0; i < half; ++i) {
+      const double inv = pow((double)cfg->rope_theta, -2.0 * i / (double)m->d);
+      for (int p = 0; p < cfg->max_seq; ++p) {
+        const double ang = (double)p * inv;
+        cs[(size_t)p * half + i] = (float)cos(ang);
+        sn[(size_t)p * half + i] = (float)sin(ang);
+      }
+    }
+    FT_CUDA(cudaMemcpyAsync(m->rope_cos, cs.data(), cs.size() * sizeof(float), cudaMemcpyHostToDevice, st));
+    FT_CUDA(cudaMemcpyAsync(m->rope_sin, sn.data(), sn.size() * sizeof(float), cudaMemcpyHostToDevice, st));
+    FT_CUDA(cudaStreamSynchronize(st));
+  }
+  return FT_OK;
+}
+
+ft_status ft_train_step(ft_model* m, const int32_t* dev_tokens, const int32_t* dev_labels, int32_t B, int32_t S,
+                        float* host_loss, float* host_gnorm) {
+  if (!m) return FT_EINVAL;
+  ft_status s = run_forward_backward(m, dev_tokens, dev_labels, B, S, true);
+  if (s) return s;
+  if ((s = run_update(m))) return s;
+  if (host_loss || host_gnorm) return finish(m, host_loss, host_gnorm);
+  return FT_OK;
+}
+
+ft_status ft_train_step_host(ft_model* m, const int32_t* host_tokens, const int32_t* host_labels, int32_t B, int32_t S,
+                             float* host_loss, float* host_gnorm) {
+  if (!m || !host_tokens || !host_labels) return fail(m, FT_EINVAL, "null argument");
+  if (B < 1 || S < 1 || B > m->cfg.max_batch || S > m->cfg.max_seq) return fail(m, FT_EINVAL, "B or S out of range");
+  const size_t bytes = (size_t)B * S * sizeof(int32_t);
+  FT_CUDA(cudaMemcpyAsync(m->tok_dev, host_tokens, bytes, cudaMemcpyHostToDevice, m->stream));
+  FT_CUDA(cudaMemcpyAsync(m->lab_dev, host_labels, bytes, cudaMemcpyHostToDevice, m->stream));
+  float loss = 0.f;
+  ft_status s = ft_train_step(m, m->tok_dev, m->lab_dev, B, S, &loss, host_gnorm);
+  if (host_loss) *host_loss = loss;
+  return s;
+}
+
+ft_status ft_forward_loss(ft_model* m, const int32_t* dev_tokens, const int32_t* dev_labels, int32_t B, int32_t S,
+                          float* host_loss) {
+  if (!m) return FT_EINVAL;
+  ft_status s = run_forward_backward(m, dev_tokens, dev_labels, B, S, false);
+  if (s) return s;
+  return finish(m, host_loss, nullptr);
+}
+
+ft_status ft_forward_backward(ft_model* m, const int32_t* dev_tokens, const int32_t* dev_labels, int32_t B, int32_t S,
+                              float* host_loss) {
+  if (!m) return FT_EINVAL;
+  ft_status s = run_forward_backward(m, dev_tokens, dev_labels, B, S, true);
+  if (s) return s;
+  return finish(m, host_loss, nullptr);
+}
+
+ft_status ft_apply_update(ft_model* m, float* host_gnorm) {
+  if (!m) return FT_EINVAL;
+  ft_status s = run_update(m);
+  if (s) return s;
+  return finish(m, nullptr, host_gnorm);
+}
+
+int32_t ft_num_params(const ft_model* m) { return m ? (int32_t)m->params.size() : 0; }
+
+ft_status ft_param_info(const ft_model* m, int32_t i, const char** name, int32_t* ndim, int64_t shape[2]) {
+  if (!m || i < 0 || i >= (int32_t)m->params.size()) return FT_EINVAL;
+  const ParamInfo& p = m->params[i];
+  if (name) *name = p.name.c_str();
+  if (ndim) *ndim = p.cols ? 2 : 1;
+  if (shape) { shape[0] = p.rows; shape[1] = p.cols ? p.cols : 1; }
+  return FT_OK;
+}
+
+static ft_status param_copy(ft_model* m, int32_t i, ft_kind kind, void* host, size_t bytes, bool to_host) {
+  if (!m || !host) return fail(m, FT_EINVAL, "null argument");
+  if (i < 0 || i >= (int32_t)m->params.size()) return fail(m, FT_EINVAL, "parameter index out of range");
+  if ((int)kind < 0 || (int)kind > (int)FT_GRAD_F32) return fail(m, FT_EINVAL, "unknown kind");
+  const ParamInfo& p = m->params[i];
+  const size_t es = kind_elem_size(kind);
+  if (bytes != p.numel() * es) return fail(m, FT_EINVAL, "byte count does not match the tensor");
+  uint8_t* dev = reinterpret_cast<uint8_t*>(kind_base(m, kind)) + p.offset * es;
+  uint8_t* hp = reinterpret_cast<uint8_t*>(host);
+  FT_CUDA(cudaStreamSynchronize(m->stream));
+  if (!p.is_wgu) {
+    if (to_host) FT_CUDA(cudaMemcpy(hp, dev, bytes, cudaMemcpyDeviceToHost));
+    else FT_CUDA(cudaMemcpy(dev, hp, bytes, cudaMemcpyHostToDevice));
+  } else {
+    // 16-row blocks of the logical tensor sit at their physical (interleaved) place
+    const size_t blk = 16 * (size_t)p.cols * es;
+    for (int64_t r0 = 0; r0 < p.rows; r0 += 16) {
+      uint8_t* d = dev + (size_t)wgu_phys_row(r0, m->f) * p.cols * es;
+      uint8_t* hrow = hp + (size_t)r0 * p.cols * es;
+      if (to_host) FT_CUDA(cudaMemcpy(hrow, d, blk, cudaMemcpyDeviceToHost));
+      else FT_CUDA(cudaMemcpy(d, hrow, blk, cudaMemcpyHostToDevice));
+    }
+  }
+  if (!to_host && kind == FT_MASTER_F32) {
+    const size_t span = align_up(p.numel(), 128);
+    FT_LAUNCH(cast_bf16(m->master + p.offset, m->pbf + p.offset, span, m->stream));
+    FT_CUDA(cudaStreamSynchronize(m->stream));
+  }
+  return FT_OK;
+}
+
+ft_status ft_get_param(ft_model* m, int32_t i, ft_kind kind, void* host_dst, size_t bytes) {
+  return param_copy(m, i, kind, host_dst, bytes, true);
+}
+ft_status ft_set_param(ft_model* m, int32_t i, ft_kind kind, const void* host_src, size_t bytes) {
+  return param_copy(m, i, kind, const_cast<void*>(host_src), bytes, false);
+}
+
+ft_status ft_get_step(const ft_model* mc, int64_t* step) {
+  ft_model* m = const_cast<ft_model*>(mc);
+  if (!m || !step) return FT_EINVAL;
+  long long s = 0;
+  FT_CUDA(cudaStreamSynchronize(m->stream));
+  FT_CUDA(cudaMemcpy(&s, &m->sc->step, sizeof(s), cudaMemcpyDeviceToHost));
+  *step = s;
+  return FT_OK;
+}
+
+ft_status ft_set_step(ft_model* m, int64_t step) {
+  if (!m || step < 0) return FT_EINVAL;
+  long long s = step;
+  FT_CUDA(cudaStreamSynchronize(m->stream));
+  FT_CUDA(cudaMemcpy(&m->sc->step, &s, sizeof(s), cudaMemcpyHostToDevice));
+  return FT_OK;
+}
+
+ft_status ft_get_tap(ft_model* m, const char* name, int32_t layer, void* host_dst, size_t bytes, size_t* out_bytes,
+                     int32_t* dtype) {
+  if (!m || !name || !host_dst) return fail(m, FT_EINVAL, "null argument");
+  if (m->lastB == 0) return fail(m, FT_ENOTFOUND, "no step has run yet");
+  const size_t T = (size_t)m->lastB * m->lastS, h = m->h, f = m->f, hq = m->hq, nqkv = m->nqkv;
+  const void* src = nullptr;
+  size_t n = 0;
+  int dt = 0;
+  const std::string nm(name);
+  if (layer < 0) {
+    if (nm == "hF") { src = m->hF; n = T * h; }
+    else if (nm == "ce_lse") { src = m->ce_lse; n = T; dt = 1; }
+    else if (nm == "d_hF" && m->have_bwd) { src = m->d_hF; n = T * h; }
+  } else if (layer < m->L) {
+    const bool fwd_ok = !m->cfg.recompute;  // with recomputation only the layer inputs / outputs survive the step
+    if (nm == "x_in") { src = m->x[layer]; n = T * h; }
+    else if (nm == "x_out" && (!m->cfg.recompute || layer == m->L - 1 || !m->have_bwd)) { src = m->x[layer + 1]; n = T * h; }
+    else if (fwd_ok) {
+      const LayerActs& a = m->acts[layer];
+      if (nm == "h1") { src = a.h1; n = T * h; }
+      else if (nm == "qkv") { src = a.qkv; n = T * nqkv; }
+      else if (nm == "attn_lse") { src = a.lse; n = T * m->cfg.n_heads; dt = 1; }
+      else if (nm == "o") { src = a.o; n = T * hq; }
+      else if (nm == "x_mid") { src = a.x_mid; n = T * h; }
+      else if (nm == "h2") { src = a.h2; n = T * h; }
+      else if (nm == "gu") { src = a.gu; n = T * 2 * f; }
+      else if (nm == "a") { src = a.a; n = T * f; }
+    }
+    if (!src && m->cfg.debug_taps && m->have_bwd) {
+      const LayerTaps& t = m->taps[layer];
+      if (nm == "d_x_out") { src = t.d_x_out; n = T * h; }
+      else if (nm == "d_a") { src = t.d_a; n = T * f; }
+      else if (nm == "d_gu") { src = t.d_gu; n = T * 2 * f; }
+      else if (nm == "d_h2") { src = t.d_h2; n = T * h; }
+      else if (nm == "d_x_mid") { src = t.d_x_mid; n = T * h; }
+      else if (nm == "d_o") { src = t.d_o; n = T * hq; }
+      else if (nm == "d_qkv") { src = t.d_qkv; n = T * nqkv; }
+      else if (nm == "d_h1") { src = t.d_h1; n = T * h; }
+      else if (nm == "d_x_in") { src = t.d_x_in; n = T * h; }
+    }
+  }
+  if (!src) return fail(m, FT_ENOTFOUND, "no such tap (or it was not kept in this mode)");
+  const size_t nbytes = n * (dt ? 4 : 2);
+  if (out_bytes) *out_bytes = nbytes;
+  if (dtype) *dtype = dt;
+  if (bytes < nbytes) return fail(m, FT_EINVAL, "destination too small");
+  FT_CUDA(cudaStreamSynchronize(m->stream));
+  FT_CUDA(cudaMemcpy(host_dst, src, nbytes, cudaMemcpyDeviceToHost));
+  if (nm == "d_gu") {
+    // undo the physical interleave: [T, 2f] columns back to gate | up
+    std::vector<uint16_t> tmp(2 * f);
+    uint16_t* rows = reinterpret_cast<uint16_t*>(host_dst);
+    for (size_t t = 0; t < T; ++t) {
+      uint16_t* r = rows + t * 2 * f;
+      for (size_t c = 0; c < 2 * f; ++c) tmp[c] = r[wgu_phys_row((int64_t)c, (int64_t)f)];
+      memcpy(r, tmp.data(), 2 * f * sizeof(uint16_t));
+    }
+  }
+  return FT_OK;
+}
+
+const char* ft_last_error(const ft_model* m) { return m ? m->err.c_str() : "null model"; }
+int64_t ft_launch_count(const ft_model* m) { return m ? m->launches : 0; }
+void ft_destroy(ft_model* m) { delete m; }
+
+// ---------------------------------------------------------------- single kernels
+ft_status ft_k_gemm(const void* dev_A, int32_t a_mn, int64_t lda, const void* dev_B, int32_t b_mn, int64_t ldb,
+                    void* dev_C, int64_t ldc, const void* dev_resid, int32_t out_kind, int32_t M, int32_t N, int32_t K,
+                    int32_t* dev_err, void* stream) {
+  if (out_kind < 0 || out_kind > 3) return FT_EINVAL;
+  GemmArgs g;
+  g.A = reinterpret_cast<const bf16*>(dev_A); g.a_mn = a_mn; g.lda = lda;
+  g.B = reinterpret_cast<const bf16*>(dev_B); g.b_mn = b_mn; g.ldb = ldb;
+  g.C = dev_C; g.ldc = ldc; g.resid = reinterpret_cast<const bf16*>(dev_resid);
+  g.epi = out_kind; g.M = M; g.N = N; g.K = K; g.err = dev_err;
+  cudaError_t e = launch_gemm(g, reinterpret_cast<cudaStream_t>(stream));
+  if (e == cudaErrorInvalidValue) return FT_EINVAL;
+  return e == cudaSuccess ? FT_OK : FT_ECUDA;
+}
+
+ft_status ft_k_attention_fwd(const void* dev_qkv, void* dev_o, float* dev_lse, int32_t B, int32_t S, int32_t n_heads,
+                             int32_t n_kv_heads, int32_t head_dim, void* stream) {
+  if (!dev_qkv || !dev_o || !dev_lse) return FT_EINVAL;
+  cudaError_t e = attention_fwd(reinterpret_cast<const bf16*>(dev_qkv), reinterpret_cast<bf16*>(dev_o), dev_lse, B, S,
+                                n_heads, n_kv_heads, head_dim, reinterpret_cast<cudaStream_t>(stream));
+  if (e == cudaErrorInvalidValue) return FT_EINVAL;
+  return e == cudaSuccess ? FT_OK : FT_ECUDA;
+}
+
+ft_status ft_k_attention_bwd(const void* dev_qkv, const void* dev_o, const void* dev_do, const float* dev_lse,
+                             float* dev_delta, void* dev_dqkv, const float* dev_cos, const float* dev_sin, int32_t B,
+                             int32_t S, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, void* stream) {
+  if (!dev_qkv || !dev_o || !dev_do || !dev_lse || !dev_delta || !dev_dqkv) return FT_EINVAL;
+  cudaError_t e = attention_bwd(reinterpret_cast<const bf16*>(dev_qkv), reinterpret_cast<const bf16*>(dev_o),
+                                reinterpret_cast<const bf16*>(dev_do), dev_lse, dev_delta,
+                                reinterpret_cast<bf16*>(dev_dqkv), dev_cos, dev_sin, B, S, n_heads, n_kv_heads, head_dim,
+                                reinterpret_cast<cudaStream_t>(stream));
+  if (e == cudaErrorInvalidValue) return FT_EINVAL;
+  return e == cudaSuccess ? FT_OK : FT_ECUDA;
+}
+
+}  // extern "C"

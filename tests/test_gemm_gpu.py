@@ -1,0 +1,92 @@
+"""tcgen05 GEMM family against the fp64 contraction of the same bf16 inputs (through the C ABI)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import decoder as D
+
+pytestmark = pytest.mark.gpu
+
+
+def _bf16_tensor(rng, shape, scale=1.0):
+    a = D.bf16_round(rng.standard_normal(shape) * scale)
+    return a, torch.from_numpy(a.astype(np.float32)).to(torch.bfloat16).cuda()
+
+
+def _run(M, N, K, a_mn, b_mn, out_kind, seed=0):
+    from paper_2609_13645_b200 import binding as B
+    rng = np.random.default_rng(seed)
+    A, At = _bf16_tensor(rng, (K, M) if a_mn else (M, K))
+    Bm, Bt = _bf16_tensor(rng, (K, N) if b_mn else (N, K))
+    ref = (A.T if a_mn else A) @ (Bm if b_mn else Bm.T)
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    resid = None
+    if out_kind in (0, 1):
+        out = torch.full((M, N), 7.0, dtype=torch.bfloat16, device="cuda")
+        if out_kind == 1:
+            R_, resid = _bf16_tensor(rng, (M, N))
+            ref = ref + R_
+        ref = D.bf16_round(ref)
+    else:
+        out = torch.full((M, N), 0.5, dtype=torch.float32, device="cuda")
+        if out_kind == 3:
+            ref = ref + 0.5
+    B.k_gemm(At, a_mn, Bt, b_mn, out, out_kind, M, N, K, err, resid)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
+    got = out.float().cpu().numpy().astype(np.float64)
+    rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
+    return rel, got, ref
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 128, 64), (256, 256, 256), (384, 768, 320), (200, 136, 72), (1000, 1376, 256),
+                                   (256, 256, 688)])
+def test_forward_layout_bf16_out(M, N, K):
+    rel, got, ref = _run(M, N, K, 0, 0, 0)
+    assert rel < 2e-3, rel
+    # apart from roundings that flip at a tie, every element is the correctly rounded fp64 result
+    assert np.mean(got != ref) < 0.02
+    assert np.max(np.abs(got - ref) / (np.abs(ref) + 1e-3)) < 2.0 ** -6
+
+
+@pytest.mark.parametrize("M,N,K", [(256, 256, 256), (200, 136, 1376), (512, 688, 256)])
+def test_data_gradient_layout(M, N, K):
+    rel, got, ref = _run(M, N, K, 0, 1, 0)
+    assert rel < 2e-3, rel
+    assert np.mean(got != ref) < 0.02
+
+
+@pytest.mark.parametrize("M,N,K", [(256, 256, 256), (768, 256, 200), (256, 688, 1000), (1376, 256, 264)])
+def test_weight_gradient_layout_fp32_out(M, N, K):
+    rel, got, ref = _run(M, N, K, 1, 1, 2)
+    assert rel < 1e-5, rel
+
+
+def test_fp32_accumulate_and_residual_epilogues():
+    rel, _, _ = _run(256, 384, 192, 1, 1, 3)
+    assert rel < 1e-5, rel
+    rel, got, ref = _run(300, 256, 128, 0, 0, 1)
+    assert rel < 2e-3 and np.mean(got != ref) < 0.02
+    rel, _, _ = _run(256, 1024, 256, 0, 0, 2)
+    assert rel < 1e-5
+
+
+def test_large_tile_variant_many_tiles():
+    # enough 128x256 tiles to fill every SM: the wide-tile kernel with its double-buffered accumulator
+    rel, got, ref = _run(2048, 4096, 512, 0, 0, 0, seed=3)
+    assert rel < 2e-3 and np.mean(got != ref) < 0.02
+    rel, _, _ = _run(4096, 2048, 384, 1, 1, 2, seed=4)
+    assert rel < 1e-5
+    rel, got, ref = _run(2048, 4096, 520, 0, 1, 0, seed=5)
+    assert rel < 2e-3
+
+
+def test_bad_arguments_are_rejected_without_launching():
+    from paper_2609_13645_b200 import binding as B
+    a = torch.zeros(128, 64, dtype=torch.bfloat16, device="cuda")
+    c = torch.zeros(128, 128, dtype=torch.bfloat16, device="cuda")
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    with pytest.raises(B.ForgeStepError):
+        B.k_gemm(a, 0, a, 0, c, 0, 128, 124, 64, err)  # N not a multiple of 8
+    with pytest.raises(B.ForgeStepError):
+        B.k_gemm(a, 1, a, 0, c, 0, 64, 128, 128, err)  # mn-major A with k-major B is not offered
