@@ -459,14 +459,14 @@ __device__ __forceinline__ unsigned long long splitmix64(unsigned long long z) {
 }
 
 __global__ void init_normal_kernel(float* __restrict__ p, size_t n, unsigned long long seed, unsigned long long tensor_id,
-                                   float stddev) {
+                                   double stddev) {
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
     const unsigned long long k = seed ^ ((tensor_id + 1ull) * 0xD1B54A32D192ED03ull) ^ ((unsigned long long)i * 0x8CB92BA72F3D8DD7ull);
     const unsigned long long r = splitmix64(k);
     const double u1 = ((double)(r >> 40) + 1.0) / 16777216.0;
     const double u2 = (double)((r >> 16) & 0xFFFFFFull) / 16777216.0;
     const double z = sqrt(-2.0 * log(u1)) * cos(6.283185307179586476925286766559 * u2);
-    p[i] = (float)(z * (double)stddev);
+    p[i] = (float)(z * stddev);
   }
 }
 
@@ -582,7 +582,7 @@ int adamw(float* p, float* m, float* v, const float* g, bf16* pb, size_t n, size
   return ok(1);
 }
 
-int init_normal(float* p, size_t n, uint64_t seed, int tensor_id, float stddev, cudaStream_t st) {
+int init_normal(float* p, size_t n, uint64_t seed, int tensor_id, double stddev, cudaStream_t st) {
   init_normal_kernel<<<grid_for(n, 256), 256, 0, st>>>(p, n, seed, (unsigned long long)tensor_id, stddev);
   return ok(1);
 }

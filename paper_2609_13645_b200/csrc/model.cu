@@ -470,10 +470,10 @@ ft_status ft_init_model(const ft_config* cfg, uint64_t seed, void* dev_workspace
     if (p.cols) {
       // element e of the LOGICAL tensor i gets draw (seed, i, e); wgu is drawn logically, then placed physically
       if (!p.is_wgu) {
-        FT_LAUNCH(init_normal(m->master + p.offset, p.numel(), seed, (int)i, 0.02f, st));
+        FT_LAUNCH(init_normal(m->master + p.offset, p.numel(), seed, (int)i, 0.02, st));
       } else {
         float* tmp = m->grad + p.offset;  // the gradient arena is free at this point
-        FT_LAUNCH(init_normal(tmp, p.numel(), seed, (int)i, 0.02f, st));
+        FT_LAUNCH(init_normal(tmp, p.numel(), seed, (int)i, 0.02, st));
         for (int64_t r0 = 0; r0 < 2 * (int64_t)m->f; r0 += 16) {
           const int64_t pr = wgu_phys_row(r0, m->f);
           FT_CUDA(cudaMemcpyAsync(m->master + p.offset + pr * p.cols, tmp + r0 * p.cols, 16 * p.cols * sizeof(float),
