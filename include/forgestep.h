@@ -97,6 +97,17 @@ ft_status ft_set_step(ft_model* m, int64_t step);
 ft_status ft_get_tap(ft_model* m, const char* name, int32_t layer, void* host_dst, size_t bytes,
                      size_t* out_bytes, int32_t* dtype);
 
+/* Per-class kernel timing with CUDA events recorded on the model's stream around every launch.  While enabled
+ * the step still never synchronises; ft_get_profile synchronises and returns, for one class, the summed device
+ * time (ms), the summed algorithmic work (FLOPs for FT_PROF_GEMM and the attention classes, bytes otherwise) and
+ * the number of kernels.  Enabling resets the totals. */
+typedef enum {
+  FT_PROF_GEMM = 0, FT_PROF_ATTN_FWD = 1, FT_PROF_ATTN_BWD = 2, FT_PROF_NORM = 3, FT_PROF_ELEMENTWISE = 4,
+  FT_PROF_CE = 5, FT_PROF_OPTIMIZER = 6, FT_PROF_CLASSES = 7
+} ft_prof_class;
+ft_status ft_set_profiling(ft_model* m, int32_t enable);
+ft_status ft_get_profile(ft_model* m, int32_t cls, double* ms, double* work, int64_t* launches);
+
 const char* ft_last_error(const ft_model* m);
 /* Number of kernels the library launched since the model was created (for launch accounting). */
 int64_t ft_launch_count(const ft_model* m);

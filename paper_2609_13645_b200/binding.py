@@ -18,6 +18,7 @@ _lib = None
 FT_OK, FT_EINVAL, FT_ENOMEM, FT_ECUDA, FT_ENONFINITE, FT_ETIMEOUT, FT_ENOTFOUND = range(7)
 STATUS_NAMES = ["FT_OK", "FT_EINVAL", "FT_ENOMEM", "FT_ECUDA", "FT_ENONFINITE", "FT_ETIMEOUT", "FT_ENOTFOUND"]
 KIND_MASTER, KIND_BF16, KIND_ADAM_M, KIND_ADAM_V, KIND_GRAD = range(5)
+PROF_CLASSES = ["gemm", "attn_fwd", "attn_bwd", "norm", "elementwise", "ce", "optimizer"]
 
 
 class FtConfig(C.Structure):
@@ -63,6 +64,10 @@ def lib():
         L.ft_last_error.argtypes = [vp]
         L.ft_launch_count.restype = i64
         L.ft_launch_count.argtypes = [vp]
+        L.ft_set_profiling.argtypes = [vp, i32]
+        L.ft_set_profiling.restype = C.c_int
+        L.ft_get_profile.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(i64)]
+        L.ft_get_profile.restype = C.c_int
         L.ft_destroy.restype = None
         L.ft_destroy.argtypes = [vp]
         L.ft_k_gemm.argtypes = [vp, i32, i64, vp, i32, i64, vp, i64, vp, i32, i32, i32, i32, vp, vp]
@@ -210,6 +215,18 @@ class Model:
         self._check(lib().ft_get_tap(self._h, name.encode(), layer, C.c_void_p(buf.ctypes.data), buf.nbytes,
                                      C.byref(need), C.byref(dt)))
         return buf.view(np.float32).copy() if dt.value == 1 else bf16_bits_to_f32(buf.view(np.uint16))
+
+    def set_profiling(self, enable: bool):
+        self._check(lib().ft_set_profiling(self._h, 1 if enable else 0))
+
+    def get_profile(self) -> Dict[str, Dict[str, float]]:
+        """Per kernel class: device milliseconds, algorithmic work (FLOPs or bytes) and kernel count."""
+        out = {}
+        for cls, name in enumerate(PROF_CLASSES):
+            ms, work, n = C.c_double(), C.c_double(), C.c_int64()
+            self._check(lib().ft_get_profile(self._h, cls, C.byref(ms), C.byref(work), C.byref(n)))
+            out[name] = dict(ms=ms.value, work=work.value, launches=int(n.value))
+        return out
 
     @property
     def launch_count(self) -> int:

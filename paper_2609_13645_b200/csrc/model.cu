@@ -80,6 +80,16 @@ struct ft_model {
   int lastB = 0, lastS = 0;
   bool have_bwd = false;
 
+  // optional per-class timing with CUDA events on the model's stream
+  struct ProfRec { cudaEvent_t a, b; int cls; double work; };
+  bool prof = false;
+  std::vector<ProfRec> prof_pending;
+  std::vector<cudaEvent_t> prof_pool;
+  double prof_ms[FT_PROF_CLASSES] = {0};
+  double prof_work[FT_PROF_CLASSES] = {0};
+  int64_t prof_launches[FT_PROF_CLASSES] = {0};
+  cudaEvent_t prof_cur = nullptr;
+
   const ParamInfo& P(int i) const { return params[i]; }
   int idx_layer(int l, int k) const { return 1 + l * 6 + k; }  // k: 0 norm1, 1 wqkv, 2 wo, 3 norm2, 4 wgu, 5 wd
   bf16* wb(int i) const { return pbf + params[i].offset; }
@@ -202,18 +212,54 @@ ft_status cuda_fail(ft_model* m, cudaError_t e, const char* where) {
     cudaError_t e__ = (call);                                      \
     if (e__ != cudaSuccess) return cuda_fail(m, e__, #call);       \
   } while (0)
-#define FT_LAUNCH(call)                                                                     \
+// cls: profiling class of the launch, work: its algorithmic bytes (or flops for contractions)
+#define FT_LAUNCH(cls, work, call)                                                          \
   do {                                                                                      \
+    prof_begin(m);                                                                          \
     int n__ = (call);                                                                       \
     if (n__ < 0) return fail(m, FT_ECUDA, std::string("kernel launch failed: ") + #call);   \
     m->launches += n__;                                                                     \
+    prof_end(m, cls, work, n__);                                                            \
   } while (0)
 #define FT_GEMM(args)                                                                       \
   do {                                                                                      \
+    prof_begin(m);                                                                          \
     cudaError_t e__ = launch_gemm(args, m->stream);                                         \
     if (e__ != cudaSuccess) return cuda_fail(m, e__, "launch_gemm");                        \
     m->launches += 1;                                                                       \
+    prof_end(m, FT_PROF_GEMM, 2.0 * (double)(args).M * (double)(args).N * (double)(args).K, 1); \
   } while (0)
+
+cudaEvent_t prof_event(ft_model* m) {
+  if (!m->prof_pool.empty()) { cudaEvent_t e = m->prof_pool.back(); m->prof_pool.pop_back(); return e; }
+  cudaEvent_t e = nullptr;
+  cudaEventCreate(&e);
+  return e;
+}
+inline void prof_begin(ft_model* m) {
+  if (!m->prof) return;
+  m->prof_cur = prof_event(m);
+  cudaEventRecord(m->prof_cur, m->stream);
+}
+inline void prof_end(ft_model* m, int cls, double work, int launches) {
+  if (!m->prof || !m->prof_cur) return;
+  ft_model::ProfRec r;
+  r.a = m->prof_cur; r.b = prof_event(m); r.cls = cls; r.work = work;
+  cudaEventRecord(r.b, m->stream);
+  m->prof_pending.push_back(r);
+  m->prof_launches[cls] += launches;
+  m->prof_cur = nullptr;
+}
+// turns finished event pairs into per-class totals (the stream must be idle)
+void prof_collect(ft_model* m) {
+  for (auto& r : m->prof_pending) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, r.a, r.b) == cudaSuccess) { m->prof_ms[r.cls] += ms; m->prof_work[r.cls] += r.work; }
+    m->prof_pool.push_back(r.a);
+    m->prof_pool.push_back(r.b);
+  }
+  m->prof_pending.clear();
+}
 
 AdamHyper hyper(const ft_model* m) {
   AdamHyper hp;
@@ -232,7 +278,7 @@ GemmArgs gemm_base(ft_model* m) {
 ft_status layer_forward(ft_model* m, int l, LayerActs& a, int B, int S) {
   const int T = B * S, h = m->h, f = m->f, hq = m->hq, nqkv = m->nqkv;
   cudaStream_t st = m->stream;
-  FT_LAUNCH(rmsnorm_fwd(m->x[l], m->wb(m->idx_layer(l, 0)), a.h1, a.r1, T, h, m->cfg.rms_eps, st));
+  FT_LAUNCH(FT_PROF_NORM, 4.0 * T * h, rmsnorm_fwd(m->x[l], m->wb(m->idx_layer(l, 0)), a.h1, a.r1, T, h, m->cfg.rms_eps, st));
   {
     GemmArgs g = gemm_base(m);
     g.A = a.h1; g.lda = h; g.B = m->wb(m->idx_layer(l, 1)); g.ldb = h; g.C = a.qkv; g.ldc = nqkv;
@@ -240,15 +286,17 @@ ft_status layer_forward(ft_model* m, int l, LayerActs& a, int B, int S) {
     g.rope_cos = m->rope_cos; g.rope_sin = m->rope_sin; g.seq = S; g.head_dim = m->d; g.rope_cols = hq + m->hkv;
     FT_GEMM(g);
   }
+  prof_begin(m);
   FT_CUDA(attention_fwd(a.qkv, a.o, a.lse, B, S, m->cfg.n_heads, m->cfg.n_kv_heads, m->d, st));
   m->launches += 1;
+  prof_end(m, FT_PROF_ATTN_FWD, 2.0 * B * m->cfg.n_heads * (double)S * S * m->d, 1);
   {
     GemmArgs g = gemm_base(m);
     g.A = a.o; g.lda = hq; g.B = m->wb(m->idx_layer(l, 2)); g.ldb = hq; g.C = a.x_mid; g.ldc = h; g.resid = m->x[l];
     g.M = T; g.N = h; g.K = hq; g.epi = EPI_BF16_RESID;
     FT_GEMM(g);
   }
-  FT_LAUNCH(rmsnorm_fwd(a.x_mid, m->wb(m->idx_layer(l, 3)), a.h2, a.r2, T, h, m->cfg.rms_eps, st));
+  FT_LAUNCH(FT_PROF_NORM, 4.0 * T * h, rmsnorm_fwd(a.x_mid, m->wb(m->idx_layer(l, 3)), a.h2, a.r2, T, h, m->cfg.rms_eps, st));
   {
     GemmArgs g = gemm_base(m);
     g.A = a.h2; g.lda = h; g.B = m->wb(m->idx_layer(l, 4)); g.ldb = h; g.C = a.a; g.ldc = f; g.gu = a.gu; g.d_ffn = f;
@@ -294,7 +342,7 @@ ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
   if (tp) { ft_status s = copy_tap(m, tp->d_x_out, m->dxA, (size_t)T * h); if (s) return s; }
   ft_status s = linear_backward(m, m->dxA, a.a, m->idx_layer(l, 5), m->d_a, T, h, f);
   if (s) return s;
-  FT_LAUNCH(swiglu_bwd(m->d_a, a.gu, m->d_gu, T, f, st));
+  FT_LAUNCH(FT_PROF_ELEMENTWISE, 10.0 * T * f, swiglu_bwd(m->d_a, a.gu, m->d_gu, T, f, st));
   s = linear_backward(m, m->d_gu, a.h2, m->idx_layer(l, 4), m->d_h, T, 2 * f, h);
   if (s) return s;
   if (tp) {
@@ -302,13 +350,15 @@ ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
     if ((s = copy_tap(m, tp->d_gu, m->d_gu, (size_t)T * 2 * f))) return s;
     if ((s = copy_tap(m, tp->d_h2, m->d_h, (size_t)T * h))) return s;
   }
-  FT_LAUNCH(rmsnorm_bwd(m->d_h, a.x_mid, a.r2, m->wb(m->idx_layer(l, 3)), m->dxA, m->dxB, m->gr(m->idx_layer(l, 3)),
-                        m->norm_partial, T, h, st));
+  FT_LAUNCH(FT_PROF_NORM, 8.0 * T * h, rmsnorm_bwd(m->d_h, a.x_mid, a.r2, m->wb(m->idx_layer(l, 3)), m->dxA, m->dxB,
+                                                    m->gr(m->idx_layer(l, 3)), m->norm_partial, T, h, st));
   s = linear_backward(m, m->dxB, a.o, m->idx_layer(l, 2), m->d_o, T, h, hq);
   if (s) return s;
+  prof_begin(m);
   FT_CUDA(attention_bwd(a.qkv, a.o, m->d_o, a.lse, m->delta, m->d_qkv, m->rope_cos, m->rope_sin, B, S, m->cfg.n_heads,
                         m->cfg.n_kv_heads, m->d, st));
   m->launches += 3;
+  prof_end(m, FT_PROF_ATTN_BWD, 4.0 * B * m->cfg.n_heads * (double)S * S * m->d, 3);
   s = linear_backward(m, m->d_qkv, a.h1, m->idx_layer(l, 1), m->d_h, T, nqkv, h);
   if (s) return s;
   if (tp) {
@@ -317,8 +367,8 @@ ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
     if ((s = copy_tap(m, tp->d_qkv, m->d_qkv, (size_t)T * nqkv))) return s;
     if ((s = copy_tap(m, tp->d_h1, m->d_h, (size_t)T * h))) return s;
   }
-  FT_LAUNCH(rmsnorm_bwd(m->d_h, m->x[l], a.r1, m->wb(m->idx_layer(l, 0)), m->dxB, m->dxA, m->gr(m->idx_layer(l, 0)),
-                        m->norm_partial, T, h, st));
+  FT_LAUNCH(FT_PROF_NORM, 8.0 * T * h, rmsnorm_bwd(m->d_h, m->x[l], a.r1, m->wb(m->idx_layer(l, 0)), m->dxB, m->dxA,
+                                                    m->gr(m->idx_layer(l, 0)), m->norm_partial, T, h, st));
   if (tp) { if ((s = copy_tap(m, tp->d_x_in, m->dxA, (size_t)T * h))) return s; }
   return FT_OK;
 }
@@ -331,14 +381,14 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
   cudaStream_t st = m->stream;
   m->lastB = B; m->lastS = S; m->have_bwd = false;
 
-  FT_LAUNCH(count_labels(lab, T, m->sc, st));
-  FT_LAUNCH(embed_fwd(tok, m->wb(0), m->x[0], T, h, V, st));
+  FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T, count_labels(lab, T, m->sc, st));
+  FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T * h, embed_fwd(tok, m->wb(0), m->x[0], T, h, V, st));
   for (int l = 0; l < L; ++l) {
     ft_status s = layer_forward(m, l, m->acts[m->cfg.recompute ? 0 : l], B, S);
     if (s) return s;
   }
   const int i_normf = 1 + 6 * L, i_head = 2 + 6 * L;
-  FT_LAUNCH(rmsnorm_fwd(m->x[L], m->wb(i_normf), m->hF, m->rF, T, h, m->cfg.rms_eps, st));
+  FT_LAUNCH(FT_PROF_NORM, 4.0 * T * h, rmsnorm_fwd(m->x[L], m->wb(i_normf), m->hF, m->rF, T, h, m->cfg.rms_eps, st));
 
   // output head + cross-entropy (+ both head gradients) in chunks of rows: the logits of one chunk at a time
   for (int r0 = 0, chunk = 0; r0 < T; r0 += m->ce_chunk, ++chunk) {
@@ -349,7 +399,8 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
       g.M = rows; g.N = V; g.K = h; g.epi = EPI_F32;
       FT_GEMM(g);
     }
-    FT_LAUNCH(cross_entropy_rows(m->z, lab + r0, m->ce_lse + r0, m->loss_row + r0, with_bwd ? m->dz : nullptr, rows, V,
+    FT_LAUNCH(FT_PROF_CE, (with_bwd ? 10.0 : 4.0) * rows * V,
+              cross_entropy_rows(m->z, lab + r0, m->ce_lse + r0, m->loss_row + r0, with_bwd ? m->dz : nullptr, rows, V,
                                  m->sc, st));
     if (with_bwd) {
       {
@@ -366,11 +417,11 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
       }
     }
   }
-  FT_LAUNCH(reduce_loss(m->loss_row, T, m->sc, st));
+  FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T, reduce_loss(m->loss_row, T, m->sc, st));
   if (!with_bwd) return FT_OK;
 
-  FT_LAUNCH(rmsnorm_bwd(m->d_hF, m->x[L], m->rF, m->wb(i_normf), nullptr, m->dxA, m->gr(i_normf), m->norm_partial, T, h,
-                        st));
+  FT_LAUNCH(FT_PROF_NORM, 6.0 * T * h,
+            rmsnorm_bwd(m->d_hF, m->x[L], m->rF, m->wb(i_normf), nullptr, m->dxA, m->gr(i_normf), m->norm_partial, T, h, st));
   for (int l = L - 1; l >= 0; --l) {
     LayerActs& a = m->acts[m->cfg.recompute ? 0 : l];
     if (m->cfg.recompute) {
@@ -382,7 +433,7 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
     ft_status s = layer_backward(m, l, a, B, S);
     if (s) return s;
   }
-  FT_LAUNCH(embed_bwd(tok, m->dxA, m->gr(0), m->keys, T, h, V, st));
+  FT_LAUNCH(FT_PROF_ELEMENTWISE, 2.0 * T * h + 4.0 * V * h, embed_bwd(tok, m->dxA, m->gr(0), m->keys, T, h, V, st));
   m->have_bwd = true;
   return FT_OK;
 }
@@ -390,9 +441,9 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
 ft_status run_update(ft_model* m) {
   cudaStream_t st = m->stream;
   const AdamHyper hp = hyper(m);
-  FT_LAUNCH(grad_norm_and_clip(m->grad, m->arena, m->sq_partial, m->sc, hp, st));
-  FT_LAUNCH(advance_step(m->sc, hp, st));
-  FT_LAUNCH(adamw(m->master, m->adam_m, m->adam_v, m->grad, m->pbf, m->arena, m->n_decay, m->sc, hp, st));
+  FT_LAUNCH(FT_PROF_OPTIMIZER, 4.0 * m->arena, grad_norm_and_clip(m->grad, m->arena, m->sq_partial, m->sc, hp, st));
+  FT_LAUNCH(FT_PROF_OPTIMIZER, 0.0, advance_step(m->sc, hp, st));
+  FT_LAUNCH(FT_PROF_OPTIMIZER, 30.0 * m->arena, adamw(m->master, m->adam_m, m->adam_v, m->grad, m->pbf, m->arena, m->n_decay, m->sc, hp, st));
   return FT_OK;
 }
 
@@ -470,10 +521,10 @@ ft_status ft_init_model(const ft_config* cfg, uint64_t seed, void* dev_workspace
     if (p.cols) {
       // element e of the LOGICAL tensor i gets draw (seed, i, e); wgu is drawn logically, then placed physically
       if (!p.is_wgu) {
-        FT_LAUNCH(init_normal(m->master + p.offset, p.numel(), seed, (int)i, 0.02, st));
+        FT_LAUNCH(FT_PROF_ELEMENTWISE, 0.0, init_normal(m->master + p.offset, p.numel(), seed, (int)i, 0.02, st));
       } else {
         float* tmp = m->grad + p.offset;  // the gradient arena is free at this point
-        FT_LAUNCH(init_normal(tmp, p.numel(), seed, (int)i, 0.02, st));
+        FT_LAUNCH(FT_PROF_ELEMENTWISE, 0.0, init_normal(tmp, p.numel(), seed, (int)i, 0.02, st));
         for (int64_t r0 = 0; r0 < 2 * (int64_t)m->f; r0 += 16) {
           const int64_t pr = wgu_phys_row(r0, m->f);
           FT_CUDA(cudaMemcpyAsync(m->master + p.offset + pr * p.cols, tmp + r0 * p.cols, 16 * p.cols * sizeof(float),
@@ -481,11 +532,11 @@ ft_status ft_init_model(const ft_config* cfg, uint64_t seed, void* dev_workspace
         }
       }
     } else {
-      FT_LAUNCH(fill_f32(m->master + p.offset, p.numel(), 1.0f, st));
+      FT_LAUNCH(FT_PROF_ELEMENTWISE, 0.0, fill_f32(m->master + p.offset, p.numel(), 1.0f, st));
     }
   }
   FT_CUDA(cudaMemsetAsync(m->grad, 0, m->arena * sizeof(float), st));
-  FT_LAUNCH(cast_bf16(m->master, m->pbf, m->arena, st));
+  FT_LAUNCH(FT_PROF_ELEMENTWISE, 0.0, cast_bf16(m->master, m->pbf, m->arena, st));
 
   // RoPE tables: angle(p, i) = p * theta^(-2i/d), evaluated in double on the host, stored as fp32
   {
@@ -588,7 +639,7 @@ static ft_status param_copy(ft_model* m, int32_t i, ft_kind kind, void* host, si
   }
   if (!to_host && kind == FT_MASTER_F32) {
     const size_t span = align_up(p.numel(), 128);
-    FT_LAUNCH(cast_bf16(m->master + p.offset, m->pbf + p.offset, span, m->stream));
+    FT_LAUNCH(FT_PROF_ELEMENTWISE, 0.0, cast_bf16(m->master + p.offset, m->pbf + p.offset, span, m->stream));
     FT_CUDA(cudaStreamSynchronize(m->stream));
   }
   return FT_OK;
@@ -680,9 +731,35 @@ ft_status ft_get_tap(ft_model* m, const char* name, int32_t layer, void* host_ds
   return FT_OK;
 }
 
+ft_status ft_set_profiling(ft_model* m, int32_t enable) {
+  if (!m) return FT_EINVAL;
+  FT_CUDA(cudaStreamSynchronize(m->stream));
+  prof_collect(m);
+  m->prof = enable != 0;
+  if (enable) {
+    for (int c = 0; c < FT_PROF_CLASSES; ++c) { m->prof_ms[c] = 0; m->prof_work[c] = 0; m->prof_launches[c] = 0; }
+  }
+  return FT_OK;
+}
+
+ft_status ft_get_profile(ft_model* m, int32_t cls, double* ms, double* work, int64_t* launches) {
+  if (!m || cls < 0 || cls >= FT_PROF_CLASSES) return FT_EINVAL;
+  FT_CUDA(cudaStreamSynchronize(m->stream));
+  prof_collect(m);
+  if (ms) *ms = m->prof_ms[cls];
+  if (work) *work = m->prof_work[cls];
+  if (launches) *launches = m->prof_launches[cls];
+  return FT_OK;
+}
+
 const char* ft_last_error(const ft_model* m) { return m ? m->err.c_str() : "null model"; }
 int64_t ft_launch_count(const ft_model* m) { return m ? m->launches : 0; }
-void ft_destroy(ft_model* m) { delete m; }
+void ft_destroy(ft_model* m) {
+  if (!m) return;
+  for (auto& r : m->prof_pending) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+  for (auto e : m->prof_pool) cudaEventDestroy(e);
+  delete m;
+}
 
 // ---------------------------------------------------------------- single kernels
 ft_status ft_k_gemm(const void* dev_A, int32_t a_mn, int64_t lda, const void* dev_B, int32_t b_mn, int64_t ldb,
