@@ -1,0 +1,94 @@
+"""Times one kernel of the library through the C ABI with CUDA events (also the target of ncu captures).
+
+    python -m paper_2609_13645_b200.kernel_bench gemm --M 8192 --N 11264 --K 2048 --layout tn --iters 20
+    python -m paper_2609_13645_b200.kernel_bench attn_fwd --B 4 --S 2048 --nh 16 --nkv 8 --d 128
+    python -m paper_2609_13645_b200.kernel_bench attn_bwd --B 4 --S 2048 --nh 16 --nkv 8 --d 128
+
+Inputs are random bf16; between timed launches a 256 MB buffer is rewritten so the operands do not sit in L2.
+Prints one JSON line with the mean launch time and the achieved TFLOP/s.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+
+sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+
+
+def main():
+    import torch
+    from paper_2609_13645_b200 import binding as B
+
+    ap = argparse.ArgumentParser()
+    ap.add_argument("kernel", choices=["gemm", "attn_fwd", "attn_bwd"])
+    ap.add_argument("--M", type=int, default=8192)
+    ap.add_argument("--N", type=int, default=4096)
+    ap.add_argument("--K", type=int, default=2048)
+    ap.add_argument("--layout", default="tn", choices=["tn", "nn", "wgrad"])
+    ap.add_argument("--B", type=int, default=4)
+    ap.add_argument("--S", type=int, default=2048)
+    ap.add_argument("--nh", type=int, default=16)
+    ap.add_argument("--nkv", type=int, default=8)
+    ap.add_argument("--d", type=int, default=128)
+    ap.add_argument("--iters", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--no-flush", action="store_true")
+    a = ap.parse_args()
+    torch.manual_seed(0)
+    dev = "cuda"
+    flush = None if a.no_flush else torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    err = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    if a.kernel == "gemm":
+        M, N, K = a.M, a.N, a.K
+        if a.layout == "tn":
+            A = torch.randn(M, K, device=dev).bfloat16(); Bm = torch.randn(N, K, device=dev).bfloat16()
+            out = torch.empty(M, N, dtype=torch.bfloat16, device=dev); amn, bmn, kind = 0, 0, 0
+        elif a.layout == "nn":
+            A = torch.randn(M, K, device=dev).bfloat16(); Bm = torch.randn(K, N, device=dev).bfloat16()
+            out = torch.empty(M, N, dtype=torch.bfloat16, device=dev); amn, bmn, kind = 0, 1, 0
+        else:
+            A = torch.randn(K, M, device=dev).bfloat16(); Bm = torch.randn(K, N, device=dev).bfloat16()
+            out = torch.empty(M, N, dtype=torch.float32, device=dev); amn, bmn, kind = 1, 1, 2
+        flops = 2.0 * M * N * K
+        run = lambda: B.k_gemm(A, amn, Bm, bmn, out, kind, M, N, K, err)
+        desc = dict(kernel="gemm", layout=a.layout, M=M, N=N, K=K)
+    else:
+        Bsz, S, nh, nkv, d = a.B, a.S, a.nh, a.nkv, a.d
+        qkv = torch.randn(Bsz * S, (nh + 2 * nkv) * d, device=dev).bfloat16()
+        o = torch.empty(Bsz * S, nh * d, dtype=torch.bfloat16, device=dev)
+        lse = torch.empty(Bsz, nh, S, dtype=torch.float32, device=dev)
+        B.k_attention_fwd(qkv, o, lse, Bsz, S, nh, nkv, d)
+        fwd_flops = 2.0 * Bsz * nh * S * S * d  # causal: half of 4 B n_h S^2 d
+        if a.kernel == "attn_fwd":
+            flops = fwd_flops
+            run = lambda: B.k_attention_fwd(qkv, o, lse, Bsz, S, nh, nkv, d)
+        else:
+            do = torch.randn(Bsz * S, nh * d, device=dev).bfloat16()
+            delta = torch.empty(Bsz, nh, S, dtype=torch.float32, device=dev)
+            dqkv = torch.empty_like(qkv)
+            flops = 2.0 * fwd_flops  # model count of the backward (the paper's 1:2 ratio)
+            run = lambda: B.k_attention_bwd(qkv, o, do, lse, delta, dqkv, Bsz, S, nh, nkv, d)
+        desc = dict(kernel=a.kernel, B=Bsz, S=S, n_heads=nh, n_kv=nkv, d=d)
+
+    for _ in range(a.warmup):
+        run()
+    torch.cuda.synchronize()
+    total = 0.0
+    for _ in range(a.iters):
+        if flush is not None:
+            flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); run(); e1.record()
+        torch.cuda.synchronize()
+        total += e0.elapsed_time(e1)
+    ms = total / a.iters
+    assert int(err.item()) == 0
+    desc.update(ms=ms, tflops=flops / (ms * 1e-3) / 1e12, iters=a.iters)
+    print(json.dumps(desc))
+
+
+if __name__ == "__main__":
+    main()
