@@ -137,6 +137,23 @@ ft_status ft_k_attention_bwd(const void* dev_qkv, const void* dev_o, const void*
                              int32_t B, int32_t S, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim,
                              void* stream);
 
+/* The same backward for callers that cannot hand over scratch memory they allocated: code running where device
+ * allocation is off limits (inside a framework's allocator callback, in a plugin that is given only its input and
+ * output tensors, under a memory budget that is already fully committed) has nowhere to get the fp32 "delta"
+ * buffer that ft_k_attention_bwd needs.  Here that buffer is a fixed 4 MiB array inside the library image, so the
+ * call allocates nothing, on the device or through any library.  (The paper has no counterpart of this call.)
+ *   - Limit: B * n_heads * S <= 1,048,576; larger problems return FT_ENOMEM and launch nothing.
+ *   - Every GPU that loads the library keeps the 4 MiB until the process exits.
+ *   - The first call on each device looks up the array's device address (once, with that device current); make
+ *     that first call before starting any stream capture.
+ *   - All calls share the one array and it keeps the last call's contents; the pre-pass of each call rewrites
+ *     every element it later reads, so no clearing is needed, but two calls whose kernels overlap on the GPU
+ *     (different streams, or different threads) race on it: run them one after the other.
+ * Inputs, outputs and results are those of ft_k_attention_bwd (same kernels, same bits). */
+ft_status ft_k_attention_bwd_noalloc(const void* dev_qkv, const void* dev_o, const void* dev_do, const float* dev_lse,
+                                     void* dev_dqkv, const float* dev_cos, const float* dev_sin, int32_t B,
+                                     int32_t S, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

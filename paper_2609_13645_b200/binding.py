@@ -73,6 +73,8 @@ def lib():
         L.ft_k_gemm.argtypes = [vp, i32, i64, vp, i32, i64, vp, i64, vp, i32, i32, i32, i32, vp, vp]
         L.ft_k_attention_fwd.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp]
         L.ft_k_attention_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]
+        L.ft_k_attention_bwd_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]
+        L.ft_k_attention_bwd_noalloc.restype = C.c_int
         for name in ("ft_init_model", "ft_train_step", "ft_train_step_host", "ft_forward_loss", "ft_forward_backward",
                      "ft_apply_update", "ft_param_info", "ft_get_param", "ft_set_param", "ft_get_step", "ft_set_step",
                      "ft_get_tap", "ft_k_gemm", "ft_k_attention_fwd", "ft_k_attention_bwd"):
@@ -259,3 +261,12 @@ def k_attention_bwd(qkv, o, d_o, lse, delta, dqkv, B, S, n_heads, n_kv, d, cos=N
                                   _stream_ptr())
     if st != FT_OK:
         raise ForgeStepError(st, "ft_k_attention_bwd")
+
+
+def k_attention_bwd_noalloc(qkv, o, d_o, lse, dqkv, B, S, n_heads, n_kv, d, cos=None, sin=None):
+    """Attention backward whose scratch lives inside the library: for callers that may not allocate device memory.
+    Returns the status code instead of raising, so a caller can tell "too large for the built-in scratch" apart."""
+    return lib().ft_k_attention_bwd_noalloc(
+        C.c_void_p(qkv.data_ptr()), C.c_void_p(o.data_ptr()), C.c_void_p(d_o.data_ptr()), C.c_void_p(lse.data_ptr()),
+        C.c_void_p(dqkv.data_ptr()), C.c_void_p(cos.data_ptr()) if cos is not None else None,
+        C.c_void_p(sin.data_ptr()) if sin is not None else None, B, S, n_heads, n_kv, d, _stream_ptr())
