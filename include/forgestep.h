@@ -108,6 +108,9 @@ typedef enum {
 ft_status ft_set_profiling(ft_model* m, int32_t enable);
 ft_status ft_get_profile(ft_model* m, int32_t cls, double* ms, double* work, int64_t* launches);
 
+/* Development switch: 1 = tcgen05 attention kernels (default), 0 = warp-level mma.sync attention kernels. */
+void ft_debug_attention_impl(int32_t impl);
+
 const char* ft_last_error(const ft_model* m);
 /* Number of kernels the library launched since the model was created (for launch accounting). */
 int64_t ft_launch_count(const ft_model* m);

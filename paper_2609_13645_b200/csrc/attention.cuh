@@ -17,4 +17,13 @@ cudaError_t attention_bwd(const bf16* qkv, const bf16* o, const bf16* d_o, const
                           const float* cos, const float* sin, int B, int S, int n_heads, int n_kv, int d,
                           cudaStream_t st);
 
+// The same forward on the tcgen05 tensor cores (accumulators in TMEM, operands by TMA).  err: device status word.
+cudaError_t attention_fwd_tc(const bf16* qkv, bf16* o, float* lse, int B, int S, int n_heads, int n_kv, int d, int* err,
+                             cudaStream_t st);
+
+// Device status word used by the single-kernel entry points (address on the current device).
+int* attention_status_word();
+// 1: tcgen05 kernels where they exist (default); 0: warp-level mma.sync kernels.
+extern int g_attention_impl;
+
 }  // namespace fs

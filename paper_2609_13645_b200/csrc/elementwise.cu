@@ -62,69 +62,86 @@ __global__ void rmsnorm_fwd_kernel(const bf16* __restrict__ x, const bf16* __res
 
 // ---------------------------------------------------------------- RMSNorm backward
 // dx_k = r g_k dy_k - x_k r^3 (1/h) sum_j g_j dy_j x_j (+ resid_k);  dg_k = sum_t dy_tk x_tk r_t.
-// One warp per row, rows strided over the grid; each lane keeps the dg of its columns in registers, the 8 warps of a
-// block are then added in warp order, and a second kernel adds the block partials in block order.
+// WPR warps share a row (1 for h <= 2048, 2 above), rows strided over the grid.  A warp loads its whole share of the
+// row with all 16-byte loads in flight at once, keeps it in registers for both the dot product and the update, and
+// keeps the dg of its columns in registers; warps owning the same columns are then added in warp order, and a second
+// kernel adds the block partials in block order (no floating-point atomics anywhere).
+template <int NCHW, int WPR>
 __global__ void __launch_bounds__(256)
 rmsnorm_bwd_kernel(const bf16* __restrict__ dy, const bf16* __restrict__ x, const float* __restrict__ r,
                    const bf16* __restrict__ g, const bf16* __restrict__ resid, bf16* __restrict__ dx,
                    float* __restrict__ partial, int T, int h) {
   extern __shared__ float s_dg[];  // [h]
+  __shared__ float s_dot[2][8];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int nch = h >> 8;
-  float dg[kNormMaxChunks][8];
+  const int sub = warp % WPR;            // which part of the row this warp owns
+  const int slot = warp / WPR;           // which of the block's concurrent rows
+  constexpr int ROWS = 8 / WPR;          // rows in flight per block
+  float dg[NCHW][8];
 #pragma unroll
-  for (int i = 0; i < kNormMaxChunks; ++i)
+  for (int i = 0; i < NCHW; ++i)
 #pragma unroll
     for (int e = 0; e < 8; ++e) dg[i][e] = 0.f;
   const float inv_h = 1.0f / (float)h;
-  for (int row = blockIdx.x * 8 + warp; row < T; row += gridDim.x * 8) {
-    const bf16* dyr = dy + (long long)row * h;
-    const bf16* xr = x + (long long)row * h;
-    const float rr = r[row];
+  int parity = 0;
+  const int nrows_iter = (T + gridDim.x * ROWS - 1) / (gridDim.x * ROWS);
+  for (int it = 0; it < nrows_iter; ++it) {
+    const int row = (it * gridDim.x + blockIdx.x) * ROWS + slot;
+    const bool live = row < T;
+    uint4 vdy[NCHW], vx[NCHW], vrs[NCHW];
+#pragma unroll
+    for (int i = 0; i < NCHW; ++i) {
+      const int c = (sub * NCHW + i) * 256 + lane * 8;
+      const bool okc = live && c < h;
+      const long long off = (long long)row * h + c;
+      vdy[i] = okc ? *reinterpret_cast<const uint4*>(dy + off) : make_uint4(0, 0, 0, 0);
+      vx[i] = okc ? *reinterpret_cast<const uint4*>(x + off) : make_uint4(0, 0, 0, 0);
+      vrs[i] = (okc && resid != nullptr) ? *reinterpret_cast<const uint4*>(resid + off) : make_uint4(0, 0, 0, 0);
+    }
+    const float rr = live ? r[row] : 0.f;
     float dot = 0.f;
 #pragma unroll
-    for (int i = 0; i < kNormMaxChunks; ++i) {
-      if (i < nch) {
-        const int c = lane * 8 + (i << 8);
-        float a[8], b[8], gg[8];
-        unpack8(*reinterpret_cast<const uint4*>(dyr + c), a);
-        unpack8(*reinterpret_cast<const uint4*>(xr + c), b);
-        unpack8(*reinterpret_cast<const uint4*>(g + c), gg);
+    for (int i = 0; i < NCHW; ++i) {
+      const int c = (sub * NCHW + i) * 256 + lane * 8;
+      float a[8], b[8], gg[8];
+      unpack8(vdy[i], a);
+      unpack8(vx[i], b);
+      unpack8(c < h ? *reinterpret_cast<const uint4*>(g + c) : make_uint4(0, 0, 0, 0), gg);  // gains stay in L1
 #pragma unroll
-        for (int e = 0; e < 8; ++e) dot += gg[e] * a[e] * b[e];
-      }
+      for (int e = 0; e < 8; ++e) dot += gg[e] * a[e] * b[e];
     }
     dot = warp_sum(dot);
+    if (WPR == 2) {
+      // the two warps of a row swap their halves of the dot product (added in a fixed order)
+      if (lane == 0) s_dot[parity][warp] = dot;
+      __syncthreads();
+      const float d0 = s_dot[parity][slot * 2], d1 = s_dot[parity][slot * 2 + 1];
+      dot = d0 + d1;
+      parity ^= 1;
+    }
     const float coef = rr * rr * rr * dot * inv_h;
 #pragma unroll
-    for (int i = 0; i < kNormMaxChunks; ++i) {
-      if (i < nch) {
-        const int c = lane * 8 + (i << 8);
-        float a[8], b[8], gg[8], o[8];
-        unpack8(*reinterpret_cast<const uint4*>(dyr + c), a);
-        unpack8(*reinterpret_cast<const uint4*>(xr + c), b);
-        unpack8(*reinterpret_cast<const uint4*>(g + c), gg);
+    for (int i = 0; i < NCHW; ++i) {
+      const int c = (sub * NCHW + i) * 256 + lane * 8;
+      float a[8], b[8], gg[8], rs[8], o[8];
+      unpack8(vdy[i], a);
+      unpack8(vx[i], b);
+      unpack8(c < h ? *reinterpret_cast<const uint4*>(g + c) : make_uint4(0, 0, 0, 0), gg);
+      unpack8(vrs[i], rs);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          o[e] = rr * gg[e] * a[e] - b[e] * coef;
-          dg[i][e] += a[e] * b[e] * rr;
-        }
-        if (resid != nullptr) {
-          float rs[8];
-          unpack8(*reinterpret_cast<const uint4*>(resid + (long long)row * h + c), rs);
-#pragma unroll
-          for (int e = 0; e < 8; ++e) o[e] += rs[e];
-        }
-        *reinterpret_cast<uint4*>(dx + (long long)row * h + c) = pack8(o);
+      for (int e = 0; e < 8; ++e) {
+        o[e] = rr * gg[e] * a[e] - b[e] * coef + rs[e];
+        dg[i][e] += a[e] * b[e] * rr;
       }
+      if (live && c < h) *reinterpret_cast<uint4*>(dx + (long long)row * h + c) = pack8(o);
     }
   }
-  for (int w = 0; w < 8; ++w) {
-    if (warp == w) {
+  for (int w = 0; w < ROWS; ++w) {
+    if (slot == w) {
 #pragma unroll
-      for (int i = 0; i < kNormMaxChunks; ++i) {
-        if (i < nch) {
-          const int c = lane * 8 + (i << 8);
+      for (int i = 0; i < NCHW; ++i) {
+        const int c = (sub * NCHW + i) * 256 + lane * 8;
+        if (c < h) {
 #pragma unroll
           for (int e = 0; e < 8; ++e) s_dg[c + e] = (w == 0 ? 0.f : s_dg[c + e]) + dg[i][e];
         }
@@ -135,12 +152,23 @@ rmsnorm_bwd_kernel(const bf16* __restrict__ dy, const bf16* __restrict__ x, cons
   for (int c = threadIdx.x; c < h; c += blockDim.x) partial[(long long)blockIdx.x * h + c] = s_dg[c];
 }
 
+// out[c] = sum over blocks of partial[b][c], in block order: 32 columns x 8 row groups per CTA, the 8 groups
+// (each a fixed strided subset of the blocks) are then added in group order.
 __global__ void colsum_kernel(const float* __restrict__ partial, float* __restrict__ out, int nblk, int h) {
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= h) return;
-  float s = 0.f;
-  for (int b = 0; b < nblk; ++b) s += partial[(long long)b * h + c];
-  out[c] = s;
+  __shared__ float s[8][33];
+  const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
+  const int c = blockIdx.x * 32 + cx;
+  float a = 0.f;
+  if (c < h)
+    for (int b = ry; b < nblk; b += 8) a += partial[(long long)b * h + c];
+  s[ry][cx] = a;
+  __syncthreads();
+  if (ry == 0 && c < h) {
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += s[w][cx];
+    out[c] = tot;
+  }
 }
 
 // ---------------------------------------------------------------- SwiGLU backward
@@ -415,11 +443,17 @@ __global__ void advance_step_kernel(StepScalars* sc, AdamHyper hp) {
   sc->bc2 = (float)(1.0 - pow((double)hp.beta2, (double)t));
 }
 
+// WITH_NORM: clipping is off (coefficient 1), so the squared gradient norm is summed in the same pass and written
+// as one partial per block (fixed order: thread-strided, warp shuffle, warp order).
+template <bool WITH_NORM>
 __global__ void __launch_bounds__(256)
 adamw_kernel(float* __restrict__ p, float* __restrict__ m, float* __restrict__ v, const float* __restrict__ g,
-             bf16* __restrict__ pb, size_t n4, size_t n4_decay, const StepScalars* __restrict__ sc, AdamHyper hp) {
-  const float clip = sc->clip, bc1 = sc->bc1, bc2 = sc->bc2;
+             bf16* __restrict__ pb, size_t n4, size_t n4_decay, const StepScalars* __restrict__ sc, AdamHyper hp,
+             float* __restrict__ sq_partial) {
+  __shared__ float s_sq[8];
+  const float clip = WITH_NORM ? 1.0f : sc->clip, bc1 = sc->bc1, bc2 = sc->bc2;
   const float omb1 = 1.0f - hp.beta1, omb2 = 1.0f - hp.beta2;
+  float sq = 0.f;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
     const float wd = i < n4_decay ? hp.wd : 0.f;
     const float4 g4 = reinterpret_cast<const float4*>(g)[i];
@@ -430,6 +464,7 @@ adamw_kernel(float* __restrict__ p, float* __restrict__ m, float* __restrict__ v
     float pp[4] = {p4.x, p4.y, p4.z, p4.w};
     float mm[4] = {m4.x, m4.y, m4.z, m4.w};
     float vv[4] = {v4.x, v4.y, v4.z, v4.w};
+    if (WITH_NORM) sq += g4.x * g4.x + g4.y * g4.y + g4.z * g4.z + g4.w * g4.w;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       const float ge = gg[e] * clip;
@@ -447,6 +482,16 @@ adamw_kernel(float* __restrict__ p, float* __restrict__ m, float* __restrict__ v
     o.x = pack_bf16(pp[0], pp[1]);
     o.y = pack_bf16(pp[2], pp[3]);
     reinterpret_cast<uint2*>(pb)[i] = o;
+  }
+  if (WITH_NORM) {
+    sq = warp_sum(sq);
+    if ((threadIdx.x & 31) == 0) s_sq[threadIdx.x >> 5] = sq;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float tot = 0.f;
+      for (int w = 0; w < 8; ++w) tot += s_sq[w];
+      sq_partial[blockIdx.x] = tot;
+    }
   }
 }
 
@@ -491,7 +536,7 @@ inline int ok(int launches) { return cudaGetLastError() == cudaSuccess ? launche
 
 int elementwise_blocks_for_norm(int T) {
   const int need = (T + 7) / 8;
-  return need < 296 ? need : 296;
+  return need < 148 ? need : 148;  // one resident CTA per SM (register-bound)
 }
 
 size_t sort_pad(size_t n) {
@@ -511,12 +556,30 @@ int rmsnorm_fwd(const bf16* x, const bf16* g, bf16* y, float* r, int T, int h, f
   return ok(1);
 }
 
+template <int NCHW, int WPR>
+static void launch_rmsnorm_bwd(int nblk, const bf16* dy, const bf16* x, const float* r, const bf16* g, const bf16* resid,
+                               bf16* dx, float* partial, int T, int h, cudaStream_t st) {
+  rmsnorm_bwd_kernel<NCHW, WPR><<<nblk, 256, h * sizeof(float), st>>>(dy, x, r, g, resid, dx, partial, T, h);
+}
+
 int rmsnorm_bwd(const bf16* dy, const bf16* x, const float* r, const bf16* g, const bf16* resid, bf16* dx, float* dg,
                 float* partial, int T, int h, cudaStream_t st) {
   if ((h & 255) || h > 256 * kNormMaxChunks) return -1;
   const int nblk = elementwise_blocks_for_norm(T);
-  rmsnorm_bwd_kernel<<<nblk, 256, h * sizeof(float), st>>>(dy, x, r, g, resid, dx, partial, T, h);
-  colsum_kernel<<<(h + 255) / 256, 256, 0, st>>>(partial, dg, nblk, h);
+  const int nch = h >> 8;
+#define FS_NORM_CASE(N, W) launch_rmsnorm_bwd<N, W>(nblk, dy, x, r, g, resid, dx, partial, T, h, st); break
+  if (nch <= 8) {
+    switch (nch) {
+      case 1: FS_NORM_CASE(1, 1); case 2: FS_NORM_CASE(2, 1); case 3: FS_NORM_CASE(3, 1); case 4: FS_NORM_CASE(4, 1);
+      case 5: FS_NORM_CASE(5, 1); case 6: FS_NORM_CASE(6, 1); case 7: FS_NORM_CASE(7, 1); default: FS_NORM_CASE(8, 1);
+    }
+  } else {
+    switch ((nch + 1) / 2) {
+      case 5: FS_NORM_CASE(5, 2); case 6: FS_NORM_CASE(6, 2); case 7: FS_NORM_CASE(7, 2); default: FS_NORM_CASE(8, 2);
+    }
+  }
+#undef FS_NORM_CASE
+  colsum_kernel<<<(h + 31) / 32, 256, 0, st>>>(partial, dg, nblk, h);
   return ok(2);
 }
 
@@ -578,8 +641,15 @@ int advance_step(StepScalars* sc, AdamHyper hp, cudaStream_t st) {
 
 int adamw(float* p, float* m, float* v, const float* g, bf16* pb, size_t n, size_t n_decay, const StepScalars* sc,
           AdamHyper hp, cudaStream_t st) {
-  adamw_kernel<<<148 * 8, 256, 0, st>>>(p, m, v, g, pb, n / 4, n_decay / 4, sc, hp);
+  adamw_kernel<false><<<kSqnormBlocks, 256, 0, st>>>(p, m, v, g, pb, n / 4, n_decay / 4, sc, hp, nullptr);
   return ok(1);
+}
+
+int adamw_with_norm(float* p, float* m, float* v, const float* g, bf16* pb, size_t n, size_t n_decay, float* partial,
+                    StepScalars* sc, AdamHyper hp, cudaStream_t st) {
+  adamw_kernel<true><<<kSqnormBlocks, 256, 0, st>>>(p, m, v, g, pb, n / 4, n_decay / 4, sc, hp, partial);
+  sqnorm_final_kernel<<<1, 256, 0, st>>>(partial, kSqnormBlocks, sc, hp);
+  return ok(2);
 }
 
 int init_normal(float* p, size_t n, uint64_t seed, int tensor_id, double stddev, cudaStream_t st) {

@@ -51,6 +51,9 @@ int advance_step(StepScalars* sc, AdamHyper hp, cudaStream_t st);
 // fused clip + Adam + decoupled decay + bf16 write-back over a flat arena; elements >= n_decay get no decay
 int adamw(float* p, float* m, float* v, const float* g, bf16* pb, size_t n, size_t n_decay, const StepScalars* sc,
           AdamHyper hp, cudaStream_t st);
+// clipping off: the same pass also sums the squared gradient norm (reported, not used by the update)
+int adamw_with_norm(float* p, float* m, float* v, const float* g, bf16* pb, size_t n, size_t n_decay, float* partial,
+                    StepScalars* sc, AdamHyper hp, cudaStream_t st);
 int init_normal(float* p, size_t n, uint64_t seed, int tensor_id, double std, cudaStream_t st);
 int fill_f32(float* p, size_t n, float v, cudaStream_t st);
 int cast_bf16(const float* src, bf16* dst, size_t n, cudaStream_t st);

@@ -9,9 +9,7 @@
 // contraction runs over the rows of the stored activations) without materialising any transpose.
 #include "gemm.cuh"
 
-#include <cuda.h>
-
-#include <mutex>
+#include "tmap.cuh"
 
 namespace fs {
 
@@ -331,38 +329,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 }
 
 // ---------------------------------------------------------------- host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn get_encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static std::once_flag once;
-  std::call_once(once, [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  });
-  return fn;
-}
-
-// 2-D bf16 tensor map over a row-major matrix [rows, row_stride] of which `cols` columns are valid;
-// box = 64 columns x box_rows rows, 128-byte swizzle, zero fill outside.
-bool make_tmap(CUtensorMap* tm, const bf16* base, uint64_t cols, uint64_t rows, uint64_t row_stride, uint32_t box_rows) {
-  EncodeTiledFn enc = get_encode_fn();
-  if (!enc) return false;
-  cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {row_stride * sizeof(bf16)};
-  cuuint32_t box[2] = {64, box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<bf16*>(base), dims, strides, box, estr,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS;
-}
-
 int sm_count() {
   static int n = 0;
   if (n == 0) {
@@ -385,8 +351,8 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
     attr_set = true;
   }
   CUtensorMap tmA, tmB;
-  bool ok = A_MN ? make_tmap(&tmA, a.A, a.M, a.K, a.lda, 64) : make_tmap(&tmA, a.A, a.K, a.M, a.lda, BM);
-  ok = ok && (B_MN ? make_tmap(&tmB, a.B, a.N, a.K, a.ldb, 64) : make_tmap(&tmB, a.B, a.K, a.N, a.ldb, BN));
+  bool ok = A_MN ? make_tmap_2d(&tmA, a.A, a.M, a.K, a.lda, 64) : make_tmap_2d(&tmA, a.A, a.K, a.M, a.lda, BM);
+  ok = ok && (B_MN ? make_tmap_2d(&tmB, a.B, a.N, a.K, a.ldb, 64) : make_tmap_2d(&tmB, a.B, a.K, a.N, a.ldb, BN));
   if (!ok) return cudaErrorInvalidValue;
   GemmDev p;
   p.C = a.C; p.resid = a.resid; p.gu = a.gu; p.rope_cos = a.rope_cos; p.rope_sin = a.rope_sin; p.err = a.err;

@@ -287,7 +287,10 @@ ft_status layer_forward(ft_model* m, int l, LayerActs& a, int B, int S) {
     FT_GEMM(g);
   }
   prof_begin(m);
-  FT_CUDA(attention_fwd(a.qkv, a.o, a.lse, B, S, m->cfg.n_heads, m->cfg.n_kv_heads, m->d, st));
+  if (g_attention_impl)
+    FT_CUDA(attention_fwd_tc(a.qkv, a.o, a.lse, B, S, m->cfg.n_heads, m->cfg.n_kv_heads, m->d, &m->sc->err, st));
+  else
+    FT_CUDA(attention_fwd(a.qkv, a.o, a.lse, B, S, m->cfg.n_heads, m->cfg.n_kv_heads, m->d, st));
   m->launches += 1;
   prof_end(m, FT_PROF_ATTN_FWD, 2.0 * B * m->cfg.n_heads * (double)S * S * m->d, 1);
   {
@@ -441,9 +444,18 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
 ft_status run_update(ft_model* m) {
   cudaStream_t st = m->stream;
   const AdamHyper hp = hyper(m);
-  FT_LAUNCH(FT_PROF_OPTIMIZER, 4.0 * m->arena, grad_norm_and_clip(m->grad, m->arena, m->sq_partial, m->sc, hp, st));
-  FT_LAUNCH(FT_PROF_OPTIMIZER, 0.0, advance_step(m->sc, hp, st));
-  FT_LAUNCH(FT_PROF_OPTIMIZER, 30.0 * m->arena, adamw(m->master, m->adam_m, m->adam_v, m->grad, m->pbf, m->arena, m->n_decay, m->sc, hp, st));
+  if (hp.max_grad_norm > 0.f) {
+    FT_LAUNCH(FT_PROF_OPTIMIZER, 4.0 * m->arena, grad_norm_and_clip(m->grad, m->arena, m->sq_partial, m->sc, hp, st));
+    FT_LAUNCH(FT_PROF_OPTIMIZER, 0.0, advance_step(m->sc, hp, st));
+    FT_LAUNCH(FT_PROF_OPTIMIZER, 30.0 * m->arena,
+              adamw(m->master, m->adam_m, m->adam_v, m->grad, m->pbf, m->arena, m->n_decay, m->sc, hp, st));
+  } else {
+    // no clipping: the update does not wait for the norm, which is summed in the same pass over the gradients
+    FT_LAUNCH(FT_PROF_OPTIMIZER, 0.0, advance_step(m->sc, hp, st));
+    FT_LAUNCH(FT_PROF_OPTIMIZER, 30.0 * m->arena,
+              adamw_with_norm(m->master, m->adam_m, m->adam_v, m->grad, m->pbf, m->arena, m->n_decay, m->sq_partial,
+                              m->sc, hp, st));
+  }
   return FT_OK;
 }
 
@@ -752,6 +764,8 @@ ft_status ft_get_profile(ft_model* m, int32_t cls, double* ms, double* work, int
   return FT_OK;
 }
 
+void ft_debug_attention_impl(int32_t impl) { g_attention_impl = impl; }
+
 const char* ft_last_error(const ft_model* m) { return m ? m->err.c_str() : "null model"; }
 int64_t ft_launch_count(const ft_model* m) { return m ? m->launches : 0; }
 void ft_destroy(ft_model* m) {
@@ -779,8 +793,16 @@ ft_status ft_k_gemm(const void* dev_A, int32_t a_mn, int64_t lda, const void* de
 ft_status ft_k_attention_fwd(const void* dev_qkv, void* dev_o, float* dev_lse, int32_t B, int32_t S, int32_t n_heads,
                              int32_t n_kv_heads, int32_t head_dim, void* stream) {
   if (!dev_qkv || !dev_o || !dev_lse) return FT_EINVAL;
-  cudaError_t e = attention_fwd(reinterpret_cast<const bf16*>(dev_qkv), reinterpret_cast<bf16*>(dev_o), dev_lse, B, S,
-                                n_heads, n_kv_heads, head_dim, reinterpret_cast<cudaStream_t>(stream));
+  cudaError_t e;
+  if (g_attention_impl) {
+    int* status = attention_status_word();
+    if (!status) return FT_ECUDA;
+    e = attention_fwd_tc(reinterpret_cast<const bf16*>(dev_qkv), reinterpret_cast<bf16*>(dev_o), dev_lse, B, S, n_heads,
+                         n_kv_heads, head_dim, status, reinterpret_cast<cudaStream_t>(stream));
+  } else {
+    e = attention_fwd(reinterpret_cast<const bf16*>(dev_qkv), reinterpret_cast<bf16*>(dev_o), dev_lse, B, S, n_heads,
+                      n_kv_heads, head_dim, reinterpret_cast<cudaStream_t>(stream));
+  }
   if (e == cudaErrorInvalidValue) return FT_EINVAL;
   return e == cudaSuccess ? FT_OK : FT_ECUDA;
 }
