@@ -110,6 +110,8 @@ ft_status ft_get_profile(ft_model* m, int32_t cls, double* ms, double* work, int
 
 /* Development switch: 1 = tcgen05 attention kernels (default), 0 = warp-level mma.sync attention kernels. */
 void ft_debug_attention_impl(int32_t impl);
+/* Development switch: force the GEMM tile width (128 or 256 columns); 0 = choose by tile count (default). */
+void ft_debug_gemm_tile(int32_t bn);
 
 const char* ft_last_error(const ft_model* m);
 /* Number of kernels the library launched since the model was created (for launch accounting). */

@@ -70,6 +70,8 @@ def lib():
         L.ft_get_profile.restype = C.c_int
         L.ft_debug_attention_impl.argtypes = [i32]
         L.ft_debug_attention_impl.restype = None
+        L.ft_debug_gemm_tile.argtypes = [i32]
+        L.ft_debug_gemm_tile.restype = None
         L.ft_destroy.restype = None
         L.ft_destroy.argtypes = [vp]
         L.ft_k_gemm.argtypes = [vp, i32, i64, vp, i32, i64, vp, i64, vp, i32, i32, i32, i32, vp, vp]

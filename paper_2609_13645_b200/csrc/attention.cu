@@ -614,6 +614,15 @@ cudaError_t attention_bwd(const bf16* qkv, const bf16* o, const bf16* d_o, const
   return cudaErrorInvalidValue;
 }
 
+cudaError_t attention_delta(const bf16* o, const bf16* d_o, float* delta, int B, int S, int nh, int d, cudaStream_t st) {
+  const long long warps = (long long)B * S * nh;
+  const int blocks = (int)((warps * 32 + 255) / 256);
+  if (d == 64) attn_delta_kernel<64><<<blocks, 256, 0, st>>>(o, d_o, delta, B, S, nh);
+  else if (d == 128) attn_delta_kernel<128><<<blocks, 256, 0, st>>>(o, d_o, delta, B, S, nh);
+  else return cudaErrorInvalidValue;
+  return cudaGetLastError();
+}
+
 }  // namespace fs
 
 // =============================================================================== entry point that allocates nothing
@@ -658,10 +667,21 @@ extern "C" ft_status ft_k_attention_bwd_noalloc(const void* dev_qkv, const void*
   if (static_delta_ptr(&delta) != cudaSuccess) return FT_ECUDA;
   // every element of delta that the two main kernels read is written by the pre-pass of this same call,
   // so nothing has to start at zero
-  cudaError_t e = fs::attention_bwd(reinterpret_cast<const fs::bf16*>(dev_qkv), reinterpret_cast<const fs::bf16*>(dev_o),
-                                    reinterpret_cast<const fs::bf16*>(dev_do), dev_lse, delta,
-                                    reinterpret_cast<fs::bf16*>(dev_dqkv), dev_cos, dev_sin, B, S, n_heads, n_kv_heads,
-                                    head_dim, reinterpret_cast<cudaStream_t>(stream));
+  // same kernels as ft_k_attention_bwd, so the same bits
+  cudaError_t e;
+  if (fs::g_attention_impl) {
+    int* status = fs::attention_status_word();
+    if (!status) return FT_ECUDA;
+    e = fs::attention_bwd_tc(reinterpret_cast<const fs::bf16*>(dev_qkv), reinterpret_cast<const fs::bf16*>(dev_o),
+                             reinterpret_cast<const fs::bf16*>(dev_do), dev_lse, delta,
+                             reinterpret_cast<fs::bf16*>(dev_dqkv), dev_cos, dev_sin, B, S, n_heads, n_kv_heads, head_dim,
+                             status, reinterpret_cast<cudaStream_t>(stream));
+  } else {
+    e = fs::attention_bwd(reinterpret_cast<const fs::bf16*>(dev_qkv), reinterpret_cast<const fs::bf16*>(dev_o),
+                          reinterpret_cast<const fs::bf16*>(dev_do), dev_lse, delta,
+                          reinterpret_cast<fs::bf16*>(dev_dqkv), dev_cos, dev_sin, B, S, n_heads, n_kv_heads, head_dim,
+                          reinterpret_cast<cudaStream_t>(stream));
+  }
   if (e == cudaErrorInvalidValue) return FT_EINVAL;
   return e == cudaSuccess ? FT_OK : FT_ECUDA;
 }

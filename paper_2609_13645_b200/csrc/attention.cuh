@@ -21,6 +21,12 @@ cudaError_t attention_bwd(const bf16* qkv, const bf16* o, const bf16* d_o, const
 cudaError_t attention_fwd_tc(const bf16* qkv, bf16* o, float* lse, int B, int S, int n_heads, int n_kv, int d, int* err,
                              cudaStream_t st);
 
+cudaError_t attention_bwd_tc(const bf16* qkv, const bf16* o, const bf16* d_o, const float* lse, float* delta, bf16* dqkv,
+                             const float* cos, const float* sin, int B, int S, int n_heads, int n_kv, int d, int* err,
+                             cudaStream_t st);
+// delta[b, n, i] = sum_k dO[b,i,n,k] O[b,i,n,k] (the backward pre-pass; one launch)
+cudaError_t attention_delta(const bf16* o, const bf16* d_o, float* delta, int B, int S, int n_heads, int d, cudaStream_t st);
+
 // Device status word used by the single-kernel entry points (address on the current device).
 int* attention_status_word();
 // 1: tcgen05 kernels where they exist (default); 0: warp-level mma.sync kernels.

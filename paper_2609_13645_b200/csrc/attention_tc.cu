@@ -298,6 +298,431 @@ cudaError_t attention_fwd_tc_t(const bf16* qkv, bf16* o, float* lse, int B, int 
   return cudaGetLastError();
 }
 
+// ============================================================================ backward
+// One kernel template for both halves of the deterministic backward.  A CTA keeps a "resident" pair of [128 x D]
+// tiles (X1, X2) and streams pairs of [64 x D] tiles (Y1, Y2):
+//   MODE_DQ : X = (Q, dO) of 128 queries, Y = (K, V) blocks          -> dQ  += dS  K
+//   MODE_DKV: X = (K, V) of 128 keys,     Y = (Q, dO) blocks, all the query heads of the GQA group in a fixed order
+//                                                                     -> dV += P^T dO,  dK += dS^T Q
+// Per streamed block:  S = X1 Y1^T and dP = X2 Y2^T (two tcgen05 GEMMs into one of two TMEM buffers); the compute
+// warps (one X row per thread) turn them into P = exp2(S c - LSE) and dS = P (dP - delta), write them as bf16
+// A-operand tiles to shared memory, and the accumulating GEMMs read the SAME streamed tiles again as mn-major B
+// operands.  warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..9 = compute (two warps per TMEM lane quarter, each
+// taking half of the 64 streamed columns).
+enum { MODE_DQ = 0, MODE_DKV = 1 };
+// barrier slots: Y ring (up to 4 stages) first, then the double-buffered TMEM / operand-tile handshakes
+enum { BB_XFULL = 0, BB_YFULL = 1, BB_YEMPTY = 5, BB_SDPFULL = 9, BB_SDPEMPTY = 11, BB_TFULL = 13, BB_TEMPTY = 15,
+       BB_ACCDONE = 17, BB_COUNT = 18 };
+constexpr int BWD_THREADS = 320;
+
+template <int D, int MODE>
+struct BwdCfg {
+  static constexpr int KC = D / 64;
+  static constexpr int X_BYTES = 128 * D * 2;
+  static constexpr int Y_BYTES = 64 * D * 2;
+  static constexpr int T_BYTES = 128 * 64 * 2;
+  static constexpr int NT = MODE == MODE_DKV ? 2 : 1;
+  static constexpr int NST = MODE == MODE_DKV ? 3 : 4;  // stages of the streamed-tile ring
+  static constexpr int OFF_X1 = 0, OFF_X2 = X_BYTES, OFF_Y = 2 * X_BYTES;
+  static constexpr int OFF_T = OFF_Y + NST * 2 * Y_BYTES;
+  static constexpr int OFF_STAT = OFF_T + 2 * NT * T_BYTES;
+  static constexpr int OFF_BAR = OFF_STAT + 2048;
+  static constexpr int SMEM_BYTES = OFF_BAR + 256;
+  static constexpr int TMEM_COLS = 512;  // buffer b: S at b*128, dP at b*128+64; accumulators from column 256
+  static constexpr int ACC0 = 256, ACC1 = 256 + D;
+};
+
+template <int W>
+__device__ __forceinline__ void tmem_load_cols(uint32_t taddr, float (&out)[W]) {
+  static_assert(W == 32 || W == 16, "chunk width");
+  if constexpr (W == 32) {
+    uint32_t t[32];
+    tmem_ld32(taddr, t);
+    tmem_ld_wait();
+#pragma unroll
+    for (int i = 0; i < 32; ++i) out[i] = __uint_as_float(t[i]);
+  } else {
+    uint32_t t[16];
+    tmem_ld16(taddr, t);
+    tmem_ld_wait();
+#pragma unroll
+    for (int i = 0; i < 16; ++i) out[i] = __uint_as_float(t[i]);
+  }
+}
+
+template <int W>
+__device__ __forceinline__ void store_bf16_row(bf16* dst, const float (&v)[W]) {
+#pragma unroll
+  for (int i = 0; i < W; i += 8) {
+    uint4 o;
+    o.x = pack_bf16(v[i], v[i + 1]);
+    o.y = pack_bf16(v[i + 2], v[i + 3]);
+    o.z = pack_bf16(v[i + 4], v[i + 5]);
+    o.w = pack_bf16(v[i + 6], v[i + 7]);
+    *reinterpret_cast<uint4*>(dst + i) = o;
+  }
+}
+
+template <int D, int MODE>
+__global__ void __launch_bounds__(BWD_THREADS, 1)
+attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_constant__ CUtensorMap tm_qkv64,
+                   const __grid_constant__ CUtensorMap tm_do128, const __grid_constant__ CUtensorMap tm_do64,
+                   const float* __restrict__ lse, const float* __restrict__ delta, bf16* __restrict__ dqkv,
+                   const float* __restrict__ rope_cos, const float* __restrict__ rope_sin, int S, int n_heads, int n_kv,
+                   float scale, float scale_log2, int* err) {
+  using C = BwdCfg<D, MODE>;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const uint32_t sbase = smem_u32(smem);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::OFF_BAR);
+  const uint32_t bar0 = sbase + C::OFF_BAR;
+  auto bar = [&](int i) { return bar0 + 8u * i; };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + BB_COUNT);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* s_stat = reinterpret_cast<float*>(smem + C::OFF_STAT);  // [stage][0: lse*log2e, 1: delta][64]
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if ((sbase & 1023u) != 0u) {
+    if (threadIdx.x == 0) atomicExch(err, (int)ERR_BAD_ALIGNMENT);
+    return;
+  }
+  const int n_rep = n_heads / n_kv;
+  const int hq = n_heads * D, hkv = n_kv * D;
+  const long long ld = hq + 2 * hkv;
+  const int b = blockIdx.z;
+  int x0, kvh, n_q = 0, iters, qb0 = 0, per_head = 1;
+  if constexpr (MODE == MODE_DQ) {
+    x0 = (gridDim.x - 1 - blockIdx.x) * 128;  // heaviest query blocks first
+    n_q = blockIdx.y;
+    kvh = n_q / n_rep;
+    iters = (min(S, x0 + 128) + 63) / 64;
+  } else {
+    x0 = blockIdx.x * 128;  // the first key blocks see the most queries
+    kvh = blockIdx.y;
+    qb0 = x0 / 64;
+    per_head = (S + 63) / 64 - qb0;
+    iters = per_head * n_rep;
+  }
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar(BB_XFULL), 1);
+    for (int i = 0; i < C::NST; ++i) {
+      mbar_init(bar(BB_YFULL + i), MODE == MODE_DKV ? 2 : 1);
+      mbar_init(bar(BB_YEMPTY + i), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar(BB_SDPFULL + i), 1);
+      mbar_init(bar(BB_SDPEMPTY + i), 8);
+      mbar_init(bar(BB_TFULL + i), 8);
+      mbar_init(bar(BB_TEMPTY + i), 1);
+    }
+    mbar_init(bar(BB_ACCDONE), 1);
+    *abort_flag = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tm_qkv128);
+    tma_prefetch_desc(&tm_qkv64);
+    tma_prefetch_desc(&tm_do128);
+    tma_prefetch_desc(&tm_do64);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_slot), C::TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      mbar_expect_tx(bar(BB_XFULL), 2 * C::X_BYTES);
+#pragma unroll
+      for (int kc = 0; kc < C::KC; ++kc) {
+        if constexpr (MODE == MODE_DQ) {
+          tma_load_3d(sbase + C::OFF_X1 + kc * 16384, &tm_qkv128, bar(BB_XFULL), n_q * D + kc * 64, x0, b);
+          tma_load_3d(sbase + C::OFF_X2 + kc * 16384, &tm_do128, bar(BB_XFULL), n_q * D + kc * 64, x0, b);
+        } else {
+          tma_load_3d(sbase + C::OFF_X1 + kc * 16384, &tm_qkv128, bar(BB_XFULL), hq + kvh * D + kc * 64, x0, b);
+          tma_load_3d(sbase + C::OFF_X2 + kc * 16384, &tm_qkv128, bar(BB_XFULL), hq + hkv + kvh * D + kc * 64, x0, b);
+        }
+      }
+    }
+    for (int it = 0; it < iters; ++it) {
+      const int st = it % C::NST;
+      bool ok = mbar_wait(bar(BB_YEMPTY + st), (((uint32_t)(it / C::NST)) & 1u) ^ 1u, abort_flag, err);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      const uint32_t ydst = sbase + C::OFF_Y + st * 2 * C::Y_BYTES;
+      if constexpr (MODE == MODE_DQ) {
+        if (lane == 0) {
+          mbar_expect_tx(bar(BB_YFULL + st), 2 * C::Y_BYTES);
+#pragma unroll
+          for (int kc = 0; kc < C::KC; ++kc) {
+            tma_load_3d(ydst + kc * 8192, &tm_qkv64, bar(BB_YFULL + st), hq + kvh * D + kc * 64, it * 64, b);
+            tma_load_3d(ydst + C::Y_BYTES + kc * 8192, &tm_qkv64, bar(BB_YFULL + st), hq + hkv + kvh * D + kc * 64,
+                        it * 64, b);
+          }
+        }
+      } else {
+        const int rep = it / per_head, qb = qb0 + it % per_head;
+        const int n = kvh * n_rep + rep;
+        if (lane == 0) {
+          mbar_expect_tx(bar(BB_YFULL + st), 2 * C::Y_BYTES);
+#pragma unroll
+          for (int kc = 0; kc < C::KC; ++kc) {
+            tma_load_3d(ydst + kc * 8192, &tm_qkv64, bar(BB_YFULL + st), n * D + kc * 64, qb * 64, b);
+            tma_load_3d(ydst + C::Y_BYTES + kc * 8192, &tm_do64, bar(BB_YFULL + st), n * D + kc * 64, qb * 64, b);
+          }
+        }
+        const long long stat = ((long long)b * n_heads + n) * S;
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int qq = qb * 64 + lane * 2 + e;
+          s_stat[st * 128 + lane * 2 + e] = qq < S ? lse[stat + qq] * 1.4426950408889634f : 0.f;
+          s_stat[st * 128 + 64 + lane * 2 + e] = qq < S ? delta[stat + qq] : 0.f;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(BB_YFULL + st));
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc_base = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 4) << 24);
+      const uint32_t idesc_sdp = idesc_base | ((uint32_t)(64 >> 3) << 17);            // N = 64, both K-major
+      const uint32_t idesc_acc = idesc_base | (1u << 16) | ((uint32_t)(D >> 3) << 17);  // N = D, B mn-major
+      auto issue_sdp = [&](int it) {
+        const int st = it % C::NST;
+        const uint32_t y1 = sbase + C::OFF_Y + st * 2 * C::Y_BYTES, y2 = y1 + C::Y_BYTES;
+        const uint32_t d_s = tmem_base + (uint32_t)((it & 1) * 128), d_p = d_s + 64;
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) {
+          const uint32_t xo = (k >> 2) * 16384 + (k & 3) * 32, yo = (k >> 2) * 8192 + (k & 3) * 32;
+          umma_bf16(d_s, umma_desc_sw128(sbase + C::OFF_X1 + xo, 0, 1024), umma_desc_sw128(y1 + yo, 0, 1024), idesc_sdp,
+                    k > 0 ? 1u : 0u);
+        }
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) {
+          const uint32_t xo = (k >> 2) * 16384 + (k & 3) * 32, yo = (k >> 2) * 8192 + (k & 3) * 32;
+          umma_bf16(d_p, umma_desc_sw128(sbase + C::OFF_X2 + xo, 0, 1024), umma_desc_sw128(y2 + yo, 0, 1024), idesc_sdp,
+                    k > 0 ? 1u : 0u);
+        }
+        umma_commit(bar(BB_SDPFULL + (it & 1)));
+      };
+      bool ok = mbar_wait(bar(BB_XFULL), 0, abort_flag, err) && mbar_wait(bar(BB_YFULL), 0, abort_flag, err);
+      if (ok) {
+        tc_fence_after();
+        issue_sdp(0);
+      }
+      for (int it = 0; it < iters && ok; ++it) {
+        if (it + 1 < iters) {
+          const int s1 = (it + 1) & 1, y1s = (it + 1) % C::NST;
+          if (!mbar_wait(bar(BB_YFULL + y1s), ((uint32_t)((it + 1) / C::NST)) & 1u, abort_flag, err)) { ok = false; break; }
+          if (!mbar_wait(bar(BB_SDPEMPTY + s1), (((uint32_t)(it + 1) >> 1) & 1u) ^ 1u, abort_flag, err)) { ok = false; break; }
+          tc_fence_after();
+          issue_sdp(it + 1);
+        }
+        const int bf = it & 1;
+        if (!mbar_wait(bar(BB_TFULL + bf), ((uint32_t)it >> 1) & 1u, abort_flag, err)) { ok = false; break; }
+        tc_fence_after();
+        const int yst = it % C::NST;
+        const uint32_t y1 = sbase + C::OFF_Y + yst * 2 * C::Y_BYTES, y2 = y1 + C::Y_BYTES;
+        const uint32_t t0 = sbase + C::OFF_T + bf * C::NT * C::T_BYTES, t1 = t0 + C::T_BYTES;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const uint32_t acc = (it > 0 || k > 0) ? 1u : 0u;
+          if constexpr (MODE == MODE_DQ) {
+            umma_bf16(tmem_base + C::ACC0, umma_desc_sw128(t0 + k * 32, 0, 1024),
+                      umma_desc_sw128(y1 + k * 2048, 8192, 1024), idesc_acc, acc);  // dQ += dS K
+          } else {
+            umma_bf16(tmem_base + C::ACC0, umma_desc_sw128(t0 + k * 32, 0, 1024),
+                      umma_desc_sw128(y2 + k * 2048, 8192, 1024), idesc_acc, acc);  // dV += P^T dO
+            umma_bf16(tmem_base + C::ACC1, umma_desc_sw128(t1 + k * 32, 0, 1024),
+                      umma_desc_sw128(y1 + k * 2048, 8192, 1024), idesc_acc, acc);  // dK += dS^T Q
+          }
+        }
+        umma_commit(bar(BB_YEMPTY + yst));
+        umma_commit(bar(BB_TEMPTY + bf));
+      }
+      if (ok) umma_commit(bar(BB_ACCDONE));
+    }
+  } else {
+    // ------------------------------------------------------------------ compute warps
+    const int q = warp & 3, ch = (warp - 2) >> 2;
+    const int rloc = q * 32 + lane;
+    const int row = x0 + rloc;  // query (MODE_DQ) or key (MODE_DKV) position
+    const uint32_t tlane = tmem_base + ((uint32_t)(q * 32) << 16);
+    float lse2_row = 0.f, delta_row = 0.f;
+    if constexpr (MODE == MODE_DQ) {
+      if (row < S) {
+        const long long stat = ((long long)b * n_heads + n_q) * S;
+        lse2_row = lse[stat + row] * 1.4426950408889634f;
+        delta_row = delta[stat + row];
+      }
+    }
+    bool ok = true;
+    for (int it = 0; it < iters; ++it) {
+      const int bf = it & 1;
+      ok = mbar_wait(bar(BB_SDPFULL + bf), ((uint32_t)it >> 1) & 1u, abort_flag, err);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      uint32_t rs[32], rp[32];
+      tmem_ld32(tlane + (uint32_t)(bf * 128 + ch * 32), rs);
+      tmem_ld32(tlane + (uint32_t)(bf * 128 + 64 + ch * 32), rp);
+      tmem_ld_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(BB_SDPEMPTY + bf));
+
+      int y0;
+      const int yst = it % C::NST;
+      const float* st_lse = s_stat + yst * 128 + ch * 32;
+      const float* st_dl = st_lse + 64;
+      if constexpr (MODE == MODE_DQ) {
+        y0 = it * 64;
+      } else {
+        y0 = (qb0 + it % per_head) * 64;
+        ok = mbar_wait(bar(BB_YFULL + yst), ((uint32_t)(it / C::NST)) & 1u, abort_flag, err);  // acquire the staged statistics
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+      }
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        const int col = y0 + ch * 32 + i;
+        float p, ds;
+        if constexpr (MODE == MODE_DQ) {
+          p = col <= row ? exp2f(__uint_as_float(rs[i]) * scale_log2 - lse2_row) : 0.f;
+          ds = p * (__uint_as_float(rp[i]) - delta_row);
+        } else {
+          p = (col >= row && col < S) ? exp2f(__uint_as_float(rs[i]) * scale_log2 - st_lse[i]) : 0.f;
+          ds = p * (__uint_as_float(rp[i]) - st_dl[i]);
+        }
+        rs[i] = __float_as_uint(p);
+        rp[i] = __float_as_uint(ds);
+      }
+      ok = mbar_wait(bar(BB_TEMPTY + bf), (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag, err);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      uint8_t* t0row = smem + C::OFF_T + bf * C::NT * C::T_BYTES + rloc * 128;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const int chunk = ((ch * 4 + c) ^ (rloc & 7)) << 4;
+        uint4 vp, vd;
+        vp.x = pack_bf16(__uint_as_float(rs[c * 8 + 0]), __uint_as_float(rs[c * 8 + 1]));
+        vp.y = pack_bf16(__uint_as_float(rs[c * 8 + 2]), __uint_as_float(rs[c * 8 + 3]));
+        vp.z = pack_bf16(__uint_as_float(rs[c * 8 + 4]), __uint_as_float(rs[c * 8 + 5]));
+        vp.w = pack_bf16(__uint_as_float(rs[c * 8 + 6]), __uint_as_float(rs[c * 8 + 7]));
+        vd.x = pack_bf16(__uint_as_float(rp[c * 8 + 0]), __uint_as_float(rp[c * 8 + 1]));
+        vd.y = pack_bf16(__uint_as_float(rp[c * 8 + 2]), __uint_as_float(rp[c * 8 + 3]));
+        vd.z = pack_bf16(__uint_as_float(rp[c * 8 + 4]), __uint_as_float(rp[c * 8 + 5]));
+        vd.w = pack_bf16(__uint_as_float(rp[c * 8 + 6]), __uint_as_float(rp[c * 8 + 7]));
+        if constexpr (MODE == MODE_DQ) {
+          *reinterpret_cast<uint4*>(t0row + chunk) = vd;
+        } else {
+          *reinterpret_cast<uint4*>(t0row + chunk) = vp;
+          *reinterpret_cast<uint4*>(t0row + C::T_BYTES + chunk) = vd;
+        }
+      }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(BB_TFULL + bf));
+    }
+    if (ok) {
+      ok = mbar_wait(bar(BB_ACCDONE), 0, abort_flag, err);
+      ok = __all_sync(0xffffffffu, ok);
+    }
+    if (ok) {
+      tc_fence_after();
+      // rotated output (dQ or dK): this warp owns columns [i0, i0+W) and their partners D/2 further
+      constexpr int W = D / 4, H = D / 2;
+      const int i0 = ch * W;
+      const uint32_t racc = tlane + (uint32_t)(MODE == MODE_DQ ? C::ACC0 : C::ACC1);
+      float lo[W], hi[W];
+      tmem_load_cols<W>(racc + (uint32_t)i0, lo);
+      tmem_load_cols<W>(racc + (uint32_t)(H + i0), hi);
+#pragma unroll
+      for (int i = 0; i < W; ++i) { lo[i] *= scale; hi[i] *= scale; }
+      if (rope_cos != nullptr) {
+        const int pos = min(row, S - 1);
+        const float* cs = rope_cos + (long long)pos * H + i0;
+        const float* sn = rope_sin + (long long)pos * H + i0;
+#pragma unroll
+        for (int i = 0; i < W; i += 4) {
+          const float4 c4 = *reinterpret_cast<const float4*>(cs + i);
+          const float4 s4 = *reinterpret_cast<const float4*>(sn + i);
+          const float cc[4] = {c4.x, c4.y, c4.z, c4.w}, ss[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const float y1 = lo[i + u], y2 = hi[i + u];
+            lo[i + u] = y1 * cc[u] + y2 * ss[u];
+            hi[i + u] = y2 * cc[u] - y1 * ss[u];
+          }
+        }
+      }
+      const int colbase = MODE == MODE_DQ ? n_q * D : hq + kvh * D;
+      if (row < S) {
+        bf16* dst = dqkv + ((long long)b * S + row) * ld + colbase;
+        store_bf16_row<W>(dst + i0, lo);
+        store_bf16_row<W>(dst + H + i0, hi);
+      }
+      if constexpr (MODE == MODE_DKV) {
+        bf16* dstv = dqkv + ((long long)b * S + row) * ld + hq + hkv + kvh * D;
+#pragma unroll 1
+        for (int c = ch * H; c < (ch + 1) * H; c += 32) {
+          float v[32];
+          tmem_load_cols<32>(tlane + (uint32_t)(C::ACC0 + c), v);
+          if (row < S) store_bf16_row<32>(dstv + c, v);
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag != 0) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000LL) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, C::TMEM_COLS);
+  }
+}
+
+template <int D>
+cudaError_t attention_bwd_tc_t(const bf16* qkv, const bf16* o, const bf16* d_o, const float* lse, float* delta, bf16* dqkv,
+                               const float* cs, const float* sn, int B, int S, int nh, int nkv, int* err, cudaStream_t st) {
+  using CQ = BwdCfg<D, MODE_DQ>;
+  using CK = BwdCfg<D, MODE_DKV>;
+  static bool once = false;
+  if (!once) {
+    cudaError_t e = cudaFuncSetAttribute(attn_bwd_tc_kernel<D, MODE_DQ>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         CQ::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_bwd_tc_kernel<D, MODE_DKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, CK::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    once = true;
+  }
+  const int hq = nh * D, nqkv = (nh + 2 * nkv) * D;
+  CUtensorMap tq128, tq64, td128, td64;
+  if (!make_tmap_3d(&tq128, qkv, nqkv, S, B, nqkv, 128) || !make_tmap_3d(&tq64, qkv, nqkv, S, B, nqkv, 64) ||
+      !make_tmap_3d(&td128, d_o, hq, S, B, hq, 128) || !make_tmap_3d(&td64, d_o, hq, S, B, hq, 64))
+    return cudaErrorInvalidValue;
+  const float scale = (float)(1.0 / sqrt((double)D));
+  const float scale_log2 = (float)((1.0 / sqrt((double)D)) * 1.4426950408889634);
+  cudaError_t e = attention_delta(o, d_o, delta, B, S, nh, D, st);
+  if (e != cudaSuccess) return e;
+  dim3 gq((S + 127) / 128, nh, B), gk((S + 127) / 128, nkv, B);
+  attn_bwd_tc_kernel<D, MODE_DQ><<<gq, BWD_THREADS, CQ::SMEM_BYTES, st>>>(tq128, tq64, td128, td64, lse, delta, dqkv, cs, sn,
+                                                                            S, nh, nkv, scale, scale_log2, err);
+  attn_bwd_tc_kernel<D, MODE_DKV><<<gk, BWD_THREADS, CK::SMEM_BYTES, st>>>(tq128, tq64, td128, td64, lse, delta, dqkv, cs,
+                                                                             sn, S, nh, nkv, scale, scale_log2, err);
+  return cudaGetLastError();
+}
+
 static __device__ int g_attn_status;
 
 }  // namespace
@@ -321,6 +746,16 @@ cudaError_t attention_fwd_tc(const bf16* qkv, bf16* o, float* lse, int B, int S,
   if (B <= 0 || S <= 0 || nh <= 0 || nkv <= 0 || nh % nkv || !err) return cudaErrorInvalidValue;
   if (d == 64) return attention_fwd_tc_t<64>(qkv, o, lse, B, S, nh, nkv, err, st);
   if (d == 128) return attention_fwd_tc_t<128>(qkv, o, lse, B, S, nh, nkv, err, st);
+  return cudaErrorInvalidValue;
+}
+
+cudaError_t attention_bwd_tc(const bf16* qkv, const bf16* o, const bf16* d_o, const float* lse, float* delta, bf16* dqkv,
+                             const float* cs, const float* sn, int B, int S, int nh, int nkv, int d, int* err,
+                             cudaStream_t st) {
+  if (B <= 0 || S <= 0 || nh <= 0 || nkv <= 0 || nh % nkv || !err) return cudaErrorInvalidValue;
+  if ((cs == nullptr) != (sn == nullptr)) return cudaErrorInvalidValue;
+  if (d == 64) return attention_bwd_tc_t<64>(qkv, o, d_o, lse, delta, dqkv, cs, sn, B, S, nh, nkv, err, st);
+  if (d == 128) return attention_bwd_tc_t<128>(qkv, o, d_o, lse, delta, dqkv, cs, sn, B, S, nh, nkv, err, st);
   return cudaErrorInvalidValue;
 }
 

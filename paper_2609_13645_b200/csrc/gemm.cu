@@ -366,6 +366,8 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
 
 }  // namespace
 
+int g_gemm_force_bn = 0;  // development knob: 0 = choose by tile count, 128 or 256 = force that tile width
+
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream) {
   if (a.M <= 0 || a.N <= 0 || a.K <= 0 || !a.A || !a.B || !a.C || !a.err) return cudaErrorInvalidValue;
   if ((a.N & 7) || (a.lda & 7) || (a.ldb & 7) || (a.ldc & 3)) return cudaErrorInvalidValue;
@@ -379,7 +381,7 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream) {
     return cudaErrorInvalidValue;
   if (a.epi == EPI_SWIGLU && (!a.gu || a.d_ffn <= 0 || a.d_ffn % 16 || a.N != 2 * a.d_ffn)) return cudaErrorInvalidValue;
   const int tiles256 = ((a.M + BM - 1) / BM) * ((a.N + 255) / 256);
-  const bool wide = tiles256 >= sm_count();
+  const bool wide = g_gemm_force_bn ? g_gemm_force_bn == 256 : tiles256 >= sm_count();
   if (!a.a_mn && !a.b_mn) return wide ? launch_variant<256, false, false>(a, stream) : launch_variant<128, false, false>(a, stream);
   if (!a.a_mn && a.b_mn) return wide ? launch_variant<256, false, true>(a, stream) : launch_variant<128, false, true>(a, stream);
   if (a.a_mn && a.b_mn) return wide ? launch_variant<256, true, true>(a, stream) : launch_variant<128, true, true>(a, stream);

@@ -41,4 +41,6 @@ struct GemmArgs {
 // Enqueues the contraction on `stream`.  Returns cudaErrorInvalidValue for shapes it does not take.
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream);
 
+extern int g_gemm_force_bn;
+
 }  // namespace fs

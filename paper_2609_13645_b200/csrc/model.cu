@@ -358,8 +358,12 @@ ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
   s = linear_backward(m, m->dxB, a.o, m->idx_layer(l, 2), m->d_o, T, h, hq);
   if (s) return s;
   prof_begin(m);
-  FT_CUDA(attention_bwd(a.qkv, a.o, m->d_o, a.lse, m->delta, m->d_qkv, m->rope_cos, m->rope_sin, B, S, m->cfg.n_heads,
-                        m->cfg.n_kv_heads, m->d, st));
+  if (g_attention_impl)
+    FT_CUDA(attention_bwd_tc(a.qkv, a.o, m->d_o, a.lse, m->delta, m->d_qkv, m->rope_cos, m->rope_sin, B, S,
+                             m->cfg.n_heads, m->cfg.n_kv_heads, m->d, &m->sc->err, st));
+  else
+    FT_CUDA(attention_bwd(a.qkv, a.o, m->d_o, a.lse, m->delta, m->d_qkv, m->rope_cos, m->rope_sin, B, S, m->cfg.n_heads,
+                          m->cfg.n_kv_heads, m->d, st));
   m->launches += 3;
   prof_end(m, FT_PROF_ATTN_BWD, 4.0 * B * m->cfg.n_heads * (double)S * S * m->d, 3);
   s = linear_backward(m, m->d_qkv, a.h1, m->idx_layer(l, 1), m->d_h, T, nqkv, h);
@@ -765,6 +769,7 @@ ft_status ft_get_profile(ft_model* m, int32_t cls, double* ms, double* work, int
 }
 
 void ft_debug_attention_impl(int32_t impl) { g_attention_impl = impl; }
+void ft_debug_gemm_tile(int32_t bn) { g_gemm_force_bn = bn; }
 
 const char* ft_last_error(const ft_model* m) { return m ? m->err.c_str() : "null model"; }
 int64_t ft_launch_count(const ft_model* m) { return m ? m->launches : 0; }
@@ -811,10 +816,19 @@ ft_status ft_k_attention_bwd(const void* dev_qkv, const void* dev_o, const void*
                              float* dev_delta, void* dev_dqkv, const float* dev_cos, const float* dev_sin, int32_t B,
                              int32_t S, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, void* stream) {
   if (!dev_qkv || !dev_o || !dev_do || !dev_lse || !dev_delta || !dev_dqkv) return FT_EINVAL;
-  cudaError_t e = attention_bwd(reinterpret_cast<const bf16*>(dev_qkv), reinterpret_cast<const bf16*>(dev_o),
-                                reinterpret_cast<const bf16*>(dev_do), dev_lse, dev_delta,
-                                reinterpret_cast<bf16*>(dev_dqkv), dev_cos, dev_sin, B, S, n_heads, n_kv_heads, head_dim,
-                                reinterpret_cast<cudaStream_t>(stream));
+  cudaError_t e;
+  if (g_attention_impl) {
+    int* status = attention_status_word();
+    if (!status) return FT_ECUDA;
+    e = attention_bwd_tc(reinterpret_cast<const bf16*>(dev_qkv), reinterpret_cast<const bf16*>(dev_o),
+                         reinterpret_cast<const bf16*>(dev_do), dev_lse, dev_delta, reinterpret_cast<bf16*>(dev_dqkv),
+                         dev_cos, dev_sin, B, S, n_heads, n_kv_heads, head_dim, status,
+                         reinterpret_cast<cudaStream_t>(stream));
+  } else {
+    e = attention_bwd(reinterpret_cast<const bf16*>(dev_qkv), reinterpret_cast<const bf16*>(dev_o),
+                      reinterpret_cast<const bf16*>(dev_do), dev_lse, dev_delta, reinterpret_cast<bf16*>(dev_dqkv),
+                      dev_cos, dev_sin, B, S, n_heads, n_kv_heads, head_dim, reinterpret_cast<cudaStream_t>(stream));
+  }
   if (e == cudaErrorInvalidValue) return FT_EINVAL;
   return e == cudaSuccess ? FT_OK : FT_ECUDA;
 }

@@ -35,8 +35,11 @@ def main():
     ap.add_argument("--iters", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--no-flush", action="store_true")
+    ap.add_argument("--bn", type=int, default=0, help="force the GEMM tile width (development)")
     a = ap.parse_args()
     torch.manual_seed(0)
+    if a.bn:
+        B.lib().ft_debug_gemm_tile(a.bn)
     dev = "cuda"
     flush = None if a.no_flush else torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     err = torch.zeros(1, dtype=torch.int32, device=dev)
