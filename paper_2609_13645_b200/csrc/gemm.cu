@@ -380,8 +380,9 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream) {
                             a.rope_cols % a.head_dim || a.N % a.head_dim))
     return cudaErrorInvalidValue;
   if (a.epi == EPI_SWIGLU && (!a.gu || a.d_ffn <= 0 || a.d_ffn % 16 || a.N != 2 * a.d_ffn)) return cudaErrorInvalidValue;
-  const int tiles256 = ((a.M + BM - 1) / BM) * ((a.N + 255) / 256);
-  const bool wide = g_gemm_force_bn ? g_gemm_force_bn == 256 : tiles256 >= sm_count();
+  // 128 x 256 tiles move 96 B of operands per tensor-core cycle through shared memory, 128 x 128 tiles 128 B: the
+  // wide tile is faster even when it leaves SMs idle (measured), so the narrow one only serves N <= 128
+  const bool wide = g_gemm_force_bn ? g_gemm_force_bn == 256 : a.N > 128;
   if (!a.a_mn && !a.b_mn) return wide ? launch_variant<256, false, false>(a, stream) : launch_variant<128, false, false>(a, stream);
   if (!a.a_mn && a.b_mn) return wide ? launch_variant<256, false, true>(a, stream) : launch_variant<128, false, true>(a, stream);
   if (a.a_mn && a.b_mn) return wide ? launch_variant<256, true, true>(a, stream) : launch_variant<128, true, true>(a, stream);
