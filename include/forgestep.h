@@ -112,6 +112,8 @@ ft_status ft_get_profile(ft_model* m, int32_t cls, double* ms, double* work, int
 void ft_debug_attention_impl(int32_t impl);
 /* Development switch: force the GEMM tile width (128 or 256 columns); 0 = choose by tile count (default). */
 void ft_debug_gemm_tile(int32_t bn);
+/* Development switch: 1 = CTA-pair (cta_group::2, 256 x 256 tile) GEMM kernel where it applies (default), 0 = off. */
+void ft_debug_gemm_pairs(int32_t on);
 
 const char* ft_last_error(const ft_model* m);
 /* Number of kernels the library launched since the model was created (for launch accounting). */

@@ -72,6 +72,8 @@ def lib():
         L.ft_debug_attention_impl.restype = None
         L.ft_debug_gemm_tile.argtypes = [i32]
         L.ft_debug_gemm_tile.restype = None
+        L.ft_debug_gemm_pairs.argtypes = [i32]
+        L.ft_debug_gemm_pairs.restype = None
         L.ft_destroy.restype = None
         L.ft_destroy.argtypes = [vp]
         L.ft_k_gemm.argtypes = [vp, i32, i64, vp, i32, i64, vp, i64, vp, i32, i32, i32, i32, vp, vp]

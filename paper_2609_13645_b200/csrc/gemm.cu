@@ -53,6 +53,138 @@ __device__ __forceinline__ void store8_bf16(bf16* dst, const float* v) {
   *reinterpret_cast<uint4*>(dst) = o;
 }
 
+// Epilogue of one accumulator tile for one thread: `row` is the global output row held by this thread's TMEM lane,
+// taddr the TMEM address of (its lane quarter, first column of the tile), n0 the tile's first output column.
+// Every tcgen05.ld is executed by all 32 lanes (rows past M only skip the stores).
+template <int BN>
+__device__ __forceinline__ void epilogue_tile(const GemmDev& p, uint32_t taddr, int row, int n0) {
+  const bool row_ok = row < p.M;
+  uint32_t r[32];
+  if (p.epi == EPI_ROPE) {
+    const int d = p.head_dim;
+    const int half = d >> 1;
+    const int pos = row_ok ? (row % p.seq) : 0;
+    bf16* crow = reinterpret_cast<bf16*>(p.C) + (long long)row * p.ldc;
+    for (int hc = 0; hc < BN; hc += d) {
+      const int g0 = n0 + hc;
+      if (g0 >= p.N) break;
+      if (g0 >= p.rope_cols) {
+        for (int c = 0; c < d; c += 32) {
+          tmem_ld32(taddr + hc + c, r);
+          tmem_ld_wait();
+          if (row_ok) {
+            float v[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) store8_bf16(crow + g0 + c + j, v + j);
+          }
+        }
+      } else {
+        uint32_t r2[32];
+        for (int i0 = 0; i0 < half; i0 += 32) {
+          tmem_ld32(taddr + hc + i0, r);
+          tmem_ld32(taddr + hc + i0 + half, r2);
+          tmem_ld_wait();
+          if (row_ok) {
+            const float* cs = p.rope_cos + (long long)pos * half + i0;
+            const float* sn = p.rope_sin + (long long)pos * half + i0;
+            float lo[32], hi[32];
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+              const float4 c4 = *reinterpret_cast<const float4*>(cs + j);
+              const float4 s4 = *reinterpret_cast<const float4*>(sn + j);
+              const float cc[4] = {c4.x, c4.y, c4.z, c4.w};
+              const float ss[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+              for (int u = 0; u < 4; ++u) {
+                const float x1 = __uint_as_float(r[j + u]);
+                const float x2 = __uint_as_float(r2[j + u]);
+                lo[j + u] = x1 * cc[u] - x2 * ss[u];
+                hi[j + u] = x2 * cc[u] + x1 * ss[u];
+              }
+            }
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+              store8_bf16(crow + g0 + i0 + j, lo + j);
+              store8_bf16(crow + g0 + i0 + half + j, hi + j);
+            }
+          }
+        }
+      }
+    }
+  } else if (p.epi == EPI_SWIGLU) {
+    // physical columns alternate 16 gate / 16 up of the same 16 logical ffn columns
+    const int f = p.d_ffn;
+    bf16* arow = reinterpret_cast<bf16*>(p.C) + (long long)row * p.ldc;
+    bf16* gurow = p.gu + (long long)row * (2LL * f);
+    for (int c = 0; c < BN; c += 32) {
+      const int gc = n0 + c;
+      if (gc >= p.N) break;
+      tmem_ld32(taddr + c, r);
+      tmem_ld_wait();
+      if (row_ok) {
+        const int lc = gc >> 1;  // logical ffn column of this 16-wide group
+        float g[16], u[16], a[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          g[j] = round_bf16(__uint_as_float(r[j]));
+          u[j] = round_bf16(__uint_as_float(r[16 + j]));
+          a[j] = g[j] / (1.0f + __expf(-g[j])) * u[j];
+        }
+        store8_bf16(gurow + lc, g);
+        store8_bf16(gurow + lc + 8, g + 8);
+        store8_bf16(gurow + f + lc, u);
+        store8_bf16(gurow + f + lc + 8, u + 8);
+        store8_bf16(arow + lc, a);
+        store8_bf16(arow + lc + 8, a + 8);
+      }
+    }
+  } else {
+    for (int c = 0; c < BN; c += 32) {
+      const int gc = n0 + c;
+      if (gc >= p.N) break;
+      tmem_ld32(taddr + c, r);
+      tmem_ld_wait();
+      if (row_ok) {
+        float v[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+        if (p.epi == EPI_BF16 || p.epi == EPI_BF16_RESID) {
+          bf16* crow = reinterpret_cast<bf16*>(p.C) + (long long)row * p.ldc + gc;
+          const bf16* rrow = p.resid + (long long)row * p.ldc + gc;
+#pragma unroll
+          for (int j = 0; j < 32; j += 8) {
+            if (gc + j < p.N) {
+              if (p.epi == EPI_BF16_RESID) {
+                const uint4 x = *reinterpret_cast<const uint4*>(rrow + j);
+                v[j + 0] += bf16_lo(x.x); v[j + 1] += bf16_hi(x.x);
+                v[j + 2] += bf16_lo(x.y); v[j + 3] += bf16_hi(x.y);
+                v[j + 4] += bf16_lo(x.z); v[j + 5] += bf16_hi(x.z);
+                v[j + 6] += bf16_lo(x.w); v[j + 7] += bf16_hi(x.w);
+              }
+              store8_bf16(crow + j, v + j);
+            }
+          }
+        } else {
+          float* crow = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + gc;
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            if (gc + j < p.N) {
+              float4 o = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+              if (p.epi == EPI_F32_ACC) {
+                const float4 x = *reinterpret_cast<const float4*>(crow + j);
+                o.x += x.x; o.y += x.y; o.z += x.z; o.w += x.w;
+              }
+              *reinterpret_cast<float4*>(crow + j) = o;
+            }
+          }
+        }
+      }
+    }
+  }
+}
+
 template <int BN, bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmDev p) {
@@ -178,132 +310,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (!ok) break;
       tc_fence_after();
       const int row = m0 + q * 32 + lane;
-      const bool row_ok = row < p.M;
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
-      uint32_t r[32];
-      if (p.epi == EPI_ROPE) {
-        const int d = p.head_dim;
-        const int half = d >> 1;
-        const int pos = row_ok ? (row % p.seq) : 0;
-        bf16* crow = reinterpret_cast<bf16*>(p.C) + (long long)row * p.ldc;
-        for (int hc = 0; hc < BN; hc += d) {
-          const int g0 = n0 + hc;
-          if (g0 >= p.N) break;
-          if (g0 >= p.rope_cols) {
-            for (int c = 0; c < d; c += 32) {
-              tmem_ld32(taddr + hc + c, r);
-              tmem_ld_wait();
-              if (row_ok) {
-                float v[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-#pragma unroll
-                for (int j = 0; j < 32; j += 8) store8_bf16(crow + g0 + c + j, v + j);
-              }
-            }
-          } else {
-            uint32_t r2[32];
-            for (int i0 = 0; i0 < half; i0 += 32) {
-              tmem_ld32(taddr + hc + i0, r);
-              tmem_ld32(taddr + hc + i0 + half, r2);
-              tmem_ld_wait();
-              if (row_ok) {
-                const float* cs = p.rope_cos + (long long)pos * half + i0;
-                const float* sn = p.rope_sin + (long long)pos * half + i0;
-                float lo[32], hi[32];
-#pragma unroll
-                for (int j = 0; j < 32; j += 4) {
-                  const float4 c4 = *reinterpret_cast<const float4*>(cs + j);
-                  const float4 s4 = *reinterpret_cast<const float4*>(sn + j);
-                  const float cc[4] = {c4.x, c4.y, c4.z, c4.w};
-                  const float ss[4] = {s4.x, s4.y, s4.z, s4.w};
-#pragma unroll
-                  for (int u = 0; u < 4; ++u) {
-                    const float x1 = __uint_as_float(r[j + u]);
-                    const float x2 = __uint_as_float(r2[j + u]);
-                    lo[j + u] = x1 * cc[u] - x2 * ss[u];
-                    hi[j + u] = x2 * cc[u] + x1 * ss[u];
-                  }
-                }
-#pragma unroll
-                for (int j = 0; j < 32; j += 8) {
-                  store8_bf16(crow + g0 + i0 + j, lo + j);
-                  store8_bf16(crow + g0 + i0 + half + j, hi + j);
-                }
-              }
-            }
-          }
-        }
-      } else if (p.epi == EPI_SWIGLU) {
-        // physical columns alternate 16 gate / 16 up of the same 16 logical ffn columns
-        const int f = p.d_ffn;
-        bf16* arow = reinterpret_cast<bf16*>(p.C) + (long long)row * p.ldc;
-        bf16* gurow = p.gu + (long long)row * (2LL * f);
-        for (int c = 0; c < BN; c += 32) {
-          const int gc = n0 + c;
-          if (gc >= p.N) break;
-          tmem_ld32(taddr + c, r);
-          tmem_ld_wait();
-          if (row_ok) {
-            const int lc = gc >> 1;  // logical ffn column of this 16-wide group
-            float g[16], u[16], a[16];
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              g[j] = round_bf16(__uint_as_float(r[j]));
-              u[j] = round_bf16(__uint_as_float(r[16 + j]));
-              a[j] = g[j] / (1.0f + __expf(-g[j])) * u[j];
-            }
-            store8_bf16(gurow + lc, g);
-            store8_bf16(gurow + lc + 8, g + 8);
-            store8_bf16(gurow + f + lc, u);
-            store8_bf16(gurow + f + lc + 8, u + 8);
-            store8_bf16(arow + lc, a);
-            store8_bf16(arow + lc + 8, a + 8);
-          }
-        }
-      } else {
-        for (int c = 0; c < BN; c += 32) {
-          const int gc = n0 + c;
-          if (gc >= p.N) break;
-          tmem_ld32(taddr + c, r);
-          tmem_ld_wait();
-          if (row_ok) {
-            float v[32];
-#pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-            if (p.epi == EPI_BF16 || p.epi == EPI_BF16_RESID) {
-              bf16* crow = reinterpret_cast<bf16*>(p.C) + (long long)row * p.ldc + gc;
-              const bf16* rrow = p.resid + (long long)row * p.ldc + gc;
-#pragma unroll
-              for (int j = 0; j < 32; j += 8) {
-                if (gc + j < p.N) {
-                  if (p.epi == EPI_BF16_RESID) {
-                    const uint4 x = *reinterpret_cast<const uint4*>(rrow + j);
-                    v[j + 0] += bf16_lo(x.x); v[j + 1] += bf16_hi(x.x);
-                    v[j + 2] += bf16_lo(x.y); v[j + 3] += bf16_hi(x.y);
-                    v[j + 4] += bf16_lo(x.z); v[j + 5] += bf16_hi(x.z);
-                    v[j + 6] += bf16_lo(x.w); v[j + 7] += bf16_hi(x.w);
-                  }
-                  store8_bf16(crow + j, v + j);
-                }
-              }
-            } else {
-              float* crow = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + gc;
-#pragma unroll
-              for (int j = 0; j < 32; j += 4) {
-                if (gc + j < p.N) {
-                  float4 o = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                  if (p.epi == EPI_F32_ACC) {
-                    const float4 x = *reinterpret_cast<const float4*>(crow + j);
-                    o.x += x.x; o.y += x.y; o.z += x.z; o.w += x.w;
-                  }
-                  *reinterpret_cast<float4*>(crow + j) = o;
-                }
-              }
-            }
-          }
-        }
-      }
+      epilogue_tile<BN>(p, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), row, n0);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(acc));
@@ -325,6 +332,176 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __syncwarp();
     tc_fence_after();
     tmem_dealloc(tmem_base, C::TMEM_COLS);
+  }
+}
+
+// ---------------------------------------------------------------- CTA-pair variant
+// Two CTAs on neighbouring SMs (a cluster of 2) share one 256 x 256 output tile: each loads its own 128 rows of A and
+// its own 128 of the 256 rows of B, the leader issues tcgen05.mma.cta_group::2 (M = 256), and each CTA's TMEM ends up
+// with its 128 rows x 256 columns of the accumulator.  Per flop this moves a third less operand data through L2 and
+// shared memory than the single-CTA 128 x 256 tile.  No TMA multicast is used: every CTA fetches its own operands.
+struct PairCfg {
+  static constexpr int BN = 256;                 // output columns of the pair's tile
+  static constexpr int HALF_B = 128;             // rows of B (output columns) each CTA loads
+  static constexpr int A_BYTES_ = BM * BK * 2;   // 16 KB
+  static constexpr int B_BYTES = HALF_B * BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES_ + B_BYTES;
+  static constexpr int STAGES = 6;
+  static constexpr int TMEM_COLS = 512;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 256 + 1024;
+};
+
+template <bool A_MN, bool B_MN>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmDev p) {
+  using C = PairCfg;
+  constexpr int BN = C::BN;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::STAGES * C::STAGE_BYTES);
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (C::STAGES + s); };
+  auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * C::STAGES + b); };
+  auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * C::STAGES + 2 + b); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * C::STAGES + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();  // 0 = leader
+  const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::STAGES; ++s) {
+      mbar_init(full_bar(s), 1);   // the leader's expect_tx arrival; both CTAs' bytes are counted on the leader's barrier
+      mbar_init(empty_bar(s), 1);  // one multicast commit
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(tfull_bar(b), 1);   // one multicast commit
+      mbar_init(tempty_bar(b), 8);  // 4 epilogue warps of each CTA, all arriving at the leader
+    }
+    *abort_flag = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tmA);
+    tma_prefetch_desc(&tmB);
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_u32(tmem_slot), C::TMEM_COLS);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // both CTAs' barriers exist before either signals the other
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int tiles_m = (p.M + 255) / 256;
+  const int tiles_n = (p.N + BN - 1) / BN;
+  const int ntiles = tiles_m * tiles_n;
+  const int kblocks = (p.K + BK - 1) / BK;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int t = pair; t < ntiles && ok; t += npairs) {
+        const int m0 = (t % tiles_m) * 256 + (int)rank * BM;       // this CTA's rows of A / of the output
+        const int nb0 = (t / tiles_m) * BN + (int)rank * C::HALF_B;  // this CTA's rows of B
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.err)) { ok = false; break; }
+          const uint32_t fb = full_bar(stage);
+          if (rank == 0) mbar_expect_tx(fb, 2 * C::STAGE_BYTES);
+          const uint32_t a_dst = smem_u32(smem + stage * C::STAGE_BYTES);
+          const uint32_t b_dst = a_dst + C::A_BYTES_;
+          if constexpr (!A_MN) {
+            tma_load_2d_pair(a_dst, &tmA, fb, kb * BK, m0);
+          } else {
+#pragma unroll
+            for (int j = 0; j < BM / 64; ++j) tma_load_2d_pair(a_dst + j * CHUNK_BYTES, &tmA, fb, m0 + 64 * j, kb * BK);
+          }
+          if constexpr (!B_MN) {
+            tma_load_2d_pair(b_dst, &tmB, fb, kb * BK, nb0);
+          } else {
+#pragma unroll
+            for (int j = 0; j < C::HALF_B / 64; ++j)
+              tma_load_2d_pair(b_dst + j * CHUNK_BYTES, &tmB, fb, nb0 + 64 * j, kb * BK);
+          }
+          if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && rank == 0) {
+      // M = 256 over the pair, N = 256
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) | ((B_MN ? 1u : 0u) << 16) |
+                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int t = pair; t < ntiles && ok; t += npairs) {
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.err)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.err)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(smem + stage * C::STAGE_BYTES);
+          const uint32_t b_addr = a_addr + C::A_BYTES_;
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            const uint64_t adesc = A_MN ? umma_desc_sw128(a_addr + k * 2048, CHUNK_BYTES, 1024)
+                                        : umma_desc_sw128(a_addr + k * 32, 0, 1024);
+            const uint64_t bdesc = B_MN ? umma_desc_sw128(b_addr + k * 2048, CHUNK_BYTES, 1024)
+                                        : umma_desc_sw128(b_addr + k * 32, 0, 1024);
+            umma_bf16_pair(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          umma_commit_pair(empty_bar(stage));  // frees the stage in both CTAs
+          if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit_pair(tfull_bar(acc));  // wakes the epilogue warps of both CTAs
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+  } else {
+    const int q = warp & 3;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    for (int t = pair; t < ntiles; t += npairs) {
+      const int m0 = (t % tiles_m) * 256 + (int)rank * BM;
+      const int n0 = (t / tiles_m) * BN;
+      bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.err);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const int row = m0 + q * 32 + lane;
+      epilogue_tile<BN>(p, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), row, n0);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_leader(tempty_bar(acc));
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1u;
+    }
+  }
+
+  // teardown: both CTAs meet before either releases shared memory or TMEM the other may still be using
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag != 0) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000LL) __nanosleep(1000);
+    __syncthreads();
+  }
+  cluster_sync_all();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
   }
 }
 
@@ -364,9 +541,46 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
   return cudaGetLastError();
 }
 
+template <bool A_MN, bool B_MN>
+cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
+  using C = PairCfg;
+  static bool attr_set = false;
+  auto kern = gemm_tc_pair_kernel<A_MN, B_MN>;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  CUtensorMap tmA, tmB;
+  bool ok = A_MN ? make_tmap_2d(&tmA, a.A, a.M, a.K, a.lda, 64) : make_tmap_2d(&tmA, a.A, a.K, a.M, a.lda, BM);
+  ok = ok && (B_MN ? make_tmap_2d(&tmB, a.B, a.N, a.K, a.ldb, 64) : make_tmap_2d(&tmB, a.B, a.K, a.N, a.ldb, C::HALF_B));
+  if (!ok) return cudaErrorInvalidValue;
+  GemmDev p;
+  p.C = a.C; p.resid = a.resid; p.gu = a.gu; p.rope_cos = a.rope_cos; p.rope_sin = a.rope_sin; p.err = a.err;
+  p.ldc = a.ldc; p.M = a.M; p.N = a.N; p.K = a.K; p.epi = a.epi;
+  p.seq = a.seq; p.head_dim = a.head_dim; p.rope_cols = a.rope_cols; p.d_ffn = a.d_ffn;
+  const int tiles = ((a.M + 255) / 256) * ((a.N + 255) / 256);
+  const int max_pairs = sm_count() / 2;
+  const int pairs = tiles < max_pairs ? tiles : max_pairs;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs, 1, 1);
+  cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = C::SMEM_BYTES;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, tmA, tmB, p);
+}
+
 }  // namespace
 
-int g_gemm_force_bn = 0;  // development knob: 0 = choose by tile count, 128 or 256 = force that tile width
+int g_gemm_force_bn = 0;
+int g_gemm_pairs = 1;  // development knob: 1 = CTA-pair kernel for outputs of at least 256 x 256, 0 = single-CTA kernel only  // development knob: 0 = choose by tile count, 128 or 256 = force that tile width
 
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream) {
   if (a.M <= 0 || a.N <= 0 || a.K <= 0 || !a.A || !a.B || !a.C || !a.err) return cudaErrorInvalidValue;
@@ -383,6 +597,12 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream) {
   // 128 x 256 tiles move 96 B of operands per tensor-core cycle through shared memory, 128 x 128 tiles 128 B: the
   // wide tile is faster even when it leaves SMs idle (measured), so the narrow one only serves N <= 128
   const bool wide = g_gemm_force_bn ? g_gemm_force_bn == 256 : a.N > 128;
+  if (g_gemm_pairs && !g_gemm_force_bn && a.M >= 256 && a.N >= 256) {
+    if (!a.a_mn && !a.b_mn) return launch_pair_variant<false, false>(a, stream);
+    if (!a.a_mn && a.b_mn) return launch_pair_variant<false, true>(a, stream);
+    if (a.a_mn && a.b_mn) return launch_pair_variant<true, true>(a, stream);
+    return cudaErrorInvalidValue;
+  }
   if (!a.a_mn && !a.b_mn) return wide ? launch_variant<256, false, false>(a, stream) : launch_variant<128, false, false>(a, stream);
   if (!a.a_mn && a.b_mn) return wide ? launch_variant<256, false, true>(a, stream) : launch_variant<128, false, true>(a, stream);
   if (a.a_mn && a.b_mn) return wide ? launch_variant<256, true, true>(a, stream) : launch_variant<128, true, true>(a, stream);

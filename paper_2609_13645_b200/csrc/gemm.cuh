@@ -42,5 +42,6 @@ struct GemmArgs {
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream);
 
 extern int g_gemm_force_bn;
+extern int g_gemm_pairs;
 
 }  // namespace fs

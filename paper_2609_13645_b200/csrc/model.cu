@@ -770,6 +770,7 @@ ft_status ft_get_profile(ft_model* m, int32_t cls, double* ms, double* work, int
 
 void ft_debug_attention_impl(int32_t impl) { g_attention_impl = impl; }
 void ft_debug_gemm_tile(int32_t bn) { g_gemm_force_bn = bn; }
+void ft_debug_gemm_pairs(int32_t on) { g_gemm_pairs = on; }
 
 const char* ft_last_error(const ft_model* m) { return m ? m->err.c_str() : "null model"; }
 int64_t ft_launch_count(const ft_model* m) { return m ? m->launches : 0; }

@@ -36,10 +36,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--no-flush", action="store_true")
     ap.add_argument("--bn", type=int, default=0, help="force the GEMM tile width (development)")
+    ap.add_argument("--pairs", type=int, default=1, help="0: single-CTA GEMM kernel only (development)")
     a = ap.parse_args()
     torch.manual_seed(0)
     if a.bn:
         B.lib().ft_debug_gemm_tile(a.bn)
+    B.lib().ft_debug_gemm_pairs(a.pairs)
     dev = "cuda"
     flush = None if a.no_flush else torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     err = torch.zeros(1, dtype=torch.int32, device=dev)
