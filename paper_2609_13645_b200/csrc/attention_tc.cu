@@ -172,26 +172,24 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
       const int k0 = j * C::BK;
       const bool need_mask = k0 + C::BK - 1 > q0 + q * 32;  // warp-uniform
+      if (need_mask) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          if (k0 + i > row) r0[i] = 0xff800000u;       // -inf
+          if (k0 + 32 + i > row) r1[i] = 0xff800000u;
+        }
+      }
       float mx = -INFINITY;
 #pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        float a = __uint_as_float(r0[i]) * scale_log2;
-        float c = __uint_as_float(r1[i]) * scale_log2;
-        if (need_mask) {
-          if (k0 + i > row) a = -INFINITY;
-          if (k0 + 32 + i > row) c = -INFINITY;
-        }
-        r0[i] = __float_as_uint(a);
-        r1[i] = __float_as_uint(c);
-        mx = fmaxf(mx, fmaxf(a, c));
-      }
-      const float mnew = fmaxf(mref, ceilf(mx));
-      const float alpha = exp2f(mref - mnew);  // exact power of two; 0 on the first block
+      for (int i = 0; i < 32; ++i) mx = fmaxf(mx, fmaxf(__uint_as_float(r0[i]), __uint_as_float(r1[i])));
+      // scale_log2 > 0, so the maximum commutes with the scaling
+      const float mnew = fmaxf(mref, ceilf(mx * scale_log2));
+      const float alpha = fast_exp2(mref - mnew);  // exact power of two; 0 on the first block
       float psum = 0.f;
 #pragma unroll
       for (int i = 0; i < 32; ++i) {
-        const float a = exp2f(__uint_as_float(r0[i]) - mnew);
-        const float c = exp2f(__uint_as_float(r1[i]) - mnew);
+        const float a = fast_exp2(fmaf(__uint_as_float(r0[i]), scale_log2, -mnew));
+        const float c = fast_exp2(fmaf(__uint_as_float(r1[i]), scale_log2, -mnew));
         psum += a + c;
         r0[i] = __float_as_uint(a);
         r1[i] = __float_as_uint(c);
@@ -587,19 +585,34 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
       }
+      // masking is only needed where the block touches the diagonal (or the end of the sequence): warp-uniform
+      const int cmin = y0 + ch * 32, rmin = x0 + q * 32;
+      bool full;
+      if constexpr (MODE == MODE_DQ) full = cmin + 31 <= rmin;            // every key <= every query of this warp
+      else full = cmin >= rmin + 31 && cmin + 32 <= S;                    // every query >= every key, and in range
+      if constexpr (MODE == MODE_DQ) {
+        const float nl = -lse2_row;
 #pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        const int col = y0 + ch * 32 + i;
-        float p, ds;
-        if constexpr (MODE == MODE_DQ) {
-          p = col <= row ? exp2f(__uint_as_float(rs[i]) * scale_log2 - lse2_row) : 0.f;
-          ds = p * (__uint_as_float(rp[i]) - delta_row);
-        } else {
-          p = (col >= row && col < S) ? exp2f(__uint_as_float(rs[i]) * scale_log2 - st_lse[i]) : 0.f;
-          ds = p * (__uint_as_float(rp[i]) - st_dl[i]);
+        for (int i = 0; i < 32; ++i) {
+          float p = fast_exp2(fmaf(__uint_as_float(rs[i]), scale_log2, nl));
+          if (!full && cmin + i > row) p = 0.f;
+          rs[i] = __float_as_uint(p);
+          rp[i] = __float_as_uint(p * (__uint_as_float(rp[i]) - delta_row));
         }
-        rs[i] = __float_as_uint(p);
-        rp[i] = __float_as_uint(ds);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+          const float4 l4 = *reinterpret_cast<const float4*>(st_lse + i);
+          const float4 d4 = *reinterpret_cast<const float4*>(st_dl + i);
+          const float ll[4] = {l4.x, l4.y, l4.z, l4.w}, dd[4] = {d4.x, d4.y, d4.z, d4.w};
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            float p = fast_exp2(fmaf(__uint_as_float(rs[i + u]), scale_log2, -ll[u]));
+            if (!full && (cmin + i + u < row || cmin + i + u >= S)) p = 0.f;
+            rs[i + u] = __float_as_uint(p);
+            rp[i + u] = __float_as_uint(p * (__uint_as_float(rp[i + u]) - dd[u]));
+          }
+        }
       }
       ok = mbar_wait(bar(BB_TEMPTY + bf), (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag, err);
       ok = __all_sync(0xffffffffu, ok);

@@ -218,6 +218,13 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr, uint32_t lbo
   return d;
 }
 
+// 2^x with the hardware approximation (relative error about 2^-22; -inf gives 0, results below 2^-126 flush to 0)
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 // ---------------------------------------------------------------- small reductions
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
