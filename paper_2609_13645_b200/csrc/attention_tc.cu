@@ -17,6 +17,13 @@ namespace fs {
 namespace {
 
 constexpr float kLn2 = 0.6931471805599453f;
+
+#ifdef FS_ATTN_TRACE
+__device__ long long g_trace[8192];
+#define FS_TRACE(slot) do { if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) g_trace[(slot)] = clock64(); } while (0)
+#else
+#define FS_TRACE(slot) do { } while (0)
+#endif
 constexpr int ATT_THREADS = 192;
 
 // barrier slots of the forward kernel
@@ -318,12 +325,9 @@ struct BwdCfg {
   static constexpr int KC = D / 64;
   static constexpr int X_BYTES = 128 * D * 2;
   static constexpr int Y_BYTES = 64 * D * 2;
-  static constexpr int T_BYTES = 128 * 64 * 2;
-  static constexpr int NT = MODE == MODE_DKV ? 2 : 1;
-  static constexpr int NST = MODE == MODE_DKV ? 3 : 4;  // stages of the streamed-tile ring
+  static constexpr int NST = 4;  // stages of the streamed-tile ring
   static constexpr int OFF_X1 = 0, OFF_X2 = X_BYTES, OFF_Y = 2 * X_BYTES;
-  static constexpr int OFF_T = OFF_Y + NST * 2 * Y_BYTES;
-  static constexpr int OFF_STAT = OFF_T + 2 * NT * T_BYTES;
+  static constexpr int OFF_STAT = OFF_Y + NST * 2 * Y_BYTES;
   static constexpr int OFF_BAR = OFF_STAT + 2048;
   static constexpr int SMEM_BYTES = OFF_BAR + 256;
   static constexpr int TMEM_COLS = 512;  // buffer b: S at b*128, dP at b*128+64; accumulators from column 256
@@ -409,9 +413,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar(BB_SDPFULL + i), 1);
-      mbar_init(bar(BB_SDPEMPTY + i), 8);
       mbar_init(bar(BB_TFULL + i), 8);
-      mbar_init(bar(BB_TEMPTY + i), 1);
     }
     mbar_init(bar(BB_ACCDONE), 1);
     *abort_flag = 0;
@@ -450,6 +452,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
       bool ok = mbar_wait(bar(BB_YEMPTY + st), (((uint32_t)(it / C::NST)) & 1u) ^ 1u, abort_flag, err);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
+      if (lane == 0 && it < 100) FS_TRACE(it * 16 + 10);
       const uint32_t ydst = sbase + C::OFF_Y + st * 2 * C::Y_BYTES;
       if constexpr (MODE == MODE_DQ) {
         if (lane == 0) {
@@ -489,21 +492,25 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
       const uint32_t idesc_base = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 4) << 24);
       const uint32_t idesc_sdp = idesc_base | ((uint32_t)(64 >> 3) << 17);            // N = 64, both K-major
       const uint32_t idesc_acc = idesc_base | (1u << 16) | ((uint32_t)(D >> 3) << 17);  // N = D, B mn-major
+      // descriptors are built once per tile; a K step of 16 elements moves the start-address field (units of 16 B)
+      // by 2 inside a 64-element chunk of a K-major tile and by 128 for an mn-major tile
+      const uint64_t dx1 = umma_desc_sw128(sbase + C::OFF_X1, 0, 1024), dx2 = umma_desc_sw128(sbase + C::OFF_X2, 0, 1024);
       auto issue_sdp = [&](int it) {
         const int st = it % C::NST;
-        const uint32_t y1 = sbase + C::OFF_Y + st * 2 * C::Y_BYTES, y2 = y1 + C::Y_BYTES;
+        const uint32_t y1 = sbase + C::OFF_Y + st * 2 * C::Y_BYTES;
+        const uint64_t dy1 = umma_desc_sw128(y1, 0, 1024), dy2 = umma_desc_sw128(y1 + C::Y_BYTES, 0, 1024);
         const uint32_t d_s = tmem_base + (uint32_t)((it & 1) * 128), d_p = d_s + 64;
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
-          const uint32_t xo = (k >> 2) * 16384 + (k & 3) * 32, yo = (k >> 2) * 8192 + (k & 3) * 32;
-          umma_bf16(d_s, umma_desc_sw128(sbase + C::OFF_X1 + xo, 0, 1024), umma_desc_sw128(y1 + yo, 0, 1024), idesc_sdp,
-                    k > 0 ? 1u : 0u);
+          const uint64_t xo = (uint64_t)(((k >> 2) * 16384 + (k & 3) * 32) >> 4);
+          const uint64_t yo = (uint64_t)(((k >> 2) * 8192 + (k & 3) * 32) >> 4);
+          umma_bf16(d_s, dx1 + xo, dy1 + yo, idesc_sdp, k > 0 ? 1u : 0u);
         }
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
-          const uint32_t xo = (k >> 2) * 16384 + (k & 3) * 32, yo = (k >> 2) * 8192 + (k & 3) * 32;
-          umma_bf16(d_p, umma_desc_sw128(sbase + C::OFF_X2 + xo, 0, 1024), umma_desc_sw128(y2 + yo, 0, 1024), idesc_sdp,
-                    k > 0 ? 1u : 0u);
+          const uint64_t xo = (uint64_t)(((k >> 2) * 16384 + (k & 3) * 32) >> 4);
+          const uint64_t yo = (uint64_t)(((k >> 2) * 8192 + (k & 3) * 32) >> 4);
+          umma_bf16(d_p, dx2 + xo, dy2 + yo, idesc_sdp, k > 0 ? 1u : 0u);
         }
         umma_commit(bar(BB_SDPFULL + (it & 1)));
       };
@@ -514,33 +521,39 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
       }
       for (int it = 0; it < iters && ok; ++it) {
         if (it + 1 < iters) {
-          const int s1 = (it + 1) & 1, y1s = (it + 1) % C::NST;
+          const int y1s = (it + 1) % C::NST;
           if (!mbar_wait(bar(BB_YFULL + y1s), ((uint32_t)((it + 1) / C::NST)) & 1u, abort_flag, err)) { ok = false; break; }
-          if (!mbar_wait(bar(BB_SDPEMPTY + s1), (((uint32_t)(it + 1) >> 1) & 1u) ^ 1u, abort_flag, err)) { ok = false; break; }
+          // buffer s1 was last read by the accumulating MMAs of block it-1, issued earlier by this thread: in order
           tc_fence_after();
+          if (it < 100) FS_TRACE(it * 16 + 0);
           issue_sdp(it + 1);
+          if (it < 100) FS_TRACE(it * 16 + 1);
         }
         const int bf = it & 1;
         if (!mbar_wait(bar(BB_TFULL + bf), ((uint32_t)it >> 1) & 1u, abort_flag, err)) { ok = false; break; }
         tc_fence_after();
+        if (it < 100) FS_TRACE(it * 16 + 2);
         const int yst = it % C::NST;
         const uint32_t y1 = sbase + C::OFF_Y + yst * 2 * C::Y_BYTES, y2 = y1 + C::Y_BYTES;
-        const uint32_t t0 = sbase + C::OFF_T + bf * C::NT * C::T_BYTES, t1 = t0 + C::T_BYTES;
+        // A operands (bf16 P^T / dS^T) sit in TMEM where S / dP were: 16 queries (K = 16) = 8 columns; the two
+        // compute warps of a lane quarter each wrote their 32 queries at the start of their own 32 fp32 columns
+        const uint32_t tp = tmem_base + (uint32_t)(bf * 128), tds = tp + 64;
+        const uint64_t by1 = umma_desc_sw128(y1, 8192, 1024), by2 = umma_desc_sw128(y2, 8192, 1024);
+        const uint32_t first = it > 0 ? 1u : 0u;
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-          const uint32_t acc = (it > 0 || k > 0) ? 1u : 0u;
+          const uint32_t acc = k > 0 ? 1u : first;
+          const uint32_t acol = (uint32_t)((k >> 1) * 32 + (k & 1) * 8);
+          const uint64_t ko = (uint64_t)((k * 2048) >> 4);
           if constexpr (MODE == MODE_DQ) {
-            umma_bf16(tmem_base + C::ACC0, umma_desc_sw128(t0 + k * 32, 0, 1024),
-                      umma_desc_sw128(y1 + k * 2048, 8192, 1024), idesc_acc, acc);  // dQ += dS K
+            umma_bf16_ts(tmem_base + C::ACC0, tds + acol, by1 + ko, idesc_acc, acc);  // dQ += dS K
           } else {
-            umma_bf16(tmem_base + C::ACC0, umma_desc_sw128(t0 + k * 32, 0, 1024),
-                      umma_desc_sw128(y2 + k * 2048, 8192, 1024), idesc_acc, acc);  // dV += P^T dO
-            umma_bf16(tmem_base + C::ACC1, umma_desc_sw128(t1 + k * 32, 0, 1024),
-                      umma_desc_sw128(y1 + k * 2048, 8192, 1024), idesc_acc, acc);  // dK += dS^T Q
+            umma_bf16_ts(tmem_base + C::ACC0, tp + acol, by2 + ko, idesc_acc, acc);   // dV += P^T dO
+            umma_bf16_ts(tmem_base + C::ACC1, tds + acol, by1 + ko, idesc_acc, acc);  // dK += dS^T Q
           }
         }
         umma_commit(bar(BB_YEMPTY + yst));
-        umma_commit(bar(BB_TEMPTY + bf));
+        if (it < 100) FS_TRACE(it * 16 + 3);
       }
       if (ok) umma_commit(bar(BB_ACCDONE));
     }
@@ -565,13 +578,12 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
+      if (threadIdx.x == 64 && it < 100) FS_TRACE(it * 16 + 4);
       uint32_t rs[32], rp[32];
       tmem_ld32(tlane + (uint32_t)(bf * 128 + ch * 32), rs);
       tmem_ld32(tlane + (uint32_t)(bf * 128 + 64 + ch * 32), rp);
       tmem_ld_wait();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(BB_SDPEMPTY + bf));
+      if (threadIdx.x == 64 && it < 100) FS_TRACE(it * 16 + 5);
 
       int y0;
       const int yst = it % C::NST;
@@ -614,32 +626,22 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
           }
         }
       }
-      ok = mbar_wait(bar(BB_TEMPTY + bf), (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag, err);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      uint8_t* t0row = smem + C::OFF_T + bf * C::NT * C::T_BYTES + rloc * 128;
+      if (threadIdx.x == 64 && it < 100) FS_TRACE(it * 16 + 6);
+      // bf16 pairs back into TMEM, over this warp's own (already loaded) fp32 columns
+      uint32_t wp[16], wd[16];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const int chunk = ((ch * 4 + c) ^ (rloc & 7)) << 4;
-        uint4 vp, vd;
-        vp.x = pack_bf16(__uint_as_float(rs[c * 8 + 0]), __uint_as_float(rs[c * 8 + 1]));
-        vp.y = pack_bf16(__uint_as_float(rs[c * 8 + 2]), __uint_as_float(rs[c * 8 + 3]));
-        vp.z = pack_bf16(__uint_as_float(rs[c * 8 + 4]), __uint_as_float(rs[c * 8 + 5]));
-        vp.w = pack_bf16(__uint_as_float(rs[c * 8 + 6]), __uint_as_float(rs[c * 8 + 7]));
-        vd.x = pack_bf16(__uint_as_float(rp[c * 8 + 0]), __uint_as_float(rp[c * 8 + 1]));
-        vd.y = pack_bf16(__uint_as_float(rp[c * 8 + 2]), __uint_as_float(rp[c * 8 + 3]));
-        vd.z = pack_bf16(__uint_as_float(rp[c * 8 + 4]), __uint_as_float(rp[c * 8 + 5]));
-        vd.w = pack_bf16(__uint_as_float(rp[c * 8 + 6]), __uint_as_float(rp[c * 8 + 7]));
-        if constexpr (MODE == MODE_DQ) {
-          *reinterpret_cast<uint4*>(t0row + chunk) = vd;
-        } else {
-          *reinterpret_cast<uint4*>(t0row + chunk) = vp;
-          *reinterpret_cast<uint4*>(t0row + C::T_BYTES + chunk) = vd;
-        }
+      for (int c = 0; c < 16; ++c) {
+        wp[c] = pack_bf16(__uint_as_float(rs[2 * c]), __uint_as_float(rs[2 * c + 1]));
+        wd[c] = pack_bf16(__uint_as_float(rp[2 * c]), __uint_as_float(rp[2 * c + 1]));
       }
-      fence_proxy_async_smem();
+      if constexpr (MODE == MODE_DKV) tmem_st16(tlane + (uint32_t)(bf * 128 + ch * 32), wp);
+      tmem_st16(tlane + (uint32_t)(bf * 128 + 64 + ch * 32), wd);
+      tmem_st_wait();
+      if (threadIdx.x == 64 && it < 100) FS_TRACE(it * 16 + 8);
+      tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(BB_TFULL + bf));
+      if (threadIdx.x == 64 && it < 100) FS_TRACE(it * 16 + 9);
     }
     if (ok) {
       ok = mbar_wait(bar(BB_ACCDONE), 0, abort_flag, err);
@@ -771,5 +773,13 @@ cudaError_t attention_bwd_tc(const bf16* qkv, const bf16* o, const bf16* d_o, co
   if (d == 128) return attention_bwd_tc_t<128>(qkv, o, d_o, lse, delta, dqkv, cs, sn, B, S, nh, nkv, err, st);
   return cudaErrorInvalidValue;
 }
+
+#ifdef FS_ATTN_TRACE
+}  // namespace fs
+extern "C" int ft_debug_attn_trace(long long* host_dst, int n) {
+  return (int)cudaMemcpyFromSymbol(host_dst, fs::g_trace, sizeof(long long) * n);
+}
+namespace fs {
+#endif
 
 }  // namespace fs
