@@ -108,8 +108,6 @@ typedef enum {
 ft_status ft_set_profiling(ft_model* m, int32_t enable);
 ft_status ft_get_profile(ft_model* m, int32_t cls, double* ms, double* work, int64_t* launches);
 
-/* Development switch: 1 = tcgen05 attention kernels (default), 0 = warp-level mma.sync attention kernels. */
-void ft_debug_attention_impl(int32_t impl);
 /* Development switch: force the GEMM tile width (128 or 256 columns); 0 = choose by tile count (default). */
 void ft_debug_gemm_tile(int32_t bn);
 /* Development switch: 1 = CTA-pair (cta_group::2, 256 x 256 tile) GEMM kernel where it applies (default), 0 = off. */

@@ -68,8 +68,6 @@ def lib():
         L.ft_set_profiling.restype = C.c_int
         L.ft_get_profile.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(i64)]
         L.ft_get_profile.restype = C.c_int
-        L.ft_debug_attention_impl.argtypes = [i32]
-        L.ft_debug_attention_impl.restype = None
         L.ft_debug_gemm_tile.argtypes = [i32]
         L.ft_debug_gemm_tile.restype = None
         L.ft_debug_gemm_pairs.argtypes = [i32]

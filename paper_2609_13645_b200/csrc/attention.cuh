@@ -1,4 +1,4 @@
-// Host-side interface of the causal flash-attention kernels.
+// Host-side interface of the causal flash-attention kernels (tcgen05 tensor cores, accumulators in TMEM, TMA loads).
 #pragma once
 #include <cuda_runtime.h>
 
@@ -7,29 +7,20 @@
 namespace fs {
 
 // qkv bf16 [B*S, (n_h + 2 n_kv) d] packed q heads | k heads | v heads (q, k rotated); o bf16 [B*S, n_h d];
-// lse fp32 [B, n_h, S] in natural log.  d in {64, 128}.  One kernel launch.
-cudaError_t attention_fwd(const bf16* qkv, bf16* o, float* lse, int B, int S, int n_heads, int n_kv, int d,
+// lse fp32 [B, n_h, S] in natural log.  d in {64, 128}.  err: device status word.  One kernel launch.
+cudaError_t attention_fwd(const bf16* qkv, bf16* o, float* lse, int B, int S, int n_heads, int n_kv, int d, int* err,
                           cudaStream_t st);
 
 // Three kernel launches (delta pre-pass, dQ, dK/dV).  delta: fp32 scratch [B, n_h, S].  dqkv has qkv's layout.
 // cos/sin: fp32 [S, d/2] or both null (then dq, dk are left in the rotated frame).
 cudaError_t attention_bwd(const bf16* qkv, const bf16* o, const bf16* d_o, const float* lse, float* delta, bf16* dqkv,
-                          const float* cos, const float* sin, int B, int S, int n_heads, int n_kv, int d,
+                          const float* cos, const float* sin, int B, int S, int n_heads, int n_kv, int d, int* err,
                           cudaStream_t st);
 
-// The same forward on the tcgen05 tensor cores (accumulators in TMEM, operands by TMA).  err: device status word.
-cudaError_t attention_fwd_tc(const bf16* qkv, bf16* o, float* lse, int B, int S, int n_heads, int n_kv, int d, int* err,
-                             cudaStream_t st);
-
-cudaError_t attention_bwd_tc(const bf16* qkv, const bf16* o, const bf16* d_o, const float* lse, float* delta, bf16* dqkv,
-                             const float* cos, const float* sin, int B, int S, int n_heads, int n_kv, int d, int* err,
-                             cudaStream_t st);
 // delta[b, n, i] = sum_k dO[b,i,n,k] O[b,i,n,k] (the backward pre-pass; one launch)
 cudaError_t attention_delta(const bf16* o, const bf16* d_o, float* delta, int B, int S, int n_heads, int d, cudaStream_t st);
 
 // Device status word used by the single-kernel entry points (address on the current device).
 int* attention_status_word();
-// 1: tcgen05 kernels where they exist (default); 0: warp-level mma.sync kernels.
-extern int g_attention_impl;
 
 }  // namespace fs

@@ -742,8 +742,6 @@ static __device__ int g_attn_status;
 
 }  // namespace
 
-int g_attention_impl = 1;
-
 int* attention_status_word() {
   static int* addr[64] = {nullptr};
   int dev = 0;
@@ -756,7 +754,7 @@ int* attention_status_word() {
   return addr[dev];
 }
 
-cudaError_t attention_fwd_tc(const bf16* qkv, bf16* o, float* lse, int B, int S, int nh, int nkv, int d, int* err,
+cudaError_t attention_fwd(const bf16* qkv, bf16* o, float* lse, int B, int S, int nh, int nkv, int d, int* err,
                              cudaStream_t st) {
   if (B <= 0 || S <= 0 || nh <= 0 || nkv <= 0 || nh % nkv || !err) return cudaErrorInvalidValue;
   if (d == 64) return attention_fwd_tc_t<64>(qkv, o, lse, B, S, nh, nkv, err, st);
@@ -764,7 +762,7 @@ cudaError_t attention_fwd_tc(const bf16* qkv, bf16* o, float* lse, int B, int S,
   return cudaErrorInvalidValue;
 }
 
-cudaError_t attention_bwd_tc(const bf16* qkv, const bf16* o, const bf16* d_o, const float* lse, float* delta, bf16* dqkv,
+cudaError_t attention_bwd(const bf16* qkv, const bf16* o, const bf16* d_o, const float* lse, float* delta, bf16* dqkv,
                              const float* cs, const float* sn, int B, int S, int nh, int nkv, int d, int* err,
                              cudaStream_t st) {
   if (B <= 0 || S <= 0 || nh <= 0 || nkv <= 0 || nh % nkv || !err) return cudaErrorInvalidValue;

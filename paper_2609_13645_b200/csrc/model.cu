@@ -287,10 +287,7 @@ ft_status layer_forward(ft_model* m, int l, LayerActs& a, int B, int S) {
     FT_GEMM(g);
   }
   prof_begin(m);
-  if (g_attention_impl)
-    FT_CUDA(attention_fwd_tc(a.qkv, a.o, a.lse, B, S, m->cfg.n_heads, m->cfg.n_kv_heads, m->d, &m->sc->err, st));
-  else
-    FT_CUDA(attention_fwd(a.qkv, a.o, a.lse, B, S, m->cfg.n_heads, m->cfg.n_kv_heads, m->d, st));
+  FT_CUDA(attention_fwd(a.qkv, a.o, a.lse, B, S, m->cfg.n_heads, m->cfg.n_kv_heads, m->d, &m->sc->err, st));
   m->launches += 1;
   prof_end(m, FT_PROF_ATTN_FWD, 2.0 * B * m->cfg.n_heads * (double)S * S * m->d, 1);
   {
@@ -358,12 +355,8 @@ ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
   s = linear_backward(m, m->dxB, a.o, m->idx_layer(l, 2), m->d_o, T, h, hq);
   if (s) return s;
   prof_begin(m);
-  if (g_attention_impl)
-    FT_CUDA(attention_bwd_tc(a.qkv, a.o, m->d_o, a.lse, m->delta, m->d_qkv, m->rope_cos, m->rope_sin, B, S,
-                             m->cfg.n_heads, m->cfg.n_kv_heads, m->d, &m->sc->err, st));
-  else
-    FT_CUDA(attention_bwd(a.qkv, a.o, m->d_o, a.lse, m->delta, m->d_qkv, m->rope_cos, m->rope_sin, B, S, m->cfg.n_heads,
-                          m->cfg.n_kv_heads, m->d, st));
+  FT_CUDA(attention_bwd(a.qkv, a.o, m->d_o, a.lse, m->delta, m->d_qkv, m->rope_cos, m->rope_sin, B, S, m->cfg.n_heads,
+                        m->cfg.n_kv_heads, m->d, &m->sc->err, st));
   m->launches += 3;
   prof_end(m, FT_PROF_ATTN_BWD, 4.0 * B * m->cfg.n_heads * (double)S * S * m->d, 3);
   s = linear_backward(m, m->d_qkv, a.h1, m->idx_layer(l, 1), m->d_h, T, nqkv, h);
@@ -768,7 +761,6 @@ ft_status ft_get_profile(ft_model* m, int32_t cls, double* ms, double* work, int
   return FT_OK;
 }
 
-void ft_debug_attention_impl(int32_t impl) { g_attention_impl = impl; }
 void ft_debug_gemm_tile(int32_t bn) { g_gemm_force_bn = bn; }
 void ft_debug_gemm_pairs(int32_t on) { g_gemm_pairs = on; }
 
@@ -799,16 +791,10 @@ ft_status ft_k_gemm(const void* dev_A, int32_t a_mn, int64_t lda, const void* de
 ft_status ft_k_attention_fwd(const void* dev_qkv, void* dev_o, float* dev_lse, int32_t B, int32_t S, int32_t n_heads,
                              int32_t n_kv_heads, int32_t head_dim, void* stream) {
   if (!dev_qkv || !dev_o || !dev_lse) return FT_EINVAL;
-  cudaError_t e;
-  if (g_attention_impl) {
-    int* status = attention_status_word();
-    if (!status) return FT_ECUDA;
-    e = attention_fwd_tc(reinterpret_cast<const bf16*>(dev_qkv), reinterpret_cast<bf16*>(dev_o), dev_lse, B, S, n_heads,
-                         n_kv_heads, head_dim, status, reinterpret_cast<cudaStream_t>(stream));
-  } else {
-    e = attention_fwd(reinterpret_cast<const bf16*>(dev_qkv), reinterpret_cast<bf16*>(dev_o), dev_lse, B, S, n_heads,
-                      n_kv_heads, head_dim, reinterpret_cast<cudaStream_t>(stream));
-  }
+  int* status = attention_status_word();
+  if (!status) return FT_ECUDA;
+  cudaError_t e = attention_fwd(reinterpret_cast<const bf16*>(dev_qkv), reinterpret_cast<bf16*>(dev_o), dev_lse, B, S,
+                                n_heads, n_kv_heads, head_dim, status, reinterpret_cast<cudaStream_t>(stream));
   if (e == cudaErrorInvalidValue) return FT_EINVAL;
   return e == cudaSuccess ? FT_OK : FT_ECUDA;
 }
@@ -817,19 +803,12 @@ ft_status ft_k_attention_bwd(const void* dev_qkv, const void* dev_o, const void*
                              float* dev_delta, void* dev_dqkv, const float* dev_cos, const float* dev_sin, int32_t B,
                              int32_t S, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, void* stream) {
   if (!dev_qkv || !dev_o || !dev_do || !dev_lse || !dev_delta || !dev_dqkv) return FT_EINVAL;
-  cudaError_t e;
-  if (g_attention_impl) {
-    int* status = attention_status_word();
-    if (!status) return FT_ECUDA;
-    e = attention_bwd_tc(reinterpret_cast<const bf16*>(dev_qkv), reinterpret_cast<const bf16*>(dev_o),
-                         reinterpret_cast<const bf16*>(dev_do), dev_lse, dev_delta, reinterpret_cast<bf16*>(dev_dqkv),
-                         dev_cos, dev_sin, B, S, n_heads, n_kv_heads, head_dim, status,
-                         reinterpret_cast<cudaStream_t>(stream));
-  } else {
-    e = attention_bwd(reinterpret_cast<const bf16*>(dev_qkv), reinterpret_cast<const bf16*>(dev_o),
-                      reinterpret_cast<const bf16*>(dev_do), dev_lse, dev_delta, reinterpret_cast<bf16*>(dev_dqkv),
-                      dev_cos, dev_sin, B, S, n_heads, n_kv_heads, head_dim, reinterpret_cast<cudaStream_t>(stream));
-  }
+  int* status = attention_status_word();
+  if (!status) return FT_ECUDA;
+  cudaError_t e = attention_bwd(reinterpret_cast<const bf16*>(dev_qkv), reinterpret_cast<const bf16*>(dev_o),
+                                reinterpret_cast<const bf16*>(dev_do), dev_lse, dev_delta,
+                                reinterpret_cast<bf16*>(dev_dqkv), dev_cos, dev_sin, B, S, n_heads, n_kv_heads, head_dim,
+                                status, reinterpret_cast<cudaStream_t>(stream));
   if (e == cudaErrorInvalidValue) return FT_EINVAL;
   return e == cudaSuccess ? FT_OK : FT_ECUDA;
 }
