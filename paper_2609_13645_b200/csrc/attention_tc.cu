@@ -318,7 +318,7 @@ enum { MODE_DQ = 0, MODE_DKV = 1 };
 // barrier slots: Y ring (up to 4 stages) first, then the double-buffered TMEM / operand-tile handshakes
 enum { BB_XFULL = 0, BB_YFULL = 1, BB_YEMPTY = 5, BB_SDPFULL = 9, BB_SDPEMPTY = 11, BB_TFULL = 13, BB_TEMPTY = 15,
        BB_ACCDONE = 17, BB_COUNT = 18 };
-constexpr int BWD_THREADS = 320;
+constexpr int BWD_THREADS = 352;  // producer, MMA issuer A, 8 compute warps, MMA issuer B
 
 template <int D, int MODE>
 struct BwdCfg {
@@ -409,13 +409,13 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
     mbar_init(bar(BB_XFULL), 1);
     for (int i = 0; i < C::NST; ++i) {
       mbar_init(bar(BB_YFULL + i), MODE == MODE_DKV ? 2 : 1);
-      mbar_init(bar(BB_YEMPTY + i), 1);
+      mbar_init(bar(BB_YEMPTY + i), 2);   // one commit from each MMA-issuing warp
     }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(bar(BB_SDPFULL + i), 1);
+      mbar_init(bar(BB_SDPFULL + i), 2);
       mbar_init(bar(BB_TFULL + i), 8);
     }
-    mbar_init(bar(BB_ACCDONE), 1);
+    mbar_init(bar(BB_ACCDONE), 2);
     *abort_flag = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tm_qkv128);
@@ -486,31 +486,29 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
         if (lane == 0) mbar_arrive(bar(BB_YFULL + st));
       }
     }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
+  } else if (warp == 1 || warp == 10) {
+    // ------------------------------------------------------------------ MMA issuers
+    // A single thread cannot issue the small (N = 64 / 128) MMAs of this kernel fast enough to keep the tensor pipe
+    // fed, so two warps issue independent accumulator chains: side 0 owns S (and dV, which reads P^T from the S
+    // columns), side 1 owns dP (and dK / dQ, which read dS from the dP columns).  Each chain stays in issue order.
     if (lane == 0) {
+      const int side = warp == 1 ? 0 : 1;
       const uint32_t idesc_base = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 4) << 24);
       const uint32_t idesc_sdp = idesc_base | ((uint32_t)(64 >> 3) << 17);            // N = 64, both K-major
       const uint32_t idesc_acc = idesc_base | (1u << 16) | ((uint32_t)(D >> 3) << 17);  // N = D, B mn-major
       // descriptors are built once per tile; a K step of 16 elements moves the start-address field (units of 16 B)
       // by 2 inside a 64-element chunk of a K-major tile and by 128 for an mn-major tile
-      const uint64_t dx1 = umma_desc_sw128(sbase + C::OFF_X1, 0, 1024), dx2 = umma_desc_sw128(sbase + C::OFF_X2, 0, 1024);
+      const uint64_t dx = umma_desc_sw128(sbase + (side == 0 ? C::OFF_X1 : C::OFF_X2), 0, 1024);
       auto issue_sdp = [&](int it) {
         const int st = it % C::NST;
-        const uint32_t y1 = sbase + C::OFF_Y + st * 2 * C::Y_BYTES;
-        const uint64_t dy1 = umma_desc_sw128(y1, 0, 1024), dy2 = umma_desc_sw128(y1 + C::Y_BYTES, 0, 1024);
-        const uint32_t d_s = tmem_base + (uint32_t)((it & 1) * 128), d_p = d_s + 64;
+        const uint32_t y = sbase + C::OFF_Y + st * 2 * C::Y_BYTES + side * C::Y_BYTES;
+        const uint64_t dy = umma_desc_sw128(y, 0, 1024);
+        const uint32_t d_t = tmem_base + (uint32_t)((it & 1) * 128 + side * 64);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
           const uint64_t xo = (uint64_t)(((k >> 2) * 16384 + (k & 3) * 32) >> 4);
           const uint64_t yo = (uint64_t)(((k >> 2) * 8192 + (k & 3) * 32) >> 4);
-          umma_bf16(d_s, dx1 + xo, dy1 + yo, idesc_sdp, k > 0 ? 1u : 0u);
-        }
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-          const uint64_t xo = (uint64_t)(((k >> 2) * 16384 + (k & 3) * 32) >> 4);
-          const uint64_t yo = (uint64_t)(((k >> 2) * 8192 + (k & 3) * 32) >> 4);
-          umma_bf16(d_p, dx2 + xo, dy2 + yo, idesc_sdp, k > 0 ? 1u : 0u);
+          umma_bf16(d_t, dx + xo, dy + yo, idesc_sdp, k > 0 ? 1u : 0u);
         }
         umma_commit(bar(BB_SDPFULL + (it & 1)));
       };
@@ -523,37 +521,34 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
         if (it + 1 < iters) {
           const int y1s = (it + 1) % C::NST;
           if (!mbar_wait(bar(BB_YFULL + y1s), ((uint32_t)((it + 1) / C::NST)) & 1u, abort_flag, err)) { ok = false; break; }
-          // buffer s1 was last read by the accumulating MMAs of block it-1, issued earlier by this thread: in order
+          // the TMEM columns this writes were last read by this same thread's accumulating MMAs of block it-1: in order
           tc_fence_after();
-          if (it < 100) FS_TRACE(it * 16 + 0);
+          if (side == 0 && it < 100) FS_TRACE(it * 16 + 0);
           issue_sdp(it + 1);
-          if (it < 100) FS_TRACE(it * 16 + 1);
+          if (side == 0 && it < 100) FS_TRACE(it * 16 + 1);
         }
         const int bf = it & 1;
         if (!mbar_wait(bar(BB_TFULL + bf), ((uint32_t)it >> 1) & 1u, abort_flag, err)) { ok = false; break; }
         tc_fence_after();
-        if (it < 100) FS_TRACE(it * 16 + 2);
+        if (side == 0 && it < 100) FS_TRACE(it * 16 + 2);
         const int yst = it % C::NST;
         const uint32_t y1 = sbase + C::OFF_Y + yst * 2 * C::Y_BYTES, y2 = y1 + C::Y_BYTES;
         // A operands (bf16 P^T / dS^T) sit in TMEM where S / dP were: 16 queries (K = 16) = 8 columns; the two
         // compute warps of a lane quarter each wrote their 32 queries at the start of their own 32 fp32 columns
-        const uint32_t tp = tmem_base + (uint32_t)(bf * 128), tds = tp + 64;
-        const uint64_t by1 = umma_desc_sw128(y1, 8192, 1024), by2 = umma_desc_sw128(y2, 8192, 1024);
+        const uint32_t ta = tmem_base + (uint32_t)(bf * 128 + side * 64);
         const uint32_t first = it > 0 ? 1u : 0u;
+        if (MODE == MODE_DKV || side == 1) {
+          // side 0: dV += P^T dO;  side 1: dK += dS^T Q  (or dQ += dS K)
+          const uint64_t by = umma_desc_sw128((MODE == MODE_DKV && side == 0) ? y2 : y1, 8192, 1024);
+          const uint32_t dacc = tmem_base + (uint32_t)((MODE == MODE_DKV && side == 1) ? C::ACC1 : C::ACC0);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const uint32_t acc = k > 0 ? 1u : first;
-          const uint32_t acol = (uint32_t)((k >> 1) * 32 + (k & 1) * 8);
-          const uint64_t ko = (uint64_t)((k * 2048) >> 4);
-          if constexpr (MODE == MODE_DQ) {
-            umma_bf16_ts(tmem_base + C::ACC0, tds + acol, by1 + ko, idesc_acc, acc);  // dQ += dS K
-          } else {
-            umma_bf16_ts(tmem_base + C::ACC0, tp + acol, by2 + ko, idesc_acc, acc);   // dV += P^T dO
-            umma_bf16_ts(tmem_base + C::ACC1, tds + acol, by1 + ko, idesc_acc, acc);  // dK += dS^T Q
+          for (int k = 0; k < 4; ++k) {
+            const uint32_t acol = (uint32_t)((k >> 1) * 32 + (k & 1) * 8);
+            umma_bf16_ts(dacc, ta + acol, by + (uint64_t)((k * 2048) >> 4), idesc_acc, k > 0 ? 1u : first);
           }
         }
         umma_commit(bar(BB_YEMPTY + yst));
-        if (it < 100) FS_TRACE(it * 16 + 3);
+        if (side == 0 && it < 100) FS_TRACE(it * 16 + 3);
       }
       if (ok) umma_commit(bar(BB_ACCDONE));
     }
