@@ -2,10 +2,11 @@
 //
 // Forward, one CTA per (128 query rows, head, batch row), two CTAs per SM so that one CTA's softmax overlaps the
 // other's matrix work:
-//   warp 0      TMA producer: Q once, then K/V blocks of 64 keys through a 2-stage ring
-//   warp 1      MMA issuer:   S_j = Q K_j^T (two S buffers in TMEM), O += P_j V_j
-//   warps 2..5  softmax: one query row per thread (TMEM lane = row), P written to shared memory as the next
-//               MMA's A operand, O rescaled in TMEM only when the row's integer reference moves
+//   warp 0      TMA producer: Q once, then K blocks of 64 keys through a 3-stage ring
+//   warp 6      TMA producer: V blocks through a 2-stage ring (V is needed a block later than K)
+//   warp 1      MMA issuer:   S_j = Q K_j^T (two S buffers in TMEM), O += P_j V_j with P read from TMEM
+//   warps 2..5  softmax: one query row per thread (TMEM lane = row), bf16 P written back over the S columns it came
+//               from, O rescaled in TMEM only when the row's integer reference moves
 // The row reference is an integer power of two (ceil of the running maximum in the log2 domain), so rescaling is
 // exact and commutes with the bf16 rounding of P: the result does not depend on the key-block size or order.
 #include <math.h>
@@ -24,23 +25,23 @@ __device__ long long g_trace[8192];
 #else
 #define FS_TRACE(slot) do { } while (0)
 #endif
-constexpr int ATT_THREADS = 192;
 
 // barrier slots of the forward kernel
-enum { B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = 3, B_SFULL = 5, B_SEMPTY = 7, B_PFULL = 9, B_ODONE = 10, B_COUNT = 11 };
+enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 4, B_VFULL = 7, B_VEMPTY = 9, B_SFULL = 11, B_PFULL = 13, B_ODONE = 15,
+       B_COUNT = 16 };
+constexpr int ATT_THREADS = 224;  // K producer, MMA issuer, 4 softmax warps, V producer
 
 template <int D>
 struct FwdCfg {
   static constexpr int BQ = 128, BK = 64, KC = D / 64;
+  static constexpr int NK = 3, NV = 2;  // K is needed one block ahead of V, so it gets the deeper ring
   static constexpr int Q_BYTES = BQ * D * 2;
   static constexpr int KV_BYTES = BK * D * 2;  // one K or one V block
-  static constexpr int P_BYTES = BQ * BK * 2;
   static constexpr int OFF_K = Q_BYTES;
-  static constexpr int OFF_V = OFF_K + 2 * KV_BYTES;
-  static constexpr int OFF_P = OFF_V + 2 * KV_BYTES;
-  static constexpr int OFF_BAR = OFF_P + P_BYTES;
-  static constexpr int SMEM_BYTES = OFF_BAR + 128;
-  static constexpr int TMEM_COLS = 256;  // S0 [0,64) S1 [64,128) O [128, 128+D)
+  static constexpr int OFF_V = OFF_K + NK * KV_BYTES;
+  static constexpr int OFF_BAR = OFF_V + NV * KV_BYTES;
+  static constexpr int SMEM_BYTES = OFF_BAR + 160;
+  static constexpr int TMEM_COLS = 256;  // S0 [0,64) S1 [64,128) (bf16 P overwrites the first 32 columns) O [128, 128+D)
   static constexpr int O_COL = 128;
 };
 
@@ -73,13 +74,20 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
   if (threadIdx.x == 0) {
     mbar_init(bar(B_QFULL), 1);
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(bar(B_KVFULL + i), 1);
-      mbar_init(bar(B_KVEMPTY + i), 1);
-      mbar_init(bar(B_SFULL + i), 1);
-      mbar_init(bar(B_SEMPTY + i), 4);
+    for (int i = 0; i < C::NK; ++i) {
+      mbar_init(bar(B_KFULL + i), 1);
+      mbar_init(bar(B_KEMPTY + i), 1);
     }
-    mbar_init(bar(B_PFULL), 4);
+    for (int i = 0; i < C::NV; ++i) {
+      mbar_init(bar(B_VFULL + i), 1);
+      mbar_init(bar(B_VEMPTY + i), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar(B_SFULL + i), 1);
+      // two P barriers: a softmax warp that does not have to rescale O may run one block ahead of a slower warp, and
+      // its arrival for block j+1 must not be counted for block j
+      mbar_init(bar(B_PFULL + i), 4);
+    }
     mbar_init(bar(B_ODONE), 1);
     *abort_flag = 0;
     mbar_fence_init();
@@ -96,68 +104,79 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
+    // ------------------------------------------------------------------ Q and K producer
     if (lane == 0) {
       mbar_expect_tx(bar(B_QFULL), C::Q_BYTES);
 #pragma unroll
       for (int kc = 0; kc < C::KC; ++kc)
         tma_load_3d(sbase + kc * (C::BQ * 128), &tmQ, bar(B_QFULL), n * D + kc * 64, q0, b);
       for (int j = 0; j < nb; ++j) {
-        const int st = j & 1;
-        if (!mbar_wait(bar(B_KVEMPTY + st), (((uint32_t)j >> 1) & 1u) ^ 1u, abort_flag, err)) break;
-        mbar_expect_tx(bar(B_KVFULL + st), 2 * C::KV_BYTES);
+        const int st = j % C::NK;
+        if (!mbar_wait(bar(B_KEMPTY + st), ((uint32_t)(j / C::NK) & 1u) ^ 1u, abort_flag, err)) break;
+        mbar_expect_tx(bar(B_KFULL + st), C::KV_BYTES);
 #pragma unroll
-        for (int kc = 0; kc < C::KC; ++kc) {
-          tma_load_3d(sbase + C::OFF_K + st * C::KV_BYTES + kc * (C::BK * 128), &tmKV, bar(B_KVFULL + st),
+        for (int kc = 0; kc < C::KC; ++kc)
+          tma_load_3d(sbase + C::OFF_K + st * C::KV_BYTES + kc * (C::BK * 128), &tmKV, bar(B_KFULL + st),
                       hq + kvh * D + kc * 64, j * C::BK, b);
-          tma_load_3d(sbase + C::OFF_V + st * C::KV_BYTES + kc * (C::BK * 128), &tmKV, bar(B_KVFULL + st),
+      }
+    }
+  } else if (warp == 6) {
+    // ------------------------------------------------------------------ V producer
+    if (lane == 0) {
+      for (int j = 0; j < nb; ++j) {
+        const int st = j % C::NV;
+        if (!mbar_wait(bar(B_VEMPTY + st), ((uint32_t)(j / C::NV) & 1u) ^ 1u, abort_flag, err)) break;
+        mbar_expect_tx(bar(B_VFULL + st), C::KV_BYTES);
+#pragma unroll
+        for (int kc = 0; kc < C::KC; ++kc)
+          tma_load_3d(sbase + C::OFF_V + st * C::KV_BYTES + kc * (C::BK * 128), &tmKV, bar(B_VFULL + st),
                       hq + hkv + kvh * D + kc * 64, j * C::BK, b);
-        }
       }
     }
   } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint32_t idesc_base = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(C::BQ >> 4) << 24);
       const uint32_t idesc_s = idesc_base | ((uint32_t)(C::BK >> 3) << 17);            // N = 64 keys, both K-major
       const uint32_t idesc_pv = idesc_base | (1u << 16) | ((uint32_t)(D >> 3) << 17);  // N = D, B (V) mn-major
-      auto issue_s = [&](int j) {
-        const int st = j & 1;
+      const uint64_t dq = umma_desc_sw128(sbase, 0, 1024);
+      // S_j overwrites the TMEM buffer that held P_{j-2}; PV_{j-2} was issued earlier by this thread, so it is ordered
+      auto issue_s = [&](int j) -> bool {
+        const int st = j % C::NK;
+        if (!mbar_wait(bar(B_KFULL + st), (uint32_t)(j / C::NK) & 1u, abort_flag, err)) return false;
+        tc_fence_after();
+        const uint64_t dk = umma_desc_sw128(sbase + C::OFF_K + st * C::KV_BYTES, 0, 1024);
         const uint32_t d_tmem = tmem_base + (uint32_t)((j & 1) * C::BK);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
-          const uint32_t a = sbase + (k >> 2) * (C::BQ * 128) + (k & 3) * 32;
-          const uint32_t bb = sbase + C::OFF_K + st * C::KV_BYTES + (k >> 2) * (C::BK * 128) + (k & 3) * 32;
-          umma_bf16(d_tmem, umma_desc_sw128(a, 0, 1024), umma_desc_sw128(bb, 0, 1024), idesc_s, k > 0 ? 1u : 0u);
+          const uint64_t qo = (uint64_t)(((k >> 2) * (C::BQ * 128) + (k & 3) * 32) >> 4);
+          const uint64_t ko = (uint64_t)(((k >> 2) * (C::BK * 128) + (k & 3) * 32) >> 4);
+          umma_bf16(d_tmem, dq + qo, dk + ko, idesc_s, k > 0 ? 1u : 0u);
         }
         umma_commit(bar(B_SFULL + (j & 1)));
+        umma_commit(bar(B_KEMPTY + st));  // K_j is free as soon as S_j is done
+        return true;
       };
-      bool ok = mbar_wait(bar(B_QFULL), 0, abort_flag, err) && mbar_wait(bar(B_KVFULL), 0, abort_flag, err);
-      if (ok) {
-        tc_fence_after();
-        issue_s(0);
-      }
+      bool ok = mbar_wait(bar(B_QFULL), 0, abort_flag, err);
+      if (ok) ok = issue_s(0);
       for (int j = 0; j < nb && ok; ++j) {
-        if (j + 1 < nb) {
-          const int s1 = (j + 1) & 1;
-          if (!mbar_wait(bar(B_KVFULL + s1), ((uint32_t)(j + 1) >> 1) & 1u, abort_flag, err)) { ok = false; break; }
-          if (!mbar_wait(bar(B_SEMPTY + s1), (((uint32_t)(j + 1) >> 1) & 1u) ^ 1u, abort_flag, err)) { ok = false; break; }
-          tc_fence_after();
-          issue_s(j + 1);
-        }
-        if (!mbar_wait(bar(B_PFULL), (uint32_t)j & 1u, abort_flag, err)) { ok = false; break; }
+        if (j + 1 < nb && !issue_s(j + 1)) { ok = false; break; }
+        const int st = j % C::NV;
+        if (!mbar_wait(bar(B_VFULL + st), (uint32_t)(j / C::NV) & 1u, abort_flag, err)) { ok = false; break; }
+        if (!mbar_wait(bar(B_PFULL + (j & 1)), ((uint32_t)j >> 1) & 1u, abort_flag, err)) { ok = false; break; }
         tc_fence_after();
-        const int st = j & 1;
+        const uint64_t dv = umma_desc_sw128(sbase + C::OFF_V + st * C::KV_BYTES, C::BK * 128, 1024);
+        const uint32_t tp = tmem_base + (uint32_t)((j & 1) * C::BK);  // bf16 P: 16 keys = 8 columns per K step
 #pragma unroll
-        for (int k = 0; k < C::BK / 16; ++k) {
-          const uint32_t a = sbase + C::OFF_P + k * 32;
-          const uint32_t bb = sbase + C::OFF_V + st * C::KV_BYTES + k * 2048;
-          umma_bf16(tmem_base + C::O_COL, umma_desc_sw128(a, 0, 1024), umma_desc_sw128(bb, C::BK * 128, 1024), idesc_pv,
-                    (j > 0 || k > 0) ? 1u : 0u);
-        }
-        umma_commit(bar(B_KVEMPTY + st));
+        for (int k = 0; k < C::BK / 16; ++k)
+          umma_bf16_ts(tmem_base + C::O_COL, tp + (uint32_t)(k * 8), dv + (uint64_t)((k * 2048) >> 4), idesc_pv,
+                       (j > 0 || k > 0) ? 1u : 0u);
+        umma_commit(bar(B_VEMPTY + st));
         umma_commit(bar(B_ODONE));
       }
     }
   } else {
+    // ------------------------------------------------------------------ softmax warps (2..5)
     const int q = warp & 3;
     const int rloc = q * 32 + lane;  // row within the tile = TMEM lane
     const int row = q0 + rloc;
@@ -173,9 +192,6 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       tmem_ld32(tlane + (uint32_t)((j & 1) * C::BK), r0);
       tmem_ld32(tlane + (uint32_t)((j & 1) * C::BK + 32), r1);
       tmem_ld_wait();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(B_SEMPTY + (j & 1)));
 
       const int k0 = j * C::BK;
       const bool need_mask = k0 + C::BK - 1 > q0 + q * 32;  // warp-uniform
@@ -193,52 +209,49 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       const float mnew = fmaxf(mref, ceilf(mx * scale_log2));
       const float alpha = fast_exp2(mref - mnew);  // exact power of two; 0 on the first block
       float psum = 0.f;
+      uint32_t pw[32];  // bf16 pairs: keys 2c, 2c+1 in word c
 #pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        const float a = fast_exp2(fmaf(__uint_as_float(r0[i]), scale_log2, -mnew));
-        const float c = fast_exp2(fmaf(__uint_as_float(r1[i]), scale_log2, -mnew));
-        psum += a + c;
-        r0[i] = __float_as_uint(a);
-        r1[i] = __float_as_uint(c);
+      for (int i = 0; i < 32; i += 2) {
+        const float a0 = fast_exp2(fmaf(__uint_as_float(r0[i]), scale_log2, -mnew));
+        const float a1 = fast_exp2(fmaf(__uint_as_float(r0[i + 1]), scale_log2, -mnew));
+        const float c0 = fast_exp2(fmaf(__uint_as_float(r1[i]), scale_log2, -mnew));
+        const float c1 = fast_exp2(fmaf(__uint_as_float(r1[i + 1]), scale_log2, -mnew));
+        psum += (a0 + a1) + (c0 + c1);
+        pw[i >> 1] = pack_bf16(a0, a1);
+        pw[16 + (i >> 1)] = pack_bf16(c0, c1);
       }
       lsum = lsum * alpha + psum;
       mref = mnew;
 
-      if (j > 0) {
-        // P_{j-1} has been consumed and O holds blocks 0..j-1: both needed before touching P or O
+      // O has to be rescaled only when this row's integer reference moved (rare after the first blocks); only then
+      // does the softmax wait for the previous P V product
+      if (j > 0 && __any_sync(0xffffffffu, alpha != 1.0f)) {
         ok = mbar_wait(bar(B_ODONE), (uint32_t)(j - 1) & 1u, abort_flag, err);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        if (__any_sync(0xffffffffu, alpha != 1.0f)) {
 #pragma unroll 1
-          for (int c = 0; c < D; c += 32) {
-            uint32_t t[32];
-            tmem_ld32(tlane + (uint32_t)(C::O_COL + c), t);
-            tmem_ld_wait();
+        for (int c = 0; c < D; c += 32) {
+          uint32_t t[32];
+          tmem_ld32(tlane + (uint32_t)(C::O_COL + c), t);
+          tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) t[i] = __float_as_uint(__uint_as_float(t[i]) * alpha);
-            tmem_st32(tlane + (uint32_t)(C::O_COL + c), t);
-          }
-          tmem_st_wait();
+          for (int i = 0; i < 32; ++i) t[i] = __float_as_uint(__uint_as_float(t[i]) * alpha);
+          tmem_st32(tlane + (uint32_t)(C::O_COL + c), t);
         }
       }
-      // P (bf16) into the 128-byte-swizzled K-major tile [128 rows x 64 keys]
-      uint8_t* prow = smem + C::OFF_P + rloc * 128;
-#pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        const uint32_t* src = c < 4 ? &r0[c * 8] : &r1[(c - 4) * 8];
-        uint4 v;
-        v.x = pack_bf16(__uint_as_float(src[0]), __uint_as_float(src[1]));
-        v.y = pack_bf16(__uint_as_float(src[2]), __uint_as_float(src[3]));
-        v.z = pack_bf16(__uint_as_float(src[4]), __uint_as_float(src[5]));
-        v.w = pack_bf16(__uint_as_float(src[6]), __uint_as_float(src[7]));
-        *reinterpret_cast<uint4*>(prow + ((c ^ (rloc & 7)) << 4)) = v;
-      }
-      fence_proxy_async_smem();
+      // bf16 P back into TMEM over the first 32 of the 64 fp32 columns it was computed from
+      tmem_st32(tlane + (uint32_t)((j & 1) * C::BK), pw);
+      tmem_st_wait();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(B_PFULL));
+      if (lane == 0) mbar_arrive(bar(B_PFULL + (j & 1)));
+    }
+    // A parity wait can only tell two consecutive phases apart.  Seeing S_j guarantees P V products up to block j-2
+    // (they were issued before S_j), so after the last block the products nb-2 and nb-1 are waited for in turn.
+    if (ok && nb >= 2) {
+      ok = mbar_wait(bar(B_ODONE), (uint32_t)(nb - 2) & 1u, abort_flag, err);
+      ok = __all_sync(0xffffffffu, ok);
     }
     if (ok) {
       ok = mbar_wait(bar(B_ODONE), (uint32_t)(nb - 1) & 1u, abort_flag, err);
