@@ -218,6 +218,7 @@ def run_cuda(args):
     clocks = sampler.stop()
     launches = model.launch_count - launches0
     prof = model.get_profile()
+    gemm_shapes = model.get_gemm_profile()
     model.set_profiling(False)
     loss_check = model.forward_loss(*dev_batches[0])
 
@@ -276,6 +277,8 @@ def run_cuda(args):
             "e2e": {"value": world * tokens_per_step / (ms_e2e / 1e3 / args.steps), "unit": "tokens/s",
                     "h2d_bytes_per_step": 2 * tokens_per_step * 4, "d2h_bytes_per_step": 64,
                     "ms_per_step": ms_e2e / args.steps, "last_loss": e2e_loss},
+            "gemm_shapes": [dict(g, ms_per_step=g["ms"] / args.steps, launches_per_step=g["launches"] / args.steps)
+                            for g in sorted(gemm_shapes, key=lambda g: -g["ms"])],
             "gpu_launches": launches, "clocks": clocks, "loss_after_run": loss_check,
         }
         if world == 1 and not args.no_cpu_baseline:

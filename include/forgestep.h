@@ -107,6 +107,9 @@ typedef enum {
 } ft_prof_class;
 ft_status ft_set_profiling(ft_model* m, int32_t enable);
 ft_status ft_get_profile(ft_model* m, int32_t cls, double* ms, double* work, int64_t* launches);
+/* The GEMM class broken down by (M, N, K, a_mn, b_mn, epilogue): entry i of the table built while profiling was on;
+ * FT_ENOTFOUND past the end.  shape = {M, N, K, a_mn, b_mn, epilogue kind}. */
+ft_status ft_get_gemm_profile(ft_model* m, int32_t i, int32_t shape[6], double* ms, int64_t* launches);
 
 /* Development switch: force the GEMM tile width (128 or 256 columns); 0 = choose by tile count (default). */
 void ft_debug_gemm_tile(int32_t bn);

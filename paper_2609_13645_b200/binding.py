@@ -72,6 +72,8 @@ def lib():
         L.ft_debug_gemm_tile.restype = None
         L.ft_debug_gemm_pairs.argtypes = [i32]
         L.ft_debug_gemm_pairs.restype = None
+        L.ft_get_gemm_profile.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(C.c_double), C.POINTER(i64)]
+        L.ft_get_gemm_profile.restype = C.c_int
         L.ft_destroy.restype = None
         L.ft_destroy.argtypes = [vp]
         L.ft_k_gemm.argtypes = [vp, i32, i64, vp, i32, i64, vp, i64, vp, i32, i32, i32, i32, vp, vp]
@@ -232,6 +234,21 @@ class Model:
             ms, work, n = C.c_double(), C.c_double(), C.c_int64()
             self._check(lib().ft_get_profile(self._h, cls, C.byref(ms), C.byref(work), C.byref(n)))
             out[name] = dict(ms=ms.value, work=work.value, launches=int(n.value))
+        return out
+
+    def get_gemm_profile(self):
+        """List of dicts (M, N, K, a_mn, b_mn, epi, ms, launches, tflops) for every GEMM shape seen while profiling."""
+        out, i = [], 0
+        while True:
+            shp, ms, n = (C.c_int32 * 6)(), C.c_double(), C.c_int64()
+            st = lib().ft_get_gemm_profile(self._h, i, shp, C.byref(ms), C.byref(n))
+            if st == FT_ENOTFOUND:
+                break
+            self._check(st)
+            M, N, K = shp[0], shp[1], shp[2]
+            out.append(dict(M=M, N=N, K=K, a_mn=shp[3], b_mn=shp[4], epi=shp[5], ms=ms.value, launches=int(n.value),
+                            tflops=2.0 * M * N * K * n.value / (ms.value * 1e-3) / 1e12 if ms.value > 0 else 0.0))
+            i += 1
         return out
 
     @property

@@ -130,7 +130,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, uint32_t taddr, 
         for (int j = 0; j < 16; ++j) {
           g[j] = round_bf16(__uint_as_float(r[j]));
           u[j] = round_bf16(__uint_as_float(r[16 + j]));
-          a[j] = g[j] / (1.0f + __expf(-g[j])) * u[j];
+          a[j] = __fdividef(g[j], 1.0f + __expf(-g[j])) * u[j];
         }
         store8_bf16(gurow + lc, g);
         store8_bf16(gurow + lc + 8, g + 8);
@@ -140,6 +140,71 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, uint32_t taddr, 
         store8_bf16(arow + lc + 8, a + 8);
       }
     }
+  } else if (p.epi == EPI_BF16_RESID) {
+    // the residual row is read one 32-column chunk ahead of the accumulator it is added to, so its latency overlaps
+    // the TMEM load and the stores of the previous chunk
+    bf16* crow = reinterpret_cast<bf16*>(p.C) + (long long)row * p.ldc;
+    const bf16* rrow = p.resid + (long long)row * p.ldc;
+    uint4 nxt[4];
+    auto fetch = [&](int gc) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        nxt[j] = (row_ok && gc + 8 * j < p.N) ? *reinterpret_cast<const uint4*>(rrow + gc + 8 * j) : make_uint4(0, 0, 0, 0);
+    };
+    fetch(n0);
+    for (int c = 0; c < BN; c += 32) {
+      const int gc = n0 + c;
+      if (gc >= p.N) break;
+      uint4 cur[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) cur[j] = nxt[j];
+      if (c + 32 < BN) fetch(gc + 32);
+      tmem_ld32(taddr + c, r);
+      tmem_ld_wait();
+      if (row_ok) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          if (gc + 8 * j < p.N) {
+            float v[8];
+            v[0] = __uint_as_float(r[8 * j + 0]) + bf16_lo(cur[j].x); v[1] = __uint_as_float(r[8 * j + 1]) + bf16_hi(cur[j].x);
+            v[2] = __uint_as_float(r[8 * j + 2]) + bf16_lo(cur[j].y); v[3] = __uint_as_float(r[8 * j + 3]) + bf16_hi(cur[j].y);
+            v[4] = __uint_as_float(r[8 * j + 4]) + bf16_lo(cur[j].z); v[5] = __uint_as_float(r[8 * j + 5]) + bf16_hi(cur[j].z);
+            v[6] = __uint_as_float(r[8 * j + 6]) + bf16_lo(cur[j].w); v[7] = __uint_as_float(r[8 * j + 7]) + bf16_hi(cur[j].w);
+            store8_bf16(crow + gc + 8 * j, v);
+          }
+        }
+      }
+    }
+  } else if (p.epi == EPI_F32_ACC) {
+    float* crow = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc;
+    float4 nxt[8];
+    auto fetch = [&](int gc) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        nxt[j] = (row_ok && gc + 4 * j < p.N) ? *reinterpret_cast<const float4*>(crow + gc + 4 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
+    };
+    fetch(n0);
+    for (int c = 0; c < BN; c += 32) {
+      const int gc = n0 + c;
+      if (gc >= p.N) break;
+      float4 cur[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) cur[j] = nxt[j];
+      if (c + 32 < BN) fetch(gc + 32);
+      tmem_ld32(taddr + c, r);
+      tmem_ld_wait();
+      if (row_ok) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          if (gc + 4 * j < p.N) {
+            float4 o = cur[j];
+            o.x += __uint_as_float(r[4 * j + 0]); o.y += __uint_as_float(r[4 * j + 1]);
+            o.z += __uint_as_float(r[4 * j + 2]); o.w += __uint_as_float(r[4 * j + 3]);
+            *reinterpret_cast<float4*>(crow + gc + 4 * j) = o;
+          }
+        }
+      }
+    }
   } else {
     for (int c = 0; c < BN; c += 32) {
       const int gc = n0 + c;
@@ -147,37 +212,24 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, uint32_t taddr, 
       tmem_ld32(taddr + c, r);
       tmem_ld_wait();
       if (row_ok) {
-        float v[32];
-#pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-        if (p.epi == EPI_BF16 || p.epi == EPI_BF16_RESID) {
+        if (p.epi == EPI_BF16) {
           bf16* crow = reinterpret_cast<bf16*>(p.C) + (long long)row * p.ldc + gc;
-          const bf16* rrow = p.resid + (long long)row * p.ldc + gc;
 #pragma unroll
           for (int j = 0; j < 32; j += 8) {
             if (gc + j < p.N) {
-              if (p.epi == EPI_BF16_RESID) {
-                const uint4 x = *reinterpret_cast<const uint4*>(rrow + j);
-                v[j + 0] += bf16_lo(x.x); v[j + 1] += bf16_hi(x.x);
-                v[j + 2] += bf16_lo(x.y); v[j + 3] += bf16_hi(x.y);
-                v[j + 4] += bf16_lo(x.z); v[j + 5] += bf16_hi(x.z);
-                v[j + 6] += bf16_lo(x.w); v[j + 7] += bf16_hi(x.w);
-              }
-              store8_bf16(crow + j, v + j);
+              float v[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(r[j + e]);
+              store8_bf16(crow + j, v);
             }
           }
         } else {
           float* crow = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + gc;
 #pragma unroll
           for (int j = 0; j < 32; j += 4) {
-            if (gc + j < p.N) {
-              float4 o = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-              if (p.epi == EPI_F32_ACC) {
-                const float4 x = *reinterpret_cast<const float4*>(crow + j);
-                o.x += x.x; o.y += x.y; o.z += x.z; o.w += x.w;
-              }
-              *reinterpret_cast<float4*>(crow + j) = o;
-            }
+            if (gc + j < p.N)
+              *reinterpret_cast<float4*>(crow + j) = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
+                                                                 __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
           }
         }
       }

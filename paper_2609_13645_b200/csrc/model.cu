@@ -81,7 +81,9 @@ struct ft_model {
   bool have_bwd = false;
 
   // optional per-class timing with CUDA events on the model's stream
-  struct ProfRec { cudaEvent_t a, b; int cls; double work; };
+  struct ProfRec { cudaEvent_t a, b; int cls; double work; int shape; };
+  struct GemmShape { int M, N, K, a_mn, b_mn, epi; double ms; long long launches; };
+  std::vector<GemmShape> prof_shapes;
   bool prof = false;
   std::vector<ProfRec> prof_pending;
   std::vector<cudaEvent_t> prof_pool;
@@ -117,8 +119,9 @@ bool valid_config(const ft_config* c, std::string* why) {
 
 int pick_ce_chunk(const ft_config* c) {
   const long long T = (long long)c->max_batch * c->max_seq;
-  long long rows = 2048;
-  while (rows > 128 && rows * (long long)c->vocab * 6 > (3ll << 30)) rows >>= 1;  // logits + dlogits scratch <= 3 GiB
+  // larger chunks mean fewer read-modify-write passes over the fp32 head gradient; logits + dlogits scratch <= 2 GiB
+  long long rows = 4096;
+  while (rows > 128 && rows * (long long)c->vocab * 6 > (2ll << 30)) rows >>= 1;
   if (rows > T) rows = (T + 7) / 8 * 8;
   return (int)rows;
 }
@@ -227,7 +230,7 @@ ft_status cuda_fail(ft_model* m, cudaError_t e, const char* where) {
     cudaError_t e__ = launch_gemm(args, m->stream);                                         \
     if (e__ != cudaSuccess) return cuda_fail(m, e__, "launch_gemm");                        \
     m->launches += 1;                                                                       \
-    prof_end(m, FT_PROF_GEMM, 2.0 * (double)(args).M * (double)(args).N * (double)(args).K, 1); \
+    prof_end(m, FT_PROF_GEMM, 2.0 * (double)(args).M * (double)(args).N * (double)(args).K, 1, prof_shape_index(m, args)); \
   } while (0)
 
 cudaEvent_t prof_event(ft_model* m) {
@@ -241,10 +244,10 @@ inline void prof_begin(ft_model* m) {
   m->prof_cur = prof_event(m);
   cudaEventRecord(m->prof_cur, m->stream);
 }
-inline void prof_end(ft_model* m, int cls, double work, int launches) {
+inline void prof_end(ft_model* m, int cls, double work, int launches, int shape = -1) {
   if (!m->prof || !m->prof_cur) return;
   ft_model::ProfRec r;
-  r.a = m->prof_cur; r.b = prof_event(m); r.cls = cls; r.work = work;
+  r.a = m->prof_cur; r.b = prof_event(m); r.cls = cls; r.work = work; r.shape = shape;
   cudaEventRecord(r.b, m->stream);
   m->prof_pending.push_back(r);
   m->prof_launches[cls] += launches;
@@ -254,11 +257,27 @@ inline void prof_end(ft_model* m, int cls, double work, int launches) {
 void prof_collect(ft_model* m) {
   for (auto& r : m->prof_pending) {
     float ms = 0.f;
-    if (cudaEventElapsedTime(&ms, r.a, r.b) == cudaSuccess) { m->prof_ms[r.cls] += ms; m->prof_work[r.cls] += r.work; }
+    if (cudaEventElapsedTime(&ms, r.a, r.b) == cudaSuccess) {
+      m->prof_ms[r.cls] += ms;
+      m->prof_work[r.cls] += r.work;
+      if (r.shape >= 0) { m->prof_shapes[r.shape].ms += ms; m->prof_shapes[r.shape].launches += 1; }
+    }
     m->prof_pool.push_back(r.a);
     m->prof_pool.push_back(r.b);
   }
   m->prof_pending.clear();
+}
+
+// index of this GEMM's (shape, layout, epilogue) in the per-shape profile table
+int prof_shape_index(ft_model* m, const GemmArgs& g) {
+  if (!m->prof) return -1;
+  for (size_t i = 0; i < m->prof_shapes.size(); ++i) {
+    const auto& s = m->prof_shapes[i];
+    if (s.M == g.M && s.N == g.N && s.K == g.K && s.a_mn == g.a_mn && s.b_mn == g.b_mn && s.epi == g.epi) return (int)i;
+  }
+  ft_model::GemmShape s = {g.M, g.N, g.K, g.a_mn, g.b_mn, g.epi, 0.0, 0};
+  m->prof_shapes.push_back(s);
+  return (int)m->prof_shapes.size() - 1;
 }
 
 AdamHyper hyper(const ft_model* m) {
@@ -747,6 +766,7 @@ ft_status ft_set_profiling(ft_model* m, int32_t enable) {
   m->prof = enable != 0;
   if (enable) {
     for (int c = 0; c < FT_PROF_CLASSES; ++c) { m->prof_ms[c] = 0; m->prof_work[c] = 0; m->prof_launches[c] = 0; }
+    m->prof_shapes.clear();
   }
   return FT_OK;
 }
@@ -763,6 +783,18 @@ ft_status ft_get_profile(ft_model* m, int32_t cls, double* ms, double* work, int
 
 void ft_debug_gemm_tile(int32_t bn) { g_gemm_force_bn = bn; }
 void ft_debug_gemm_pairs(int32_t on) { g_gemm_pairs = on; }
+
+ft_status ft_get_gemm_profile(ft_model* m, int32_t i, int32_t shape[6], double* ms, int64_t* launches) {
+  if (!m || !shape) return FT_EINVAL;
+  FT_CUDA(cudaStreamSynchronize(m->stream));
+  prof_collect(m);
+  if (i < 0 || i >= (int32_t)m->prof_shapes.size()) return FT_ENOTFOUND;
+  const auto& s = m->prof_shapes[i];
+  shape[0] = s.M; shape[1] = s.N; shape[2] = s.K; shape[3] = s.a_mn; shape[4] = s.b_mn; shape[5] = s.epi;
+  if (ms) *ms = s.ms;
+  if (launches) *launches = s.launches;
+  return FT_OK;
+}
 
 const char* ft_last_error(const ft_model* m) { return m ? m->err.c_str() : "null model"; }
 int64_t ft_launch_count(const ft_model* m) { return m ? m->launches : 0; }

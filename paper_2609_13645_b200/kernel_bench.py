@@ -35,6 +35,7 @@ def main():
     ap.add_argument("--iters", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--no-flush", action="store_true")
+    ap.add_argument("--out", default="auto", choices=["auto", "bf16", "resid", "f32", "f32acc"], help="GEMM epilogue")
     ap.add_argument("--bn", type=int, default=0, help="force the GEMM tile width (development)")
     ap.add_argument("--pairs", type=int, default=1, help="0: single-CTA GEMM kernel only (development)")
     a = ap.parse_args()
@@ -57,9 +58,15 @@ def main():
         else:
             A = torch.randn(K, M, device=dev).bfloat16(); Bm = torch.randn(K, N, device=dev).bfloat16()
             out = torch.empty(M, N, dtype=torch.float32, device=dev); amn, bmn, kind = 1, 1, 2
+        resid = None
+        if a.out != "auto":
+            kind = {"bf16": 0, "resid": 1, "f32": 2, "f32acc": 3}[a.out]
+            out = torch.zeros(M, N, dtype=torch.bfloat16 if kind < 2 else torch.float32, device=dev)
+            if kind == 1:
+                resid = torch.randn(M, N, device=dev).bfloat16()
         flops = 2.0 * M * N * K
-        run = lambda: B.k_gemm(A, amn, Bm, bmn, out, kind, M, N, K, err)
-        desc = dict(kernel="gemm", layout=a.layout, M=M, N=N, K=K)
+        run = lambda: B.k_gemm(A, amn, Bm, bmn, out, kind, M, N, K, err, resid)
+        desc = dict(kernel="gemm", layout=a.layout, out=a.out, M=M, N=N, K=K)
     else:
         Bsz, S, nh, nkv, d = a.B, a.S, a.nh, a.nkv, a.d
         qkv = torch.randn(Bsz * S, (nh + 2 * nkv) * d, device=dev).bfloat16()
