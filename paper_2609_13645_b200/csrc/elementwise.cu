@@ -536,7 +536,7 @@ inline int ok(int launches) { return cudaGetLastError() == cudaSuccess ? launche
 
 int elementwise_blocks_for_norm(int T) {
   const int need = (T + 7) / 8;
-  return need < 148 ? need : 148;  // one resident CTA per SM (register-bound)
+  return need < 296 ? need : 296;  // two resident CTAs per SM
 }
 
 size_t sort_pad(size_t n) {
@@ -568,14 +568,15 @@ int rmsnorm_bwd(const bf16* dy, const bf16* x, const float* r, const bf16* g, co
   const int nblk = elementwise_blocks_for_norm(T);
   const int nch = h >> 8;
 #define FS_NORM_CASE(N, W) launch_rmsnorm_bwd<N, W>(nblk, dy, x, r, g, resid, dx, partial, T, h, st); break
-  if (nch <= 8) {
+  if (nch <= 4) {
     switch (nch) {
       case 1: FS_NORM_CASE(1, 1); case 2: FS_NORM_CASE(2, 1); case 3: FS_NORM_CASE(3, 1); case 4: FS_NORM_CASE(4, 1);
-      case 5: FS_NORM_CASE(5, 1); case 6: FS_NORM_CASE(6, 1); case 7: FS_NORM_CASE(7, 1); default: FS_NORM_CASE(8, 1);
+      default: FS_NORM_CASE(4, 1);
     }
   } else {
+    // two warps per row from h = 1280 up: half the registers per thread, so two CTAs fit on an SM
     switch ((nch + 1) / 2) {
-      case 5: FS_NORM_CASE(5, 2); case 6: FS_NORM_CASE(6, 2); case 7: FS_NORM_CASE(7, 2); default: FS_NORM_CASE(8, 2);
+      case 3: FS_NORM_CASE(3, 2); case 4: FS_NORM_CASE(4, 2); case 5: FS_NORM_CASE(5, 2); case 6: FS_NORM_CASE(6, 2); case 7: FS_NORM_CASE(7, 2); default: FS_NORM_CASE(8, 2);
     }
   }
 #undef FS_NORM_CASE
