@@ -65,6 +65,13 @@ ft_status ft_init_model(const ft_config* cfg, uint64_t seed, void* dev_workspace
 ft_status ft_train_step(ft_model* m, const int32_t* dev_tokens, const int32_t* dev_labels, int32_t B, int32_t S,
                         float* host_loss, float* host_gnorm);
 
+/* Whole-step CUDA graph (the paper's full-step graph capture): when enabled, the first ft_train_step of a (B, S)
+ * runs launch by launch, the second is captured into a graph, later ones replay it (ids are first copied into the
+ * model's own buffers).  Needs a capturable stream (not the legacy default stream; otherwise it switches itself
+ * off); not used while profiling or with debug_taps.  ft_graph_replays counts the replays so far. */
+ft_status ft_set_graph(ft_model* m, int32_t enable);
+int64_t ft_graph_replays(const ft_model* m);
+
 /* Same call with HOST token and label arrays: copies them to the device, runs the step, returns the loss. */
 ft_status ft_train_step_host(ft_model* m, const int32_t* host_tokens, const int32_t* host_labels, int32_t B,
                              int32_t S, float* host_loss, float* host_gnorm);

@@ -74,6 +74,10 @@ def lib():
         L.ft_debug_gemm_pairs.restype = None
         L.ft_get_gemm_profile.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(C.c_double), C.POINTER(i64)]
         L.ft_get_gemm_profile.restype = C.c_int
+        L.ft_set_graph.argtypes = [vp, i32]
+        L.ft_set_graph.restype = C.c_int
+        L.ft_graph_replays.argtypes = [vp]
+        L.ft_graph_replays.restype = i64
         L.ft_destroy.restype = None
         L.ft_destroy.argtypes = [vp]
         L.ft_k_gemm.argtypes = [vp, i32, i64, vp, i32, i64, vp, i64, vp, i32, i32, i32, i32, vp, vp]
@@ -223,6 +227,14 @@ class Model:
         self._check(lib().ft_get_tap(self._h, name.encode(), layer, C.c_void_p(buf.ctypes.data), buf.nbytes,
                                      C.byref(need), C.byref(dt)))
         return buf.view(np.float32).copy() if dt.value == 1 else bf16_bits_to_f32(buf.view(np.uint16))
+
+    def set_graph(self, enable: bool):
+        """Capture the whole step into a CUDA graph on its second run and replay it afterwards."""
+        self._check(lib().ft_set_graph(self._h, 1 if enable else 0))
+
+    @property
+    def graph_replays(self) -> int:
+        return int(lib().ft_graph_replays(self._h))
 
     def set_profiling(self, enable: bool):
         self._check(lib().ft_set_profiling(self._h, 1 if enable else 0))

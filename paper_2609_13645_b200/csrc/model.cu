@@ -80,6 +80,13 @@ struct ft_model {
   int lastB = 0, lastS = 0;
   bool have_bwd = false;
 
+  // whole-step CUDA graph: the first step of a (B, S) runs launch by launch, the second is captured, later ones replay
+  bool graph_enabled = false;
+  int graph_B = 0, graph_S = 0, warm_B = 0, warm_S = 0;
+  cudaGraphExec_t graph_exec = nullptr;
+  int64_t graph_launches = 0;
+  int64_t graph_replays = 0;
+
   // optional per-class timing with CUDA events on the model's stream
   struct ProfRec { cudaEvent_t a, b; int cls; double work; int shape; };
   struct GemmShape { int M, N, K, a_mn, b_mn, epi; double ms; long long launches; };
@@ -490,6 +497,14 @@ ft_status finish(ft_model* m, float* host_loss, float* host_gnorm) {
   return FT_OK;
 }
 
+// Host <-> device copy ordered on the model's stream and finished on return.  (A plain cudaMemcpy from pageable host
+// memory may return while the DMA is still in flight, and is only ordered against the legacy default stream.)
+cudaError_t copy_sync(ft_model* m, void* dst, const void* src, size_t bytes, cudaMemcpyKind kind) {
+  cudaError_t e = cudaMemcpyAsync(dst, src, bytes, kind, m->stream);
+  if (e != cudaSuccess) return e;
+  return cudaStreamSynchronize(m->stream);
+}
+
 // wgu rows: logical (gate 0..f-1, up 0..f-1) <-> physical (16 gate rows, 16 up rows, alternating)
 inline int64_t wgu_phys_row(int64_t r, int64_t f) {
   const int64_t i = r < f ? r : r - f;
@@ -585,15 +600,80 @@ ft_status ft_init_model(const ft_config* cfg, uint64_t seed, void* dev_workspace
   return FT_OK;
 }
 
+// One full step enqueued launch by launch.
+static ft_status step_direct(ft_model* m, const int32_t* tok, const int32_t* lab, int32_t B, int32_t S) {
+  ft_status s = run_forward_backward(m, tok, lab, B, S, true);
+  if (s) return s;
+  return run_update(m);
+}
+
+// The same step through a captured graph when that is enabled and possible.  The graph reads the token and label
+// ids from the model's own buffers (the caller's pointers may change from step to step), every other address in
+// it is fixed, and the optimizer scalars it needs live in device memory, so a replay needs no host value.
+static ft_status step_maybe_graphed(ft_model* m, const int32_t* tok, const int32_t* lab, int32_t B, int32_t S) {
+  if (!m->graph_enabled || m->prof || m->cfg.debug_taps) return step_direct(m, tok, lab, B, S);
+  if (B < 1 || S < 1 || B > m->cfg.max_batch || S > m->cfg.max_seq) return fail(m, FT_EINVAL, "B or S out of range");
+  if (!tok || !lab) return fail(m, FT_EINVAL, "null argument");
+  if (!(m->graph_exec && m->graph_B == B && m->graph_S == S)) {
+    if (!(m->warm_B == B && m->warm_S == S)) {  // first step of this shape: plain launches (one-time kernel set-up)
+      m->warm_B = B; m->warm_S = S;
+      return step_direct(m, tok, lab, B, S);
+    }
+    if (m->graph_exec) { cudaGraphExecDestroy(m->graph_exec); m->graph_exec = nullptr; }
+    if (cudaStreamBeginCapture(m->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+      cudaGetLastError();          // e.g. the legacy default stream cannot be captured: keep working without a graph
+      m->graph_enabled = false;
+      return step_direct(m, tok, lab, B, S);
+    }
+    const int64_t before = m->launches;
+    ft_status s = step_direct(m, m->tok_dev, m->lab_dev, B, S);
+    cudaGraph_t graph = nullptr;
+    cudaError_t e = cudaStreamEndCapture(m->stream, &graph);
+    m->graph_launches = m->launches - before;
+    m->launches = before;  // nothing ran yet
+    if (s != FT_OK || e != cudaSuccess || !graph) {
+      if (graph) cudaGraphDestroy(graph);
+      cudaGetLastError();
+      m->graph_enabled = false;
+      if (s != FT_OK) return s;
+      return step_direct(m, tok, lab, B, S);
+    }
+    e = cudaGraphInstantiate(&m->graph_exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (e != cudaSuccess) {
+      m->graph_exec = nullptr;
+      m->graph_enabled = false;
+      return step_direct(m, tok, lab, B, S);
+    }
+    m->graph_B = B; m->graph_S = S;
+  }
+  const size_t bytes = (size_t)B * S * sizeof(int32_t);
+  if (tok != m->tok_dev) FT_CUDA(cudaMemcpyAsync(m->tok_dev, tok, bytes, cudaMemcpyDeviceToDevice, m->stream));
+  if (lab != m->lab_dev) FT_CUDA(cudaMemcpyAsync(m->lab_dev, lab, bytes, cudaMemcpyDeviceToDevice, m->stream));
+  FT_CUDA(cudaGraphLaunch(m->graph_exec, m->stream));
+  m->launches += m->graph_launches;
+  m->graph_replays += 1;
+  m->lastB = B; m->lastS = S; m->have_bwd = true;
+  return FT_OK;
+}
+
 ft_status ft_train_step(ft_model* m, const int32_t* dev_tokens, const int32_t* dev_labels, int32_t B, int32_t S,
                         float* host_loss, float* host_gnorm) {
   if (!m) return FT_EINVAL;
-  ft_status s = run_forward_backward(m, dev_tokens, dev_labels, B, S, true);
+  ft_status s = step_maybe_graphed(m, dev_tokens, dev_labels, B, S);
   if (s) return s;
-  if ((s = run_update(m))) return s;
   if (host_loss || host_gnorm) return finish(m, host_loss, host_gnorm);
   return FT_OK;
 }
+
+ft_status ft_set_graph(ft_model* m, int32_t enable) {
+  if (!m) return FT_EINVAL;
+  m->graph_enabled = enable != 0;
+  if (!enable && m->graph_exec) { cudaGraphExecDestroy(m->graph_exec); m->graph_exec = nullptr; }
+  return FT_OK;
+}
+
+int64_t ft_graph_replays(const ft_model* m) { return m ? m->graph_replays : 0; }
 
 ft_status ft_train_step_host(ft_model* m, const int32_t* host_tokens, const int32_t* host_labels, int32_t B, int32_t S,
                              float* host_loss, float* host_gnorm) {
@@ -653,16 +733,16 @@ static ft_status param_copy(ft_model* m, int32_t i, ft_kind kind, void* host, si
   uint8_t* hp = reinterpret_cast<uint8_t*>(host);
   FT_CUDA(cudaStreamSynchronize(m->stream));
   if (!p.is_wgu) {
-    if (to_host) FT_CUDA(cudaMemcpy(hp, dev, bytes, cudaMemcpyDeviceToHost));
-    else FT_CUDA(cudaMemcpy(dev, hp, bytes, cudaMemcpyHostToDevice));
+    if (to_host) FT_CUDA(copy_sync(m, hp, dev, bytes, cudaMemcpyDeviceToHost));
+    else FT_CUDA(copy_sync(m, dev, hp, bytes, cudaMemcpyHostToDevice));
   } else {
     // 16-row blocks of the logical tensor sit at their physical (interleaved) place
     const size_t blk = 16 * (size_t)p.cols * es;
     for (int64_t r0 = 0; r0 < p.rows; r0 += 16) {
       uint8_t* d = dev + (size_t)wgu_phys_row(r0, m->f) * p.cols * es;
       uint8_t* hrow = hp + (size_t)r0 * p.cols * es;
-      if (to_host) FT_CUDA(cudaMemcpy(hrow, d, blk, cudaMemcpyDeviceToHost));
-      else FT_CUDA(cudaMemcpy(d, hrow, blk, cudaMemcpyHostToDevice));
+      if (to_host) FT_CUDA(copy_sync(m, hrow, d, blk, cudaMemcpyDeviceToHost));
+      else FT_CUDA(copy_sync(m, d, hrow, blk, cudaMemcpyHostToDevice));
     }
   }
   if (!to_host && kind == FT_MASTER_F32) {
@@ -685,7 +765,7 @@ ft_status ft_get_step(const ft_model* mc, int64_t* step) {
   if (!m || !step) return FT_EINVAL;
   long long s = 0;
   FT_CUDA(cudaStreamSynchronize(m->stream));
-  FT_CUDA(cudaMemcpy(&s, &m->sc->step, sizeof(s), cudaMemcpyDeviceToHost));
+  FT_CUDA(copy_sync(m, &s, &m->sc->step, sizeof(s), cudaMemcpyDeviceToHost));
   *step = s;
   return FT_OK;
 }
@@ -694,7 +774,7 @@ ft_status ft_set_step(ft_model* m, int64_t step) {
   if (!m || step < 0) return FT_EINVAL;
   long long s = step;
   FT_CUDA(cudaStreamSynchronize(m->stream));
-  FT_CUDA(cudaMemcpy(&m->sc->step, &s, sizeof(s), cudaMemcpyHostToDevice));
+  FT_CUDA(copy_sync(m, &m->sc->step, &s, sizeof(s), cudaMemcpyHostToDevice));
   return FT_OK;
 }
 
@@ -745,7 +825,7 @@ ft_status ft_get_tap(ft_model* m, const char* name, int32_t layer, void* host_ds
   if (dtype) *dtype = dt;
   if (bytes < nbytes) return fail(m, FT_EINVAL, "destination too small");
   FT_CUDA(cudaStreamSynchronize(m->stream));
-  FT_CUDA(cudaMemcpy(host_dst, src, nbytes, cudaMemcpyDeviceToHost));
+  FT_CUDA(copy_sync(m, host_dst, src, nbytes, cudaMemcpyDeviceToHost));
   if (nm == "d_gu") {
     // undo the physical interleave: [T, 2f] columns back to gate | up
     std::vector<uint16_t> tmp(2 * f);
@@ -802,6 +882,7 @@ void ft_destroy(ft_model* m) {
   if (!m) return;
   for (auto& r : m->prof_pending) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
   for (auto e : m->prof_pool) cudaEventDestroy(e);
+  if (m->graph_exec) cudaGraphExecDestroy(m->graph_exec);
   delete m;
 }
 

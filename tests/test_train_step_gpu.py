@@ -236,3 +236,24 @@ def test_error_paths_return_codes_and_keep_the_context_usable():
     model.set_param("norm_f", w)
     assert np.isfinite(model.forward_loss(to_dev(tok), to_dev(lab)))
     model.close()
+
+
+def test_whole_step_graph_replay_is_bit_identical_to_plain_launches():
+    from paper_2609_13645_b200 import binding as B
+    ocfg, _ = _c1()
+    params = D.init_params(ocfg, SI.WEIGHT_SEED)
+    plain, l_plain = _run_steps(ocfg, params, 5)
+    side = torch.cuda.Stream()  # the legacy default stream cannot be captured
+    with torch.cuda.stream(side):
+        graphed = B.Model(lib_config(B, ocfg, 2, 128), seed=1)
+        load_params(graphed, params)
+        graphed.set_graph(True)
+        _, l_graph = _run_steps(ocfg, params, 5, model=graphed)
+        side.synchronize()
+        assert graphed.graph_replays >= 3  # step 1 plain, step 2 captured and replayed, steps 3..5 replayed
+        assert np.array_equal(np.float32(l_plain).view(np.uint32), np.float32(l_graph).view(np.uint32))
+        for a, b in zip(_state_bits(plain), _state_bits(graphed)):
+            assert np.array_equal(a, b)
+        assert graphed.step == 5
+        graphed.close()
+    plain.close()
