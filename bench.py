@@ -99,6 +99,21 @@ class ClockSampler:
                 "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(values, world, device=None):
+    """Element-wise maximum of a list of floats over all ranks (the slowest rank defines a multi-GPU time)."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def job_tokens_per_s(tokens_per_step_per_rank, world, ms_total, steps):
+    """Whole-job throughput of `world` independent replicas that all took ms_total (max over ranks) for `steps` steps."""
+    return world * tokens_per_step_per_rank / (ms_total / 1e3 / steps)
+
+
 def model_flops(w, seq):
     return flops_per_token(w["n_layers"], w["d_model"], w["n_heads"], w["n_kv_heads"], w["head_dim"], w["d_ffn"],
                            w["vocab"], seq)
@@ -252,15 +267,12 @@ def run_cuda(args):
     barrier()
     ms_e2e = ev2.elapsed_time(ev3)
 
-    tms = torch.tensor([ms_total, ms_e2e, ms_prof], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
-    ms_total, ms_e2e, ms_prof = float(tms[0]), float(tms[1]), float(tms[2])
+    ms_total, ms_e2e, ms_prof = max_over_ranks([ms_total, ms_e2e, ms_prof], world, device="cuda")
 
     if rank == 0:
         fl = model_flops(w, S)
         step_s = ms_total / 1e3 / args.steps
-        tok_s = world * tokens_per_step / step_s
+        tok_s = job_tokens_per_s(tokens_per_step, world, ms_total, args.steps)
         model_tflops = fl["total"] * tokens_per_step / step_s / 1e12
         g = prof["gemm"]
         gemm_tflops = g["work"] / (g["ms"] / 1e3) / 1e12 if g["ms"] > 0 else None
@@ -290,7 +302,7 @@ def run_cuda(args):
                     "vs_measured_sustained": model_tflops / peak_tf,
                     "vs_nominal_2250": model_tflops / NOMINAL_BF16_TFLOPS, "peaks": peak_kind},
             "roofline": roof, "ms_per_step_profiled": ms_prof / args.steps, "kernel_classes": classes,
-            "e2e": {"value": world * tokens_per_step / (ms_e2e / 1e3 / args.steps), "unit": "tokens/s",
+            "e2e": {"value": job_tokens_per_s(tokens_per_step, world, ms_e2e, args.steps), "unit": "tokens/s",
                     "h2d_bytes_per_step": 2 * tokens_per_step * 4, "d2h_bytes_per_step": 64,
                     "ms_per_step": ms_e2e / args.steps, "last_loss": e2e_loss},
             "gemm_shapes": [dict(g, ms_per_step=g["ms"] / args.steps, launches_per_step=g["launches"] / args.steps)

@@ -257,3 +257,25 @@ def test_whole_step_graph_replay_is_bit_identical_to_plain_launches():
         assert graphed.step == 5
         graphed.close()
     plain.close()
+
+
+def test_ten_step_loss_and_gradient_norm_trajectory_matches_oracle():
+    """Ten consecutive steps on fresh batches: per-step loss within 1e-2, gradient norm within 1 %, and the masters
+    after ten steps within the sign-flip bound of one step (the error does not pile up)."""
+    from paper_2609_13645_b200 import binding as B
+    ocfg = oracle_config(n_layers=2, d_model=256, n_heads=4, n_kv_heads=2, head_dim=64, d_ffn=352, vocab=512)
+    params = D.init_params(ocfg, 2024)
+    st = D.TrainState(ocfg, params)
+    model = B.Model(lib_config(B, ocfg, 2, 96), seed=1)
+    load_params(model, params)
+    for step in range(10):
+        tok, lab = SI.batch(ocfg.vocab, 2, 96, "zipf", step=step)
+        loss_o, gn_o, _, _ = st.train_step(tok, lab)
+        loss_g, gn_g = model.train_step(to_dev(tok), to_dev(lab))
+        assert abs(loss_g - loss_o) < TOL_LOSS, (step, loss_g, loss_o)
+        assert abs(gn_g - gn_o) / gn_o < 1e-2, (step, gn_g, gn_o)
+    assert model.step == 10
+    for name in params:
+        e = rel_l2(model.get_param(name), st.params[name])
+        assert e < 1e-2, (name, e)
+    model.close()
