@@ -139,6 +139,17 @@ ft_status ft_k_gemm(const void* dev_A, int32_t a_mn, int64_t lda, const void* de
                     void* dev_C, int64_t ldc, const void* dev_resid, int32_t out_kind,
                     int32_t M, int32_t N, int32_t K, int32_t* dev_err, void* stream);
 
+/* Weight-gradient contraction (Section 4.3, "dW = X^T dY"): C fp32 [M, N] (+)= A^T B with A bf16 [K, lda] (M
+ * contiguous) and B bf16 [K, ldb] (N contiguous), K the token dimension.  When the output has too few 256 x 256
+ * tiles to occupy every SM pair and K is long, the K range is divided into up to 8 parts that run concurrently,
+ * each writing an fp32 partial [M, N] into dev_scratch; a second kernel adds the parts in index order (and the old
+ * C when accumulate != 0), so the result is bit-identical from run to run.  dev_scratch: device memory owned by the
+ * caller, scratch_bytes of it; with less than 2 * M * N * 4 bytes the call degrades to the single-pass kernel.
+ * M, N, K multiples of 8; lda, ldb multiples of 8; ldc a multiple of 4.  dev_err as in ft_k_gemm. */
+ft_status ft_k_gemm_splitk(const void* dev_A, int64_t lda, const void* dev_B, int64_t ldb, float* dev_C, int64_t ldc,
+                           int32_t accumulate, int32_t M, int32_t N, int32_t K, float* dev_scratch,
+                           uint64_t scratch_bytes, int32_t* dev_err, void* stream);
+
 /* Causal attention core forward on a packed qkv buffer bf16 [B*S, (n_h + 2 n_kv) * d] (q heads, k heads,
  * v heads; q, k already rotated): o bf16 [B*S, n_h*d], lse fp32 [B, n_h, S] (natural log). d in {64, 128}. */
 ft_status ft_k_attention_fwd(const void* dev_qkv, void* dev_o, float* dev_lse, int32_t B, int32_t S,

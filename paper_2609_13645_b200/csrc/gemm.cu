@@ -42,6 +42,8 @@ struct GemmDev {
   int M, N, K;
   int epi;
   int seq, head_dim, rope_cols, d_ffn;
+  int ksplit;              // > 1: the K blocks are divided over ksplit work units per output tile
+  long long split_stride;  // elements between the partial outputs of consecutive K parts
 };
 
 __device__ __forceinline__ void store8_bf16(bf16* dst, const float* v) {
@@ -450,8 +452,10 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
   const int tiles_m = (p.M + 255) / 256;
   const int tiles_n = (p.N + BN - 1) / BN;
-  const int ntiles = tiles_m * tiles_n;
-  const int kblocks = (p.K + BK - 1) / BK;
+  const int tiles_mn = tiles_m * tiles_n;
+  const int ntiles = tiles_mn * p.ksplit;  // work units: (output tile, K part)
+  const int kblocks_all = (p.K + BK - 1) / BK;
+  const int kpb = (kblocks_all + p.ksplit - 1) / p.ksplit;  // K blocks per part (every part is non-empty by construction)
 
   if (warp == 0) {
     if (lane == 0) {
@@ -459,9 +463,10 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       uint32_t phase = 0;
       bool ok = true;
       for (int t = pair; t < ntiles && ok; t += npairs) {
-        const int m0 = (t % tiles_m) * 256 + (int)rank * BM;       // this CTA's rows of A / of the output
-        const int nb0 = (t / tiles_m) * BN + (int)rank * C::HALF_B;  // this CTA's rows of B
-        for (int kb = 0; kb < kblocks; ++kb) {
+        const int tt = t % tiles_mn, kb0 = (t / tiles_mn) * kpb, kb1 = min(kblocks_all, kb0 + kpb);
+        const int m0 = (tt % tiles_m) * 256 + (int)rank * BM;       // this CTA's rows of A / of the output
+        const int nb0 = (tt / tiles_m) * BN + (int)rank * C::HALF_B;  // this CTA's rows of B
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.err)) { ok = false; break; }
           const uint32_t fb = full_bar(stage);
           if (rank == 0) mbar_expect_tx(fb, 2 * C::STAGE_BYTES);
@@ -498,7 +503,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.err)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-        for (int kb = 0; kb < kblocks; ++kb) {
+        const int kb0 = (t / tiles_mn) * kpb, kb1 = min(kblocks_all, kb0 + kpb);
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag, p.err)) { ok = false; break; }
           tc_fence_after();
           const uint32_t a_addr = smem_u32(smem + stage * C::STAGE_BYTES);
@@ -509,7 +515,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                                         : umma_desc_sw128(a_addr + k * 32, 0, 1024);
             const uint64_t bdesc = B_MN ? umma_desc_sw128(b_addr + k * 2048, CHUNK_BYTES, 1024)
                                         : umma_desc_sw128(b_addr + k * 32, 0, 1024);
-            umma_bf16_pair(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+            umma_bf16_pair(d_tmem, adesc, bdesc, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
           }
           umma_commit_pair(empty_bar(stage));  // frees the stage in both CTAs
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
@@ -525,14 +531,21 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     int acc = 0;
     uint32_t acc_phase = 0;
     for (int t = pair; t < ntiles; t += npairs) {
-      const int m0 = (t % tiles_m) * 256 + (int)rank * BM;
-      const int n0 = (t / tiles_m) * BN;
+      const int tt = t % tiles_mn;
+      const int m0 = (tt % tiles_m) * 256 + (int)rank * BM;
+      const int n0 = (tt / tiles_m) * BN;
       bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.err);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
       const int row = m0 + q * 32 + lane;
-      epilogue_tile<BN>(p, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), row, n0);
+      if (p.ksplit > 1) {
+        GemmDev pp = p;  // this K part's own fp32 partial output
+        pp.C = reinterpret_cast<float*>(p.C) + (long long)(t / tiles_mn) * p.split_stride;
+        epilogue_tile<BN>(pp, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), row, n0);
+      } else {
+        epilogue_tile<BN>(p, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), row, n0);
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_leader(tempty_bar(acc));
@@ -554,6 +567,22 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     __syncwarp();
     tc_fence_after();
     tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
+  }
+}
+
+// out[r, c] (+)= sum over K parts of partial[s][r, c], parts added in index order (deterministic)
+__global__ void splitk_reduce_kernel(const float* __restrict__ partial, int nsplit, long long stride, float* __restrict__ out,
+                                     long long ldc, int M, int N, int accumulate) {
+  const long long n4 = (long long)M * (N / 4);
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (long long)gridDim.x * blockDim.x) {
+    const long long r = i / (N / 4);
+    const int c = (int)(i % (N / 4)) * 4;
+    float4 a = accumulate ? *reinterpret_cast<const float4*>(out + r * ldc + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < nsplit; ++s) {
+      const float4 v = *reinterpret_cast<const float4*>(partial + s * stride + r * N + c);
+      a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+    }
+    *reinterpret_cast<float4*>(out + r * ldc + c) = a;
   }
 }
 
@@ -587,6 +616,7 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
   p.C = a.C; p.resid = a.resid; p.gu = a.gu; p.rope_cos = a.rope_cos; p.rope_sin = a.rope_sin; p.err = a.err;
   p.ldc = a.ldc; p.M = a.M; p.N = a.N; p.K = a.K; p.epi = a.epi;
   p.seq = a.seq; p.head_dim = a.head_dim; p.rope_cols = a.rope_cols; p.d_ffn = a.d_ffn;
+  p.ksplit = 1; p.split_stride = 0;
   const int tiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN);
   const int grid = tiles < sm_count() ? tiles : sm_count();
   kern<<<grid, GEMM_THREADS, C::SMEM_BYTES, stream>>>(tmA, tmB, p);
@@ -613,7 +643,24 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
   p.seq = a.seq; p.head_dim = a.head_dim; p.rope_cols = a.rope_cols; p.d_ffn = a.d_ffn;
   const int tiles = ((a.M + 255) / 256) * ((a.N + 255) / 256);
   const int max_pairs = sm_count() / 2;
-  const int pairs = tiles < max_pairs ? tiles : max_pairs;
+  // split-K for weight gradients whose output has too few tiles to occupy the machine
+  int ksplit = 1;
+  const int kblocks = (a.K + BK - 1) / BK;
+  if (A_MN && B_MN && (a.epi == EPI_F32 || a.epi == EPI_F32_ACC) && a.splitk_scratch && tiles * 2 <= max_pairs) {
+    int want = max_pairs / tiles;
+    if (want > 8) want = 8;
+    if (want > kblocks / 8) want = kblocks / 8;  // at least 8 K blocks per part
+    if (want >= 2) {
+      const int kpb = (kblocks + want - 1) / want;
+      want = (kblocks + kpb - 1) / kpb;  // every part non-empty
+      if (want >= 2 && (size_t)want * a.M * a.N * sizeof(float) <= a.splitk_bytes) ksplit = want;
+    }
+  }
+  p.ksplit = ksplit;
+  p.split_stride = (long long)a.M * a.N;
+  if (ksplit > 1) { p.C = a.splitk_scratch; p.ldc = a.N; p.epi = EPI_F32; }
+  const int work = tiles * ksplit;
+  const int pairs = work < max_pairs ? work : max_pairs;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs, 1, 1);
   cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
@@ -626,7 +673,13 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, tmA, tmB, p);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, p);
+  if (e != cudaSuccess || ksplit == 1) return e;
+  const long long n4 = (long long)a.M * (a.N / 4);
+  const int blocks = (int)((n4 + 255) / 256 < 1184 ? (n4 + 255) / 256 : 1184);
+  splitk_reduce_kernel<<<blocks, 256, 0, stream>>>(a.splitk_scratch, ksplit, p.split_stride, reinterpret_cast<float*>(a.C),
+                                                   a.ldc, a.M, a.N, a.epi == EPI_F32_ACC ? 1 : 0);
+  return cudaGetLastError();
 }
 
 }  // namespace

@@ -36,6 +36,10 @@ struct GemmArgs {
   bf16* gu = nullptr;  // [M, 2f] gate | up
   int d_ffn = 0;
   int* err = nullptr;  // device status word
+  // Optional fp32 scratch for split-K: weight-gradient GEMMs with few output tiles split their (long) contraction over
+  // several CTA pairs, write partial tiles here and add them in a fixed order.  Unused when null or too small.
+  float* splitk_scratch = nullptr;
+  size_t splitk_bytes = 0;
 };
 
 // Enqueues the contraction on `stream`.  Returns cudaErrorInvalidValue for shapes it does not take.

@@ -19,6 +19,7 @@ using namespace fs;
 namespace {
 
 constexpr size_t kAlign = 256;
+constexpr size_t kSplitKFloats = 6u << 20;  // 24 MiB of split-K partial tiles (74 tiles of 256 x 256 fp32 at most)
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct ParamInfo {
@@ -74,7 +75,7 @@ struct ft_model {
   float *rF, *ce_lse, *loss_row;
   bf16 *hF, *d_hF;
   bf16 *dxA, *dxB, *d_h, *d_a, *d_gu, *d_o, *d_qkv;
-  float *delta, *norm_partial, *sq_partial, *z;
+  float *delta, *norm_partial, *sq_partial, *z, *splitk;
   bf16* dz;
   unsigned long long* keys;
   int lastB = 0, lastS = 0;
@@ -194,6 +195,7 @@ size_t carve(ft_model* m, uint8_t* base) {
   m->delta = cv.take<float>(T * c.n_heads);
   m->norm_partial = cv.take<float>((size_t)elementwise_blocks_for_norm((int)T) * h);
   m->sq_partial = cv.take<float>(kSqnormBlocks);
+  m->splitk = cv.take<float>(kSplitKFloats);
   m->z = cv.take<float>((size_t)m->ce_chunk * V);
   m->dz = cv.take<bf16>((size_t)m->ce_chunk * V);
   m->keys = cv.take<unsigned long long>(sort_pad(T));
@@ -297,6 +299,8 @@ AdamHyper hyper(const ft_model* m) {
 GemmArgs gemm_base(ft_model* m) {
   GemmArgs g;
   g.err = &m->sc->err;
+  g.splitk_scratch = m->splitk;
+  g.splitk_bytes = kSplitKFloats * sizeof(float);
   return g;
 }
 
@@ -896,6 +900,21 @@ ft_status ft_k_gemm(const void* dev_A, int32_t a_mn, int64_t lda, const void* de
   g.B = reinterpret_cast<const bf16*>(dev_B); g.b_mn = b_mn; g.ldb = ldb;
   g.C = dev_C; g.ldc = ldc; g.resid = reinterpret_cast<const bf16*>(dev_resid);
   g.epi = out_kind; g.M = M; g.N = N; g.K = K; g.err = dev_err;
+  cudaError_t e = launch_gemm(g, reinterpret_cast<cudaStream_t>(stream));
+  if (e == cudaErrorInvalidValue) return FT_EINVAL;
+  return e == cudaSuccess ? FT_OK : FT_ECUDA;
+}
+
+ft_status ft_k_gemm_splitk(const void* dev_A, int64_t lda, const void* dev_B, int64_t ldb, float* dev_C, int64_t ldc,
+                           int32_t accumulate, int32_t M, int32_t N, int32_t K, float* dev_scratch, uint64_t scratch_bytes,
+                           int32_t* dev_err, void* stream) {
+  if (!dev_A || !dev_B || !dev_C || !dev_scratch) return FT_EINVAL;
+  GemmArgs g;
+  g.A = reinterpret_cast<const bf16*>(dev_A); g.a_mn = 1; g.lda = lda;
+  g.B = reinterpret_cast<const bf16*>(dev_B); g.b_mn = 1; g.ldb = ldb;
+  g.C = dev_C; g.ldc = ldc;
+  g.epi = accumulate ? EPI_F32_ACC : EPI_F32; g.M = M; g.N = N; g.K = K; g.err = dev_err;
+  g.splitk_scratch = dev_scratch; g.splitk_bytes = scratch_bytes;
   cudaError_t e = launch_gemm(g, reinterpret_cast<cudaStream_t>(stream));
   if (e == cudaErrorInvalidValue) return FT_EINVAL;
   return e == cudaSuccess ? FT_OK : FT_ECUDA;

@@ -90,3 +90,35 @@ def test_bad_arguments_are_rejected_without_launching():
         B.k_gemm(a, 0, a, 0, c, 0, 128, 124, 64, err)  # N not a multiple of 8
     with pytest.raises(B.ForgeStepError):
         B.k_gemm(a, 1, a, 0, c, 0, 64, 128, 128, err)  # mn-major A with k-major B is not offered
+
+
+@pytest.mark.parametrize("M,N,K,acc", [(768, 768, 8192, False), (512, 256, 4096, True), (1000, 520, 2056, True),
+                                       (256, 256, 1024, False), (768, 2304, 8192, False), (256, 256, 960, True)])
+def test_split_k_weight_gradient_matches_the_contraction_and_repeats_bit_for_bit(M, N, K, acc):
+    """Few output tiles, long K: the K range is divided over concurrent CTA pairs and the parts are added in a
+    fixed order.  Checked against the fp64 contraction, against run-to-run bit identity, and (ragged K, ragged
+    tiles) against the padding rules of the single-pass kernel."""
+    from paper_2609_13645_b200 import binding as B
+    rng = np.random.default_rng(11)
+    A, At = _bf16_tensor(rng, (K, M))
+    Bm, Bt = _bf16_tensor(rng, (K, N))
+    ref = A.T @ Bm + (0.5 if acc else 0.0)
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    scratch = torch.full((8 * M * N,), float("nan"), dtype=torch.float32, device="cuda")
+    outs = []
+    for _ in range(2):
+        out = torch.full((M, N), 0.5, dtype=torch.float32, device="cuda")
+        B.k_gemm_splitk(At, Bt, out, M, N, K, scratch, err, accumulate=acc)
+        torch.cuda.synchronize()
+        assert int(err.item()) == 0
+        outs.append(out.cpu().numpy())
+    assert np.array_equal(outs[0], outs[1])
+    got = outs[0].astype(np.float64)
+    assert np.all(np.isfinite(got))
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) < 1e-5
+    # a scratch buffer too small for two parts falls back to the single-pass kernel and still gives the result
+    out = torch.full((M, N), 0.5, dtype=torch.float32, device="cuda")
+    B.k_gemm_splitk(At, Bt, out, M, N, K, scratch[:M * N], err, accumulate=acc)
+    torch.cuda.synchronize()
+    got1 = out.cpu().numpy().astype(np.float64)
+    assert np.linalg.norm(got1 - ref) / np.linalg.norm(ref) < 1e-5
