@@ -122,6 +122,8 @@ ft_status ft_get_gemm_profile(ft_model* m, int32_t i, int32_t shape[6], double* 
 void ft_debug_gemm_tile(int32_t bn);
 /* Development switch: 1 = CTA-pair (cta_group::2, 256 x 256 tile) GEMM kernel where it applies (default), 0 = off. */
 void ft_debug_gemm_pairs(int32_t on);
+/* Development switch: 1 = balanced-K schedule where it applies and scratch is available (default), 0 = round-robin tiles. */
+void ft_debug_gemm_balanced(int32_t on);
 
 const char* ft_last_error(const ft_model* m);
 /* Number of kernels the library launched since the model was created (for launch accounting). */
@@ -139,16 +141,21 @@ ft_status ft_k_gemm(const void* dev_A, int32_t a_mn, int64_t lda, const void* de
                     void* dev_C, int64_t ldc, const void* dev_resid, int32_t out_kind,
                     int32_t M, int32_t N, int32_t K, int32_t* dev_err, void* stream);
 
-/* Weight-gradient contraction (Section 4.3, "dW = X^T dY"): C fp32 [M, N] (+)= A^T B with A bf16 [K, lda] (M
- * contiguous) and B bf16 [K, ldb] (N contiguous), K the token dimension.  When the output has too few 256 x 256
- * tiles to occupy every SM pair and K is long, the K range is divided into up to 8 parts that run concurrently,
- * each writing an fp32 partial [M, N] into dev_scratch; a second kernel adds the parts in index order (and the old
- * C when accumulate != 0), so the result is bit-identical from run to run.  dev_scratch: device memory owned by the
- * caller, scratch_bytes of it; with less than 2 * M * N * 4 bytes the call degrades to the single-pass kernel.
- * M, N, K multiples of 8; lda, ldb multiples of 8; ldc a multiple of 4.  dev_err as in ft_k_gemm. */
-ft_status ft_k_gemm_splitk(const void* dev_A, int64_t lda, const void* dev_B, int64_t ldb, float* dev_C, int64_t ldc,
-                           int32_t accumulate, int32_t M, int32_t N, int32_t K, float* dev_scratch,
-                           uint64_t scratch_bytes, int32_t* dev_err, void* stream);
+/* ft_k_gemm with a device scratch buffer that lets the kernel divide work along K (Section 4.3: weight gradients
+ * contract over the token dimension, the long one).  Results stay bit-identical from run to run:
+ *  - weight-gradient layout (a_mn = b_mn = 1, fp32 output) with few 256 x 256 output tiles: up to 8 K parts run
+ *    concurrently into fp32 partial outputs and a second kernel adds them in index order;
+ *  - any layout whose tile count is not a multiple of the number of SM pairs: every pair takes an equally long range
+ *    of (tile, K block) units; a tile cut by a range boundary is completed by the pair holding its first K block, which
+ *    adds the other pairs' fp32 partial tiles in pair order before the usual epilogue.
+ * dev_scratch: caller-owned device memory, 16-byte aligned, scratch_bytes long; its contents on entry do not matter
+ * (the call clears the 1 KiB of counters at its start with a stream-ordered memset) and are unspecified afterwards.
+ * 20 MiB covers every case; with less the call degrades to the plain schedule of ft_k_gemm.  Two calls that share a
+ * scratch buffer must not overlap on the GPU. */
+ft_status ft_k_gemm_ws(const void* dev_A, int32_t a_mn, int64_t lda, const void* dev_B, int32_t b_mn, int64_t ldb,
+                       void* dev_C, int64_t ldc, const void* dev_resid, int32_t out_kind,
+                       int32_t M, int32_t N, int32_t K, float* dev_scratch, uint64_t scratch_bytes,
+                       int32_t* dev_err, void* stream);
 
 /* Causal attention core forward on a packed qkv buffer bf16 [B*S, (n_h + 2 n_kv) * d] (q heads, k heads,
  * v heads; q, k already rotated): o bf16 [B*S, n_h*d], lse fp32 [B, n_h, S] (natural log). d in {64, 128}. */

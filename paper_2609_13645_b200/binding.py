@@ -81,8 +81,8 @@ def lib():
         L.ft_destroy.restype = None
         L.ft_destroy.argtypes = [vp]
         L.ft_k_gemm.argtypes = [vp, i32, i64, vp, i32, i64, vp, i64, vp, i32, i32, i32, i32, vp, vp]
-        L.ft_k_gemm_splitk.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, i32, vp, C.c_uint64, vp, vp]
-        L.ft_k_gemm_splitk.restype = C.c_int
+        L.ft_k_gemm_ws.argtypes = [vp, i32, i64, vp, i32, i64, vp, i64, vp, i32, i32, i32, i32, vp, C.c_uint64, vp, vp]
+        L.ft_k_gemm_ws.restype = C.c_int
         L.ft_k_attention_fwd.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp]
         L.ft_k_attention_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]
         L.ft_k_attention_bwd_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]
@@ -281,15 +281,15 @@ def k_gemm(A, a_mn: int, B, b_mn: int, Cout, out_kind: int, M: int, N: int, K: i
         raise ForgeStepError(st, "ft_k_gemm")
 
 
-def k_gemm_splitk(A, B, Cout, M: int, N: int, K: int, scratch, err, accumulate: bool = False):
-    """Weight-gradient contraction C[M,N] (+)= A^T B (A [K, M], B [K, N] bf16, C fp32) with a deterministic split of
-    K over concurrent CTA pairs; `scratch` is an fp32 device tensor for the partial outputs."""
-    st = lib().ft_k_gemm_splitk(C.c_void_p(A.data_ptr()), A.stride(0), C.c_void_p(B.data_ptr()), B.stride(0),
-                                C.c_void_p(Cout.data_ptr()), Cout.stride(0), int(accumulate), M, N, K,
-                                C.c_void_p(scratch.data_ptr()), scratch.numel() * 4, C.c_void_p(err.data_ptr()),
-                                _stream_ptr())
+def k_gemm_ws(A, a_mn: int, B, b_mn: int, Cout, out_kind: int, M: int, N: int, K: int, scratch, err, resid=None):
+    """k_gemm with an fp32 device scratch tensor, which enables the deterministic split-K / balanced-K schedules."""
+    st = lib().ft_k_gemm_ws(C.c_void_p(A.data_ptr()), a_mn, A.stride(0), C.c_void_p(B.data_ptr()), b_mn, B.stride(0),
+                            C.c_void_p(Cout.data_ptr()), Cout.stride(0),
+                            C.c_void_p(resid.data_ptr()) if resid is not None else None, out_kind, M, N, K,
+                            C.c_void_p(scratch.data_ptr()), scratch.numel() * 4, C.c_void_p(err.data_ptr()),
+                            _stream_ptr())
     if st != FT_OK:
-        raise ForgeStepError(st, "ft_k_gemm_splitk")
+        raise ForgeStepError(st, "ft_k_gemm_ws")
 
 
 def k_attention_fwd(qkv, o, lse, B, S, n_heads, n_kv, d):

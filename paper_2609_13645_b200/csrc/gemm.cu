@@ -13,7 +13,11 @@
 
 namespace fs {
 
+int g_gemm_balanced = 1;  // development knob: 0 = always the round-robin tile schedule
+
 namespace {
+
+constexpr size_t kScratchFlagFloats = 256;
 
 constexpr int BM = 128;
 constexpr int BK = 64;  // 64 bf16 = 128 bytes = one swizzle row
@@ -44,7 +48,74 @@ struct GemmDev {
   int seq, head_dim, rope_cols, d_ffn;
   int ksplit;              // > 1: the K blocks are divided over ksplit work units per output tile
   long long split_stride;  // elements between the partial outputs of consecutive K parts
+  int balanced;            // 1: the last partial wave of tiles is divided along K and runs first (see WorkIter)
+  int sw_first;            // balanced: first tile of the divided wave (tiles before it run whole, round-robin)
+  int sw_parts;            // balanced: K parts per tile of the divided wave
+  int sw_kpb;              // balanced: K blocks per part
+  int* flags;              // balanced: one arrival counter per pair (zero between launches)
+  float* slots;            // balanced: one fp32 partial tile [256][256] per pair
 };
+
+// The work of one CTA pair as a sequence of pieces (output tile, K blocks [kb0, kb1), K part).
+// Round-robin schedule: piece i is unit pair + i * npairs of (tile, K part).
+// Balanced schedule, for a tile count that leaves a last wave with at most half of the pairs busy: the tiles of that
+// wave are divided into sw_parts K parts each and run FIRST, pair q taking part q % sw_parts of tile sw_first +
+// q / sw_parts.  Parts > 0 leave their accumulator in the pair's scratch slot; the pair with part 0 adds them in its
+// epilogue (which overlaps its next tile's main loop).  All pairs then walk the remaining tiles round-robin, in step
+// with one another as in the plain schedule, which keeps concurrent CTAs on the same K blocks of shared operands.
+struct WorkIter {
+  int tiles_mn, kblocks, kpb, nunits, npairs, t;
+  int sw_tile, sw_kb0, sw_kb1, sw_part;  // this pair's piece of the divided wave (sw_tile < 0: none)
+  __device__ WorkIter(const GemmDev& p, int tiles, int kb, int pair, int np)
+      : tiles_mn(tiles), kblocks(kb), kpb((kb + p.ksplit - 1) / p.ksplit), nunits(tiles * p.ksplit), npairs(np), t(pair),
+        sw_tile(-1), sw_kb0(0), sw_kb1(0), sw_part(0) {
+    if (p.balanced) {
+      nunits = p.sw_first;
+      const int j = pair / p.sw_parts;
+      if (p.sw_first + j < tiles) {
+        sw_tile = p.sw_first + j;
+        sw_part = pair % p.sw_parts;
+        sw_kb0 = sw_part * p.sw_kpb;
+        sw_kb1 = min(kb, sw_kb0 + p.sw_kpb);
+      }
+    }
+  }
+  // split: the piece belongs to the divided wave
+  __device__ bool next(int& tile, int& kb0, int& kb1, int& part, bool& split) {
+    if (sw_tile >= 0) {
+      tile = sw_tile; kb0 = sw_kb0; kb1 = sw_kb1; part = sw_part; split = true;
+      sw_tile = -1;
+      return true;
+    }
+    split = false;
+    if (t >= nunits) return false;
+    tile = t % tiles_mn;
+    part = t / tiles_mn;
+    kb0 = part * kpb;
+    kb1 = min(kblocks, kb0 + kpb);
+    t += npairs;
+    return true;
+  }
+};
+
+// Bounded wait for `flag` to reach `target` (acquire).  One lane calls it.
+__device__ __forceinline__ bool flag_wait(const int* flag, int target, volatile int* abort_flag, int* err) {
+  const long long t0 = clock64();
+  for (uint32_t it = 1;; ++it) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+    if (v >= target) return true;
+    if ((it & 63u) == 0u) {
+      if (*abort_flag != 0) return false;
+      if (clock64() - t0 > kWaitLimitCycles) {
+        *abort_flag = 1;
+        atomicExch(err, (int)ERR_WAIT_TIMEOUT);
+        return false;
+      }
+    }
+    __nanosleep(64);
+  }
+}
 
 __device__ __forceinline__ void store8_bf16(bf16* dst, const float* v) {
   uint4 o;
@@ -55,25 +126,77 @@ __device__ __forceinline__ void store8_bf16(bf16* dst, const float* v) {
   *reinterpret_cast<uint4*>(dst) = o;
 }
 
+#ifdef FS_GEMM_TRACE
+// development trace: per CTA pair and piece, globaltimer at (accumulator ready, partials ready, epilogue done)
+__device__ unsigned long long g_gemm_trace[148 * 32 * 4];
+__device__ __forceinline__ unsigned long long gtimer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+#define FS_GTRACE(pair, piece, k) do { if ((piece) < 32) g_gemm_trace[((pair) * 32 + (piece)) * 4 + (k)] = gtimer(); } while (0)
+#else
+#define FS_GTRACE(pair, piece, k) do { } while (0)
+#endif
+
+constexpr int SLOT_FLOATS = 256 * 256;  // one fp32 partial tile of a CTA pair
+
+// Partial accumulators of the same output tile that other CTA pairs left in scratch.  A slot holds a pair's 256 x 256
+// fp32 accumulator in the order the epilogue threads touch it, so that every warp access is one contiguous 512 bytes:
+// float4 index = ((cta * 4 + lane quarter) * 64 + (column / 32) * 8 + j) * 32 + lane for columns 32 * (column / 32) +
+// 4 j .. + 3 of the row held by `lane`.  `base` points at this thread's first float4 of the first partial.
+constexpr int SLOT_F4 = SLOT_FLOATS / 4;
+struct Fixup {
+  const float4* base = nullptr;
+  int n = 0;
+};
+__device__ __forceinline__ int slot_thread_f4(int cta, int quarter, int lane) { return (cta * 4 + quarter) * 2048 + lane; }
+
+// 32 accumulator columns of this thread's row from TMEM (+ the partials of the same columns, added in index order)
+__device__ __forceinline__ void ld_acc32(uint32_t taddr, int coloff, uint32_t (&r)[32], const Fixup& fx) {
+  tmem_ld32(taddr + coloff, r);
+  if (fx.n == 0) {
+    tmem_ld_wait();
+    return;
+  }
+  // one round trip to L2 per partial: the trips, not the bytes, bound this loop (the launcher limits their number)
+  const float4* src = fx.base + (coloff >> 5) * 256;
+  float4 v[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) v[j] = __ldcg(src + j * 32);
+  tmem_ld_wait();
+  for (int s = 0;;) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      r[4 * j + 0] = __float_as_uint(__uint_as_float(r[4 * j + 0]) + v[j].x);
+      r[4 * j + 1] = __float_as_uint(__uint_as_float(r[4 * j + 1]) + v[j].y);
+      r[4 * j + 2] = __float_as_uint(__uint_as_float(r[4 * j + 2]) + v[j].z);
+      r[4 * j + 3] = __float_as_uint(__uint_as_float(r[4 * j + 3]) + v[j].w);
+    }
+    if (++s >= fx.n) break;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = __ldcg(src + (long long)s * SLOT_F4 + j * 32);
+  }
+}
+
 // Epilogue of one accumulator tile for one thread: `row` is the global output row held by this thread's TMEM lane,
 // taddr the TMEM address of (its lane quarter, first column of the tile), n0 the tile's first output column.
 // Every tcgen05.ld is executed by all 32 lanes (rows past M only skip the stores).
 template <int BN>
-__device__ __forceinline__ void epilogue_tile(const GemmDev& p, uint32_t taddr, int row, int n0) {
+__device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint32_t taddr, int row, int n0, const Fixup fx = Fixup()) {
   const bool row_ok = row < p.M;
   uint32_t r[32];
   if (p.epi == EPI_ROPE) {
     const int d = p.head_dim;
     const int half = d >> 1;
     const int pos = row_ok ? (row % p.seq) : 0;
-    bf16* crow = reinterpret_cast<bf16*>(p.C) + (long long)row * p.ldc;
+    bf16* crow = reinterpret_cast<bf16*>(cptr) + (long long)row * p.ldc;
     for (int hc = 0; hc < BN; hc += d) {
       const int g0 = n0 + hc;
       if (g0 >= p.N) break;
       if (g0 >= p.rope_cols) {
         for (int c = 0; c < d; c += 32) {
-          tmem_ld32(taddr + hc + c, r);
-          tmem_ld_wait();
+          ld_acc32(taddr, hc + c, r, fx);
           if (row_ok) {
             float v[32];
 #pragma unroll
@@ -85,9 +208,14 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, uint32_t taddr, 
       } else {
         uint32_t r2[32];
         for (int i0 = 0; i0 < half; i0 += 32) {
-          tmem_ld32(taddr + hc + i0, r);
-          tmem_ld32(taddr + hc + i0 + half, r2);
-          tmem_ld_wait();
+          if (fx.n == 0) {
+            tmem_ld32(taddr + hc + i0, r);
+            tmem_ld32(taddr + hc + i0 + half, r2);
+            tmem_ld_wait();
+          } else {
+            ld_acc32(taddr, hc + i0, r, fx);
+            ld_acc32(taddr, hc + i0 + half, r2, fx);
+          }
           if (row_ok) {
             const float* cs = p.rope_cos + (long long)pos * half + i0;
             const float* sn = p.rope_sin + (long long)pos * half + i0;
@@ -118,13 +246,12 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, uint32_t taddr, 
   } else if (p.epi == EPI_SWIGLU) {
     // physical columns alternate 16 gate / 16 up of the same 16 logical ffn columns
     const int f = p.d_ffn;
-    bf16* arow = reinterpret_cast<bf16*>(p.C) + (long long)row * p.ldc;
+    bf16* arow = reinterpret_cast<bf16*>(cptr) + (long long)row * p.ldc;
     bf16* gurow = p.gu + (long long)row * (2LL * f);
     for (int c = 0; c < BN; c += 32) {
       const int gc = n0 + c;
       if (gc >= p.N) break;
-      tmem_ld32(taddr + c, r);
-      tmem_ld_wait();
+      ld_acc32(taddr, c, r, fx);
       if (row_ok) {
         const int lc = gc >> 1;  // logical ffn column of this 16-wide group
         float g[16], u[16], a[16];
@@ -145,7 +272,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, uint32_t taddr, 
   } else if (p.epi == EPI_BF16_RESID) {
     // the residual row is read one 32-column chunk ahead of the accumulator it is added to, so its latency overlaps
     // the TMEM load and the stores of the previous chunk
-    bf16* crow = reinterpret_cast<bf16*>(p.C) + (long long)row * p.ldc;
+    bf16* crow = reinterpret_cast<bf16*>(cptr) + (long long)row * p.ldc;
     const bf16* rrow = p.resid + (long long)row * p.ldc;
     uint4 nxt[4];
     auto fetch = [&](int gc) {
@@ -161,8 +288,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, uint32_t taddr, 
 #pragma unroll
       for (int j = 0; j < 4; ++j) cur[j] = nxt[j];
       if (c + 32 < BN) fetch(gc + 32);
-      tmem_ld32(taddr + c, r);
-      tmem_ld_wait();
+      ld_acc32(taddr, c, r, fx);
       if (row_ok) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -178,7 +304,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, uint32_t taddr, 
       }
     }
   } else if (p.epi == EPI_F32_ACC) {
-    float* crow = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc;
+    float* crow = reinterpret_cast<float*>(cptr) + (long long)row * p.ldc;
     float4 nxt[8];
     auto fetch = [&](int gc) {
 #pragma unroll
@@ -193,8 +319,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, uint32_t taddr, 
 #pragma unroll
       for (int j = 0; j < 8; ++j) cur[j] = nxt[j];
       if (c + 32 < BN) fetch(gc + 32);
-      tmem_ld32(taddr + c, r);
-      tmem_ld_wait();
+      ld_acc32(taddr, c, r, fx);
       if (row_ok) {
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -211,11 +336,10 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, uint32_t taddr, 
     for (int c = 0; c < BN; c += 32) {
       const int gc = n0 + c;
       if (gc >= p.N) break;
-      tmem_ld32(taddr + c, r);
-      tmem_ld_wait();
+      ld_acc32(taddr, c, r, fx);
       if (row_ok) {
         if (p.epi == EPI_BF16) {
-          bf16* crow = reinterpret_cast<bf16*>(p.C) + (long long)row * p.ldc + gc;
+          bf16* crow = reinterpret_cast<bf16*>(cptr) + (long long)row * p.ldc + gc;
 #pragma unroll
           for (int j = 0; j < 32; j += 8) {
             if (gc + j < p.N) {
@@ -226,7 +350,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, uint32_t taddr, 
             }
           }
         } else {
-          float* crow = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + gc;
+          float* crow = reinterpret_cast<float*>(cptr) + (long long)row * p.ldc + gc;
 #pragma unroll
           for (int j = 0; j < 32; j += 4) {
             if (gc + j < p.N)
@@ -364,7 +488,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (!ok) break;
       tc_fence_after();
       const int row = m0 + q * 32 + lane;
-      epilogue_tile<BN>(p, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), row, n0);
+      epilogue_tile<BN>(p, p.C, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), row, n0);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(acc));
@@ -453,19 +577,19 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const int tiles_m = (p.M + 255) / 256;
   const int tiles_n = (p.N + BN - 1) / BN;
   const int tiles_mn = tiles_m * tiles_n;
-  const int ntiles = tiles_mn * p.ksplit;  // work units: (output tile, K part)
   const int kblocks_all = (p.K + BK - 1) / BK;
-  const int kpb = (kblocks_all + p.ksplit - 1) / p.ksplit;  // K blocks per part (every part is non-empty by construction)
+  WorkIter work(p, tiles_mn, kblocks_all, pair, npairs);
+  int tile, kb0, kb1, part;
+  bool split;
 
   if (warp == 0) {
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int t = pair; t < ntiles && ok; t += npairs) {
-        const int tt = t % tiles_mn, kb0 = (t / tiles_mn) * kpb, kb1 = min(kblocks_all, kb0 + kpb);
-        const int m0 = (tt % tiles_m) * 256 + (int)rank * BM;       // this CTA's rows of A / of the output
-        const int nb0 = (tt / tiles_m) * BN + (int)rank * C::HALF_B;  // this CTA's rows of B
+      while (ok && work.next(tile, kb0, kb1, part, split)) {
+        const int m0 = (tile % tiles_m) * 256 + (int)rank * BM;       // this CTA's rows of A / of the output
+        const int nb0 = (tile / tiles_m) * BN + (int)rank * C::HALF_B;  // this CTA's rows of B
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.err)) { ok = false; break; }
           const uint32_t fb = full_bar(stage);
@@ -499,11 +623,10 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
-      for (int t = pair; t < ntiles && ok; t += npairs) {
+      while (ok && work.next(tile, kb0, kb1, part, split)) {
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.err)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-        const int kb0 = (t / tiles_mn) * kpb, kb1 = min(kblocks_all, kb0 + kpb);
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag, p.err)) { ok = false; break; }
           tc_fence_after();
@@ -530,25 +653,60 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const int q = warp & 3;
     int acc = 0;
     uint32_t acc_phase = 0;
-    for (int t = pair; t < ntiles; t += npairs) {
-      const int tt = t % tiles_mn;
-      const int m0 = (tt % tiles_m) * 256 + (int)rank * BM;
-      const int n0 = (tt / tiles_m) * BN;
+    [[maybe_unused]] int piece = 0;
+    [[maybe_unused]] const bool tracer = (warp == 2 && lane == 0 && rank == 0);
+    if (tracer) FS_GTRACE(pair, 31, 0);
+    while (work.next(tile, kb0, kb1, part, split)) {
+      const int m0 = (tile % tiles_m) * 256 + (int)rank * BM;
+      const int n0 = (tile / tiles_m) * BN;
       bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.err);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
       const int row = m0 + q * 32 + lane;
-      if (p.ksplit > 1) {
-        GemmDev pp = p;  // this K part's own fp32 partial output
-        pp.C = reinterpret_cast<float*>(p.C) + (long long)(t / tiles_mn) * p.split_stride;
-        epilogue_tile<BN>(pp, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), row, n0);
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
+      const int slot_f4 = slot_thread_f4((int)rank, q, lane);
+      if (tracer) { FS_GTRACE(pair, piece, 0); FS_GTRACE(pair, piece, 1); }
+      if (split && part > 0) {
+        // a later K part of a divided tile: leave this partial accumulator in the pair's slot
+        float4* dst = reinterpret_cast<float4*>(p.slots) + (long long)pair * SLOT_F4 + slot_f4;
+        uint32_t r[32];
+        for (int c = 0; c < BN && n0 + c < p.N; c += 32) {
+          tmem_ld32(taddr + c, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            __stcg(dst + (c >> 5) * 256 + j * 32,
+                   make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
+                               __uint_as_float(r[4 * j + 3])));
+        }
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) atomicAdd(p.flags + pair, 1);
       } else {
-        epilogue_tile<BN>(p, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), row, n0);
+        Fixup fx;
+        void* cptr = p.C;
+        if (split && p.sw_parts > 1) {
+          // part 0 of a divided tile: wait for the other parts (they run at the same time on the next pairs) and add
+          // them in pair order
+          fx.n = p.sw_parts - 1;
+          fx.base = reinterpret_cast<const float4*>(p.slots) + (long long)(pair + 1) * SLOT_F4 + slot_f4;
+          int got = 1;
+          if (lane == 0)
+            for (int s = 0; s < fx.n && got; ++s) got = flag_wait(p.flags + pair + 1 + s, 8, abort_flag, p.err) ? 1 : 0;
+          got = __shfl_sync(0xffffffffu, got, 0);
+          if (!got) break;
+          if (tracer) FS_GTRACE(pair, piece, 1);
+        } else if (p.ksplit > 1) {
+          cptr = reinterpret_cast<float*>(p.C) + (long long)part * p.split_stride;  // this K part's own fp32 partial output
+        }
+        epilogue_tile<BN>(p, cptr, taddr, row, n0, fx);
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_leader(tempty_bar(acc));
+      if (tracer) FS_GTRACE(pair, piece, 2);
+      ++piece;
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
     }
@@ -563,6 +721,12 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     __syncthreads();
   }
   cluster_sync_all();
+  if (p.balanced && rank == 0 && threadIdx.x == 0) {
+    // every warp of the pair has consumed the partials: clear the arrival counters this pair waited on for the next launch
+    WorkIter mine(p, tiles_mn, kblocks_all, pair, npairs);
+    if (mine.sw_tile >= 0 && mine.sw_part == 0)
+      for (int s2 = 1; s2 < p.sw_parts; ++s2) p.flags[pair + s2] = 0;
+  }
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
@@ -616,7 +780,7 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
   p.C = a.C; p.resid = a.resid; p.gu = a.gu; p.rope_cos = a.rope_cos; p.rope_sin = a.rope_sin; p.err = a.err;
   p.ldc = a.ldc; p.M = a.M; p.N = a.N; p.K = a.K; p.epi = a.epi;
   p.seq = a.seq; p.head_dim = a.head_dim; p.rope_cols = a.rope_cols; p.d_ffn = a.d_ffn;
-  p.ksplit = 1; p.split_stride = 0;
+  p.ksplit = 1; p.split_stride = 0; p.balanced = 0; p.sw_first = 0; p.sw_parts = 1; p.sw_kpb = 0; p.flags = nullptr; p.slots = nullptr;
   const int tiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN);
   const int grid = tiles < sm_count() ? tiles : sm_count();
   kern<<<grid, GEMM_THREADS, C::SMEM_BYTES, stream>>>(tmA, tmB, p);
@@ -643,24 +807,51 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
   p.seq = a.seq; p.head_dim = a.head_dim; p.rope_cols = a.rope_cols; p.d_ffn = a.d_ffn;
   const int tiles = ((a.M + 255) / 256) * ((a.N + 255) / 256);
   const int max_pairs = sm_count() / 2;
+  // scratch layout: 256 arrival counters (kept zero between launches), then fp32 partial tiles
+  int* flags = reinterpret_cast<int*>(a.scratch);
+  float* data = a.scratch ? a.scratch + kScratchFlagFloats : nullptr;
+  const size_t data_bytes = a.scratch_bytes > kScratchFlagFloats * sizeof(float) ? a.scratch_bytes - kScratchFlagFloats * sizeof(float) : 0;
+  const int kblocks = (a.K + BK - 1) / BK;
   // split-K for weight gradients whose output has too few tiles to occupy the machine
   int ksplit = 1;
-  const int kblocks = (a.K + BK - 1) / BK;
-  if (A_MN && B_MN && (a.epi == EPI_F32 || a.epi == EPI_F32_ACC) && a.splitk_scratch && tiles * 2 <= max_pairs) {
+  if (A_MN && B_MN && (a.epi == EPI_F32 || a.epi == EPI_F32_ACC) && data && tiles * 2 <= max_pairs) {
     int want = max_pairs / tiles;
     if (want > 8) want = 8;
     if (want > kblocks / 8) want = kblocks / 8;  // at least 8 K blocks per part
     if (want >= 2) {
       const int kpb = (kblocks + want - 1) / want;
       want = (kblocks + kpb - 1) / kpb;  // every part non-empty
-      if (want >= 2 && (size_t)want * a.M * a.N * sizeof(float) <= a.splitk_bytes) ksplit = want;
+      if (want >= 2 && (size_t)want * a.M * a.N * sizeof(float) <= data_bytes) ksplit = want;
     }
   }
   p.ksplit = ksplit;
   p.split_stride = (long long)a.M * a.N;
-  if (ksplit > 1) { p.C = a.splitk_scratch; p.ldc = a.N; p.epi = EPI_F32; }
+  if (ksplit > 1) { p.C = data; p.ldc = a.N; p.epi = EPI_F32; }
+  // balanced schedule: a last wave that would keep at most half of the pairs busy is divided along K
+  p.balanced = 0; p.sw_first = tiles; p.sw_parts = 1; p.sw_kpb = kblocks; p.flags = flags; p.slots = data;
+  const int left = tiles % max_pairs;
+  if (g_gemm_balanced && ksplit == 1 && data && tiles > max_pairs && left > 0 && max_pairs <= 256 &&
+      (size_t)max_pairs * SLOT_FLOATS * sizeof(float) <= data_bytes) {
+    int parts = max_pairs / left;
+    // The pair with part 0 adds the other parts' tiles while its next tile's main loop runs; the longer that loop (K),
+    // the more partials fit into it without delaying the tile after.
+    const int cap = kblocks < 48 ? 2 : (kblocks < 80 ? 3 : (kblocks < 112 ? 5 : 8));
+    if (parts > cap) parts = cap;
+    if (parts > kblocks / 4) parts = kblocks / 4;  // at least 4 K blocks per part
+    const int waves = (tiles + max_pairs - 1) / max_pairs;
+    if (parts >= 2 && (parts - 1) * 50 < parts * waves) parts = 1;  // saves under 2 % of the kernel: not worth the traffic
+    if (parts >= 2) {
+      const int kpb = (kblocks + parts - 1) / parts;
+      parts = (kblocks + kpb - 1) / kpb;  // every part non-empty
+      if (parts >= 2) { p.balanced = 1; p.sw_first = tiles - left; p.sw_parts = parts; p.sw_kpb = kpb; }
+    }
+  }
   const int work = tiles * ksplit;
-  const int pairs = work < max_pairs ? work : max_pairs;
+  const int pairs = p.balanced ? max_pairs : (work < max_pairs ? work : max_pairs);
+  if (p.balanced && a.scratch_reset) {
+    cudaError_t e0 = cudaMemsetAsync(flags, 0, kScratchFlagFloats * sizeof(float), stream);
+    if (e0 != cudaSuccess) return e0;
+  }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs, 1, 1);
   cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
@@ -677,12 +868,20 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
   if (e != cudaSuccess || ksplit == 1) return e;
   const long long n4 = (long long)a.M * (a.N / 4);
   const int blocks = (int)((n4 + 255) / 256 < 1184 ? (n4 + 255) / 256 : 1184);
-  splitk_reduce_kernel<<<blocks, 256, 0, stream>>>(a.splitk_scratch, ksplit, p.split_stride, reinterpret_cast<float*>(a.C),
+  splitk_reduce_kernel<<<blocks, 256, 0, stream>>>(data, ksplit, p.split_stride, reinterpret_cast<float*>(a.C),
                                                    a.ldc, a.M, a.N, a.epi == EPI_F32_ACC ? 1 : 0);
   return cudaGetLastError();
 }
 
 }  // namespace
+
+#ifdef FS_GEMM_TRACE
+}  // namespace fs
+extern "C" int ft_debug_gemm_trace(unsigned long long* host_dst, int n) {
+  return (int)cudaMemcpyFromSymbol(host_dst, fs::g_gemm_trace, sizeof(unsigned long long) * n);
+}
+namespace fs {
+#endif
 
 int g_gemm_force_bn = 0;
 int g_gemm_pairs = 1;  // development knob: 1 = CTA-pair kernel for outputs of at least 256 x 256, 0 = single-CTA kernel only  // development knob: 0 = choose by tile count, 128 or 256 = force that tile width

@@ -36,10 +36,15 @@ struct GemmArgs {
   bf16* gu = nullptr;  // [M, 2f] gate | up
   int d_ffn = 0;
   int* err = nullptr;  // device status word
-  // Optional fp32 scratch for split-K: weight-gradient GEMMs with few output tiles split their (long) contraction over
-  // several CTA pairs, write partial tiles here and add them in a fixed order.  Unused when null or too small.
-  float* splitk_scratch = nullptr;
-  size_t splitk_bytes = 0;
+  // Optional device scratch that lets the CTA-pair kernel divide work along K (both deterministic):
+  //  - split-K: weight gradients with few output tiles run up to 8 K parts concurrently, a second kernel adds them;
+  //  - balanced-K: when the tile count is not a multiple of the pair count, every pair takes an equally long range of
+  //    (tile, K block) units and tiles cut by a range boundary are completed from fp32 partials.
+  // The first 1 KiB holds arrival counters that must be zero at launch; the kernel leaves them zero.  With
+  // scratch_reset the launcher clears them itself (one memset node) before a balanced-K launch.
+  float* scratch = nullptr;
+  size_t scratch_bytes = 0;
+  bool scratch_reset = false;
 };
 
 // Enqueues the contraction on `stream`.  Returns cudaErrorInvalidValue for shapes it does not take.
@@ -47,5 +52,6 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream);
 
 extern int g_gemm_force_bn;
 extern int g_gemm_pairs;
+extern int g_gemm_balanced;
 
 }  // namespace fs

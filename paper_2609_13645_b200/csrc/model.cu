@@ -299,8 +299,8 @@ AdamHyper hyper(const ft_model* m) {
 GemmArgs gemm_base(ft_model* m) {
   GemmArgs g;
   g.err = &m->sc->err;
-  g.splitk_scratch = m->splitk;
-  g.splitk_bytes = kSplitKFloats * sizeof(float);
+  g.scratch = m->splitk;
+  g.scratch_bytes = kSplitKFloats * sizeof(float);
   return g;
 }
 
@@ -563,6 +563,7 @@ ft_status ft_init_model(const ft_config* cfg, uint64_t seed, void* dev_workspace
   FT_CUDA(cudaMemsetAsync(m->grad, 0, m->arena * sizeof(float), st));
   FT_CUDA(cudaMemsetAsync(m->master, 0, m->arena * sizeof(float), st));
   FT_CUDA(cudaMemsetAsync(m->sc, 0, sizeof(StepScalars), st));
+  FT_CUDA(cudaMemsetAsync(m->splitk, 0, 1024, st));  // the GEMM scratch's arrival counters start at zero
   for (size_t i = 0; i < m->params.size(); ++i) {
     const ParamInfo& p = m->params[i];
     if (p.cols) {
@@ -866,6 +867,7 @@ ft_status ft_get_profile(ft_model* m, int32_t cls, double* ms, double* work, int
 }
 
 void ft_debug_gemm_tile(int32_t bn) { g_gemm_force_bn = bn; }
+void ft_debug_gemm_balanced(int32_t on) { g_gemm_balanced = on; }
 void ft_debug_gemm_pairs(int32_t on) { g_gemm_pairs = on; }
 
 ft_status ft_get_gemm_profile(ft_model* m, int32_t i, int32_t shape[6], double* ms, int64_t* launches) {
@@ -905,16 +907,16 @@ ft_status ft_k_gemm(const void* dev_A, int32_t a_mn, int64_t lda, const void* de
   return e == cudaSuccess ? FT_OK : FT_ECUDA;
 }
 
-ft_status ft_k_gemm_splitk(const void* dev_A, int64_t lda, const void* dev_B, int64_t ldb, float* dev_C, int64_t ldc,
-                           int32_t accumulate, int32_t M, int32_t N, int32_t K, float* dev_scratch, uint64_t scratch_bytes,
-                           int32_t* dev_err, void* stream) {
-  if (!dev_A || !dev_B || !dev_C || !dev_scratch) return FT_EINVAL;
+ft_status ft_k_gemm_ws(const void* dev_A, int32_t a_mn, int64_t lda, const void* dev_B, int32_t b_mn, int64_t ldb,
+                       void* dev_C, int64_t ldc, const void* dev_resid, int32_t out_kind, int32_t M, int32_t N, int32_t K,
+                       float* dev_scratch, uint64_t scratch_bytes, int32_t* dev_err, void* stream) {
+  if (out_kind < 0 || out_kind > 3 || !dev_scratch) return FT_EINVAL;
   GemmArgs g;
-  g.A = reinterpret_cast<const bf16*>(dev_A); g.a_mn = 1; g.lda = lda;
-  g.B = reinterpret_cast<const bf16*>(dev_B); g.b_mn = 1; g.ldb = ldb;
-  g.C = dev_C; g.ldc = ldc;
-  g.epi = accumulate ? EPI_F32_ACC : EPI_F32; g.M = M; g.N = N; g.K = K; g.err = dev_err;
-  g.splitk_scratch = dev_scratch; g.splitk_bytes = scratch_bytes;
+  g.A = reinterpret_cast<const bf16*>(dev_A); g.a_mn = a_mn; g.lda = lda;
+  g.B = reinterpret_cast<const bf16*>(dev_B); g.b_mn = b_mn; g.ldb = ldb;
+  g.C = dev_C; g.ldc = ldc; g.resid = reinterpret_cast<const bf16*>(dev_resid);
+  g.epi = out_kind; g.M = M; g.N = N; g.K = K; g.err = dev_err;
+  g.scratch = dev_scratch; g.scratch_bytes = scratch_bytes; g.scratch_reset = true;
   cudaError_t e = launch_gemm(g, reinterpret_cast<cudaStream_t>(stream));
   if (e == cudaErrorInvalidValue) return FT_EINVAL;
   return e == cudaSuccess ? FT_OK : FT_ECUDA;

@@ -37,7 +37,7 @@ def main():
     ap.add_argument("--no-flush", action="store_true")
     ap.add_argument("--out", default="auto", choices=["auto", "bf16", "resid", "f32", "f32acc"], help="GEMM epilogue")
     ap.add_argument("--bn", type=int, default=0, help="force the GEMM tile width (development)")
-    ap.add_argument("--splitk", action="store_true", help="wgrad layout: the split-K entry point with 8 parts of scratch")
+    ap.add_argument("--ws", action="store_true", help="GEMM with a scratch buffer (split-K / balanced-K schedules)")
     ap.add_argument("--pairs", type=int, default=1, help="0: single-CTA GEMM kernel only (development)")
     a = ap.parse_args()
     torch.manual_seed(0)
@@ -67,11 +67,10 @@ def main():
                 resid = torch.randn(M, N, device=dev).bfloat16()
         flops = 2.0 * M * N * K
         run = lambda: B.k_gemm(A, amn, Bm, bmn, out, kind, M, N, K, err, resid)
-        if a.splitk:
-            assert a.layout == "wgrad" and kind in (2, 3)
-            scratch = torch.empty(8 * M * N, dtype=torch.float32, device=dev)
-            run = lambda: B.k_gemm_splitk(A, Bm, out, M, N, K, scratch, err, accumulate=(kind == 3))
-        desc = dict(kernel="gemm", layout=a.layout, out=a.out, M=M, N=N, K=K, splitk=bool(a.splitk))
+        if a.ws:
+            scratch = torch.empty(6 << 20, dtype=torch.float32, device=dev)
+            run = lambda: B.k_gemm_ws(A, amn, Bm, bmn, out, kind, M, N, K, scratch, err, resid)
+        desc = dict(kernel="gemm", layout=a.layout, out=a.out, M=M, N=N, K=K, ws=bool(a.ws))
     else:
         Bsz, S, nh, nkv, d = a.B, a.S, a.nh, a.nkv, a.d
         qkv = torch.randn(Bsz * S, (nh + 2 * nkv) * d, device=dev).bfloat16()

@@ -13,7 +13,7 @@ def _bf16_tensor(rng, shape, scale=1.0):
     return a, torch.from_numpy(a.astype(np.float32)).to(torch.bfloat16).cuda()
 
 
-def _run(M, N, K, a_mn, b_mn, out_kind, seed=0):
+def _run(M, N, K, a_mn, b_mn, out_kind, seed=0, ws=False):
     from paper_2609_13645_b200 import binding as B
     rng = np.random.default_rng(seed)
     A, At = _bf16_tensor(rng, (K, M) if a_mn else (M, K))
@@ -31,7 +31,11 @@ def _run(M, N, K, a_mn, b_mn, out_kind, seed=0):
         out = torch.full((M, N), 0.5, dtype=torch.float32, device="cuda")
         if out_kind == 3:
             ref = ref + 0.5
-    B.k_gemm(At, a_mn, Bt, b_mn, out, out_kind, M, N, K, err, resid)
+    if ws:
+        scratch = torch.full((5 << 20,), float("nan"), dtype=torch.float32, device="cuda")
+        B.k_gemm_ws(At, a_mn, Bt, b_mn, out, out_kind, M, N, K, scratch, err, resid)
+    else:
+        B.k_gemm(At, a_mn, Bt, b_mn, out, out_kind, M, N, K, err, resid)
     torch.cuda.synchronize()
     assert int(err.item()) == 0
     got = out.float().cpu().numpy().astype(np.float64)
@@ -104,11 +108,11 @@ def test_split_k_weight_gradient_matches_the_contraction_and_repeats_bit_for_bit
     Bm, Bt = _bf16_tensor(rng, (K, N))
     ref = A.T @ Bm + (0.5 if acc else 0.0)
     err = torch.zeros(1, dtype=torch.int32, device="cuda")
-    scratch = torch.full((8 * M * N,), float("nan"), dtype=torch.float32, device="cuda")
+    scratch = torch.full((256 + 8 * M * N,), float("nan"), dtype=torch.float32, device="cuda")
     outs = []
     for _ in range(2):
         out = torch.full((M, N), 0.5, dtype=torch.float32, device="cuda")
-        B.k_gemm_splitk(At, Bt, out, M, N, K, scratch, err, accumulate=acc)
+        B.k_gemm_ws(At, 1, Bt, 1, out, 3 if acc else 2, M, N, K, scratch, err)
         torch.cuda.synchronize()
         assert int(err.item()) == 0
         outs.append(out.cpu().numpy())
@@ -118,7 +122,45 @@ def test_split_k_weight_gradient_matches_the_contraction_and_repeats_bit_for_bit
     assert np.linalg.norm(got - ref) / np.linalg.norm(ref) < 1e-5
     # a scratch buffer too small for two parts falls back to the single-pass kernel and still gives the result
     out = torch.full((M, N), 0.5, dtype=torch.float32, device="cuda")
-    B.k_gemm_splitk(At, Bt, out, M, N, K, scratch[:M * N], err, accumulate=acc)
+    B.k_gemm_ws(At, 1, Bt, 1, out, 3 if acc else 2, M, N, K, scratch[:M * N], err)
     torch.cuda.synchronize()
     got1 = out.cpu().numpy().astype(np.float64)
     assert np.linalg.norm(got1 - ref) / np.linalg.norm(ref) < 1e-5
+
+
+# Shapes with more 256 x 256 tiles than the 74 SM pairs and a last wave of at most 37 tiles: the balanced schedule
+# divides that wave into 2 .. 8 K parts.  Ragged M, N and K (parts of unequal length) included.
+BALANCED = [(2048, 2560, 512), (2048, 2560, 1024), (4096, 4096, 520), (2000, 2568, 1000), (8192, 2048, 704),
+            (2304, 2304, 2048), (2560, 2560, 512)]
+
+
+@pytest.mark.parametrize("M,N,K", BALANCED)
+@pytest.mark.parametrize("a_mn,b_mn,kind", [(0, 0, 0), (0, 1, 0), (1, 1, 2), (1, 1, 3), (0, 0, 1)])
+def test_balanced_k_schedule_matches_the_contraction(M, N, K, a_mn, b_mn, kind):
+    rel, got, ref = _run(M, N, K, a_mn, b_mn, kind, seed=21, ws=True)
+    assert np.all(np.isfinite(got))
+    if kind >= 2:
+        assert rel < 1e-5, rel
+    else:
+        assert rel < 2e-3 and np.mean(got != ref) < 0.02
+        # one bf16 rounding of a sum whose fp32 accumulation error is far below the typical magnitude sqrt(K)
+        assert np.all(np.abs(got - ref) <= 2.0 ** -7 * np.abs(ref) + 1e-2)
+
+
+def test_balanced_k_schedule_repeats_bit_for_bit_and_leaves_its_counters_clear():
+    from paper_2609_13645_b200 import binding as B
+    M, N, K = 2048, 2560, 1024
+    rng = np.random.default_rng(5)
+    _, At = _bf16_tensor(rng, (M, K))
+    _, Bt = _bf16_tensor(rng, (N, K))
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    scratch = torch.full((5 << 20,), float("nan"), dtype=torch.float32, device="cuda")
+    outs = []
+    for _ in range(3):
+        out = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        B.k_gemm_ws(At, 0, Bt, 0, out, 0, M, N, K, scratch, err)
+        torch.cuda.synchronize()
+        assert int(err.item()) == 0
+        assert int(scratch[:256].view(torch.int32).abs().sum().item()) == 0
+        outs.append(out.view(torch.int16).cpu().numpy())
+    assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])

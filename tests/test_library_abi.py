@@ -17,7 +17,7 @@ def declared_symbols():
 def test_header_declares_the_boundary():
     syms = declared_symbols()
     for need in ("ft_workspace_bytes", "ft_init_model", "ft_train_step", "ft_train_step_host", "ft_forward_loss",
-                 "ft_get_param", "ft_set_param", "ft_get_tap", "ft_apply_update", "ft_k_gemm", "ft_k_gemm_splitk", "ft_k_attention_fwd",
+                 "ft_get_param", "ft_set_param", "ft_get_tap", "ft_apply_update", "ft_k_gemm", "ft_k_gemm_ws", "ft_k_attention_fwd",
                  "ft_k_attention_bwd"):
         assert need in syms
 
