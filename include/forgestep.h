@@ -65,6 +65,16 @@ ft_status ft_init_model(const ft_config* cfg, uint64_t seed, void* dev_workspace
 ft_status ft_train_step(ft_model* m, const int32_t* dev_tokens, const int32_t* dev_labels, int32_t B, int32_t S,
                         float* host_loss, float* host_gnorm);
 
+/* Optimizer-tail fusion (Section 5.3's fused clip + Adam, taken one step further): with gradient clipping off
+ * (max_grad_norm <= 0) the update of a weight matrix does not depend on the global norm, so ft_train_step applies
+ * AdamW inside the epilogue of the weight-gradient GEMM (or of its split-K reduction): the finished fp32 gradient
+ * never goes to memory, and the separate optimizer pass shrinks to the embedding table and the gains.  The update
+ * arithmetic is the same function, so parameters, moments and losses are bit-identical to the unfused step; the
+ * reported gradient norm is summed in a different (still fixed) order.  On by default; off automatically when
+ * clipping is on or debug_taps is set.  After a fusing ft_train_step, FT_GRAD_F32 of the matrices holds stale
+ * values (use ft_forward_backward to materialise gradients).  Changing the setting drops a captured graph. */
+ft_status ft_set_fused_update(ft_model* m, int32_t enable);
+
 /* Whole-step CUDA graph (the paper's full-step graph capture): when enabled, the first ft_train_step of a (B, S)
  * runs launch by launch, the second is captured into a graph, later ones replay it (ids are first copied into the
  * model's own buffers).  Needs a capturable stream (not the legacy default stream; otherwise it switches itself

@@ -74,6 +74,8 @@ def lib():
         L.ft_debug_gemm_pairs.restype = None
         L.ft_get_gemm_profile.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(C.c_double), C.POINTER(i64)]
         L.ft_get_gemm_profile.restype = C.c_int
+        L.ft_set_fused_update.argtypes = [vp, i32]
+        L.ft_set_fused_update.restype = C.c_int
         L.ft_set_graph.argtypes = [vp, i32]
         L.ft_set_graph.restype = C.c_int
         L.ft_graph_replays.argtypes = [vp]
@@ -229,6 +231,10 @@ class Model:
         self._check(lib().ft_get_tap(self._h, name.encode(), layer, C.c_void_p(buf.ctypes.data), buf.nbytes,
                                      C.byref(need), C.byref(dt)))
         return buf.view(np.float32).copy() if dt.value == 1 else bf16_bits_to_f32(buf.view(np.uint16))
+
+    def set_fused_update(self, enable: bool):
+        """AdamW inside the weight-gradient GEMM epilogues (default on; only takes effect with clipping off)."""
+        self._check(lib().ft_set_fused_update(self._h, 1 if enable else 0))
 
     def set_graph(self, enable: bool):
         """Capture the whole step into a CUDA graph on its second run and replay it afterwards."""

@@ -2,6 +2,8 @@
 // atomics), so results are bit-identical from run to run; all global accesses are 16-byte vectors.
 #include "elementwise.cuh"
 
+#include "adamw_math.cuh"
+
 #include <math.h>
 
 namespace fs {
@@ -451,8 +453,8 @@ adamw_kernel(float* __restrict__ p, float* __restrict__ m, float* __restrict__ v
              bf16* __restrict__ pb, size_t n4, size_t n4_decay, const StepScalars* __restrict__ sc, AdamHyper hp,
              float* __restrict__ sq_partial) {
   __shared__ float s_sq[8];
-  const float clip = WITH_NORM ? 1.0f : sc->clip, bc1 = sc->bc1, bc2 = sc->bc2;
-  const float omb1 = 1.0f - hp.beta1, omb2 = 1.0f - hp.beta2;
+  const float clip = WITH_NORM ? 1.0f : sc->clip;
+  const AdamCoef c = make_adam_coef(hp.lr, hp.beta1, hp.beta2, hp.eps, sc->bc1, sc->bc2);
   float sq = 0.f;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
     const float wd = i < n4_decay ? hp.wd : 0.f;
@@ -466,15 +468,7 @@ adamw_kernel(float* __restrict__ p, float* __restrict__ m, float* __restrict__ v
     float vv[4] = {v4.x, v4.y, v4.z, v4.w};
     if (WITH_NORM) sq += g4.x * g4.x + g4.y * g4.y + g4.z * g4.z + g4.w * g4.w;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const float ge = gg[e] * clip;
-      mm[e] = hp.beta1 * mm[e] + omb1 * ge;
-      vv[e] = hp.beta2 * vv[e] + omb2 * ge * ge;
-      const float mhat = mm[e] / bc1;
-      const float vhat = vv[e] / bc2;
-      const float upd = mhat / (sqrtf(vhat) + hp.eps) + wd * pp[e];
-      pp[e] = pp[e] - hp.lr * upd;
-    }
+    for (int e = 0; e < 4; ++e) adamw_elem(__fmul_rn(gg[e], clip), wd, c, pp[e], mm[e], vv[e]);
     reinterpret_cast<float4*>(p)[i] = make_float4(pp[0], pp[1], pp[2], pp[3]);
     reinterpret_cast<float4*>(m)[i] = make_float4(mm[0], mm[1], mm[2], mm[3]);
     reinterpret_cast<float4*>(v)[i] = make_float4(vv[0], vv[1], vv[2], vv[3]);
@@ -651,6 +645,17 @@ int adamw_with_norm(float* p, float* m, float* v, const float* g, bf16* pb, size
   adamw_kernel<true><<<kSqnormBlocks, 256, 0, st>>>(p, m, v, g, pb, n / 4, n_decay / 4, sc, hp, partial);
   sqnorm_final_kernel<<<1, 256, 0, st>>>(partial, kSqnormBlocks, sc, hp);
   return ok(2);
+}
+
+int adamw_range_with_norm(float* p, float* m, float* v, const float* g, bf16* pb, size_t n, size_t n_decay, float* partial,
+                          const StepScalars* sc, AdamHyper hp, cudaStream_t st) {
+  adamw_kernel<true><<<kSqnormBlocks, 256, 0, st>>>(p, m, v, g, pb, n / 4, n_decay / 4, sc, hp, partial);
+  return ok(1);
+}
+
+int sqnorm_final(const float* partial, int count, StepScalars* sc, AdamHyper hp, cudaStream_t st) {
+  sqnorm_final_kernel<<<1, 256, 0, st>>>(partial, count, sc, hp);
+  return ok(1);
 }
 
 int init_normal(float* p, size_t n, uint64_t seed, int tensor_id, double stddev, cudaStream_t st) {

@@ -54,6 +54,11 @@ int adamw(float* p, float* m, float* v, const float* g, bf16* pb, size_t n, size
 // clipping off: the same pass also sums the squared gradient norm (reported, not used by the update)
 int adamw_with_norm(float* p, float* m, float* v, const float* g, bf16* pb, size_t n, size_t n_decay, float* partial,
                     StepScalars* sc, AdamHyper hp, cudaStream_t st);
+// AdamW over one range of the arenas (clipping off), writing kSqnormBlocks partial sums of g^2 to `partial` and leaving
+// the final sum to sqnorm_final, which adds `count` partials in index order and stores the norm in sc.
+int adamw_range_with_norm(float* p, float* m, float* v, const float* g, bf16* pb, size_t n, size_t n_decay, float* partial,
+                          const StepScalars* sc, AdamHyper hp, cudaStream_t st);
+int sqnorm_final(const float* partial, int count, StepScalars* sc, AdamHyper hp, cudaStream_t st);
 int init_normal(float* p, size_t n, uint64_t seed, int tensor_id, double std, cudaStream_t st);
 int fill_f32(float* p, size_t n, float v, cudaStream_t st);
 int cast_bf16(const float* src, bf16* dst, size_t n, cudaStream_t st);

@@ -9,11 +9,14 @@
 // contraction runs over the rows of the stored activations) without materialising any transpose.
 #include "gemm.cuh"
 
+#include "adamw_math.cuh"
+#include "elementwise.cuh"
 #include "tmap.cuh"
 
 namespace fs {
 
-int g_gemm_balanced = 1;  // development knob: 0 = always the round-robin tile schedule
+int g_gemm_balanced = 1;
+int g_gemm_last_launches = 1;  // development knob: 0 = always the round-robin tile schedule
 
 namespace {
 
@@ -25,6 +28,13 @@ constexpr int A_BYTES = BM * BK * 2;
 constexpr int CHUNK_BYTES = 64 * BK * 2;  // one 64 x 64 box of an mn-major operand
 constexpr int GEMM_THREADS = 192;
 
+// Per epilogue warp, a 32 x 32 fp32 staging tile that turns "one thread per output row" into coalesced 128-byte row
+// segments.  The 16-byte column group j of row r sits at group j ^ (r & 7): conflict-free both for a thread writing
+// its row and for 8 lanes reading one row.
+constexpr int EPI_STAGE_FLOATS = 32 * 32;
+constexpr int EPI_WARPS_MAX = 8;
+constexpr int EPI_STAGE_BYTES = EPI_WARPS_MAX * EPI_STAGE_FLOATS * 4;
+
 template <int BN>
 struct Cfg {
   static constexpr int B_BYTES = BN * BK * 2;
@@ -32,7 +42,7 @@ struct Cfg {
   static constexpr int STAGES = (BN == 256) ? 4 : 6;
   static constexpr int TMEM_COLS = 2 * BN;
   static constexpr int BAR_BYTES = 256;
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024;  // + slack to align to 1024
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + EPI_STAGE_BYTES + 1024;  // + slack to align to 1024
 };
 
 struct GemmDev {
@@ -54,7 +64,32 @@ struct GemmDev {
   int sw_kpb;              // balanced: K blocks per part
   int* flags;              // balanced: one arrival counter per pair (zero between launches)
   float* slots;            // balanced: one fp32 partial tile [256][256] per pair
+  // fused AdamW (null adam_p: off)
+  float* adam_p;
+  float* adam_m;
+  float* adam_v;
+  bf16* adam_pb;
+  const StepScalars* adam_sc;
+  float* adam_sq;
+  float adam_lr, adam_beta1, adam_beta2, adam_eps, adam_wd;
 };
+
+__device__ __forceinline__ AdamCoef adam_coef(const GemmDev& p) {
+  return make_adam_coef(p.adam_lr, p.adam_beta1, p.adam_beta2, p.adam_eps, p.adam_sc->bc1, p.adam_sc->bc2);
+}
+
+// Fused AdamW: the epilogue streams master, moments (and, when accumulating, the earlier gradient) of its block with
+// few loads in flight, too few to cover DRAM latency.  Each lane therefore asks L2, one 32-column chunk ahead, for the
+// 128-byte line of every stream at (its row, that chunk).  (Plain prefetch instructions: bulk prefetches go through
+// the TMA unit and were measured to slow the operand loads of the main loop.)
+__device__ __forceinline__ void adam_prefetch_chunk(const GemmDev& p, const void* cptr, int row, int gc) {
+  if (row >= p.M || gc >= p.N) return;
+  const long long o = (long long)row * p.ldc + gc;
+  asm volatile("prefetch.global.L2 [%0];" ::"l"(p.adam_p + o));
+  asm volatile("prefetch.global.L2 [%0];" ::"l"(p.adam_m + o));
+  asm volatile("prefetch.global.L2 [%0];" ::"l"(p.adam_v + o));
+  if (p.epi == EPI_F32_ACC) asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const float*>(cptr) + o));
+}
 
 // The work of one CTA pair as a sequence of pieces (output tile, K blocks [kb0, kb1), K part).
 // Round-robin schedule: piece i is unit pair + i * npairs of (tile, K part).
@@ -183,15 +218,80 @@ __device__ __forceinline__ void ld_acc32(uint32_t taddr, int coloff, uint32_t (&
 // taddr the TMEM address of (its lane quarter, first column of the tile), n0 the tile's first output column.
 // Every tcgen05.ld is executed by all 32 lanes (rows past M only skip the stores).
 template <int BN>
-__device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint32_t taddr, int row, int n0, const Fixup fx = Fixup()) {
+__device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint32_t taddr, int row, int n0, float& sq,
+                                              float* stage, int cb, int ce, const Fixup fx = Fixup()) {
   const bool row_ok = row < p.M;
   uint32_t r[32];
-  if (p.epi == EPI_ROPE) {
+  if (p.adam_p != nullptr) {
+    // Weight gradient consumed in place: g = accumulator (+ the gradient of earlier chunks for EPI_F32_ACC), then
+    // AdamW on master, moments and bf16 copy at the same position.  The 32 x 32 chunk goes through the warp's staging
+    // tile so that 8 lanes cover 128 contiguous bytes of one row: all seven streams are read and written coalesced.
+    const AdamCoef c = adam_coef(p);
+    const int lane = threadIdx.x & 31;
+    const int row0 = row - lane;                 // first row of this warp's 32
+    const int sub = lane >> 3, col4 = (lane & 7) * 4;
+    for (int c0 = cb; c0 < ce; c0 += 32) {
+      const int gc = n0 + c0;
+      if (gc >= p.N) break;
+      if (c0 + 32 < ce) adam_prefetch_chunk(p, cptr, row, gc + 32);
+      ld_acc32(taddr, c0, r, fx);
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        *reinterpret_cast<float4*>(stage + lane * 32 + 4 * (j ^ (lane & 7))) =
+            make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
+                        __uint_as_float(r[4 * j + 3]));
+      __syncwarp();
+      if (gc + col4 < p.N) {
+        // all loads of the chunk are issued before the first store (the compiler cannot prove the streams distinct,
+        // so it would otherwise serialise one row's loads behind the previous row's stores)
+#pragma unroll
+        for (int hb = 0; hb < 8; hb += 4) {
+          float4 P4[4], M4[4], V4[4], O4[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int rr = (hb + i) * 4 + sub;
+            const bool okr = row0 + rr < p.M;
+            const long long o = (long long)(row0 + rr) * p.ldc + gc + col4;
+            const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+            P4[i] = okr ? *reinterpret_cast<const float4*>(p.adam_p + o) : z;
+            M4[i] = okr ? *reinterpret_cast<const float4*>(p.adam_m + o) : z;
+            V4[i] = okr ? *reinterpret_cast<const float4*>(p.adam_v + o) : z;
+            O4[i] = (okr && p.epi == EPI_F32_ACC) ? *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(cptr) + o) : z;
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int rr = (hb + i) * 4 + sub;
+            if (row0 + rr < p.M) {
+              const long long o = (long long)(row0 + rr) * p.ldc + gc + col4;
+              const float4 g4 = *reinterpret_cast<const float4*>(stage + rr * 32 + 4 * ((col4 >> 2) ^ (rr & 7)));
+              float g[4] = {g4.x, g4.y, g4.z, g4.w};
+              if (p.epi == EPI_F32_ACC) { g[0] += O4[i].x; g[1] += O4[i].y; g[2] += O4[i].z; g[3] += O4[i].w; }
+              float pp[4] = {P4[i].x, P4[i].y, P4[i].z, P4[i].w}, mm[4] = {M4[i].x, M4[i].y, M4[i].z, M4[i].w},
+                    vv[4] = {V4[i].x, V4[i].y, V4[i].z, V4[i].w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                sq += g[e] * g[e];
+                adamw_elem(g[e], p.adam_wd, c, pp[e], mm[e], vv[e]);
+              }
+              *reinterpret_cast<float4*>(p.adam_p + o) = make_float4(pp[0], pp[1], pp[2], pp[3]);
+              *reinterpret_cast<float4*>(p.adam_m + o) = make_float4(mm[0], mm[1], mm[2], mm[3]);
+              *reinterpret_cast<float4*>(p.adam_v + o) = make_float4(vv[0], vv[1], vv[2], vv[3]);
+              uint2 ob;
+              ob.x = pack_bf16(pp[0], pp[1]);
+              ob.y = pack_bf16(pp[2], pp[3]);
+              *reinterpret_cast<uint2*>(p.adam_pb + o) = ob;
+            }
+          }
+        }
+      }
+      __syncwarp();
+    }
+  } else if (p.epi == EPI_ROPE) {
     const int d = p.head_dim;
     const int half = d >> 1;
     const int pos = row_ok ? (row % p.seq) : 0;
     bf16* crow = reinterpret_cast<bf16*>(cptr) + (long long)row * p.ldc;
-    for (int hc = 0; hc < BN; hc += d) {
+    for (int hc = cb; hc < ce; hc += d) {
       const int g0 = n0 + hc;
       if (g0 >= p.N) break;
       if (g0 >= p.rope_cols) {
@@ -248,7 +348,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
     const int f = p.d_ffn;
     bf16* arow = reinterpret_cast<bf16*>(cptr) + (long long)row * p.ldc;
     bf16* gurow = p.gu + (long long)row * (2LL * f);
-    for (int c = 0; c < BN; c += 32) {
+    for (int c = cb; c < ce; c += 32) {
       const int gc = n0 + c;
       if (gc >= p.N) break;
       ld_acc32(taddr, c, r, fx);
@@ -280,14 +380,14 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
       for (int j = 0; j < 4; ++j)
         nxt[j] = (row_ok && gc + 8 * j < p.N) ? *reinterpret_cast<const uint4*>(rrow + gc + 8 * j) : make_uint4(0, 0, 0, 0);
     };
-    fetch(n0);
-    for (int c = 0; c < BN; c += 32) {
+    fetch(n0 + cb);
+    for (int c = cb; c < ce; c += 32) {
       const int gc = n0 + c;
       if (gc >= p.N) break;
       uint4 cur[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) cur[j] = nxt[j];
-      if (c + 32 < BN) fetch(gc + 32);
+      if (c + 32 < ce) fetch(gc + 32);
       ld_acc32(taddr, c, r, fx);
       if (row_ok) {
 #pragma unroll
@@ -311,14 +411,14 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
       for (int j = 0; j < 8; ++j)
         nxt[j] = (row_ok && gc + 4 * j < p.N) ? *reinterpret_cast<const float4*>(crow + gc + 4 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
     };
-    fetch(n0);
-    for (int c = 0; c < BN; c += 32) {
+    fetch(n0 + cb);
+    for (int c = cb; c < ce; c += 32) {
       const int gc = n0 + c;
       if (gc >= p.N) break;
       float4 cur[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j) cur[j] = nxt[j];
-      if (c + 32 < BN) fetch(gc + 32);
+      if (c + 32 < ce) fetch(gc + 32);
       ld_acc32(taddr, c, r, fx);
       if (row_ok) {
 #pragma unroll
@@ -333,7 +433,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
       }
     }
   } else {
-    for (int c = 0; c < BN; c += 32) {
+    for (int c = cb; c < ce; c += 32) {
       const int gc = n0 + c;
       if (gc >= p.N) break;
       ld_acc32(taddr, c, r, fx);
@@ -480,20 +580,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int q = warp & 3;  // TMEM lane quarter this warp may read
     int acc = 0;
     uint32_t acc_phase = 0;
+    float sq = 0.f;  // fused AdamW: this thread's share of the squared gradient norm
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x) {
       const int m0 = (t % tiles_m) * BM;
       const int n0 = (t / tiles_m) * BN;
+      if (p.adam_p != nullptr) adam_prefetch_chunk(p, p.C, m0 + q * 32 + lane, n0);
       bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.err);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
       const int row = m0 + q * 32 + lane;
-      epilogue_tile<BN>(p, p.C, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), row, n0);
+      epilogue_tile<BN>(p, p.C, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), row, n0, sq,
+                        reinterpret_cast<float*>(smem + C::STAGES * C::STAGE_BYTES + C::BAR_BYTES) + q * EPI_STAGE_FLOATS, 0, BN);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(acc));
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
+    }
+    if (p.adam_p != nullptr) {
+      sq = warp_sum(sq);
+      if (lane == 0) p.adam_sq[blockIdx.x * 4 + q] = sq;
     }
   }
 
@@ -526,11 +633,14 @@ struct PairCfg {
   static constexpr int STAGE_BYTES = A_BYTES_ + B_BYTES;
   static constexpr int STAGES = 6;
   static constexpr int TMEM_COLS = 512;
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 256 + 1024;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 256 + EPI_STAGE_BYTES + 1024;
 };
 
+// 10 warps: TMA producer, MMA issuer, and 8 epilogue warps (two per TMEM lane quarter, 128 of the tile's 256 columns each)
+constexpr int PAIR_THREADS = 320;
+
 template <bool A_MN, bool B_MN>
-__global__ void __launch_bounds__(GEMM_THREADS, 1)
+__global__ void __launch_bounds__(PAIR_THREADS, 1)
 gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmDev p) {
   using C = PairCfg;
   constexpr int BN = C::BN;
@@ -557,7 +667,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(tfull_bar(b), 1);   // one multicast commit
-      mbar_init(tempty_bar(b), 8);  // 4 epilogue warps of each CTA, all arriving at the leader
+      mbar_init(tempty_bar(b), 16);  // 8 epilogue warps of each CTA, all arriving at the leader
     }
     *abort_flag = 0;
     mbar_fence_init();
@@ -650,15 +760,20 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       }
     }
   } else {
-    const int q = warp & 3;
+    const int q = warp & 3;                 // TMEM lane quarter this warp may read
+    const int cb = ((warp - 2) >> 2) * 128;  // its half of the tile's columns
+    const int ce = cb + 128;
+    float* stage = reinterpret_cast<float*>(smem + C::STAGES * C::STAGE_BYTES + 256) + (warp - 2) * EPI_STAGE_FLOATS;
     int acc = 0;
     uint32_t acc_phase = 0;
+    float sq = 0.f;  // fused AdamW: this thread's share of the squared gradient norm
     [[maybe_unused]] int piece = 0;
     [[maybe_unused]] const bool tracer = (warp == 2 && lane == 0 && rank == 0);
     if (tracer) FS_GTRACE(pair, 31, 0);
     while (work.next(tile, kb0, kb1, part, split)) {
       const int m0 = (tile % tiles_m) * 256 + (int)rank * BM;
       const int n0 = (tile / tiles_m) * BN;
+      if (p.adam_p != nullptr && !(split && part > 0)) adam_prefetch_chunk(p, p.C, m0 + q * 32 + lane, n0 + cb);
       bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.err);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -671,7 +786,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         // a later K part of a divided tile: leave this partial accumulator in the pair's slot
         float4* dst = reinterpret_cast<float4*>(p.slots) + (long long)pair * SLOT_F4 + slot_f4;
         uint32_t r[32];
-        for (int c = 0; c < BN && n0 + c < p.N; c += 32) {
+        for (int c = cb; c < ce && n0 + c < p.N; c += 32) {
           tmem_ld32(taddr + c, r);
           tmem_ld_wait();
 #pragma unroll
@@ -693,14 +808,14 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           fx.base = reinterpret_cast<const float4*>(p.slots) + (long long)(pair + 1) * SLOT_F4 + slot_f4;
           int got = 1;
           if (lane == 0)
-            for (int s = 0; s < fx.n && got; ++s) got = flag_wait(p.flags + pair + 1 + s, 8, abort_flag, p.err) ? 1 : 0;
+            for (int s = 0; s < fx.n && got; ++s) got = flag_wait(p.flags + pair + 1 + s, 16, abort_flag, p.err) ? 1 : 0;
           got = __shfl_sync(0xffffffffu, got, 0);
           if (!got) break;
           if (tracer) FS_GTRACE(pair, piece, 1);
         } else if (p.ksplit > 1) {
           cptr = reinterpret_cast<float*>(p.C) + (long long)part * p.split_stride;  // this K part's own fp32 partial output
         }
-        epilogue_tile<BN>(p, cptr, taddr, row, n0, fx);
+        epilogue_tile<BN>(p, cptr, taddr, row, n0, sq, stage, cb, ce, fx);
       }
       tc_fence_before();
       __syncwarp();
@@ -709,6 +824,10 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       ++piece;
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
+    }
+    if (p.adam_p != nullptr) {
+      sq = warp_sum(sq);
+      if (lane == 0) p.adam_sq[blockIdx.x * 8 + (warp - 2)] = sq;
     }
   }
 
@@ -734,9 +853,16 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   }
 }
 
-// out[r, c] (+)= sum over K parts of partial[s][r, c], parts added in index order (deterministic)
-__global__ void splitk_reduce_kernel(const float* __restrict__ partial, int nsplit, long long stride, float* __restrict__ out,
-                                     long long ldc, int M, int N, int accumulate) {
+// out[r, c] (+)= sum over K parts of partial[s][r, c], parts added in index order (deterministic).  ADAM: the sum is
+// the finished gradient and goes straight into the AdamW update at (r, c) instead of being stored.
+template <bool ADAM>
+__global__ void __launch_bounds__(256)
+splitk_reduce_kernel(const float* __restrict__ partial, int nsplit, long long stride, float* __restrict__ out, long long ldc,
+                     int M, int N, int accumulate, const GemmDev p) {
+  __shared__ float s_sq[8];
+  float sq = 0.f;
+  AdamCoef cf = {};
+  if (ADAM) cf = adam_coef(p);
   const long long n4 = (long long)M * (N / 4);
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (long long)gridDim.x * blockDim.x) {
     const long long r = i / (N / 4);
@@ -746,11 +872,52 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ partial, int nspl
       const float4 v = *reinterpret_cast<const float4*>(partial + s * stride + r * N + c);
       a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
     }
-    *reinterpret_cast<float4*>(out + r * ldc + c) = a;
+    if (!ADAM) {
+      *reinterpret_cast<float4*>(out + r * ldc + c) = a;
+    } else {
+      const long long o = r * ldc + c;
+      const float g[4] = {a.x, a.y, a.z, a.w};
+      const float4 p4 = *reinterpret_cast<const float4*>(p.adam_p + o);
+      const float4 m4 = *reinterpret_cast<const float4*>(p.adam_m + o);
+      const float4 v4 = *reinterpret_cast<const float4*>(p.adam_v + o);
+      float pp[4] = {p4.x, p4.y, p4.z, p4.w}, mm[4] = {m4.x, m4.y, m4.z, m4.w}, vv[4] = {v4.x, v4.y, v4.z, v4.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        sq += g[e] * g[e];
+        adamw_elem(g[e], p.adam_wd, cf, pp[e], mm[e], vv[e]);
+      }
+      *reinterpret_cast<float4*>(p.adam_p + o) = make_float4(pp[0], pp[1], pp[2], pp[3]);
+      *reinterpret_cast<float4*>(p.adam_m + o) = make_float4(mm[0], mm[1], mm[2], mm[3]);
+      *reinterpret_cast<float4*>(p.adam_v + o) = make_float4(vv[0], vv[1], vv[2], vv[3]);
+      uint2 ob;
+      ob.x = pack_bf16(pp[0], pp[1]);
+      ob.y = pack_bf16(pp[2], pp[3]);
+      *reinterpret_cast<uint2*>(p.adam_pb + o) = ob;
+    }
+  }
+  if (ADAM) {
+    sq = warp_sum(sq);
+    if ((threadIdx.x & 31) == 0) s_sq[threadIdx.x >> 5] = sq;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float tot = 0.f;
+      for (int w = 0; w < 8; ++w) tot += s_sq[w];
+      p.adam_sq[blockIdx.x] = tot;
+    }
   }
 }
 
 // ---------------------------------------------------------------- host side
+void set_adam(GemmDev& p, const GemmArgs& a) {
+  p.adam_p = nullptr; p.adam_m = nullptr; p.adam_v = nullptr; p.adam_pb = nullptr; p.adam_sc = nullptr; p.adam_sq = nullptr;
+  p.adam_lr = p.adam_beta1 = p.adam_beta2 = p.adam_eps = p.adam_wd = 0.f;
+  if (!a.adam) return;
+  p.adam_p = a.adam->p; p.adam_m = a.adam->m; p.adam_v = a.adam->v; p.adam_pb = a.adam->pb;
+  p.adam_sc = reinterpret_cast<const StepScalars*>(a.adam->scalars); p.adam_sq = a.adam->sq_slots;
+  p.adam_lr = a.adam->lr; p.adam_beta1 = a.adam->beta1; p.adam_beta2 = a.adam->beta2; p.adam_eps = a.adam->eps;
+  p.adam_wd = a.adam->wd;
+}
+
 int sm_count() {
   static int n = 0;
   if (n == 0) {
@@ -780,6 +947,7 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
   p.C = a.C; p.resid = a.resid; p.gu = a.gu; p.rope_cos = a.rope_cos; p.rope_sin = a.rope_sin; p.err = a.err;
   p.ldc = a.ldc; p.M = a.M; p.N = a.N; p.K = a.K; p.epi = a.epi;
   p.seq = a.seq; p.head_dim = a.head_dim; p.rope_cols = a.rope_cols; p.d_ffn = a.d_ffn;
+  set_adam(p, a);
   p.ksplit = 1; p.split_stride = 0; p.balanced = 0; p.sw_first = 0; p.sw_parts = 1; p.sw_kpb = 0; p.flags = nullptr; p.slots = nullptr;
   const int tiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN);
   const int grid = tiles < sm_count() ? tiles : sm_count();
@@ -805,6 +973,7 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
   p.C = a.C; p.resid = a.resid; p.gu = a.gu; p.rope_cos = a.rope_cos; p.rope_sin = a.rope_sin; p.err = a.err;
   p.ldc = a.ldc; p.M = a.M; p.N = a.N; p.K = a.K; p.epi = a.epi;
   p.seq = a.seq; p.head_dim = a.head_dim; p.rope_cols = a.rope_cols; p.d_ffn = a.d_ffn;
+  set_adam(p, a);
   const int tiles = ((a.M + 255) / 256) * ((a.N + 255) / 256);
   const int max_pairs = sm_count() / 2;
   // scratch layout: 256 arrival counters (kept zero between launches), then fp32 partial tiles
@@ -826,7 +995,7 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
   }
   p.ksplit = ksplit;
   p.split_stride = (long long)a.M * a.N;
-  if (ksplit > 1) { p.C = data; p.ldc = a.N; p.epi = EPI_F32; }
+  if (ksplit > 1) { p.C = data; p.ldc = a.N; p.epi = EPI_F32; p.adam_p = nullptr; }  // the reduction applies AdamW instead
   // balanced schedule: a last wave that would keep at most half of the pairs busy is divided along K
   p.balanced = 0; p.sw_first = tiles; p.sw_parts = 1; p.sw_kpb = kblocks; p.flags = flags; p.slots = data;
   const int left = tiles % max_pairs;
@@ -854,7 +1023,7 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs, 1, 1);
-  cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
+  cfg.blockDim = dim3(PAIR_THREADS, 1, 1);
   cfg.dynamicSmemBytes = C::SMEM_BYTES;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
@@ -864,12 +1033,21 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  g_gemm_last_launches = ksplit > 1 ? 2 : 1;
   cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, p);
   if (e != cudaSuccess || ksplit == 1) return e;
   const long long n4 = (long long)a.M * (a.N / 4);
-  const int blocks = (int)((n4 + 255) / 256 < 1184 ? (n4 + 255) / 256 : 1184);
-  splitk_reduce_kernel<<<blocks, 256, 0, stream>>>(data, ksplit, p.split_stride, reinterpret_cast<float*>(a.C),
-                                                   a.ldc, a.M, a.N, a.epi == EPI_F32_ACC ? 1 : 0);
+  if (a.adam) {
+    GemmDev pa = p;
+    set_adam(pa, a);
+    const int blocks = (int)((n4 + 255) / 256 < kAdamFuseSlots ? (n4 + 255) / 256 : kAdamFuseSlots);
+    splitk_reduce_kernel<true><<<blocks, 256, 0, stream>>>(data, ksplit, p.split_stride, reinterpret_cast<float*>(a.C), a.ldc,
+                                                           a.M, a.N, a.epi == EPI_F32_ACC ? 1 : 0, pa);
+  } else {
+    const int blocks = (int)((n4 + 255) / 256 < 1184 ? (n4 + 255) / 256 : 1184);
+    splitk_reduce_kernel<false><<<blocks, 256, 0, stream>>>(data, ksplit, p.split_stride, reinterpret_cast<float*>(a.C),
+                                                            a.ldc, a.M, a.N, a.epi == EPI_F32_ACC ? 1 : 0, p);
+  }
   return cudaGetLastError();
 }
 
@@ -887,6 +1065,7 @@ int g_gemm_force_bn = 0;
 int g_gemm_pairs = 1;  // development knob: 1 = CTA-pair kernel for outputs of at least 256 x 256, 0 = single-CTA kernel only  // development knob: 0 = choose by tile count, 128 or 256 = force that tile width
 
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream) {
+  g_gemm_last_launches = 1;
   if (a.M <= 0 || a.N <= 0 || a.K <= 0 || !a.A || !a.B || !a.C || !a.err) return cudaErrorInvalidValue;
   if ((a.N & 7) || (a.lda & 7) || (a.ldb & 7) || (a.ldc & 3)) return cudaErrorInvalidValue;
   if ((a.a_mn ? a.M : a.K) & 7) return cudaErrorInvalidValue;
@@ -894,6 +1073,9 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream) {
   if ((reinterpret_cast<uintptr_t>(a.A) | reinterpret_cast<uintptr_t>(a.B) | reinterpret_cast<uintptr_t>(a.C)) & 15)
     return cudaErrorInvalidValue;
   if (a.epi == EPI_BF16_RESID && !a.resid) return cudaErrorInvalidValue;
+  if (a.adam && ((a.epi != EPI_F32 && a.epi != EPI_F32_ACC) || !a.adam->p || !a.adam->m || !a.adam->v || !a.adam->pb ||
+                 !a.adam->scalars || !a.adam->sq_slots))
+    return cudaErrorInvalidValue;
   if (a.epi == EPI_ROPE && (!a.rope_cos || !a.rope_sin || (a.head_dim != 64 && a.head_dim != 128) || a.seq <= 0 ||
                             a.rope_cols % a.head_dim || a.N % a.head_dim))
     return cudaErrorInvalidValue;

@@ -16,6 +16,21 @@ enum GemmEpilogue : int {
   EPI_SWIGLU = 5       // acc columns alternate 16 gate / 16 up: writes gate|up to gu bf16 [M, 2f] and a = R(silu(G) U) to C [M, f]
 };
 
+// Weight-gradient GEMMs (EPI_F32 / EPI_F32_ACC) can hand the finished gradient straight to AdamW instead of storing it:
+// the epilogue reads the master weight and both moments at the gradient's position, applies the update, and writes
+// master, moments and the bf16 copy.  Only valid with gradient clipping off (the update then does not depend on the
+// global norm); the squared norm is still summed, one partial per epilogue warp, into sq_slots.
+struct AdamFuse {
+  float* p = nullptr;   // fp32 master weights, same shape and row stride (ldc) as C
+  float* m = nullptr;   // first moment
+  float* v = nullptr;   // second moment
+  bf16* pb = nullptr;   // bf16 copy of the weights
+  const void* scalars = nullptr;  // device StepScalars (bias corrections of the current step)
+  float lr = 0, beta1 = 0, beta2 = 0, eps = 0, wd = 0;
+  float* sq_slots = nullptr;  // kAdamFuseSlots floats, zeroed by the caller; unused ones stay zero
+};
+constexpr int kAdamFuseSlots = 1280;
+
 struct GemmArgs {
   const bf16* A = nullptr;  // a_mn = 0: [M, lda] row-major (k contiguous); a_mn = 1: [K, lda] row-major (m contiguous)
   int a_mn = 0;
@@ -45,6 +60,7 @@ struct GemmArgs {
   float* scratch = nullptr;
   size_t scratch_bytes = 0;
   bool scratch_reset = false;
+  const AdamFuse* adam = nullptr;
 };
 
 // Enqueues the contraction on `stream`.  Returns cudaErrorInvalidValue for shapes it does not take.
@@ -52,6 +68,7 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream);
 
 extern int g_gemm_force_bn;
 extern int g_gemm_pairs;
+extern int g_gemm_last_launches;  // kernels the last launch_gemm call enqueued
 extern int g_gemm_balanced;
 
 }  // namespace fs

@@ -81,6 +81,14 @@ struct ft_model {
   int lastB = 0, lastS = 0;
   bool have_bwd = false;
 
+  // AdamW inside the weight-gradient GEMM epilogues (clipping off): the train step then never stores those gradients
+  bool fused_update = true;   // policy switch (ft_set_fused_update)
+  bool fusing = false;        // true while a step that fuses is being enqueued
+  int fuse_idx = 0;           // next slot region of fuse_sq
+  float* fuse_sq = nullptr;   // partial sums of the squared gradient norm: [4L+1][kAdamFuseSlots] + 2 x [kSqnormBlocks]
+  std::vector<AdamFuse> fuse_args;  // kept alive until the launches are enqueued
+  size_t fuse_sq_count() const { return (size_t)(4 * L + 1) * kAdamFuseSlots + 2 * (size_t)kSqnormBlocks; }
+
   // whole-step CUDA graph: the first step of a (B, S) runs launch by launch, the second is captured, later ones replay
   bool graph_enabled = false;
   int graph_B = 0, graph_S = 0, warm_B = 0, warm_S = 0;
@@ -195,6 +203,7 @@ size_t carve(ft_model* m, uint8_t* base) {
   m->delta = cv.take<float>(T * c.n_heads);
   m->norm_partial = cv.take<float>((size_t)elementwise_blocks_for_norm((int)T) * h);
   m->sq_partial = cv.take<float>(kSqnormBlocks);
+  m->fuse_sq = cv.take<float>(m->fuse_sq_count());
   m->splitk = cv.take<float>(kSplitKFloats);
   m->z = cv.take<float>((size_t)m->ce_chunk * V);
   m->dz = cv.take<bf16>((size_t)m->ce_chunk * V);
@@ -238,7 +247,7 @@ ft_status cuda_fail(ft_model* m, cudaError_t e, const char* where) {
     prof_begin(m);                                                                          \
     cudaError_t e__ = launch_gemm(args, m->stream);                                         \
     if (e__ != cudaSuccess) return cuda_fail(m, e__, "launch_gemm");                        \
-    m->launches += 1;                                                                       \
+    m->launches += g_gemm_last_launches;                                                    \
     prof_end(m, FT_PROF_GEMM, 2.0 * (double)(args).M * (double)(args).N * (double)(args).K, 1, prof_shape_index(m, args)); \
   } while (0)
 
@@ -304,6 +313,19 @@ GemmArgs gemm_base(ft_model* m) {
   return g;
 }
 
+// AdamW arguments for the weight-gradient GEMM of parameter wi (a matrix: decayed), with the next norm-slot region
+const AdamFuse* fuse_for(ft_model* m, int wi) {
+  const size_t off = m->params[wi].offset;
+  AdamFuse a;
+  a.p = m->master + off; a.m = m->adam_m + off; a.v = m->adam_v + off; a.pb = m->pbf + off;
+  a.scalars = m->sc;
+  a.lr = m->cfg.lr; a.beta1 = m->cfg.beta1; a.beta2 = m->cfg.beta2; a.eps = m->cfg.adam_eps; a.wd = m->cfg.weight_decay;
+  a.sq_slots = m->fuse_sq + (size_t)m->fuse_idx * kAdamFuseSlots;
+  m->fuse_idx += 1;
+  m->fuse_args.push_back(a);
+  return &m->fuse_args.back();
+}
+
 // forward of layer l from m->x[l] into activation slot `a`, output to m->x[l+1]
 ft_status layer_forward(ft_model* m, int l, LayerActs& a, int B, int S) {
   const int T = B * S, h = m->h, f = m->f, hq = m->hq, nqkv = m->nqkv;
@@ -359,6 +381,7 @@ ft_status linear_backward(ft_model* m, const bf16* dY, const bf16* X, int wi, bf
     GemmArgs g = gemm_base(m);
     g.A = dY; g.a_mn = 1; g.lda = n_out; g.B = X; g.b_mn = 1; g.ldb = n_in; g.C = m->gr(wi); g.ldc = n_in;
     g.M = n_out; g.N = n_in; g.K = T; g.epi = EPI_F32;
+    if (m->fusing) g.adam = fuse_for(m, wi);
     FT_GEMM(g);
   }
   return FT_OK;
@@ -404,12 +427,22 @@ ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
 }
 
 // forward (+ backward when with_bwd) of one batch; everything is enqueued, nothing is synchronised
-ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* lab, int B, int S, bool with_bwd) {
+ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* lab, int B, int S, bool with_bwd,
+                               bool fuse = false) {
   if (!m || !tok || !lab) return fail(m, FT_EINVAL, "null argument");
   if (B < 1 || S < 1 || B > m->cfg.max_batch || S > m->cfg.max_seq) return fail(m, FT_EINVAL, "B or S out of range");
   const int T = B * S, h = m->h, V = m->V, L = m->L;
   cudaStream_t st = m->stream;
   m->lastB = B; m->lastS = S; m->have_bwd = false;
+  m->fusing = fuse && with_bwd;
+  m->fuse_idx = 0;
+  m->fuse_args.clear();
+  m->fuse_args.reserve((size_t)4 * L + 1);  // pointers into it are handed to the launcher
+  if (m->fusing) {
+    // the optimizer step counter and bias corrections must be current before the first weight-gradient epilogue
+    FT_CUDA(cudaMemsetAsync(m->fuse_sq, 0, m->fuse_sq_count() * sizeof(float), st));
+    FT_LAUNCH(FT_PROF_OPTIMIZER, 0.0, advance_step(m->sc, hyper(m), st));
+  }
 
   FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T, count_labels(lab, T, m->sc, st));
   FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T * h, embed_fwd(tok, m->wb(0), m->x[0], T, h, V, st));
@@ -443,6 +476,7 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
         GemmArgs g = gemm_base(m);
         g.A = m->dz; g.a_mn = 1; g.lda = V; g.B = m->hF + (size_t)r0 * h; g.b_mn = 1; g.ldb = h; g.C = m->gr(i_head);
         g.ldc = h; g.M = V; g.N = h; g.K = rows; g.epi = chunk == 0 ? EPI_F32 : EPI_F32_ACC;
+        if (m->fusing && r0 + rows >= T) g.adam = fuse_for(m, i_head);  // the last chunk completes the gradient
         FT_GEMM(g);
       }
     }
@@ -464,7 +498,7 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
     if (s) return s;
   }
   FT_LAUNCH(FT_PROF_ELEMENTWISE, 2.0 * T * h + 4.0 * V * h, embed_bwd(tok, m->dxA, m->gr(0), m->keys, T, h, V, st));
-  m->have_bwd = true;
+  m->have_bwd = !m->fusing;  // a fusing step leaves no gradients of the matrices behind
   return FT_OK;
 }
 
@@ -483,6 +517,25 @@ ft_status run_update(ft_model* m) {
               adamw_with_norm(m->master, m->adam_m, m->adam_v, m->grad, m->pbf, m->arena, m->n_decay, m->sq_partial,
                               m->sc, hp, st));
   }
+  return FT_OK;
+}
+
+// What is left of the update after a fusing backward: the embedding table and the gains (their gradients do not
+// come from a GEMM), and the gradient norm from all partial sums in slot order.
+ft_status run_update_rest(ft_model* m) {
+  cudaStream_t st = m->stream;
+  const AdamHyper hp = hyper(m);
+  const size_t fused_slots = (size_t)(4 * m->L + 1) * kAdamFuseSlots;
+  const size_t embed_span = (m->params[0].numel() + 127) / 128 * 128;  // embed is the first tensor of the arenas
+  FT_LAUNCH(FT_PROF_OPTIMIZER, 30.0 * embed_span,
+            adamw_range_with_norm(m->master, m->adam_m, m->adam_v, m->grad, m->pbf, embed_span, embed_span,
+                                  m->fuse_sq + fused_slots, m->sc, hp, st));
+  const size_t g0 = m->n_decay, gn = m->arena - m->n_decay;
+  FT_LAUNCH(FT_PROF_OPTIMIZER, 30.0 * gn,
+            adamw_range_with_norm(m->master + g0, m->adam_m + g0, m->adam_v + g0, m->grad + g0, m->pbf + g0, gn, 0,
+                                  m->fuse_sq + fused_slots + kSqnormBlocks, m->sc, hp, st));
+  FT_LAUNCH(FT_PROF_OPTIMIZER, 4.0 * m->fuse_sq_count(), sqnorm_final(m->fuse_sq, (int)m->fuse_sq_count(), m->sc, hp, st));
+  m->fusing = false;
   return FT_OK;
 }
 
@@ -607,9 +660,10 @@ ft_status ft_init_model(const ft_config* cfg, uint64_t seed, void* dev_workspace
 
 // One full step enqueued launch by launch.
 static ft_status step_direct(ft_model* m, const int32_t* tok, const int32_t* lab, int32_t B, int32_t S) {
-  ft_status s = run_forward_backward(m, tok, lab, B, S, true);
+  const bool fuse = m->fused_update && m->cfg.max_grad_norm <= 0.f && !m->cfg.debug_taps;
+  ft_status s = run_forward_backward(m, tok, lab, B, S, true, fuse);
   if (s) return s;
-  return run_update(m);
+  return fuse ? run_update_rest(m) : run_update(m);
 }
 
 // The same step through a captured graph when that is enabled and possible.  The graph reads the token and label
@@ -658,7 +712,8 @@ static ft_status step_maybe_graphed(ft_model* m, const int32_t* tok, const int32
   FT_CUDA(cudaGraphLaunch(m->graph_exec, m->stream));
   m->launches += m->graph_launches;
   m->graph_replays += 1;
-  m->lastB = B; m->lastS = S; m->have_bwd = true;
+  m->lastB = B; m->lastS = S;
+  m->have_bwd = !(m->fused_update && m->cfg.max_grad_norm <= 0.f);  // a fusing step leaves no matrix gradients behind
   return FT_OK;
 }
 
@@ -668,6 +723,13 @@ ft_status ft_train_step(ft_model* m, const int32_t* dev_tokens, const int32_t* d
   ft_status s = step_maybe_graphed(m, dev_tokens, dev_labels, B, S);
   if (s) return s;
   if (host_loss || host_gnorm) return finish(m, host_loss, host_gnorm);
+  return FT_OK;
+}
+
+ft_status ft_set_fused_update(ft_model* m, int32_t enable) {
+  if (!m) return FT_EINVAL;
+  m->fused_update = enable != 0;
+  if (m->graph_exec) { cudaGraphExecDestroy(m->graph_exec); m->graph_exec = nullptr; }  // captured with the old setting
   return FT_OK;
 }
 

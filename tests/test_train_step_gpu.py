@@ -279,3 +279,39 @@ def test_ten_step_loss_and_gradient_norm_trajectory_matches_oracle():
         e = rel_l2(model.get_param(name), st.params[name])
         assert e < 1e-2, (name, e)
     model.close()
+
+
+@pytest.mark.parametrize("shape", ["c1", "split_k", "balanced"])
+def test_adamw_inside_the_weight_gradient_epilogue_equals_the_separate_optimizer_pass(shape):
+    """Clipping is off, so the train step applies AdamW where the weight gradient is finished (GEMM epilogue, split-K
+    reduction, or the epilogue that completes a tile divided along K).  Same update function, same gradient bits:
+    parameters, moments, bf16 copies and losses must equal the unfused step bit for bit over several steps; the
+    gradient norm is summed in another order and agrees to rounding."""
+    from paper_2609_13645_b200 import binding as B
+    if shape == "c1":
+        ocfg, _ = _c1()
+        Bsz, S = 2, 128
+    elif shape == "split_k":   # weight gradients with few tiles and 2048 tokens: K split over 4 parts
+        ocfg = oracle_config(n_layers=2, d_model=512, n_heads=4, n_kv_heads=2, head_dim=128, d_ffn=1024, vocab=2048)
+        Bsz, S = 2, 1024
+    else:                      # gate/up gradient of 18 x 5 = 90 tiles: the 16 tiles past the 74 pairs are divided
+        ocfg = oracle_config(n_layers=1, d_model=1280, n_heads=10, n_kv_heads=2, head_dim=128, d_ffn=2304, vocab=2048)
+        Bsz, S = 1, 1024
+    runs = []
+    for fused in (True, False):
+        model = B.Model(lib_config(B, ocfg, Bsz, S), seed=3)
+        model.set_fused_update(fused)
+        out = []
+        for s in range(3):
+            tok, lab = SI.batch(ocfg.vocab, Bsz, S, "uniform", step=s)
+            out.append(model.train_step(to_dev(tok), to_dev(lab)))
+        runs.append((model, out))
+    (mf, lf), (mu, lu) = runs
+    assert np.array_equal(np.float32([x[0] for x in lf]).view(np.uint32), np.float32([x[0] for x in lu]).view(np.uint32))
+    for (_, gf), (_, gu) in zip(lf, lu):
+        assert abs(gf - gu) <= 1e-5 * gu
+    for a, b in zip(_state_bits(mf), _state_bits(mu)):
+        assert np.array_equal(a, b)
+    assert mf.step == 3 and mu.step == 3
+    mf.close()
+    mu.close()
