@@ -636,7 +636,10 @@ struct PairCfg {
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 256 + EPI_STAGE_BYTES + 1024;
 };
 
-// 10 warps: TMA producer, MMA issuer, and 8 epilogue warps (two per TMEM lane quarter, 128 of the tile's 256 columns each)
+// Warps: TMA producer, MMA issuer, then the epilogue warps.  Launched with 192 threads there are four (one per TMEM lane
+// quarter, all 256 columns of the tile each); with 320 there are eight (two per quarter, 128 columns each), which the
+// fused AdamW epilogue needs to keep enough loads in flight.  (Eight warps cost the plain epilogues about 4 % of tensor
+// activity, measured on the gate/up shape, so they are used only where the epilogue is the heavy part.)
 constexpr int PAIR_THREADS = 320;
 
 template <bool A_MN, bool B_MN>
@@ -667,7 +670,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(tfull_bar(b), 1);   // one multicast commit
-      mbar_init(tempty_bar(b), 16);  // 8 epilogue warps of each CTA, all arriving at the leader
+      mbar_init(tempty_bar(b), 2 * (blockDim.x / 32 - 2));  // the epilogue warps of both CTAs, all arriving at the leader
     }
     *abort_flag = 0;
     mbar_fence_init();
@@ -761,8 +764,9 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
   } else {
     const int q = warp & 3;                 // TMEM lane quarter this warp may read
-    const int cb = ((warp - 2) >> 2) * 128;  // its half of the tile's columns
-    const int ce = cb + 128;
+    const int ncols = blockDim.x == PAIR_THREADS ? 128 : 256;  // columns of the tile per epilogue warp
+    const int cb = ((warp - 2) >> 2) * ncols;
+    const int ce = cb + ncols;
     float* stage = reinterpret_cast<float*>(smem + C::STAGES * C::STAGE_BYTES + 256) + (warp - 2) * EPI_STAGE_FLOATS;
     int acc = 0;
     uint32_t acc_phase = 0;
@@ -808,7 +812,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           fx.base = reinterpret_cast<const float4*>(p.slots) + (long long)(pair + 1) * SLOT_F4 + slot_f4;
           int got = 1;
           if (lane == 0)
-            for (int s = 0; s < fx.n && got; ++s) got = flag_wait(p.flags + pair + 1 + s, 16, abort_flag, p.err) ? 1 : 0;
+            for (int s = 0; s < fx.n && got; ++s) got = flag_wait(p.flags + pair + 1 + s, 2 * ((int)blockDim.x / 32 - 2), abort_flag, p.err) ? 1 : 0;
           got = __shfl_sync(0xffffffffu, got, 0);
           if (!got) break;
           if (tracer) FS_GTRACE(pair, piece, 1);
@@ -1023,7 +1027,7 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs, 1, 1);
-  cfg.blockDim = dim3(PAIR_THREADS, 1, 1);
+  cfg.blockDim = dim3(a.adam ? PAIR_THREADS : GEMM_THREADS, 1, 1);
   cfg.dynamicSmemBytes = C::SMEM_BYTES;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
