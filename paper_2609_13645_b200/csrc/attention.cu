@@ -12,37 +12,53 @@ namespace fs {
 namespace {
 
 // ============================================================================ backward pre-pass
-// delta[b, n, i] = sum_k dO[b,i,n,k] O[b,i,n,k]; one warp per (token, head).
+// delta[b, n, i] = sum_k dO[b,i,n,k] O[b,i,n,k].  D/8 lanes share one (token, head) row with one 16-byte load per
+// tensor each; every warp keeps two groups of rows in flight and walks the rows grid-strided.  The D products of a
+// row are added in a fixed order (8 per lane, then a butterfly over the row's lanes).
 template <int D>
-__global__ void attn_delta_kernel(const bf16* __restrict__ o, const bf16* __restrict__ d_o, float* __restrict__ delta,
-                                  int B, int S, int n_heads) {
-  const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int lane = threadIdx.x & 31;
+__global__ void __launch_bounds__(256)
+attn_delta_kernel(const bf16* __restrict__ o, const bf16* __restrict__ d_o, float* __restrict__ delta, int B, int S,
+                  int n_heads) {
+  constexpr int LPR = D / 8;    // lanes per row
+  constexpr int RPW = 32 / LPR;  // rows per warp and load
+  const int lane = threadIdx.x & 31, sub = lane / LPR, l = lane % LPR;
   const long long total = (long long)B * S * n_heads;
-  if (w >= total) return;
-  const int n = (int)(w % n_heads);
-  const long long tok = w / n_heads;
-  const bf16* po = o + (tok * n_heads + n) * D;
-  const bf16* pd = d_o + (tok * n_heads + n) * D;
-  float acc = 0.f;
+  const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long base = (((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5) * (2 * RPW); base < total;
+       base += nwarps * (2 * RPW)) {
+    uint4 a[2], d[2];
 #pragma unroll
-  for (int c = lane * 2; c < D; c += 64) {
-    const uint32_t a = *reinterpret_cast<const uint32_t*>(po + c);
-    const uint32_t d = *reinterpret_cast<const uint32_t*>(pd + c);
-    acc += bf16_lo(a) * bf16_lo(d) + bf16_hi(a) * bf16_hi(d);
-  }
-  acc = warp_sum(acc);
-  if (lane == 0) {
-    const int b = (int)(tok / S), i = (int)(tok % S);
-    delta[((long long)b * n_heads + n) * S + i] = acc;
+    for (int u = 0; u < 2; ++u) {
+      const long long w = base + u * RPW + sub;
+      const bool ok = w < total;
+      a[u] = ok ? *reinterpret_cast<const uint4*>(o + w * D + l * 8) : make_uint4(0, 0, 0, 0);
+      d[u] = ok ? *reinterpret_cast<const uint4*>(d_o + w * D + l * 8) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      float acc = bf16_lo(a[u].x) * bf16_lo(d[u].x) + bf16_hi(a[u].x) * bf16_hi(d[u].x);
+      acc += bf16_lo(a[u].y) * bf16_lo(d[u].y) + bf16_hi(a[u].y) * bf16_hi(d[u].y);
+      acc += bf16_lo(a[u].z) * bf16_lo(d[u].z) + bf16_hi(a[u].z) * bf16_hi(d[u].z);
+      acc += bf16_lo(a[u].w) * bf16_lo(d[u].w) + bf16_hi(a[u].w) * bf16_hi(d[u].w);
+#pragma unroll
+      for (int off = LPR / 2; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+      const long long w = base + u * RPW + sub;
+      if (l == 0 && w < total) {
+        const int n = (int)(w % n_heads);
+        const long long tok = w / n_heads;
+        const int b = (int)(tok / S), i = (int)(tok % S);
+        delta[((long long)b * n_heads + n) * S + i] = acc;
+      }
+    }
   }
 }
 
 }  // namespace
 
 cudaError_t attention_delta(const bf16* o, const bf16* d_o, float* delta, int B, int S, int nh, int d, cudaStream_t st) {
-  const long long warps = (long long)B * S * nh;
-  const int blocks = (int)((warps * 32 + 255) / 256);
+  const long long rows = (long long)B * S * nh;
+  const long long want = (rows * (d / 8) + 2 * 256 - 1) / (2 * 256);  // blocks if every thread took one load pair
+  const int blocks = (int)(want < 148 * 8 ? (want > 0 ? want : 1) : 148 * 8);
   if (d == 64) attn_delta_kernel<64><<<blocks, 256, 0, st>>>(o, d_o, delta, B, S, nh);
   else if (d == 128) attn_delta_kernel<128><<<blocks, 256, 0, st>>>(o, d_o, delta, B, S, nh);
   else return cudaErrorInvalidValue;

@@ -352,8 +352,10 @@ __global__ void bitonic_global_kernel(unsigned long long* __restrict__ keys, int
   }
 }
 
-// block i works only if sorted position i starts a run of equal tokens; its 8 warps take contiguous eighths of the
-// run (position order), and the eight partial rows are added in warp order.
+// block (i, y) works only if sorted position i starts a run of equal tokens; it owns columns [256 y, 256 y + 256) of
+// that token's gradient row.  Its 8 warps take contiguous eighths of the run (position order, four rows in flight,
+// added in position order), and the eight partial rows are added in warp order.  A token as frequent as id 0 of a
+// Zipf stream (14 % of the positions) is thus spread over h / 256 blocks instead of one.
 __global__ void __launch_bounds__(256)
 embed_bwd_kernel(const unsigned long long* __restrict__ keys, const bf16* __restrict__ dx, float* __restrict__ dE, int T,
                  int h) {
@@ -376,29 +378,43 @@ embed_bwd_kernel(const unsigned long long* __restrict__ keys, const bf16* __rest
   const int len = s_end - i;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r0 = i + (int)(((long long)len * warp) / 8), r1 = i + (int)(((long long)len * (warp + 1)) / 8);
-  for (int slab = 0; slab < h; slab += 256) {
-    const int c = slab + lane * 8;
-    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    if (c < h) {
-      for (int rpos = r0; rpos < r1; ++rpos) {
-        const unsigned pos = (unsigned)(keys[rpos] & 0xffffffffull);
+  const int slab = blockIdx.y * 256;
+  const int c = slab + lane * 8;
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  if (c < h) {
+    int rpos = r0;
+    for (; rpos + 4 <= r1; rpos += 4) {
+      uint4 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const unsigned pos = (unsigned)(keys[rpos + u] & 0xffffffffull);
+        v[u] = *reinterpret_cast<const uint4*>(dx + (long long)pos * h + c);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
         float f[8];
-        unpack8(*reinterpret_cast<const uint4*>(dx + (long long)pos * h + c), f);
+        unpack8(v[u], f);
 #pragma unroll
         for (int e = 0; e < 8; ++e) acc[e] += f[e];
       }
     }
+    for (; rpos < r1; ++rpos) {
+      const unsigned pos = (unsigned)(keys[rpos] & 0xffffffffull);
+      float f[8];
+      unpack8(*reinterpret_cast<const uint4*>(dx + (long long)pos * h + c), f);
 #pragma unroll
-    for (int e = 0; e < 8; ++e) s_part[warp][lane * 8 + e] = acc[e];
-    __syncthreads();
-    const int col = slab + threadIdx.x;
-    if (col < h) {
-      float tot = 0.f;
-#pragma unroll
-      for (int w = 0; w < 8; ++w) tot += s_part[w][threadIdx.x];
-      dE[(long long)tokid * h + col] = tot;
+      for (int e = 0; e < 8; ++e) acc[e] += f[e];
     }
-    __syncthreads();
+  }
+#pragma unroll
+  for (int e = 0; e < 8; ++e) s_part[warp][lane * 8 + e] = acc[e];
+  __syncthreads();
+  const int col = slab + threadIdx.x;
+  if (col < h) {
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += s_part[w][threadIdx.x];
+    dE[(long long)tokid * h + col] = tot;
   }
 }
 
@@ -618,7 +634,7 @@ int embed_bwd(const int32_t* tok, const bf16* dx, float* dE, unsigned long long*
     ++launches;
   }
   if (cudaMemsetAsync(dE, 0, (size_t)vocab * h * sizeof(float), st) != cudaSuccess) return -1;
-  embed_bwd_kernel<<<T, 256, 0, st>>>(keys, dx, dE, T, h);
+  embed_bwd_kernel<<<dim3(T, (h + 255) / 256), 256, 0, st>>>(keys, dx, dE, T, h);
   ++launches;
   return ok(launches);
 }
