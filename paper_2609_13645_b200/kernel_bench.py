@@ -3,6 +3,11 @@
     python -m paper_2609_13645_b200.kernel_bench gemm --M 8192 --N 11264 --K 2048 --layout tn --iters 20
     python -m paper_2609_13645_b200.kernel_bench attn_fwd --B 4 --S 2048 --nh 16 --nkv 8 --d 128
     python -m paper_2609_13645_b200.kernel_bench attn_bwd --B 4 --S 2048 --nh 16 --nkv 8 --d 128
+    python -m paper_2609_13645_b200.kernel_bench step --workload c3_1b --layers 1 --iters 3
+
+`step` runs whole train steps of a workload cut down to --layers layers (a few GB on the device): the in-situ target
+for ncu captures of the kernels that have no entry point of their own (norms, SwiGLU backward, cross-entropy, the
+weight-gradient GEMM with AdamW in its epilogue, the leftover optimizer pass).
 
 Inputs are random bf16; between timed launches a 256 MB buffer is rewritten so the operands do not sit in L2.
 Prints one JSON line with the mean launch time and the achieved TFLOP/s.
@@ -22,7 +27,10 @@ def main():
     from paper_2609_13645_b200 import binding as B
 
     ap = argparse.ArgumentParser()
-    ap.add_argument("kernel", choices=["gemm", "attn_fwd", "attn_bwd"])
+    ap.add_argument("kernel", choices=["gemm", "attn_fwd", "attn_bwd", "step"])
+    ap.add_argument("--workload", default="c3_1b")
+    ap.add_argument("--layers", type=int, default=1)
+    ap.add_argument("--unfused", action="store_true", help="step: separate optimizer pass instead of the fused epilogue")
     ap.add_argument("--M", type=int, default=8192)
     ap.add_argument("--N", type=int, default=4096)
     ap.add_argument("--K", type=int, default=2048)
@@ -45,6 +53,27 @@ def main():
         B.lib().ft_debug_gemm_tile(a.bn)
     B.lib().ft_debug_gemm_pairs(a.pairs)
     dev = "cuda"
+    if a.kernel == "step":
+        import synth_inputs as SI
+        w = SI.WORKLOADS[a.workload]
+        Bsz, S = w["batch"], w["seq"]
+        cfg = B.make_config(a.layers, w["d_model"], w["n_heads"], w["n_kv_heads"], w["head_dim"], w["d_ffn"], w["vocab"],
+                            Bsz, S, recompute=w.get("recompute", 0))
+        model = B.Model(cfg, seed=SI.WEIGHT_SEED)
+        model.set_fused_update(not a.unfused)
+        total = 0.0
+        for it in range(a.warmup + a.iters):
+            tok, lab = SI.batch(w["vocab"], Bsz, S, w["dist"], step=it)
+            tok, lab = torch.from_numpy(tok).cuda(), torch.from_numpy(lab).cuda()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); model.train_step(tok, lab, want_loss=False); e1.record()
+            torch.cuda.synchronize()
+            if it >= a.warmup:
+                total += e0.elapsed_time(e1)
+        print(json.dumps(dict(kernel="step", workload=a.workload, layers=a.layers, fused=not a.unfused, ms=total / a.iters,
+                              iters=a.iters)))
+        model.close()
+        return
     flush = None if a.no_flush else torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     err = torch.zeros(1, dtype=torch.int32, device=dev)
 
