@@ -205,6 +205,8 @@ def run_cuda(args):
     torch.cuda.set_stream(side)
     model = B.Model(cfg, seed=SI.WEIGHT_SEED)
     model.set_graph(not args.no_graph)
+    model.set_overlap(not args.no_overlap)
+    model.set_fused_update(not args.no_fused_update)
     n_batches = args.steps + args.warmup
     host_batches = [SI.batch(w["vocab"], Bsz, S, w["dist"], seed=SI.DATA_SEED + 1000 * rank, step=i)
                     for i in range(n_batches)]
@@ -328,6 +330,8 @@ def main():
     ap.add_argument("--workload", default="c3_1b", choices=sorted(SI.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel separately in the timed region")
+    ap.add_argument("--no-overlap", action="store_true", help="ablation: weight-gradient GEMMs on the main stream")
+    ap.add_argument("--no-fused-update", action="store_true", help="ablation: separate AdamW pass over all parameters")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

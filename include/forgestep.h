@@ -75,6 +75,14 @@ ft_status ft_train_step(ft_model* m, const int32_t* dev_tokens, const int32_t* d
  * values (use ft_forward_backward to materialise gradients).  Changing the setting drops a captured graph. */
 ft_status ft_set_fused_update(ft_model* m, int32_t enable);
 
+/* Weight-gradient overlap: nothing later in the backward pass depends on a layer's weight gradients (Section 4.3's
+ * fused dgrad + wgrad observation, turned into concurrency), so the library enqueues those GEMMs on a second stream
+ * of its own, ordered by events against the kernels that produce their inputs and against the kernels that later
+ * overwrite the buffers they read; they occupy the SMs that the main chain leaves idle in the last wave of each
+ * kernel.  Results do not change by a bit (every kernel keeps its own fixed summation order and its own scratch).
+ * On by default; switched off internally while profiling or with debug_taps.  Changing it drops a captured graph. */
+ft_status ft_set_overlap(ft_model* m, int32_t enable);
+
 /* Whole-step CUDA graph (the paper's full-step graph capture): when enabled, the first ft_train_step of a (B, S)
  * runs launch by launch, the second is captured into a graph, later ones replay it (ids are first copied into the
  * model's own buffers).  Needs a capturable stream (not the legacy default stream; otherwise it switches itself

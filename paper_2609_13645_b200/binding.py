@@ -76,6 +76,8 @@ def lib():
         L.ft_get_gemm_profile.restype = C.c_int
         L.ft_set_fused_update.argtypes = [vp, i32]
         L.ft_set_fused_update.restype = C.c_int
+        L.ft_set_overlap.argtypes = [vp, i32]
+        L.ft_set_overlap.restype = C.c_int
         L.ft_set_graph.argtypes = [vp, i32]
         L.ft_set_graph.restype = C.c_int
         L.ft_graph_replays.argtypes = [vp]
@@ -235,6 +237,10 @@ class Model:
     def set_fused_update(self, enable: bool):
         """AdamW inside the weight-gradient GEMM epilogues (default on; only takes effect with clipping off)."""
         self._check(lib().ft_set_fused_update(self._h, 1 if enable else 0))
+
+    def set_overlap(self, enable: bool):
+        """Weight-gradient GEMMs on a second stream, concurrent with the rest of the backward pass (default on)."""
+        self._check(lib().ft_set_overlap(self._h, 1 if enable else 0))
 
     def set_graph(self, enable: bool):
         """Capture the whole step into a CUDA graph on its second run and replay it afterwards."""

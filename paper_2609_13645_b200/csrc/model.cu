@@ -81,6 +81,18 @@ struct ft_model {
   int lastB = 0, lastS = 0;
   bool have_bwd = false;
 
+  // Weight-gradient GEMMs on a second stream: nothing later in the backward pass depends on them, so they fill the SMs
+  // that the main chain's kernels leave idle in their last wave.  ev_d orders a weight gradient after the data
+  // gradient of the same layer (which still reads the bf16 weights the fused update overwrites); ev_w[k] lets the main
+  // stream wait before it overwrites a buffer the k-th weight gradient of the previous layer still reads.
+  bool overlap = true;        // policy switch (ft_set_overlap)
+  cudaStream_t side = nullptr;
+  cudaEvent_t ev_d = nullptr;
+  cudaEvent_t ev_w[4] = {nullptr, nullptr, nullptr, nullptr};
+  bool w_pending[4] = {false, false, false, false};
+  bool overlapping = false;   // true while a backward pass that uses the second stream is being enqueued
+  float* splitk2 = nullptr;   // GEMM scratch of the second stream
+
   // AdamW inside the weight-gradient GEMM epilogues (clipping off): the train step then never stores those gradients
   bool fused_update = true;   // policy switch (ft_set_fused_update)
   bool fusing = false;        // true while a step that fuses is being enqueued
@@ -205,6 +217,7 @@ size_t carve(ft_model* m, uint8_t* base) {
   m->sq_partial = cv.take<float>(kSqnormBlocks);
   m->fuse_sq = cv.take<float>(m->fuse_sq_count());
   m->splitk = cv.take<float>(kSplitKFloats);
+  m->splitk2 = cv.take<float>(kSplitKFloats);
   m->z = cv.take<float>((size_t)m->ce_chunk * V);
   m->dz = cv.take<bf16>((size_t)m->ce_chunk * V);
   m->keys = cv.take<unsigned long long>(sort_pad(T));
@@ -242,10 +255,11 @@ ft_status cuda_fail(ft_model* m, cudaError_t e, const char* where) {
     m->launches += n__;                                                                     \
     prof_end(m, cls, work, n__);                                                            \
   } while (0)
-#define FT_GEMM(args)                                                                       \
+#define FT_GEMM(args) FT_GEMM_ON(args, m->stream)
+#define FT_GEMM_ON(args, stream_)                                                           \
   do {                                                                                      \
     prof_begin(m);                                                                          \
-    cudaError_t e__ = launch_gemm(args, m->stream);                                         \
+    cudaError_t e__ = launch_gemm(args, stream_);                                           \
     if (e__ != cudaSuccess) return cuda_fail(m, e__, "launch_gemm");                        \
     m->launches += g_gemm_last_launches;                                                    \
     prof_end(m, FT_PROF_GEMM, 2.0 * (double)(args).M * (double)(args).N * (double)(args).K, 1, prof_shape_index(m, args)); \
@@ -370,7 +384,16 @@ ft_status copy_tap(ft_model* m, bf16* dst, const bf16* src, size_t n) {
 }
 
 // data gradient  dX[T, n_in] = dY[T, n_out] W[n_out, n_in]  and weight gradient  dW[n_out, n_in] = dY^T X
-ft_status linear_backward(ft_model* m, const bf16* dY, const bf16* X, int wi, bf16* dX, int T, int n_out, int n_in) {
+// Main stream waits until the k-th weight gradient enqueued on the second stream has finished (no-op when none is).
+ft_status wait_wgrad(ft_model* m, int k) {
+  if (!m->w_pending[k]) return FT_OK;
+  FT_CUDA(cudaStreamWaitEvent(m->stream, m->ev_w[k], 0));
+  m->w_pending[k] = false;
+  return FT_OK;
+}
+
+// dX = dY W (data gradient) and dW = dY^T X (weight gradient, slot k of the layer's four)
+ft_status linear_backward(ft_model* m, const bf16* dY, const bf16* X, int wi, bf16* dX, int T, int n_out, int n_in, int k) {
   {
     GemmArgs g = gemm_base(m);
     g.A = dY; g.lda = n_out; g.B = m->wb(wi); g.b_mn = 1; g.ldb = n_in; g.C = dX; g.ldc = n_in;
@@ -382,7 +405,18 @@ ft_status linear_backward(ft_model* m, const bf16* dY, const bf16* X, int wi, bf
     g.A = dY; g.a_mn = 1; g.lda = n_out; g.B = X; g.b_mn = 1; g.ldb = n_in; g.C = m->gr(wi); g.ldc = n_in;
     g.M = n_out; g.N = n_in; g.K = T; g.epi = EPI_F32;
     if (m->fusing) g.adam = fuse_for(m, wi);
-    FT_GEMM(g);
+    if (!m->overlapping) {
+      FT_GEMM(g);
+    } else {
+      ft_status s = wait_wgrad(m, k);  // one weight gradient per slot in flight
+      if (s) return s;
+      FT_CUDA(cudaEventRecord(m->ev_d, m->stream));
+      FT_CUDA(cudaStreamWaitEvent(m->side, m->ev_d, 0));
+      g.scratch = m->splitk2;
+      FT_GEMM_ON(g, m->side);
+      FT_CUDA(cudaEventRecord(m->ev_w[k], m->side));
+      m->w_pending[k] = true;
+    }
   }
   return FT_OK;
 }
@@ -393,26 +427,29 @@ ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
   LayerTaps* tp = m->cfg.debug_taps ? &m->taps[l] : nullptr;
   // m->dxA holds d_x_out
   if (tp) { ft_status s = copy_tap(m, tp->d_x_out, m->dxA, (size_t)T * h); if (s) return s; }
-  ft_status s = linear_backward(m, m->dxA, a.a, m->idx_layer(l, 5), m->d_a, T, h, f);
+  ft_status s = linear_backward(m, m->dxA, a.a, m->idx_layer(l, 5), m->d_a, T, h, f, 0);
   if (s) return s;
+  if ((s = wait_wgrad(m, 1))) return s;  // the previous layer's gate/up weight gradient still reads d_gu
   FT_LAUNCH(FT_PROF_ELEMENTWISE, 10.0 * T * f, swiglu_bwd(m->d_a, a.gu, m->d_gu, T, f, st));
-  s = linear_backward(m, m->d_gu, a.h2, m->idx_layer(l, 4), m->d_h, T, 2 * f, h);
+  s = linear_backward(m, m->d_gu, a.h2, m->idx_layer(l, 4), m->d_h, T, 2 * f, h, 1);
   if (s) return s;
   if (tp) {
     if ((s = copy_tap(m, tp->d_a, m->d_a, (size_t)T * f))) return s;
     if ((s = copy_tap(m, tp->d_gu, m->d_gu, (size_t)T * 2 * f))) return s;
     if ((s = copy_tap(m, tp->d_h2, m->d_h, (size_t)T * h))) return s;
   }
+  if ((s = wait_wgrad(m, 2))) return s;  // the previous layer's output-projection weight gradient still reads dxB
   FT_LAUNCH(FT_PROF_NORM, 8.0 * T * h, rmsnorm_bwd(m->d_h, a.x_mid, a.r2, m->wb(m->idx_layer(l, 3)), m->dxA, m->dxB,
                                                     m->gr(m->idx_layer(l, 3)), m->norm_partial, T, h, st));
-  s = linear_backward(m, m->dxB, a.o, m->idx_layer(l, 2), m->d_o, T, h, hq);
+  s = linear_backward(m, m->dxB, a.o, m->idx_layer(l, 2), m->d_o, T, h, hq, 2);
   if (s) return s;
+  if ((s = wait_wgrad(m, 3))) return s;  // the previous layer's qkv weight gradient still reads d_qkv
   prof_begin(m);
   FT_CUDA(attention_bwd(a.qkv, a.o, m->d_o, a.lse, m->delta, m->d_qkv, m->rope_cos, m->rope_sin, B, S, m->cfg.n_heads,
                         m->cfg.n_kv_heads, m->d, &m->sc->err, st));
   m->launches += 3;
   prof_end(m, FT_PROF_ATTN_BWD, 4.0 * B * m->cfg.n_heads * (double)S * S * m->d, 3);
-  s = linear_backward(m, m->d_qkv, a.h1, m->idx_layer(l, 1), m->d_h, T, nqkv, h);
+  s = linear_backward(m, m->d_qkv, a.h1, m->idx_layer(l, 1), m->d_h, T, nqkv, h, 3);
   if (s) return s;
   if (tp) {
     if ((s = copy_tap(m, tp->d_x_mid, m->dxB, (size_t)T * h))) return s;
@@ -420,6 +457,7 @@ ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
     if ((s = copy_tap(m, tp->d_qkv, m->d_qkv, (size_t)T * nqkv))) return s;
     if ((s = copy_tap(m, tp->d_h1, m->d_h, (size_t)T * h))) return s;
   }
+  if ((s = wait_wgrad(m, 0))) return s;  // this layer's down-projection weight gradient still reads dxA
   FT_LAUNCH(FT_PROF_NORM, 8.0 * T * h, rmsnorm_bwd(m->d_h, m->x[l], a.r1, m->wb(m->idx_layer(l, 0)), m->dxB, m->dxA,
                                                     m->gr(m->idx_layer(l, 0)), m->norm_partial, T, h, st));
   if (tp) { if ((s = copy_tap(m, tp->d_x_in, m->dxA, (size_t)T * h))) return s; }
@@ -435,6 +473,7 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
   cudaStream_t st = m->stream;
   m->lastB = B; m->lastS = S; m->have_bwd = false;
   m->fusing = fuse && with_bwd;
+  m->overlapping = with_bwd && m->overlap && m->side != nullptr && !m->prof && !m->cfg.debug_taps;
   m->fuse_idx = 0;
   m->fuse_args.clear();
   m->fuse_args.reserve((size_t)4 * L + 1);  // pointers into it are handed to the launcher
@@ -489,6 +528,8 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
   for (int l = L - 1; l >= 0; --l) {
     LayerActs& a = m->acts[m->cfg.recompute ? 0 : l];
     if (m->cfg.recompute) {
+      // the weight gradients of the layer above read the one activation slot that the recomputation overwrites
+      for (int k = 0; k < 4; ++k) { ft_status sw = wait_wgrad(m, k); if (sw) return sw; }
       // rerun the layer's forward from its saved input (same kernels, so the same bits as the first time);
       // its output lands in x[l+1], which nothing reads any more
       ft_status s = layer_forward(m, l, a, B, S);
@@ -498,6 +539,8 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
     if (s) return s;
   }
   FT_LAUNCH(FT_PROF_ELEMENTWISE, 2.0 * T * h + 4.0 * V * h, embed_bwd(tok, m->dxA, m->gr(0), m->keys, T, h, V, st));
+  for (int k = 0; k < 4; ++k) { ft_status sw = wait_wgrad(m, k); if (sw) return sw; }  // join the second stream
+  m->overlapping = false;
   m->have_bwd = !m->fusing;  // a fusing step leaves no gradients of the matrices behind
   return FT_OK;
 }
@@ -610,6 +653,9 @@ ft_status ft_init_model(const ft_config* cfg, uint64_t seed, void* dev_workspace
   FT_CUDA(cudaGetDevice(&dev));
   FT_CUDA(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
   if (major != 10) return fail(m, FT_ECUDA, "this library needs an sm_100 device");
+  FT_CUDA(cudaStreamCreateWithFlags(&m->side, cudaStreamNonBlocking));
+  FT_CUDA(cudaEventCreateWithFlags(&m->ev_d, cudaEventDisableTiming));
+  for (int k = 0; k < 4; ++k) FT_CUDA(cudaEventCreateWithFlags(&m->ev_w[k], cudaEventDisableTiming));
 
   FT_CUDA(cudaMemsetAsync(m->adam_m, 0, m->arena * sizeof(float), st));
   FT_CUDA(cudaMemsetAsync(m->adam_v, 0, m->arena * sizeof(float), st));
@@ -617,6 +663,7 @@ ft_status ft_init_model(const ft_config* cfg, uint64_t seed, void* dev_workspace
   FT_CUDA(cudaMemsetAsync(m->master, 0, m->arena * sizeof(float), st));
   FT_CUDA(cudaMemsetAsync(m->sc, 0, sizeof(StepScalars), st));
   FT_CUDA(cudaMemsetAsync(m->splitk, 0, 1024, st));  // the GEMM scratch's arrival counters start at zero
+  FT_CUDA(cudaMemsetAsync(m->splitk2, 0, 1024, st));
   for (size_t i = 0; i < m->params.size(); ++i) {
     const ParamInfo& p = m->params[i];
     if (p.cols) {
@@ -723,6 +770,13 @@ ft_status ft_train_step(ft_model* m, const int32_t* dev_tokens, const int32_t* d
   ft_status s = step_maybe_graphed(m, dev_tokens, dev_labels, B, S);
   if (s) return s;
   if (host_loss || host_gnorm) return finish(m, host_loss, host_gnorm);
+  return FT_OK;
+}
+
+ft_status ft_set_overlap(ft_model* m, int32_t enable) {
+  if (!m) return FT_EINVAL;
+  m->overlap = enable != 0;
+  if (m->graph_exec) { cudaGraphExecDestroy(m->graph_exec); m->graph_exec = nullptr; }  // captured with the old setting
   return FT_OK;
 }
 
@@ -951,6 +1005,9 @@ void ft_destroy(ft_model* m) {
   for (auto& r : m->prof_pending) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
   for (auto e : m->prof_pool) cudaEventDestroy(e);
   if (m->graph_exec) cudaGraphExecDestroy(m->graph_exec);
+  if (m->side) cudaStreamDestroy(m->side);
+  if (m->ev_d) cudaEventDestroy(m->ev_d);
+  for (auto e : m->ev_w) if (e) cudaEventDestroy(e);
   delete m;
 }
 

@@ -315,3 +315,28 @@ def test_adamw_inside_the_weight_gradient_epilogue_equals_the_separate_optimizer
     assert mf.step == 3 and mu.step == 3
     mf.close()
     mu.close()
+
+
+@pytest.mark.parametrize("recompute", [0, 1])
+def test_weight_gradients_on_the_second_stream_change_no_bit(recompute):
+    """The weight-gradient GEMMs run on a second stream, concurrent with the rest of the backward pass; events order
+    them against the producers of their inputs and against later writers of the buffers they read (with recomputation
+    all layers share one activation slot).  Three steps of a three-layer model must equal the single-stream run."""
+    from paper_2609_13645_b200 import binding as B
+    ocfg = oracle_config(n_layers=3, d_model=512, n_heads=4, n_kv_heads=2, head_dim=128, d_ffn=1024, vocab=2048)
+    Bsz, S = 2, 512
+    runs = []
+    for overlap in (True, False):
+        model = B.Model(lib_config(B, ocfg, Bsz, S, recompute=recompute), seed=5)
+        model.set_overlap(overlap)
+        out = []
+        for s in range(3):
+            tok, lab = SI.batch(ocfg.vocab, Bsz, S, "uniform", step=s)
+            out.append(model.train_step(to_dev(tok), to_dev(lab)))
+        runs.append((model, out))
+    (mo, lo), (ms, ls) = runs
+    assert lo == ls
+    for a, b in zip(_state_bits(mo), _state_bits(ms)):
+        assert np.array_equal(a, b)
+    mo.close()
+    ms.close()
