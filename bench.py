@@ -99,6 +99,13 @@ class ClockSampler:
                 "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
+# DRAM read + write bytes of one launch of the dominant kernel, from the committed ncu capture of the gate/up GEMM
+# (dram__bytes_read.sum 87.9 MB + dram__bytes_write.sum 147.7 MB; the algorithmic bytes of that launch are 264.3 MB)
+NCU_GEMM_TRAFFIC_BYTES = 235.6e6
+NCU_GEMM_TRAFFIC_OF = ("one launch of gemm_tc_pair_kernel at M 8192, N 11264, K 2048 (gate/up projection of c3_1b), ncu capture "
+                       "summarised in profiles/gemm_tc_pair_kernel_tn_8192x11264x2048.md; algorithmic bytes 264.3e6")
+
+
 def max_over_ranks(values, world, device=None):
     """Element-wise maximum of a list of floats over all ranks (the slowest rank defines a multi-GPU time)."""
     import torch
@@ -281,7 +288,8 @@ def run_cuda(args):
         peak_tf = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
         roof = {"bound": "tensor", "kernel": "gemm_tc_kernel (all tcgen05 GEMMs of the step)",
                 "achieved": gemm_tflops, "peak": peak_tf, "unit": "TFLOP/s",
-                "frac": gemm_tflops / peak_tf if gemm_tflops else None, "traffic": None,
+                "frac": gemm_tflops / peak_tf if gemm_tflops else None, "traffic": NCU_GEMM_TRAFFIC_BYTES,
+                "traffic_of": NCU_GEMM_TRAFFIC_OF,
                 "peak_kind": f"{peak_kind} sustained bf16 (kernels timed inside a long step)",
                 "share_of_step": g["ms"] / ms_prof,
                 "measured_in": "the profiled pass (same K steps, CUDA events around every launch, no graph)"}
