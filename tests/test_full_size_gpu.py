@@ -230,3 +230,55 @@ def test_head_loss_and_weight_gradients_on_sampled_entries(run):
     dzc = R(dzc / T)
     gH = m.get_param("lm_head", B.KIND_GRAD).astype(np.float64)
     assert rel_l2(gH[vv], dzc.T @ hF_all) < 1e-3
+
+
+@pytest.mark.parametrize("name", ["c3_1b", "c4_8b_slice"])
+def test_bench_launch_configuration_equals_the_plain_step_bit_for_bit(name):
+    """bench.py times the step as a replayed CUDA graph with AdamW inside the weight-gradient epilogues and the weight
+    gradients on a second stream.  At full size (16 layers at c3; recomputation at c4, where all layers share one
+    activation slot) that configuration must leave the same bits as the plain step (one stream, separate optimizer
+    pass, launch by launch), whose kernels the sampled-parity tests above tie to the oracle."""
+    import gc
+    from paper_2609_13645_b200 import binding as B
+    w = SI.WORKLOADS[name]
+    ocfg = oracle_config(**{k: w[k] for k in SI.MODEL_KEYS})
+    cfg = lib_config(B, ocfg, w["batch"], w["seq"], recompute=w["recompute"])
+    gc.collect()
+    torch.cuda.empty_cache()
+    if torch.cuda.mem_get_info()[0] < B.workspace_bytes(cfg) + (4 << 30):
+        pytest.skip("not enough free device memory")
+    L = ocfg.n_layers
+    names = ["embed", "lm_head", "norm_f"] + [f"layers.{l}.{t}" for l in (0, L // 2, L - 1)
+                                              for t in ("wqkv", "wo", "wgu", "wd", "norm1", "norm2")]
+    batches = [SI.batch(ocfg.vocab, w["batch"], w["seq"], w["dist"], step=s) for s in range(3)]
+
+    def state(model):
+        out = []
+        for n in names:
+            for kind in (B.KIND_MASTER, B.KIND_ADAM_M, B.KIND_ADAM_V, B.KIND_BF16):
+                out.append(model.get_param(n, kind).view(np.uint32).copy())
+        return out
+
+    plain = B.Model(cfg, seed=SI.WEIGHT_SEED)
+    plain.set_fused_update(False)
+    plain.set_overlap(False)
+    l_plain = [plain.train_step(to_dev(t), to_dev(l))[0] for t, l in batches]
+    s_plain = state(plain)
+    plain.close()
+    plain.workspace = None
+    gc.collect()
+    torch.cuda.empty_cache()
+
+    side = torch.cuda.Stream()  # the legacy default stream cannot be captured
+    with torch.cuda.stream(side):
+        fast = B.Model(cfg, seed=SI.WEIGHT_SEED)
+        fast.set_graph(True)
+        l_fast = [fast.train_step(to_dev(t), to_dev(l))[0] for t, l in batches]
+        side.synchronize()
+        assert fast.graph_replays >= 2  # step 1 plain launches, step 2 captured and replayed, step 3 replayed
+        s_fast = state(fast)
+        fast.close()
+        fast.workspace = None
+    assert np.array_equal(np.float32(l_plain).view(np.uint32), np.float32(l_fast).view(np.uint32))
+    for a, b in zip(s_plain, s_fast):
+        assert np.array_equal(a, b)
