@@ -142,6 +142,11 @@ void ft_debug_gemm_tile(int32_t bn);
 void ft_debug_gemm_pairs(int32_t on);
 /* Development switch: 1 = balanced-K schedule where it applies and scratch is available (default), 0 = round-robin tiles. */
 void ft_debug_gemm_balanced(int32_t on);
+/* Development switch (process-wide): 1 = the GEMM, attention, norm, SwiGLU-backward and cross-entropy kernels are launched
+ * with programmatic stream serialization (Section 5.2's PDL: a kernel's blocks are scheduled and run their set-up while the
+ * previous kernel drains, then wait for its completion inside the kernel), the default; 0 = ordinary stream order.  Graphs
+ * captured under one setting keep it. */
+void ft_debug_pdl(int32_t on);
 
 const char* ft_last_error(const ft_model* m);
 /* Number of kernels the library launched since the model was created (for launch accounting). */

@@ -19,6 +19,8 @@ template <int D>
 __global__ void __launch_bounds__(256)
 attn_delta_kernel(const bf16* __restrict__ o, const bf16* __restrict__ d_o, float* __restrict__ delta, int B, int S,
                   int n_heads) {
+  pdl_trigger();
+  pdl_wait();
   constexpr int LPR = D / 8;    // lanes per row
   constexpr int RPW = 32 / LPR;  // rows per warp and load
   const int lane = threadIdx.x & 31, sub = lane / LPR, l = lane % LPR;
@@ -59,10 +61,9 @@ cudaError_t attention_delta(const bf16* o, const bf16* d_o, float* delta, int B,
   const long long rows = (long long)B * S * nh;
   const long long want = (rows * (d / 8) + 2 * 256 - 1) / (2 * 256);  // blocks if every thread took one load pair
   const int blocks = (int)(want < 148 * 8 ? (want > 0 ? want : 1) : 148 * 8);
-  if (d == 64) attn_delta_kernel<64><<<blocks, 256, 0, st>>>(o, d_o, delta, B, S, nh);
-  else if (d == 128) attn_delta_kernel<128><<<blocks, 256, 0, st>>>(o, d_o, delta, B, S, nh);
-  else return cudaErrorInvalidValue;
-  return cudaGetLastError();
+  if (d == 64) return launch_pdl(attn_delta_kernel<64>, blocks, 256, 0, st, o, d_o, delta, B, S, nh);
+  if (d == 128) return launch_pdl(attn_delta_kernel<128>, blocks, 256, 0, st, o, d_o, delta, B, S, nh);
+  return cudaErrorInvalidValue;
 }
 
 }  // namespace fs

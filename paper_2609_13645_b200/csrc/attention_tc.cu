@@ -102,6 +102,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_trigger();
+  pdl_wait();  // set-up done; from here on the kernel touches what its predecessor wrote
 
   if (warp == 0) {
     // ------------------------------------------------------------------ Q and K producer
@@ -312,7 +314,8 @@ cudaError_t attention_fwd_tc_t(const bf16* qkv, bf16* o, float* lse, int B, int 
     return cudaErrorInvalidValue;
   const float scale_log2 = (float)((1.0 / sqrt((double)D)) * 1.4426950408889634);
   dim3 grid((S + C::BQ - 1) / C::BQ, nh, B);
-  attn_fwd_tc_kernel<D><<<grid, ATT_THREADS, C::SMEM_BYTES, st>>>(tmQ, tmKV, o, lse, S, nh, nkv, scale_log2, err);
+  cudaError_t el = launch_pdl(attn_fwd_tc_kernel<D>, grid, ATT_THREADS, C::SMEM_BYTES, st, tmQ, tmKV, o, lse, S, nh, nkv, scale_log2, err);
+  if (el != cudaSuccess) return el;
   return cudaGetLastError();
 }
 
@@ -444,6 +447,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_trigger();
+  pdl_wait();  // set-up done; from here on the kernel touches what its predecessor wrote
 
   if (warp == 0) {
     // ------------------------------------------------------------------ producer
@@ -739,11 +744,11 @@ cudaError_t attention_bwd_tc_t(const bf16* qkv, const bf16* o, const bf16* d_o, 
   cudaError_t e = attention_delta(o, d_o, delta, B, S, nh, D, st);
   if (e != cudaSuccess) return e;
   dim3 gq((S + 127) / 128, nh, B), gk((S + 127) / 128, nkv, B);
-  attn_bwd_tc_kernel<D, MODE_DQ><<<gq, BWD_THREADS, CQ::SMEM_BYTES, st>>>(tq128, tq64, td128, td64, lse, delta, dqkv, cs, sn,
-                                                                            S, nh, nkv, scale, scale_log2, err);
-  attn_bwd_tc_kernel<D, MODE_DKV><<<gk, BWD_THREADS, CK::SMEM_BYTES, st>>>(tq128, tq64, td128, td64, lse, delta, dqkv, cs,
-                                                                             sn, S, nh, nkv, scale, scale_log2, err);
-  return cudaGetLastError();
+  e = launch_pdl(attn_bwd_tc_kernel<D, MODE_DQ>, gq, BWD_THREADS, CQ::SMEM_BYTES, st, tq128, tq64, td128, td64, lse, delta,
+                 dqkv, cs, sn, S, nh, nkv, scale, scale_log2, err);
+  if (e != cudaSuccess) return e;
+  return launch_pdl(attn_bwd_tc_kernel<D, MODE_DKV>, gk, BWD_THREADS, CK::SMEM_BYTES, st, tq128, tq64, td128, td64, lse, delta,
+                    dqkv, cs, sn, S, nh, nkv, scale, scale_log2, err);
 }
 
 static __device__ int g_attn_status;

@@ -242,6 +242,32 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// A kernel launched with launch_pdl() may be scheduled while its predecessor in the stream is still running: its
+// blocks come up on SMs the predecessor has left, run their set-up, and park in pdl_wait() until the predecessor has
+// finished and its writes are visible.  Every kernel launched that way executes pdl_wait() before its first access to
+// global memory (reads and writes alike); pdl_trigger() at the top of a kernel lets its own successor start early.
+// Both are no-ops in a kernel that was launched the ordinary way.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+extern int g_pdl;  // host switch: 1 = launch_pdl() sets the attribute (default), 0 = ordinary stream order
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = g_pdl ? 1 : 0;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 // ---------------------------------------------------------------- small reductions
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

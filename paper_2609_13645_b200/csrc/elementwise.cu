@@ -24,6 +24,8 @@ __device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
 // ---------------------------------------------------------------- embedding forward
 __global__ void embed_fwd_kernel(const int32_t* __restrict__ tok, const bf16* __restrict__ E, bf16* __restrict__ x,
                                  long long total_chunks, int chunks_per_row, int h, int vocab) {
+  pdl_trigger();
+  pdl_wait();
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total_chunks;
        i += (long long)gridDim.x * blockDim.x) {
     const long long t = i / chunks_per_row;
@@ -37,6 +39,8 @@ __global__ void embed_fwd_kernel(const int32_t* __restrict__ tok, const bf16* __
 // ---------------------------------------------------------------- RMSNorm forward: one warp per row
 __global__ void rmsnorm_fwd_kernel(const bf16* __restrict__ x, const bf16* __restrict__ g, bf16* __restrict__ y,
                                    float* __restrict__ r, int T, int h, float eps) {
+  pdl_trigger();
+  pdl_wait();
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= T) return;
@@ -73,6 +77,8 @@ __global__ void __launch_bounds__(256)
 rmsnorm_bwd_kernel(const bf16* __restrict__ dy, const bf16* __restrict__ x, const float* __restrict__ r,
                    const bf16* __restrict__ g, const bf16* __restrict__ resid, bf16* __restrict__ dx,
                    float* __restrict__ partial, int T, int h) {
+  pdl_trigger();
+  pdl_wait();
   extern __shared__ float s_dg[];  // [h]
   __shared__ float s_dot[2][8];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -157,6 +163,8 @@ rmsnorm_bwd_kernel(const bf16* __restrict__ dy, const bf16* __restrict__ x, cons
 // out[c] = sum over blocks of partial[b][c], in block order: 32 columns x 8 row groups per CTA, the 8 groups
 // (each a fixed strided subset of the blocks) are then added in group order.
 __global__ void colsum_kernel(const float* __restrict__ partial, float* __restrict__ out, int nblk, int h) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float s[8][33];
   const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
   const int c = blockIdx.x * 32 + cx;
@@ -176,6 +184,8 @@ __global__ void colsum_kernel(const float* __restrict__ partial, float* __restri
 // ---------------------------------------------------------------- SwiGLU backward
 __global__ void swiglu_bwd_kernel(const bf16* __restrict__ d_a, const bf16* __restrict__ gu, bf16* __restrict__ d_gu,
                                   long long total_chunks, int chunks_per_row, int f) {
+  pdl_trigger();
+  pdl_wait();
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total_chunks;
        i += (long long)gridDim.x * blockDim.x) {
     const long long t = i / chunks_per_row;
@@ -217,6 +227,8 @@ __global__ void count_labels_kernel(const int32_t* __restrict__ labels, int T, S
 __global__ void __launch_bounds__(256)
 cross_entropy_kernel(const float* __restrict__ z, const int32_t* __restrict__ labels, float* __restrict__ lse_out,
                      float* __restrict__ loss_row, bf16* __restrict__ dz, int V, const StepScalars* __restrict__ sc) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float s_m[8], s_s[8];
   __shared__ float s_lse;
   const int row = blockIdx.x;
@@ -557,19 +569,19 @@ size_t sort_pad(size_t n) {
 
 int embed_fwd(const int32_t* tok, const bf16* E, bf16* x, int T, int h, int vocab, cudaStream_t st) {
   const long long total = (long long)T * (h / 8);
-  embed_fwd_kernel<<<grid_for(total, 256), 256, 0, st>>>(tok, E, x, total, h / 8, h, vocab);
+  if (launch_pdl(embed_fwd_kernel, grid_for(total, 256), 256, 0, st, tok, E, x, total, h / 8, h, vocab) != cudaSuccess) return -1;
   return ok(1);
 }
 
 int rmsnorm_fwd(const bf16* x, const bf16* g, bf16* y, float* r, int T, int h, float eps, cudaStream_t st) {
-  rmsnorm_fwd_kernel<<<(T + 7) / 8, 256, 0, st>>>(x, g, y, r, T, h, eps);
+  if (launch_pdl(rmsnorm_fwd_kernel, (T + 7) / 8, 256, 0, st, x, g, y, r, T, h, eps) != cudaSuccess) return -1;
   return ok(1);
 }
 
 template <int NCHW, int WPR>
 static void launch_rmsnorm_bwd(int nblk, const bf16* dy, const bf16* x, const float* r, const bf16* g, const bf16* resid,
                                bf16* dx, float* partial, int T, int h, cudaStream_t st) {
-  rmsnorm_bwd_kernel<NCHW, WPR><<<nblk, 256, h * sizeof(float), st>>>(dy, x, r, g, resid, dx, partial, T, h);
+  launch_pdl(rmsnorm_bwd_kernel<NCHW, WPR>, nblk, 256, h * sizeof(float), st, dy, x, r, g, resid, dx, partial, T, h);
 }
 
 int rmsnorm_bwd(const bf16* dy, const bf16* x, const float* r, const bf16* g, const bf16* resid, bf16* dx, float* dg,
@@ -590,13 +602,13 @@ int rmsnorm_bwd(const bf16* dy, const bf16* x, const float* r, const bf16* g, co
     }
   }
 #undef FS_NORM_CASE
-  colsum_kernel<<<(h + 31) / 32, 256, 0, st>>>(partial, dg, nblk, h);
+  if (launch_pdl(colsum_kernel, (h + 31) / 32, 256, 0, st, partial, dg, nblk, h) != cudaSuccess) return -1;
   return ok(2);
 }
 
 int swiglu_bwd(const bf16* d_a, const bf16* gu, bf16* d_gu, int T, int f, cudaStream_t st) {
   const long long total = (long long)T * (f / 8);
-  swiglu_bwd_kernel<<<grid_for(total, 256), 256, 0, st>>>(d_a, gu, d_gu, total, f / 8, f);
+  if (launch_pdl(swiglu_bwd_kernel, grid_for(total, 256), 256, 0, st, d_a, gu, d_gu, total, f / 8, f) != cudaSuccess) return -1;
   return ok(1);
 }
 
@@ -607,7 +619,7 @@ int count_labels(const int32_t* labels, int T, StepScalars* sc, cudaStream_t st)
 
 int cross_entropy_rows(const float* z, const int32_t* labels, float* lse, float* loss_row, bf16* dz, int rows, int V,
                        const StepScalars* sc, cudaStream_t st) {
-  cross_entropy_kernel<<<rows, 256, 0, st>>>(z, labels, lse, loss_row, dz, V, sc);
+  if (launch_pdl(cross_entropy_kernel, rows, 256, 0, st, z, labels, lse, loss_row, dz, V, sc) != cudaSuccess) return -1;
   return ok(1);
 }
 

@@ -15,6 +15,7 @@
 
 namespace fs {
 
+int g_pdl = 1;
 int g_gemm_balanced = 1;
 int g_gemm_last_launches = 1;  // development knob: 0 = always the round-robin tile schedule
 
@@ -525,6 +526,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_trigger();
+  pdl_wait();  // barriers, TMEM and descriptors are set up; everything from here on touches the predecessor's data
 
   const int tiles_m = (p.M + BM - 1) / BM;
   const int tiles_n = (p.N + BN - 1) / BN;
@@ -709,6 +712,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   cluster_sync_all();  // both CTAs' barriers exist before either signals the other
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_trigger();
+  pdl_wait();  // barriers, TMEM and descriptors are set up; everything from here on touches the predecessor's data
 
   const int tiles_m = (p.M + 255) / 256;
   const int tiles_n = (p.N + BN - 1) / BN;
@@ -891,6 +896,8 @@ __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(const float* __restrict__ partial, int nsplit, long long stride, float* __restrict__ out, long long ldc,
                      int M, int N, int accumulate, const GemmDev p) {
   __shared__ float s_sq[8];
+  pdl_trigger();
+  pdl_wait();
   float sq = 0.f;
   AdamCoef cf = {};
   if (ADAM) cf = adam_coef(p);
@@ -983,8 +990,7 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
   p.ksplit = 1; p.split_stride = 0; p.balanced = 0; p.sw_first = 0; p.sw_parts = 1; p.sw_kpb = 0; p.flags = nullptr; p.slots = nullptr;
   const int tiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN);
   const int grid = tiles < sm_count() ? tiles : sm_count();
-  kern<<<grid, GEMM_THREADS, C::SMEM_BYTES, stream>>>(tmA, tmB, p);
-  return cudaGetLastError();
+  return launch_pdl(kern, grid, GEMM_THREADS, C::SMEM_BYTES, stream, tmA, tmB, p);
 }
 
 template <bool A_MN, bool B_MN>
@@ -1059,13 +1065,15 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
   cfg.blockDim = dim3(a.adam ? PAIR_THREADS : GEMM_THREADS, 1, 1);
   cfg.dynamicSmemBytes = C::SMEM_BYTES;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = g_pdl ? 1 : 0;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   g_gemm_last_launches = ksplit > 1 ? 2 : 1;
   cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, p);
   if (e != cudaSuccess || ksplit == 1) return e;
@@ -1074,12 +1082,12 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
     GemmDev pa = p;
     set_adam(pa, a);
     const int blocks = (int)((n4 + 255) / 256 < kAdamFuseSlots ? (n4 + 255) / 256 : kAdamFuseSlots);
-    splitk_reduce_kernel<true><<<blocks, 256, 0, stream>>>(data, ksplit, p.split_stride, reinterpret_cast<float*>(a.C), a.ldc,
-                                                           a.M, a.N, a.epi == EPI_F32_ACC ? 1 : 0, pa);
+    return launch_pdl(splitk_reduce_kernel<true>, blocks, 256, 0, stream, data, ksplit, p.split_stride,
+                      reinterpret_cast<float*>(a.C), a.ldc, a.M, a.N, a.epi == EPI_F32_ACC ? 1 : 0, pa);
   } else {
     const int blocks = (int)((n4 + 255) / 256 < 1184 ? (n4 + 255) / 256 : 1184);
-    splitk_reduce_kernel<false><<<blocks, 256, 0, stream>>>(data, ksplit, p.split_stride, reinterpret_cast<float*>(a.C),
-                                                            a.ldc, a.M, a.N, a.epi == EPI_F32_ACC ? 1 : 0, p);
+    return launch_pdl(splitk_reduce_kernel<false>, blocks, 256, 0, stream, data, ksplit, p.split_stride,
+                      reinterpret_cast<float*>(a.C), a.ldc, a.M, a.N, a.epi == EPI_F32_ACC ? 1 : 0, p);
   }
   return cudaGetLastError();
 }
