@@ -266,43 +266,45 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
       if (gc + col4 < p.N) {
         // all loads of the chunk are issued before the first store (the compiler cannot prove the streams distinct,
         // so it would otherwise serialise one row's loads behind the previous row's stores)
+        // Rolling window over the chunk's 8 row groups: the loads of group i + 4 are issued before group i is updated
+        // and stored, so four groups of loads stay in flight behind the arithmetic.  (Loads are placed explicitly: the
+        // compiler cannot prove the streams distinct and would not move them above earlier stores.)
+        float4 P4[8], M4[8], V4[8], O4[8];
+        auto fetch = [&](int i) {
+          const int rr = i * 4 + sub;
+          const bool okr = row0 + rr < p.M;
+          const long long o = (long long)(row0 + rr) * p.ldc + gc + col4;
+          const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+          P4[i] = okr ? *reinterpret_cast<const float4*>(p.adam_p + o) : z;
+          M4[i] = okr ? *reinterpret_cast<const float4*>(p.adam_m + o) : z;
+          V4[i] = okr ? *reinterpret_cast<const float4*>(p.adam_v + o) : z;
+          O4[i] = (okr && p.epi == EPI_F32_ACC) ? *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(cptr) + o) : z;
+        };
 #pragma unroll
-        for (int hb = 0; hb < 8; hb += 4) {
-          float4 P4[4], M4[4], V4[4], O4[4];
+        for (int i = 0; i < 4; ++i) fetch(i);
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const int rr = (hb + i) * 4 + sub;
-            const bool okr = row0 + rr < p.M;
+        for (int i = 0; i < 8; ++i) {
+          if (i + 4 < 8) fetch(i + 4);
+          const int rr = i * 4 + sub;
+          if (row0 + rr < p.M) {
             const long long o = (long long)(row0 + rr) * p.ldc + gc + col4;
-            const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-            P4[i] = okr ? *reinterpret_cast<const float4*>(p.adam_p + o) : z;
-            M4[i] = okr ? *reinterpret_cast<const float4*>(p.adam_m + o) : z;
-            V4[i] = okr ? *reinterpret_cast<const float4*>(p.adam_v + o) : z;
-            O4[i] = (okr && p.epi == EPI_F32_ACC) ? *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(cptr) + o) : z;
-          }
+            const float4 g4 = *reinterpret_cast<const float4*>(stage + rr * 32 + 4 * ((col4 >> 2) ^ (rr & 7)));
+            float g[4] = {g4.x, g4.y, g4.z, g4.w};
+            if (p.epi == EPI_F32_ACC) { g[0] += O4[i].x; g[1] += O4[i].y; g[2] += O4[i].z; g[3] += O4[i].w; }
+            float pp[4] = {P4[i].x, P4[i].y, P4[i].z, P4[i].w}, mm[4] = {M4[i].x, M4[i].y, M4[i].z, M4[i].w},
+                  vv[4] = {V4[i].x, V4[i].y, V4[i].z, V4[i].w};
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const int rr = (hb + i) * 4 + sub;
-            if (row0 + rr < p.M) {
-              const long long o = (long long)(row0 + rr) * p.ldc + gc + col4;
-              const float4 g4 = *reinterpret_cast<const float4*>(stage + rr * 32 + 4 * ((col4 >> 2) ^ (rr & 7)));
-              float g[4] = {g4.x, g4.y, g4.z, g4.w};
-              if (p.epi == EPI_F32_ACC) { g[0] += O4[i].x; g[1] += O4[i].y; g[2] += O4[i].z; g[3] += O4[i].w; }
-              float pp[4] = {P4[i].x, P4[i].y, P4[i].z, P4[i].w}, mm[4] = {M4[i].x, M4[i].y, M4[i].z, M4[i].w},
-                    vv[4] = {V4[i].x, V4[i].y, V4[i].z, V4[i].w};
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                sq += g[e] * g[e];
-                adamw_elem(g[e], p.adam_wd, c, pp[e], mm[e], vv[e]);
-              }
-              *reinterpret_cast<float4*>(p.adam_p + o) = make_float4(pp[0], pp[1], pp[2], pp[3]);
-              *reinterpret_cast<float4*>(p.adam_m + o) = make_float4(mm[0], mm[1], mm[2], mm[3]);
-              *reinterpret_cast<float4*>(p.adam_v + o) = make_float4(vv[0], vv[1], vv[2], vv[3]);
-              uint2 ob;
-              ob.x = pack_bf16(pp[0], pp[1]);
-              ob.y = pack_bf16(pp[2], pp[3]);
-              *reinterpret_cast<uint2*>(p.adam_pb + o) = ob;
+            for (int e = 0; e < 4; ++e) {
+              sq += g[e] * g[e];
+              adamw_elem(g[e], p.adam_wd, c, pp[e], mm[e], vv[e]);
             }
+            *reinterpret_cast<float4*>(p.adam_p + o) = make_float4(pp[0], pp[1], pp[2], pp[3]);
+            *reinterpret_cast<float4*>(p.adam_m + o) = make_float4(mm[0], mm[1], mm[2], mm[3]);
+            *reinterpret_cast<float4*>(p.adam_v + o) = make_float4(vv[0], vv[1], vv[2], vv[3]);
+            uint2 ob;
+            ob.x = pack_bf16(pp[0], pp[1]);
+            ob.y = pack_bf16(pp[2], pp[3]);
+            *reinterpret_cast<uint2*>(p.adam_pb + o) = ob;
           }
         }
       }
