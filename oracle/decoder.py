@@ -58,6 +58,17 @@ class Config:
     weight_decay: float = 0.1
     max_grad_norm: float = 0.0  # <= 0: clipping off
     clip_eps: float = 1e-6
+    # Variants of the paper's model families (appendix "Model Architectures", rows "Tied input/output embeddings" and
+    # "muP (scale_emb, dim_model_base, scale_depth)").  The paper gives the three muP numbers, not where they act;
+    # the reading taken here is the published MiniCPM convention, reduced to three plain factors:
+    #   emb_scale   (scale_emb)                     x_0 = R(emb_scale * E[token])
+    #   resid_scale (scale_depth / sqrt(n_layers))  x <- R(x + resid_scale * branch) for both branches of a layer
+    #   logit_scale (dim_model_base / d_model)      z = logit_scale * (h_F W^T)
+    # All 1 (and untied) reproduces the plain decoder exactly.
+    emb_scale: float = 1.0
+    resid_scale: float = 1.0
+    logit_scale: float = 1.0
+    tie_embeddings: bool = False  # the output head reads the embedding table; its gradient is the sum of both uses
 
     @property
     def h_q(self) -> int:
@@ -118,7 +129,9 @@ def param_specs(cfg: Config) -> List[Tuple[str, Tuple[int, ...]]]:
             (p + "wgu", (2 * cfg.d_ffn, cfg.d_model)),  # rows: gate 0..f-1, then up 0..f-1
             (p + "wd", (cfg.d_model, cfg.d_ffn)),
         ]
-    specs += [("norm_f", (cfg.d_model,)), ("lm_head", (cfg.vocab, cfg.d_model))]
+    specs += [("norm_f", (cfg.d_model,))]
+    if not cfg.tie_embeddings:
+        specs += [("lm_head", (cfg.vocab, cfg.d_model))]
     return specs
 
 
@@ -317,8 +330,10 @@ def forward_backward(cfg: Config, params: Dict[str, np.ndarray], tokens: np.ndar
     W = {k_: R(np.asarray(v_, dtype=np.float64)) for k_, v_ in params.items()}
     cos, sin = rope_tables(S, d, cfg.rope_theta)
 
-    # 2. embedding: exact row copy
-    x = W["embed"][tokens]  # [B,S,h]
+    # 2. embedding: row copy (exact when emb_scale is 1: R of a bf16 value is itself)
+    s_e, s_r, s_l = float(cfg.emb_scale), float(cfg.resid_scale), float(cfg.logit_scale)
+    head = "embed" if cfg.tie_embeddings else "lm_head"
+    x = R(s_e * W["embed"][tokens])  # [B,S,h]
     saved = []
     for l in range(cfg.n_layers):
         p = f"layers.{l}."
@@ -334,14 +349,14 @@ def forward_backward(cfg: Config, params: Dict[str, np.ndarray], tokens: np.ndar
         v = R(v)
         o, lse = attention_fwd(q, k, v, n_rep, R, contract)
         o2 = o.reshape(B, S, hq)
-        x_mid = R(x_in + o2 @ W[p + "wo"].T)
+        x_mid = R(x_in + s_r * (o2 @ W[p + "wo"].T))
         y, r2 = rmsnorm_fwd(x_mid, W[p + "norm2"], cfg.rms_eps)
         h2 = R(y)
         gu = h2 @ W[p + "wgu"].T
         G = R(gu[..., :f])
         U = R(gu[..., f:])
         a = R(G * sigmoid(G) * U)
-        x_out = R(x_mid + a @ W[p + "wd"].T)
+        x_out = R(x_mid + s_r * (a @ W[p + "wd"].T))
         saved.append(dict(x_in=x_in, r1=r1, h1=h1, q=q, k=k, v=v, o=o, lse=lse, x_mid=x_mid, r2=r2, h2=h2,
                           G=G, U=U, a=a))
         for nm, val in (("x_in", x_in), ("h1", h1), ("q", q), ("k", k), ("v", v), ("attn_lse", lse), ("o", o2),
@@ -351,7 +366,7 @@ def forward_backward(cfg: Config, params: Dict[str, np.ndarray], tokens: np.ndar
 
     y, rF = rmsnorm_fwd(x, W["norm_f"], cfg.rms_eps)
     hF = R(y)
-    z = hF @ W["lm_head"].T  # logits stay unrounded
+    z = s_l * (hF @ W[head].T)  # logits stay unrounded
     zmax = np.max(z, axis=-1, keepdims=True)
     ce_lse = (zmax + np.log(np.sum(np.exp(z - zmax), axis=-1, keepdims=True)))[..., 0]
     counted = labels >= 0
@@ -367,14 +382,17 @@ def forward_backward(cfg: Config, params: Dict[str, np.ndarray], tokens: np.ndar
         return loss, {}, taps
 
     grads: Dict[str, np.ndarray] = {}
-    # B1: dz = R((softmax(z) - onehot(y)) / n_counted), zero rows for ignored labels
+    # B1: dz = R(logit_scale (softmax(z) - onehot(y)) / n_counted), zero rows for ignored labels: the gradient with
+    # respect to the unscaled product h_F W^T, rounded once
     pz = np.exp(z - ce_lse[..., None])
     onehot = np.zeros_like(pz)
     np.put_along_axis(onehot, safe_lab[..., None], 1.0, axis=-1)
-    dz = R(np.where(counted[..., None], (pz - onehot) / max(n_cnt, 1), 0.0))
+    dz = R(np.where(counted[..., None], s_l * (pz - onehot) / max(n_cnt, 1), 0.0))
     del pz, onehot
-    d_hF = R(dz @ W["lm_head"])
-    grads["lm_head"] = dz.reshape(T, V).T @ hF.reshape(T, h)
+    d_hF = R(dz @ W[head])
+    g_head = dz.reshape(T, V).T @ hF.reshape(T, h)
+    if not cfg.tie_embeddings:
+        grads["lm_head"] = g_head
     del dz
     tap("d_hF", d_hF)
     dxn, grads["norm_f"] = rmsnorm_bwd(d_hF, x, rF, W["norm_f"])
@@ -384,8 +402,9 @@ def forward_backward(cfg: Config, params: Dict[str, np.ndarray], tokens: np.ndar
         p = f"layers.{l}."
         sv = saved[l]
         tap(p + "d_x_out", dx)
-        d_a = R(dx @ W[p + "wd"])
-        grads[p + "wd"] = dx.reshape(T, h).T @ sv["a"].reshape(T, f)
+        # the branch output entered the residual stream times resid_scale: its gradient is resid_scale * dx (not rounded)
+        d_a = R((s_r * dx) @ W[p + "wd"])
+        grads[p + "wd"] = (s_r * dx).reshape(T, h).T @ sv["a"].reshape(T, f)
         G, U = sv["G"], sv["U"]
         sg = sigmoid(G)
         dU = R(d_a * G * sg)
@@ -395,8 +414,8 @@ def forward_backward(cfg: Config, params: Dict[str, np.ndarray], tokens: np.ndar
         grads[p + "wgu"] = dGU.reshape(T, 2 * f).T @ sv["h2"].reshape(T, h)
         dxn, grads[p + "norm2"] = rmsnorm_bwd(d_h2, sv["x_mid"], sv["r2"], W[p + "norm2"])
         d_x_mid = R(dx + dxn)
-        d_o = R(d_x_mid @ W[p + "wo"])
-        grads[p + "wo"] = d_x_mid.reshape(T, h).T @ sv["o"].reshape(T, hq)
+        d_o = R((s_r * d_x_mid) @ W[p + "wo"])
+        grads[p + "wo"] = (s_r * d_x_mid).reshape(T, h).T @ sv["o"].reshape(T, hq)
         dq, dk, dv = attention_bwd(sv["q"], sv["k"], sv["v"], sv["o"], d_o.reshape(B, S, nh, d), sv["lse"],
                                    n_rep, R)
         dq = R(rope_apply_transpose(dq, cos, sin))
@@ -417,7 +436,7 @@ def forward_backward(cfg: Config, params: Dict[str, np.ndarray], tokens: np.ndar
     # B10: dE[v,:] = sum over positions holding token v
     dE = np.zeros((V, h), dtype=np.float64)
     np.add.at(dE, tokens.reshape(-1), dx.reshape(T, h))
-    grads["embed"] = dE
+    grads["embed"] = s_e * dE + (g_head if cfg.tie_embeddings else 0.0)
     return loss, grads, taps
 
 

@@ -66,8 +66,13 @@ def test_bf16_round_ties_to_even_and_idempotent():
 
 
 # ---------------------------------------------------------------- whole backward: finite differences
-def test_gradients_match_central_finite_differences():
-    cfg = tiny_cfg()
+VARIANTS = [dict(), dict(emb_scale=12.0, resid_scale=1.4 / math.sqrt(2), logit_scale=256.0 / 1024.0),
+            dict(tie_embeddings=True), dict(tie_embeddings=True, emb_scale=3.0, resid_scale=0.7, logit_scale=0.5)]
+
+
+@pytest.mark.parametrize("variant", VARIANTS, ids=["plain", "mup", "tied", "tied+mup"])
+def test_gradients_match_central_finite_differences(variant):
+    cfg = tiny_cfg(**variant)
     params = tiny_params(cfg)
     tok, lab = tiny_batch(cfg)
     lab[0, 2] = -1  # one ignored label
@@ -116,7 +121,9 @@ def _torch_loss(cfg, tp, tok, lab):
     def rms(x, g):
         return x * torch.rsqrt(x.pow(2).mean(-1, keepdim=True) + cfg.rms_eps) * g
 
-    x = F.embedding(torch.from_numpy(tok.astype(np.int64)), tp["embed"])
+    # model variants, written the way the published muP decoders apply them: embeddings times scale_emb, every branch
+    # output times scale_depth / sqrt(n_layers) before the residual add, final hidden state times the logit factor
+    x = F.embedding(torch.from_numpy(tok.astype(np.int64)), tp["embed"]) * cfg.emb_scale
     for l in range(cfg.n_layers):
         p = f"layers.{l}."
         qkv = F.linear(rms(x, tp[p + "norm1"]), tp[p + "wqkv"])
@@ -125,12 +132,36 @@ def _torch_loss(cfg, tp, tok, lab):
         k = rope(k.reshape(B, S, nkv, d)).transpose(1, 2).repeat_interleave(nh // nkv, dim=1)
         v = v.reshape(B, S, nkv, d).transpose(1, 2).repeat_interleave(nh // nkv, dim=1)
         o = F.scaled_dot_product_attention(q, k, v, is_causal=True)
-        x = x + F.linear(o.transpose(1, 2).reshape(B, S, cfg.h_q), tp[p + "wo"])
+        x = x + F.linear(o.transpose(1, 2).reshape(B, S, cfg.h_q), tp[p + "wo"]) * cfg.resid_scale
         g, u = torch.chunk(F.linear(rms(x, tp[p + "norm2"]), tp[p + "wgu"]), 2, dim=-1)
-        x = x + F.linear(F.silu(g) * u, tp[p + "wd"])
-    z = F.linear(rms(x, tp["norm_f"]), tp["lm_head"])
+        x = x + F.linear(F.silu(g) * u, tp[p + "wd"]) * cfg.resid_scale
+    z = F.linear(rms(x, tp["norm_f"]) * cfg.logit_scale, tp["embed"] if cfg.tie_embeddings else tp["lm_head"])
     return F.cross_entropy(z.reshape(B * S, -1), torch.from_numpy(lab.astype(np.int64)).reshape(-1),
                            ignore_index=-1), z
+
+
+@pytest.mark.parametrize("variant", VARIANTS[1:], ids=["mup", "tied", "tied+mup"])
+def test_model_variants_match_torch_autograd(variant):
+    cfg = tiny_cfg(**variant)
+    params = tiny_params(cfg, seed=21)
+    assert ("lm_head" in params) == (not cfg.tie_embeddings)
+    tok, lab = tiny_batch(cfg, B=2, S=7, seed=22)
+    loss, grads, taps = D.forward_backward(cfg, params, tok, lab, mode="exact", keep_logits=True)
+    tp = {k: torch.tensor(v, dtype=torch.float64, requires_grad=True) for k, v in params.items()}
+    tl, z = _torch_loss(cfg, tp, tok, lab)
+    tl.backward()
+    assert abs(loss - tl.item()) < 1e-12
+    assert np.allclose(taps["logits"], z.detach().numpy(), rtol=0, atol=1e-11)
+    for name in params:
+        tg = tp[name].grad.numpy()
+        assert np.linalg.norm(grads[name] - tg) / np.linalg.norm(tg) < 1e-11, name
+    # all factors 1 and untied is the plain decoder bit for bit
+    plain = tiny_cfg()
+    pp = tiny_params(plain, seed=21)
+    a = D.forward_backward(plain, pp, tok, lab, mode="contract")
+    b = D.forward_backward(tiny_cfg(emb_scale=1.0, resid_scale=1.0, logit_scale=1.0, tie_embeddings=False), pp, tok, lab,
+                           mode="contract")
+    assert a[0] == b[0] and all(np.array_equal(a[1][k], b[1][k]) for k in a[1])
 
 
 @pytest.mark.parametrize("nkv", [4, 2, 1])
