@@ -106,6 +106,14 @@ NCU_GEMM_TRAFFIC_OF = ("one launch of gemm_tc_pair_kernel at M 8192, N 11264, K 
                        "summarised in profiles/gemm_tc_pair_kernel_tn_8192x11264x2048.md; algorithmic bytes 264.3e6")
 
 
+def variant_kwargs(args, w):
+    """--variant mup_tied: the muP factors of the paper's MiniCPM rows (scale_emb 12, scale_depth 1.4, dim_model_base 256)
+    and tied input/output embeddings on top of the workload's shape; the default is the plain decoder."""
+    if args.variant == "plain":
+        return {}
+    return dict(emb_scale=12.0, resid_scale=1.4 / w["n_layers"] ** 0.5, logit_scale=256.0 / w["d_model"], tie_embeddings=1)
+
+
 def max_over_ranks(values, world, device=None):
     """Element-wise maximum of a list of floats over all ranks (the slowest rank defines a multi-GPU time)."""
     import torch
@@ -206,7 +214,7 @@ def run_cuda(args):
     w = SI.WORKLOADS[args.workload]
     Bsz, S = w["batch"], w["seq"]
     cfg = B.make_config(w["n_layers"], w["d_model"], w["n_heads"], w["n_kv_heads"], w["head_dim"], w["d_ffn"],
-                        w["vocab"], Bsz, S, recompute=w["recompute"])
+                        w["vocab"], Bsz, S, recompute=w["recompute"], **variant_kwargs(args, w))
     # The model lives on its own (capturable) stream; everything below is enqueued and timed on that stream.
     side = torch.cuda.Stream()
     torch.cuda.set_stream(side)
@@ -304,7 +312,7 @@ def run_cuda(args):
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": args.workload, "batch": Bsz, "seq_len": S, "tokens_per_step_per_gpu": tokens_per_step,
                        "parallelism": "replicas only (single-GPU path, no collectives)" if world > 1 else "1 GPU",
-                       "recompute": w["recompute"], "cuda_graph": graph_replays > 0,
+                       "recompute": w["recompute"], "cuda_graph": graph_replays > 0, "variant": args.variant,
                        "l2": "no flush needed: weights + activations touched per step are far larger than the 126 MB L2",
                        "token_ids": w["dist"]},
             "mfu": {"model_tflops": model_tflops, "model_gflop_per_token": fl["total"] / 1e9,
@@ -338,6 +346,8 @@ def main():
     ap.add_argument("--workload", default="c3_1b", choices=sorted(SI.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel separately in the timed region")
+    ap.add_argument("--variant", default="plain", choices=["plain", "mup_tied"],
+                    help="model variant on the workload's shape (default: the plain decoder the metric is quoted on)")
     ap.add_argument("--no-overlap", action="store_true", help="ablation: weight-gradient GEMMs on the main stream")
     ap.add_argument("--no-fused-update", action="store_true", help="ablation: separate AdamW pass over all parameters")
     args = ap.parse_args()

@@ -40,6 +40,12 @@ typedef struct {
   float max_grad_norm;            /* <= 0: clipping off; else coeff = min(1, max/(norm + 1e-6)) */
   int32_t recompute;              /* 0: keep every layer's activations; 1: keep layer inputs, rerun the layer forward in backward */
   int32_t debug_taps;             /* 1: keep the backward intermediates of every layer for ft_get_tap (needs recompute = 0) */
+  /* Variants of the paper's model families (appendix "Model Architectures": rows "Tied input/output embeddings" and
+   * "muP (scale_emb, dim_model_base, scale_depth)").  A factor of 0 means 1, so a zero-filled tail is the plain decoder. */
+  float emb_scale;                /* x_0 = R(emb_scale * E[token])                         (muP: scale_emb) */
+  float resid_scale;              /* x <- R(x + resid_scale * branch), both branches       (muP: scale_depth / sqrt(n_layers)) */
+  float logit_scale;              /* z = logit_scale * (h_F W^T)                            (muP: dim_model_base / d_model) */
+  int32_t tie_embeddings;         /* 1: no lm_head parameter; the head reads the embedding table and both gradients add */
 } ft_config;
 
 typedef struct ft_model ft_model;

@@ -23,7 +23,7 @@ __device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
 
 // ---------------------------------------------------------------- embedding forward
 __global__ void embed_fwd_kernel(const int32_t* __restrict__ tok, const bf16* __restrict__ E, bf16* __restrict__ x,
-                                 long long total_chunks, int chunks_per_row, int h, int vocab) {
+                                 long long total_chunks, int chunks_per_row, int h, int vocab, float scale) {
   pdl_trigger();
   pdl_wait();
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total_chunks;
@@ -32,7 +32,15 @@ __global__ void embed_fwd_kernel(const int32_t* __restrict__ tok, const bf16* __
     const int c = (int)(i % chunks_per_row) * 8;
     int id = tok[t];
     id = id < 0 ? 0 : (id >= vocab ? vocab - 1 : id);
-    *reinterpret_cast<uint4*>(x + t * h + c) = *reinterpret_cast<const uint4*>(E + (long long)id * h + c);
+    uint4 v = *reinterpret_cast<const uint4*>(E + (long long)id * h + c);
+    if (scale != 1.0f) {  // x_0 = R(scale * E[token])
+      float f[8];
+      unpack8(v, f);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) f[e] *= scale;
+      v = pack8(f);
+    }
+    *reinterpret_cast<uint4*>(x + t * h + c) = v;
   }
 }
 
@@ -226,7 +234,8 @@ __global__ void count_labels_kernel(const int32_t* __restrict__ labels, int T, S
 // one block per row of logits
 __global__ void __launch_bounds__(256)
 cross_entropy_kernel(const float* __restrict__ z, const int32_t* __restrict__ labels, float* __restrict__ lse_out,
-                     float* __restrict__ loss_row, bf16* __restrict__ dz, int V, const StepScalars* __restrict__ sc) {
+                     float* __restrict__ loss_row, bf16* __restrict__ dz, int V, const StepScalars* __restrict__ sc,
+                     float dz_scale) {
   pdl_trigger();
   pdl_wait();
   __shared__ float s_m[8], s_s[8];
@@ -273,7 +282,7 @@ cross_entropy_kernel(const float* __restrict__ z, const int32_t* __restrict__ la
   const float lse = s_lse;
   const int y = labels[row];
   const bool counted = y >= 0 && y < V;
-  const float w = counted ? sc->inv_count : 0.f;
+  const float w = counted ? sc->inv_count * dz_scale : 0.f;  // dz_scale: the logit factor, folded into the one rounding
   bf16* dr = dz + (long long)row * V;
   for (int c = threadIdx.x * 4; c < V; c += 1024) {
     const float4 v = *reinterpret_cast<const float4*>(zr + c);
@@ -370,7 +379,7 @@ __global__ void bitonic_global_kernel(unsigned long long* __restrict__ keys, int
 // Zipf stream (14 % of the positions) is thus spread over h / 256 blocks instead of one.
 __global__ void __launch_bounds__(256)
 embed_bwd_kernel(const unsigned long long* __restrict__ keys, const bf16* __restrict__ dx, float* __restrict__ dE, int T,
-                 int h) {
+                 int h, float scale, int accumulate) {
   __shared__ int s_end;
   __shared__ float s_part[8][256];
   const int i = blockIdx.x;
@@ -426,7 +435,9 @@ embed_bwd_kernel(const unsigned long long* __restrict__ keys, const bf16* __rest
     float tot = 0.f;
 #pragma unroll
     for (int w = 0; w < 8; ++w) tot += s_part[w][threadIdx.x];
-    dE[(long long)tokid * h + col] = tot;
+    // tied embeddings: the table's gradient already holds the output head's part, this row's sum is added to it
+    float* dst = dE + (long long)tokid * h + col;
+    *dst = accumulate ? *dst + scale * tot : scale * tot;
   }
 }
 
@@ -567,9 +578,9 @@ size_t sort_pad(size_t n) {
   return p;
 }
 
-int embed_fwd(const int32_t* tok, const bf16* E, bf16* x, int T, int h, int vocab, cudaStream_t st) {
+int embed_fwd(const int32_t* tok, const bf16* E, bf16* x, int T, int h, int vocab, float scale, cudaStream_t st) {
   const long long total = (long long)T * (h / 8);
-  if (launch_pdl(embed_fwd_kernel, grid_for(total, 256), 256, 0, st, tok, E, x, total, h / 8, h, vocab) != cudaSuccess) return -1;
+  if (launch_pdl(embed_fwd_kernel, grid_for(total, 256), 256, 0, st, tok, E, x, total, h / 8, h, vocab, scale) != cudaSuccess) return -1;
   return ok(1);
 }
 
@@ -618,8 +629,8 @@ int count_labels(const int32_t* labels, int T, StepScalars* sc, cudaStream_t st)
 }
 
 int cross_entropy_rows(const float* z, const int32_t* labels, float* lse, float* loss_row, bf16* dz, int rows, int V,
-                       const StepScalars* sc, cudaStream_t st) {
-  if (launch_pdl(cross_entropy_kernel, rows, 256, 0, st, z, labels, lse, loss_row, dz, V, sc) != cudaSuccess) return -1;
+                       const StepScalars* sc, float dz_scale, cudaStream_t st) {
+  if (launch_pdl(cross_entropy_kernel, rows, 256, 0, st, z, labels, lse, loss_row, dz, V, sc, dz_scale) != cudaSuccess) return -1;
   return ok(1);
 }
 
@@ -629,7 +640,7 @@ int reduce_loss(const float* loss_row, int T, StepScalars* sc, cudaStream_t st) 
 }
 
 int embed_bwd(const int32_t* tok, const bf16* dx, float* dE, unsigned long long* keys, int T, int h, int vocab,
-              cudaStream_t st) {
+              float scale, bool accumulate, cudaStream_t st) {
   const int n_pad = (int)sort_pad((size_t)T);
   int launches = 0;
   make_keys_kernel<<<(n_pad + 255) / 256, 256, 0, st>>>(tok, keys, T, n_pad, vocab);
@@ -645,8 +656,8 @@ int embed_bwd(const int32_t* tok, const bf16* dx, float* dE, unsigned long long*
     bitonic_chunk_kernel<<<nchunks, kSortThreads, 0, st>>>(keys, k, k);
     ++launches;
   }
-  if (cudaMemsetAsync(dE, 0, (size_t)vocab * h * sizeof(float), st) != cudaSuccess) return -1;
-  embed_bwd_kernel<<<dim3(T, (h + 255) / 256), 256, 0, st>>>(keys, dx, dE, T, h);
+  if (!accumulate && cudaMemsetAsync(dE, 0, (size_t)vocab * h * sizeof(float), st) != cudaSuccess) return -1;
+  embed_bwd_kernel<<<dim3(T, (h + 255) / 256), 256, 0, st>>>(keys, dx, dE, T, h, scale, accumulate ? 1 : 0);
   ++launches;
   return ok(launches);
 }

@@ -31,7 +31,7 @@ constexpr int kSqnormBlocks = 1184;               // partial sums of the gradien
 size_t sort_pad(size_t n);                         // padded key count of the embedding-backward sort
 
 // each returns the number of kernels it launched, or a negative value after a CUDA launch error
-int embed_fwd(const int32_t* tok, const bf16* E, bf16* x, int T, int h, int vocab, cudaStream_t st);
+int embed_fwd(const int32_t* tok, const bf16* E, bf16* x, int T, int h, int vocab, float scale, cudaStream_t st);
 int rmsnorm_fwd(const bf16* x, const bf16* g, bf16* y, float* r, int T, int h, float eps, cudaStream_t st);
 // dx = R(resid + rmsnorm_bwd(dy)) (resid may be null); dg = column sums (fp32, fixed order) via `partial`.
 int rmsnorm_bwd(const bf16* dy, const bf16* x, const float* r, const bf16* g, const bf16* resid, bf16* dx, float* dg,
@@ -40,12 +40,14 @@ int rmsnorm_bwd(const bf16* dy, const bf16* x, const float* r, const bf16* g, co
 int swiglu_bwd(const bf16* d_a, const bf16* gu, bf16* d_gu, int T, int f, cudaStream_t st);
 int count_labels(const int32_t* labels, int T, StepScalars* sc, cudaStream_t st);
 // per row: lse, loss contribution, and (if dz != null) dz = R((softmax(z) - onehot) * inv_count), zero for ignored rows
+// dz = R(dz_scale * (softmax(z) - onehot) / counted labels)
 int cross_entropy_rows(const float* z, const int32_t* labels, float* lse, float* loss_row, bf16* dz, int rows, int V,
-                       const StepScalars* sc, cudaStream_t st);
+                       const StepScalars* sc, float dz_scale, cudaStream_t st);
 int reduce_loss(const float* loss_row, int T, StepScalars* sc, cudaStream_t st);
-// dE[v,:] = sum over positions with token v (fp32, position order); keys: scratch of sort_pad(T) uint64
+// dE[v,:] (+)= scale * sum over positions with token v (fp32, position order); keys: scratch of sort_pad(T) uint64.
+// accumulate: dE already holds another gradient of the same table (tied output head) and is not cleared first.
 int embed_bwd(const int32_t* tok, const bf16* dx, float* dE, unsigned long long* keys, int T, int h, int vocab,
-              cudaStream_t st);
+              float scale, bool accumulate, cudaStream_t st);
 int grad_norm_and_clip(const float* g, size_t n, float* partial, StepScalars* sc, AdamHyper hp, cudaStream_t st);
 int advance_step(StepScalars* sc, AdamHyper hp, cudaStream_t st);
 // fused clip + Adam + decoupled decay + bf16 write-back over a flat arena; elements >= n_decay get no decay

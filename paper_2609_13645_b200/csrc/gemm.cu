@@ -58,6 +58,7 @@ struct GemmDev {
   int epi;
   int seq, head_dim, rope_cols, d_ffn;
   int panel;               // tile numbering (see tile_coords)
+  float alpha;             // accumulator scale (1: off)
   int ksplit;              // > 1: the K blocks are divided over ksplit work units per output tile
   long long split_stride;  // elements between the partial outputs of consecutive K parts
   int balanced;            // 1: the last partial wave of tiles is divided along K and runs first (see WorkIter)
@@ -210,10 +211,18 @@ struct Fixup {
 __device__ __forceinline__ int slot_thread_f4(int cta, int quarter, int lane) { return (cta * 4 + quarter) * 2048 + lane; }
 
 // 32 accumulator columns of this thread's row from TMEM (+ the partials of the same columns, added in index order)
-__device__ __forceinline__ void ld_acc32(uint32_t taddr, int coloff, uint32_t (&r)[32], const Fixup& fx) {
+__device__ __forceinline__ void scale32(uint32_t (&r)[32], float alpha) {
+  if (alpha != 1.0f) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * alpha);
+  }
+}
+
+__device__ __forceinline__ void ld_acc32(uint32_t taddr, int coloff, uint32_t (&r)[32], const Fixup& fx, float alpha) {
   tmem_ld32(taddr + coloff, r);
   if (fx.n == 0) {
     tmem_ld_wait();
+    scale32(r, alpha);
     return;
   }
   // one round trip to L2 per partial: the trips, not the bytes, bound this loop (the launcher limits their number)
@@ -234,6 +243,7 @@ __device__ __forceinline__ void ld_acc32(uint32_t taddr, int coloff, uint32_t (&
 #pragma unroll
     for (int j = 0; j < 8; ++j) v[j] = __ldcg(src + (long long)s * SLOT_F4 + j * 32);
   }
+  scale32(r, alpha);
 }
 
 // Epilogue of one accumulator tile for one thread: `row` is the global output row held by this thread's TMEM lane,
@@ -256,7 +266,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
       const int gc = n0 + c0;
       if (gc >= p.N) break;
       if (c0 + 32 < ce) adam_prefetch_chunk(p, cptr, row, gc + 32);
-      ld_acc32(taddr, c0, r, fx);
+      ld_acc32(taddr, c0, r, fx, p.alpha);
 #pragma unroll
       for (int j = 0; j < 8; ++j)
         *reinterpret_cast<float4*>(stage + lane * 32 + 4 * (j ^ (lane & 7))) =
@@ -320,7 +330,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
       if (g0 >= p.N) break;
       if (g0 >= p.rope_cols) {
         for (int c = 0; c < d; c += 32) {
-          ld_acc32(taddr, hc + c, r, fx);
+          ld_acc32(taddr, hc + c, r, fx, 1.0f);
           if (row_ok) {
             float v[32];
 #pragma unroll
@@ -337,8 +347,8 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
             tmem_ld32(taddr + hc + i0 + half, r2);
             tmem_ld_wait();
           } else {
-            ld_acc32(taddr, hc + i0, r, fx);
-            ld_acc32(taddr, hc + i0 + half, r2, fx);
+            ld_acc32(taddr, hc + i0, r, fx, 1.0f);
+            ld_acc32(taddr, hc + i0 + half, r2, fx, 1.0f);
           }
           if (row_ok) {
             const float* cs = p.rope_cos + (long long)pos * half + i0;
@@ -375,7 +385,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
     for (int c = cb; c < ce; c += 32) {
       const int gc = n0 + c;
       if (gc >= p.N) break;
-      ld_acc32(taddr, c, r, fx);
+      ld_acc32(taddr, c, r, fx, p.alpha);
       if (row_ok) {
         const int lc = gc >> 1;  // logical ffn column of this 16-wide group
         float g[16], u[16], a[16];
@@ -412,7 +422,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
 #pragma unroll
       for (int j = 0; j < 4; ++j) cur[j] = nxt[j];
       if (c + 32 < ce) fetch(gc + 32);
-      ld_acc32(taddr, c, r, fx);
+      ld_acc32(taddr, c, r, fx, p.alpha);
       if (row_ok) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -443,7 +453,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
 #pragma unroll
       for (int j = 0; j < 8; ++j) cur[j] = nxt[j];
       if (c + 32 < ce) fetch(gc + 32);
-      ld_acc32(taddr, c, r, fx);
+      ld_acc32(taddr, c, r, fx, p.alpha);
       if (row_ok) {
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -460,7 +470,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
     for (int c = cb; c < ce; c += 32) {
       const int gc = n0 + c;
       if (gc >= p.N) break;
-      ld_acc32(taddr, c, r, fx);
+      ld_acc32(taddr, c, r, fx, p.alpha);
       if (row_ok) {
         if (p.epi == EPI_BF16) {
           bf16* crow = reinterpret_cast<bf16*>(cptr) + (long long)row * p.ldc + gc;
@@ -988,6 +998,7 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
   p.ldc = a.ldc; p.M = a.M; p.N = a.N; p.K = a.K; p.epi = a.epi;
   p.seq = a.seq; p.head_dim = a.head_dim; p.rope_cols = a.rope_cols; p.d_ffn = a.d_ffn;
   set_adam(p, a);
+  p.alpha = a.alpha;
   p.panel = (size_t)a.M * a.K * sizeof(bf16) > (48u << 20) ? 1 : 0;
   p.ksplit = 1; p.split_stride = 0; p.balanced = 0; p.sw_first = 0; p.sw_parts = 1; p.sw_kpb = 0; p.flags = nullptr; p.slots = nullptr;
   const int tiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN);
@@ -1014,6 +1025,7 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
   p.ldc = a.ldc; p.M = a.M; p.N = a.N; p.K = a.K; p.epi = a.epi;
   p.seq = a.seq; p.head_dim = a.head_dim; p.rope_cols = a.rope_cols; p.d_ffn = a.d_ffn;
   set_adam(p, a);
+  p.alpha = a.alpha;
   p.panel = (size_t)a.M * a.K * sizeof(bf16) > (48u << 20) ? 1 : 0;
   const int tiles = ((a.M + 255) / 256) * ((a.N + 255) / 256);
   const int max_pairs = sm_count() / 2;
@@ -1116,6 +1128,7 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream) {
   if ((reinterpret_cast<uintptr_t>(a.A) | reinterpret_cast<uintptr_t>(a.B) | reinterpret_cast<uintptr_t>(a.C)) & 15)
     return cudaErrorInvalidValue;
   if (a.epi == EPI_BF16_RESID && !a.resid) return cudaErrorInvalidValue;
+  if (a.alpha != 1.0f && (a.epi == EPI_ROPE || a.epi == EPI_SWIGLU)) return cudaErrorInvalidValue;
   if (a.adam && ((a.epi != EPI_F32 && a.epi != EPI_F32_ACC) || !a.adam->p || !a.adam->m || !a.adam->v || !a.adam->pb ||
                  !a.adam->scalars || !a.adam->sq_slots))
     return cudaErrorInvalidValue;

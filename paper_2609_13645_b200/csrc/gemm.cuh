@@ -43,6 +43,7 @@ struct GemmArgs {
   const bf16* resid = nullptr;
   int epi = EPI_BF16;
   int M = 0, N = 0, K = 0;
+  float alpha = 1.0f;  // the accumulator is multiplied by alpha before the epilogue (not for EPI_ROPE / EPI_SWIGLU)
   // EPI_ROPE
   const float* rope_cos = nullptr;  // fp32 [seq, head_dim/2]
   const float* rope_sin = nullptr;

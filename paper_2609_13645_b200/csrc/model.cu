@@ -128,6 +128,13 @@ struct ft_model {
 
 namespace {
 
+// a factor of 0 in the configuration means 1
+void normalise(ft_config& c) {
+  if (c.emb_scale == 0.f) c.emb_scale = 1.f;
+  if (c.resid_scale == 0.f) c.resid_scale = 1.f;
+  if (c.logit_scale == 0.f) c.logit_scale = 1.f;
+}
+
 bool valid_config(const ft_config* c, std::string* why) {
   auto bad = [&](const char* m) { if (why) *why = m; return false; };
   if (!c) return bad("null config");
@@ -142,6 +149,8 @@ bool valid_config(const ft_config* c, std::string* why) {
   if ((long long)c->max_batch * c->max_seq > (1ll << 24)) return bad("max_batch * max_seq too large");
   if (c->debug_taps && c->recompute) return bad("debug_taps needs recompute = 0");
   if (!(c->rms_eps > 0.f) || !(c->rope_theta > 0.f)) return bad("rms_eps and rope_theta must be positive");
+  if (c->emb_scale < 0.f || c->resid_scale < 0.f || c->logit_scale < 0.f) return bad("negative scale factor");
+  if (c->tie_embeddings != 0 && c->tie_embeddings != 1) return bad("tie_embeddings must be 0 or 1");
   return true;
 }
 
@@ -180,7 +189,7 @@ size_t carve(ft_model* m, uint8_t* base) {
     add(p + "wd", h, f, false);
   }
   add("norm_f", h, 0, false);
-  add("lm_head", V, h, false);
+  if (!c.tie_embeddings) add("lm_head", V, h, false);
   size_t off = 0;
   for (auto& p : m->params) if (p.cols) { p.offset = off; off += align_up(p.numel(), 128); }
   m->n_decay = off;
@@ -359,7 +368,7 @@ ft_status layer_forward(ft_model* m, int l, LayerActs& a, int B, int S) {
   {
     GemmArgs g = gemm_base(m);
     g.A = a.o; g.lda = hq; g.B = m->wb(m->idx_layer(l, 2)); g.ldb = hq; g.C = a.x_mid; g.ldc = h; g.resid = m->x[l];
-    g.M = T; g.N = h; g.K = hq; g.epi = EPI_BF16_RESID;
+    g.M = T; g.N = h; g.K = hq; g.epi = EPI_BF16_RESID; g.alpha = m->cfg.resid_scale;
     FT_GEMM(g);
   }
   FT_LAUNCH(FT_PROF_NORM, 4.0 * T * h, rmsnorm_fwd(a.x_mid, m->wb(m->idx_layer(l, 3)), a.h2, a.r2, T, h, m->cfg.rms_eps, st));
@@ -372,7 +381,7 @@ ft_status layer_forward(ft_model* m, int l, LayerActs& a, int B, int S) {
   {
     GemmArgs g = gemm_base(m);
     g.A = a.a; g.lda = f; g.B = m->wb(m->idx_layer(l, 5)); g.ldb = f; g.C = m->x[l + 1]; g.ldc = h; g.resid = a.x_mid;
-    g.M = T; g.N = h; g.K = f; g.epi = EPI_BF16_RESID;
+    g.M = T; g.N = h; g.K = f; g.epi = EPI_BF16_RESID; g.alpha = m->cfg.resid_scale;
     FT_GEMM(g);
   }
   return FT_OK;
@@ -393,17 +402,19 @@ ft_status wait_wgrad(ft_model* m, int k) {
 }
 
 // dX = dY W (data gradient) and dW = dY^T X (weight gradient, slot k of the layer's four)
-ft_status linear_backward(ft_model* m, const bf16* dY, const bf16* X, int wi, bf16* dX, int T, int n_out, int n_in, int k) {
+// alpha: factor the branch output carried into the residual stream (its gradient is alpha * dY, never rounded)
+ft_status linear_backward(ft_model* m, const bf16* dY, const bf16* X, int wi, bf16* dX, int T, int n_out, int n_in, int k,
+                          float alpha = 1.0f) {
   {
     GemmArgs g = gemm_base(m);
     g.A = dY; g.lda = n_out; g.B = m->wb(wi); g.b_mn = 1; g.ldb = n_in; g.C = dX; g.ldc = n_in;
-    g.M = T; g.N = n_in; g.K = n_out; g.epi = EPI_BF16;
+    g.M = T; g.N = n_in; g.K = n_out; g.epi = EPI_BF16; g.alpha = alpha;
     FT_GEMM(g);
   }
   {
     GemmArgs g = gemm_base(m);
     g.A = dY; g.a_mn = 1; g.lda = n_out; g.B = X; g.b_mn = 1; g.ldb = n_in; g.C = m->gr(wi); g.ldc = n_in;
-    g.M = n_out; g.N = n_in; g.K = T; g.epi = EPI_F32;
+    g.M = n_out; g.N = n_in; g.K = T; g.epi = EPI_F32; g.alpha = alpha;
     if (m->fusing) g.adam = fuse_for(m, wi);
     if (!m->overlapping) {
       FT_GEMM(g);
@@ -427,7 +438,7 @@ ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
   LayerTaps* tp = m->cfg.debug_taps ? &m->taps[l] : nullptr;
   // m->dxA holds d_x_out
   if (tp) { ft_status s = copy_tap(m, tp->d_x_out, m->dxA, (size_t)T * h); if (s) return s; }
-  ft_status s = linear_backward(m, m->dxA, a.a, m->idx_layer(l, 5), m->d_a, T, h, f, 0);
+  ft_status s = linear_backward(m, m->dxA, a.a, m->idx_layer(l, 5), m->d_a, T, h, f, 0, m->cfg.resid_scale);
   if (s) return s;
   if ((s = wait_wgrad(m, 1))) return s;  // the previous layer's gate/up weight gradient still reads d_gu
   FT_LAUNCH(FT_PROF_ELEMENTWISE, 10.0 * T * f, swiglu_bwd(m->d_a, a.gu, m->d_gu, T, f, st));
@@ -441,7 +452,7 @@ ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
   if ((s = wait_wgrad(m, 2))) return s;  // the previous layer's output-projection weight gradient still reads dxB
   FT_LAUNCH(FT_PROF_NORM, 8.0 * T * h, rmsnorm_bwd(m->d_h, a.x_mid, a.r2, m->wb(m->idx_layer(l, 3)), m->dxA, m->dxB,
                                                     m->gr(m->idx_layer(l, 3)), m->norm_partial, T, h, st));
-  s = linear_backward(m, m->dxB, a.o, m->idx_layer(l, 2), m->d_o, T, h, hq, 2);
+  s = linear_backward(m, m->dxB, a.o, m->idx_layer(l, 2), m->d_o, T, h, hq, 2, m->cfg.resid_scale);
   if (s) return s;
   if ((s = wait_wgrad(m, 3))) return s;  // the previous layer's qkv weight gradient still reads d_qkv
   prof_begin(m);
@@ -484,12 +495,13 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
   }
 
   FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T, count_labels(lab, T, m->sc, st));
-  FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T * h, embed_fwd(tok, m->wb(0), m->x[0], T, h, V, st));
+  FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T * h, embed_fwd(tok, m->wb(0), m->x[0], T, h, V, m->cfg.emb_scale, st));
   for (int l = 0; l < L; ++l) {
     ft_status s = layer_forward(m, l, m->acts[m->cfg.recompute ? 0 : l], B, S);
     if (s) return s;
   }
-  const int i_normf = 1 + 6 * L, i_head = 2 + 6 * L;
+  const bool tied = m->cfg.tie_embeddings != 0;
+  const int i_normf = 1 + 6 * L, i_head = tied ? 0 : 2 + 6 * L;  // tied: the head reads (and adds its gradient to) the table
   FT_LAUNCH(FT_PROF_NORM, 4.0 * T * h, rmsnorm_fwd(m->x[L], m->wb(i_normf), m->hF, m->rF, T, h, m->cfg.rms_eps, st));
 
   // output head + cross-entropy (+ both head gradients) in chunks of rows: the logits of one chunk at a time
@@ -498,12 +510,12 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
     {
       GemmArgs g = gemm_base(m);
       g.A = m->hF + (size_t)r0 * h; g.lda = h; g.B = m->wb(i_head); g.ldb = h; g.C = m->z; g.ldc = V;
-      g.M = rows; g.N = V; g.K = h; g.epi = EPI_F32;
+      g.M = rows; g.N = V; g.K = h; g.epi = EPI_F32; g.alpha = m->cfg.logit_scale;
       FT_GEMM(g);
     }
     FT_LAUNCH(FT_PROF_CE, (with_bwd ? 10.0 : 4.0) * rows * V,
               cross_entropy_rows(m->z, lab + r0, m->ce_lse + r0, m->loss_row + r0, with_bwd ? m->dz : nullptr, rows, V,
-                                 m->sc, st));
+                                 m->sc, m->cfg.logit_scale, st));
     if (with_bwd) {
       {
         GemmArgs g = gemm_base(m);
@@ -515,7 +527,8 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
         GemmArgs g = gemm_base(m);
         g.A = m->dz; g.a_mn = 1; g.lda = V; g.B = m->hF + (size_t)r0 * h; g.b_mn = 1; g.ldb = h; g.C = m->gr(i_head);
         g.ldc = h; g.M = V; g.N = h; g.K = rows; g.epi = chunk == 0 ? EPI_F32 : EPI_F32_ACC;
-        if (m->fusing && r0 + rows >= T) g.adam = fuse_for(m, i_head);  // the last chunk completes the gradient
+        // the last chunk completes the gradient (with tied embeddings the table's own part is still to come)
+        if (m->fusing && !tied && r0 + rows >= T) g.adam = fuse_for(m, i_head);
         FT_GEMM(g);
       }
     }
@@ -538,7 +551,7 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
     ft_status s = layer_backward(m, l, a, B, S);
     if (s) return s;
   }
-  FT_LAUNCH(FT_PROF_ELEMENTWISE, 2.0 * T * h + 4.0 * V * h, embed_bwd(tok, m->dxA, m->gr(0), m->keys, T, h, V, st));
+  FT_LAUNCH(FT_PROF_ELEMENTWISE, 2.0 * T * h + 4.0 * V * h, embed_bwd(tok, m->dxA, m->gr(0), m->keys, T, h, V, m->cfg.emb_scale, tied, st));
   for (int k = 0; k < 4; ++k) { ft_status sw = wait_wgrad(m, k); if (sw) return sw; }  // join the second stream
   m->overlapping = false;
   m->have_bwd = !m->fusing;  // a fusing step leaves no gradients of the matrices behind
@@ -632,6 +645,7 @@ size_t ft_workspace_bytes(const ft_config* cfg) {
   if (!valid_config(cfg, nullptr)) return 0;
   ft_model tmp;
   tmp.cfg = *cfg;
+  normalise(tmp.cfg);
   return carve(&tmp, nullptr);
 }
 
@@ -644,6 +658,7 @@ ft_status ft_init_model(const ft_config* cfg, uint64_t seed, void* dev_workspace
   if (!dev_workspace || (reinterpret_cast<uintptr_t>(dev_workspace) & (kAlign - 1))) return FT_EINVAL;
   ft_model* m = new ft_model();
   m->cfg = *cfg;
+  normalise(m->cfg);
   m->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   const size_t need = carve(m, reinterpret_cast<uint8_t*>(dev_workspace));
   if (bytes < need) { delete m; return FT_ENOMEM; }

@@ -12,7 +12,8 @@ def f32(x):
 def oracle_config(**kw):
     """Oracle config whose hyper-parameters carry the fp32 values the C struct holds."""
     c = D.Config(**kw)
-    for k in ("rms_eps", "rope_theta", "lr", "beta1", "beta2", "adam_eps", "weight_decay", "max_grad_norm"):
+    for k in ("rms_eps", "rope_theta", "lr", "beta1", "beta2", "adam_eps", "weight_decay", "max_grad_norm", "emb_scale",
+              "resid_scale", "logit_scale"):
         setattr(c, k, f32(getattr(c, k)))
     return c
 
@@ -21,7 +22,8 @@ def lib_config(B, ocfg, max_batch, max_seq, **extra):
     return B.make_config(ocfg.n_layers, ocfg.d_model, ocfg.n_heads, ocfg.n_kv_heads, ocfg.head_dim, ocfg.d_ffn,
                          ocfg.vocab, max_batch, max_seq, rms_eps=ocfg.rms_eps, rope_theta=ocfg.rope_theta, lr=ocfg.lr,
                          beta1=ocfg.beta1, beta2=ocfg.beta2, adam_eps=ocfg.adam_eps, weight_decay=ocfg.weight_decay,
-                         max_grad_norm=ocfg.max_grad_norm, **extra)
+                         max_grad_norm=ocfg.max_grad_norm, emb_scale=ocfg.emb_scale, resid_scale=ocfg.resid_scale,
+                         logit_scale=ocfg.logit_scale, tie_embeddings=int(ocfg.tie_embeddings), **extra)
 
 
 def rel_l2(a, b):

@@ -98,6 +98,23 @@ def test_gqa_head_dim_128_two_layers_with_ignored_labels():
     _check_step(ocfg, tok, lab, params)
 
 
+@pytest.mark.parametrize("variant", ["mup", "tied", "tied+mup"])
+def test_model_variants_match_oracle_on_every_tap_gradient_and_master(variant):
+    """The paper's model families differ from the plain decoder by tied input/output embeddings and by the muP factors
+    on the embedding, the residual branches and the logits: same full-step parity as configuration 1."""
+    import math
+    kw = dict(n_layers=2, d_model=256, n_heads=4, n_kv_heads=2, head_dim=64, d_ffn=688, vocab=1024)
+    if "mup" in variant:  # MiniCPM's numbers: scale_emb 12, scale_depth 1.4, dim_model_base 256 (here d_model = 256 -> 0.5 used)
+        kw.update(emb_scale=12.0, resid_scale=1.4 / math.sqrt(2), logit_scale=0.5)
+    if "tied" in variant:
+        kw.update(tie_embeddings=True)
+    ocfg = oracle_config(**kw)
+    params = D.init_params(ocfg, SI.WEIGHT_SEED)
+    assert ("lm_head" in params) == ("tied" not in variant)
+    tok, lab = SI.batch(ocfg.vocab, 2, 128, "uniform", step=0)
+    _check_step(ocfg, tok, lab, params)
+
+
 def test_seeded_initialisation_matches_the_oracles_generator():
     from paper_2609_13645_b200 import binding as B
     ocfg, w = _c1()
@@ -281,7 +298,7 @@ def test_ten_step_loss_and_gradient_norm_trajectory_matches_oracle():
     model.close()
 
 
-@pytest.mark.parametrize("shape", ["c1", "split_k", "balanced"])
+@pytest.mark.parametrize("shape", ["c1", "split_k", "balanced", "tied_mup"])
 def test_adamw_inside_the_weight_gradient_epilogue_equals_the_separate_optimizer_pass(shape):
     """Clipping is off, so the train step applies AdamW where the weight gradient is finished (GEMM epilogue, split-K
     reduction, or the epilogue that completes a tile divided along K).  Same update function, same gradient bits:
@@ -291,6 +308,10 @@ def test_adamw_inside_the_weight_gradient_epilogue_equals_the_separate_optimizer
     if shape == "c1":
         ocfg, _ = _c1()
         Bsz, S = 2, 128
+    elif shape == "tied_mup":  # the head's gradient joins the table's: it stays with the separate pass; factors in the epilogues
+        ocfg = oracle_config(n_layers=2, d_model=512, n_heads=4, n_kv_heads=2, head_dim=128, d_ffn=1024, vocab=2048,
+                             tie_embeddings=True, emb_scale=12.0, resid_scale=0.99, logit_scale=0.5)
+        Bsz, S = 2, 1024
     elif shape == "split_k":   # weight gradients with few tiles and 2048 tokens: K split over 4 parts
         ocfg = oracle_config(n_layers=2, d_model=512, n_heads=4, n_kv_heads=2, head_dim=128, d_ffn=1024, vocab=2048)
         Bsz, S = 2, 1024
