@@ -69,6 +69,11 @@ class Config:
     resid_scale: float = 1.0
     logit_scale: float = 1.0
     tie_embeddings: bool = False  # the output head reads the embedding table; its gradient is the sum of both uses
+    # Per-head QK-Norm (appendix "Model Architectures", Qwen3 column: "RoPE (theta = 1e6, QK-Norm)"): the d entries of
+    # every query and key head are RMS-normalised with a learned gain of d entries (one for all query heads, one for all
+    # key heads of a layer; eps = rms_eps) before the rotation.  The paper names it without a formula; this is the
+    # published Qwen3 definition.
+    qk_norm: bool = False
 
     @property
     def h_q(self) -> int:
@@ -129,6 +134,8 @@ def param_specs(cfg: Config) -> List[Tuple[str, Tuple[int, ...]]]:
             (p + "wgu", (2 * cfg.d_ffn, cfg.d_model)),  # rows: gate 0..f-1, then up 0..f-1
             (p + "wd", (cfg.d_model, cfg.d_ffn)),
         ]
+        if cfg.qk_norm:
+            specs += [(p + "q_norm", (cfg.head_dim,)), (p + "k_norm", (cfg.head_dim,))]
     specs += [("norm_f", (cfg.d_model,))]
     if not cfg.tie_embeddings:
         specs += [("lm_head", (cfg.vocab, cfg.d_model))]
@@ -344,6 +351,10 @@ def forward_backward(cfg: Config, params: Dict[str, np.ndarray], tokens: np.ndar
         q = qkv[..., :hq].reshape(B, S, nh, d)
         k = qkv[..., hq:hq + hkv].reshape(B, S, nkv, d)
         v = qkv[..., hq + hkv:].reshape(B, S, nkv, d)
+        if cfg.qk_norm:  # per-head RMSNorm of the unrounded accumulators, then the rotation, then one rounding
+            q, rq = rmsnorm_fwd(q, W[p + "q_norm"], cfg.rms_eps)  # rq [B,S,n_h]; q is now the normalised, gained value
+            k, rk = rmsnorm_fwd(k, W[p + "k_norm"], cfg.rms_eps)
+            q_hat, k_hat = q / W[p + "q_norm"], k / W[p + "k_norm"]  # unit-RMS values (pre-gain) for the backward pass
         q = R(rope_apply(q, cos, sin))  # RoPE on the unrounded q, k; one rounding after it
         k = R(rope_apply(k, cos, sin))
         v = R(v)
@@ -359,6 +370,8 @@ def forward_backward(cfg: Config, params: Dict[str, np.ndarray], tokens: np.ndar
         x_out = R(x_mid + s_r * (a @ W[p + "wd"].T))
         saved.append(dict(x_in=x_in, r1=r1, h1=h1, q=q, k=k, v=v, o=o, lse=lse, x_mid=x_mid, r2=r2, h2=h2,
                           G=G, U=U, a=a))
+        if cfg.qk_norm:
+            saved[-1].update(q_hat=q_hat, k_hat=k_hat, rq=rq, rk=rk)
         for nm, val in (("x_in", x_in), ("h1", h1), ("q", q), ("k", k), ("v", v), ("attn_lse", lse), ("o", o2),
                         ("x_mid", x_mid), ("h2", h2), ("G", G), ("U", U), ("a", a), ("x_out", x_out)):
             tap(p + nm, val)
@@ -421,6 +434,16 @@ def forward_backward(cfg: Config, params: Dict[str, np.ndarray], tokens: np.ndar
         dq = R(rope_apply_transpose(dq, cos, sin))
         dk = R(rope_apply_transpose(dk, cos, sin))
         dv = R(dv)
+        if cfg.qk_norm:
+            # backward of y = x_hat * g with x_hat = x r: dx = r (g dy - x_hat mean_k(g dy x_hat)), dg = sum dy x_hat;
+            # dy is the rounded gradient above, dx is rounded once more (it is what the projection's backward reads)
+            def head_norm_bwd(dy, x_hat, r, g):
+                gdy = dy * g
+                dx = r[..., None] * (gdy - x_hat * np.mean(gdy * x_hat, axis=-1, keepdims=True))
+                return dx, np.sum((dy * x_hat).reshape(-1, d), axis=0)
+            dq, grads[p + "q_norm"] = head_norm_bwd(dq, sv["q_hat"], sv["rq"], W[p + "q_norm"])
+            dk, grads[p + "k_norm"] = head_norm_bwd(dk, sv["k_hat"], sv["rk"], W[p + "k_norm"])
+            dq, dk = R(dq), R(dk)
         dqkv = np.concatenate([dq.reshape(B, S, hq), dk.reshape(B, S, hkv), dv.reshape(B, S, hkv)], axis=-1)
         d_h1 = R(dqkv @ W[p + "wqkv"])
         grads[p + "wqkv"] = dqkv.reshape(T, hq + 2 * hkv).T @ sv["h1"].reshape(T, h)

@@ -67,10 +67,12 @@ def test_bf16_round_ties_to_even_and_idempotent():
 
 # ---------------------------------------------------------------- whole backward: finite differences
 VARIANTS = [dict(), dict(emb_scale=12.0, resid_scale=1.4 / math.sqrt(2), logit_scale=256.0 / 1024.0),
-            dict(tie_embeddings=True), dict(tie_embeddings=True, emb_scale=3.0, resid_scale=0.7, logit_scale=0.5)]
+            dict(tie_embeddings=True), dict(tie_embeddings=True, emb_scale=3.0, resid_scale=0.7, logit_scale=0.5),
+            dict(qk_norm=True), dict(qk_norm=True, tie_embeddings=True, n_kv_heads=1)]
+VARIANT_IDS = ["plain", "mup", "tied", "tied+mup", "qknorm", "qknorm+tied+mqa"]
 
 
-@pytest.mark.parametrize("variant", VARIANTS, ids=["plain", "mup", "tied", "tied+mup"])
+@pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_IDS)
 def test_gradients_match_central_finite_differences(variant):
     cfg = tiny_cfg(**variant)
     params = tiny_params(cfg)
@@ -128,8 +130,11 @@ def _torch_loss(cfg, tp, tok, lab):
         p = f"layers.{l}."
         qkv = F.linear(rms(x, tp[p + "norm1"]), tp[p + "wqkv"])
         q, k, v = torch.split(qkv, [cfg.h_q, cfg.h_kv, cfg.h_kv], dim=-1)
-        q = rope(q.reshape(B, S, nh, d)).transpose(1, 2)
-        k = rope(k.reshape(B, S, nkv, d)).transpose(1, 2).repeat_interleave(nh // nkv, dim=1)
+        q, k = q.reshape(B, S, nh, d), k.reshape(B, S, nkv, d)
+        if cfg.qk_norm:  # per-head RMSNorm over head_dim before the rotation, as in the published QK-Norm decoders
+            q, k = rms(q, tp[p + "q_norm"]), rms(k, tp[p + "k_norm"])
+        q = rope(q).transpose(1, 2)
+        k = rope(k).transpose(1, 2).repeat_interleave(nh // nkv, dim=1)
         v = v.reshape(B, S, nkv, d).transpose(1, 2).repeat_interleave(nh // nkv, dim=1)
         o = F.scaled_dot_product_attention(q, k, v, is_causal=True)
         x = x + F.linear(o.transpose(1, 2).reshape(B, S, cfg.h_q), tp[p + "wo"]) * cfg.resid_scale
@@ -140,7 +145,7 @@ def _torch_loss(cfg, tp, tok, lab):
                            ignore_index=-1), z
 
 
-@pytest.mark.parametrize("variant", VARIANTS[1:], ids=["mup", "tied", "tied+mup"])
+@pytest.mark.parametrize("variant", VARIANTS[1:], ids=VARIANT_IDS[1:])
 def test_model_variants_match_torch_autograd(variant):
     cfg = tiny_cfg(**variant)
     params = tiny_params(cfg, seed=21)
