@@ -108,9 +108,12 @@ NCU_GEMM_TRAFFIC_OF = ("one launch of gemm_tc_pair_kernel at M 8192, N 11264, K 
 
 def variant_kwargs(args, w):
     """--variant mup_tied: the muP factors of the paper's MiniCPM rows (scale_emb 12, scale_depth 1.4, dim_model_base 256)
-    and tied input/output embeddings on top of the workload's shape; the default is the plain decoder."""
+    and tied input/output embeddings on top of the workload's shape; --variant qknorm_tied: per-head QK-Norm and tied
+    embeddings (the paper's Qwen3 row); the default is the plain decoder."""
     if args.variant == "plain":
         return {}
+    if args.variant == "qknorm_tied":  # the Qwen3 column: per-head QK-Norm, tied embeddings, no muP
+        return dict(qk_norm=1, tie_embeddings=1)
     return dict(emb_scale=12.0, resid_scale=1.4 / w["n_layers"] ** 0.5, logit_scale=256.0 / w["d_model"], tie_embeddings=1)
 
 
@@ -346,7 +349,7 @@ def main():
     ap.add_argument("--workload", default="c3_1b", choices=sorted(SI.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel separately in the timed region")
-    ap.add_argument("--variant", default="plain", choices=["plain", "mup_tied"],
+    ap.add_argument("--variant", default="plain", choices=["plain", "mup_tied", "qknorm_tied"],
                     help="model variant on the workload's shape (default: the plain decoder the metric is quoted on)")
     ap.add_argument("--no-overlap", action="store_true", help="ablation: weight-gradient GEMMs on the main stream")
     ap.add_argument("--no-fused-update", action="store_true", help="ablation: separate AdamW pass over all parameters")

@@ -46,6 +46,8 @@ typedef struct {
   float resid_scale;              /* x <- R(x + resid_scale * branch), both branches       (muP: scale_depth / sqrt(n_layers)) */
   float logit_scale;              /* z = logit_scale * (h_F W^T)                            (muP: dim_model_base / d_model) */
   int32_t tie_embeddings;         /* 1: no lm_head parameter; the head reads the embedding table and both gradients add */
+  int32_t qk_norm;                /* 1: per-head RMSNorm of q and k before the rotation (Qwen3 column of the same appendix);
+                                     adds the gains layers.{l}.q_norm and layers.{l}.k_norm [head_dim], eps = rms_eps */
 } ft_config;
 
 typedef struct ft_model ft_model;

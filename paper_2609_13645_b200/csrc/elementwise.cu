@@ -189,6 +189,27 @@ __global__ void colsum_kernel(const float* __restrict__ partial, float* __restri
   }
 }
 
+// the same for a partial buffer of 2 d columns whose halves belong to two output tensors (query gain | key gain)
+__global__ void colsum2_kernel(const float* __restrict__ partial, float* __restrict__ out_a, float* __restrict__ out_b,
+                               int nblk, int d) {
+  pdl_trigger();
+  pdl_wait();
+  __shared__ float s[8][33];
+  const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
+  const int c = blockIdx.x * 32 + cx;
+  float a = 0.f;
+  if (c < 2 * d)
+    for (int b = ry; b < nblk; b += 8) a += partial[(long long)b * 2 * d + c];
+  s[ry][cx] = a;
+  __syncthreads();
+  if (ry == 0 && c < 2 * d) {
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += s[w][cx];
+    if (c < d) out_a[c] = tot; else out_b[c - d] = tot;
+  }
+}
+
 // ---------------------------------------------------------------- SwiGLU backward
 __global__ void swiglu_bwd_kernel(const bf16* __restrict__ d_a, const bf16* __restrict__ gu, bf16* __restrict__ d_gu,
                                   long long total_chunks, int chunks_per_row, int f) {
@@ -528,6 +549,106 @@ adamw_kernel(float* __restrict__ p, float* __restrict__ m, float* __restrict__ v
   }
 }
 
+// ---------------------------------------------------------------- per-head QK-Norm backward
+// D/8 lanes per (token, head) row of D entries of dqkv (query heads, then key heads), in place.  dy = the row as the
+// attention backward left it (gradient with respect to the normalised, gained, un-rotated head).  The unit-RMS value
+// x_hat = x r is rebuilt from the stored rotated head: x_hat = rotate^-1(q) / gain.  Then
+//   dx = r (gain dy - x_hat mean_k(gain dy x_hat)),   dgain_k += dy_k x_hat_k.
+// Rows are dealt to warps in a fixed grid-strided order and every warp keeps its dgain sums in registers; warps are
+// added in warp order into one partial row per block ([block][2][D]: query gain, key gain), blocks by colsum.
+template <int D>
+__global__ void __launch_bounds__(256)
+qknorm_bwd_kernel(bf16* __restrict__ dqkv, const bf16* __restrict__ qkv, const float* __restrict__ rr,
+                  const bf16* __restrict__ gain_q, const bf16* __restrict__ gain_k, const float* __restrict__ cosT,
+                  const float* __restrict__ sinT, float* __restrict__ partial, int T, int S, int nh, int nkv) {
+  pdl_trigger();
+  pdl_wait();
+  constexpr int HALF = D / 2;
+  constexpr int LPR = D / 8;     // lanes per row: each owns columns 4 l .. 4 l + 3 and the same + D/2 (8-byte accesses)
+  constexpr int RPW = 32 / LPR;  // rows a warp handles at once
+  __shared__ float s_dg[8][2][D];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int sub = lane / LPR, l = lane % LPR, c0 = 4 * l;
+  const int heads = nh + nkv, nqkv = (nh + 2 * nkv) * D;
+  float dgq[8], dgk[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) { dgq[e] = 0.f; dgk[e] = 0.f; }
+  auto load4 = [](const bf16* p, float* f) {
+    const uint2 v = *reinterpret_cast<const uint2*>(p);
+    f[0] = bf16_lo(v.x); f[1] = bf16_hi(v.x); f[2] = bf16_lo(v.y); f[3] = bf16_hi(v.y);
+  };
+  const long long rows = (long long)T * heads;
+  const long long stride = (long long)gridDim.x * 8 * RPW;
+  for (long long base = ((long long)blockIdx.x * 8 + warp) * RPW; base < rows; base += stride) {
+    const long long row = base + sub;
+    const bool live = row < rows;
+    const long long rw = live ? row : 0;
+    const int t = (int)(rw / heads), hd = (int)(rw % heads);
+    const bool is_q = hd < nh;
+    const long long off = (long long)t * nqkv + (is_q ? hd * D : nh * D + (hd - nh) * D) + c0;
+    const bf16* g = (is_q ? gain_q : gain_k) + c0;
+    const int pos = t % S;
+    float q1[4], q2[4], dy[8], gn[8], xh[8];
+    load4(qkv + off, q1);
+    load4(qkv + off + HALF, q2);
+    load4(dqkv + off, dy);
+    load4(dqkv + off + HALF, dy + 4);
+    load4(g, gn);
+    load4(g + HALF, gn + 4);
+    const float4 cs4 = *reinterpret_cast<const float4*>(cosT + (long long)pos * HALF + c0);
+    const float4 sn4 = *reinterpret_cast<const float4*>(sinT + (long long)pos * HALF + c0);
+    const float cs[4] = {cs4.x, cs4.y, cs4.z, cs4.w}, sn[4] = {sn4.x, sn4.y, sn4.z, sn4.w};
+    float dot = 0.f;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      xh[e] = (q1[e] * cs[e] + q2[e] * sn[e]) / gn[e];          // inverse rotation, then the gain divided out
+      xh[4 + e] = (q2[e] * cs[e] - q1[e] * sn[e]) / gn[4 + e];
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) dot += gn[e] * dy[e] * xh[e];
+#pragma unroll
+    for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+    dot *= 1.0f / (float)D;
+    const float r = live ? rr[row] : 0.f;
+    if (live) {
+      float o[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) o[e] = r * (gn[e] * dy[e] - xh[e] * dot);
+      uint2 w0, w1;
+      w0.x = pack_bf16(o[0], o[1]); w0.y = pack_bf16(o[2], o[3]);
+      w1.x = pack_bf16(o[4], o[5]); w1.y = pack_bf16(o[6], o[7]);
+      *reinterpret_cast<uint2*>(dqkv + off) = w0;
+      *reinterpret_cast<uint2*>(dqkv + off + HALF) = w1;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        if (is_q) dgq[e] += dy[e] * xh[e]; else dgk[e] += dy[e] * xh[e];
+      }
+    }
+  }
+  // the RPW row groups of a warp, added in group order (lane sub 0 collects), then warps in warp order
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    float aq = 0.f, ak = 0.f;
+#pragma unroll
+    for (int u = 0; u < RPW; ++u) {
+      aq += __shfl_sync(0xffffffffu, dgq[e], u * LPR + l);
+      ak += __shfl_sync(0xffffffffu, dgk[e], u * LPR + l);
+    }
+    if (sub == 0) {
+      const int c = (e < 4) ? c0 + e : HALF + c0 + (e - 4);
+      s_dg[warp][0][c] = aq;
+      s_dg[warp][1][c] = ak;
+    }
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < 2 * D; i += blockDim.x) {
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += s_dg[w][i / D][i % D];
+    partial[(long long)blockIdx.x * 2 * D + i] = tot;
+  }
+}
+
 // ---------------------------------------------------------------- initialisation
 __device__ __forceinline__ unsigned long long splitmix64(unsigned long long z) {
   z += 0x9E3779B97F4A7C15ull;
@@ -614,6 +735,27 @@ int rmsnorm_bwd(const bf16* dy, const bf16* x, const float* r, const bf16* g, co
   }
 #undef FS_NORM_CASE
   if (launch_pdl(colsum_kernel, (h + 31) / 32, 256, 0, st, partial, dg, nblk, h) != cudaSuccess) return -1;
+  return ok(2);
+}
+
+int qknorm_bwd(bf16* dqkv, const bf16* qkv, const float* r, const bf16* gain_q, const bf16* gain_k, const float* cosT,
+               const float* sinT, float* dgain_q, float* dgain_k, float* partial, size_t partial_floats, int T, int S,
+               int nh, int nkv, int d, cudaStream_t st) {
+  // many small blocks: the kernel is a chain of short dependent loads per row, so it lives on blocks in flight
+  const long long rows = (long long)T * (nh + nkv);
+  long long want = (rows + 8 * (32 / (d / 8)) - 1) / (8 * (32 / (d / 8)));
+  const long long cap = (long long)(partial_floats / (2 * (size_t)d));
+  if (want > 148 * 8) want = 148 * 8;
+  if (want > cap) want = cap;
+  if (want < 1) return -1;
+  const int nblk = (int)want;
+  cudaError_t e;
+  if (d == 64) e = launch_pdl(qknorm_bwd_kernel<64>, nblk, 256, 0, st, dqkv, qkv, r, gain_q, gain_k, cosT, sinT, partial, T, S, nh, nkv);
+  else if (d == 128) e = launch_pdl(qknorm_bwd_kernel<128>, nblk, 256, 0, st, dqkv, qkv, r, gain_q, gain_k, cosT, sinT, partial, T, S, nh, nkv);
+  else return -1;
+  if (e != cudaSuccess) return -1;
+  // partial is [nblk][2 d]: column sums give dgain_q | dgain_k side by side; they land in two gradient tensors
+  if (launch_pdl(colsum2_kernel, (2 * d + 31) / 32, 256, 0, st, partial, dgain_q, dgain_k, nblk, d) != cudaSuccess) return -1;
   return ok(2);
 }
 

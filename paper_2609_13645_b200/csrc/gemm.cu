@@ -59,6 +59,11 @@ struct GemmDev {
   int seq, head_dim, rope_cols, d_ffn;
   int panel;               // tile numbering (see tile_coords)
   float alpha;             // accumulator scale (1: off)
+  float* qk_r;             // per-head QK-Norm in the RoPE epilogue (null: off)
+  const bf16* qk_gain_q;
+  const bf16* qk_gain_k;
+  int n_q_heads;
+  float qk_eps;
   int ksplit;              // > 1: the K blocks are divided over ksplit work units per output tile
   long long split_stride;  // elements between the partial outputs of consecutive K parts
   int balanced;            // 1: the last partial wave of tiles is divided along K and runs first (see WorkIter)
@@ -341,6 +346,22 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
         }
       } else {
         uint32_t r2[32];
+        // per-head QK-Norm: a first pass over the head's accumulators for r, which is applied (with the gain) in the
+        // rotation pass below
+        float qr = 1.0f;
+        const bf16* gain = nullptr;
+        if (p.qk_r != nullptr) {
+          float ss = 0.f;
+          for (int c = 0; c < d; c += 32) {
+            ld_acc32(taddr, hc + c, r, fx, 1.0f);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) ss = fmaf(__uint_as_float(r[j]), __uint_as_float(r[j]), ss);
+          }
+          qr = 1.0f / sqrtf(ss / (float)d + p.qk_eps);
+          const int head = g0 / d;
+          gain = head < p.n_q_heads ? p.qk_gain_q : p.qk_gain_k;
+          if (row_ok) p.qk_r[(long long)row * (p.rope_cols / d) + head] = qr;
+        }
         for (int i0 = 0; i0 < half; i0 += 32) {
           if (fx.n == 0) {
             tmem_ld32(taddr + hc + i0, r);
@@ -362,8 +383,12 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
               const float ss[4] = {s4.x, s4.y, s4.z, s4.w};
 #pragma unroll
               for (int u = 0; u < 4; ++u) {
-                const float x1 = __uint_as_float(r[j + u]);
-                const float x2 = __uint_as_float(r2[j + u]);
+                float x1 = __uint_as_float(r[j + u]);
+                float x2 = __uint_as_float(r2[j + u]);
+                if (gain != nullptr) {
+                  x1 = x1 * qr * __bfloat162float(gain[i0 + j + u]);
+                  x2 = x2 * qr * __bfloat162float(gain[i0 + half + j + u]);
+                }
                 lo[j + u] = x1 * cc[u] - x2 * ss[u];
                 hi[j + u] = x2 * cc[u] + x1 * ss[u];
               }
@@ -999,6 +1024,7 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
   p.seq = a.seq; p.head_dim = a.head_dim; p.rope_cols = a.rope_cols; p.d_ffn = a.d_ffn;
   set_adam(p, a);
   p.alpha = a.alpha;
+  p.qk_r = a.qk_r; p.qk_gain_q = a.qk_gain_q; p.qk_gain_k = a.qk_gain_k; p.n_q_heads = a.n_q_heads; p.qk_eps = a.qk_eps;
   p.panel = (size_t)a.M * a.K * sizeof(bf16) > (48u << 20) ? 1 : 0;
   p.ksplit = 1; p.split_stride = 0; p.balanced = 0; p.sw_first = 0; p.sw_parts = 1; p.sw_kpb = 0; p.flags = nullptr; p.slots = nullptr;
   const int tiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN);
@@ -1026,6 +1052,7 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
   p.seq = a.seq; p.head_dim = a.head_dim; p.rope_cols = a.rope_cols; p.d_ffn = a.d_ffn;
   set_adam(p, a);
   p.alpha = a.alpha;
+  p.qk_r = a.qk_r; p.qk_gain_q = a.qk_gain_q; p.qk_gain_k = a.qk_gain_k; p.n_q_heads = a.n_q_heads; p.qk_eps = a.qk_eps;
   p.panel = (size_t)a.M * a.K * sizeof(bf16) > (48u << 20) ? 1 : 0;
   const int tiles = ((a.M + 255) / 256) * ((a.N + 255) / 256);
   const int max_pairs = sm_count() / 2;
@@ -1129,6 +1156,7 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream) {
     return cudaErrorInvalidValue;
   if (a.epi == EPI_BF16_RESID && !a.resid) return cudaErrorInvalidValue;
   if (a.alpha != 1.0f && (a.epi == EPI_ROPE || a.epi == EPI_SWIGLU)) return cudaErrorInvalidValue;
+  if (a.qk_r && (a.epi != EPI_ROPE || !a.qk_gain_q || !a.qk_gain_k)) return cudaErrorInvalidValue;
   if (a.adam && ((a.epi != EPI_F32 && a.epi != EPI_F32_ACC) || !a.adam->p || !a.adam->m || !a.adam->v || !a.adam->pb ||
                  !a.adam->scalars || !a.adam->sq_slots))
     return cudaErrorInvalidValue;

@@ -48,6 +48,14 @@ struct GemmArgs {
   const float* rope_cos = nullptr;  // fp32 [seq, head_dim/2]
   const float* rope_sin = nullptr;
   int seq = 1, head_dim = 64, rope_cols = 0;
+  // EPI_ROPE with per-head QK-Norm (null qk_r: off): every rotated head is first RMS-normalised over its head_dim
+  // accumulators and multiplied by a gain (heads below n_q_heads use gain_q, the others gain_k); r = (mean x^2 + eps)^(-1/2)
+  // of every (row, head) is written to qk_r [M, rope_cols / head_dim] for the backward pass
+  float* qk_r = nullptr;
+  const bf16* qk_gain_q = nullptr;
+  const bf16* qk_gain_k = nullptr;
+  int n_q_heads = 0;
+  float qk_eps = 0.f;
   // EPI_SWIGLU
   bf16* gu = nullptr;  // [M, 2f] gate | up
   int d_ffn = 0;

@@ -45,6 +45,7 @@ struct Carver {
 struct LayerActs {
   bf16 *h1, *qkv, *o, *x_mid, *h2, *gu, *a;
   float *lse, *r1, *r2;
+  float* qk_r;  // per-head QK-Norm: r of every (token, query or key head); null when the variant is off
 };
 
 struct LayerTaps {  // debug copies of one layer's backward intermediates
@@ -121,7 +122,9 @@ struct ft_model {
   cudaEvent_t prof_cur = nullptr;
 
   const ParamInfo& P(int i) const { return params[i]; }
-  int idx_layer(int l, int k) const { return 1 + l * 6 + k; }  // k: 0 norm1, 1 wqkv, 2 wo, 3 norm2, 4 wgu, 5 wd
+  int per_layer() const { return cfg.qk_norm ? 8 : 6; }
+  // k: 0 norm1, 1 wqkv, 2 wo, 3 norm2, 4 wgu, 5 wd, (QK-Norm: 6 q_norm, 7 k_norm)
+  int idx_layer(int l, int k) const { return 1 + l * per_layer() + k; }
   bf16* wb(int i) const { return pbf + params[i].offset; }
   float* gr(int i) const { return grad + params[i].offset; }
 };
@@ -151,6 +154,7 @@ bool valid_config(const ft_config* c, std::string* why) {
   if (!(c->rms_eps > 0.f) || !(c->rope_theta > 0.f)) return bad("rms_eps and rope_theta must be positive");
   if (c->emb_scale < 0.f || c->resid_scale < 0.f || c->logit_scale < 0.f) return bad("negative scale factor");
   if (c->tie_embeddings != 0 && c->tie_embeddings != 1) return bad("tie_embeddings must be 0 or 1");
+  if (c->qk_norm != 0 && c->qk_norm != 1) return bad("qk_norm must be 0 or 1");
   return true;
 }
 
@@ -187,6 +191,10 @@ size_t carve(ft_model* m, uint8_t* base) {
     add(p + "norm2", h, 0, false);
     add(p + "wgu", 2 * f, h, true);
     add(p + "wd", h, f, false);
+    if (c.qk_norm) {
+      add(p + "q_norm", c.head_dim, 0, false);
+      add(p + "k_norm", c.head_dim, 0, false);
+    }
   }
   add("norm_f", h, 0, false);
   if (!c.tie_embeddings) add("lm_head", V, h, false);
@@ -215,6 +223,7 @@ size_t carve(ft_model* m, uint8_t* base) {
     a.x_mid = cv.take<bf16>(T * h); a.h2 = cv.take<bf16>(T * h); a.gu = cv.take<bf16>(T * 2 * f);
     a.a = cv.take<bf16>(T * f); a.lse = cv.take<float>(T * c.n_heads); a.r1 = cv.take<float>(T);
     a.r2 = cv.take<float>(T);
+    a.qk_r = c.qk_norm ? cv.take<float>(T * (size_t)(c.n_heads + c.n_kv_heads)) : nullptr;
   }
   m->rF = cv.take<float>(T); m->ce_lse = cv.take<float>(T); m->loss_row = cv.take<float>(T);
   m->hF = cv.take<bf16>(T * h); m->d_hF = cv.take<bf16>(T * h);
@@ -359,6 +368,10 @@ ft_status layer_forward(ft_model* m, int l, LayerActs& a, int B, int S) {
     g.A = a.h1; g.lda = h; g.B = m->wb(m->idx_layer(l, 1)); g.ldb = h; g.C = a.qkv; g.ldc = nqkv;
     g.M = T; g.N = nqkv; g.K = h; g.epi = EPI_ROPE;
     g.rope_cos = m->rope_cos; g.rope_sin = m->rope_sin; g.seq = S; g.head_dim = m->d; g.rope_cols = hq + m->hkv;
+    if (m->cfg.qk_norm) {
+      g.qk_r = a.qk_r; g.qk_gain_q = m->wb(m->idx_layer(l, 6)); g.qk_gain_k = m->wb(m->idx_layer(l, 7));
+      g.n_q_heads = m->cfg.n_heads; g.qk_eps = m->cfg.rms_eps;
+    }
     FT_GEMM(g);
   }
   prof_begin(m);
@@ -460,6 +473,14 @@ ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
                         m->cfg.n_kv_heads, m->d, &m->sc->err, st));
   m->launches += 3;
   prof_end(m, FT_PROF_ATTN_BWD, 4.0 * B * m->cfg.n_heads * (double)S * S * m->d, 3);
+  if (m->cfg.qk_norm) {
+    // d_q, d_k so far are gradients of the normalised heads: through the per-head norm, in place, and the two gain gradients
+    FT_LAUNCH(FT_PROF_NORM, 6.0 * T * (hq + m->hkv),
+              qknorm_bwd(m->d_qkv, a.qkv, a.qk_r, m->wb(m->idx_layer(l, 6)), m->wb(m->idx_layer(l, 7)), m->rope_cos,
+                         m->rope_sin, m->gr(m->idx_layer(l, 6)), m->gr(m->idx_layer(l, 7)), m->norm_partial,
+                         (size_t)elementwise_blocks_for_norm(m->maxT) * h, T, S,
+                         m->cfg.n_heads, m->cfg.n_kv_heads, m->d, st));
+  }
   s = linear_backward(m, m->d_qkv, a.h1, m->idx_layer(l, 1), m->d_h, T, nqkv, h, 3);
   if (s) return s;
   if (tp) {
@@ -501,7 +522,7 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
     if (s) return s;
   }
   const bool tied = m->cfg.tie_embeddings != 0;
-  const int i_normf = 1 + 6 * L, i_head = tied ? 0 : 2 + 6 * L;  // tied: the head reads (and adds its gradient to) the table
+  const int i_normf = 1 + m->per_layer() * L, i_head = tied ? 0 : i_normf + 1;  // tied: the head reads (and adds its gradient to) the table
   FT_LAUNCH(FT_PROF_NORM, 4.0 * T * h, rmsnorm_fwd(m->x[L], m->wb(i_normf), m->hF, m->rF, T, h, m->cfg.rms_eps, st));
 
   // output head + cross-entropy (+ both head gradients) in chunks of rows: the logits of one chunk at a time

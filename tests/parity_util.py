@@ -23,7 +23,8 @@ def lib_config(B, ocfg, max_batch, max_seq, **extra):
                          ocfg.vocab, max_batch, max_seq, rms_eps=ocfg.rms_eps, rope_theta=ocfg.rope_theta, lr=ocfg.lr,
                          beta1=ocfg.beta1, beta2=ocfg.beta2, adam_eps=ocfg.adam_eps, weight_decay=ocfg.weight_decay,
                          max_grad_norm=ocfg.max_grad_norm, emb_scale=ocfg.emb_scale, resid_scale=ocfg.resid_scale,
-                         logit_scale=ocfg.logit_scale, tie_embeddings=int(ocfg.tie_embeddings), **extra)
+                         logit_scale=ocfg.logit_scale, tie_embeddings=int(ocfg.tie_embeddings), qk_norm=int(ocfg.qk_norm),
+                         **extra)
 
 
 def rel_l2(a, b):

@@ -98,7 +98,7 @@ def test_gqa_head_dim_128_two_layers_with_ignored_labels():
     _check_step(ocfg, tok, lab, params)
 
 
-@pytest.mark.parametrize("variant", ["mup", "tied", "tied+mup"])
+@pytest.mark.parametrize("variant", ["mup", "tied", "tied+mup", "qknorm", "qknorm128+tied+mup"])
 def test_model_variants_match_oracle_on_every_tap_gradient_and_master(variant):
     """The paper's model families differ from the plain decoder by tied input/output embeddings and by the muP factors
     on the embedding, the residual branches and the logits: same full-step parity as configuration 1."""
@@ -108,8 +108,17 @@ def test_model_variants_match_oracle_on_every_tap_gradient_and_master(variant):
         kw.update(emb_scale=12.0, resid_scale=1.4 / math.sqrt(2), logit_scale=0.5)
     if "tied" in variant:
         kw.update(tie_embeddings=True)
+    if "qknorm" in variant:  # the Qwen3 column: per-head RMSNorm of q and k before the rotation
+        kw.update(qk_norm=True)
+    if "128" in variant:
+        kw.update(d_model=512, head_dim=128)
     ocfg = oracle_config(**kw)
     params = D.init_params(ocfg, SI.WEIGHT_SEED)
+    if ocfg.qk_norm:  # gains away from 1, so that a missing or misplaced gain shows
+        rng = np.random.default_rng(3)
+        for l in range(ocfg.n_layers):
+            for nm in ("q_norm", "k_norm"):
+                params[f"layers.{l}.{nm}"] = (1.0 + 0.25 * rng.standard_normal(ocfg.head_dim)).astype(np.float32)
     assert ("lm_head" in params) == ("tied" not in variant)
     tok, lab = SI.batch(ocfg.vocab, 2, 128, "uniform", step=0)
     _check_step(ocfg, tok, lab, params)
@@ -310,7 +319,7 @@ def test_adamw_inside_the_weight_gradient_epilogue_equals_the_separate_optimizer
         Bsz, S = 2, 128
     elif shape == "tied_mup":  # the head's gradient joins the table's: it stays with the separate pass; factors in the epilogues
         ocfg = oracle_config(n_layers=2, d_model=512, n_heads=4, n_kv_heads=2, head_dim=128, d_ffn=1024, vocab=2048,
-                             tie_embeddings=True, emb_scale=12.0, resid_scale=0.99, logit_scale=0.5)
+                             tie_embeddings=True, emb_scale=12.0, resid_scale=0.99, logit_scale=0.5, qk_norm=True)
         Bsz, S = 2, 1024
     elif shape == "split_k":   # weight gradients with few tiles and 2048 tokens: K split over 4 parts
         ocfg = oracle_config(n_layers=2, d_model=512, n_heads=4, n_kv_heads=2, head_dim=128, d_ffn=1024, vocab=2048)
