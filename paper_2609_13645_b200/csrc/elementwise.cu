@@ -189,23 +189,24 @@ __global__ void colsum_kernel(const float* __restrict__ partial, float* __restri
   }
 }
 
-// the same for a partial buffer of 2 d columns whose halves belong to two output tensors (query gain | key gain)
-__global__ void colsum2_kernel(const float* __restrict__ partial, float* __restrict__ out_a, float* __restrict__ out_b,
-                               int nblk, int d) {
+// the same for a partial buffer of 2 d columns whose halves belong to two output tensors (query gain | key gain);
+// 32 row groups per block (the buffer has up to 1184 rows), added in group order
+__global__ void __launch_bounds__(1024)
+colsum2_kernel(const float* __restrict__ partial, float* __restrict__ out_a, float* __restrict__ out_b, int nblk, int d) {
   pdl_trigger();
   pdl_wait();
-  __shared__ float s[8][33];
+  __shared__ float s[32][33];
   const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
   const int c = blockIdx.x * 32 + cx;
   float a = 0.f;
   if (c < 2 * d)
-    for (int b = ry; b < nblk; b += 8) a += partial[(long long)b * 2 * d + c];
+    for (int b = ry; b < nblk; b += 32) a += partial[(long long)b * 2 * d + c];
   s[ry][cx] = a;
   __syncthreads();
   if (ry == 0 && c < 2 * d) {
     float tot = 0.f;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) tot += s[w][cx];
+    for (int w = 0; w < 32; ++w) tot += s[w][cx];
     if (c < d) out_a[c] = tot; else out_b[c - d] = tot;
   }
 }
@@ -577,32 +578,37 @@ qknorm_bwd_kernel(bf16* __restrict__ dqkv, const bf16* __restrict__ qkv, const f
     const uint2 v = *reinterpret_cast<const uint2*>(p);
     f[0] = bf16_lo(v.x); f[1] = bf16_hi(v.x); f[2] = bf16_lo(v.y); f[3] = bf16_hi(v.y);
   };
-  const long long rows = (long long)T * heads;
-  const long long stride = (long long)gridDim.x * 8 * RPW;
-  for (long long base = ((long long)blockIdx.x * 8 + warp) * RPW; base < rows; base += stride) {
-    const long long row = base + sub;
+  // this lane's eight gains of either kind and their reciprocals (rounded once), the same for every row
+  float gq[8], gk[8], rgq[8], rgk[8];
+  load4(gain_q + c0, gq); load4(gain_q + c0 + HALF, gq + 4);
+  load4(gain_k + c0, gk); load4(gain_k + c0 + HALF, gk + 4);
+#pragma unroll
+  for (int e = 0; e < 8; ++e) { rgq[e] = __frcp_rn(gq[e]); rgk[e] = __frcp_rn(gk[e]); }
+  const int rows = T * heads;  // at most 2^24 tokens x heads: fits
+  const int stride = (int)gridDim.x * 8 * RPW;
+  for (int base = ((int)blockIdx.x * 8 + warp) * RPW; base < rows; base += stride) {
+    const int row = base + sub;
     const bool live = row < rows;
-    const long long rw = live ? row : 0;
-    const int t = (int)(rw / heads), hd = (int)(rw % heads);
+    const int rw = live ? row : 0;
+    const int t = rw / heads, hd = rw - t * heads;
     const bool is_q = hd < nh;
     const long long off = (long long)t * nqkv + (is_q ? hd * D : nh * D + (hd - nh) * D) + c0;
-    const bf16* g = (is_q ? gain_q : gain_k) + c0;
     const int pos = t % S;
-    float q1[4], q2[4], dy[8], gn[8], xh[8];
+    float q1[4], q2[4], dy[8], gn[8], rg[8], xh[8];
     load4(qkv + off, q1);
     load4(qkv + off + HALF, q2);
     load4(dqkv + off, dy);
     load4(dqkv + off + HALF, dy + 4);
-    load4(g, gn);
-    load4(g + HALF, gn + 4);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) { gn[e] = is_q ? gq[e] : gk[e]; rg[e] = is_q ? rgq[e] : rgk[e]; }
     const float4 cs4 = *reinterpret_cast<const float4*>(cosT + (long long)pos * HALF + c0);
     const float4 sn4 = *reinterpret_cast<const float4*>(sinT + (long long)pos * HALF + c0);
     const float cs[4] = {cs4.x, cs4.y, cs4.z, cs4.w}, sn[4] = {sn4.x, sn4.y, sn4.z, sn4.w};
     float dot = 0.f;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      xh[e] = (q1[e] * cs[e] + q2[e] * sn[e]) / gn[e];          // inverse rotation, then the gain divided out
-      xh[4 + e] = (q2[e] * cs[e] - q1[e] * sn[e]) / gn[4 + e];
+      xh[e] = (q1[e] * cs[e] + q2[e] * sn[e]) * rg[e];          // inverse rotation, then the gain divided out
+      xh[4 + e] = (q2[e] * cs[e] - q1[e] * sn[e]) * rg[4 + e];
     }
 #pragma unroll
     for (int e = 0; e < 8; ++e) dot += gn[e] * dy[e] * xh[e];
@@ -755,7 +761,7 @@ int qknorm_bwd(bf16* dqkv, const bf16* qkv, const float* r, const bf16* gain_q, 
   else return -1;
   if (e != cudaSuccess) return -1;
   // partial is [nblk][2 d]: column sums give dgain_q | dgain_k side by side; they land in two gradient tensors
-  if (launch_pdl(colsum2_kernel, (2 * d + 31) / 32, 256, 0, st, partial, dgain_q, dgain_k, nblk, d) != cudaSuccess) return -1;
+  if (launch_pdl(colsum2_kernel, (2 * d + 31) / 32, 1024, 0, st, partial, dgain_q, dgain_k, nblk, d) != cudaSuccess) return -1;
   return ok(2);
 }
 

@@ -30,6 +30,7 @@ def main():
     ap.add_argument("kernel", choices=["gemm", "attn_fwd", "attn_bwd", "step"])
     ap.add_argument("--workload", default="c3_1b")
     ap.add_argument("--layers", type=int, default=1)
+    ap.add_argument("--qk-norm", action="store_true", help="step: per-head QK-Norm variant")
     ap.add_argument("--unfused", action="store_true", help="step: separate optimizer pass instead of the fused epilogue")
     ap.add_argument("--M", type=int, default=8192)
     ap.add_argument("--N", type=int, default=4096)
@@ -58,7 +59,7 @@ def main():
         w = SI.WORKLOADS[a.workload]
         Bsz, S = w["batch"], w["seq"]
         cfg = B.make_config(a.layers, w["d_model"], w["n_heads"], w["n_kv_heads"], w["head_dim"], w["d_ffn"], w["vocab"],
-                            Bsz, S, recompute=w.get("recompute", 0))
+                            Bsz, S, recompute=w.get("recompute", 0), qk_norm=int(a.qk_norm))
         model = B.Model(cfg, seed=SI.WEIGHT_SEED)
         model.set_fused_update(not a.unfused)
         total = 0.0
