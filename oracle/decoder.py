@@ -32,7 +32,7 @@ from __future__ import annotations
 
 import dataclasses
 import math
-from typing import Dict, List, Tuple
+from typing import Dict, List, Optional, Tuple
 
 import numpy as np
 
@@ -74,6 +74,12 @@ class Config:
     # key heads of a layer; eps = rms_eps) before the rotation.  The paper names it without a formula; this is the
     # published Qwen3 definition.
     qk_norm: bool = False
+    # LongRoPE (appendix "Model Architectures", MiniCPM4 rows: "Position encoding: LongRoPE"): the paper names it
+    # without its constants; reading = the published method's form, a per-frequency rescale factor lambda_i and one
+    # magnitude factor: angle(p, i) = p * theta^(-2i/d) / lambda_i, and cos, sin are multiplied by rope_mscale.
+    # None / 1 is plain RoPE.  (Which lambda_i a checkpoint uses is model data, passed in like the weights.)
+    rope_factors: Optional[Tuple[float, ...]] = None
+    rope_mscale: float = 1.0
 
     @property
     def h_q(self) -> int:
@@ -188,13 +194,15 @@ def init_params(cfg: Config, seed: int) -> Dict[str, np.ndarray]:
 # --------------------------------------------------------------------------
 # building blocks (each in fp64, inputs already carry any contract rounding)
 # --------------------------------------------------------------------------
-def rope_tables(S: int, d: int, theta: float) -> Tuple[np.ndarray, np.ndarray]:
-    """cos/sin of p * theta**(-2i/d), p = 0..S-1, i = 0..d/2-1: fp64 values stored as fp32."""
+def rope_tables(S: int, d: int, theta: float, factors=None, mscale: float = 1.0) -> Tuple[np.ndarray, np.ndarray]:
+    """mscale * cos/sin of p * theta**(-2i/d) / factors_i, p = 0..S-1, i = 0..d/2-1: fp64 values stored as fp32."""
     i = np.arange(d // 2, dtype=np.float64)
     inv_freq = np.power(float(theta), -2.0 * i / d)
+    if factors is not None:
+        inv_freq = inv_freq / np.asarray(factors, dtype=np.float64)
     ang = np.arange(S, dtype=np.float64)[:, None] * inv_freq[None, :]
-    c = np.cos(ang).astype(np.float32).astype(np.float64)
-    s = np.sin(ang).astype(np.float32).astype(np.float64)
+    c = (float(mscale) * np.cos(ang)).astype(np.float32).astype(np.float64)
+    s = (float(mscale) * np.sin(ang)).astype(np.float32).astype(np.float64)
     return c, s
 
 
@@ -335,7 +343,7 @@ def forward_backward(cfg: Config, params: Dict[str, np.ndarray], tokens: np.ndar
 
     # 1. compute copies: W^b = R(W) for every parameter (matrices and gains)
     W = {k_: R(np.asarray(v_, dtype=np.float64)) for k_, v_ in params.items()}
-    cos, sin = rope_tables(S, d, cfg.rope_theta)
+    cos, sin = rope_tables(S, d, cfg.rope_theta, cfg.rope_factors, cfg.rope_mscale)
 
     # 2. embedding: row copy (exact when emb_scale is 1: R of a bf16 value is itself)
     s_e, s_r, s_l = float(cfg.emb_scale), float(cfg.resid_scale), float(cfg.logit_scale)

@@ -68,8 +68,9 @@ def test_bf16_round_ties_to_even_and_idempotent():
 # ---------------------------------------------------------------- whole backward: finite differences
 VARIANTS = [dict(), dict(emb_scale=12.0, resid_scale=1.4 / math.sqrt(2), logit_scale=256.0 / 1024.0),
             dict(tie_embeddings=True), dict(tie_embeddings=True, emb_scale=3.0, resid_scale=0.7, logit_scale=0.5),
-            dict(qk_norm=True), dict(qk_norm=True, tie_embeddings=True, n_kv_heads=1)]
-VARIANT_IDS = ["plain", "mup", "tied", "tied+mup", "qknorm", "qknorm+tied+mqa"]
+            dict(qk_norm=True), dict(qk_norm=True, tie_embeddings=True, n_kv_heads=1),
+            dict(rope_factors=(1.0, 1.7, 3.1, 4.9), rope_mscale=1.19, qk_norm=True)]
+VARIANT_IDS = ["plain", "mup", "tied", "tied+mup", "qknorm", "qknorm+tied+mqa", "longrope+qknorm"]
 
 
 @pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_IDS)
@@ -110,9 +111,11 @@ def _torch_loss(cfg, tp, tok, lab):
     d, nh, nkv = cfg.head_dim, cfg.n_heads, cfg.n_kv_heads
     pos = torch.arange(S, dtype=torch.float64)
     inv = torch.tensor(cfg.rope_theta, dtype=torch.float64) ** (-torch.arange(0, d, 2, dtype=torch.float64) / d)
+    if cfg.rope_factors is not None:  # LongRoPE: per-frequency rescale factors, one magnitude factor on cos and sin
+        inv = inv / torch.tensor(cfg.rope_factors, dtype=torch.float64)
     ang = torch.outer(pos, inv)
-    cos = torch.cos(ang).to(torch.float32).to(torch.float64)  # the cos/sin tables are stored as fp32
-    sin = torch.sin(ang).to(torch.float32).to(torch.float64)
+    cos = (cfg.rope_mscale * torch.cos(ang)).to(torch.float32).to(torch.float64)  # the tables are stored as fp32
+    sin = (cfg.rope_mscale * torch.sin(ang)).to(torch.float32).to(torch.float64)
 
     def rope(x):  # x [B,S,n,d]; rotate-half form
         half = torch.cat([-x[..., d // 2:], x[..., :d // 2]], dim=-1)
@@ -338,6 +341,20 @@ def test_rope_properties():
     assert abs(np.sum(rx * y) - np.sum(x * D.rope_apply_transpose(y, c[:S], s[:S]))) < 1e-10
     # angle of (p, i) is p * theta^(-2i/d)
     assert abs(c[3, 1] - np.float32(math.cos(3 * 1e4 ** (-2 / 8)))) < 1e-7
+    # LongRoPE form: angle / lambda_i, magnitude factor on both tables: norms scale by it, the relative-position
+    # property and the transpose survive, factors of 1 change nothing
+    lam, ms = (1.0, 2.0, 3.5, 8.0), 1.25
+    c2, s2 = D.rope_tables(S + 5, d, 1e4, lam, ms)
+    assert abs(c2[3, 1] - np.float32(ms * math.cos(3 * 1e4 ** (-2 / 8) / 2.0))) < 1e-7
+    assert abs(s2[7, 3] - np.float32(ms * math.sin(7 * 1e4 ** (-6 / 8) / 8.0))) < 1e-7
+    r2 = D.rope_apply(x, c2[:S], s2[:S])
+    assert np.allclose(np.linalg.norm(r2, axis=-1), ms * np.linalg.norm(x, axis=-1), rtol=1e-6)
+    a0 = np.einsum("bmnd,bknd->bnmk", r2, D.rope_apply(y, c2[:S], s2[:S]))
+    a5 = np.einsum("bmnd,bknd->bnmk", D.rope_apply(x, c2[5:S + 5], s2[5:S + 5]), D.rope_apply(y, c2[5:S + 5], s2[5:S + 5]))
+    assert np.allclose(a0, a5, atol=4e-6)
+    assert abs(np.sum(r2 * y) - np.sum(x * D.rope_apply_transpose(y, c2[:S], s2[:S]))) < 1e-10
+    c1, s1 = D.rope_tables(S, d, 1e4, (1.0,) * (d // 2), 1.0)
+    assert np.array_equal(c1, c[:S]) and np.array_equal(s1, s[:S])
 
 
 def test_rmsnorm_properties():
