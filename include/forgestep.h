@@ -83,6 +83,11 @@ ft_status ft_train_step(ft_model* m, const int32_t* dev_tokens, const int32_t* d
  * values (use ft_forward_backward to materialise gradients).  Changing the setting drops a captured graph. */
 ft_status ft_set_fused_update(ft_model* m, int32_t enable);
 
+/* Position tables in the LongRoPE form (appendix "Model Architectures", MiniCPM4 rows): angle(p, i) = p * theta^(-2i/d) /
+ * host_factors[i] for i < head_dim / 2 (NULL: all 1), and cos, sin multiplied by mscale (> 0).  Rebuilds both tables on the
+ * host in double precision and copies them (synchronises the model's stream).  The factors are model data, like weights. */
+ft_status ft_set_rope_scaling(ft_model* m, const float* host_factors, float mscale);
+
 /* Weight-gradient overlap: nothing later in the backward pass depends on a layer's weight gradients (Section 4.3's
  * fused dgrad + wgrad observation, turned into concurrency), so the library enqueues those GEMMs on a second stream
  * of its own, ordered by events against the kernels that produce their inputs and against the kernels that later

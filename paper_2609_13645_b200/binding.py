@@ -78,6 +78,8 @@ def lib():
         L.ft_get_gemm_profile.restype = C.c_int
         L.ft_set_fused_update.argtypes = [vp, i32]
         L.ft_set_fused_update.restype = C.c_int
+        L.ft_set_rope_scaling.argtypes = [vp, vp, C.c_float]
+        L.ft_set_rope_scaling.restype = C.c_int
         L.ft_set_overlap.argtypes = [vp, i32]
         L.ft_set_overlap.restype = C.c_int
         L.ft_set_graph.argtypes = [vp, i32]
@@ -240,6 +242,12 @@ class Model:
     def set_fused_update(self, enable: bool):
         """AdamW inside the weight-gradient GEMM epilogues (default on; only takes effect with clipping off)."""
         self._check(lib().ft_set_fused_update(self._h, 1 if enable else 0))
+
+    def set_rope_scaling(self, factors=None, mscale: float = 1.0):
+        """LongRoPE-form position tables: per-frequency rescale factors (head_dim / 2 floats, None = 1) and a magnitude
+        factor on cos and sin."""
+        f = None if factors is None else np.ascontiguousarray(factors, dtype=np.float32)
+        self._check(lib().ft_set_rope_scaling(self._h, None if f is None else C.c_void_p(f.ctypes.data), float(mscale)))
 
     def set_overlap(self, enable: bool):
         """Weight-gradient GEMMs on a second stream, concurrent with the rest of the backward pass (default on)."""

@@ -561,7 +561,8 @@ template <int D>
 __global__ void __launch_bounds__(256)
 qknorm_bwd_kernel(bf16* __restrict__ dqkv, const bf16* __restrict__ qkv, const float* __restrict__ rr,
                   const bf16* __restrict__ gain_q, const bf16* __restrict__ gain_k, const float* __restrict__ cosT,
-                  const float* __restrict__ sinT, float* __restrict__ partial, int T, int S, int nh, int nkv) {
+                  const float* __restrict__ sinT, float* __restrict__ partial, float inv_mscale2, int T, int S, int nh,
+                  int nkv) {
   pdl_trigger();
   pdl_wait();
   constexpr int HALF = D / 2;
@@ -583,7 +584,8 @@ qknorm_bwd_kernel(bf16* __restrict__ dqkv, const bf16* __restrict__ qkv, const f
   load4(gain_q + c0, gq); load4(gain_q + c0 + HALF, gq + 4);
   load4(gain_k + c0, gk); load4(gain_k + c0 + HALF, gk + 4);
 #pragma unroll
-  for (int e = 0; e < 8; ++e) { rgq[e] = __frcp_rn(gq[e]); rgk[e] = __frcp_rn(gk[e]); }
+  // the tables carry a magnitude factor m (LongRoPE form): rotating back with them gives m^2 x, hence inv_mscale2
+  for (int e = 0; e < 8; ++e) { rgq[e] = __frcp_rn(gq[e]) * inv_mscale2; rgk[e] = __frcp_rn(gk[e]) * inv_mscale2; }
   const int rows = T * heads;  // at most 2^24 tokens x heads: fits
   const int stride = (int)gridDim.x * 8 * RPW;
   for (int base = ((int)blockIdx.x * 8 + warp) * RPW; base < rows; base += stride) {
@@ -745,8 +747,8 @@ int rmsnorm_bwd(const bf16* dy, const bf16* x, const float* r, const bf16* g, co
 }
 
 int qknorm_bwd(bf16* dqkv, const bf16* qkv, const float* r, const bf16* gain_q, const bf16* gain_k, const float* cosT,
-               const float* sinT, float* dgain_q, float* dgain_k, float* partial, size_t partial_floats, int T, int S,
-               int nh, int nkv, int d, cudaStream_t st) {
+               const float* sinT, float* dgain_q, float* dgain_k, float* partial, size_t partial_floats, float inv_mscale2,
+               int T, int S, int nh, int nkv, int d, cudaStream_t st) {
   // many small blocks: the kernel is a chain of short dependent loads per row, so it lives on blocks in flight
   const long long rows = (long long)T * (nh + nkv);
   long long want = (rows + 8 * (32 / (d / 8)) - 1) / (8 * (32 / (d / 8)));
@@ -756,8 +758,8 @@ int qknorm_bwd(bf16* dqkv, const bf16* qkv, const float* r, const bf16* gain_q, 
   if (want < 1) return -1;
   const int nblk = (int)want;
   cudaError_t e;
-  if (d == 64) e = launch_pdl(qknorm_bwd_kernel<64>, nblk, 256, 0, st, dqkv, qkv, r, gain_q, gain_k, cosT, sinT, partial, T, S, nh, nkv);
-  else if (d == 128) e = launch_pdl(qknorm_bwd_kernel<128>, nblk, 256, 0, st, dqkv, qkv, r, gain_q, gain_k, cosT, sinT, partial, T, S, nh, nkv);
+  if (d == 64) e = launch_pdl(qknorm_bwd_kernel<64>, nblk, 256, 0, st, dqkv, qkv, r, gain_q, gain_k, cosT, sinT, partial, inv_mscale2, T, S, nh, nkv);
+  else if (d == 128) e = launch_pdl(qknorm_bwd_kernel<128>, nblk, 256, 0, st, dqkv, qkv, r, gain_q, gain_k, cosT, sinT, partial, inv_mscale2, T, S, nh, nkv);
   else return -1;
   if (e != cudaSuccess) return -1;
   // partial is [nblk][2 d]: column sums give dgain_q | dgain_k side by side; they land in two gradient tensors

@@ -40,8 +40,8 @@ int rmsnorm_bwd(const bf16* dy, const bf16* x, const float* r, const bf16* g, co
 // Per-head QK-Norm backward, in place on dqkv's query and key heads (see the kernel); dgain_q, dgain_k [d] fp32 are
 // overwritten; partial: scratch of partial_floats floats (one row of 2 d per block; more room, more blocks, up to 1184).
 int qknorm_bwd(bf16* dqkv, const bf16* qkv, const float* r, const bf16* gain_q, const bf16* gain_k, const float* cosT,
-               const float* sinT, float* dgain_q, float* dgain_k, float* partial, size_t partial_floats, int T, int S,
-               int nh, int nkv, int d, cudaStream_t st);
+               const float* sinT, float* dgain_q, float* dgain_k, float* partial, size_t partial_floats, float inv_mscale2,
+               int T, int S, int nh, int nkv, int d, cudaStream_t st);
 int swiglu_bwd(const bf16* d_a, const bf16* gu, bf16* d_gu, int T, int f, cudaStream_t st);
 int count_labels(const int32_t* labels, int T, StepScalars* sc, cudaStream_t st);
 // per row: lse, loss contribution, and (if dz != null) dz = R((softmax(z) - onehot) * inv_count), zero for ignored rows

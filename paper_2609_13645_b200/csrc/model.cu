@@ -68,6 +68,7 @@ struct ft_model {
   float *master, *adam_m, *adam_v, *grad;
   bf16* pbf;
   float *rope_cos, *rope_sin;
+  float rope_mscale = 1.0f;  // magnitude factor folded into both tables (LongRoPE form)
   StepScalars* sc;
   int32_t *tok_dev, *lab_dev;
   std::vector<bf16*> x;  // x[l] = input of layer l, x[L] = output of the last layer
@@ -478,7 +479,7 @@ ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
     FT_LAUNCH(FT_PROF_NORM, 6.0 * T * (hq + m->hkv),
               qknorm_bwd(m->d_qkv, a.qkv, a.qk_r, m->wb(m->idx_layer(l, 6)), m->wb(m->idx_layer(l, 7)), m->rope_cos,
                          m->rope_sin, m->gr(m->idx_layer(l, 6)), m->gr(m->idx_layer(l, 7)), m->norm_partial,
-                         (size_t)elementwise_blocks_for_norm(m->maxT) * h, T, S,
+                         (size_t)elementwise_blocks_for_norm(m->maxT) * h, 1.0f / (m->rope_mscale * m->rope_mscale), T, S,
                          m->cfg.n_heads, m->cfg.n_kv_heads, m->d, st));
   }
   s = linear_backward(m, m->d_qkv, a.h1, m->idx_layer(l, 1), m->d_h, T, nqkv, h, 3);
@@ -670,6 +671,29 @@ size_t ft_workspace_bytes(const ft_config* cfg) {
   return carve(&tmp, nullptr);
 }
 
+// RoPE tables: mscale * cos/sin of angle(p, i) = p * theta^(-2i/d) / factors[i], evaluated in double on the host, stored
+// as fp32 [max_seq, d/2].  factors == nullptr: all 1.
+static ft_status build_rope_tables(ft_model* m, const float* factors, float mscale) {
+  const ft_config* cfg = &m->cfg;
+  cudaStream_t st = m->stream;
+  const int half = m->d / 2;
+  std::vector<float> cs((size_t)cfg->max_seq * half), sn((size_t)cfg->max_seq * half);
+  for (int i = 0; i < half; ++i) {
+    double inv = pow((double)cfg->rope_theta, -2.0 * i / (double)m->d);
+    if (factors) inv /= (double)factors[i];
+    for (int p = 0; p < cfg->max_seq; ++p) {
+      const double ang = (double)p * inv;
+      cs[(size_t)p * half + i] = (float)((double)mscale * cos(ang));
+      sn[(size_t)p * half + i] = (float)((double)mscale * sin(ang));
+    }
+  }
+  FT_CUDA(cudaMemcpyAsync(m->rope_cos, cs.data(), cs.size() * sizeof(float), cudaMemcpyHostToDevice, st));
+  FT_CUDA(cudaMemcpyAsync(m->rope_sin, sn.data(), sn.size() * sizeof(float), cudaMemcpyHostToDevice, st));
+  FT_CUDA(cudaStreamSynchronize(st));
+  m->rope_mscale = mscale;
+  return FT_OK;
+}
+
 ft_status ft_init_model(const ft_config* cfg, uint64_t seed, void* dev_workspace, size_t bytes, void* cuda_stream,
                         ft_model** out) {
   if (!out) return FT_EINVAL;
@@ -722,21 +746,9 @@ ft_status ft_init_model(const ft_config* cfg, uint64_t seed, void* dev_workspace
   FT_CUDA(cudaMemsetAsync(m->grad, 0, m->arena * sizeof(float), st));
   FT_LAUNCH(FT_PROF_ELEMENTWISE, 0.0, cast_bf16(m->master, m->pbf, m->arena, st));
 
-  // RoPE tables: angle(p, i) = p * theta^(-2i/d), evaluated in double on the host, stored as fp32
   {
-    const int half = m->d / 2;
-    std::vector<float> cs((size_t)cfg->max_seq * half), sn((size_t)cfg->max_seq * half);
-    for (int i = 0; i < half; ++i) {
-      const double inv = pow((double)cfg->rope_theta, -2.0 * i / (double)m->d);
-      for (int p = 0; p < cfg->max_seq; ++p) {
-        const double ang = (double)p * inv;
-        cs[(size_t)p * half + i] = (float)cos(ang);
-        sn[(size_t)p * half + i] = (float)sin(ang);
-      }
-    }
-    FT_CUDA(cudaMemcpyAsync(m->rope_cos, cs.data(), cs.size() * sizeof(float), cudaMemcpyHostToDevice, st));
-    FT_CUDA(cudaMemcpyAsync(m->rope_sin, sn.data(), sn.size() * sizeof(float), cudaMemcpyHostToDevice, st));
-    FT_CUDA(cudaStreamSynchronize(st));
+    ft_status sr = build_rope_tables(m, nullptr, 1.0f);
+    if (sr) return sr;
   }
   return FT_OK;
 }
@@ -807,6 +819,15 @@ ft_status ft_train_step(ft_model* m, const int32_t* dev_tokens, const int32_t* d
   if (s) return s;
   if (host_loss || host_gnorm) return finish(m, host_loss, host_gnorm);
   return FT_OK;
+}
+
+ft_status ft_set_rope_scaling(ft_model* m, const float* host_factors, float mscale) {
+  if (!m) return FT_EINVAL;
+  if (!(mscale > 0.f)) return fail(m, FT_EINVAL, "mscale must be positive");
+  if (host_factors)
+    for (int i = 0; i < m->d / 2; ++i)
+      if (!(host_factors[i] > 0.f)) return fail(m, FT_EINVAL, "rescale factors must be positive");
+  return build_rope_tables(m, host_factors, mscale);  // same device addresses: a captured graph stays valid
 }
 
 ft_status ft_set_overlap(ft_model* m, int32_t enable) {

@@ -31,6 +31,8 @@ def _check_step(ocfg, tok, lab, params, debug=True, recompute=0, report=None):
     Bsz, S = tok.shape
     T = Bsz * S
     model = B.Model(lib_config(B, ocfg, Bsz, S, debug_taps=1 if debug else 0, recompute=recompute), seed=1)
+    if ocfg.rope_factors is not None or ocfg.rope_mscale != 1.0:
+        model.set_rope_scaling(ocfg.rope_factors, ocfg.rope_mscale)
     load_params(model, params)
     st = D.TrainState(ocfg, params)
     loss_o, gn_o, grads_o, taps_o = st.train_step(tok, lab, mode="contract", want_taps=True)
@@ -98,7 +100,7 @@ def test_gqa_head_dim_128_two_layers_with_ignored_labels():
     _check_step(ocfg, tok, lab, params)
 
 
-@pytest.mark.parametrize("variant", ["mup", "tied", "tied+mup", "qknorm", "qknorm128+tied+mup"])
+@pytest.mark.parametrize("variant", ["mup", "tied", "tied+mup", "qknorm", "qknorm128+tied+mup", "longrope+qknorm"])
 def test_model_variants_match_oracle_on_every_tap_gradient_and_master(variant):
     """The paper's model families differ from the plain decoder by tied input/output embeddings and by the muP factors
     on the embedding, the residual branches and the logits: same full-step parity as configuration 1."""
@@ -112,6 +114,9 @@ def test_model_variants_match_oracle_on_every_tap_gradient_and_master(variant):
         kw.update(qk_norm=True)
     if "128" in variant:
         kw.update(d_model=512, head_dim=128)
+    if "longrope" in variant:  # per-frequency rescale factors growing with the index, magnitude factor on cos / sin
+        kw.update(rope_factors=tuple(float(np.float32(1.0 + 0.2 * i)) for i in range(kw["head_dim"] // 2)),
+                  rope_mscale=float(np.float32(1.1)))
     ocfg = oracle_config(**kw)
     params = D.init_params(ocfg, SI.WEIGHT_SEED)
     if ocfg.qk_norm:  # gains away from 1, so that a missing or misplaced gain shows
