@@ -36,11 +36,21 @@ def test_workspace_size_and_config_validation_run_on_the_host():
     n = B.workspace_bytes(ok)
     assert n > 0 and n % 256 == 0
     assert B.workspace_bytes(B.make_config(1, 256, 4, 4, 64, 688, 1024, 4, 128)) > n
-    for bad in (dict(head_dim=96), dict(d_model=100), dict(d_ffn=100), dict(n_kv_heads=3), dict(vocab=1001)):
+    for bad in (dict(head_dim=96), dict(d_model=100), dict(d_ffn=100), dict(n_kv_heads=3), dict(vocab=1001),
+                dict(emb_scale=-1.0), dict(resid_scale=-0.5), dict(logit_scale=-2.0), dict(tie_embeddings=2),
+                dict(qk_norm=3)):
         kw = dict(n_layers=1, d_model=256, n_heads=4, n_kv_heads=4, head_dim=64, d_ffn=688, vocab=1024, max_batch=2,
                   max_seq=128)
         kw.update(bad)
         assert B.workspace_bytes(B.make_config(**kw)) == 0, bad
+    # model variants: a tied head drops the lm_head tensors from every arena; QK-Norm adds gains and the saved r; a
+    # zero factor means 1 and changes nothing
+    base = dict(n_layers=2, d_model=256, n_heads=4, n_kv_heads=2, head_dim=64, d_ffn=688, vocab=1024, max_batch=2,
+                max_seq=128)
+    n0 = B.workspace_bytes(B.make_config(**base))
+    assert B.workspace_bytes(B.make_config(**base, tie_embeddings=1)) < n0
+    assert B.workspace_bytes(B.make_config(**base, qk_norm=1)) > n0
+    assert B.workspace_bytes(B.make_config(**base, emb_scale=0.0, resid_scale=0.0, logit_scale=0.0)) == n0
     # the 1B-shaped workload fits one B200 with room to spare
     big = B.make_config(16, 2048, 16, 8, 128, 5632, 32000, 4, 2048)
     assert B.workspace_bytes(big) < 60 * 2 ** 30

@@ -256,6 +256,10 @@ def test_error_paths_return_codes_and_keep_the_context_usable():
     assert e.value.status == B.FT_EINVAL
     with pytest.raises(B.ForgeStepError):
         model.get_tap("no_such_tap", 0)
+    for bad in ((None, 0.0), (np.zeros(ocfg.head_dim // 2), 1.0), (-np.ones(ocfg.head_dim // 2), 1.0)):
+        with pytest.raises(B.ForgeStepError) as e:
+            model.set_rope_scaling(*bad)
+        assert e.value.status == B.FT_EINVAL
     # a non-finite master makes the loss non-finite: reported, not fatal
     w = model.get_param("norm_f")
     w[0] = np.inf
