@@ -57,6 +57,7 @@ struct GemmDev {
   int M, N, K;
   int epi;
   int seq, head_dim, rope_cols, d_ffn;
+  long long rope_ld;
   int panel;               // tile numbering (see tile_coords)
   float alpha;             // accumulator scale (1: off)
   float* qk_r;             // per-head QK-Norm in the RoPE epilogue (null: off)
@@ -372,26 +373,20 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
             ld_acc32(taddr, hc + i0 + half, r2, fx, 1.0f);
           }
           if (row_ok) {
-            const float* cs = p.rope_cos + (long long)pos * half + i0;
-            const float* sn = p.rope_sin + (long long)pos * half + i0;
+            const float* cs = p.rope_cos + (long long)i0 * p.rope_ld + pos;
+            const float* sn = p.rope_sin + (long long)i0 * p.rope_ld + pos;
             float lo[32], hi[32];
 #pragma unroll
-            for (int j = 0; j < 32; j += 4) {
-              const float4 c4 = *reinterpret_cast<const float4*>(cs + j);
-              const float4 s4 = *reinterpret_cast<const float4*>(sn + j);
-              const float cc[4] = {c4.x, c4.y, c4.z, c4.w};
-              const float ss[4] = {s4.x, s4.y, s4.z, s4.w};
-#pragma unroll
-              for (int u = 0; u < 4; ++u) {
-                float x1 = __uint_as_float(r[j + u]);
-                float x2 = __uint_as_float(r2[j + u]);
-                if (gain != nullptr) {
-                  x1 = x1 * qr * __bfloat162float(gain[i0 + j + u]);
-                  x2 = x2 * qr * __bfloat162float(gain[i0 + half + j + u]);
-                }
-                lo[j + u] = x1 * cc[u] - x2 * ss[u];
-                hi[j + u] = x2 * cc[u] + x1 * ss[u];
+            for (int j = 0; j < 32; ++j) {
+              const float cc = cs[(long long)j * p.rope_ld], ss = sn[(long long)j * p.rope_ld];
+              float x1 = __uint_as_float(r[j]);
+              float x2 = __uint_as_float(r2[j]);
+              if (gain != nullptr) {
+                x1 = x1 * qr * __bfloat162float(gain[i0 + j]);
+                x2 = x2 * qr * __bfloat162float(gain[i0 + half + j]);
               }
+              lo[j] = x1 * cc - x2 * ss;
+              hi[j] = x2 * cc + x1 * ss;
             }
 #pragma unroll
             for (int j = 0; j < 32; j += 8) {
@@ -1021,7 +1016,7 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
   GemmDev p;
   p.C = a.C; p.resid = a.resid; p.gu = a.gu; p.rope_cos = a.rope_cos; p.rope_sin = a.rope_sin; p.err = a.err;
   p.ldc = a.ldc; p.M = a.M; p.N = a.N; p.K = a.K; p.epi = a.epi;
-  p.seq = a.seq; p.head_dim = a.head_dim; p.rope_cols = a.rope_cols; p.d_ffn = a.d_ffn;
+  p.seq = a.seq; p.head_dim = a.head_dim; p.rope_cols = a.rope_cols; p.d_ffn = a.d_ffn; p.rope_ld = a.rope_ld;
   set_adam(p, a);
   p.alpha = a.alpha;
   p.qk_r = a.qk_r; p.qk_gain_q = a.qk_gain_q; p.qk_gain_k = a.qk_gain_k; p.n_q_heads = a.n_q_heads; p.qk_eps = a.qk_eps;
@@ -1049,7 +1044,7 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
   GemmDev p;
   p.C = a.C; p.resid = a.resid; p.gu = a.gu; p.rope_cos = a.rope_cos; p.rope_sin = a.rope_sin; p.err = a.err;
   p.ldc = a.ldc; p.M = a.M; p.N = a.N; p.K = a.K; p.epi = a.epi;
-  p.seq = a.seq; p.head_dim = a.head_dim; p.rope_cols = a.rope_cols; p.d_ffn = a.d_ffn;
+  p.seq = a.seq; p.head_dim = a.head_dim; p.rope_cols = a.rope_cols; p.d_ffn = a.d_ffn; p.rope_ld = a.rope_ld;
   set_adam(p, a);
   p.alpha = a.alpha;
   p.qk_r = a.qk_r; p.qk_gain_q = a.qk_gain_q; p.qk_gain_k = a.qk_gain_k; p.n_q_heads = a.n_q_heads; p.qk_eps = a.qk_eps;
@@ -1160,7 +1155,7 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream) {
   if (a.adam && ((a.epi != EPI_F32 && a.epi != EPI_F32_ACC) || !a.adam->p || !a.adam->m || !a.adam->v || !a.adam->pb ||
                  !a.adam->scalars || !a.adam->sq_slots))
     return cudaErrorInvalidValue;
-  if (a.epi == EPI_ROPE && (!a.rope_cos || !a.rope_sin || (a.head_dim != 64 && a.head_dim != 128) || a.seq <= 0 ||
+  if (a.epi == EPI_ROPE && (!a.rope_cos || !a.rope_sin || a.rope_ld < a.seq || (a.head_dim != 64 && a.head_dim != 128) || a.seq <= 0 ||
                             a.rope_cols % a.head_dim || a.N % a.head_dim))
     return cudaErrorInvalidValue;
   if (a.epi == EPI_SWIGLU && (!a.gu || a.d_ffn <= 0 || a.d_ffn % 16 || a.N != 2 * a.d_ffn)) return cudaErrorInvalidValue;

@@ -45,8 +45,11 @@ struct GemmArgs {
   int M = 0, N = 0, K = 0;
   float alpha = 1.0f;  // the accumulator is multiplied by alpha before the epilogue (not for EPI_ROPE / EPI_SWIGLU)
   // EPI_ROPE
-  const float* rope_cos = nullptr;  // fp32 [seq, head_dim/2]
+  // fp32 tables TRANSPOSED, [head_dim/2][rope_ld] (entry (i, position) at i * rope_ld + position): the 32 rows a warp
+  // holds are consecutive positions, so each load of one i is one 128-byte line
+  const float* rope_cos = nullptr;
   const float* rope_sin = nullptr;
+  int64_t rope_ld = 0;
   int seq = 1, head_dim = 64, rope_cols = 0;
   // EPI_ROPE with per-head QK-Norm (null qk_r: off): every rotated head is first RMS-normalised over its head_dim
   // accumulators and multiplied by a gain (heads below n_q_heads use gain_q, the others gain_k); r = (mean x^2 + eps)^(-1/2)

@@ -67,7 +67,8 @@ struct ft_model {
   size_t arena = 0, n_decay = 0;
   float *master, *adam_m, *adam_v, *grad;
   bf16* pbf;
-  float *rope_cos, *rope_sin;
+  float *rope_cos, *rope_sin;    // [max_seq][d/2]: attention backward, QK-Norm backward
+  float *rope_cosT, *rope_sinT;  // the same transposed, [d/2][max_seq]: the QKV GEMM's epilogue
   float rope_mscale = 1.0f;  // magnitude factor folded into both tables (LongRoPE form)
   StepScalars* sc;
   int32_t *tok_dev, *lab_dev;
@@ -211,6 +212,8 @@ size_t carve(ft_model* m, uint8_t* base) {
   m->adam_v = cv.take<float>(m->arena);
   m->grad = cv.take<float>(m->arena);
   m->pbf = cv.take<bf16>(m->arena);
+  m->rope_cosT = cv.take<float>((size_t)c.max_seq * (m->d / 2));
+  m->rope_sinT = cv.take<float>((size_t)c.max_seq * (m->d / 2));
   m->rope_cos = cv.take<float>((size_t)c.max_seq * (m->d / 2));
   m->rope_sin = cv.take<float>((size_t)c.max_seq * (m->d / 2));
   m->sc = cv.take<StepScalars>(1);
@@ -368,7 +371,8 @@ ft_status layer_forward(ft_model* m, int l, LayerActs& a, int B, int S) {
     GemmArgs g = gemm_base(m);
     g.A = a.h1; g.lda = h; g.B = m->wb(m->idx_layer(l, 1)); g.ldb = h; g.C = a.qkv; g.ldc = nqkv;
     g.M = T; g.N = nqkv; g.K = h; g.epi = EPI_ROPE;
-    g.rope_cos = m->rope_cos; g.rope_sin = m->rope_sin; g.seq = S; g.head_dim = m->d; g.rope_cols = hq + m->hkv;
+    g.rope_cos = m->rope_cosT; g.rope_sin = m->rope_sinT; g.rope_ld = m->cfg.max_seq; g.seq = S; g.head_dim = m->d;
+    g.rope_cols = hq + m->hkv;
     if (m->cfg.qk_norm) {
       g.qk_r = a.qk_r; g.qk_gain_q = m->wb(m->idx_layer(l, 6)); g.qk_gain_k = m->wb(m->idx_layer(l, 7));
       g.n_q_heads = m->cfg.n_heads; g.qk_eps = m->cfg.rms_eps;
@@ -687,8 +691,16 @@ static ft_status build_rope_tables(ft_model* m, const float* factors, float msca
       sn[(size_t)p * half + i] = (float)((double)mscale * sin(ang));
     }
   }
+  std::vector<float> csT(cs.size()), snT(sn.size());
+  for (int i = 0; i < half; ++i)
+    for (int p = 0; p < cfg->max_seq; ++p) {
+      csT[(size_t)i * cfg->max_seq + p] = cs[(size_t)p * half + i];
+      snT[(size_t)i * cfg->max_seq + p] = sn[(size_t)p * half + i];
+    }
   FT_CUDA(cudaMemcpyAsync(m->rope_cos, cs.data(), cs.size() * sizeof(float), cudaMemcpyHostToDevice, st));
   FT_CUDA(cudaMemcpyAsync(m->rope_sin, sn.data(), sn.size() * sizeof(float), cudaMemcpyHostToDevice, st));
+  FT_CUDA(cudaMemcpyAsync(m->rope_cosT, csT.data(), csT.size() * sizeof(float), cudaMemcpyHostToDevice, st));
+  FT_CUDA(cudaMemcpyAsync(m->rope_sinT, snT.data(), snT.size() * sizeof(float), cudaMemcpyHostToDevice, st));
   FT_CUDA(cudaStreamSynchronize(st));
   m->rope_mscale = mscale;
   return FT_OK;
