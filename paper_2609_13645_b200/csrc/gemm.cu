@@ -17,6 +17,7 @@ namespace fs {
 
 int g_pdl = 1;
 int g_gemm_balanced = 1;
+int g_gemm_epi8_kblocks = 16;
 int g_gemm_last_launches = 1;  // development knob: 0 = always the round-robin tile schedule
 
 namespace {
@@ -60,6 +61,7 @@ struct GemmDev {
   long long rope_ld;
   int panel;               // tile numbering (see tile_coords)
   float alpha;             // accumulator scale (1: off)
+  int wide_store;          // 1: C, ldc and N allow 32-byte stores (bf16 output)
   float* qk_r;             // per-head QK-Norm in the RoPE epilogue (null: off)
   const bf16* qk_gain_q;
   const bf16* qk_gain_k;
@@ -179,6 +181,29 @@ __device__ __forceinline__ bool flag_wait(const int* flag, int target, volatile 
     }
     __nanosleep(64);
   }
+}
+
+// 16 bf16 = 32 bytes in one store (256-bit stores exist from sm_100 on): one full 32-byte sector per request instead of
+// two half-sector requests
+__device__ __forceinline__ void store16_bf16(bf16* dst, const float* v) {
+  uint32_t w[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) w[i] = pack_bf16(v[2 * i], v[2 * i + 1]);
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+               "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+               : "memory");
+}
+
+__device__ __forceinline__ void store8_f32(float* dst, const uint32_t* w) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+               "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+               : "memory");
+}
+__device__ __forceinline__ void load8_b32(const void* src, uint32_t* w) {
+  asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+               : "l"(src)
+               : "memory");
 }
 
 __device__ __forceinline__ void store8_bf16(bf16* dst, const float* v) {
@@ -341,8 +366,13 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
             float v[32];
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+            if (p.wide_store) {
 #pragma unroll
-            for (int j = 0; j < 32; j += 8) store8_bf16(crow + g0 + c + j, v + j);
+              for (int j = 0; j < 32; j += 16) store16_bf16(crow + g0 + c + j, v + j);
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; j += 8) store8_bf16(crow + g0 + c + j, v + j);
+            }
           }
         }
       } else {
@@ -388,10 +418,18 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
               lo[j] = x1 * cc - x2 * ss;
               hi[j] = x2 * cc + x1 * ss;
             }
+            if (p.wide_store) {
 #pragma unroll
-            for (int j = 0; j < 32; j += 8) {
-              store8_bf16(crow + g0 + i0 + j, lo + j);
-              store8_bf16(crow + g0 + i0 + half + j, hi + j);
+              for (int j = 0; j < 32; j += 16) {
+                store16_bf16(crow + g0 + i0 + j, lo + j);
+                store16_bf16(crow + g0 + i0 + half + j, hi + j);
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; j += 8) {
+                store8_bf16(crow + g0 + i0 + j, lo + j);
+                store8_bf16(crow + g0 + i0 + half + j, hi + j);
+              }
             }
           }
         }
@@ -415,12 +453,18 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
           u[j] = round_bf16(__uint_as_float(r[16 + j]));
           a[j] = __fdividef(g[j], 1.0f + __expf(-g[j])) * u[j];
         }
-        store8_bf16(gurow + lc, g);
-        store8_bf16(gurow + lc + 8, g + 8);
-        store8_bf16(gurow + f + lc, u);
-        store8_bf16(gurow + f + lc + 8, u + 8);
-        store8_bf16(arow + lc, a);
-        store8_bf16(arow + lc + 8, a + 8);
+        if (p.wide_store) {
+          store16_bf16(gurow + lc, g);
+          store16_bf16(gurow + f + lc, u);
+          store16_bf16(arow + lc, a);
+        } else {
+          store8_bf16(gurow + lc, g);
+          store8_bf16(gurow + lc + 8, g + 8);
+          store8_bf16(gurow + f + lc, u);
+          store8_bf16(gurow + f + lc + 8, u + 8);
+          store8_bf16(arow + lc, a);
+          store8_bf16(arow + lc + 8, a + 8);
+        }
       }
     }
   } else if (p.epi == EPI_BF16_RESID) {
@@ -430,9 +474,24 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
     const bf16* rrow = p.resid + (long long)row * p.ldc;
     uint4 nxt[4];
     auto fetch = [&](int gc) {
+      if (p.wide_store) {  // two 32-byte loads
 #pragma unroll
-      for (int j = 0; j < 4; ++j)
-        nxt[j] = (row_ok && gc + 8 * j < p.N) ? *reinterpret_cast<const uint4*>(rrow + gc + 8 * j) : make_uint4(0, 0, 0, 0);
+        for (int j = 0; j < 4; j += 2) {
+          if (row_ok && gc + 8 * j < p.N) {
+            uint32_t w[8];
+            load8_b32(rrow + gc + 8 * j, w);
+            nxt[j] = make_uint4(w[0], w[1], w[2], w[3]);
+            nxt[j + 1] = make_uint4(w[4], w[5], w[6], w[7]);
+          } else {
+            nxt[j] = make_uint4(0, 0, 0, 0);
+            nxt[j + 1] = make_uint4(0, 0, 0, 0);
+          }
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          nxt[j] = (row_ok && gc + 8 * j < p.N) ? *reinterpret_cast<const uint4*>(rrow + gc + 8 * j) : make_uint4(0, 0, 0, 0);
+      }
     };
     fetch(n0 + cb);
     for (int c = cb; c < ce; c += 32) {
@@ -444,45 +503,68 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
       if (c + 32 < ce) fetch(gc + 32);
       ld_acc32(taddr, c, r, fx, p.alpha);
       if (row_ok) {
+        float v[32];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          if (gc + 8 * j < p.N) {
-            float v[8];
-            v[0] = __uint_as_float(r[8 * j + 0]) + bf16_lo(cur[j].x); v[1] = __uint_as_float(r[8 * j + 1]) + bf16_hi(cur[j].x);
-            v[2] = __uint_as_float(r[8 * j + 2]) + bf16_lo(cur[j].y); v[3] = __uint_as_float(r[8 * j + 3]) + bf16_hi(cur[j].y);
-            v[4] = __uint_as_float(r[8 * j + 4]) + bf16_lo(cur[j].z); v[5] = __uint_as_float(r[8 * j + 5]) + bf16_hi(cur[j].z);
-            v[6] = __uint_as_float(r[8 * j + 6]) + bf16_lo(cur[j].w); v[7] = __uint_as_float(r[8 * j + 7]) + bf16_hi(cur[j].w);
-            store8_bf16(crow + gc + 8 * j, v);
-          }
+          v[8 * j + 0] = __uint_as_float(r[8 * j + 0]) + bf16_lo(cur[j].x); v[8 * j + 1] = __uint_as_float(r[8 * j + 1]) + bf16_hi(cur[j].x);
+          v[8 * j + 2] = __uint_as_float(r[8 * j + 2]) + bf16_lo(cur[j].y); v[8 * j + 3] = __uint_as_float(r[8 * j + 3]) + bf16_hi(cur[j].y);
+          v[8 * j + 4] = __uint_as_float(r[8 * j + 4]) + bf16_lo(cur[j].z); v[8 * j + 5] = __uint_as_float(r[8 * j + 5]) + bf16_hi(cur[j].z);
+          v[8 * j + 6] = __uint_as_float(r[8 * j + 6]) + bf16_lo(cur[j].w); v[8 * j + 7] = __uint_as_float(r[8 * j + 7]) + bf16_hi(cur[j].w);
+        }
+        if (p.wide_store) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 16)
+            if (gc + j < p.N) store16_bf16(crow + gc + j, v + j);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; j += 8)
+            if (gc + j < p.N) store8_bf16(crow + gc + j, v + j);
         }
       }
     }
   } else if (p.epi == EPI_F32_ACC) {
     float* crow = reinterpret_cast<float*>(cptr) + (long long)row * p.ldc;
-    float4 nxt[8];
+    uint32_t nxt[32];
     auto fetch = [&](int gc) {
 #pragma unroll
-      for (int j = 0; j < 8; ++j)
-        nxt[j] = (row_ok && gc + 4 * j < p.N) ? *reinterpret_cast<const float4*>(crow + gc + 4 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int j = 0; j < 32; j += 8) {
+        if (row_ok && gc + j < p.N) {
+          if (p.wide_store) {
+            load8_b32(crow + gc + j, nxt + j);
+          } else {
+            const float4 a = *reinterpret_cast<const float4*>(crow + gc + j);
+            const float4 b4 = (gc + j + 4 < p.N) ? *reinterpret_cast<const float4*>(crow + gc + j + 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+            nxt[j] = __float_as_uint(a.x); nxt[j + 1] = __float_as_uint(a.y); nxt[j + 2] = __float_as_uint(a.z); nxt[j + 3] = __float_as_uint(a.w);
+            nxt[j + 4] = __float_as_uint(b4.x); nxt[j + 5] = __float_as_uint(b4.y); nxt[j + 6] = __float_as_uint(b4.z); nxt[j + 7] = __float_as_uint(b4.w);
+          }
+        } else {
+#pragma unroll
+          for (int e = 0; e < 8; ++e) nxt[j + e] = 0u;
+        }
+      }
     };
     fetch(n0 + cb);
     for (int c = cb; c < ce; c += 32) {
       const int gc = n0 + c;
       if (gc >= p.N) break;
-      float4 cur[8];
+      uint32_t cur[32];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) cur[j] = nxt[j];
+      for (int j = 0; j < 32; ++j) cur[j] = nxt[j];
       if (c + 32 < ce) fetch(gc + 32);
       ld_acc32(taddr, c, r, fx, p.alpha);
       if (row_ok) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          if (gc + 4 * j < p.N) {
-            float4 o = cur[j];
-            o.x += __uint_as_float(r[4 * j + 0]); o.y += __uint_as_float(r[4 * j + 1]);
-            o.z += __uint_as_float(r[4 * j + 2]); o.w += __uint_as_float(r[4 * j + 3]);
-            *reinterpret_cast<float4*>(crow + gc + 4 * j) = o;
-          }
+        for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(cur[j]) + __uint_as_float(r[j]));
+        if (p.wide_store) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 8)
+            if (gc + j < p.N) store8_f32(crow + gc + j, r + j);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; j += 4)
+            if (gc + j < p.N)
+              *reinterpret_cast<float4*>(crow + gc + j) = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
+                                                                      __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
         }
       }
     }
@@ -494,22 +576,40 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
       if (row_ok) {
         if (p.epi == EPI_BF16) {
           bf16* crow = reinterpret_cast<bf16*>(cptr) + (long long)row * p.ldc + gc;
+          if (p.wide_store) {
 #pragma unroll
-          for (int j = 0; j < 32; j += 8) {
-            if (gc + j < p.N) {
-              float v[8];
+            for (int j = 0; j < 32; j += 16) {
+              if (gc + j < p.N) {
+                float v[16];
 #pragma unroll
-              for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(r[j + e]);
-              store8_bf16(crow + j, v);
+                for (int e = 0; e < 16; ++e) v[e] = __uint_as_float(r[j + e]);
+                store16_bf16(crow + j, v);
+              }
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+              if (gc + j < p.N) {
+                float v[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(r[j + e]);
+                store8_bf16(crow + j, v);
+              }
             }
           }
         } else {
           float* crow = reinterpret_cast<float*>(cptr) + (long long)row * p.ldc + gc;
+          if (p.wide_store) {
 #pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            if (gc + j < p.N)
-              *reinterpret_cast<float4*>(crow + j) = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
-                                                                 __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+            for (int j = 0; j < 32; j += 8)
+              if (gc + j < p.N) store8_f32(crow + j, r + j);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+              if (gc + j < p.N)
+                *reinterpret_cast<float4*>(crow + j) = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
+                                                                   __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+            }
           }
         }
       }
@@ -1019,6 +1119,14 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
   p.seq = a.seq; p.head_dim = a.head_dim; p.rope_cols = a.rope_cols; p.d_ffn = a.d_ffn; p.rope_ld = a.rope_ld;
   set_adam(p, a);
   p.alpha = a.alpha;
+  {
+    const bool f32out = a.epi == EPI_F32 || a.epi == EPI_F32_ACC;
+    const int m = f32out ? 7 : 15;  // elements per 32 bytes, minus one
+    bool ok32 = (reinterpret_cast<uintptr_t>(a.C) & 31) == 0 && (a.ldc & m) == 0 && (a.N & m) == 0;
+    if (a.epi == EPI_BF16_RESID) ok32 = ok32 && (reinterpret_cast<uintptr_t>(a.resid) & 31) == 0;
+    if (a.epi == EPI_SWIGLU) ok32 = ok32 && (reinterpret_cast<uintptr_t>(a.gu) & 31) == 0;
+    p.wide_store = ok32 ? 1 : 0;
+  }
   p.qk_r = a.qk_r; p.qk_gain_q = a.qk_gain_q; p.qk_gain_k = a.qk_gain_k; p.n_q_heads = a.n_q_heads; p.qk_eps = a.qk_eps;
   p.panel = (size_t)a.M * a.K * sizeof(bf16) > (48u << 20) ? 1 : 0;
   p.ksplit = 1; p.split_stride = 0; p.balanced = 0; p.sw_first = 0; p.sw_parts = 1; p.sw_kpb = 0; p.flags = nullptr; p.slots = nullptr;
@@ -1047,6 +1155,14 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
   p.seq = a.seq; p.head_dim = a.head_dim; p.rope_cols = a.rope_cols; p.d_ffn = a.d_ffn; p.rope_ld = a.rope_ld;
   set_adam(p, a);
   p.alpha = a.alpha;
+  {
+    const bool f32out = a.epi == EPI_F32 || a.epi == EPI_F32_ACC;
+    const int m = f32out ? 7 : 15;  // elements per 32 bytes, minus one
+    bool ok32 = (reinterpret_cast<uintptr_t>(a.C) & 31) == 0 && (a.ldc & m) == 0 && (a.N & m) == 0;
+    if (a.epi == EPI_BF16_RESID) ok32 = ok32 && (reinterpret_cast<uintptr_t>(a.resid) & 31) == 0;
+    if (a.epi == EPI_SWIGLU) ok32 = ok32 && (reinterpret_cast<uintptr_t>(a.gu) & 31) == 0;
+    p.wide_store = ok32 ? 1 : 0;
+  }
   p.qk_r = a.qk_r; p.qk_gain_q = a.qk_gain_q; p.qk_gain_k = a.qk_gain_k; p.n_q_heads = a.n_q_heads; p.qk_eps = a.qk_eps;
   p.panel = (size_t)a.M * a.K * sizeof(bf16) > (48u << 20) ? 1 : 0;
   const int tiles = ((a.M + 255) / 256) * ((a.N + 255) / 256);
@@ -1098,7 +1214,9 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs, 1, 1);
-  cfg.blockDim = dim3(a.adam ? PAIR_THREADS : GEMM_THREADS, 1, 1);
+  // eight epilogue warps where the epilogue is the long pole: the fused update, and short contractions whose main loop
+  // per tile (K / 64 blocks of ~0.3 us) is shorter than the four-warp epilogue (~5 us)
+  cfg.blockDim = dim3((a.adam || kblocks <= g_gemm_epi8_kblocks) ? PAIR_THREADS : GEMM_THREADS, 1, 1);
   cfg.dynamicSmemBytes = C::SMEM_BYTES;
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
