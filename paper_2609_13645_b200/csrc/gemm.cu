@@ -17,7 +17,6 @@ namespace fs {
 
 int g_pdl = 1;
 int g_gemm_balanced = 1;
-int g_gemm_epi8_kblocks = 16;
 int g_gemm_last_launches = 1;  // development knob: 0 = always the round-robin tile schedule
 
 namespace {
@@ -1214,9 +1213,9 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs, 1, 1);
-  // eight epilogue warps where the epilogue is the long pole: the fused update, and short contractions whose main loop
-  // per tile (K / 64 blocks of ~0.3 us) is shorter than the four-warp epilogue (~5 us)
-  cfg.blockDim = dim3((a.adam || kblocks <= g_gemm_epi8_kblocks) ? PAIR_THREADS : GEMM_THREADS, 1, 1);
+  // eight epilogue warps only for the fused update (for short contractions, whose epilogue is the long pole too, they
+  // changed nothing: that epilogue is bound by L2 store requests, not by warps)
+  cfg.blockDim = dim3(a.adam ? PAIR_THREADS : GEMM_THREADS, 1, 1);
   cfg.dynamicSmemBytes = C::SMEM_BYTES;
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
