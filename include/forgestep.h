@@ -96,6 +96,12 @@ ft_status ft_set_rope_scaling(ft_model* m, const float* host_factors, float msca
  * On by default; switched off internally while profiling or with debug_taps.  Changing it drops a captured graph. */
 ft_status ft_set_overlap(ft_model* m, int32_t enable);
 
+/* Stored-dS attention backward (see ft_k_attention_bwd_ws): when max_seq is a multiple of 128 and
+ * 2 * max_batch * n_heads * max_seq^2 bytes is at most 24 GiB, the workspace holds one layer's dS^T and the step
+ * uses that path for sequences that are multiples of 128; other sequences, and models over the limit, use the
+ * recomputing dQ kernel.  On by default; 0 selects the recomputing kernel always.  Changing it drops a captured graph. */
+ft_status ft_set_attention_stored_ds(ft_model* m, int32_t enable);
+
 /* Whole-step CUDA graph (the paper's full-step graph capture): when enabled, the first ft_train_step of a (B, S)
  * runs launch by launch, the second is captured into a graph, later ones replay it (ids are first copied into the
  * model's own buffers).  Needs a capturable stream (not the legacy default stream; otherwise it switches itself
@@ -205,6 +211,18 @@ ft_status ft_k_attention_bwd(const void* dev_qkv, const void* dev_o, const void*
                              float* dev_delta, void* dev_dqkv, const float* dev_cos, const float* dev_sin,
                              int32_t B, int32_t S, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim,
                              void* stream);
+
+/* The same backward with a second scratch array, dev_ds: bf16 [B * n_h, S, S] (ds_bytes >= 2 B n_h S^2, 128-byte
+ * aligned, caller-owned device memory; contents on entry do not matter, unspecified afterwards).  The dK/dV kernel
+ * writes the rounded dS of Sec. 2.2's attention backward (dS = P o (dP - delta)) there, transposed, and dQ = dS K / sqrt(d)
+ * is then one causally truncated batched contraction over the stored tiles: five tile products per (query block, key
+ * block) pair instead of seven, the same dS bits feeding dK and dQ.  Needs S % 128 == 0; with dev_ds NULL, ds_bytes too
+ * small, a misaligned dev_ds or any other S the call is ft_k_attention_bwd.  Results are deterministic; they agree with
+ * ft_k_attention_bwd to rounding, not bit for bit. */
+ft_status ft_k_attention_bwd_ws(const void* dev_qkv, const void* dev_o, const void* dev_do, const float* dev_lse,
+                                float* dev_delta, void* dev_dqkv, const float* dev_cos, const float* dev_sin,
+                                void* dev_ds, uint64_t ds_bytes, int32_t B, int32_t S, int32_t n_heads,
+                                int32_t n_kv_heads, int32_t head_dim, void* stream);
 
 /* The same backward for callers that cannot hand over scratch memory they allocated: code running where device
  * allocation is off limits (inside a framework's allocator callback, in a plugin that is given only its input and

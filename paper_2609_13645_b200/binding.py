@@ -82,6 +82,8 @@ def lib():
         L.ft_set_rope_scaling.restype = C.c_int
         L.ft_set_overlap.argtypes = [vp, i32]
         L.ft_set_overlap.restype = C.c_int
+        L.ft_set_attention_stored_ds.argtypes = [vp, i32]
+        L.ft_set_attention_stored_ds.restype = C.c_int
         L.ft_set_graph.argtypes = [vp, i32]
         L.ft_set_graph.restype = C.c_int
         L.ft_graph_replays.argtypes = [vp]
@@ -93,6 +95,8 @@ def lib():
         L.ft_k_gemm_ws.restype = C.c_int
         L.ft_k_attention_fwd.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp]
         L.ft_k_attention_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]
+        L.ft_k_attention_bwd_ws.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_uint64, i32, i32, i32, i32, i32, vp]
+        L.ft_k_attention_bwd_ws.restype = C.c_int
         L.ft_k_attention_bwd_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]
         L.ft_k_attention_bwd_noalloc.restype = C.c_int
         for name in ("ft_init_model", "ft_train_step", "ft_train_step_host", "ft_forward_loss", "ft_forward_backward",
@@ -253,6 +257,10 @@ class Model:
         """Weight-gradient GEMMs on a second stream, concurrent with the rest of the backward pass (default on)."""
         self._check(lib().ft_set_overlap(self._h, 1 if enable else 0))
 
+    def set_attention_stored_ds(self, enable: bool):
+        """Attention backward that stores dS^T once and computes dQ as one batched contraction (default on)."""
+        self._check(lib().ft_set_attention_stored_ds(self._h, 1 if enable else 0))
+
     def set_graph(self, enable: bool):
         """Capture the whole step into a CUDA graph on its second run and replay it afterwards."""
         self._check(lib().ft_set_graph(self._h, 1 if enable else 0))
@@ -330,6 +338,19 @@ def k_attention_bwd(qkv, o, d_o, lse, delta, dqkv, B, S, n_heads, n_kv, d, cos=N
                                   _stream_ptr())
     if st != FT_OK:
         raise ForgeStepError(st, "ft_k_attention_bwd")
+
+
+def k_attention_bwd_ws(qkv, o, d_o, lse, delta, dqkv, ds, B, S, n_heads, n_kv, d, cos=None, sin=None):
+    """Attention backward with a dS^T scratch tensor `ds` (bf16, at least B * n_heads * S * S elements) or None."""
+    st = lib().ft_k_attention_bwd_ws(C.c_void_p(qkv.data_ptr()), C.c_void_p(o.data_ptr()), C.c_void_p(d_o.data_ptr()),
+                                     C.c_void_p(lse.data_ptr()), C.c_void_p(delta.data_ptr()),
+                                     C.c_void_p(dqkv.data_ptr()), C.c_void_p(cos.data_ptr()) if cos is not None else None,
+                                     C.c_void_p(sin.data_ptr()) if sin is not None else None,
+                                     C.c_void_p(ds.data_ptr()) if ds is not None else None,
+                                     ds.numel() * ds.element_size() if ds is not None else 0, B, S, n_heads, n_kv, d,
+                                     _stream_ptr())
+    if st != FT_OK:
+        raise ForgeStepError(st, "ft_k_attention_bwd_ws")
 
 
 def k_attention_bwd_noalloc(qkv, o, d_o, lse, dqkv, B, S, n_heads, n_kv, d, cos=None, sin=None):

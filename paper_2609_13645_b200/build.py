@@ -8,7 +8,7 @@ import sys
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libforgestep.so")
-SOURCES = ["gemm.cu", "attention.cu", "attention_tc.cu", "elementwise.cu", "model.cu"]
+SOURCES = ["gemm.cu", "attention.cu", "attention_tc.cu", "attention_dq.cu", "elementwise.cu", "model.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr",

@@ -17,6 +17,19 @@ cudaError_t attention_bwd(const bf16* qkv, const bf16* o, const bf16* d_o, const
                           const float* cos, const float* sin, int B, int S, int n_heads, int n_kv, int d, int* err,
                           cudaStream_t st);
 
+// The same with a scratch array for dS^T (bf16 [B n_h, S, S], attention_bwd_ds_bytes() bytes, 128-byte aligned): the
+// dK/dV kernel leaves its rounded dS tiles there and dQ becomes one causally truncated batched contraction over them
+// (delta pre-pass, dK/dV, dQ: three launches, five tile products per block pair instead of seven).  Needs S % 128 == 0;
+// with ds == nullptr, too small a scratch or another S this is attention_bwd().
+size_t attention_bwd_ds_bytes(int B, int S, int n_heads);
+cudaError_t attention_bwd_ws(const bf16* qkv, const bf16* o, const bf16* d_o, const float* lse, float* delta, bf16* dqkv,
+                             const float* cos, const float* sin, bf16* ds, size_t ds_bytes, int B, int S, int n_heads,
+                             int n_kv, int d, int* err, cudaStream_t st);
+
+// dQ from stored dS^T (the last launch of attention_bwd_ws).
+cudaError_t attention_dq_from_ds(const bf16* ds, const bf16* qkv, bf16* dqkv, const float* cos, const float* sin, int B, int S,
+                                 int n_heads, int n_kv, int d, int* err, cudaStream_t st);
+
 // delta[b, n, i] = sum_k dO[b,i,n,k] O[b,i,n,k] (the backward pre-pass; one launch)
 cudaError_t attention_delta(const bf16* o, const bf16* d_o, float* delta, int B, int S, int n_heads, int d, cudaStream_t st);
 

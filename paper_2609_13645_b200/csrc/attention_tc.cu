@@ -350,6 +350,12 @@ struct BwdCfg {
   static constexpr int ACC0 = 256, ACC1 = 256 + D;
 };
 
+__device__ __forceinline__ void store8_b32(void* dst, const uint32_t* w) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+               "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+               : "memory");
+}
+
 template <int W>
 __device__ __forceinline__ void tmem_load_cols(uint32_t taddr, float (&out)[W]) {
   static_assert(W == 32 || W == 16, "chunk width");
@@ -386,8 +392,8 @@ __global__ void __launch_bounds__(BWD_THREADS, 1)
 attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_constant__ CUtensorMap tm_qkv64,
                    const __grid_constant__ CUtensorMap tm_do128, const __grid_constant__ CUtensorMap tm_do64,
                    const float* __restrict__ lse, const float* __restrict__ delta, bf16* __restrict__ dqkv,
-                   const float* __restrict__ rope_cos, const float* __restrict__ rope_sin, int S, int n_heads, int n_kv,
-                   float scale, float scale_log2, int* err) {
+                   bf16* __restrict__ ds_out, const float* __restrict__ rope_cos, const float* __restrict__ rope_sin, int S,
+                   int n_heads, int n_kv, float scale, float scale_log2, int* err) {
   using C = BwdCfg<D, MODE>;
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sbase = smem_u32(smem);
@@ -655,6 +661,16 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(BB_TFULL + bf));
       if (threadIdx.x == 64 && it < 100) FS_TRACE(it * 16 + 9);
+      if constexpr (MODE == MODE_DKV) {
+        // after the arrival, off the MMA chain's critical path: the same rounded dS also goes to dS^T[b, head][key][query]
+        // for the dQ contraction that follows (S % 128 == 0 there)
+        if (ds_out != nullptr) {
+          const int n = kvh * n_rep + it / per_head;
+          bf16* dsp = ds_out + (((long long)b * n_heads + n) * S + row) * S + cmin;
+          store8_b32(dsp, wd);
+          store8_b32(dsp + 16, wd + 8);
+        }
+      }
     }
     if (ok) {
       ok = mbar_wait(bar(BB_ACCDONE), 0, abort_flag, err);
@@ -722,7 +738,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
 
 template <int D>
 cudaError_t attention_bwd_tc_t(const bf16* qkv, const bf16* o, const bf16* d_o, const float* lse, float* delta, bf16* dqkv,
-                               const float* cs, const float* sn, int B, int S, int nh, int nkv, int* err, cudaStream_t st) {
+                               const float* cs, const float* sn, bf16* ds, int B, int S, int nh, int nkv, int* err,
+                               cudaStream_t st) {
   using CQ = BwdCfg<D, MODE_DQ>;
   using CK = BwdCfg<D, MODE_DKV>;
   static bool once = false;
@@ -744,11 +761,19 @@ cudaError_t attention_bwd_tc_t(const bf16* qkv, const bf16* o, const bf16* d_o, 
   cudaError_t e = attention_delta(o, d_o, delta, B, S, nh, D, st);
   if (e != cudaSuccess) return e;
   dim3 gq((S + 127) / 128, nh, B), gk((S + 127) / 128, nkv, B);
+  bf16* none = nullptr;
+  if (ds != nullptr) {
+    // dK/dV first, leaving dS^T behind; dQ is then one causally truncated batched contraction over it
+    e = launch_pdl(attn_bwd_tc_kernel<D, MODE_DKV>, gk, BWD_THREADS, CK::SMEM_BYTES, st, tq128, tq64, td128, td64, lse, delta,
+                   dqkv, ds, cs, sn, S, nh, nkv, scale, scale_log2, err);
+    if (e != cudaSuccess) return e;
+    return attention_dq_from_ds(ds, qkv, dqkv, cs, sn, B, S, nh, nkv, D, err, st);
+  }
   e = launch_pdl(attn_bwd_tc_kernel<D, MODE_DQ>, gq, BWD_THREADS, CQ::SMEM_BYTES, st, tq128, tq64, td128, td64, lse, delta,
-                 dqkv, cs, sn, S, nh, nkv, scale, scale_log2, err);
+                 dqkv, none, cs, sn, S, nh, nkv, scale, scale_log2, err);
   if (e != cudaSuccess) return e;
   return launch_pdl(attn_bwd_tc_kernel<D, MODE_DKV>, gk, BWD_THREADS, CK::SMEM_BYTES, st, tq128, tq64, td128, td64, lse, delta,
-                    dqkv, cs, sn, S, nh, nkv, scale, scale_log2, err);
+                    dqkv, none, cs, sn, S, nh, nkv, scale, scale_log2, err);
 }
 
 static __device__ int g_attn_status;
@@ -775,14 +800,26 @@ cudaError_t attention_fwd(const bf16* qkv, bf16* o, float* lse, int B, int S, in
   return cudaErrorInvalidValue;
 }
 
-cudaError_t attention_bwd(const bf16* qkv, const bf16* o, const bf16* d_o, const float* lse, float* delta, bf16* dqkv,
-                             const float* cs, const float* sn, int B, int S, int nh, int nkv, int d, int* err,
-                             cudaStream_t st) {
+size_t attention_bwd_ds_bytes(int B, int S, int nh) {
+  if (B <= 0 || S <= 0 || nh <= 0 || S % 128 != 0) return 0;
+  return (size_t)B * nh * S * S * sizeof(bf16);
+}
+
+cudaError_t attention_bwd_ws(const bf16* qkv, const bf16* o, const bf16* d_o, const float* lse, float* delta, bf16* dqkv,
+                             const float* cs, const float* sn, bf16* ds, size_t ds_bytes, int B, int S, int nh, int nkv, int d,
+                             int* err, cudaStream_t st) {
   if (B <= 0 || S <= 0 || nh <= 0 || nkv <= 0 || nh % nkv || !err) return cudaErrorInvalidValue;
   if ((cs == nullptr) != (sn == nullptr)) return cudaErrorInvalidValue;
-  if (d == 64) return attention_bwd_tc_t<64>(qkv, o, d_o, lse, delta, dqkv, cs, sn, B, S, nh, nkv, err, st);
-  if (d == 128) return attention_bwd_tc_t<128>(qkv, o, d_o, lse, delta, dqkv, cs, sn, B, S, nh, nkv, err, st);
+  const size_t need = attention_bwd_ds_bytes(B, S, nh);
+  if (ds != nullptr && (need == 0 || ds_bytes < need || (reinterpret_cast<uintptr_t>(ds) & 127u) != 0)) ds = nullptr;
+  if (d == 64) return attention_bwd_tc_t<64>(qkv, o, d_o, lse, delta, dqkv, cs, sn, ds, B, S, nh, nkv, err, st);
+  if (d == 128) return attention_bwd_tc_t<128>(qkv, o, d_o, lse, delta, dqkv, cs, sn, ds, B, S, nh, nkv, err, st);
   return cudaErrorInvalidValue;
+}
+
+cudaError_t attention_bwd(const bf16* qkv, const bf16* o, const bf16* d_o, const float* lse, float* delta, bf16* dqkv,
+                          const float* cs, const float* sn, int B, int S, int nh, int nkv, int d, int* err, cudaStream_t st) {
+  return attention_bwd_ws(qkv, o, d_o, lse, delta, dqkv, cs, sn, nullptr, 0, B, S, nh, nkv, d, err, st);
 }
 
 #ifdef FS_ATTN_TRACE

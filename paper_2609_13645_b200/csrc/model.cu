@@ -19,6 +19,7 @@ using namespace fs;
 namespace {
 
 constexpr size_t kAlign = 256;
+constexpr size_t kAttnDsMaxBytes = 24ull << 30;  // largest dS^T scratch the workspace will carry
 constexpr size_t kSplitKFloats = 6u << 20;  // 24 MiB of split-K partial tiles (74 tiles of 256 x 256 fp32 at most)
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -95,6 +96,9 @@ struct ft_model {
   bool w_pending[4] = {false, false, false, false};
   bool overlapping = false;   // true while a backward pass that uses the second stream is being enqueued
   float* splitk2 = nullptr;   // GEMM scratch of the second stream
+  bf16* attn_ds = nullptr;    // dS^T scratch of the attention backward (one layer's worth), or null
+  size_t attn_ds_bytes = 0;
+  bool attn_ds_on = true;
 
   // AdamW inside the weight-gradient GEMM epilogues (clipping off): the train step then never stores those gradients
   bool fused_update = true;   // policy switch (ft_set_fused_update)
@@ -235,6 +239,10 @@ size_t carve(ft_model* m, uint8_t* base) {
   m->d_a = cv.take<bf16>(T * f); m->d_gu = cv.take<bf16>(T * 2 * f); m->d_o = cv.take<bf16>(T * hq);
   m->d_qkv = cv.take<bf16>(T * nqkv);
   m->delta = cv.take<float>(T * c.n_heads);
+  // dS^T of one layer's attention backward, when the longest sequence allows the stored-dS path and it stays modest
+  m->attn_ds_bytes = attention_bwd_ds_bytes(c.max_batch, c.max_seq, c.n_heads);
+  if (m->attn_ds_bytes > kAttnDsMaxBytes) m->attn_ds_bytes = 0;
+  m->attn_ds = m->attn_ds_bytes ? cv.take<bf16>(m->attn_ds_bytes / sizeof(bf16)) : nullptr;
   m->norm_partial = cv.take<float>((size_t)elementwise_blocks_for_norm((int)T) * h);
   m->sq_partial = cv.take<float>(kSqnormBlocks);
   m->fuse_sq = cv.take<float>(m->fuse_sq_count());
@@ -474,8 +482,9 @@ ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
   if (s) return s;
   if ((s = wait_wgrad(m, 3))) return s;  // the previous layer's qkv weight gradient still reads d_qkv
   prof_begin(m);
-  FT_CUDA(attention_bwd(a.qkv, a.o, m->d_o, a.lse, m->delta, m->d_qkv, m->rope_cos, m->rope_sin, B, S, m->cfg.n_heads,
-                        m->cfg.n_kv_heads, m->d, &m->sc->err, st));
+  FT_CUDA(attention_bwd_ws(a.qkv, a.o, m->d_o, a.lse, m->delta, m->d_qkv, m->rope_cos, m->rope_sin,
+                           m->attn_ds_on ? m->attn_ds : nullptr, m->attn_ds_bytes, B, S, m->cfg.n_heads, m->cfg.n_kv_heads,
+                           m->d, &m->sc->err, st));
   m->launches += 3;
   prof_end(m, FT_PROF_ATTN_BWD, 4.0 * B * m->cfg.n_heads * (double)S * S * m->d, 3);
   if (m->cfg.qk_norm) {
@@ -849,6 +858,13 @@ ft_status ft_set_overlap(ft_model* m, int32_t enable) {
   return FT_OK;
 }
 
+ft_status ft_set_attention_stored_ds(ft_model* m, int32_t enable) {
+  if (!m) return FT_EINVAL;
+  m->attn_ds_on = enable != 0;
+  if (m->graph_exec) { cudaGraphExecDestroy(m->graph_exec); m->graph_exec = nullptr; }  // captured with the old setting
+  return FT_OK;
+}
+
 ft_status ft_set_fused_update(ft_model* m, int32_t enable) {
   if (!m) return FT_EINVAL;
   m->fused_update = enable != 0;
@@ -1132,6 +1148,22 @@ ft_status ft_k_attention_bwd(const void* dev_qkv, const void* dev_o, const void*
                                 reinterpret_cast<const bf16*>(dev_do), dev_lse, dev_delta,
                                 reinterpret_cast<bf16*>(dev_dqkv), dev_cos, dev_sin, B, S, n_heads, n_kv_heads, head_dim,
                                 status, reinterpret_cast<cudaStream_t>(stream));
+  if (e == cudaErrorInvalidValue) return FT_EINVAL;
+  return e == cudaSuccess ? FT_OK : FT_ECUDA;
+}
+
+ft_status ft_k_attention_bwd_ws(const void* dev_qkv, const void* dev_o, const void* dev_do, const float* dev_lse,
+                                float* dev_delta, void* dev_dqkv, const float* dev_cos, const float* dev_sin, void* dev_ds,
+                                uint64_t ds_bytes, int32_t B, int32_t S, int32_t n_heads, int32_t n_kv_heads,
+                                int32_t head_dim, void* stream) {
+  if (!dev_qkv || !dev_o || !dev_do || !dev_lse || !dev_delta || !dev_dqkv) return FT_EINVAL;
+  int* status = attention_status_word();
+  if (!status) return FT_ECUDA;
+  cudaError_t e = attention_bwd_ws(reinterpret_cast<const bf16*>(dev_qkv), reinterpret_cast<const bf16*>(dev_o),
+                                   reinterpret_cast<const bf16*>(dev_do), dev_lse, dev_delta,
+                                   reinterpret_cast<bf16*>(dev_dqkv), dev_cos, dev_sin, reinterpret_cast<bf16*>(dev_ds),
+                                   (size_t)ds_bytes, B, S, n_heads, n_kv_heads, head_dim, status,
+                                   reinterpret_cast<cudaStream_t>(stream));
   if (e == cudaErrorInvalidValue) return FT_EINVAL;
   return e == cudaSuccess ? FT_OK : FT_ECUDA;
 }

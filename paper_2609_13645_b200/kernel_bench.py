@@ -46,7 +46,7 @@ def main():
     ap.add_argument("--no-flush", action="store_true")
     ap.add_argument("--out", default="auto", choices=["auto", "bf16", "resid", "f32", "f32acc"], help="GEMM epilogue")
     ap.add_argument("--bn", type=int, default=0, help="force the GEMM tile width (development)")
-    ap.add_argument("--ws", action="store_true", help="GEMM with a scratch buffer (split-K / balanced-K schedules)")
+    ap.add_argument("--ws", action="store_true", help="GEMM with a scratch buffer (split-K / balanced-K schedules); attn_bwd with the dS^T scratch")
     ap.add_argument("--pairs", type=int, default=1, help="0: single-CTA GEMM kernel only (development)")
     a = ap.parse_args()
     torch.manual_seed(0)
@@ -117,7 +117,10 @@ def main():
             dqkv = torch.empty_like(qkv)
             flops = 2.0 * fwd_flops  # model count of the backward (the paper's 1:2 ratio)
             run = lambda: B.k_attention_bwd(qkv, o, do, lse, delta, dqkv, Bsz, S, nh, nkv, d)
-        desc = dict(kernel=a.kernel, B=Bsz, S=S, n_heads=nh, n_kv=nkv, d=d)
+            if a.ws:
+                ds = torch.empty(Bsz * nh, S, S, dtype=torch.bfloat16, device=dev)
+                run = lambda: B.k_attention_bwd_ws(qkv, o, do, lse, delta, dqkv, ds, Bsz, S, nh, nkv, d)
+        desc = dict(kernel=a.kernel, B=Bsz, S=S, n_heads=nh, n_kv=nkv, d=d, ws=bool(a.ws))
 
     for _ in range(a.warmup):
         run()

@@ -26,13 +26,14 @@ def _small_gqa():
     return oracle_config(n_layers=2, d_model=512, n_heads=4, n_kv_heads=2, head_dim=128, d_ffn=720, vocab=2048)
 
 
-def _check_step(ocfg, tok, lab, params, debug=True, recompute=0, report=None):
+def _check_step(ocfg, tok, lab, params, debug=True, recompute=0, report=None, stored_ds=True):
     from paper_2609_13645_b200 import binding as B
     Bsz, S = tok.shape
     T = Bsz * S
     model = B.Model(lib_config(B, ocfg, Bsz, S, debug_taps=1 if debug else 0, recompute=recompute), seed=1)
     if ocfg.rope_factors is not None or ocfg.rope_mscale != 1.0:
         model.set_rope_scaling(ocfg.rope_factors, ocfg.rope_mscale)
+    model.set_attention_stored_ds(stored_ds)
     load_params(model, params)
     st = D.TrainState(ocfg, params)
     loss_o, gn_o, grads_o, taps_o = st.train_step(tok, lab, mode="contract", want_taps=True)
@@ -98,6 +99,16 @@ def test_gqa_head_dim_128_two_layers_with_ignored_labels():
     lab = lab.copy()
     lab[0, :7] = -1
     _check_step(ocfg, tok, lab, params)
+
+
+@pytest.mark.parametrize("stored_ds", [False, True])
+def test_both_attention_backward_paths_match_oracle_on_a_multi_tile_sequence(stored_ds):
+    """S = 384 is a multiple of 128, so the step may keep dS^T and compute dQ as one batched contraction; with the
+    switch off it recomputes S and dP in a dQ kernel.  Same parity bars either way."""
+    ocfg = _small_gqa()
+    params = D.init_params(ocfg, 99)
+    tok, lab = SI.batch(ocfg.vocab, 1, 384, "zipf", seed=6)
+    _check_step(ocfg, tok, lab, params, stored_ds=stored_ds)
 
 
 @pytest.mark.parametrize("variant", ["mup", "tied", "tied+mup", "qknorm", "qknorm128+tied+mup", "longrope+qknorm"])
