@@ -212,8 +212,9 @@ ft_status ft_k_attention_bwd(const void* dev_qkv, const void* dev_o, const void*
                              int32_t B, int32_t S, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim,
                              void* stream);
 
-/* The same backward with a second scratch array, dev_ds: bf16 [B * n_h, S, S] (ds_bytes >= 2 B n_h S^2, 128-byte
- * aligned, caller-owned device memory; contents on entry do not matter, unspecified afterwards).  The dK/dV kernel
+/* The same backward with a second scratch array, dev_ds: B * n_h * S * S bf16 in a chunked order private to the
+ * library (ds_bytes >= 2 B n_h S^2, 128-byte aligned, caller-owned device memory; contents on entry do not matter,
+ * unspecified afterwards).  The dK/dV kernel
  * writes the rounded dS of Sec. 2.2's attention backward (dS = P o (dP - delta)) there, transposed, and dQ = dS K / sqrt(d)
  * is then one causally truncated batched contraction over the stored tiles: five tile products per (query block, key
  * block) pair instead of seven, the same dS bits feeding dK and dQ.  Needs S % 128 == 0; with dev_ds NULL, ds_bytes too

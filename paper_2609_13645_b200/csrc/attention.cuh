@@ -17,7 +17,7 @@ cudaError_t attention_bwd(const bf16* qkv, const bf16* o, const bf16* d_o, const
                           const float* cos, const float* sin, int B, int S, int n_heads, int n_kv, int d, int* err,
                           cudaStream_t st);
 
-// The same with a scratch array for dS^T (bf16 [B n_h, S, S], attention_bwd_ds_bytes() bytes, 128-byte aligned): the
+// The same with a scratch array for dS^T (B n_h S^2 bf16 in 32-query chunks, attention_bwd_ds_bytes() bytes, 128-byte aligned): the
 // dK/dV kernel leaves its rounded dS tiles there and dQ becomes one causally truncated batched contraction over them
 // (delta pre-pass, dK/dV, dQ: three launches, five tile products per block pair instead of seven).  Needs S % 128 == 0;
 // with ds == nullptr, too small a scratch or another S this is attention_bwd().

@@ -1,9 +1,16 @@
 // dQ of the attention backward as one batched, causally truncated contraction over the stored dS^T tiles:
 //   dQ[b, h, i, :] = scale * sum_{j <= i} dS[b, h, i, j] K[b, kv(h), j, :]
-// The dK/dV kernel computes dS (bf16) anyway; when it also writes its tiles to a scratch array dS^T[b*n_h + h][j][i],
-// dQ needs neither S nor dP again: 5 tile products per (query block, key block) pair in the whole backward pass instead
-// of 7, and every dS value is rounded exactly once for both of its uses.  Each dQ element is the sum of one CTA's MMAs
-// in a fixed order, so the result is deterministic without atomics.
+// The dK/dV kernel computes dS (bf16) anyway; when it also writes its tiles to a scratch array, dQ needs neither S nor
+// dP again: 5 tile products per (query block, key block) pair in the whole backward pass instead of 7, and every dS
+// value is rounded exactly once for both of its uses.  Each dQ element is the sum of one CTA's MMAs in a fixed order,
+// so the result is deterministic without atomics.
+//
+// Scratch layout: element (z = b n_h + h, key j, query i) at ((z * S/32 + i / 32) * S + j) * 32 + i % 32, i.e. 32-query
+// chunks [z][i / 32][j][32].  A thread of the dK/dV kernel (one key, 32 queries) then stores one contiguous 64-byte
+// row, its warp a 2 KiB run, and a TMA box of 64 keys x 4 chunks lands in shared memory as the MN-major operand layout
+// of the 64-byte swizzle (4 blocks of [64 keys][64 bytes]).  Measured against the alternatives at B 4, S 2048, 16/8
+// heads of 128: row-major dS^T (128-byte swizzle) costs the dK/dV kernel 40 us of scattered 32-byte stores; 16-query
+// chunks (32-byte swizzle) give back those 40 us but slow this kernel's TMA loads by 15 us; this layout loses neither.
 //
 // Persistent, warp-specialised like the GEMM: warp 0 TMA producer, warp 1 MMA issuer, warps 2..5 epilogue (scale,
 // inverse rotation, one rounding to bf16).  A tile is 128 queries of one (batch, head); its K range ends at the diagonal.
@@ -23,7 +30,7 @@ constexpr int DQ_BK = 64;   // keys per pipeline stage
 
 template <int D>
 struct DqCfg {
-  static constexpr int A_BYTES = DQ_BK * DQ_BM * 2;  // two 64 x 64 boxes of dS^T
+  static constexpr int A_BYTES = DQ_BK * DQ_BM * 2;  // one box of dS^T: 4 chunks of [64 keys][32 queries]
   static constexpr int B_BYTES = DQ_BK * D * 2;      // D / 64 boxes of K
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STAGES = 3;
@@ -108,8 +115,7 @@ attn_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_ds, const __grid_cons
           mbar_expect_tx(fb, C::STAGE_BYTES);
           const uint32_t a_dst = sbase + stage * C::STAGE_BYTES;
           const uint32_t b_dst = a_dst + C::A_BYTES;
-#pragma unroll
-          for (int j = 0; j < DQ_BM / 64; ++j) tma_load_3d(a_dst + j * 8192, &tm_ds, fb, q0 + 64 * j, kb * DQ_BK, z);
+          tma_load_4d(a_dst, &tm_ds, fb, 0, kb * DQ_BK, q0 / 32, z);  // 4 chunks of [64 keys][32 queries]
 #pragma unroll
           for (int j = 0; j < D / 64; ++j) tma_load_3d(b_dst + j * 8192, &tm_qkv, fb, hq + kvh * D + 64 * j, kb * DQ_BK, b);
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
@@ -140,7 +146,7 @@ attn_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_ds, const __grid_cons
           const uint32_t b_addr = a_addr + C::A_BYTES;
 #pragma unroll
           for (int k = 0; k < DQ_BK / 16; ++k) {
-            const uint64_t adesc = umma_desc_sw128(a_addr + k * 2048, 8192, 1024);
+            const uint64_t adesc = umma_desc_sw64(a_addr + k * 1024, 4096, 512);
             const uint64_t bdesc = umma_desc_sw128(b_addr + k * 2048, 8192, 1024);
             umma_bf16(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
           }
@@ -243,7 +249,7 @@ cudaError_t launch_dq(const bf16* ds, const bf16* qkv, bf16* dqkv, const float* 
   }
   const int nqkv = (nh + 2 * nkv) * D;
   CUtensorMap tm_ds, tm_qkv;
-  if (!make_tmap_3d(&tm_ds, ds, S, S, (uint64_t)B * nh, S, 64) || !make_tmap_3d(&tm_qkv, qkv, nqkv, S, B, nqkv, 64))
+  if (!make_tmap_ds_chunked(&tm_ds, ds, S, (uint64_t)B * nh) || !make_tmap_3d(&tm_qkv, qkv, nqkv, S, B, nqkv, 64))
     return cudaErrorInvalidValue;
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);

@@ -662,11 +662,12 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
       if (lane == 0) mbar_arrive(bar(BB_TFULL + bf));
       if (threadIdx.x == 64 && it < 100) FS_TRACE(it * 16 + 9);
       if constexpr (MODE == MODE_DKV) {
-        // after the arrival, off the MMA chain's critical path: the same rounded dS also goes to dS^T[b, head][key][query]
-        // for the dQ contraction that follows (S % 128 == 0 there)
+        // after the arrival, off the MMA chain's critical path: the same rounded dS also goes to the dS^T scratch
+        // of the dQ contraction that follows (S % 128 == 0 there)
         if (ds_out != nullptr) {
           const int n = kvh * n_rep + it / per_head;
-          bf16* dsp = ds_out + (((long long)b * n_heads + n) * S + row) * S + cmin;
+          // 32-query chunks [b n_h + n][query / 32][key][query % 32]: one contiguous 64-byte row per thread
+          bf16* dsp = ds_out + ((((long long)b * n_heads + n) * (S >> 5) + (cmin >> 5)) * S + row) * 32;
           store8_b32(dsp, wd);
           store8_b32(dsp + 16, wd + 8);
         }

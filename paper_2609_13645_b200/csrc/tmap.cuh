@@ -57,4 +57,21 @@ inline bool make_tmap_3d(CUtensorMap* tm, const bf16* base, uint64_t cols, uint6
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 4-D map over the chunked dS^T scratch of the attention backward, bf16 [nz][S / 32][S][32]: element (z, key j, query i)
+// sits at ((z * S/32 + i / 32) * S + j) * 32 + i % 32, so that consecutive keys of one 32-query chunk are contiguous
+// 64-byte rows (what the lanes of a warp of the dK/dV kernel store).  A box is 64 keys of 4 chunks (128 queries) and
+// lands in shared memory as 4 blocks of [64 keys][32 queries], 64-byte rows with the 64-byte swizzle: the MN-major
+// operand layout of that swizzle mode.  Strides ascend with the dimension.
+inline bool make_tmap_ds_chunked(CUtensorMap* tm, const bf16* base, uint64_t S, uint64_t nz) {
+  EncodeTiledFn enc = get_encode_fn();
+  if (!enc || S % 128 != 0) return false;
+  cuuint64_t dims[4] = {32, S, S / 32, nz};
+  cuuint64_t strides[3] = {32 * sizeof(bf16), S * 32 * sizeof(bf16), S * S * sizeof(bf16)};
+  cuuint32_t box[4] = {32, 64, 4, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<bf16*>(base), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace fs
