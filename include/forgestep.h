@@ -113,6 +113,20 @@ int64_t ft_graph_replays(const ft_model* m);
 ft_status ft_train_step_host(ft_model* m, const int32_t* host_tokens, const int32_t* host_labels, int32_t B,
                              int32_t S, float* host_loss, float* host_gnorm);
 
+/* Pipelined form of ft_train_step_host for training loops that do not need a step's loss before enqueueing the next
+ * step (the paper's rule of keeping host synchronisation out of the hot loop, Section 5.2 / Appendix "optimization
+ * catalog": device-side norm and clipping, no .item() in the step).  ft_submit_step_host enqueues, on the model's
+ * stream, the copies of this step's ids, the whole step and a copy of its scalars into a pinned slot owned by the
+ * library, and returns without waiting; ft_collect_step waits for the OLDEST submitted step that has not been
+ * collected and returns its loss, gradient norm and status.  At most FT_MAX_IN_FLIGHT steps may be outstanding (one
+ * more submit returns FT_EINVAL and enqueues nothing); ft_collect_step with nothing outstanding returns FT_ENOTFOUND.
+ * host_tokens / host_labels must stay unchanged until that step has been collected; they should be pinned memory
+ * (pageable memory works but makes the copy, and so the call, wait for the stream).  Results are bit-identical to
+ * ft_train_step_host on the same inputs.  Do not interleave with other step calls while steps are outstanding. */
+#define FT_MAX_IN_FLIGHT 2
+ft_status ft_submit_step_host(ft_model* m, const int32_t* host_tokens, const int32_t* host_labels, int32_t B, int32_t S);
+ft_status ft_collect_step(ft_model* m, float* host_loss, float* host_gnorm);
+
 /* Forward and loss only; no gradients, no update. */
 ft_status ft_forward_loss(ft_model* m, const int32_t* dev_tokens, const int32_t* dev_labels, int32_t B, int32_t S,
                           float* host_loss);

@@ -18,6 +18,7 @@ _lib = None
 FT_OK, FT_EINVAL, FT_ENOMEM, FT_ECUDA, FT_ENONFINITE, FT_ETIMEOUT, FT_ENOTFOUND = range(7)
 STATUS_NAMES = ["FT_OK", "FT_EINVAL", "FT_ENOMEM", "FT_ECUDA", "FT_ENONFINITE", "FT_ETIMEOUT", "FT_ENOTFOUND"]
 KIND_MASTER, KIND_BF16, KIND_ADAM_M, KIND_ADAM_V, KIND_GRAD = range(5)
+MAX_IN_FLIGHT = 2  # FT_MAX_IN_FLIGHT of the header
 PROF_CLASSES = ["gemm", "attn_fwd", "attn_bwd", "norm", "elementwise", "ce", "optimizer"]
 
 
@@ -82,6 +83,10 @@ def lib():
         L.ft_set_rope_scaling.restype = C.c_int
         L.ft_set_overlap.argtypes = [vp, i32]
         L.ft_set_overlap.restype = C.c_int
+        L.ft_submit_step_host.argtypes = [vp, vp, vp, i32, i32]
+        L.ft_submit_step_host.restype = C.c_int
+        L.ft_collect_step.argtypes = [vp, vp, vp]
+        L.ft_collect_step.restype = C.c_int
         L.ft_set_attention_stored_ds.argtypes = [vp, i32]
         L.ft_set_attention_stored_ds.restype = C.c_int
         L.ft_set_graph.argtypes = [vp, i32]
@@ -142,6 +147,7 @@ class Model:
             raise ForgeStepError(FT_EINVAL, "invalid config")
         self.workspace = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
         self._h = C.c_void_p()
+        self._pending = []
         st = lib().ft_init_model(C.byref(cfg), C.c_uint64(seed), C.c_void_p(self.workspace.data_ptr()), nbytes,
                                  _stream_ptr(), C.byref(self._h))
         self._check(st)
@@ -183,6 +189,22 @@ class Model:
         loss, gn = C.c_float(), C.c_float()
         st = lib().ft_train_step_host(self._h, C.c_void_p(tokens.ctypes.data), C.c_void_p(labels.ctypes.data), B, S,
                                       C.byref(loss), C.byref(gn))
+        self._check(st)
+        return loss.value, gn.value
+
+    def submit_step_host(self, tokens: np.ndarray, labels: np.ndarray):
+        """Enqueue one train step on host int32 arrays [B, S] (ideally pinned) without waiting for it; at most
+        MAX_IN_FLIGHT steps may be outstanding.  The arrays must stay unchanged until the step is collected."""
+        B, S = tokens.shape
+        self._pending.append((tokens, labels))  # keep the buffers alive while the copy may still run
+        self._check(lib().ft_submit_step_host(self._h, C.c_void_p(tokens.ctypes.data), C.c_void_p(labels.ctypes.data), B, S))
+
+    def collect_step(self):
+        """Wait for the oldest submitted step; returns its (loss, gradient norm)."""
+        loss, gn = C.c_float(), C.c_float()
+        st = lib().ft_collect_step(self._h, C.byref(loss), C.byref(gn))
+        if self._pending:
+            self._pending.pop(0)
         self._check(st)
         return loss.value, gn.value
 

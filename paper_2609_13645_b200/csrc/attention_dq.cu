@@ -241,12 +241,9 @@ template <int D>
 cudaError_t launch_dq(const bf16* ds, const bf16* qkv, bf16* dqkv, const float* cs, const float* sn, int B, int S, int nh,
                       int nkv, int* err, cudaStream_t st) {
   using C = DqCfg<D>;
-  static bool once = false;
-  if (!once) {
-    cudaError_t e = cudaFuncSetAttribute(attn_dq_gemm_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    once = true;
-  }
+  static unsigned long long smem_set = 0;
+  cudaError_t e0 = ensure_dynamic_smem(attn_dq_gemm_kernel<D>, C::SMEM_BYTES, smem_set);
+  if (e0 != cudaSuccess) return e0;
   const int nqkv = (nh + 2 * nkv) * D;
   CUtensorMap tm_ds, tm_qkv;
   if (!make_tmap_ds_chunked(&tm_ds, ds, S, (uint64_t)B * nh) || !make_tmap_3d(&tm_qkv, qkv, nqkv, S, B, nqkv, 64))

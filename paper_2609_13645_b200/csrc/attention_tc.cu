@@ -302,12 +302,9 @@ template <int D>
 cudaError_t attention_fwd_tc_t(const bf16* qkv, bf16* o, float* lse, int B, int S, int nh, int nkv, int* err,
                                cudaStream_t st) {
   using C = FwdCfg<D>;
-  static bool once = false;
-  if (!once) {
-    cudaError_t e = cudaFuncSetAttribute(attn_fwd_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    once = true;
-  }
+  static unsigned long long smem_set = 0;
+  cudaError_t e0 = ensure_dynamic_smem(attn_fwd_tc_kernel<D>, C::SMEM_BYTES, smem_set);
+  if (e0 != cudaSuccess) return e0;
   const int nqkv = (nh + 2 * nkv) * D;
   CUtensorMap tmQ, tmKV;
   if (!make_tmap_3d(&tmQ, qkv, nqkv, S, B, nqkv, C::BQ) || !make_tmap_3d(&tmKV, qkv, nqkv, S, B, nqkv, C::BK))
@@ -743,15 +740,11 @@ cudaError_t attention_bwd_tc_t(const bf16* qkv, const bf16* o, const bf16* d_o, 
                                cudaStream_t st) {
   using CQ = BwdCfg<D, MODE_DQ>;
   using CK = BwdCfg<D, MODE_DKV>;
-  static bool once = false;
-  if (!once) {
-    cudaError_t e = cudaFuncSetAttribute(attn_bwd_tc_kernel<D, MODE_DQ>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         CQ::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_bwd_tc_kernel<D, MODE_DKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, CK::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    once = true;
-  }
+  static unsigned long long smem_set_q = 0, smem_set_k = 0;
+  cudaError_t e0 = ensure_dynamic_smem(attn_bwd_tc_kernel<D, MODE_DQ>, CQ::SMEM_BYTES, smem_set_q);
+  if (e0 != cudaSuccess) return e0;
+  e0 = ensure_dynamic_smem(attn_bwd_tc_kernel<D, MODE_DKV>, CK::SMEM_BYTES, smem_set_k);
+  if (e0 != cudaSuccess) return e0;
   const int hq = nh * D, nqkv = (nh + 2 * nkv) * D;
   CUtensorMap tq128, tq64, td128, td64;
   if (!make_tmap_3d(&tq128, qkv, nqkv, S, B, nqkv, 128) || !make_tmap_3d(&tq64, qkv, nqkv, S, B, nqkv, 64) ||

@@ -287,6 +287,20 @@ inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, siz
 }
 
 // ---------------------------------------------------------------- small reductions
+// cudaFuncSetAttribute acts on the current device only, so the "already done" memory of a launcher is a bit per device
+// (one static mask per kernel instantiation at the call site).  Devices past 63 set the attribute every time.
+template <typename Kern>
+inline cudaError_t ensure_dynamic_smem(Kern kern, int bytes, unsigned long long& done_mask) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const bool tracked = dev >= 0 && dev < 64;
+  if (tracked && ((done_mask >> dev) & 1ull)) return cudaSuccess;
+  e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess && tracked) done_mask |= 1ull << dev;
+  return e;
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

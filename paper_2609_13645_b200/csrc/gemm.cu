@@ -1088,26 +1088,23 @@ void set_adam(GemmDev& p, const GemmArgs& a) {
 }
 
 int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    if (n <= 0) n = 148;
-  }
+  static int cache[64] = {0};
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  if (dev >= 0 && dev < 64 && cache[dev] > 0) return cache[dev];
+  cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+  if (n <= 0) n = 148;
+  if (dev >= 0 && dev < 64) cache[dev] = n;
   return n;
 }
 
 template <int BN, bool A_MN, bool B_MN>
 cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
   using C = Cfg<BN>;
-  static bool attr_set = false;
   auto kern = gemm_tc_kernel<BN, A_MN, B_MN>;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static unsigned long long smem_set = 0;
+  cudaError_t e0 = ensure_dynamic_smem(kern, C::SMEM_BYTES, smem_set);
+  if (e0 != cudaSuccess) return e0;
   CUtensorMap tmA, tmB;
   bool ok = A_MN ? make_tmap_2d(&tmA, a.A, a.M, a.K, a.lda, 64) : make_tmap_2d(&tmA, a.A, a.K, a.M, a.lda, BM);
   ok = ok && (B_MN ? make_tmap_2d(&tmB, a.B, a.N, a.K, a.ldb, 64) : make_tmap_2d(&tmB, a.B, a.K, a.N, a.ldb, BN));
@@ -1137,13 +1134,10 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
 template <bool A_MN, bool B_MN>
 cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
   using C = PairCfg;
-  static bool attr_set = false;
   auto kern = gemm_tc_pair_kernel<A_MN, B_MN>;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static unsigned long long smem_set = 0;
+  cudaError_t e0 = ensure_dynamic_smem(kern, C::SMEM_BYTES, smem_set);
+  if (e0 != cudaSuccess) return e0;
   CUtensorMap tmA, tmB;
   bool ok = A_MN ? make_tmap_2d(&tmA, a.A, a.M, a.K, a.lda, 64) : make_tmap_2d(&tmA, a.A, a.K, a.M, a.lda, BM);
   ok = ok && (B_MN ? make_tmap_2d(&tmB, a.B, a.N, a.K, a.ldb, 64) : make_tmap_2d(&tmB, a.B, a.K, a.N, a.ldb, C::HALF_B));

@@ -96,6 +96,10 @@ struct ft_model {
   bool w_pending[4] = {false, false, false, false};
   bool overlapping = false;   // true while a backward pass that uses the second stream is being enqueued
   float* splitk2 = nullptr;   // GEMM scratch of the second stream
+  // pipelined host entry: pinned result slots and one event per slot, oldest-first
+  StepScalars* ring = nullptr;
+  cudaEvent_t ring_ev[FT_MAX_IN_FLIGHT] = {};
+  unsigned ring_head = 0, ring_tail = 0;  // submitted, collected (monotonic counters)
   bf16* attn_ds = nullptr;    // dS^T scratch of the attention backward (one layer's worth), or null
   size_t attn_ds_bytes = 0;
   bool attn_ds_on = true;
@@ -894,6 +898,43 @@ ft_status ft_train_step_host(ft_model* m, const int32_t* host_tokens, const int3
   return s;
 }
 
+ft_status ft_submit_step_host(ft_model* m, const int32_t* host_tokens, const int32_t* host_labels, int32_t B, int32_t S) {
+  if (!m || !host_tokens || !host_labels) return fail(m, FT_EINVAL, "null argument");
+  if (B < 1 || S < 1 || B > m->cfg.max_batch || S > m->cfg.max_seq) return fail(m, FT_EINVAL, "B or S out of range");
+  if (m->ring_head - m->ring_tail >= FT_MAX_IN_FLIGHT) return fail(m, FT_EINVAL, "too many steps in flight: collect one first");
+  if (!m->ring) {
+    FT_CUDA(cudaHostAlloc(reinterpret_cast<void**>(&m->ring), FT_MAX_IN_FLIGHT * sizeof(StepScalars), cudaHostAllocDefault));
+    for (auto& e : m->ring_ev) FT_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  }
+  const size_t bytes = (size_t)B * S * sizeof(int32_t);
+  FT_CUDA(cudaMemcpyAsync(m->tok_dev, host_tokens, bytes, cudaMemcpyHostToDevice, m->stream));
+  FT_CUDA(cudaMemcpyAsync(m->lab_dev, host_labels, bytes, cudaMemcpyHostToDevice, m->stream));
+  ft_status s = step_maybe_graphed(m, m->tok_dev, m->lab_dev, B, S);
+  if (s) return s;
+  const unsigned slot = m->ring_head % FT_MAX_IN_FLIGHT;
+  FT_CUDA(cudaMemcpyAsync(&m->ring[slot], m->sc, sizeof(StepScalars), cudaMemcpyDeviceToHost, m->stream));
+  FT_CUDA(cudaEventRecord(m->ring_ev[slot], m->stream));
+  ++m->ring_head;
+  return FT_OK;
+}
+
+ft_status ft_collect_step(ft_model* m, float* host_loss, float* host_gnorm) {
+  if (!m) return FT_EINVAL;
+  if (m->ring_head == m->ring_tail) return fail(m, FT_ENOTFOUND, "no step in flight");
+  const unsigned slot = m->ring_tail % FT_MAX_IN_FLIGHT;
+  FT_CUDA(cudaEventSynchronize(m->ring_ev[slot]));
+  ++m->ring_tail;
+  const StepScalars hs = m->ring[slot];
+  if (host_loss) *host_loss = hs.loss;
+  if (host_gnorm) *host_gnorm = hs.gnorm;
+  if (hs.err != 0) {
+    FT_CUDA(cudaMemsetAsync(&m->sc->err, 0, sizeof(int), m->stream));
+    return fail(m, FT_ETIMEOUT, "a device-side wait ran out of time");
+  }
+  if (hs.nonfinite) return fail(m, FT_ENONFINITE, "loss is not finite");
+  return FT_OK;
+}
+
 ft_status ft_forward_loss(ft_model* m, const int32_t* dev_tokens, const int32_t* dev_labels, int32_t B, int32_t S,
                           float* host_loss) {
   if (!m) return FT_EINVAL;
@@ -1094,6 +1135,8 @@ void ft_destroy(ft_model* m) {
   if (m->side) cudaStreamDestroy(m->side);
   if (m->ev_d) cudaEventDestroy(m->ev_d);
   for (auto e : m->ev_w) if (e) cudaEventDestroy(e);
+  for (auto e : m->ring_ev) if (e) cudaEventDestroy(e);
+  if (m->ring) cudaFreeHost(m->ring);
   delete m;
 }
 

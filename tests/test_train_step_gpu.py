@@ -256,6 +256,58 @@ def test_host_buffer_entry_point_equals_device_entry_point():
     b.close()
 
 
+def test_pipelined_host_steps_equal_the_synchronous_host_steps_bit_for_bit():
+    """submit_step_host / collect_step keep one step in flight; losses, norms and the final state are those of
+    train_step_host, and the in-flight limit and the empty collect are reported, not silently accepted."""
+    from paper_2609_13645_b200 import binding as B
+    ocfg, w = _c1()
+    Bsz, S = w["batch"], w["seq"]
+    batches = [SI.batch(ocfg.vocab, Bsz, S, "zipf", step=i) for i in range(5)]
+    pinned = [(torch.from_numpy(t).pin_memory(), torch.from_numpy(l).pin_memory()) for t, l in batches]
+
+    def run(pipelined):
+        model = B.Model(lib_config(B, ocfg, Bsz, S), seed=3)
+        out = []
+        if not pipelined:
+            for t, l in pinned:
+                out.append(model.train_step_host(t.numpy(), l.numpy()))
+        else:
+            with pytest.raises(B.ForgeStepError) as ei:
+                model.collect_step()
+            assert ei.value.status == B.FT_ENOTFOUND
+            for i, (t, l) in enumerate(pinned):
+                model.submit_step_host(t.numpy(), l.numpy())
+                if i > 0:
+                    out.append(model.collect_step())
+            out.append(model.collect_step())
+            # the limit: two submits are accepted, the third is refused and enqueues nothing
+            model.submit_step_host(pinned[0][0].numpy(), pinned[0][1].numpy())
+            model.submit_step_host(pinned[1][0].numpy(), pinned[1][1].numpy())
+            with pytest.raises(B.ForgeStepError) as ei:
+                model.submit_step_host(pinned[2][0].numpy(), pinned[2][1].numpy())
+            assert ei.value.status == B.FT_EINVAL
+            model._pending.pop()
+            extra = [model.collect_step(), model.collect_step()]
+            assert all(np.isfinite(x[0]) for x in extra) and model.step == 7
+            model.close()
+            return out, None
+        state = {n: model.get_param(n, B.KIND_MASTER) for n, _ in model.params}
+        model.close()
+        return out, state
+
+    sync_out, sync_state = run(False)
+    pipe_out, _ = run(True)
+    assert sync_out == pipe_out
+    # and the state after the same five pipelined steps
+    model = B.Model(lib_config(B, ocfg, Bsz, S), seed=3)
+    for t, l in pinned:
+        model.submit_step_host(t.numpy(), l.numpy())
+        model.collect_step()
+    for n, _ in model.params:
+        assert np.array_equal(model.get_param(n, B.KIND_MASTER), sync_state[n])
+    model.close()
+
+
 def test_error_paths_return_codes_and_keep_the_context_usable():
     from paper_2609_13645_b200 import binding as B
     ocfg, _ = _c1()
