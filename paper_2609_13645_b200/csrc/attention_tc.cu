@@ -18,6 +18,7 @@ namespace fs {
 namespace {
 
 constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kRefSlack = 8.0f;
 
 #ifdef FS_ATTN_TRACE
 __device__ long long g_trace[8192];
@@ -207,8 +208,12 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       float mx = -INFINITY;
 #pragma unroll
       for (int i = 0; i < 32; ++i) mx = fmaxf(mx, fmaxf(__uint_as_float(r0[i]), __uint_as_float(r1[i])));
-      // scale_log2 > 0, so the maximum commutes with the scaling
-      const float mnew = fmaxf(mref, ceilf(mx * scale_log2));
+      // scale_log2 > 0, so the maximum commutes with the scaling.  The reference only moves once the block maximum
+      // has passed it by more than 2^kRefSlack (P stays below that, far from overflow): with 32 rows per warp some
+      // row's maximum crosses an integer in almost every block, and each move costs the whole warp a wait for the
+      // previous P V product and a pass over O.  Powers of two commute with the roundings, so nothing else changes.
+      const float mcand = ceilf(mx * scale_log2);
+      const float mnew = mcand > mref + kRefSlack ? mcand : mref;
       const float alpha = fast_exp2(mref - mnew);  // exact power of two; 0 on the first block
       float psum = 0.f;
       uint32_t pw[32];  // bf16 pairs: keys 2c, 2c+1 in word c
