@@ -353,6 +353,58 @@ def run_cuda(args):
     return 0
 
 
+def run_dp(args):
+    """Opt-in (--dp): the same workload as ONE data-parallel job over all ranks (paper_2609_13645_b200/dp.py): bucketed
+    reduce-scatter behind the backward pass, sharded AdamW, per-bucket all-gather.  The default arm stays replicas.
+    Every step reads its loss (the driver's collect), so this is an end-to-end style number."""
+    import torch
+    import torch.distributed as dist
+    from paper_2609_13645_b200 import binding as B
+    from paper_2609_13645_b200.dp import DataParallel, LibraryBackend
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    else:
+        dist.init_process_group("nccl", init_method="tcp://127.0.0.1:29771", rank=0, world_size=1)
+    w = SI.WORKLOADS[args.workload]
+    Bsz, S = w["batch"], w["seq"]
+    cfg = B.make_config(w["n_layers"], w["d_model"], w["n_heads"], w["n_kv_heads"], w["head_dim"], w["d_ffn"],
+                        w["vocab"], Bsz, S, recompute=w["recompute"], **variant_kwargs(args, w))
+    side = torch.cuda.Stream()
+    torch.cuda.set_stream(side)
+    model = B.Model(cfg, seed=SI.WEIGHT_SEED)
+    dp = DataParallel(LibraryBackend(model))
+    n_batches = args.steps + args.warmup
+    batches = [SI.batch(w["vocab"], Bsz, S, w["dist"], seed=SI.DATA_SEED + 1000 * rank, step=i) for i in range(n_batches)]
+    batches = [(torch.from_numpy(t).cuda(), torch.from_numpy(l).cuda()) for t, l in batches]
+    for i in range(args.warmup):
+        dp.step(*batches[i])
+    dist.barrier(); torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    loss = None
+    for i in range(args.steps):
+        loss, gnorm = dp.step(*batches[args.warmup + i])
+    ev1.record()
+    dist.barrier(); torch.cuda.synchronize()
+    ms = max_over_ranks([ev0.elapsed_time(ev1)], world, device="cuda")[0]
+    if rank == 0:
+        print(json.dumps({
+            "metric": "train_tokens_per_sec", "value": job_tokens_per_s(Bsz * S, world, ms, args.steps), "unit": "tokens/s",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": args.workload, "batch_per_gpu": Bsz, "seq_len": S, "global_batch": Bsz * world,
+                       "parallelism": f"dp{world}: reduce-scatter per gradient bucket behind the backward pass, sharded AdamW, "
+                                      "all-gather of the bf16 copy per bucket", "buckets": len(dp.buckets)},
+            "last_loss": loss, "mode": "dp"}))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -361,6 +413,7 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="c3_1b", choices=sorted(SI.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--dp", action="store_true", help="one data-parallel job over the ranks instead of independent replicas")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel separately in the timed region")
     ap.add_argument("--variant", default="plain", choices=["plain", "mup_tied", "qknorm_tied"],
                     help="model variant on the workload's shape (default: the plain decoder the metric is quoted on)")
@@ -369,6 +422,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.dp:
+        return run_dp(args)
     return run_cuda(args)
 
 

@@ -113,6 +113,49 @@ int64_t ft_graph_replays(const ft_model* m);
 ft_status ft_train_step_host(ft_model* m, const int32_t* host_tokens, const int32_t* host_labels, int32_t B,
                              int32_t S, float* host_loss, float* host_gnorm);
 
+/* ---- Data-parallel hooks (Section 5.2, "bucketed reduce-scatter overlapped with backward", "ZeRO-1 sharded optimizer,
+ * per-bucket all-gather interleaved with Adam").  The library itself holds no communicator: these calls expose what a
+ * data-parallel driver needs, and paper_2609_13645_b200/dp.py drives them with torch.distributed (NCCL).
+ *
+ * The flat fp32 gradient arena (and the identically laid out master / moment / bf16 arenas, ft_arena_ptr) is cut into
+ * buckets in the order in which the backward pass completes them: the untied LM head first, then the layers from the
+ * last to the first (each layer's four matrices, contiguous), then the embedding table, then all gains.  Every bucket
+ * starts on a multiple of 128 elements and has a multiple of 128 elements, so it divides evenly over 2, 4, ... 128
+ * ranks.
+ *   ft_dp_num_buckets / ft_dp_bucket   number of buckets; arena offset and element count of bucket i.
+ *   ft_arena_ptr                       device address and element count of an arena (FT_GRAD_F32, FT_COMPUTE_BF16, ...).
+ *   ft_dp_set_label_count              number of labels >= 0 over ALL ranks' batches of the next step: the loss mean and
+ *                                      the logit gradients divide by it, so that the SUM of the ranks' gradients is the
+ *                                      gradient of the global mean loss (0: this batch's own count, the default).
+ *   ft_dp_backward                     enqueues forward + backward of this rank's batch on the model's stream (gradients
+ *                                      materialised, weight gradients in stream order), recording one event per bucket;
+ *                                      returns without waiting.
+ *   ft_dp_stream_wait_bucket           makes `stream` wait (device side) for bucket i of the last ft_dp_backward.
+ *   ft_dp_sqnorm                       *dev_out = sum of squares of the gradient range, fixed summation order, on `stream`.
+ *   ft_dp_begin_update                 advances the step counter and bias corrections; with dev_sq_total (the sum of
+ *                                      squares over all ranks' shards) it also sets the norm and the clip coefficient,
+ *                                      with NULL the coefficient is 1 (only valid when clipping is off).  Once per step,
+ *                                      on `stream`, before the first ft_dp_update_range.
+ *   ft_dp_update_range                 AdamW (master, moments, bf16 copy) on arena range [offset, offset + count) from
+ *                                      the gradient values found there (the reduced shard), on `stream`.
+ *   ft_dp_set_norm                     records the norm for reporting when clipping is off (after the update).
+ *   ft_dp_collect                      waits for the model's stream; returns this rank's loss share (sum of its label
+ *                                      losses / total label count) and the recorded norm, and any device-side status.
+ *   ft_dp_scratch                      4 floats of device memory for the driver's scalar reductions.
+ * offset and count are multiples of 4.  `stream` may be the model's stream or another one; the driver orders it. */
+int32_t ft_dp_num_buckets(ft_model* m);
+ft_status ft_dp_bucket(ft_model* m, int32_t i, int64_t* offset, int64_t* count);
+ft_status ft_arena_ptr(ft_model* m, ft_kind kind, void** dev_ptr, int64_t* numel);
+ft_status ft_dp_scratch(ft_model* m, float** dev_ptr);
+ft_status ft_dp_set_label_count(ft_model* m, int64_t total_count);
+ft_status ft_dp_backward(ft_model* m, const int32_t* dev_tokens, const int32_t* dev_labels, int32_t B, int32_t S);
+ft_status ft_dp_stream_wait_bucket(ft_model* m, int32_t i, void* stream);
+ft_status ft_dp_sqnorm(ft_model* m, int64_t offset, int64_t count, float* dev_out, void* stream);
+ft_status ft_dp_begin_update(ft_model* m, const float* dev_sq_total, void* stream);
+ft_status ft_dp_update_range(ft_model* m, int64_t offset, int64_t count, void* stream);
+ft_status ft_dp_set_norm(ft_model* m, const float* dev_sq_total, void* stream);
+ft_status ft_dp_collect(ft_model* m, float* host_loss, float* host_gnorm);
+
 /* Pipelined form of ft_train_step_host for training loops that do not need a step's loss before enqueueing the next
  * step (the paper's rule of keeping host synchronisation out of the hot loop, Section 5.2 / Appendix "optimization
  * catalog": device-side norm and clipping, no .item() in the step).  ft_submit_step_host enqueues, on the model's

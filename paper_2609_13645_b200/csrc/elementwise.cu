@@ -237,7 +237,7 @@ __global__ void swiglu_bwd_kernel(const bf16* __restrict__ d_a, const bf16* __re
 }
 
 // ---------------------------------------------------------------- loss
-__global__ void count_labels_kernel(const int32_t* __restrict__ labels, int T, StepScalars* sc) {
+__global__ void count_labels_kernel(const int32_t* __restrict__ labels, int T, StepScalars* sc, long long denom_override) {
   __shared__ int s[32];
   int c = 0;
   for (int i = threadIdx.x; i < T; i += blockDim.x) c += labels[i] >= 0 ? 1 : 0;
@@ -249,7 +249,9 @@ __global__ void count_labels_kernel(const int32_t* __restrict__ labels, int T, S
     int tot = 0;
     for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += s[w];
     sc->count = tot;
-    sc->inv_count = 1.0f / (float)(tot > 0 ? tot : 1);
+    // data parallelism: the mean runs over the labels of all ranks, whose number the caller provides
+    const long long denom = denom_override > 0 ? denom_override : (long long)(tot > 0 ? tot : 1);
+    sc->inv_count = 1.0f / (float)denom;
   }
 }
 
@@ -497,6 +499,27 @@ __global__ void sqnorm_final_kernel(const float* __restrict__ partial, int nblk,
     sc->gnorm = gn;
     sc->clip = hp.max_grad_norm > 0.f ? fminf(1.0f, hp.max_grad_norm / (gn + 1e-6f)) : 1.0f;
   }
+}
+
+// sum of the block partials in index order -> *out (one block)
+__global__ void sqnorm_sum_kernel(const float* __restrict__ partial, int nblk, float* __restrict__ out) {
+  __shared__ float s[256];
+  float a = 0.f;
+  for (int i = threadIdx.x; i < nblk; i += 256) a += partial[i];
+  s[threadIdx.x] = a;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if ((int)threadIdx.x < o) s[threadIdx.x] += s[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *out = s[0];
+}
+
+// norm and clip coefficient from a sum of squares that was formed elsewhere (over all ranks' shards)
+__global__ void clip_from_sq_kernel(const float* __restrict__ sq_total, StepScalars* sc, AdamHyper hp) {
+  const float gn = sqrtf(fmaxf(*sq_total, 0.f));
+  sc->gnorm = gn;
+  sc->clip = hp.max_grad_norm > 0.f ? fminf(1.0f, hp.max_grad_norm / (gn + 1e-6f)) : 1.0f;
 }
 
 __global__ void advance_step_kernel(StepScalars* sc, AdamHyper hp) {
@@ -773,8 +796,8 @@ int swiglu_bwd(const bf16* d_a, const bf16* gu, bf16* d_gu, int T, int f, cudaSt
   return ok(1);
 }
 
-int count_labels(const int32_t* labels, int T, StepScalars* sc, cudaStream_t st) {
-  count_labels_kernel<<<1, 1024, 0, st>>>(labels, T, sc);
+int count_labels(const int32_t* labels, int T, StepScalars* sc, long long denom_override, cudaStream_t st) {
+  count_labels_kernel<<<1, 1024, 0, st>>>(labels, T, sc, denom_override);
   return ok(1);
 }
 
@@ -816,6 +839,17 @@ int grad_norm_and_clip(const float* g, size_t n, float* partial, StepScalars* sc
   sqnorm_partial_kernel<<<kSqnormBlocks, 256, 0, st>>>(g, n / 4, partial);
   sqnorm_final_kernel<<<1, 256, 0, st>>>(partial, kSqnormBlocks, sc, hp);
   return ok(2);
+}
+
+int sqnorm_to(const float* g, size_t n, float* partial, float* out, cudaStream_t st) {
+  sqnorm_partial_kernel<<<kSqnormBlocks, 256, 0, st>>>(g, n / 4, partial);
+  sqnorm_sum_kernel<<<1, 256, 0, st>>>(partial, kSqnormBlocks, out);
+  return ok(2);
+}
+
+int clip_from_sq(const float* sq_total, StepScalars* sc, AdamHyper hp, cudaStream_t st) {
+  clip_from_sq_kernel<<<1, 1, 0, st>>>(sq_total, sc, hp);
+  return ok(1);
 }
 
 int advance_step(StepScalars* sc, AdamHyper hp, cudaStream_t st) {

@@ -43,7 +43,8 @@ int qknorm_bwd(bf16* dqkv, const bf16* qkv, const float* r, const bf16* gain_q, 
                const float* sinT, float* dgain_q, float* dgain_k, float* partial, size_t partial_floats, float inv_mscale2,
                int T, int S, int nh, int nkv, int d, cudaStream_t st);
 int swiglu_bwd(const bf16* d_a, const bf16* gu, bf16* d_gu, int T, int f, cudaStream_t st);
-int count_labels(const int32_t* labels, int T, StepScalars* sc, cudaStream_t st);
+// denom_override > 0: the loss mean (and the logit gradient) divide by it instead of by this batch's own label count
+int count_labels(const int32_t* labels, int T, StepScalars* sc, long long denom_override, cudaStream_t st);
 // per row: lse, loss contribution, and (if dz != null) dz = R((softmax(z) - onehot) * inv_count), zero for ignored rows
 // dz = R(dz_scale * (softmax(z) - onehot) / counted labels)
 int cross_entropy_rows(const float* z, const int32_t* labels, float* lse, float* loss_row, bf16* dz, int rows, int V,
@@ -55,6 +56,10 @@ int embed_bwd(const int32_t* tok, const bf16* dx, float* dE, unsigned long long*
               float scale, bool accumulate, cudaStream_t st);
 int grad_norm_and_clip(const float* g, size_t n, float* partial, StepScalars* sc, AdamHyper hp, cudaStream_t st);
 int advance_step(StepScalars* sc, AdamHyper hp, cudaStream_t st);
+// *out = sum of squares of g[0, n) (n a multiple of 4), fixed order; partial: kSqnormBlocks floats of scratch
+int sqnorm_to(const float* g, size_t n, float* partial, float* out, cudaStream_t st);
+// gradient norm and clip coefficient in sc from a sum of squares formed elsewhere
+int clip_from_sq(const float* sq_total, StepScalars* sc, AdamHyper hp, cudaStream_t st);
 // fused clip + Adam + decoupled decay + bf16 write-back over a flat arena; elements >= n_decay get no decay
 int adamw(float* p, float* m, float* v, const float* g, bf16* pb, size_t n, size_t n_decay, const StepScalars* sc,
           AdamHyper hp, cudaStream_t st);

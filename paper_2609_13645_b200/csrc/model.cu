@@ -100,6 +100,14 @@ struct ft_model {
   StepScalars* ring = nullptr;
   cudaEvent_t ring_ev[FT_MAX_IN_FLIGHT] = {};
   unsigned ring_head = 0, ring_tail = 0;  // submitted, collected (monotonic counters)
+  // data-parallel hooks: gradient buckets of the flat arena in the order the backward pass completes them, one event
+  // per bucket recorded on the model's stream, and the label count of all ranks for the loss mean
+  struct DpBucket { size_t offset, count; };
+  std::vector<DpBucket> dp_buckets;
+  std::vector<cudaEvent_t> dp_ev;
+  bool dp_mode = false;
+  long long label_count_override = 0;
+  float* dp_sq = nullptr;     // 4 floats of device scratch for the callers' norm reduction
   bf16* attn_ds = nullptr;    // dS^T scratch of the attention backward (one layer's worth), or null
   size_t attn_ds_bytes = 0;
   bool attn_ds_on = true;
@@ -249,6 +257,7 @@ size_t carve(ft_model* m, uint8_t* base) {
   m->attn_ds = m->attn_ds_bytes ? cv.take<bf16>(m->attn_ds_bytes / sizeof(bf16)) : nullptr;
   m->norm_partial = cv.take<float>((size_t)elementwise_blocks_for_norm((int)T) * h);
   m->sq_partial = cv.take<float>(kSqnormBlocks);
+  m->dp_sq = cv.take<float>(4);
   m->fuse_sq = cv.take<float>(m->fuse_sq_count());
   m->splitk = cv.take<float>(kSplitKFloats);
   m->splitk2 = cv.take<float>(kSplitKFloats);
@@ -523,7 +532,7 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
   cudaStream_t st = m->stream;
   m->lastB = B; m->lastS = S; m->have_bwd = false;
   m->fusing = fuse && with_bwd;
-  m->overlapping = with_bwd && m->overlap && m->side != nullptr && !m->prof && !m->cfg.debug_taps;
+  m->overlapping = with_bwd && m->overlap && m->side != nullptr && !m->prof && !m->cfg.debug_taps && !m->dp_mode;
   m->fuse_idx = 0;
   m->fuse_args.clear();
   m->fuse_args.reserve((size_t)4 * L + 1);  // pointers into it are handed to the launcher
@@ -533,7 +542,7 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
     FT_LAUNCH(FT_PROF_OPTIMIZER, 0.0, advance_step(m->sc, hyper(m), st));
   }
 
-  FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T, count_labels(lab, T, m->sc, st));
+  FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T, count_labels(lab, T, m->sc, m->label_count_override, st));
   FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T * h, embed_fwd(tok, m->wb(0), m->x[0], T, h, V, m->cfg.emb_scale, st));
   for (int l = 0; l < L; ++l) {
     ft_status s = layer_forward(m, l, m->acts[m->cfg.recompute ? 0 : l], B, S);
@@ -574,6 +583,8 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
   }
   FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T, reduce_loss(m->loss_row, T, m->sc, st));
   if (!with_bwd) return FT_OK;
+  const int dp_base = tied ? 0 : 1;  // bucket 0 is the untied head, complete here
+  if (m->dp_mode && !tied) FT_CUDA(cudaEventRecord(m->dp_ev[0], st));
 
   FT_LAUNCH(FT_PROF_NORM, 6.0 * T * h,
             rmsnorm_bwd(m->d_hF, m->x[L], m->rF, m->wb(i_normf), nullptr, m->dxA, m->gr(i_normf), m->norm_partial, T, h, st));
@@ -589,9 +600,14 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
     }
     ft_status s = layer_backward(m, l, a, B, S);
     if (s) return s;
+    if (m->dp_mode) FT_CUDA(cudaEventRecord(m->dp_ev[dp_base + (L - 1 - l)], st));
   }
   FT_LAUNCH(FT_PROF_ELEMENTWISE, 2.0 * T * h + 4.0 * V * h, embed_bwd(tok, m->dxA, m->gr(0), m->keys, T, h, V, m->cfg.emb_scale, tied, st));
   for (int k = 0; k < 4; ++k) { ft_status sw = wait_wgrad(m, k); if (sw) return sw; }  // join the second stream
+  if (m->dp_mode) {  // the embedding table and the gains (summed over the whole pass) are complete only now
+    FT_CUDA(cudaEventRecord(m->dp_ev[dp_base + L], st));
+    FT_CUDA(cudaEventRecord(m->dp_ev[dp_base + L + 1], st));
+  }
   m->overlapping = false;
   m->have_bwd = !m->fusing;  // a fusing step leaves no gradients of the matrices behind
   return FT_OK;
@@ -935,6 +951,133 @@ ft_status ft_collect_step(ft_model* m, float* host_loss, float* host_gnorm) {
   return FT_OK;
 }
 
+// ---------------------------------------------------------------- data-parallel hooks
+namespace {
+void dp_build_buckets(ft_model* m) {
+  if (!m->dp_buckets.empty()) return;
+  const int L = m->L, per = m->per_layer();
+  auto span = [&](int first, int last) {  // arena range of the matrices first..last (consecutive in the arena)
+    ft_model::DpBucket b;
+    b.offset = m->params[first].offset;
+    b.count = m->params[last].offset + align_up(m->params[last].numel(), 128) - b.offset;
+    return b;
+  };
+  if (!m->cfg.tie_embeddings) { const int ih = 1 + per * L + 1; m->dp_buckets.push_back(span(ih, ih)); }
+  for (int l = L - 1; l >= 0; --l) {
+    // a layer's matrices in parameter order: wqkv, wo, wgu, wd (the gains between them live in the gains region)
+    m->dp_buckets.push_back(span(m->idx_layer(l, 1), m->idx_layer(l, 5)));
+  }
+  m->dp_buckets.push_back(span(0, 0));
+  ft_model::DpBucket g; g.offset = m->n_decay; g.count = m->arena - m->n_decay;
+  m->dp_buckets.push_back(g);
+}
+}  // namespace
+
+int32_t ft_dp_num_buckets(ft_model* m) {
+  if (!m) return 0;
+  dp_build_buckets(m);
+  return (int32_t)m->dp_buckets.size();
+}
+
+ft_status ft_dp_bucket(ft_model* m, int32_t i, int64_t* offset, int64_t* count) {
+  if (!m || !offset || !count) return FT_EINVAL;
+  dp_build_buckets(m);
+  if (i < 0 || i >= (int32_t)m->dp_buckets.size()) return FT_ENOTFOUND;
+  *offset = (int64_t)m->dp_buckets[i].offset;
+  *count = (int64_t)m->dp_buckets[i].count;
+  return FT_OK;
+}
+
+ft_status ft_arena_ptr(ft_model* m, ft_kind kind, void** dev_ptr, int64_t* numel) {
+  if (!m || !dev_ptr || !numel) return FT_EINVAL;
+  void* b = kind_base(m, kind);
+  if (!b) return FT_EINVAL;
+  *dev_ptr = b;
+  *numel = (int64_t)m->arena;
+  return FT_OK;
+}
+
+ft_status ft_dp_scratch(ft_model* m, float** dev_ptr) {
+  if (!m || !dev_ptr) return FT_EINVAL;
+  *dev_ptr = m->dp_sq;
+  return FT_OK;
+}
+
+ft_status ft_dp_set_label_count(ft_model* m, int64_t total_count) {
+  if (!m || total_count < 0) return FT_EINVAL;
+  m->label_count_override = total_count;
+  if (m->graph_exec) { cudaGraphExecDestroy(m->graph_exec); m->graph_exec = nullptr; }  // the count is a launch argument
+  return FT_OK;
+}
+
+ft_status ft_dp_backward(ft_model* m, const int32_t* dev_tokens, const int32_t* dev_labels, int32_t B, int32_t S) {
+  if (!m) return FT_EINVAL;
+  if (m->cfg.debug_taps) return fail(m, FT_EINVAL, "data-parallel hooks are not available with debug_taps");
+  dp_build_buckets(m);
+  if (m->dp_ev.empty()) {
+    m->dp_ev.assign(m->dp_buckets.size(), nullptr);
+    for (auto& e : m->dp_ev) FT_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  }
+  m->dp_mode = true;
+  ft_status s = run_forward_backward(m, dev_tokens, dev_labels, B, S, true, false);
+  m->dp_mode = false;
+  return s;
+}
+
+ft_status ft_dp_stream_wait_bucket(ft_model* m, int32_t i, void* stream) {
+  if (!m || i < 0 || i >= (int32_t)m->dp_ev.size() || !m->dp_ev[i]) return FT_EINVAL;
+  FT_CUDA(cudaStreamWaitEvent(reinterpret_cast<cudaStream_t>(stream), m->dp_ev[i], 0));
+  return FT_OK;
+}
+
+namespace {
+bool dp_range_ok(const ft_model* m, int64_t offset, int64_t count) {
+  return offset >= 0 && count > 0 && (offset & 3) == 0 && (count & 3) == 0 && (size_t)(offset + count) <= m->arena;
+}
+}  // namespace
+
+ft_status ft_dp_sqnorm(ft_model* m, int64_t offset, int64_t count, float* dev_out, void* stream) {
+  if (!m || !dev_out || !dp_range_ok(m, offset, count)) return FT_EINVAL;
+  if (sqnorm_to(m->grad + offset, (size_t)count, m->sq_partial, dev_out, reinterpret_cast<cudaStream_t>(stream)) < 0) return FT_ECUDA;
+  return FT_OK;
+}
+
+ft_status ft_dp_begin_update(ft_model* m, const float* dev_sq_total, void* stream) {
+  if (!m) return FT_EINVAL;
+  const AdamHyper hp = hyper(m);
+  if (!dev_sq_total && hp.max_grad_norm > 0.f) return fail(m, FT_EINVAL, "clipping needs the global sum of squares first");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (advance_step(m->sc, hp, st) < 0) return FT_ECUDA;
+  if (!dev_sq_total) {
+    FT_CUDA(cudaMemsetAsync(m->dp_sq + 3, 0, sizeof(float), st));
+    dev_sq_total = m->dp_sq + 3;  // coefficient 1; the norm is reported later (ft_dp_set_norm)
+  }
+  if (clip_from_sq(dev_sq_total, m->sc, hp, st) < 0) return FT_ECUDA;
+  return FT_OK;
+}
+
+ft_status ft_dp_set_norm(ft_model* m, const float* dev_sq_total, void* stream) {
+  if (!m || !dev_sq_total) return FT_EINVAL;
+  if (clip_from_sq(dev_sq_total, m->sc, hyper(m), reinterpret_cast<cudaStream_t>(stream)) < 0) return FT_ECUDA;
+  return FT_OK;
+}
+
+ft_status ft_dp_update_range(ft_model* m, int64_t offset, int64_t count, void* stream) {
+  if (!m || !dp_range_ok(m, offset, count)) return FT_EINVAL;
+  const size_t off = (size_t)offset, n = (size_t)count;
+  const size_t n_decay = m->n_decay > off ? (m->n_decay - off < n ? m->n_decay - off : n) : 0;
+  if (adamw(m->master + off, m->adam_m + off, m->adam_v + off, m->grad + off, m->pbf + off, n, n_decay, m->sc, hyper(m),
+            reinterpret_cast<cudaStream_t>(stream)) < 0)
+    return FT_ECUDA;
+  m->have_bwd = false;
+  return FT_OK;
+}
+
+ft_status ft_dp_collect(ft_model* m, float* host_loss, float* host_gnorm) {
+  if (!m) return FT_EINVAL;
+  return finish(m, host_loss, host_gnorm);
+}
+
 ft_status ft_forward_loss(ft_model* m, const int32_t* dev_tokens, const int32_t* dev_labels, int32_t B, int32_t S,
                           float* host_loss) {
   if (!m) return FT_EINVAL;
@@ -1136,6 +1279,7 @@ void ft_destroy(ft_model* m) {
   if (m->ev_d) cudaEventDestroy(m->ev_d);
   for (auto e : m->ev_w) if (e) cudaEventDestroy(e);
   for (auto e : m->ring_ev) if (e) cudaEventDestroy(e);
+  for (auto e : m->dp_ev) if (e) cudaEventDestroy(e);
   if (m->ring) cudaFreeHost(m->ring);
   delete m;
 }

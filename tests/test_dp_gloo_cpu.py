@@ -1,0 +1,168 @@
+"""The data-parallel driver (paper_2609_13645_b200/dp.py) on CPU: two gloo ranks and a stand-in backend.
+
+The stand-in keeps flat fp32 arenas like the library's (tensors padded to 128 elements, a few buckets in completion
+order) and fills them from the ORACLE: gradients of the rank's half batch, AdamW on a range with the oracle's update.
+What is under test is the driver: global label count, in-order buckets, reduce-scatter slices, sharded update, all-gather
+of the compute copy, norm over all ranks' slices, clipping.  After two steps every rank's compute copy and its owned
+master slices must equal one oracle process that trained on the concatenated batch.
+"""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+WORKER = r"""
+import os, sys, json
+sys.path.insert(0, {root!r})
+import numpy as np, torch, torch.distributed as dist
+from contextlib import nullcontext
+from oracle import decoder as D
+from paper_2609_13645_b200.dp import DataParallel
+import synth_inputs as SI
+
+rank = int(os.environ["RANK"]); world = int(os.environ["WORLD_SIZE"])
+clip = float(sys.argv[1])
+dist.init_process_group("gloo")
+cfg = D.Config(n_layers=2, d_model=64, n_heads=2, n_kv_heads=1, head_dim=32, d_ffn=96, vocab=128, max_grad_norm=clip, lr=1e-2)
+params = D.init_params(cfg, 7)
+names = list(params)
+mats = [n for n in names if params[n].ndim == 2]
+gains = [n for n in names if params[n].ndim == 1]
+pad = lambda n: (n + 127) // 128 * 128
+
+
+class OracleBackend:
+    # flat arenas: matrices first, gains after, each padded to 128 elements; AdamW through the oracle's update
+    def __init__(self):
+        self.clipping = clip > 0
+        self.off, o = {{}}, 0
+        for n in mats + gains:
+            self.off[n] = o; o += pad(params[n].size)
+        self.n_decay = self.off[gains[0]]
+        self.arena = o
+        z = lambda dt: torch.zeros(o, dtype=dt)
+        self.master, self.m, self.v, self.g = z(torch.float64), z(torch.float64), z(torch.float64), z(torch.float32)
+        self.comp = z(torch.float32)
+        for n in names:
+            self.master[self.off[n]:self.off[n] + params[n].size] = torch.from_numpy(params[n].astype(np.float64).ravel())
+        self.comp.copy_(self.master.float())
+        self.step_no, self.clipc, self.gnorm, self.loss_share, self.total = 0, 1.0, 0.0, 0.0, 0
+        self.events = []
+    def buckets(self):
+        # completion order: last matrices first, gains last; three matrix buckets
+        k = len(mats) // 3
+        groups = [mats[2 * k:], mats[k:2 * k], mats[:k]]
+        out = [(self.off[g[0]], self.off[g[-1]] + pad(params[g[-1]].size) - self.off[g[0]]) for g in groups]
+        out.append((self.n_decay, self.arena - self.n_decay))
+        return out
+    def grad(self): return self.g
+    def compute_copy(self): return self.comp
+    def new_scalars(self, n): return torch.zeros(n, dtype=torch.float32)
+    def count_labels(self, labels): return torch.tensor([int((labels >= 0).sum())], dtype=torch.int64)
+    def set_label_count(self, n): self.total = n
+    def cur_params(self):
+        return {{n: self.comp[self.off[n]:self.off[n] + params[n].size].numpy().reshape(params[n].shape).astype(np.float32) for n in names}}
+    def backward(self, tokens, labels):
+        loss, grads, _ = D.forward_backward(cfg, self.cur_params(), tokens.numpy(), labels.numpy(), "exact", False)
+        w = float((labels >= 0).sum()) / self.total  # local mean -> share of the global mean
+        self.loss_share = loss * w
+        self.g.zero_()
+        for n in names:
+            self.g[self.off[n]:self.off[n] + params[n].size] = torch.from_numpy((grads[n] * w).astype(np.float32).ravel())
+        self.events.append("backward")
+    def comm(self): return nullcontext()
+    def begin_comm(self): pass
+    def end_comm(self): pass
+    def wait_bucket(self, i): self.events.append(("wait", i))
+    def sqnorm(self, off, cnt, out): out[0] = float((self.g[off:off + cnt].double() ** 2).sum())
+    def begin_update(self, sq):
+        self.step_no += 1
+        if sq is not None:
+            self.gnorm = float(sq[0]) ** 0.5
+            self.clipc = min(1.0, clip / (self.gnorm + 1e-6)) if clip > 0 else 1.0
+        else:
+            assert clip == 0
+            self.clipc = 1.0
+    def set_norm(self, sq): self.gnorm = float(sq[0]) ** 0.5
+    def update_range(self, off, cnt):
+        for lo, hi, wd in ((off, min(off + cnt, self.n_decay), cfg.weight_decay), (max(off, self.n_decay), off + cnt, 0.0)):
+            if hi <= lo: continue
+            p, m, v = D.adamw_update(self.master[lo:hi].numpy(), self.g[lo:hi].numpy(), self.m[lo:hi].numpy(), self.v[lo:hi].numpy(),
+                                     self.step_no, cfg, wd, self.clipc)
+            self.master[lo:hi] = torch.from_numpy(p); self.m[lo:hi] = torch.from_numpy(m); self.v[lo:hi] = torch.from_numpy(v)
+            self.comp[lo:hi] = self.master[lo:hi].float()
+        self.events.append(("update", off, cnt))
+    def collect(self): return self.loss_share, self.gnorm
+
+
+be = OracleBackend()
+dp = DataParallel(be)
+ref = D.TrainState(cfg, params)   # one process on the concatenated batch, exact arithmetic, fp32 state
+out = dict(rank=rank, losses=[], ref_losses=[], gnorms=[], ref_gnorms=[])
+for step in range(2):
+    tok, lab = SI.batch(cfg.vocab, 4, 16, "uniform", step=step)
+    lab = lab.copy(); lab[0, :5] = -1            # unequal label counts on the two ranks
+    lo, hi = rank * 2, rank * 2 + 2
+    loss, gn = dp.step(torch.from_numpy(tok[lo:hi].copy()), torch.from_numpy(lab[lo:hi].copy()))
+    rl, rg, _, _ = ref.train_step(tok, lab, mode="exact")
+    out["losses"].append(loss); out["ref_losses"].append(float(rl)); out["gnorms"].append(gn); out["ref_gnorms"].append(float(rg))
+# every rank's compute copy equals the reference parameters; its owned master slices too
+worst = 0.0
+for n in names:
+    got = be.comp[be.off[n]:be.off[n] + params[n].size].numpy().reshape(params[n].shape)
+    worst = max(worst, float(np.max(np.abs(got - ref.params[n]))) / cfg.lr)
+out["worst_in_units_of_lr"] = worst
+owned = 0.0
+for i in range(len(dp.buckets)):
+    so, sn = dp.slice_of(i)
+    owned = max(owned, float((be.master[so:so + sn].float() - be.comp[so:so + sn]).abs().max()))
+out["owned_master_vs_copy"] = owned
+out["events"] = [e if isinstance(e, str) else list(e) for e in be.events[:12]]
+out["slices"] = [list(dp.slice_of(i)) for i in range(len(dp.buckets))]
+out["buckets"] = [list(b) for b in dp.buckets]
+with open(os.path.join(sys.argv[2], f"rank{{rank}}.json"), "w") as fh:   # (two ranks printing at once interleave)
+    json.dump(out, fh)
+dist.barrier()
+dist.destroy_process_group()
+"""
+
+
+def _run(tmp_path, clip, port):
+    script = tmp_path / "dp_worker.py"
+    script.write_text(WORKER.format(root=ROOT))
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), str(script), str(clip), str(tmp_path)]
+    r = subprocess.run(cmd, cwd=ROOT, env=dict(os.environ), capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-3000:]
+    return [json.loads((tmp_path / f"rank{k}.json").read_text()) for k in range(2)]
+
+
+@pytest.mark.parametrize("clip", [0.0, 0.05])
+def test_two_rank_data_parallel_step_equals_one_process_on_the_whole_batch(tmp_path, clip):
+    res = _run(tmp_path, clip, 29741 if clip == 0.0 else 29743)
+    for d in res:
+        for a, b in zip(d["losses"], d["ref_losses"]):
+            assert abs(a - b) < 1e-5, (a, b)
+        for a, b in zip(d["gnorms"], d["ref_gnorms"]):
+            assert abs(a - b) < 1e-4 * max(1.0, b), (a, b)
+        # The ranks' fp32 gradient shares are summed in fp32; where they nearly cancel, the sum's relative error is large
+        # and Adam's g / (|g| + eps) turns it into a visible fraction of one update (lr).  Measured 0.3 % of lr; a
+        # wrong slice, a missing all-gather or a wrong label count shows as whole multiples of lr.
+        assert d["worst_in_units_of_lr"] < 0.02, d["worst_in_units_of_lr"]
+        assert d["owned_master_vs_copy"] == 0.0
+    # both ranks report the same loss and norm
+    assert res[0]["losses"] == res[1]["losses"] and res[0]["gnorms"] == res[1]["gnorms"]
+    # slices: rank r owns the r-th half of every bucket, 16-byte groups, and the two halves tile the bucket
+    for (off, cnt), s0, s1 in zip(res[0]["buckets"], res[0]["slices"], res[1]["slices"]):
+        assert s0 == [off, cnt // 2] and s1 == [off + cnt // 2, cnt // 2] and cnt % 8 == 0
+    # order of a step: backward enqueued first, then per bucket wait -> (update when clipping is off)
+    ev = res[0]["events"]
+    assert ev[0] == "backward" and ev[1] == ["wait", 0]
+    if clip == 0.0:
+        assert ev[2][0] == "update" and ev[3] == ["wait", 1]
+    else:
+        assert ev[2] == ["wait", 1]
