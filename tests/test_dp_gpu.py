@@ -24,12 +24,13 @@ def one_rank_group():
     dist.destroy_process_group()
 
 
-@pytest.mark.parametrize("clip,tied", [(0.0, False), (0.5, False), (0.0, True)])
-def test_one_rank_data_parallel_steps_equal_plain_steps(one_rank_group, clip, tied):
+@pytest.mark.parametrize("clip,tied,recompute,qk_norm", [(0.0, False, 0, False), (0.5, False, 0, False), (0.0, True, 0, False),
+                                                         (0.0, False, 1, False), (0.0, True, 0, True)])
+def test_one_rank_data_parallel_steps_equal_plain_steps(one_rank_group, clip, tied, recompute, qk_norm):
     from paper_2609_13645_b200 import binding as B
     from paper_2609_13645_b200.dp import DataParallel, LibraryBackend
     ocfg = oracle_config(n_layers=2, d_model=256, n_heads=4, n_kv_heads=2, head_dim=64, d_ffn=688, vocab=1024,
-                         max_grad_norm=clip, tie_embeddings=tied)
+                         max_grad_norm=clip, tie_embeddings=tied, qk_norm=qk_norm)
     Bsz, S = 2, 128
     batches = []
     for i in range(3):
@@ -37,7 +38,7 @@ def test_one_rank_data_parallel_steps_equal_plain_steps(one_rank_group, clip, ti
         l = l.copy(); l[0, :9] = -1
         batches.append((torch.from_numpy(t).cuda(), torch.from_numpy(l).cuda()))
 
-    plain = B.Model(lib_config(B, ocfg, Bsz, S), seed=11)
+    plain = B.Model(lib_config(B, ocfg, Bsz, S, recompute=recompute), seed=11)
     plain.set_fused_update(False)
     ref = []
     for t, l in batches:
@@ -45,7 +46,7 @@ def test_one_rank_data_parallel_steps_equal_plain_steps(one_rank_group, clip, ti
         gn = plain.apply_update()
         ref.append((loss, gn))
 
-    model = B.Model(lib_config(B, ocfg, Bsz, S), seed=11)
+    model = B.Model(lib_config(B, ocfg, Bsz, S, recompute=recompute), seed=11)
     be = LibraryBackend(model)
     dp = DataParallel(be)
     # the buckets tile the arena exactly once, in 128-element units
