@@ -102,6 +102,15 @@ ft_status ft_set_overlap(ft_model* m, int32_t enable);
  * recomputing dQ kernel.  On by default; 0 selects the recomputing kernel always.  Changing it drops a captured graph. */
 ft_status ft_set_attention_stored_ds(ft_model* m, int32_t enable);
 
+/* Streaming cross-entropy (the appendix' "chunked / streaming cross-entropy" that folds the LM-head GEMM, the loss and
+ * the logit gradient into one chunked loop without ever holding logits): the logits GEMM of a row chunk reduces every
+ * 256-column tile of a row to (max, sum of exponentials) in its epilogue, a small kernel combines the pairs into the
+ * row's log-sum-exp and loss, and the same GEMM runs a second time with an epilogue that writes the bf16 logit
+ * gradient directly.  Neither fp32 logits nor a separate cross-entropy pass exist; the price is the second GEMM.  Off
+ * by default, as in the paper (slower than the chunked path at the measured shapes).  Results agree with the default
+ * path to rounding (the sums are formed per tile, then combined).  Changing it drops a captured graph. */
+ft_status ft_set_streaming_ce(ft_model* m, int32_t enable);
+
 /* Whole-step CUDA graph (the paper's full-step graph capture): when enabled, the first ft_train_step of a (B, S)
  * runs launch by launch, the second is captured into a graph, later ones replay it (ids are first copied into the
  * model's own buffers).  Needs a capturable stream (not the legacy default stream; otherwise it switches itself

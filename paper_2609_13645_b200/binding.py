@@ -87,6 +87,8 @@ def lib():
         L.ft_submit_step_host.restype = C.c_int
         L.ft_collect_step.argtypes = [vp, vp, vp]
         L.ft_collect_step.restype = C.c_int
+        L.ft_set_streaming_ce.argtypes = [vp, i32]
+        L.ft_set_streaming_ce.restype = C.c_int
         L.ft_set_attention_stored_ds.argtypes = [vp, i32]
         L.ft_set_attention_stored_ds.restype = C.c_int
         L.ft_set_graph.argtypes = [vp, i32]
@@ -278,6 +280,10 @@ class Model:
     def set_overlap(self, enable: bool):
         """Weight-gradient GEMMs on a second stream, concurrent with the rest of the backward pass (default on)."""
         self._check(lib().ft_set_overlap(self._h, 1 if enable else 0))
+
+    def set_streaming_ce(self, enable: bool):
+        """Cross-entropy inside the logits GEMM's epilogues (no logits in memory, the GEMM runs twice); default off."""
+        self._check(lib().ft_set_streaming_ce(self._h, 1 if enable else 0))
 
     def set_attention_stored_ds(self, enable: bool):
         """Attention backward that stores dS^T once and computes dQ as one batched contraction (default on)."""

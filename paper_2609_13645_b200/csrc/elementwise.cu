@@ -322,6 +322,42 @@ cross_entropy_kernel(const float* __restrict__ z, const int32_t* __restrict__ la
   }
 }
 
+// Streaming cross-entropy, second stage: one warp per row combines the (max, sum of e^(z - max)) pairs that the
+// logits GEMM left per 256-column tile, in a fixed order, into the row's log-sum-exp and loss.
+__global__ void __launch_bounds__(256)
+ce_combine_kernel(const float2* __restrict__ part, int tiles, const float* __restrict__ zy, const int32_t* __restrict__ labels,
+                  float* __restrict__ lse_out, float* __restrict__ loss_row, int rows, int V) {
+  pdl_trigger();
+  pdl_wait();
+  const int row = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  float m = -INFINITY, s = 0.f;
+  for (int t = lane; t < tiles; t += 32) {
+    const float2 ps = part[(long long)row * tiles + t];
+    const float mn = fmaxf(m, ps.x);
+    const float a = (m == -INFINITY) ? 0.f : s * expf(m - mn);
+    const float b = (ps.x == -INFINITY) ? 0.f : ps.y * expf(ps.x - mn);
+    s = a + b;
+    m = mn;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float m2 = __shfl_xor_sync(0xffffffffu, m, o);
+    const float s2 = __shfl_xor_sync(0xffffffffu, s, o);
+    const float mm = fmaxf(m, m2);
+    const float a = (m == -INFINITY) ? 0.f : s * expf(m - mm);
+    const float b = (m2 == -INFINITY) ? 0.f : s2 * expf(m2 - mm);
+    s = (m >= m2) ? a + b : b + a;  // both partners add in the same order
+    m = mm;
+  }
+  if (lane == 0) {
+    const float lse = m + logf(s);
+    lse_out[row] = lse;
+    const int y = labels[row];
+    loss_row[row] = (y >= 0 && y < V) ? lse - zy[row] : 0.f;
+  }
+}
+
 __global__ void reduce_loss_kernel(const float* __restrict__ loss_row, int T, StepScalars* sc) {
   __shared__ float s[1024];
   float a = 0.f;
@@ -804,6 +840,12 @@ int count_labels(const int32_t* labels, int T, StepScalars* sc, long long denom_
 int cross_entropy_rows(const float* z, const int32_t* labels, float* lse, float* loss_row, bf16* dz, int rows, int V,
                        const StepScalars* sc, float dz_scale, cudaStream_t st) {
   if (launch_pdl(cross_entropy_kernel, rows, 256, 0, st, z, labels, lse, loss_row, dz, V, sc, dz_scale) != cudaSuccess) return -1;
+  return ok(1);
+}
+
+int ce_combine(const float2* part, int tiles, const float* zy, const int32_t* labels, float* lse, float* loss_row, int rows,
+               int V, cudaStream_t st) {
+  if (launch_pdl(ce_combine_kernel, (rows + 7) / 8, 256, 0, st, part, tiles, zy, labels, lse, loss_row, rows, V) != cudaSuccess) return -1;
   return ok(1);
 }
 

@@ -49,6 +49,9 @@ int count_labels(const int32_t* labels, int T, StepScalars* sc, long long denom_
 // dz = R(dz_scale * (softmax(z) - onehot) / counted labels)
 int cross_entropy_rows(const float* z, const int32_t* labels, float* lse, float* loss_row, bf16* dz, int rows, int V,
                        const StepScalars* sc, float dz_scale, cudaStream_t st);
+// streaming cross-entropy: per-tile (max, sum) pairs [rows, tiles] + the label logits -> lse and loss per row
+int ce_combine(const float2* part, int tiles, const float* zy, const int32_t* labels, float* lse, float* loss_row, int rows,
+               int V, cudaStream_t st);
 int reduce_loss(const float* loss_row, int T, StepScalars* sc, cudaStream_t st);
 // dE[v,:] (+)= scale * sum over positions with token v (fp32, position order); keys: scratch of sort_pad(T) uint64.
 // accumulate: dE already holds another gradient of the same table (tied output head) and is not cleared first.

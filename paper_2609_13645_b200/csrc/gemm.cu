@@ -82,6 +82,14 @@ struct GemmDev {
   const StepScalars* adam_sc;
   float* adam_sq;
   float adam_lr, adam_beta1, adam_beta2, adam_eps, adam_wd;
+  // streaming cross-entropy (CE instantiation of the pair kernel only)
+  int ce_mode, ce_tiles;
+  float2* ce_part;
+  float* ce_zy;
+  const float* ce_lse;
+  const int32_t* ce_labels;
+  const StepScalars* ce_sc;
+  float ce_scale;
 };
 
 __device__ __forceinline__ AdamCoef adam_coef(const GemmDev& p) {
@@ -279,11 +287,71 @@ __device__ __forceinline__ void ld_acc32(uint32_t taddr, int coloff, uint32_t (&
 // Epilogue of one accumulator tile for one thread: `row` is the global output row held by this thread's TMEM lane,
 // taddr the TMEM address of (its lane quarter, first column of the tile), n0 the tile's first output column.
 // Every tcgen05.ld is executed by all 32 lanes (rows past M only skip the stores).
-template <int BN>
+template <int BN, bool CE = false>
 __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint32_t taddr, int row, int n0, float& sq,
                                               float* stage, int cb, int ce, const Fixup fx = Fixup()) {
   const bool row_ok = row < p.M;
   uint32_t r[32];
+  if constexpr (CE) {
+    // Streaming cross-entropy: this thread holds row `row` of a 256-column tile of logits.
+    const int y = row_ok ? p.ce_labels[row] : -1;
+    if (p.ce_mode == 1) {
+      float m = -INFINITY, s = 0.f, zy = 0.f;
+      for (int c = cb; c < ce; c += 32) {
+        const int gc = n0 + c;
+        if (gc >= p.N) break;
+        ld_acc32(taddr, c, r, fx, p.alpha);
+        float cm = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          if (gc + j >= p.N) r[j] = 0xff800000u;  // -inf past the last column
+          cm = fmaxf(cm, __uint_as_float(r[j]));
+        }
+        const float mn = fmaxf(m, cm);
+        float cs = 0.f;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) cs += __expf(__uint_as_float(r[j]) - mn);
+        s = s * __expf(m - mn) + cs;  // m = -inf on the first chunk: e^(-inf) = 0
+        m = mn;
+        if (y >= gc && y < gc + 32) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (gc + j == y) zy = __uint_as_float(r[j]);
+        }
+      }
+      if (row_ok) {
+        p.ce_part[(long long)row * p.ce_tiles + n0 / BN] = make_float2(m, s);
+        if (y >= n0 && y < n0 + BN && y < p.N) p.ce_zy[row] = zy;
+      }
+    } else {
+      const float lse = row_ok ? p.ce_lse[row] : 0.f;
+      const float w = (row_ok && y >= 0 && y < p.N) ? p.ce_sc->inv_count * p.ce_scale : 0.f;
+      bf16* crow = reinterpret_cast<bf16*>(cptr) + (long long)row * p.ldc;
+      for (int c = cb; c < ce; c += 32) {
+        const int gc = n0 + c;
+        if (gc >= p.N) break;
+        ld_acc32(taddr, c, r, fx, p.alpha);
+        if (row_ok) {
+          float v[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            float pj = __expf(__uint_as_float(r[j]) - lse);
+            if (gc + j == y) pj -= 1.0f;
+            v[j] = pj * w;
+          }
+          if (p.wide_store) {
+            if (gc < p.N) store16_bf16(crow + gc, v);
+            if (gc + 16 < p.N) store16_bf16(crow + gc + 16, v + 16);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; j += 8)
+              if (gc + j < p.N) store8_bf16(crow + gc + j, v + j);
+          }
+        }
+      }
+    }
+    return;
+  }
   if (p.adam_p != nullptr) {
     // Weight gradient consumed in place: g = accumulator (+ the gradient of earlier chunks for EPI_F32_ACC), then
     // AdamW on master, moments and bf16 copy at the same position.  The 32 x 32 chunk goes through the warp's staging
@@ -799,7 +867,7 @@ struct PairCfg {
 // activity, measured on the gate/up shape, so they are used only where the epilogue is the heavy part.)
 constexpr int PAIR_THREADS = 320;
 
-template <bool A_MN, bool B_MN>
+template <bool A_MN, bool B_MN, bool CE = false>
 __global__ void __launch_bounds__(PAIR_THREADS, 1)
 gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmDev p) {
   using C = PairCfg;
@@ -982,7 +1050,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         } else if (p.ksplit > 1) {
           cptr = reinterpret_cast<float*>(p.C) + (long long)part * p.split_stride;  // this K part's own fp32 partial output
         }
-        epilogue_tile<BN>(p, cptr, taddr, row, n0, sq, stage, cb, ce, fx);
+        epilogue_tile<BN, CE>(p, cptr, taddr, row, n0, sq, stage, cb, ce, fx);
       }
       tc_fence_before();
       __syncwarp();
@@ -1126,15 +1194,17 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
   p.qk_r = a.qk_r; p.qk_gain_q = a.qk_gain_q; p.qk_gain_k = a.qk_gain_k; p.n_q_heads = a.n_q_heads; p.qk_eps = a.qk_eps;
   p.panel = (size_t)a.M * a.K * sizeof(bf16) > (48u << 20) ? 1 : 0;
   p.ksplit = 1; p.split_stride = 0; p.balanced = 0; p.sw_first = 0; p.sw_parts = 1; p.sw_kpb = 0; p.flags = nullptr; p.slots = nullptr;
+  p.ce_mode = 0; p.ce_tiles = 0; p.ce_part = nullptr; p.ce_zy = nullptr; p.ce_lse = nullptr; p.ce_labels = nullptr;
+  p.ce_sc = nullptr; p.ce_scale = 1.0f;
   const int tiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN);
   const int grid = tiles < sm_count() ? tiles : sm_count();
   return launch_pdl(kern, grid, GEMM_THREADS, C::SMEM_BYTES, stream, tmA, tmB, p);
 }
 
-template <bool A_MN, bool B_MN>
+template <bool A_MN, bool B_MN, bool CE = false>
 cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
   using C = PairCfg;
-  auto kern = gemm_tc_pair_kernel<A_MN, B_MN>;
+  auto kern = gemm_tc_pair_kernel<A_MN, B_MN, CE>;
   static unsigned long long smem_set = 0;
   cudaError_t e0 = ensure_dynamic_smem(kern, C::SMEM_BYTES, smem_set);
   if (e0 != cudaSuccess) return e0;
@@ -1183,7 +1253,9 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
   // balanced schedule: a last wave that would keep at most half of the pairs busy is divided along K
   p.balanced = 0; p.sw_first = tiles; p.sw_parts = 1; p.sw_kpb = kblocks; p.flags = flags; p.slots = data;
   const int left = tiles % max_pairs;
-  if (g_gemm_balanced && ksplit == 1 && data && tiles > max_pairs && left > 0 && max_pairs <= 256 &&
+  p.ce_mode = CE ? a.ce_mode : 0; p.ce_tiles = a.ce_tiles; p.ce_part = a.ce_part; p.ce_zy = a.ce_zy; p.ce_lse = a.ce_lse;
+  p.ce_labels = a.ce_labels; p.ce_sc = a.ce_scalars; p.ce_scale = a.ce_scale;
+  if (!CE && g_gemm_balanced && ksplit == 1 && data && tiles > max_pairs && left > 0 && max_pairs <= 256 &&
       (size_t)max_pairs * SLOT_FLOATS * sizeof(float) <= data_bytes) {
     int parts = max_pairs / left;
     // The pair with part 0 adds the other parts' tiles while its next tile's main loop runs; the longer that loop (K),
@@ -1273,6 +1345,15 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream) {
   // 128 x 256 tiles move 96 B of operands per tensor-core cycle through shared memory, 128 x 128 tiles 128 B: the
   // wide tile is faster even when it leaves SMs idle (measured), so the narrow one only serves N <= 128
   const bool wide = g_gemm_force_bn ? g_gemm_force_bn == 256 : a.N > 128;
+  if (a.ce_mode != 0) {
+    // streaming cross-entropy: the CTA-pair kernel's own instantiation; the caller pads nothing, rows and columns may be ragged
+    if (a.a_mn || a.b_mn || a.adam || a.M < 1 || (a.ce_mode != 1 && a.ce_mode != 2) || !a.ce_labels ||
+        a.ce_tiles != (a.N + 255) / 256)
+      return cudaErrorInvalidValue;
+    if (a.ce_mode == 1 && (!a.ce_part || !a.ce_zy)) return cudaErrorInvalidValue;
+    if (a.ce_mode == 2 && (!a.ce_lse || !a.ce_scalars || a.epi != EPI_BF16)) return cudaErrorInvalidValue;
+    return launch_pair_variant<false, false, true>(a, stream);
+  }
   if (g_gemm_pairs && !g_gemm_force_bn && a.M >= 256 && a.N >= 256) {
     if (!a.a_mn && !a.b_mn) return launch_pair_variant<false, false>(a, stream);
     if (!a.a_mn && a.b_mn) return launch_pair_variant<false, true>(a, stream);

@@ -73,6 +73,19 @@ struct GemmArgs {
   size_t scratch_bytes = 0;
   bool scratch_reset = false;
   const AdamFuse* adam = nullptr;
+  // Streaming cross-entropy on the logits GEMM (A, B both K-major, CTA-pair kernel; alpha = logit factor).  No logits
+  // are stored.  ce_mode 1: every thread reduces its row's 256 accumulator columns to (max, sum of e^(z - max)) and
+  // stores the pair at ce_part[row * ce_tiles + column tile]; the tile that holds the row's label column also stores that
+  // logit to ce_zy[row].  ce_mode 2: C receives bf16 dz = (e^(z - ce_lse[row]) - [column == label]) * w, with
+  // w = inv_count * ce_scale for rows whose label is counted (0 <= label < N) and 0 otherwise.
+  int ce_mode = 0;
+  float2* ce_part = nullptr;
+  int ce_tiles = 0;             // column tiles of 256 per row = (N + 255) / 256
+  float* ce_zy = nullptr;
+  const float* ce_lse = nullptr;
+  const int32_t* ce_labels = nullptr;
+  const struct StepScalars* ce_scalars = nullptr;
+  float ce_scale = 1.0f;
 };
 
 // Enqueues the contraction on `stream`.  Returns cudaErrorInvalidValue for shapes it does not take.

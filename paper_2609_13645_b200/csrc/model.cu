@@ -108,6 +108,9 @@ struct ft_model {
   bool dp_mode = false;
   long long label_count_override = 0;
   float* dp_sq = nullptr;     // 4 floats of device scratch for the callers' norm reduction
+  bool streaming_ce = false;  // policy switch (ft_set_streaming_ce): cross-entropy inside the logits GEMM, recomputed for dz
+  float2* ce_part = nullptr;  // [ce_chunk, ceil(V / 256)] per-tile (max, sum) pairs
+  float* ce_zy = nullptr;     // [ce_chunk] logit at the label
   bf16* attn_ds = nullptr;    // dS^T scratch of the attention backward (one layer's worth), or null
   size_t attn_ds_bytes = 0;
   bool attn_ds_on = true;
@@ -258,6 +261,8 @@ size_t carve(ft_model* m, uint8_t* base) {
   m->norm_partial = cv.take<float>((size_t)elementwise_blocks_for_norm((int)T) * h);
   m->sq_partial = cv.take<float>(kSqnormBlocks);
   m->dp_sq = cv.take<float>(4);
+  m->ce_part = cv.take<float2>((size_t)m->ce_chunk * ((V + 255) / 256));
+  m->ce_zy = cv.take<float>((size_t)m->ce_chunk);
   m->fuse_sq = cv.take<float>(m->fuse_sq_count());
   m->splitk = cv.take<float>(kSplitKFloats);
   m->splitk2 = cv.take<float>(kSplitKFloats);
@@ -555,15 +560,31 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
   // output head + cross-entropy (+ both head gradients) in chunks of rows: the logits of one chunk at a time
   for (int r0 = 0, chunk = 0; r0 < T; r0 += m->ce_chunk, ++chunk) {
     const int rows = (T - r0) < m->ce_chunk ? (T - r0) : m->ce_chunk;
-    {
+    if (m->streaming_ce) {
+      // no logits in memory: the GEMM's epilogue reduces each 256-column tile of a row to (max, sum), a small kernel
+      // combines them, and the same GEMM runs again with an epilogue that turns its accumulators into bf16 dz
       GemmArgs g = gemm_base(m);
-      g.A = m->hF + (size_t)r0 * h; g.lda = h; g.B = m->wb(i_head); g.ldb = h; g.C = m->z; g.ldc = V;
-      g.M = rows; g.N = V; g.K = h; g.epi = EPI_F32; g.alpha = m->cfg.logit_scale;
+      g.A = m->hF + (size_t)r0 * h; g.lda = h; g.B = m->wb(i_head); g.ldb = h; g.C = m->dz; g.ldc = V;
+      g.M = rows; g.N = V; g.K = h; g.epi = EPI_BF16; g.alpha = m->cfg.logit_scale;
+      g.ce_mode = 1; g.ce_part = m->ce_part; g.ce_tiles = (V + 255) / 256; g.ce_zy = m->ce_zy; g.ce_labels = lab + r0;
       FT_GEMM(g);
+      FT_LAUNCH(FT_PROF_CE, 8.0 * rows * g.ce_tiles,
+                ce_combine(m->ce_part, g.ce_tiles, m->ce_zy, lab + r0, m->ce_lse + r0, m->loss_row + r0, rows, V, st));
+      if (with_bwd) {
+        g.ce_mode = 2; g.ce_lse = m->ce_lse + r0; g.ce_scalars = m->sc; g.ce_scale = m->cfg.logit_scale;
+        FT_GEMM(g);
+      }
+    } else {
+      {
+        GemmArgs g = gemm_base(m);
+        g.A = m->hF + (size_t)r0 * h; g.lda = h; g.B = m->wb(i_head); g.ldb = h; g.C = m->z; g.ldc = V;
+        g.M = rows; g.N = V; g.K = h; g.epi = EPI_F32; g.alpha = m->cfg.logit_scale;
+        FT_GEMM(g);
+      }
+      FT_LAUNCH(FT_PROF_CE, (with_bwd ? 10.0 : 4.0) * rows * V,
+                cross_entropy_rows(m->z, lab + r0, m->ce_lse + r0, m->loss_row + r0, with_bwd ? m->dz : nullptr, rows, V,
+                                   m->sc, m->cfg.logit_scale, st));
     }
-    FT_LAUNCH(FT_PROF_CE, (with_bwd ? 10.0 : 4.0) * rows * V,
-              cross_entropy_rows(m->z, lab + r0, m->ce_lse + r0, m->loss_row + r0, with_bwd ? m->dz : nullptr, rows, V,
-                                 m->sc, m->cfg.logit_scale, st));
     if (with_bwd) {
       {
         GemmArgs g = gemm_base(m);
@@ -881,6 +902,13 @@ ft_status ft_set_overlap(ft_model* m, int32_t enable) {
 ft_status ft_set_attention_stored_ds(ft_model* m, int32_t enable) {
   if (!m) return FT_EINVAL;
   m->attn_ds_on = enable != 0;
+  if (m->graph_exec) { cudaGraphExecDestroy(m->graph_exec); m->graph_exec = nullptr; }  // captured with the old setting
+  return FT_OK;
+}
+
+ft_status ft_set_streaming_ce(ft_model* m, int32_t enable) {
+  if (!m) return FT_EINVAL;
+  m->streaming_ce = enable != 0;
   if (m->graph_exec) { cudaGraphExecDestroy(m->graph_exec); m->graph_exec = nullptr; }  // captured with the old setting
   return FT_OK;
 }

@@ -26,7 +26,7 @@ def _small_gqa():
     return oracle_config(n_layers=2, d_model=512, n_heads=4, n_kv_heads=2, head_dim=128, d_ffn=720, vocab=2048)
 
 
-def _check_step(ocfg, tok, lab, params, debug=True, recompute=0, report=None, stored_ds=True):
+def _check_step(ocfg, tok, lab, params, debug=True, recompute=0, report=None, stored_ds=True, streaming_ce=False):
     from paper_2609_13645_b200 import binding as B
     Bsz, S = tok.shape
     T = Bsz * S
@@ -34,6 +34,7 @@ def _check_step(ocfg, tok, lab, params, debug=True, recompute=0, report=None, st
     if ocfg.rope_factors is not None or ocfg.rope_mscale != 1.0:
         model.set_rope_scaling(ocfg.rope_factors, ocfg.rope_mscale)
     model.set_attention_stored_ds(stored_ds)
+    model.set_streaming_ce(streaming_ce)
     load_params(model, params)
     st = D.TrainState(ocfg, params)
     loss_o, gn_o, grads_o, taps_o = st.train_step(tok, lab, mode="contract", want_taps=True)
@@ -99,6 +100,37 @@ def test_gqa_head_dim_128_two_layers_with_ignored_labels():
     lab = lab.copy()
     lab[0, :7] = -1
     _check_step(ocfg, tok, lab, params)
+
+
+@pytest.mark.parametrize("shape", ["c1", "ragged_tied_mup"])
+def test_streaming_cross_entropy_matches_oracle_and_the_default_path(shape):
+    """Cross-entropy inside the logits GEMM's epilogues (per-tile max / sum pairs, then the GEMM again for dz): the same
+    parity bars as the default path, and losses / gradients that agree with it to rounding.  The ragged case has a
+    vocabulary that ends inside a 256-column tile, rows that end inside a 128-row tile, ignored labels, tied
+    embeddings and a logit factor."""
+    from paper_2609_13645_b200 import binding as B
+    if shape == "c1":
+        ocfg, w = _c1()
+        tok, lab = SI.workload_batch("c1_tiny")
+    else:
+        ocfg = oracle_config(n_layers=1, d_model=256, n_heads=4, n_kv_heads=2, head_dim=64, d_ffn=688, vocab=1000,
+                             tie_embeddings=True, logit_scale=0.5, emb_scale=4.0)
+        tok, lab = SI.batch(ocfg.vocab, 3, 70, "zipf", seed=21)
+        lab = lab.copy(); lab[1, 3:11] = -1
+    params = D.init_params(ocfg, SI.WEIGHT_SEED)
+    _check_step(ocfg, tok, lab, params, streaming_ce=True)
+    Bsz, S = tok.shape
+    out = []
+    for streaming in (False, True):
+        m = B.Model(lib_config(B, ocfg, Bsz, S), seed=1)
+        load_params(m, params)
+        m.set_streaming_ce(streaming)
+        loss = m.forward_backward(to_dev(tok), to_dev(lab))
+        out.append((loss, {n: m.get_param(n, B.KIND_GRAD) for n in params}))
+        m.close()
+    assert abs(out[0][0] - out[1][0]) < 2e-6 * abs(out[0][0])
+    for n in params:
+        assert rel_l2(out[1][1][n], out[0][1][n]) < 3e-3, n
 
 
 @pytest.mark.parametrize("stored_ds", [False, True])
