@@ -849,7 +849,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 // Two CTAs on neighbouring SMs (a cluster of 2) share one 256 x 256 output tile: each loads its own 128 rows of A and
 // its own 128 of the 256 rows of B, the leader issues tcgen05.mma.cta_group::2 (M = 256), and each CTA's TMEM ends up
 // with its 128 rows x 256 columns of the accumulator.  Per flop this moves a third less operand data through L2 and
-// shared memory than the single-CTA 128 x 256 tile.  No TMA multicast is used: every CTA fetches its own operands.
+// shared memory than the single-CTA 128 x 256 tile.  Every CTA fetches its own operands with its own TMA copies.
 struct PairCfg {
   static constexpr int BN = 256;                 // output columns of the pair's tile
   static constexpr int HALF_B = 128;             // rows of B (output columns) each CTA loads
@@ -891,10 +891,10 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::STAGES; ++s) {
       mbar_init(full_bar(s), 1);   // the leader's expect_tx arrival; both CTAs' bytes are counted on the leader's barrier
-      mbar_init(empty_bar(s), 1);  // one multicast commit
+      mbar_init(empty_bar(s), 1);  // one commit, arriving in both CTAs
     }
     for (int b = 0; b < 2; ++b) {
-      mbar_init(tfull_bar(b), 1);   // one multicast commit
+      mbar_init(tfull_bar(b), 1);   // one commit, arriving in both CTAs
       mbar_init(tempty_bar(b), 2 * (blockDim.x / 32 - 2));  // the epilogue warps of both CTAs, all arriving at the leader
     }
     *abort_flag = 0;
