@@ -136,6 +136,9 @@ ft_status ft_train_step_host(ft_model* m, const int32_t* host_tokens, const int3
  *   ft_dp_set_label_count              number of labels >= 0 over ALL ranks' batches of the next step: the loss mean and
  *                                      the logit gradients divide by it, so that the SUM of the ranks' gradients is the
  *                                      gradient of the global mean loss (0: this batch's own count, the default).
+ *   ft_dp_set_label_count_device       the same number as a device int64 that the step reads when it runs (NULL: off), so
+ *                                      that the ranks' counts can be summed on the device with no host round trip; it
+ *                                      takes precedence over ft_dp_set_label_count while set.
  *   ft_dp_backward                     enqueues forward + backward of this rank's batch on the model's stream (gradients
  *                                      materialised, weight gradients in stream order), recording one event per bucket;
  *                                      returns without waiting.
@@ -157,6 +160,7 @@ ft_status ft_dp_bucket(ft_model* m, int32_t i, int64_t* offset, int64_t* count);
 ft_status ft_arena_ptr(ft_model* m, ft_kind kind, void** dev_ptr, int64_t* numel);
 ft_status ft_dp_scratch(ft_model* m, float** dev_ptr);
 ft_status ft_dp_set_label_count(ft_model* m, int64_t total_count);
+ft_status ft_dp_set_label_count_device(ft_model* m, const int64_t* dev_total_count);
 ft_status ft_dp_backward(ft_model* m, const int32_t* dev_tokens, const int32_t* dev_labels, int32_t B, int32_t S);
 ft_status ft_dp_stream_wait_bucket(ft_model* m, int32_t i, void* stream);
 ft_status ft_dp_sqnorm(ft_model* m, int64_t offset, int64_t count, float* dev_out, void* stream);

@@ -237,7 +237,8 @@ __global__ void swiglu_bwd_kernel(const bf16* __restrict__ d_a, const bf16* __re
 }
 
 // ---------------------------------------------------------------- loss
-__global__ void count_labels_kernel(const int32_t* __restrict__ labels, int T, StepScalars* sc, long long denom_override) {
+__global__ void count_labels_kernel(const int32_t* __restrict__ labels, int T, StepScalars* sc, long long denom_override,
+                                    const long long* __restrict__ denom_dev) {
   __shared__ int s[32];
   int c = 0;
   for (int i = threadIdx.x; i < T; i += blockDim.x) c += labels[i] >= 0 ? 1 : 0;
@@ -250,6 +251,7 @@ __global__ void count_labels_kernel(const int32_t* __restrict__ labels, int T, S
     for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += s[w];
     sc->count = tot;
     // data parallelism: the mean runs over the labels of all ranks, whose number the caller provides
+    if (denom_dev != nullptr) denom_override = *denom_dev;  // the count of all ranks, reduced on the device
     const long long denom = denom_override > 0 ? denom_override : (long long)(tot > 0 ? tot : 1);
     sc->inv_count = 1.0f / (float)denom;
   }
@@ -832,8 +834,9 @@ int swiglu_bwd(const bf16* d_a, const bf16* gu, bf16* d_gu, int T, int f, cudaSt
   return ok(1);
 }
 
-int count_labels(const int32_t* labels, int T, StepScalars* sc, long long denom_override, cudaStream_t st) {
-  count_labels_kernel<<<1, 1024, 0, st>>>(labels, T, sc, denom_override);
+int count_labels(const int32_t* labels, int T, StepScalars* sc, long long denom_override, const long long* denom_dev,
+                 cudaStream_t st) {
+  count_labels_kernel<<<1, 1024, 0, st>>>(labels, T, sc, denom_override, denom_dev);
   return ok(1);
 }
 

@@ -44,7 +44,9 @@ int qknorm_bwd(bf16* dqkv, const bf16* qkv, const float* r, const bf16* gain_q, 
                int T, int S, int nh, int nkv, int d, cudaStream_t st);
 int swiglu_bwd(const bf16* d_a, const bf16* gu, bf16* d_gu, int T, int f, cudaStream_t st);
 // denom_override > 0: the loss mean (and the logit gradient) divide by it instead of by this batch's own label count
-int count_labels(const int32_t* labels, int T, StepScalars* sc, long long denom_override, cudaStream_t st);
+// (denom_dev != null: the same number read from device memory when the kernel runs)
+int count_labels(const int32_t* labels, int T, StepScalars* sc, long long denom_override, const long long* denom_dev,
+                 cudaStream_t st);
 // per row: lse, loss contribution, and (if dz != null) dz = R((softmax(z) - onehot) * inv_count), zero for ignored rows
 // dz = R(dz_scale * (softmax(z) - onehot) / counted labels)
 int cross_entropy_rows(const float* z, const int32_t* labels, float* lse, float* loss_row, bf16* dz, int rows, int V,

@@ -107,6 +107,7 @@ struct ft_model {
   std::vector<cudaEvent_t> dp_ev;
   bool dp_mode = false;
   long long label_count_override = 0;
+  const long long* label_count_dev = nullptr;  // the same, read from device memory at run time (no host round trip)
   float* dp_sq = nullptr;     // 4 floats of device scratch for the callers' norm reduction
   bool streaming_ce = false;  // policy switch (ft_set_streaming_ce): cross-entropy inside the logits GEMM, recomputed for dz
   float2* ce_part = nullptr;  // [ce_chunk, ceil(V / 256)] per-tile (max, sum) pairs
@@ -547,7 +548,7 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
     FT_LAUNCH(FT_PROF_OPTIMIZER, 0.0, advance_step(m->sc, hyper(m), st));
   }
 
-  FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T, count_labels(lab, T, m->sc, m->label_count_override, st));
+  FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T, count_labels(lab, T, m->sc, m->label_count_override, m->label_count_dev, st));
   FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T * h, embed_fwd(tok, m->wb(0), m->x[0], T, h, V, m->cfg.emb_scale, st));
   for (int l = 0; l < L; ++l) {
     ft_status s = layer_forward(m, l, m->acts[m->cfg.recompute ? 0 : l], B, S);
@@ -1035,6 +1036,13 @@ ft_status ft_dp_set_label_count(ft_model* m, int64_t total_count) {
   if (!m || total_count < 0) return FT_EINVAL;
   m->label_count_override = total_count;
   if (m->graph_exec) { cudaGraphExecDestroy(m->graph_exec); m->graph_exec = nullptr; }  // the count is a launch argument
+  return FT_OK;
+}
+
+ft_status ft_dp_set_label_count_device(ft_model* m, const int64_t* dev_total_count) {
+  if (!m) return FT_EINVAL;
+  m->label_count_dev = reinterpret_cast<const long long*>(dev_total_count);
+  if (m->graph_exec) { cudaGraphExecDestroy(m->graph_exec); m->graph_exec = nullptr; }  // the pointer is a launch argument
   return FT_OK;
 }
 

@@ -5,8 +5,9 @@ compute copy interleaved with it.
 The exchange is `torch.distributed` (NCCL between GPUs); everything else — forward, backward, norm, AdamW — runs in the
 library's own kernels through `ft_dp_*`.  One process per GPU.  Per step and rank:
 
-  1. the number of labels >= 0 is summed over the ranks (one 8-byte all-reduce) and handed to the library, so that every
-     rank's loss and gradients are already divided by the GLOBAL count and the reduction is a plain sum;
+  1. the number of labels >= 0 is summed over the ranks (one 8-byte all-reduce, on the device) and handed to the library
+     as a device pointer (no host round trip), so that every rank's loss and gradients are already divided by the GLOBAL
+     count and the reduction is a plain sum;
   2. `ft_dp_backward` enqueues forward + backward on the model's stream and records one event per gradient bucket, in
      the order the backward pass completes them (head, layers last to first, embedding table, gains);
   3. on a second stream, per bucket: wait for its event, reduce-scatter it in place (rank r keeps slice r), and, when
@@ -40,6 +41,7 @@ class LibraryBackend:
         L.ft_arena_ptr.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(i64)]
         L.ft_dp_scratch.argtypes = [vp, C.POINTER(vp)]
         L.ft_dp_set_label_count.argtypes = [vp, i64]
+        L.ft_dp_set_label_count_device.argtypes = [vp, vp]
         L.ft_dp_backward.argtypes = [vp, vp, vp, i32, i32]
         L.ft_dp_stream_wait_bucket.argtypes = [vp, i32, vp]
         L.ft_dp_sqnorm.argtypes = [vp, i64, i64, vp, vp]
@@ -47,8 +49,8 @@ class LibraryBackend:
         L.ft_dp_update_range.argtypes = [vp, i64, i64, vp]
         L.ft_dp_set_norm.argtypes = [vp, vp, vp]
         L.ft_dp_collect.argtypes = [vp, vp, vp]
-        for n in ("ft_dp_bucket", "ft_arena_ptr", "ft_dp_scratch", "ft_dp_set_label_count", "ft_dp_backward",
-                  "ft_dp_stream_wait_bucket", "ft_dp_sqnorm", "ft_dp_begin_update", "ft_dp_update_range", "ft_dp_set_norm",
+        for n in ("ft_dp_bucket", "ft_arena_ptr", "ft_dp_scratch", "ft_dp_set_label_count", "ft_dp_set_label_count_device",
+                  "ft_dp_backward", "ft_dp_stream_wait_bucket", "ft_dp_sqnorm", "ft_dp_begin_update", "ft_dp_update_range", "ft_dp_set_norm",
                   "ft_dp_collect"):
             getattr(L, n).restype = C.c_int
         self.L = L
@@ -89,8 +91,10 @@ class LibraryBackend:
     def count_labels(self, labels):
         return (labels >= 0).sum().to(self.torch.int64).reshape(1)
 
-    def set_label_count(self, n: int):
-        self.model._check(self.L.ft_dp_set_label_count(self.model._h, int(n)))
+    def set_label_count(self, total):
+        """total: int64 tensor of one element on the device holding the label count of all ranks (kept by the caller)."""
+        self._total = total
+        self.model._check(self.L.ft_dp_set_label_count_device(self.model._h, C.c_void_p(total.data_ptr())))
 
     def backward(self, tokens, labels):
         Bsz, S = tokens.shape
@@ -174,7 +178,7 @@ class DataParallel:
         be, dist = self.backend, self.dist
         total = be.count_labels(labels)
         dist.all_reduce(total, op=dist.ReduceOp.SUM, group=self.group)
-        be.set_label_count(int(total.item()))
+        be.set_label_count(total)  # stays on the device: no host round trip before the step is enqueued
         be.backward(tokens, labels)
         grad, comp = be.grad(), be.compute_copy()
         be.begin_comm()

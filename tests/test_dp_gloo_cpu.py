@@ -63,7 +63,7 @@ class OracleBackend:
     def compute_copy(self): return self.comp
     def new_scalars(self, n): return torch.zeros(n, dtype=torch.float32)
     def count_labels(self, labels): return torch.tensor([int((labels >= 0).sum())], dtype=torch.int64)
-    def set_label_count(self, n): self.total = n
+    def set_label_count(self, t): self.total = int(t[0])
     def cur_params(self):
         return {{n: self.comp[self.off[n]:self.off[n] + params[n].size].numpy().reshape(params[n].shape).astype(np.float32) for n in names}}
     def backward(self, tokens, labels):

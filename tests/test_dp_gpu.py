@@ -68,7 +68,7 @@ def test_one_rank_data_parallel_steps_equal_plain_steps(one_rank_group, clip, ti
                 assert np.array_equal(a, b), (name, kind)
     assert model.step == 3
     # and the ordinary step still works on the same model afterwards (the count override is only the driver's)
-    model._check(B.lib().ft_dp_set_label_count(model._h, 0))
+    model._check(B.lib().ft_dp_set_label_count_device(model._h, None))
     loss, _ = model.train_step(*batches[0])
     assert np.isfinite(loss)
     model.close(); plain.close()
