@@ -80,6 +80,15 @@ class Config:
     # None / 1 is plain RoPE.  (Which lambda_i a checkpoint uses is model data, passed in like the weights.)
     rope_factors: Optional[Tuple[float, ...]] = None
     rope_mscale: float = 1.0
+    # One-layer multi-token-prediction (Eagle) head (appendix "Model Architectures", row "MTP / Eagle head: On (1 layer)";
+    # appendix "Ascend Model-FLOPs Utilization": the head "repeats the backbone layer's attention, projection, and FFN
+    # plus a second output head").  The paper fixes that much and no more; reading = the published depth-1 MTP module:
+    #   h'_i = R(R(hn_i Wh^T) + en_i We^T),  hn = R(rmsnorm(x_L; g_h)),  en = R(rmsnorm(R(emb_scale E[tok_{i+1}]); g_e)),
+    #   x' = one more decoder layer on h' (parameters "mtp.layer.*"), z' = logit_scale * R(rmsnorm(x'; g_f)) W_head^T
+    #   with the backbone's output head, trained on the token after next: label'_i = label_{i+1}; the last position of a
+    #   sequence has no successor and does not count.  loss = loss_backbone + mtp_weight * mean CE(z', label').
+    mtp: bool = False
+    mtp_weight: float = 1.0
 
     @property
     def h_q(self) -> int:
@@ -145,6 +154,23 @@ def param_specs(cfg: Config) -> List[Tuple[str, Tuple[int, ...]]]:
     specs += [("norm_f", (cfg.d_model,))]
     if not cfg.tie_embeddings:
         specs += [("lm_head", (cfg.vocab, cfg.d_model))]
+    if cfg.mtp:
+        p = "mtp.layer."
+        specs += [
+            ("mtp.norm_h", (cfg.d_model,)),
+            ("mtp.norm_e", (cfg.d_model,)),
+            ("mtp.proj_h", (cfg.d_model, cfg.d_model)),
+            ("mtp.proj_e", (cfg.d_model, cfg.d_model)),
+            (p + "norm1", (cfg.d_model,)),
+            (p + "wqkv", (cfg.h_q + 2 * cfg.h_kv, cfg.d_model)),
+            (p + "wo", (cfg.d_model, cfg.h_q)),
+            (p + "norm2", (cfg.d_model,)),
+            (p + "wgu", (2 * cfg.d_ffn, cfg.d_model)),
+            (p + "wd", (cfg.d_model, cfg.d_ffn)),
+        ]
+        if cfg.qk_norm:
+            specs += [(p + "q_norm", (cfg.head_dim,)), (p + "k_norm", (cfg.head_dim,))]
+        specs += [("mtp.norm_f", (cfg.d_model,))]
     return specs
 
 
@@ -349,10 +375,8 @@ def forward_backward(cfg: Config, params: Dict[str, np.ndarray], tokens: np.ndar
     s_e, s_r, s_l = float(cfg.emb_scale), float(cfg.resid_scale), float(cfg.logit_scale)
     head = "embed" if cfg.tie_embeddings else "lm_head"
     x = R(s_e * W["embed"][tokens])  # [B,S,h]
-    saved = []
-    for l in range(cfg.n_layers):
-        p = f"layers.{l}."
-        x_in = x
+    def layer_fwd(x_in, p):
+        """One decoder layer with the parameters named p + "...": returns (x_out, what its backward needs)."""
         y, r1 = rmsnorm_fwd(x_in, W[p + "norm1"], cfg.rms_eps)
         h1 = R(y)
         qkv = h1 @ W[p + "wqkv"].T  # unrounded accumulators
@@ -376,52 +400,74 @@ def forward_backward(cfg: Config, params: Dict[str, np.ndarray], tokens: np.ndar
         U = R(gu[..., f:])
         a = R(G * sigmoid(G) * U)
         x_out = R(x_mid + s_r * (a @ W[p + "wd"].T))
-        saved.append(dict(x_in=x_in, r1=r1, h1=h1, q=q, k=k, v=v, o=o, lse=lse, x_mid=x_mid, r2=r2, h2=h2,
-                          G=G, U=U, a=a))
+        sv = dict(x_in=x_in, r1=r1, h1=h1, q=q, k=k, v=v, o=o, lse=lse, x_mid=x_mid, r2=r2, h2=h2, G=G, U=U, a=a)
         if cfg.qk_norm:
-            saved[-1].update(q_hat=q_hat, k_hat=k_hat, rq=rq, rk=rk)
+            sv.update(q_hat=q_hat, k_hat=k_hat, rq=rq, rk=rk)
         for nm, val in (("x_in", x_in), ("h1", h1), ("q", q), ("k", k), ("v", v), ("attn_lse", lse), ("o", o2),
                         ("x_mid", x_mid), ("h2", h2), ("G", G), ("U", U), ("a", a), ("x_out", x_out)):
             tap(p + nm, val)
-        x = x_out
+        return x_out, sv
 
-    y, rF = rmsnorm_fwd(x, W["norm_f"], cfg.rms_eps)
+    saved = []
+    for l in range(cfg.n_layers):
+        x, sv = layer_fwd(x, f"layers.{l}.")
+        saved.append(sv)
+
+    def head_fwd(hF_, labels_):
+        """Logits (unrounded), per-row log-sum-exp and the mean loss over the counted labels."""
+        z_ = s_l * (hF_ @ W[head].T)
+        zmax = np.max(z_, axis=-1, keepdims=True)
+        lse_ = (zmax + np.log(np.sum(np.exp(z_ - zmax), axis=-1, keepdims=True)))[..., 0]
+        counted_ = labels_ >= 0
+        n_ = int(np.sum(counted_))
+        safe_ = np.where(counted_, labels_, 0)
+        z_y = np.take_along_axis(z_, safe_[..., None], axis=-1)[..., 0]
+        loss_ = float(np.sum(np.where(counted_, lse_ - z_y, 0.0)) / max(n_, 1))
+        return z_, lse_, loss_, (counted_, n_, safe_)
+
+    def head_bwd(z_, lse_, hF_, meta, weight):
+        """B1: dz = R(weight * logit_scale (softmax(z) - onehot(y)) / n_counted), zero rows for ignored labels: the
+        gradient with respect to the unscaled product h_F W^T, rounded once.  Returns (d_hF, head gradient)."""
+        counted_, n_, safe_ = meta
+        pz = np.exp(z_ - lse_[..., None])
+        onehot = np.zeros_like(pz)
+        np.put_along_axis(onehot, safe_[..., None], 1.0, axis=-1)
+        dz = R(np.where(counted_[..., None], weight * s_l * (pz - onehot) / max(n_, 1), 0.0))
+        return R(dz @ W[head]), dz.reshape(T, V).T @ hF_.reshape(T, h)
+
+    x_L = x
+    y, rF = rmsnorm_fwd(x_L, W["norm_f"], cfg.rms_eps)
     hF = R(y)
-    z = s_l * (hF @ W[head].T)  # logits stay unrounded
-    zmax = np.max(z, axis=-1, keepdims=True)
-    ce_lse = (zmax + np.log(np.sum(np.exp(z - zmax), axis=-1, keepdims=True)))[..., 0]
-    counted = labels >= 0
-    n_cnt = int(np.sum(counted))
-    safe_lab = np.where(counted, labels, 0)
-    z_y = np.take_along_axis(z, safe_lab[..., None], axis=-1)[..., 0]
-    loss = float(np.sum(np.where(counted, ce_lse - z_y, 0.0)) / max(n_cnt, 1))
+    z, ce_lse, loss, meta = head_fwd(hF, labels)
     tap("hF", hF)
     tap("ce_lse", ce_lse)
     if keep_logits:
         taps["logits"] = z
+    if cfg.mtp:
+        # the token after next: ids shifted by one inside every sequence, the last position does not count
+        tok2 = np.concatenate([tokens[:, 1:], tokens[:, -1:]], axis=1)
+        lab2 = np.concatenate([labels[:, 1:], np.full((B, 1), -1, dtype=labels.dtype)], axis=1)
+        y, r_h = rmsnorm_fwd(x_L, W["mtp.norm_h"], cfg.rms_eps)
+        hn = R(y)
+        xe = R(s_e * W["embed"][tok2])
+        y, r_e = rmsnorm_fwd(xe, W["mtp.norm_e"], cfg.rms_eps)
+        en = R(y)
+        u1 = R(hn @ W["mtp.proj_h"].T)
+        hp = R(u1 + en @ W["mtp.proj_e"].T)
+        x2, sv2 = layer_fwd(hp, "mtp.layer.")
+        y, rF2 = rmsnorm_fwd(x2, W["mtp.norm_f"], cfg.rms_eps)
+        hF2 = R(y)
+        z2, lse2, loss2, meta2 = head_fwd(hF2, lab2)
+        tap("mtp.hn", hn); tap("mtp.en", en); tap("mtp.h_in", hp); tap("mtp.hF", hF2); tap("mtp.ce_lse", lse2)
+        taps["mtp.loss"] = loss2
+        loss = loss + float(cfg.mtp_weight) * loss2
     if not backward:
         return loss, {}, taps
 
     grads: Dict[str, np.ndarray] = {}
-    # B1: dz = R(logit_scale (softmax(z) - onehot(y)) / n_counted), zero rows for ignored labels: the gradient with
-    # respect to the unscaled product h_F W^T, rounded once
-    pz = np.exp(z - ce_lse[..., None])
-    onehot = np.zeros_like(pz)
-    np.put_along_axis(onehot, safe_lab[..., None], 1.0, axis=-1)
-    dz = R(np.where(counted[..., None], s_l * (pz - onehot) / max(n_cnt, 1), 0.0))
-    del pz, onehot
-    d_hF = R(dz @ W[head])
-    g_head = dz.reshape(T, V).T @ hF.reshape(T, h)
-    if not cfg.tie_embeddings:
-        grads["lm_head"] = g_head
-    del dz
-    tap("d_hF", d_hF)
-    dxn, grads["norm_f"] = rmsnorm_bwd(d_hF, x, rF, W["norm_f"])
-    dx = R(dxn)
 
-    for l in reversed(range(cfg.n_layers)):
-        p = f"layers.{l}."
-        sv = saved[l]
+    def layer_bwd(dx, sv, p):
+        """Backward of layer_fwd: gradient of the layer's input; parameter gradients go to grads[p + ...]."""
         tap(p + "d_x_out", dx)
         # the branch output entered the residual stream times resid_scale: its gradient is resid_scale * dx (not rounded)
         d_a = R((s_r * dx) @ W[p + "wd"])
@@ -447,8 +493,8 @@ def forward_backward(cfg: Config, params: Dict[str, np.ndarray], tokens: np.ndar
             # dy is the rounded gradient above, dx is rounded once more (it is what the projection's backward reads)
             def head_norm_bwd(dy, x_hat, r, g):
                 gdy = dy * g
-                dx = r[..., None] * (gdy - x_hat * np.mean(gdy * x_hat, axis=-1, keepdims=True))
-                return dx, np.sum((dy * x_hat).reshape(-1, d), axis=0)
+                dxh = r[..., None] * (gdy - x_hat * np.mean(gdy * x_hat, axis=-1, keepdims=True))
+                return dxh, np.sum((dy * x_hat).reshape(-1, d), axis=0)
             dq, grads[p + "q_norm"] = head_norm_bwd(dq, sv["q_hat"], sv["rq"], W[p + "q_norm"])
             dk, grads[p + "k_norm"] = head_norm_bwd(dk, sv["k_hat"], sv["rk"], W[p + "k_norm"])
             dq, dk = R(dq), R(dk)
@@ -461,11 +507,37 @@ def forward_backward(cfg: Config, params: Dict[str, np.ndarray], tokens: np.ndar
                         ("d_o", d_o), ("d_q", dq.reshape(B, S, hq)), ("d_k", dk.reshape(B, S, hkv)),
                         ("d_v", dv.reshape(B, S, hkv)), ("d_h1", d_h1), ("d_x_in", d_x_in)):
             tap(p + nm, val)
-        dx = d_x_in
+        return d_x_in
+
+    d_hF, g_head = head_bwd(z, ce_lse, hF, meta, 1.0)
+    tap("d_hF", d_hF)
+    dE = np.zeros((V, h), dtype=np.float64)
+    d_xL_mtp = 0.0
+    if cfg.mtp:
+        d_hF2, g_head2 = head_bwd(z2, lse2, hF2, meta2, float(cfg.mtp_weight))
+        g_head = g_head + g_head2
+        dxn, grads["mtp.norm_f"] = rmsnorm_bwd(d_hF2, x2, rF2, W["mtp.norm_f"])
+        d_hp = layer_bwd(R(dxn), sv2, "mtp.layer.")
+        # h' = R(u1 + en We^T), u1 = R(hn Wh^T): the add passes the gradient to both terms unchanged
+        d_en = R(d_hp @ W["mtp.proj_e"])
+        grads["mtp.proj_e"] = d_hp.reshape(T, h).T @ en.reshape(T, h)
+        d_hn = R(d_hp @ W["mtp.proj_h"])
+        grads["mtp.proj_h"] = d_hp.reshape(T, h).T @ hn.reshape(T, h)
+        dxn, grads["mtp.norm_e"] = rmsnorm_bwd(d_en, xe, r_e, W["mtp.norm_e"])
+        np.add.at(dE, tok2.reshape(-1), R(dxn).reshape(T, h))
+        dxn, grads["mtp.norm_h"] = rmsnorm_bwd(d_hn, x_L, r_h, W["mtp.norm_h"])
+        d_xL_mtp = R(dxn)  # joins the backbone's gradient of x_L below, inside its one rounding
+        tap("mtp.d_hF", d_hF2); tap("mtp.d_h_in", d_hp); tap("mtp.d_x_L", d_xL_mtp)
+    if not cfg.tie_embeddings:
+        grads["lm_head"] = g_head
+    dxn, grads["norm_f"] = rmsnorm_bwd(d_hF, x_L, rF, W["norm_f"])
+    dx = R(dxn + d_xL_mtp)
+
+    for l in reversed(range(cfg.n_layers)):
+        dx = layer_bwd(dx, saved[l], f"layers.{l}.")
         saved[l] = None
 
     # B10: dE[v,:] = sum over positions holding token v
-    dE = np.zeros((V, h), dtype=np.float64)
     np.add.at(dE, tokens.reshape(-1), dx.reshape(T, h))
     grads["embed"] = s_e * dE + (g_head if cfg.tie_embeddings else 0.0)
     return loss, grads, taps

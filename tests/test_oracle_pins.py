@@ -69,8 +69,10 @@ def test_bf16_round_ties_to_even_and_idempotent():
 VARIANTS = [dict(), dict(emb_scale=12.0, resid_scale=1.4 / math.sqrt(2), logit_scale=256.0 / 1024.0),
             dict(tie_embeddings=True), dict(tie_embeddings=True, emb_scale=3.0, resid_scale=0.7, logit_scale=0.5),
             dict(qk_norm=True), dict(qk_norm=True, tie_embeddings=True, n_kv_heads=1),
-            dict(rope_factors=(1.0, 1.7, 3.1, 4.9), rope_mscale=1.19, qk_norm=True)]
-VARIANT_IDS = ["plain", "mup", "tied", "tied+mup", "qknorm", "qknorm+tied+mqa", "longrope+qknorm"]
+            dict(rope_factors=(1.0, 1.7, 3.1, 4.9), rope_mscale=1.19, qk_norm=True),
+            dict(mtp=True, mtp_weight=0.3), dict(mtp=True, mtp_weight=1.0, tie_embeddings=True, qk_norm=True, emb_scale=3.0,
+                                                 resid_scale=0.7, logit_scale=0.5)]
+VARIANT_IDS = ["plain", "mup", "tied", "tied+mup", "qknorm", "qknorm+tied+mqa", "longrope+qknorm", "mtp", "mtp+tied+qknorm+mup"]
 
 
 @pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_IDS)
@@ -128,9 +130,7 @@ def _torch_loss(cfg, tp, tok, lab):
 
     # model variants, written the way the published muP decoders apply them: embeddings times scale_emb, every branch
     # output times scale_depth / sqrt(n_layers) before the residual add, final hidden state times the logit factor
-    x = F.embedding(torch.from_numpy(tok.astype(np.int64)), tp["embed"]) * cfg.emb_scale
-    for l in range(cfg.n_layers):
-        p = f"layers.{l}."
+    def layer(x, p):
         qkv = F.linear(rms(x, tp[p + "norm1"]), tp[p + "wqkv"])
         q, k, v = torch.split(qkv, [cfg.h_q, cfg.h_kv, cfg.h_kv], dim=-1)
         q, k = q.reshape(B, S, nh, d), k.reshape(B, S, nkv, d)
@@ -142,10 +142,28 @@ def _torch_loss(cfg, tp, tok, lab):
         o = F.scaled_dot_product_attention(q, k, v, is_causal=True)
         x = x + F.linear(o.transpose(1, 2).reshape(B, S, cfg.h_q), tp[p + "wo"]) * cfg.resid_scale
         g, u = torch.chunk(F.linear(rms(x, tp[p + "norm2"]), tp[p + "wgu"]), 2, dim=-1)
-        x = x + F.linear(F.silu(g) * u, tp[p + "wd"]) * cfg.resid_scale
-    z = F.linear(rms(x, tp["norm_f"]) * cfg.logit_scale, tp["embed"] if cfg.tie_embeddings else tp["lm_head"])
-    return F.cross_entropy(z.reshape(B * S, -1), torch.from_numpy(lab.astype(np.int64)).reshape(-1),
-                           ignore_index=-1), z
+        return x + F.linear(F.silu(g) * u, tp[p + "wd"]) * cfg.resid_scale
+
+    head = tp["embed"] if cfg.tie_embeddings else tp["lm_head"]
+    ids = torch.from_numpy(tok.astype(np.int64))
+    labels = torch.from_numpy(lab.astype(np.int64))
+    x = F.embedding(ids, tp["embed"]) * cfg.emb_scale
+    for l in range(cfg.n_layers):
+        x = layer(x, f"layers.{l}.")
+    z = F.linear(rms(x, tp["norm_f"]) * cfg.logit_scale, head)
+    loss = F.cross_entropy(z.reshape(B * S, -1), labels.reshape(-1), ignore_index=-1)
+    if cfg.mtp:
+        # the published depth-1 multi-token-prediction module: the backbone's last hidden state and the embedding of the
+        # NEXT token, each normalised, concatenated and projected back to the model width by ONE matrix [h, 2h]; one
+        # more decoder layer; the backbone's output head; trained on the token after next
+        nxt = torch.cat([ids[:, 1:], ids[:, -1:]], dim=1)
+        lab2 = torch.cat([labels[:, 1:], torch.full((B, 1), -1, dtype=torch.int64)], dim=1)
+        cat = torch.cat([rms(x, tp["mtp.norm_h"]), rms(F.embedding(nxt, tp["embed"]) * cfg.emb_scale, tp["mtp.norm_e"])], dim=-1)
+        w_cat = torch.cat([tp["mtp.proj_h"], tp["mtp.proj_e"]], dim=1)
+        x2 = layer(F.linear(cat, w_cat), "mtp.layer.")
+        z2 = F.linear(rms(x2, tp["mtp.norm_f"]) * cfg.logit_scale, head)
+        loss = loss + cfg.mtp_weight * F.cross_entropy(z2.reshape(B * S, -1), lab2.reshape(-1), ignore_index=-1)
+    return loss, z
 
 
 @pytest.mark.parametrize("variant", VARIANTS[1:], ids=VARIANT_IDS[1:])
@@ -450,3 +468,38 @@ def test_flop_formula_reproduces_the_papers_tables():
         fl = flops_per_token(int(L), int(h), int(nh), int(nkv), int(d), int(f), int(V), int(s))
         for key, want in (("ffn", ffn), ("core", core), ("head", head), ("proj", proj), ("total", total)):
             assert abs(fl[key] / 1e9 - want) < 6e-4, (name, key, fl[key] / 1e9, want)
+
+
+def test_mtp_head_properties():
+    """What the reading of the one-layer MTP head implies without any arithmetic of its own: weight 0 switches it off for
+    the backbone; its loss ignores the first label of a sequence and the last position; it adds exactly weight * its own
+    mean cross-entropy; at initialisation that cross-entropy is close to ln V like the backbone's."""
+    cfg = tiny_cfg(mtp=True, mtp_weight=0.0)
+    params = tiny_params(cfg)
+    tok, lab = tiny_batch(cfg)
+    plain = tiny_cfg()
+    pp = {k: v for k, v in params.items() if not k.startswith("mtp.")}
+    l0, g0, _ = D.forward_backward(plain, pp, tok, lab, mode="exact")
+    l1, g1, t1 = D.forward_backward(cfg, params, tok, lab, mode="exact")
+    assert l0 == l1
+    for k in g0:
+        assert np.array_equal(g0[k], g1[k]), k
+    assert all(not np.any(g1[k]) for k in g1 if k.startswith("mtp."))
+    # weight w adds w * (the head's own loss), which does not see labels[:, 0] nor anything at the last position
+    cfg_w = tiny_cfg(mtp=True, mtp_weight=0.7)
+    lw, _, tw = D.forward_backward(cfg_w, params, tok, lab, mode="exact", backward=False)
+    assert abs(lw - (l0 + 0.7 * tw["mtp.loss"])) < 1e-12
+    lab2 = lab.copy(); lab2[:, 0] = (lab2[:, 0] + 1) % cfg.vocab
+    _, _, ta = D.forward_backward(cfg_w, params, tok, lab2, mode="exact", backward=False)
+    assert ta["mtp.loss"] == tw["mtp.loss"]
+    tok2 = tok.copy(); tok2[:, -1] = (tok2[:, -1] + 1) % cfg.vocab  # the last token only feeds the uncounted last position...
+    _, _, tb = D.forward_backward(cfg_w, params, tok2, lab, mode="exact", backward=False)
+    # ... as itself and as position S-2's "next token": so the head's loss may move, but only through rows that are causal
+    # successors of S-2; the backbone rows before the last are untouched
+    assert np.array_equal(tb["ce_lse"][:, :-1], tw["ce_lse"][:, :-1])
+    # at the real initialisation scale the head starts at ln V
+    c = D.Config(n_layers=1, d_model=64, n_heads=2, n_kv_heads=1, head_dim=32, d_ffn=96, vocab=512, mtp=True)
+    p = D.init_params(c, 3)
+    t, l = tiny_batch(c, B=2, S=16)
+    _, _, tt = D.forward_backward(c, p, t, l, mode="contract", backward=False)
+    assert abs(tt["mtp.loss"] - np.log(512)) < 0.05
