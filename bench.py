@@ -114,6 +114,8 @@ def variant_kwargs(args, w):
         return {}
     if args.variant == "qknorm_tied":  # the Qwen3 column: per-head QK-Norm, tied embeddings, no muP
         return dict(qk_norm=1, tie_embeddings=1)
+    if args.variant == "mup_mtp":  # the MiniCPM5 1B column: muP factors, untied, one-layer MTP (Eagle) head
+        return dict(emb_scale=12.0, resid_scale=1.4 / w["n_layers"] ** 0.5, logit_scale=256.0 / w["d_model"], mtp=1, mtp_weight=1.0)
     return dict(emb_scale=12.0, resid_scale=1.4 / w["n_layers"] ** 0.5, logit_scale=256.0 / w["d_model"], tie_embeddings=1)
 
 
@@ -132,9 +134,9 @@ def job_tokens_per_s(tokens_per_step_per_rank, world, ms_total, steps):
     return world * tokens_per_step_per_rank / (ms_total / 1e3 / steps)
 
 
-def model_flops(w, seq):
+def model_flops(w, seq, mtp=False):
     return flops_per_token(w["n_layers"], w["d_model"], w["n_heads"], w["n_kv_heads"], w["head_dim"], w["d_ffn"],
-                           w["vocab"], seq)
+                           w["vocab"], seq, mtp=mtp)
 
 
 # ------------------------------------------------------------------------------------------ CPU oracle legs
@@ -302,7 +304,7 @@ def run_cuda(args):
     ms_total, ms_e2e, ms_prof = max_over_ranks([ms_total, ms_e2e, ms_prof], world, device="cuda")
 
     if rank == 0:
-        fl = model_flops(w, S)
+        fl = model_flops(w, S, mtp=args.variant == "mup_mtp")  # the MTP head's own row of the paper's FLOP table
         step_s = ms_total / 1e3 / args.steps
         tok_s = job_tokens_per_s(tokens_per_step, world, ms_total, args.steps)
         model_tflops = fl["total"] * tokens_per_step / step_s / 1e12
@@ -416,7 +418,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--dp", action="store_true", help="one data-parallel job over the ranks instead of independent replicas")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel separately in the timed region")
-    ap.add_argument("--variant", default="plain", choices=["plain", "mup_tied", "qknorm_tied"],
+    ap.add_argument("--variant", default="plain", choices=["plain", "mup_tied", "qknorm_tied", "mup_mtp"],
                     help="model variant on the workload's shape (default: the plain decoder the metric is quoted on)")
     ap.add_argument("--no-overlap", action="store_true", help="ablation: weight-gradient GEMMs on the main stream")
     ap.add_argument("--no-fused-update", action="store_true", help="ablation: separate AdamW pass over all parameters")

@@ -48,6 +48,15 @@ typedef struct {
   int32_t tie_embeddings;         /* 1: no lm_head parameter; the head reads the embedding table and both gradients add */
   int32_t qk_norm;                /* 1: per-head RMSNorm of q and k before the rotation (Qwen3 column of the same appendix);
                                      adds the gains layers.{l}.q_norm and layers.{l}.k_norm [head_dim], eps = rms_eps */
+  int32_t mtp;                    /* 1: one-layer multi-token-prediction (Eagle) head (same appendix, row "MTP / Eagle head:
+                                     On (1 layer)"; it "repeats the backbone layer's attention, projection, and FFN plus a
+                                     second output head"): h' = R(R(hn Wh^T) + en We^T) from the normalised last hidden
+                                     state hn and the normalised embedding en of the NEXT token, one more decoder layer, its
+                                     own final norm, the backbone's output head, trained on the token after next.
+                                     Parameters mtp.norm_h, mtp.norm_e [h], mtp.proj_h, mtp.proj_e [h, h], mtp.layer.*
+                                     (a layer's set), mtp.norm_f [h].  The step then applies AdamW in a separate pass
+                                     and the data-parallel hooks are not available. */
+  float mtp_weight;               /* loss = backbone loss + mtp_weight * (mean cross-entropy of the MTP head); 0 means 1 */
 } ft_config;
 
 typedef struct ft_model ft_model;

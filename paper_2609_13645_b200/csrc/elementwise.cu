@@ -360,6 +360,24 @@ ce_combine_kernel(const float2* __restrict__ part, int tiles, const float* __res
   }
 }
 
+// MTP head inputs: inside every sequence the ids move up by one (the last position keeps its own id) and the labels
+// move up by one (the last position gets -1: no successor, not counted)
+__global__ void mtp_shift_kernel(const int32_t* __restrict__ tok, const int32_t* __restrict__ lab, int32_t* __restrict__ tok2,
+                                 int32_t* __restrict__ lab2, int T, int S) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= T) return;
+  const bool last = (i % S) == S - 1;
+  tok2[i] = last ? tok[i] : tok[i + 1];
+  lab2[i] = last ? -1 : lab[i + 1];
+}
+
+// loss <- loss + weight * (the MTP head's mean cross-entropy)
+__global__ void add_loss_kernel(StepScalars* sc, const StepScalars* sc2, float weight) {
+  const float loss = sc->loss + weight * sc2->loss;
+  sc->loss = loss;
+  sc->nonfinite = isfinite(loss) ? 0 : 1;
+}
+
 __global__ void reduce_loss_kernel(const float* __restrict__ loss_row, int T, StepScalars* sc) {
   __shared__ float s[1024];
   float a = 0.f;
@@ -849,6 +867,16 @@ int cross_entropy_rows(const float* z, const int32_t* labels, float* lse, float*
 int ce_combine(const float2* part, int tiles, const float* zy, const int32_t* labels, float* lse, float* loss_row, int rows,
                int V, cudaStream_t st) {
   if (launch_pdl(ce_combine_kernel, (rows + 7) / 8, 256, 0, st, part, tiles, zy, labels, lse, loss_row, rows, V) != cudaSuccess) return -1;
+  return ok(1);
+}
+
+int mtp_shift(const int32_t* tok, const int32_t* lab, int32_t* tok2, int32_t* lab2, int T, int S, cudaStream_t st) {
+  mtp_shift_kernel<<<(T + 255) / 256, 256, 0, st>>>(tok, lab, tok2, lab2, T, S);
+  return ok(1);
+}
+
+int add_loss(StepScalars* sc, const StepScalars* sc2, float weight, cudaStream_t st) {
+  add_loss_kernel<<<1, 1, 0, st>>>(sc, sc2, weight);
   return ok(1);
 }
 

@@ -54,6 +54,9 @@ int cross_entropy_rows(const float* z, const int32_t* labels, float* lse, float*
 // streaming cross-entropy: per-tile (max, sum) pairs [rows, tiles] + the label logits -> lse and loss per row
 int ce_combine(const float2* part, int tiles, const float* zy, const int32_t* labels, float* lse, float* loss_row, int rows,
                int V, cudaStream_t st);
+// MTP head: ids and labels shifted by one inside every sequence of length S; loss <- loss + weight * sc2->loss
+int mtp_shift(const int32_t* tok, const int32_t* lab, int32_t* tok2, int32_t* lab2, int T, int S, cudaStream_t st);
+int add_loss(StepScalars* sc, const StepScalars* sc2, float weight, cudaStream_t st);
 int reduce_loss(const float* loss_row, int T, StepScalars* sc, cudaStream_t st);
 // dE[v,:] (+)= scale * sum over positions with token v (fp32, position order); keys: scratch of sort_pad(T) uint64.
 // accumulate: dE already holds another gradient of the same table (tied output head) and is not cleared first.

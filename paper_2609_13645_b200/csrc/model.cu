@@ -109,6 +109,13 @@ struct ft_model {
   long long label_count_override = 0;
   const long long* label_count_dev = nullptr;  // the same, read from device memory at run time (no host round trip)
   float* dp_sq = nullptr;     // 4 floats of device scratch for the callers' norm reduction
+  // one-layer MTP head: its layer's activations, inputs, shifted ids and its own loss scalars
+  LayerActs acts_mtp{};
+  bf16 *mtp_hn = nullptr, *mtp_xe = nullptr, *mtp_en = nullptr, *mtp_u1 = nullptr, *mtp_hF = nullptr, *mtp_d_hF = nullptr,
+       *mtp_d_en = nullptr, *mtp_d_hn = nullptr, *mtp_d_xe = nullptr, *mtp_d_xL = nullptr;
+  float *mtp_rh = nullptr, *mtp_re = nullptr, *mtp_rF = nullptr, *mtp_lse = nullptr;
+  int32_t *mtp_tok = nullptr, *mtp_lab = nullptr;
+  StepScalars* sc_mtp = nullptr;
   bool streaming_ce = false;  // policy switch (ft_set_streaming_ce): cross-entropy inside the logits GEMM, recomputed for dz
   float2* ce_part = nullptr;  // [ce_chunk, ceil(V / 256)] per-tile (max, sum) pairs
   float* ce_zy = nullptr;     // [ce_chunk] logit at the label
@@ -146,7 +153,9 @@ struct ft_model {
   const ParamInfo& P(int i) const { return params[i]; }
   int per_layer() const { return cfg.qk_norm ? 8 : 6; }
   // k: 0 norm1, 1 wqkv, 2 wo, 3 norm2, 4 wgu, 5 wd, (QK-Norm: 6 q_norm, 7 k_norm)
-  int idx_layer(int l, int k) const { return 1 + l * per_layer() + k; }
+  // layer index L + 1 (the slot of the residual stream after the MTP head's input) addresses the MTP head's layer
+  int idx_layer(int l, int k) const { return l < L ? 1 + l * per_layer() + k : i_mtp + 4 + k; }
+  int i_mtp = -1;  // index of mtp.norm_h: norm_h, norm_e, proj_h, proj_e, then a layer's set, then mtp.norm_f
   bf16* wb(int i) const { return pbf + params[i].offset; }
   float* gr(int i) const { return grad + params[i].offset; }
 };
@@ -158,6 +167,7 @@ void normalise(ft_config& c) {
   if (c.emb_scale == 0.f) c.emb_scale = 1.f;
   if (c.resid_scale == 0.f) c.resid_scale = 1.f;
   if (c.logit_scale == 0.f) c.logit_scale = 1.f;
+  if (c.mtp_weight == 0.f) c.mtp_weight = 1.f;
 }
 
 bool valid_config(const ft_config* c, std::string* why) {
@@ -177,6 +187,9 @@ bool valid_config(const ft_config* c, std::string* why) {
   if (c->emb_scale < 0.f || c->resid_scale < 0.f || c->logit_scale < 0.f) return bad("negative scale factor");
   if (c->tie_embeddings != 0 && c->tie_embeddings != 1) return bad("tie_embeddings must be 0 or 1");
   if (c->qk_norm != 0 && c->qk_norm != 1) return bad("qk_norm must be 0 or 1");
+  if (c->mtp != 0 && c->mtp != 1) return bad("mtp must be 0 or 1");
+  if (c->mtp_weight < 0.f) return bad("negative mtp_weight");
+  if (c->mtp && c->debug_taps) return bad("debug_taps is not available with the MTP head");
   return true;
 }
 
@@ -220,6 +233,26 @@ size_t carve(ft_model* m, uint8_t* base) {
   }
   add("norm_f", h, 0, false);
   if (!c.tie_embeddings) add("lm_head", V, h, false);
+  m->i_mtp = -1;
+  if (c.mtp) {
+    m->i_mtp = (int)m->params.size();
+    add("mtp.norm_h", h, 0, false);
+    add("mtp.norm_e", h, 0, false);
+    add("mtp.proj_h", h, h, false);
+    add("mtp.proj_e", h, h, false);
+    const std::string p = "mtp.layer.";
+    add(p + "norm1", h, 0, false);
+    add(p + "wqkv", nqkv, h, false);
+    add(p + "wo", h, hq, false);
+    add(p + "norm2", h, 0, false);
+    add(p + "wgu", 2 * f, h, true);
+    add(p + "wd", h, f, false);
+    if (c.qk_norm) {
+      add(p + "q_norm", c.head_dim, 0, false);
+      add(p + "k_norm", c.head_dim, 0, false);
+    }
+    add("mtp.norm_f", h, 0, false);
+  }
   size_t off = 0;
   for (auto& p : m->params) if (p.cols) { p.offset = off; off += align_up(p.numel(), 128); }
   m->n_decay = off;
@@ -240,7 +273,8 @@ size_t carve(ft_model* m, uint8_t* base) {
   m->tok_dev = cv.take<int32_t>(T);
   m->lab_dev = cv.take<int32_t>(T);
   m->x.assign(m->L + 1, nullptr);
-  for (int l = 0; l <= m->L; ++l) m->x[l] = cv.take<bf16>(T * h);
+  if (c.mtp) m->x.assign(m->L + 3, nullptr);  // x[L+1]: input of the MTP head's layer, x[L+2]: its output
+  for (size_t l = 0; l < m->x.size(); ++l) m->x[l] = cv.take<bf16>(T * h);
   m->acts.assign(m->n_slots, LayerActs());
   for (auto& a : m->acts) {
     a.h1 = cv.take<bf16>(T * h); a.qkv = cv.take<bf16>(T * nqkv); a.o = cv.take<bf16>(T * hq);
@@ -248,6 +282,21 @@ size_t carve(ft_model* m, uint8_t* base) {
     a.a = cv.take<bf16>(T * f); a.lse = cv.take<float>(T * c.n_heads); a.r1 = cv.take<float>(T);
     a.r2 = cv.take<float>(T);
     a.qk_r = c.qk_norm ? cv.take<float>(T * (size_t)(c.n_heads + c.n_kv_heads)) : nullptr;
+  }
+  if (c.mtp) {
+    LayerActs& a = m->acts_mtp;
+    a.h1 = cv.take<bf16>(T * h); a.qkv = cv.take<bf16>(T * nqkv); a.o = cv.take<bf16>(T * hq);
+    a.x_mid = cv.take<bf16>(T * h); a.h2 = cv.take<bf16>(T * h); a.gu = cv.take<bf16>(T * 2 * f);
+    a.a = cv.take<bf16>(T * f); a.lse = cv.take<float>(T * c.n_heads); a.r1 = cv.take<float>(T);
+    a.r2 = cv.take<float>(T);
+    a.qk_r = c.qk_norm ? cv.take<float>(T * (size_t)(c.n_heads + c.n_kv_heads)) : nullptr;
+    m->mtp_hn = cv.take<bf16>(T * h); m->mtp_xe = cv.take<bf16>(T * h); m->mtp_en = cv.take<bf16>(T * h);
+    m->mtp_u1 = cv.take<bf16>(T * h); m->mtp_hF = cv.take<bf16>(T * h); m->mtp_d_hF = cv.take<bf16>(T * h);
+    m->mtp_d_en = cv.take<bf16>(T * h); m->mtp_d_hn = cv.take<bf16>(T * h); m->mtp_d_xe = cv.take<bf16>(T * h);
+    m->mtp_d_xL = cv.take<bf16>(T * h);
+    m->mtp_rh = cv.take<float>(T); m->mtp_re = cv.take<float>(T); m->mtp_rF = cv.take<float>(T); m->mtp_lse = cv.take<float>(T);
+    m->mtp_tok = cv.take<int32_t>(T); m->mtp_lab = cv.take<int32_t>(T);
+    m->sc_mtp = cv.take<StepScalars>(1);
   }
   m->rF = cv.take<float>(T); m->ce_lse = cv.take<float>(T); m->loss_row = cv.take<float>(T);
   m->hF = cv.take<bf16>(T * h); m->d_hF = cv.take<bf16>(T * h);
@@ -529,6 +578,119 @@ ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
   return FT_OK;
 }
 
+// Output head + cross-entropy (+ both head gradients) of the hidden states hF against `lab`, in chunks of rows: the
+// logits of one chunk at a time.  sc holds the label count the mean runs over; dz_scale multiplies the logit gradient
+// (logit factor, times the loss weight of this head); accumulate: the head's weight gradient already holds another
+// head's contribution; fuse_last: the last chunk completes that gradient and may carry AdamW.
+ft_status head_pass(ft_model* m, const bf16* hF, const int32_t* lab, float* lse, bf16* d_hF, StepScalars* sc, float dz_scale,
+                    int i_head, int T, bool with_bwd, bool accumulate, bool fuse_last) {
+  const int h = m->h, V = m->V;
+  cudaStream_t st = m->stream;
+  for (int r0 = 0, chunk = 0; r0 < T; r0 += m->ce_chunk, ++chunk) {
+    const int rows = (T - r0) < m->ce_chunk ? (T - r0) : m->ce_chunk;
+    if (m->streaming_ce) {
+      // no logits in memory: the GEMM's epilogue reduces each 256-column tile of a row to (max, sum), a small kernel
+      // combines them, and the same GEMM runs again with an epilogue that turns its accumulators into bf16 dz
+      GemmArgs g = gemm_base(m);
+      g.A = hF + (size_t)r0 * h; g.lda = h; g.B = m->wb(i_head); g.ldb = h; g.C = m->dz; g.ldc = V;
+      g.M = rows; g.N = V; g.K = h; g.epi = EPI_BF16; g.alpha = m->cfg.logit_scale;
+      g.ce_mode = 1; g.ce_part = m->ce_part; g.ce_tiles = (V + 255) / 256; g.ce_zy = m->ce_zy; g.ce_labels = lab + r0;
+      FT_GEMM(g);
+      FT_LAUNCH(FT_PROF_CE, 8.0 * rows * g.ce_tiles,
+                ce_combine(m->ce_part, g.ce_tiles, m->ce_zy, lab + r0, lse + r0, m->loss_row + r0, rows, V, st));
+      if (with_bwd) {
+        g.ce_mode = 2; g.ce_lse = lse + r0; g.ce_scalars = sc; g.ce_scale = dz_scale;
+        FT_GEMM(g);
+      }
+    } else {
+      {
+        GemmArgs g = gemm_base(m);
+        g.A = hF + (size_t)r0 * h; g.lda = h; g.B = m->wb(i_head); g.ldb = h; g.C = m->z; g.ldc = V;
+        g.M = rows; g.N = V; g.K = h; g.epi = EPI_F32; g.alpha = m->cfg.logit_scale;
+        FT_GEMM(g);
+      }
+      FT_LAUNCH(FT_PROF_CE, (with_bwd ? 10.0 : 4.0) * rows * V,
+                cross_entropy_rows(m->z, lab + r0, lse + r0, m->loss_row + r0, with_bwd ? m->dz : nullptr, rows, V,
+                                   sc, dz_scale, st));
+    }
+    if (with_bwd) {
+      {
+        GemmArgs g = gemm_base(m);
+        g.A = m->dz; g.lda = V; g.B = m->wb(i_head); g.b_mn = 1; g.ldb = h; g.C = d_hF + (size_t)r0 * h; g.ldc = h;
+        g.M = rows; g.N = h; g.K = V; g.epi = EPI_BF16;
+        FT_GEMM(g);
+      }
+      {
+        GemmArgs g = gemm_base(m);
+        g.A = m->dz; g.a_mn = 1; g.lda = V; g.B = hF + (size_t)r0 * h; g.b_mn = 1; g.ldb = h; g.C = m->gr(i_head);
+        g.ldc = h; g.M = V; g.N = h; g.K = rows; g.epi = (chunk == 0 && !accumulate) ? EPI_F32 : EPI_F32_ACC;
+        // the last chunk completes the gradient (with tied embeddings the table's own part is still to come)
+        if (m->fusing && fuse_last && r0 + rows >= T) g.adam = fuse_for(m, i_head);
+        FT_GEMM(g);
+      }
+    }
+  }
+  return FT_OK;
+}
+
+// One-layer MTP head, forward and its own output-head pass: the normalised last hidden state and the normalised
+// embedding of the next token are projected (two h x h matrices, the second GEMM adds the first's rounded output) into
+// the input of one more decoder layer; its normalised output goes through the backbone's output head against the
+// labels shifted by one; the step's loss becomes loss + mtp_weight * (this head's mean cross-entropy).
+ft_status mtp_forward_and_head(ft_model* m, const int32_t* tok, const int32_t* lab, int B, int S, int i_head, bool with_bwd) {
+  const int T = B * S, h = m->h, V = m->V, L = m->L, i0 = m->i_mtp, i_nf = i0 + 4 + m->per_layer();
+  cudaStream_t st = m->stream;
+  FT_LAUNCH(FT_PROF_ELEMENTWISE, 16.0 * T, mtp_shift(tok, lab, m->mtp_tok, m->mtp_lab, T, S, st));
+  FT_LAUNCH(FT_PROF_NORM, 4.0 * T * h, rmsnorm_fwd(m->x[L], m->wb(i0), m->mtp_hn, m->mtp_rh, T, h, m->cfg.rms_eps, st));
+  FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T * h, embed_fwd(m->mtp_tok, m->wb(0), m->mtp_xe, T, h, V, m->cfg.emb_scale, st));
+  FT_LAUNCH(FT_PROF_NORM, 4.0 * T * h, rmsnorm_fwd(m->mtp_xe, m->wb(i0 + 1), m->mtp_en, m->mtp_re, T, h, m->cfg.rms_eps, st));
+  {
+    GemmArgs g = gemm_base(m);
+    g.A = m->mtp_hn; g.lda = h; g.B = m->wb(i0 + 2); g.ldb = h; g.C = m->mtp_u1; g.ldc = h;
+    g.M = T; g.N = h; g.K = h; g.epi = EPI_BF16;
+    FT_GEMM(g);
+  }
+  {
+    GemmArgs g = gemm_base(m);
+    g.A = m->mtp_en; g.lda = h; g.B = m->wb(i0 + 3); g.ldb = h; g.C = m->x[L + 1]; g.ldc = h; g.resid = m->mtp_u1;
+    g.M = T; g.N = h; g.K = h; g.epi = EPI_BF16_RESID;
+    FT_GEMM(g);
+  }
+  ft_status s = layer_forward(m, L + 1, m->acts_mtp, B, S);
+  if (s) return s;
+  FT_LAUNCH(FT_PROF_NORM, 4.0 * T * h, rmsnorm_fwd(m->x[L + 2], m->wb(i_nf), m->mtp_hF, m->mtp_rF, T, h, m->cfg.rms_eps, st));
+  FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T, count_labels(m->mtp_lab, T, m->sc_mtp, 0, nullptr, st));
+  s = head_pass(m, m->mtp_hF, m->mtp_lab, m->mtp_lse, m->mtp_d_hF, m->sc_mtp, m->cfg.logit_scale * m->cfg.mtp_weight, i_head, T,
+                with_bwd, true, false);
+  if (s) return s;
+  FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T, reduce_loss(m->loss_row, T, m->sc_mtp, st));
+  FT_LAUNCH(FT_PROF_ELEMENTWISE, 0.0, add_loss(m->sc, m->sc_mtp, m->cfg.mtp_weight, st));
+  return FT_OK;
+}
+
+// Its backward: through the head's final norm, the layer, the two projections and the two input norms.  Leaves the
+// gradient with respect to the backbone's last hidden state in mtp_d_xL (bf16; the backbone's final-norm backward adds
+// it inside its one rounding) and scatters the next-token embedding gradient into the table's gradient.
+ft_status mtp_backward(ft_model* m, int B, int S, bool tied) {
+  const int T = B * S, h = m->h, V = m->V, L = m->L, i0 = m->i_mtp, i_nf = i0 + 4 + m->per_layer();
+  cudaStream_t st = m->stream;
+  FT_LAUNCH(FT_PROF_NORM, 6.0 * T * h, rmsnorm_bwd(m->mtp_d_hF, m->x[L + 2], m->mtp_rF, m->wb(i_nf), nullptr, m->dxA, m->gr(i_nf),
+                                                    m->norm_partial, T, h, st));
+  ft_status s = layer_backward(m, L + 1, m->acts_mtp, B, S);
+  if (s) return s;
+  // h' = R(u1 + en We^T), u1 = R(hn Wh^T): the add hands the same gradient (dxA) to both projections
+  if ((s = linear_backward(m, m->dxA, m->mtp_en, i0 + 3, m->mtp_d_en, T, h, h, 0))) return s;
+  if ((s = linear_backward(m, m->dxA, m->mtp_hn, i0 + 2, m->mtp_d_hn, T, h, h, 0))) return s;
+  FT_LAUNCH(FT_PROF_NORM, 6.0 * T * h, rmsnorm_bwd(m->mtp_d_en, m->mtp_xe, m->mtp_re, m->wb(i0 + 1), nullptr, m->mtp_d_xe,
+                                                    m->gr(i0 + 1), m->norm_partial, T, h, st));
+  // with tied embeddings the head passes have already written the table's gradient; otherwise this is its first part
+  FT_LAUNCH(FT_PROF_ELEMENTWISE, 2.0 * T * h + 4.0 * V * h,
+            embed_bwd(m->mtp_tok, m->mtp_d_xe, m->gr(0), m->keys, T, h, V, m->cfg.emb_scale, tied, st));
+  FT_LAUNCH(FT_PROF_NORM, 6.0 * T * h, rmsnorm_bwd(m->mtp_d_hn, m->x[L], m->mtp_rh, m->wb(i0), nullptr, m->mtp_d_xL, m->gr(i0),
+                                                    m->norm_partial, T, h, st));
+  return FT_OK;
+}
+
 // forward (+ backward when with_bwd) of one batch; everything is enqueued, nothing is synchronised
 ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* lab, int B, int S, bool with_bwd,
                                bool fuse = false) {
@@ -558,58 +720,28 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
   const int i_normf = 1 + m->per_layer() * L, i_head = tied ? 0 : i_normf + 1;  // tied: the head reads (and adds its gradient to) the table
   FT_LAUNCH(FT_PROF_NORM, 4.0 * T * h, rmsnorm_fwd(m->x[L], m->wb(i_normf), m->hF, m->rF, T, h, m->cfg.rms_eps, st));
 
-  // output head + cross-entropy (+ both head gradients) in chunks of rows: the logits of one chunk at a time
-  for (int r0 = 0, chunk = 0; r0 < T; r0 += m->ce_chunk, ++chunk) {
-    const int rows = (T - r0) < m->ce_chunk ? (T - r0) : m->ce_chunk;
-    if (m->streaming_ce) {
-      // no logits in memory: the GEMM's epilogue reduces each 256-column tile of a row to (max, sum), a small kernel
-      // combines them, and the same GEMM runs again with an epilogue that turns its accumulators into bf16 dz
-      GemmArgs g = gemm_base(m);
-      g.A = m->hF + (size_t)r0 * h; g.lda = h; g.B = m->wb(i_head); g.ldb = h; g.C = m->dz; g.ldc = V;
-      g.M = rows; g.N = V; g.K = h; g.epi = EPI_BF16; g.alpha = m->cfg.logit_scale;
-      g.ce_mode = 1; g.ce_part = m->ce_part; g.ce_tiles = (V + 255) / 256; g.ce_zy = m->ce_zy; g.ce_labels = lab + r0;
-      FT_GEMM(g);
-      FT_LAUNCH(FT_PROF_CE, 8.0 * rows * g.ce_tiles,
-                ce_combine(m->ce_part, g.ce_tiles, m->ce_zy, lab + r0, m->ce_lse + r0, m->loss_row + r0, rows, V, st));
-      if (with_bwd) {
-        g.ce_mode = 2; g.ce_lse = m->ce_lse + r0; g.ce_scalars = m->sc; g.ce_scale = m->cfg.logit_scale;
-        FT_GEMM(g);
-      }
-    } else {
-      {
-        GemmArgs g = gemm_base(m);
-        g.A = m->hF + (size_t)r0 * h; g.lda = h; g.B = m->wb(i_head); g.ldb = h; g.C = m->z; g.ldc = V;
-        g.M = rows; g.N = V; g.K = h; g.epi = EPI_F32; g.alpha = m->cfg.logit_scale;
-        FT_GEMM(g);
-      }
-      FT_LAUNCH(FT_PROF_CE, (with_bwd ? 10.0 : 4.0) * rows * V,
-                cross_entropy_rows(m->z, lab + r0, m->ce_lse + r0, m->loss_row + r0, with_bwd ? m->dz : nullptr, rows, V,
-                                   m->sc, m->cfg.logit_scale, st));
-    }
-    if (with_bwd) {
-      {
-        GemmArgs g = gemm_base(m);
-        g.A = m->dz; g.lda = V; g.B = m->wb(i_head); g.b_mn = 1; g.ldb = h; g.C = m->d_hF + (size_t)r0 * h; g.ldc = h;
-        g.M = rows; g.N = h; g.K = V; g.epi = EPI_BF16;
-        FT_GEMM(g);
-      }
-      {
-        GemmArgs g = gemm_base(m);
-        g.A = m->dz; g.a_mn = 1; g.lda = V; g.B = m->hF + (size_t)r0 * h; g.b_mn = 1; g.ldb = h; g.C = m->gr(i_head);
-        g.ldc = h; g.M = V; g.N = h; g.K = rows; g.epi = chunk == 0 ? EPI_F32 : EPI_F32_ACC;
-        // the last chunk completes the gradient (with tied embeddings the table's own part is still to come)
-        if (m->fusing && !tied && r0 + rows >= T) g.adam = fuse_for(m, i_head);
-        FT_GEMM(g);
-      }
-    }
+  {
+    ft_status sh = head_pass(m, m->hF, lab, m->ce_lse, m->d_hF, m->sc, m->cfg.logit_scale, i_head, T, with_bwd, false,
+                             !tied && !m->cfg.mtp);
+    if (sh) return sh;
   }
   FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T, reduce_loss(m->loss_row, T, m->sc, st));
+  if (m->cfg.mtp) {
+    ft_status sm = mtp_forward_and_head(m, tok, lab, B, S, i_head, with_bwd);
+    if (sm) return sm;
+  }
   if (!with_bwd) return FT_OK;
   const int dp_base = tied ? 0 : 1;  // bucket 0 is the untied head, complete here
   if (m->dp_mode && !tied) FT_CUDA(cudaEventRecord(m->dp_ev[0], st));
 
+  if (m->cfg.mtp) {
+    ft_status sm = mtp_backward(m, B, S, tied);
+    if (sm) return sm;
+    if ((sm = wait_wgrad(m, 0))) return sm;  // the projections' weight gradients still read dxA
+  }
   FT_LAUNCH(FT_PROF_NORM, 6.0 * T * h,
-            rmsnorm_bwd(m->d_hF, m->x[L], m->rF, m->wb(i_normf), nullptr, m->dxA, m->gr(i_normf), m->norm_partial, T, h, st));
+            rmsnorm_bwd(m->d_hF, m->x[L], m->rF, m->wb(i_normf), m->cfg.mtp ? m->mtp_d_xL : nullptr, m->dxA, m->gr(i_normf),
+                        m->norm_partial, T, h, st));
   for (int l = L - 1; l >= 0; --l) {
     LayerActs& a = m->acts[m->cfg.recompute ? 0 : l];
     if (m->cfg.recompute) {
@@ -624,7 +756,7 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
     if (s) return s;
     if (m->dp_mode) FT_CUDA(cudaEventRecord(m->dp_ev[dp_base + (L - 1 - l)], st));
   }
-  FT_LAUNCH(FT_PROF_ELEMENTWISE, 2.0 * T * h + 4.0 * V * h, embed_bwd(tok, m->dxA, m->gr(0), m->keys, T, h, V, m->cfg.emb_scale, tied, st));
+  FT_LAUNCH(FT_PROF_ELEMENTWISE, 2.0 * T * h + 4.0 * V * h, embed_bwd(tok, m->dxA, m->gr(0), m->keys, T, h, V, m->cfg.emb_scale, tied || m->cfg.mtp, st));
   for (int k = 0; k < 4; ++k) { ft_status sw = wait_wgrad(m, k); if (sw) return sw; }  // join the second stream
   if (m->dp_mode) {  // the embedding table and the gains (summed over the whole pass) are complete only now
     FT_CUDA(cudaEventRecord(m->dp_ev[dp_base + L], st));
@@ -818,7 +950,7 @@ ft_status ft_init_model(const ft_config* cfg, uint64_t seed, void* dev_workspace
 
 // One full step enqueued launch by launch.
 static ft_status step_direct(ft_model* m, const int32_t* tok, const int32_t* lab, int32_t B, int32_t S) {
-  const bool fuse = m->fused_update && m->cfg.max_grad_norm <= 0.f && !m->cfg.debug_taps;
+  const bool fuse = m->fused_update && m->cfg.max_grad_norm <= 0.f && !m->cfg.debug_taps && !m->cfg.mtp;
   ft_status s = run_forward_backward(m, tok, lab, B, S, true, fuse);
   if (s) return s;
   return fuse ? run_update_rest(m) : run_update(m);
@@ -1049,6 +1181,7 @@ ft_status ft_dp_set_label_count_device(ft_model* m, const int64_t* dev_total_cou
 ft_status ft_dp_backward(ft_model* m, const int32_t* dev_tokens, const int32_t* dev_labels, int32_t B, int32_t S) {
   if (!m) return FT_EINVAL;
   if (m->cfg.debug_taps) return fail(m, FT_EINVAL, "data-parallel hooks are not available with debug_taps");
+  if (m->cfg.mtp) return fail(m, FT_EINVAL, "data-parallel hooks are not available with the MTP head");
   dp_build_buckets(m);
   if (m->dp_ev.empty()) {
     m->dp_ev.assign(m->dp_buckets.size(), nullptr);

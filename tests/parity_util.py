@@ -13,7 +13,7 @@ def oracle_config(**kw):
     """Oracle config whose hyper-parameters carry the fp32 values the C struct holds."""
     c = D.Config(**kw)
     for k in ("rms_eps", "rope_theta", "lr", "beta1", "beta2", "adam_eps", "weight_decay", "max_grad_norm", "emb_scale",
-              "resid_scale", "logit_scale"):
+              "resid_scale", "logit_scale", "mtp_weight"):
         setattr(c, k, f32(getattr(c, k)))
     return c
 
@@ -24,7 +24,7 @@ def lib_config(B, ocfg, max_batch, max_seq, **extra):
                          beta1=ocfg.beta1, beta2=ocfg.beta2, adam_eps=ocfg.adam_eps, weight_decay=ocfg.weight_decay,
                          max_grad_norm=ocfg.max_grad_norm, emb_scale=ocfg.emb_scale, resid_scale=ocfg.resid_scale,
                          logit_scale=ocfg.logit_scale, tie_embeddings=int(ocfg.tie_embeddings), qk_norm=int(ocfg.qk_norm),
-                         **extra)
+                         mtp=int(ocfg.mtp), mtp_weight=ocfg.mtp_weight, **extra)
 
 
 def rel_l2(a, b):

@@ -470,6 +470,23 @@ def test_flop_formula_reproduces_the_papers_tables():
             assert abs(fl[key] / 1e9 - want) < 6e-4, (name, key, fl[key] / 1e9, want)
 
 
+def test_flop_formula_with_the_mtp_head_reproduces_the_papers_row():
+    """The printed 1.452 GFLOP/token of the MTP row fixes what the head consists of: one more layer, a second output
+    head and a [h, 2h] projection (a layer plus a head alone gives 1.423)."""
+    from paper_2609_13645_b200.flops import flops_per_token
+    for line in open(os.path.join(GOLDEN, "paper_flops_mtp.txt")):
+        if not line.strip() or line[0] == "#":
+            continue
+        left, right = line.split("|")
+        name, L, h, f, nh, nkv, d, V, s = left.split()
+        ffn, core, head, proj, mtp, total = map(float, right.split())
+        fl = flops_per_token(int(L), int(h), int(nh), int(nkv), int(d), int(f), int(V), int(s), mtp=True)
+        for key, want in (("ffn", ffn), ("core", core), ("head", head), ("proj", proj), ("mtp", mtp), ("total", total)):
+            assert abs(fl[key] / 1e9 - want) < 6e-4, (name, key, fl[key] / 1e9, want)
+        layer_and_head = fl["mtp"] - 3 * 2 * (2 * int(h)) * int(h)
+        assert abs(layer_and_head / 1e9 - mtp) > 0.02
+
+
 def test_mtp_head_properties():
     """What the reading of the one-layer MTP head implies without any arithmetic of its own: weight 0 switches it off for
     the backbone; its loss ignores the first label of a sequence and the last position; it adds exactly weight * its own

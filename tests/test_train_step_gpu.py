@@ -102,6 +102,56 @@ def test_gqa_head_dim_128_two_layers_with_ignored_labels():
     _check_step(ocfg, tok, lab, params)
 
 
+@pytest.mark.parametrize("variant", ["mtp", "mtp+tied+qknorm+mup", "mtp+ragged+streaming"])
+def test_mtp_head_step_matches_oracle_on_loss_every_gradient_and_master(variant):
+    """The one-layer MTP (Eagle) head of the paper's 1B configuration: the normalised last hidden state and the normalised
+    embedding of the next token, projected, through one more decoder layer and the backbone's output head, trained on
+    the token after next with its own weight.  Full-step parity with the oracle: loss, every gradient (backbone, head,
+    embedding table with its three contributions when tied, all mtp.* tensors), AdamW, masters."""
+    import math
+    kw = dict(n_layers=2, d_model=256, n_heads=4, n_kv_heads=2, head_dim=64, d_ffn=688, vocab=1024, mtp=True, mtp_weight=0.3)
+    Bsz, S = 2, 128
+    streaming = False
+    if "tied" in variant:
+        kw.update(tie_embeddings=True, qk_norm=True, emb_scale=12.0, resid_scale=1.4 / math.sqrt(2), logit_scale=0.5,
+                  mtp_weight=1.0)
+    if "ragged" in variant:
+        kw.update(vocab=1000, d_ffn=720)
+        Bsz, S, streaming = 3, 70, True
+    ocfg = oracle_config(**kw)
+    params = D.init_params(ocfg, SI.WEIGHT_SEED)
+    assert "mtp.proj_e" in params and "mtp.layer.wgu" in params
+    tok, lab = SI.batch(ocfg.vocab, Bsz, S, "zipf", seed=31)
+    lab = lab.copy(); lab[0, 5:9] = -1
+    _check_step(ocfg, tok, lab, params, debug=False, streaming_ce=streaming)
+
+
+def test_mtp_head_step_is_bit_identical_with_graph_recomputation_and_second_stream():
+    from paper_2609_13645_b200 import binding as B
+    ocfg = oracle_config(n_layers=2, d_model=256, n_heads=4, n_kv_heads=2, head_dim=64, d_ffn=688, vocab=1024, mtp=True,
+                         mtp_weight=0.5)
+    Bsz, S = 2, 128
+    batches = [SI.batch(ocfg.vocab, Bsz, S, "zipf", step=i) for i in range(4)]
+    outs = []
+    for recompute, overlap, graph in [(0, False, False), (1, True, False), (0, True, True)]:
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            model = B.Model(lib_config(B, ocfg, Bsz, S, recompute=recompute), seed=5)
+            model.set_overlap(overlap)
+            model.set_graph(graph)
+            losses = [model.train_step(to_dev(t), to_dev(l))[0] for t, l in batches]
+            side.synchronize()
+            state = [model.get_param(n, B.KIND_MASTER).view(np.uint32).copy() for n, _ in model.params]
+            if graph:
+                assert model.graph_replays >= 2
+            model.close()
+        outs.append((np.float32(losses).view(np.uint32), state))
+    for o in outs[1:]:
+        assert np.array_equal(o[0], outs[0][0])
+        for a, b in zip(o[1], outs[0][1]):
+            assert np.array_equal(a, b)
+
+
 @pytest.mark.parametrize("shape", ["c1", "ragged_tied_mup"])
 def test_streaming_cross_entropy_matches_oracle_and_the_default_path(shape):
     """Cross-entropy inside the logits GEMM's epilogues (per-tile max / sum pairs, then the GEMM again for dz): the same
