@@ -54,8 +54,7 @@ typedef struct {
                                      state hn and the normalised embedding en of the NEXT token, one more decoder layer, its
                                      own final norm, the backbone's output head, trained on the token after next.
                                      Parameters mtp.norm_h, mtp.norm_e [h], mtp.proj_h, mtp.proj_e [h, h], mtp.layer.*
-                                     (a layer's set), mtp.norm_f [h].  The step then applies AdamW in a separate pass
-                                     and the data-parallel hooks are not available. */
+                                     (a layer's set), mtp.norm_f [h].  The data-parallel hooks are not available with it. */
   float mtp_weight;               /* loss = backbone loss + mtp_weight * (mean cross-entropy of the MTP head); 0 means 1 */
 } ft_config;
 

@@ -129,7 +129,10 @@ struct ft_model {
   int fuse_idx = 0;           // next slot region of fuse_sq
   float* fuse_sq = nullptr;   // partial sums of the squared gradient norm: [4L+1][kAdamFuseSlots] + 2 x [kSqnormBlocks]
   std::vector<AdamFuse> fuse_args;  // kept alive until the launches are enqueued
-  size_t fuse_sq_count() const { return (size_t)(4 * L + 1) * kAdamFuseSlots + 2 * (size_t)kSqnormBlocks; }
+  // weight-gradient GEMMs that can carry AdamW: four per layer, the untied head, and with the MTP head its layer's four
+  // and its two projections
+  int n_fused() const { return 4 * L + 1 + (cfg.mtp ? 6 : 0); }
+  size_t fuse_sq_count() const { return (size_t)n_fused() * kAdamFuseSlots + 2 * (size_t)kSqnormBlocks; }
 
   // whole-step CUDA graph: the first step of a (B, S) runs launch by launch, the second is captured, later ones replay
   bool graph_enabled = false;
@@ -660,8 +663,9 @@ ft_status mtp_forward_and_head(ft_model* m, const int32_t* tok, const int32_t* l
   if (s) return s;
   FT_LAUNCH(FT_PROF_NORM, 4.0 * T * h, rmsnorm_fwd(m->x[L + 2], m->wb(i_nf), m->mtp_hF, m->mtp_rF, T, h, m->cfg.rms_eps, st));
   FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T, count_labels(m->mtp_lab, T, m->sc_mtp, 0, nullptr, st));
+  // this pass completes the head's weight gradient: its last chunk may carry AdamW (untied head only)
   s = head_pass(m, m->mtp_hF, m->mtp_lab, m->mtp_lse, m->mtp_d_hF, m->sc_mtp, m->cfg.logit_scale * m->cfg.mtp_weight, i_head, T,
-                with_bwd, true, false);
+                with_bwd, true, m->cfg.tie_embeddings == 0);
   if (s) return s;
   FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T, reduce_loss(m->loss_row, T, m->sc_mtp, st));
   FT_LAUNCH(FT_PROF_ELEMENTWISE, 0.0, add_loss(m->sc, m->sc_mtp, m->cfg.mtp_weight, st));
@@ -703,7 +707,7 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
   m->overlapping = with_bwd && m->overlap && m->side != nullptr && !m->prof && !m->cfg.debug_taps && !m->dp_mode;
   m->fuse_idx = 0;
   m->fuse_args.clear();
-  m->fuse_args.reserve((size_t)4 * L + 1);  // pointers into it are handed to the launcher
+  m->fuse_args.reserve((size_t)m->n_fused());  // pointers into it are handed to the launcher
   if (m->fusing) {
     // the optimizer step counter and bias corrections must be current before the first weight-gradient epilogue
     FT_CUDA(cudaMemsetAsync(m->fuse_sq, 0, m->fuse_sq_count() * sizeof(float), st));
@@ -790,7 +794,7 @@ ft_status run_update(ft_model* m) {
 ft_status run_update_rest(ft_model* m) {
   cudaStream_t st = m->stream;
   const AdamHyper hp = hyper(m);
-  const size_t fused_slots = (size_t)(4 * m->L + 1) * kAdamFuseSlots;
+  const size_t fused_slots = (size_t)m->n_fused() * kAdamFuseSlots;
   const size_t embed_span = (m->params[0].numel() + 127) / 128 * 128;  // embed is the first tensor of the arenas
   FT_LAUNCH(FT_PROF_OPTIMIZER, 30.0 * embed_span,
             adamw_range_with_norm(m->master, m->adam_m, m->adam_v, m->grad, m->pbf, embed_span, embed_span,
@@ -950,7 +954,7 @@ ft_status ft_init_model(const ft_config* cfg, uint64_t seed, void* dev_workspace
 
 // One full step enqueued launch by launch.
 static ft_status step_direct(ft_model* m, const int32_t* tok, const int32_t* lab, int32_t B, int32_t S) {
-  const bool fuse = m->fused_update && m->cfg.max_grad_norm <= 0.f && !m->cfg.debug_taps && !m->cfg.mtp;
+  const bool fuse = m->fused_update && m->cfg.max_grad_norm <= 0.f && !m->cfg.debug_taps;
   ft_status s = run_forward_backward(m, tok, lab, B, S, true, fuse);
   if (s) return s;
   return fuse ? run_update_rest(m) : run_update(m);

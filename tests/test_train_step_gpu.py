@@ -35,6 +35,8 @@ def _check_step(ocfg, tok, lab, params, debug=True, recompute=0, report=None, st
         model.set_rope_scaling(ocfg.rope_factors, ocfg.rope_mscale)
     model.set_attention_stored_ds(stored_ds)
     model.set_streaming_ce(streaming_ce)
+    if not debug:  # gradients are compared below: keep them (the fused epilogues consume them; their bits are tested apart)
+        model.set_fused_update(False)
     load_params(model, params)
     st = D.TrainState(ocfg, params)
     loss_o, gn_o, grads_o, taps_o = st.train_step(tok, lab, mode="contract", want_taps=True)
@@ -126,18 +128,20 @@ def test_mtp_head_step_matches_oracle_on_loss_every_gradient_and_master(variant)
     _check_step(ocfg, tok, lab, params, debug=False, streaming_ce=streaming)
 
 
-def test_mtp_head_step_is_bit_identical_with_graph_recomputation_and_second_stream():
+def test_mtp_head_step_is_bit_identical_with_graph_recomputation_second_stream_and_fused_update():
     from paper_2609_13645_b200 import binding as B
     ocfg = oracle_config(n_layers=2, d_model=256, n_heads=4, n_kv_heads=2, head_dim=64, d_ffn=688, vocab=1024, mtp=True,
                          mtp_weight=0.5)
     Bsz, S = 2, 128
     batches = [SI.batch(ocfg.vocab, Bsz, S, "zipf", step=i) for i in range(4)]
     outs = []
-    for recompute, overlap, graph in [(0, False, False), (1, True, False), (0, True, True)]:
+    for recompute, overlap, graph, fused in [(0, False, False, False), (1, True, False, True), (0, True, True, True),
+                                             (0, False, False, True)]:
         side = torch.cuda.Stream()
         with torch.cuda.stream(side):
             model = B.Model(lib_config(B, ocfg, Bsz, S, recompute=recompute), seed=5)
             model.set_overlap(overlap)
+            model.set_fused_update(fused)
             model.set_graph(graph)
             losses = [model.train_step(to_dev(t), to_dev(l))[0] for t, l in batches]
             side.synchronize()
