@@ -54,7 +54,7 @@ typedef struct {
                                      state hn and the normalised embedding en of the NEXT token, one more decoder layer, its
                                      own final norm, the backbone's output head, trained on the token after next.
                                      Parameters mtp.norm_h, mtp.norm_e [h], mtp.proj_h, mtp.proj_e [h, h], mtp.layer.*
-                                     (a layer's set), mtp.norm_f [h].  The data-parallel hooks are not available with it. */
+                                     (a layer's set), mtp.norm_f [h]. */
   float mtp_weight;               /* loss = backbone loss + mtp_weight * (mean cross-entropy of the MTP head); 0 means 1 */
 } ft_config;
 
@@ -136,7 +136,8 @@ ft_status ft_train_step_host(ft_model* m, const int32_t* host_tokens, const int3
  *
  * The flat fp32 gradient arena (and the identically laid out master / moment / bf16 arenas, ft_arena_ptr) is cut into
  * buckets in the order in which the backward pass completes them: the untied LM head first, then the layers from the
- * last to the first (each layer's four matrices, contiguous), then the embedding table, then all gains.  Every bucket
+ * last to the first (each layer's four matrices, contiguous), then the embedding table, then all gains; with the MTP
+ * head its six matrices form a bucket between the output head and the last layer.  Every bucket
  * starts on a multiple of 128 elements and has a multiple of 128 elements, so it divides evenly over 2, 4, ... 128
  * ranks.
  *   ft_dp_num_buckets / ft_dp_bucket   number of buckets; arena offset and element count of bucket i.
@@ -146,7 +147,9 @@ ft_status ft_train_step_host(ft_model* m, const int32_t* host_tokens, const int3
  *                                      gradient of the global mean loss (0: this batch's own count, the default).
  *   ft_dp_set_label_count_device       the same number as a device int64 that the step reads when it runs (NULL: off), so
  *                                      that the ranks' counts can be summed on the device with no host round trip; it
- *                                      takes precedence over ft_dp_set_label_count while set.
+ *                                      takes precedence over ft_dp_set_label_count while set.  With the MTP head the
+ *                                      pointer addresses TWO int64: the labels' count and the count of the labels
+ *                                      shifted by one (labels[:, 1:] >= 0) over all ranks.
  *   ft_dp_backward                     enqueues forward + backward of this rank's batch on the model's stream (gradients
  *                                      materialised, weight gradients in stream order), recording one event per bucket;
  *                                      returns without waiting.

@@ -662,7 +662,9 @@ ft_status mtp_forward_and_head(ft_model* m, const int32_t* tok, const int32_t* l
   ft_status s = layer_forward(m, L + 1, m->acts_mtp, B, S);
   if (s) return s;
   FT_LAUNCH(FT_PROF_NORM, 4.0 * T * h, rmsnorm_fwd(m->x[L + 2], m->wb(i_nf), m->mtp_hF, m->mtp_rF, T, h, m->cfg.rms_eps, st));
-  FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T, count_labels(m->mtp_lab, T, m->sc_mtp, 0, nullptr, st));
+  // data parallelism: the second element of the device count array is the shifted labels' count over all ranks
+  FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T,
+            count_labels(m->mtp_lab, T, m->sc_mtp, 0, m->label_count_dev ? m->label_count_dev + 1 : nullptr, st));
   // this pass completes the head's weight gradient: its last chunk may carry AdamW (untied head only)
   s = head_pass(m, m->mtp_hF, m->mtp_lab, m->mtp_lse, m->mtp_d_hF, m->sc_mtp, m->cfg.logit_scale * m->cfg.mtp_weight, i_head, T,
                 with_bwd, true, m->cfg.tie_embeddings == 0);
@@ -735,13 +737,15 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
     if (sm) return sm;
   }
   if (!with_bwd) return FT_OK;
-  const int dp_base = tied ? 0 : 1;  // bucket 0 is the untied head, complete here
+  // bucket 0 is the untied head, complete here (after the MTP head's pass when there is one); then the MTP head's matrices
+  const int dp_base = (tied ? 0 : 1) + (m->cfg.mtp ? 1 : 0);
   if (m->dp_mode && !tied) FT_CUDA(cudaEventRecord(m->dp_ev[0], st));
 
   if (m->cfg.mtp) {
     ft_status sm = mtp_backward(m, B, S, tied);
     if (sm) return sm;
     if ((sm = wait_wgrad(m, 0))) return sm;  // the projections' weight gradients still read dxA
+    if (m->dp_mode) FT_CUDA(cudaEventRecord(m->dp_ev[dp_base - 1], st));
   }
   FT_LAUNCH(FT_PROF_NORM, 6.0 * T * h,
             rmsnorm_bwd(m->d_hF, m->x[L], m->rF, m->wb(i_normf), m->cfg.mtp ? m->mtp_d_xL : nullptr, m->dxA, m->gr(i_normf),
@@ -1128,6 +1132,9 @@ void dp_build_buckets(ft_model* m) {
     return b;
   };
   if (!m->cfg.tie_embeddings) { const int ih = 1 + per * L + 1; m->dp_buckets.push_back(span(ih, ih)); }
+  // the MTP head's matrices (two projections, then its layer's four: consecutive in the arena) are complete before the
+  // backbone's backward pass starts
+  if (m->cfg.mtp) m->dp_buckets.push_back(span(m->i_mtp + 2, m->i_mtp + 4 + 5));
   for (int l = L - 1; l >= 0; --l) {
     // a layer's matrices in parameter order: wqkv, wo, wgu, wd (the gains between them live in the gains region)
     m->dp_buckets.push_back(span(m->idx_layer(l, 1), m->idx_layer(l, 5)));
@@ -1185,7 +1192,6 @@ ft_status ft_dp_set_label_count_device(ft_model* m, const int64_t* dev_total_cou
 ft_status ft_dp_backward(ft_model* m, const int32_t* dev_tokens, const int32_t* dev_labels, int32_t B, int32_t S) {
   if (!m) return FT_EINVAL;
   if (m->cfg.debug_taps) return fail(m, FT_EINVAL, "data-parallel hooks are not available with debug_taps");
-  if (m->cfg.mtp) return fail(m, FT_EINVAL, "data-parallel hooks are not available with the MTP head");
   dp_build_buckets(m);
   if (m->dp_ev.empty()) {
     m->dp_ev.assign(m->dp_buckets.size(), nullptr);

@@ -89,10 +89,12 @@ class LibraryBackend:
         return self.torch.zeros(n, dtype=self.torch.float32, device=self.device)
 
     def count_labels(self, labels):
-        return (labels >= 0).sum().to(self.torch.int64).reshape(1)
+        """[labels counted by the backbone's loss, labels counted by the MTP head's loss (shifted by one)] as int64."""
+        t = self.torch
+        return t.stack([(labels >= 0).sum(), (labels[:, 1:] >= 0).sum()]).to(t.int64)
 
     def set_label_count(self, total):
-        """total: int64 tensor of one element on the device holding the label count of all ranks (kept by the caller)."""
+        """total: int64 tensor on the device holding the label counts of all ranks (kept alive here)."""
         self._total = total
         self.model._check(self.L.ft_dp_set_label_count_device(self.model._h, C.c_void_p(total.data_ptr())))
 
