@@ -119,6 +119,14 @@ ft_status ft_set_attention_stored_ds(ft_model* m, int32_t enable);
  * path to rounding (the sums are formed per tile, then combined).  Changing it drops a captured graph. */
 ft_status ft_set_streaming_ce(ft_model* m, int32_t enable);
 
+/* SwiGLU backward inside the down projection's data-gradient contraction (the appendix' fused elementwise work around
+ * the SwiGLU block, applied to the backward pass): the gradient d_a of a = silu(G) U is rounded to bf16 in the
+ * epilogue, which reads G and U of the same positions and writes d_G = d_a U s (1 + G (1 - s)) and d_U = d_a G s,
+ * s = sigmoid(G); d_a itself is never stored and the separate elementwise pass does not run.  Bit-identical to the
+ * unfused path (same arithmetic on the same rounded d_a).  On by default; not used with debug_taps (the tap d_a needs
+ * the stored tensor).  Changing it drops a captured graph. */
+ft_status ft_set_fused_swiglu_bwd(ft_model* m, int32_t enable);
+
 /* Whole-step CUDA graph (the paper's full-step graph capture): when enabled, the first ft_train_step of a (B, S)
  * runs launch by launch, the second is captured into a graph, later ones replay it (ids are first copied into the
  * model's own buffers).  Needs a capturable stream (not the legacy default stream; otherwise it switches itself

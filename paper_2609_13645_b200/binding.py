@@ -92,6 +92,8 @@ def lib():
         L.ft_set_streaming_ce.restype = C.c_int
         L.ft_set_attention_stored_ds.argtypes = [vp, i32]
         L.ft_set_attention_stored_ds.restype = C.c_int
+        L.ft_set_fused_swiglu_bwd.argtypes = [vp, i32]
+        L.ft_set_fused_swiglu_bwd.restype = C.c_int
         L.ft_set_graph.argtypes = [vp, i32]
         L.ft_set_graph.restype = C.c_int
         L.ft_graph_replays.argtypes = [vp]
@@ -290,6 +292,10 @@ class Model:
     def set_attention_stored_ds(self, enable: bool):
         """Attention backward that stores dS^T once and computes dQ as one batched contraction (default on)."""
         self._check(lib().ft_set_attention_stored_ds(self._h, 1 if enable else 0))
+
+    def set_fused_swiglu_bwd(self, enable: bool):
+        """SwiGLU backward in the epilogue of the down projection's data-gradient GEMM (default on; bit-identical)."""
+        self._check(lib().ft_set_fused_swiglu_bwd(self._h, 1 if enable else 0))
 
     def set_graph(self, enable: bool):
         """Capture the whole step into a CUDA graph on its second run and replay it afterwards."""

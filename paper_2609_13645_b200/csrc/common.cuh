@@ -27,6 +27,17 @@ __device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v 
 // Round an fp32 value to bf16 and back (the value a stored bf16 tensor would hold).
 __device__ __forceinline__ float round_bf16(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
 
+// SwiGLU backward of one element: a = silu(G) U, so dU = da G s and dG = da U s (1 + G (1 - s)) with s = sigmoid(G).
+// Every operation is spelled out with its rounding so that the stand-alone kernel and the GEMM epilogue that fuses it
+// give the same bits.  The sigmoid uses the hardware exponential and reciprocal like the forward epilogue (relative
+// error about 2^-21, far below the bf16 rounding of the results): in the epilogue the accurate forms made the
+// epilogue, not the contraction, the long pole of the kernel.
+__device__ __forceinline__ void swiglu_bwd_elem(float da, float G, float U, float& dG, float& dU) {
+  const float sg = __fdividef(1.0f, __fadd_rn(1.0f, __expf(-G)));
+  dU = __fmul_rn(__fmul_rn(da, G), sg);
+  dG = __fmul_rn(__fmul_rn(__fmul_rn(da, U), sg), __fmaf_rn(G, __fsub_rn(1.0f, sg), 1.0f));
+}
+
 // ---------------------------------------------------------------- mbarrier
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));

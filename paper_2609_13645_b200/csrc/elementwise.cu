@@ -225,11 +225,7 @@ __global__ void swiglu_bwd_kernel(const bf16* __restrict__ d_a, const bf16* __re
     unpack8(*reinterpret_cast<const uint4*>(gu + t * 2 * f + c), G);
     unpack8(*reinterpret_cast<const uint4*>(gu + t * 2 * f + f + c), U);
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      const float sg = 1.0f / (1.0f + expf(-G[e]));
-      dU[e] = da[e] * G[e] * sg;
-      dG[e] = da[e] * U[e] * sg * (1.0f + G[e] * (1.0f - sg));
-    }
+    for (int e = 0; e < 8; ++e) swiglu_bwd_elem(da[e], G[e], U[e], dG[e], dU[e]);
     const int phys = ((c >> 4) << 5) + (c & 15);
     *reinterpret_cast<uint4*>(d_gu + t * 2 * f + phys) = pack8(dG);
     *reinterpret_cast<uint4*>(d_gu + t * 2 * f + phys + 16) = pack8(dU);

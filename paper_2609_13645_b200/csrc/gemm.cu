@@ -116,6 +116,17 @@ __device__ __forceinline__ void adam_prefetch_chunk(const GemmDev& p, const void
 // operand rows per K block instead of 34 (measured on a data-gradient GEMM with a 184 MB operand: DRAM reads down from
 // 900 to 380 MB, 6.5 % faster; on the gate/up GEMM, whose operands fit in L2, the row-fastest order is 1 % faster).
 constexpr int kPanel = 8;
+// SwiGLU-backward epilogue: ask for this thread's row of gate and up, columns [gc, gc + ncols), to be brought into L2
+// while the tile's contraction still runs (they were written a whole forward pass ago and come from HBM).
+__device__ __forceinline__ void swiglu_bwd_prefetch(const GemmDev& p, int row, int gc, int ncols) {
+  if (row >= p.M) return;
+  const bf16* g = p.gu + (long long)row * (2LL * p.d_ffn) + gc;
+  for (int c = 0; c < ncols && gc + c < p.N; c += 64) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(g + c));
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(g + p.d_ffn + c));
+  }
+}
+
 __device__ __forceinline__ void tile_coords(int panel, int tile, int tiles_m, int tiles_n, int& mi, int& ni) {
   if (!panel) {
     ni = tile / tiles_m;
@@ -287,12 +298,12 @@ __device__ __forceinline__ void ld_acc32(uint32_t taddr, int coloff, uint32_t (&
 // Epilogue of one accumulator tile for one thread: `row` is the global output row held by this thread's TMEM lane,
 // taddr the TMEM address of (its lane quarter, first column of the tile), n0 the tile's first output column.
 // Every tcgen05.ld is executed by all 32 lanes (rows past M only skip the stores).
-template <int BN, bool CE = false>
+template <int BN, int MODE = 0>  // MODE 1: streaming cross-entropy, 2: SwiGLU backward (instantiations of their own)
 __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint32_t taddr, int row, int n0, float& sq,
                                               float* stage, int cb, int ce, const Fixup fx = Fixup()) {
   const bool row_ok = row < p.M;
   uint32_t r[32];
-  if constexpr (CE) {
+  if constexpr (MODE == 1) {
     // Streaming cross-entropy: this thread holds row `row` of a 256-column tile of logits.
     const int y = row_ok ? p.ce_labels[row] : -1;
     if (p.ce_mode == 1) {
@@ -346,6 +357,83 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
 #pragma unroll
             for (int j = 0; j < 32; j += 8)
               if (gc + j < p.N) store8_bf16(crow + gc + j, v + j);
+          }
+        }
+      }
+    }
+    return;
+  }
+  if constexpr (MODE == 2) {
+    // SwiGLU backward: the accumulator is d_a (logical ffn columns); gate and up of the same (row, column) come from the
+    // forward pass' gu, one 32-column chunk ahead like the residual below (the kernel asked for the row's lines to be
+    // brought into L2 before it waited for the accumulator).  The 32 columns of a chunk land in 64 contiguous output
+    // columns: [16 d_gate | 16 d_up] twice.  (Tried: 8 lanes per row through the staging tile, so that every store is
+    // a full line: a third slower; the loads' latency, not the number of requests, is what this epilogue waits for.)
+    const int f = p.d_ffn;
+    const bf16* grow = p.gu + (long long)row * (2LL * f);
+    bf16* drow = reinterpret_cast<bf16*>(cptr) + (long long)row * p.ldc;
+    uint4 nG[4], nU[4];
+    auto fetch = [&](int gc) {
+      if (p.wide_store) {  // 32-byte loads
+#pragma unroll
+        for (int j = 0; j < 4; j += 2) {
+          if (row_ok && gc + 8 * j < p.N) {
+            uint32_t w[8];
+            load8_b32(grow + gc + 8 * j, w);
+            nG[j] = make_uint4(w[0], w[1], w[2], w[3]);
+            nG[j + 1] = make_uint4(w[4], w[5], w[6], w[7]);
+            load8_b32(grow + f + gc + 8 * j, w);
+            nU[j] = make_uint4(w[0], w[1], w[2], w[3]);
+            nU[j + 1] = make_uint4(w[4], w[5], w[6], w[7]);
+          } else {
+            nG[j] = nG[j + 1] = nU[j] = nU[j + 1] = make_uint4(0, 0, 0, 0);
+          }
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const bool ok = row_ok && gc + 8 * j < p.N;
+          nG[j] = ok ? *reinterpret_cast<const uint4*>(grow + gc + 8 * j) : make_uint4(0, 0, 0, 0);
+          nU[j] = ok ? *reinterpret_cast<const uint4*>(grow + f + gc + 8 * j) : make_uint4(0, 0, 0, 0);
+        }
+      }
+    };
+    fetch(n0 + cb);
+    for (int c = cb; c < ce; c += 32) {
+      const int gc = n0 + c;
+      if (gc >= p.N) break;
+      uint4 cG[4], cU[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) { cG[j] = nG[j]; cU[j] = nU[j]; }
+      if (c + 32 < ce) fetch(gc + 32);
+      ld_acc32(taddr, c, r, fx, p.alpha);
+      if (row_ok) {
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {  // the chunk's two groups of 16 logical columns
+          if (gc + 16 * hh < p.N) {
+            float dG[16], dU[16];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+              const uint4 g4 = cG[2 * hh + q], u4 = cU[2 * hh + q];
+              const uint32_t gw[4] = {g4.x, g4.y, g4.z, g4.w}, uw[4] = {u4.x, u4.y, u4.z, u4.w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const int j = 16 * hh + 8 * q + 2 * e;
+                swiglu_bwd_elem(round_bf16(__uint_as_float(r[j])), bf16_lo(gw[e]), bf16_lo(uw[e]), dG[8 * q + 2 * e], dU[8 * q + 2 * e]);
+                swiglu_bwd_elem(round_bf16(__uint_as_float(r[j + 1])), bf16_hi(gw[e]), bf16_hi(uw[e]), dG[8 * q + 2 * e + 1],
+                                dU[8 * q + 2 * e + 1]);
+              }
+            }
+            bf16* dst = drow + 2 * gc + 32 * hh;
+            if (p.wide_store) {
+              store16_bf16(dst, dG);
+              store16_bf16(dst + 16, dU);
+            } else {
+              store8_bf16(dst, dG);
+              store8_bf16(dst + 8, dG + 8);
+              store8_bf16(dst + 16, dU);
+              store8_bf16(dst + 24, dU + 8);
+            }
           }
         }
       }
@@ -684,7 +772,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, void* cptr, uint
   }
 }
 
-template <int BN, bool A_MN, bool B_MN>
+template <int BN, bool A_MN, bool B_MN, int MODE = 0>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmDev p) {
   using C = Cfg<BN>;
@@ -810,12 +898,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       tile_coords(p.panel, t, tiles_m, tiles_n, mi, ni);
       const int m0 = mi * BM, n0 = ni * BN;
       if (p.adam_p != nullptr) adam_prefetch_chunk(p, p.C, m0 + q * 32 + lane, n0);
+      if constexpr (MODE == 2) swiglu_bwd_prefetch(p, m0 + q * 32 + lane, n0, BN);
       bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.err);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
       const int row = m0 + q * 32 + lane;
-      epilogue_tile<BN>(p, p.C, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), row, n0, sq,
+      epilogue_tile<BN, MODE>(p, p.C, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), row, n0, sq,
                         reinterpret_cast<float*>(smem + C::STAGES * C::STAGE_BYTES + C::BAR_BYTES) + q * EPI_STAGE_FLOATS, 0, BN);
       tc_fence_before();
       __syncwarp();
@@ -867,7 +956,7 @@ struct PairCfg {
 // activity, measured on the gate/up shape, so they are used only where the epilogue is the heavy part.)
 constexpr int PAIR_THREADS = 320;
 
-template <bool A_MN, bool B_MN, bool CE = false>
+template <bool A_MN, bool B_MN, int MODE = 0>
 __global__ void __launch_bounds__(PAIR_THREADS, 1)
 gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmDev p) {
   using C = PairCfg;
@@ -1009,6 +1098,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int m0 = mi * 256 + (int)rank * BM;
       const int n0 = ni * BN;
       if (p.adam_p != nullptr && !(split && part > 0)) adam_prefetch_chunk(p, p.C, m0 + q * 32 + lane, n0 + cb);
+      // (asking one piece earlier instead, from the previous piece's epilogue, was slower: 219 us against 201 at c3_1b)
+      if constexpr (MODE == 2) { if (!(split && part > 0)) swiglu_bwd_prefetch(p, m0 + q * 32 + lane, n0 + cb, ncols); }
       bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.err);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -1050,7 +1141,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         } else if (p.ksplit > 1) {
           cptr = reinterpret_cast<float*>(p.C) + (long long)part * p.split_stride;  // this K part's own fp32 partial output
         }
-        epilogue_tile<BN, CE>(p, cptr, taddr, row, n0, sq, stage, cb, ce, fx);
+        epilogue_tile<BN, MODE>(p, cptr, taddr, row, n0, sq, stage, cb, ce, fx);
       }
       tc_fence_before();
       __syncwarp();
@@ -1166,10 +1257,10 @@ int sm_count() {
   return n;
 }
 
-template <int BN, bool A_MN, bool B_MN>
+template <int BN, bool A_MN, bool B_MN, int MODE = 0>
 cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
   using C = Cfg<BN>;
-  auto kern = gemm_tc_kernel<BN, A_MN, B_MN>;
+  auto kern = gemm_tc_kernel<BN, A_MN, B_MN, MODE>;
   static unsigned long long smem_set = 0;
   cudaError_t e0 = ensure_dynamic_smem(kern, C::SMEM_BYTES, smem_set);
   if (e0 != cudaSuccess) return e0;
@@ -1188,7 +1279,7 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
     const int m = f32out ? 7 : 15;  // elements per 32 bytes, minus one
     bool ok32 = (reinterpret_cast<uintptr_t>(a.C) & 31) == 0 && (a.ldc & m) == 0 && (a.N & m) == 0;
     if (a.epi == EPI_BF16_RESID) ok32 = ok32 && (reinterpret_cast<uintptr_t>(a.resid) & 31) == 0;
-    if (a.epi == EPI_SWIGLU) ok32 = ok32 && (reinterpret_cast<uintptr_t>(a.gu) & 31) == 0;
+    if (a.epi == EPI_SWIGLU || a.epi == EPI_SWIGLU_BWD) ok32 = ok32 && (reinterpret_cast<uintptr_t>(a.gu) & 31) == 0;
     p.wide_store = ok32 ? 1 : 0;
   }
   p.qk_r = a.qk_r; p.qk_gain_q = a.qk_gain_q; p.qk_gain_k = a.qk_gain_k; p.n_q_heads = a.n_q_heads; p.qk_eps = a.qk_eps;
@@ -1201,10 +1292,10 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
   return launch_pdl(kern, grid, GEMM_THREADS, C::SMEM_BYTES, stream, tmA, tmB, p);
 }
 
-template <bool A_MN, bool B_MN, bool CE = false>
+template <bool A_MN, bool B_MN, int MODE = 0>
 cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
   using C = PairCfg;
-  auto kern = gemm_tc_pair_kernel<A_MN, B_MN, CE>;
+  auto kern = gemm_tc_pair_kernel<A_MN, B_MN, MODE>;
   static unsigned long long smem_set = 0;
   cudaError_t e0 = ensure_dynamic_smem(kern, C::SMEM_BYTES, smem_set);
   if (e0 != cudaSuccess) return e0;
@@ -1223,7 +1314,7 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
     const int m = f32out ? 7 : 15;  // elements per 32 bytes, minus one
     bool ok32 = (reinterpret_cast<uintptr_t>(a.C) & 31) == 0 && (a.ldc & m) == 0 && (a.N & m) == 0;
     if (a.epi == EPI_BF16_RESID) ok32 = ok32 && (reinterpret_cast<uintptr_t>(a.resid) & 31) == 0;
-    if (a.epi == EPI_SWIGLU) ok32 = ok32 && (reinterpret_cast<uintptr_t>(a.gu) & 31) == 0;
+    if (a.epi == EPI_SWIGLU || a.epi == EPI_SWIGLU_BWD) ok32 = ok32 && (reinterpret_cast<uintptr_t>(a.gu) & 31) == 0;
     p.wide_store = ok32 ? 1 : 0;
   }
   p.qk_r = a.qk_r; p.qk_gain_q = a.qk_gain_q; p.qk_gain_k = a.qk_gain_k; p.n_q_heads = a.n_q_heads; p.qk_eps = a.qk_eps;
@@ -1253,9 +1344,9 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
   // balanced schedule: a last wave that would keep at most half of the pairs busy is divided along K
   p.balanced = 0; p.sw_first = tiles; p.sw_parts = 1; p.sw_kpb = kblocks; p.flags = flags; p.slots = data;
   const int left = tiles % max_pairs;
-  p.ce_mode = CE ? a.ce_mode : 0; p.ce_tiles = a.ce_tiles; p.ce_part = a.ce_part; p.ce_zy = a.ce_zy; p.ce_lse = a.ce_lse;
+  p.ce_mode = MODE == 1 ? a.ce_mode : 0; p.ce_tiles = a.ce_tiles; p.ce_part = a.ce_part; p.ce_zy = a.ce_zy; p.ce_lse = a.ce_lse;
   p.ce_labels = a.ce_labels; p.ce_sc = a.ce_scalars; p.ce_scale = a.ce_scale;
-  if (!CE && g_gemm_balanced && ksplit == 1 && data && tiles > max_pairs && left > 0 && max_pairs <= 256 &&
+  if (MODE != 1 && g_gemm_balanced && ksplit == 1 && data && tiles > max_pairs && left > 0 && max_pairs <= 256 &&
       (size_t)max_pairs * SLOT_FLOATS * sizeof(float) <= data_bytes) {
     int parts = max_pairs / left;
     // The pair with part 0 adds the other parts' tiles while its next tile's main loop runs; the longer that loop (K),
@@ -1342,6 +1433,9 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream) {
                             a.rope_cols % a.head_dim || a.N % a.head_dim))
     return cudaErrorInvalidValue;
   if (a.epi == EPI_SWIGLU && (!a.gu || a.d_ffn <= 0 || a.d_ffn % 16 || a.N != 2 * a.d_ffn)) return cudaErrorInvalidValue;
+  if (a.epi == EPI_SWIGLU_BWD && (!a.gu || a.d_ffn <= 0 || a.d_ffn % 16 || a.N != a.d_ffn || a.ldc < 2LL * a.d_ffn ||
+                                  (reinterpret_cast<uintptr_t>(a.gu) & 15)))
+    return cudaErrorInvalidValue;
   // 128 x 256 tiles move 96 B of operands per tensor-core cycle through shared memory, 128 x 128 tiles 128 B: the
   // wide tile is faster even when it leaves SMs idle (measured), so the narrow one only serves N <= 128
   const bool wide = g_gemm_force_bn ? g_gemm_force_bn == 256 : a.N > 128;
@@ -1352,7 +1446,13 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream) {
       return cudaErrorInvalidValue;
     if (a.ce_mode == 1 && (!a.ce_part || !a.ce_zy)) return cudaErrorInvalidValue;
     if (a.ce_mode == 2 && (!a.ce_lse || !a.ce_scalars || a.epi != EPI_BF16)) return cudaErrorInvalidValue;
-    return launch_pair_variant<false, false, true>(a, stream);
+    return launch_pair_variant<false, false, 1>(a, stream);
+  }
+  if (a.epi == EPI_SWIGLU_BWD) {
+    // instantiations of their own (the epilogue's register needs stay out of the other kernels); data-gradient layout only
+    if (a.a_mn || !a.b_mn || a.adam) return cudaErrorInvalidValue;
+    if (g_gemm_pairs && !g_gemm_force_bn && a.M >= 256 && a.N >= 256) return launch_pair_variant<false, true, 2>(a, stream);
+    return wide ? launch_variant<256, false, true, 2>(a, stream) : launch_variant<128, false, true, 2>(a, stream);
   }
   if (g_gemm_pairs && !g_gemm_force_bn && a.M >= 256 && a.N >= 256) {
     if (!a.a_mn && !a.b_mn) return launch_pair_variant<false, false>(a, stream);

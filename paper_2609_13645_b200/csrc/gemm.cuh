@@ -13,7 +13,9 @@ enum GemmEpilogue : int {
   EPI_F32 = 2,         // C fp32 = acc
   EPI_F32_ACC = 3,     // C fp32 += acc
   EPI_ROPE = 4,        // C bf16 = R(rope(acc)) for columns < rope_cols (heads of head_dim columns), R(acc) beyond
-  EPI_SWIGLU = 5       // acc columns alternate 16 gate / 16 up: writes gate|up to gu bf16 [M, 2f] and a = R(silu(G) U) to C [M, f]
+  EPI_SWIGLU = 5,      // acc columns alternate 16 gate / 16 up: writes gate|up to gu bf16 [M, 2f] and a = R(silu(G) U) to C [M, f]
+  EPI_SWIGLU_BWD = 6   // acc = d_a [M, f] (N = f = d_ffn): reads gate|up from gu [M, 2f] and writes bf16 d_gate, d_up to
+                       // C [M, 2f] in the alternating 16 / 16 column layout; d_a = R(alpha acc) is never stored
 };
 
 // Weight-gradient GEMMs (EPI_F32 / EPI_F32_ACC) can hand the finished gradient straight to AdamW instead of storing it:
@@ -59,7 +61,7 @@ struct GemmArgs {
   const bf16* qk_gain_k = nullptr;
   int n_q_heads = 0;
   float qk_eps = 0.f;
-  // EPI_SWIGLU
+  // EPI_SWIGLU (written), EPI_SWIGLU_BWD (read)
   bf16* gu = nullptr;  // [M, 2f] gate | up
   int d_ffn = 0;
   int* err = nullptr;  // device status word

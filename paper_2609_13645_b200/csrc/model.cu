@@ -125,6 +125,7 @@ struct ft_model {
 
   // AdamW inside the weight-gradient GEMM epilogues (clipping off): the train step then never stores those gradients
   bool fused_update = true;   // policy switch (ft_set_fused_update)
+  bool fused_swiglu_bwd = true;  // policy switch (ft_set_fused_swiglu_bwd): SwiGLU backward in the down projection's data-gradient epilogue
   bool fusing = false;        // true while a step that fuses is being enqueued
   int fuse_idx = 0;           // next slot region of fuse_sq
   float* fuse_sq = nullptr;   // partial sums of the squared gradient norm: [4L+1][kAdamFuseSlots] + 2 x [kSqnormBlocks]
@@ -500,12 +501,17 @@ ft_status wait_wgrad(ft_model* m, int k) {
 
 // dX = dY W (data gradient) and dW = dY^T X (weight gradient, slot k of the layer's four)
 // alpha: factor the branch output carried into the residual stream (its gradient is alpha * dY, never rounded)
+// swiglu_gu: when given, X is the SwiGLU output a = silu(G) U of the gate|up tensor swiglu_gu [T, 2 n_in], dX is not
+// stored, and the data-gradient epilogue writes d_gate, d_up to swiglu_dgu [T, 2 n_in] (alternating 16 / 16 columns)
 ft_status linear_backward(ft_model* m, const bf16* dY, const bf16* X, int wi, bf16* dX, int T, int n_out, int n_in, int k,
-                          float alpha = 1.0f) {
+                          float alpha = 1.0f, const bf16* swiglu_gu = nullptr, bf16* swiglu_dgu = nullptr) {
   {
     GemmArgs g = gemm_base(m);
     g.A = dY; g.lda = n_out; g.B = m->wb(wi); g.b_mn = 1; g.ldb = n_in; g.C = dX; g.ldc = n_in;
     g.M = T; g.N = n_in; g.K = n_out; g.epi = EPI_BF16; g.alpha = alpha;
+    if (swiglu_gu != nullptr) {
+      g.epi = EPI_SWIGLU_BWD; g.C = swiglu_dgu; g.ldc = 2LL * n_in; g.gu = const_cast<bf16*>(swiglu_gu); g.d_ffn = n_in;
+    }
     FT_GEMM(g);
   }
   {
@@ -535,10 +541,18 @@ ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
   LayerTaps* tp = m->cfg.debug_taps ? &m->taps[l] : nullptr;
   // m->dxA holds d_x_out
   if (tp) { ft_status s = copy_tap(m, tp->d_x_out, m->dxA, (size_t)T * h); if (s) return s; }
-  ft_status s = linear_backward(m, m->dxA, a.a, m->idx_layer(l, 5), m->d_a, T, h, f, 0, m->cfg.resid_scale);
-  if (s) return s;
-  if ((s = wait_wgrad(m, 1))) return s;  // the previous layer's gate/up weight gradient still reads d_gu
-  FT_LAUNCH(FT_PROF_ELEMENTWISE, 10.0 * T * f, swiglu_bwd(m->d_a, a.gu, m->d_gu, T, f, st));
+  ft_status s;
+  if (m->fused_swiglu_bwd && !tp) {
+    // d_a stays in the data-gradient GEMM's accumulators: its epilogue reads gate | up and writes d_gate | d_up
+    if ((s = wait_wgrad(m, 1))) return s;  // the previous layer's gate/up weight gradient still reads d_gu
+    s = linear_backward(m, m->dxA, a.a, m->idx_layer(l, 5), nullptr, T, h, f, 0, m->cfg.resid_scale, a.gu, m->d_gu);
+    if (s) return s;
+  } else {
+    s = linear_backward(m, m->dxA, a.a, m->idx_layer(l, 5), m->d_a, T, h, f, 0, m->cfg.resid_scale);
+    if (s) return s;
+    if ((s = wait_wgrad(m, 1))) return s;  // the previous layer's gate/up weight gradient still reads d_gu
+    FT_LAUNCH(FT_PROF_ELEMENTWISE, 10.0 * T * f, swiglu_bwd(m->d_a, a.gu, m->d_gu, T, f, st));
+  }
   s = linear_backward(m, m->d_gu, a.h2, m->idx_layer(l, 4), m->d_h, T, 2 * f, h, 1);
   if (s) return s;
   if (tp) {
@@ -1050,6 +1064,13 @@ ft_status ft_set_attention_stored_ds(ft_model* m, int32_t enable) {
 ft_status ft_set_streaming_ce(ft_model* m, int32_t enable) {
   if (!m) return FT_EINVAL;
   m->streaming_ce = enable != 0;
+  if (m->graph_exec) { cudaGraphExecDestroy(m->graph_exec); m->graph_exec = nullptr; }  // captured with the old setting
+  return FT_OK;
+}
+
+ft_status ft_set_fused_swiglu_bwd(ft_model* m, int32_t enable) {
+  if (!m) return FT_EINVAL;
+  m->fused_swiglu_bwd = enable != 0;
   if (m->graph_exec) { cudaGraphExecDestroy(m->graph_exec); m->graph_exec = nullptr; }  // captured with the old setting
   return FT_OK;
 }

@@ -58,9 +58,14 @@ def test_one_rank_data_parallel_steps_equal_plain_steps(one_rank_group, clip, ti
     assert len(dp.buckets) == ocfg.n_layers + (2 if tied else 3) + (1 if mtp else 0)
     got = [dp.step(t, l) for t, l in batches]
     torch.cuda.synchronize()
-    for (l0, g0), (l1, g1) in zip(ref, got):
-        assert l0 == l1
-        assert abs(g0 - g1) <= 2e-6 * g0
+    for i, ((l0, g0), (l1, g1)) in enumerate(zip(ref, got)):
+        if clip > 0 and i > 0:
+            # after a clipped update the two runs hold parameters that differ in last bits (see below), and so do
+            # their next losses and norms
+            assert abs(l0 - l1) <= 1e-5 * abs(l0) and abs(g0 - g1) <= 1e-4 * g0
+        else:
+            assert l0 == l1
+            assert abs(g0 - g1) <= 2e-6 * g0
     for name, _ in model.params:
         for kind in (B.KIND_MASTER, B.KIND_ADAM_M, B.KIND_ADAM_V, B.KIND_BF16):
             a, b = plain.get_param(name, kind), model.get_param(name, kind)
@@ -75,7 +80,7 @@ def test_one_rank_data_parallel_steps_equal_plain_steps(one_rank_group, clip, ti
                 else:
                     tol = 0.05 * ocfg.lr * len(batches)
                     if kind == B.KIND_BF16:  # a master that moved by less than that can still cross a bf16 boundary: one ulp
-                        tol = max(tol, 2.0 ** -8 * float(np.max(np.abs(a))))
+                        tol = max(tol, 2.0 ** -7 * float(np.max(np.abs(a))))  # a bf16 ulp is up to 2^-7 of the value
                     assert np.max(np.abs(a - b)) <= tol, (name, kind)
             else:
                 assert np.array_equal(a, b), (name, kind)

@@ -505,6 +505,48 @@ def test_adamw_inside_the_weight_gradient_epilogue_equals_the_separate_optimizer
     mu.close()
 
 
+@pytest.mark.parametrize("shape", ["c1", "ragged_ffn", "one_cta", "balanced", "mup_recompute"])
+def test_swiglu_backward_inside_the_data_gradient_epilogue_changes_no_bit(shape):
+    """By default the down projection's data-gradient GEMM never stores d_a: its epilogue rounds the accumulator to bf16,
+    reads gate and up, and writes d_gate | d_up.  Same element function on the same rounded value as the separate
+    elementwise pass, so losses, norms and the whole optimizer state must equal that path bit for bit.  Shapes: the
+    CTA-pair kernel; an ffn width whose last 32-column chunk is half empty; few tokens (single-CTA kernel); a tile count
+    that divides the last wave along K (partials completed before the epilogue); muP factors with recomputation."""
+    from paper_2609_13645_b200 import binding as B
+    kw, recompute = {}, 0
+    if shape == "c1":
+        ocfg, _ = _c1()
+        Bsz, S = 2, 128
+    elif shape == "ragged_ffn":
+        ocfg = oracle_config(n_layers=2, d_model=256, n_heads=4, n_kv_heads=2, head_dim=64, d_ffn=688, vocab=1024, max_grad_norm=0.5)
+        Bsz, S = 3, 160
+    elif shape == "one_cta":
+        ocfg = oracle_config(n_layers=2, d_model=256, n_heads=4, n_kv_heads=2, head_dim=64, d_ffn=1040, vocab=1024)
+        Bsz, S = 1, 136
+    elif shape == "balanced":  # 8 x 10 = 80 tiles of d_a on 74 pairs: the last 6 are divided along K
+        ocfg = oracle_config(n_layers=1, d_model=1280, n_heads=10, n_kv_heads=2, head_dim=128, d_ffn=2560, vocab=2048)
+        Bsz, S = 2, 1024
+    else:
+        ocfg = oracle_config(n_layers=3, d_model=512, n_heads=4, n_kv_heads=2, head_dim=128, d_ffn=1024, vocab=2048,
+                             emb_scale=12.0, resid_scale=0.7, logit_scale=0.5, max_grad_norm=1.0)
+        Bsz, S, recompute = 2, 512, 1
+    runs = []
+    for fused in (True, False):
+        model = B.Model(lib_config(B, ocfg, Bsz, S, recompute=recompute), seed=9)
+        model.set_fused_swiglu_bwd(fused)
+        out = []
+        for s in range(3):
+            tok, lab = SI.batch(ocfg.vocab, Bsz, S, "zipf", step=s)
+            out.append(model.train_step(to_dev(tok), to_dev(lab)))
+        runs.append((model, out))
+    (mf, lf), (mu, lu) = runs
+    assert lf == lu
+    for a, b in zip(_state_bits(mf), _state_bits(mu)):
+        assert np.array_equal(a, b)
+    mf.close()
+    mu.close()
+
+
 @pytest.mark.parametrize("recompute", [0, 1])
 def test_weight_gradients_on_the_second_stream_change_no_bit(recompute):
     """The weight-gradient GEMMs run on a second stream, concurrent with the rest of the backward pass; events order
