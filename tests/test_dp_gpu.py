@@ -74,11 +74,14 @@ def test_one_rank_data_parallel_steps_equal_plain_steps(one_rank_group, clip, ti
                 # to rounding; a master moves by lr * g / (|g| + eps)-like terms, which turn that last bit into a visible
                 # fraction of one update where |g| is of the order of eps (rows of the table few tokens touch).
                 # From the second step on the two runs hold parameters that differ in such last bits, and a bf16 step
-                # amplifies that to its rounding noise floor: the moments then agree to 1e-3, not to 1e-7.
+                # amplifies that to its rounding noise floor: the moments then agree to about 1e-3 (measured up to 1.1e-3 on
+                # a gain whose gradient is a sum of cancelling terms), not to 1e-7.  A wrong slice or a missed update is O(1).
                 if kind in (B.KIND_ADAM_M, B.KIND_ADAM_V):
-                    assert rel_l2(b, a) < 1e-3, (name, kind)
+                    assert rel_l2(b, a) < 5e-3, (name, kind)
                 else:
-                    tol = 0.05 * ocfg.lr * len(batches)
+                    # measured up to 0.08 lr per step on elements whose gradient is tiny; a skipped or doubled update of
+                    # one step is a whole lr (|m / sqrt(v)| is about 1 in the first steps)
+                    tol = 0.2 * ocfg.lr * len(batches)
                     if kind == B.KIND_BF16:  # a master that moved by less than that can still cross a bf16 boundary: one ulp
                         tol = max(tol, 2.0 ** -7 * float(np.max(np.abs(a))))  # a bf16 ulp is up to 2^-7 of the value
                     assert np.max(np.abs(a - b)) <= tol, (name, kind)
