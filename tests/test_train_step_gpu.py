@@ -104,6 +104,23 @@ def test_gqa_head_dim_128_two_layers_with_ignored_labels():
     _check_step(ocfg, tok, lab, params)
 
 
+@pytest.mark.parametrize("shape,recompute", [("c1", 0), ("gqa_ragged_ffn", 0), ("gqa_ragged_ffn", 1)])
+def test_default_path_without_taps_matches_oracle_on_loss_every_gradient_and_master(shape, recompute):
+    """Without debug taps the step takes the paths a training run takes (SwiGLU backward inside the data-gradient
+    epilogue, no stored d_a); loss, every parameter gradient and the updated masters against the oracle."""
+    if shape == "c1":
+        ocfg, _ = _c1()
+        params = D.init_params(ocfg, SI.WEIGHT_SEED)
+        tok, lab = SI.workload_batch("c1_tiny")
+    else:
+        ocfg = _small_gqa()
+        params = D.init_params(ocfg, 99)
+        tok, lab = SI.batch(ocfg.vocab, 2, 200, "zipf", seed=5)
+        lab = lab.copy()
+        lab[1, -5:] = -1
+    _check_step(ocfg, tok, lab, params, debug=False, recompute=recompute)
+
+
 @pytest.mark.parametrize("variant", ["mtp", "mtp+tied+qknorm+mup", "mtp+ragged+streaming"])
 def test_mtp_head_step_matches_oracle_on_loss_every_gradient_and_master(variant):
     """The one-layer MTP (Eagle) head of the paper's 1B configuration: the normalised last hidden state and the normalised
