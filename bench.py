@@ -227,6 +227,7 @@ def run_cuda(args):
     model.set_graph(not args.no_graph)
     model.set_overlap(not args.no_overlap)
     model.set_fused_update(not args.no_fused_update)
+    model.set_fused_swiglu_bwd(not args.no_fused_swiglu_bwd)
     model.set_streaming_ce(args.streaming_ce)
     n_batches = args.steps + args.warmup
     host_batches = [SI.batch(w["vocab"], Bsz, S, w["dist"], seed=SI.DATA_SEED + 1000 * rank, step=i)
@@ -422,6 +423,8 @@ def main():
                     help="model variant on the workload's shape (default: the plain decoder the metric is quoted on)")
     ap.add_argument("--no-overlap", action="store_true", help="ablation: weight-gradient GEMMs on the main stream")
     ap.add_argument("--no-fused-update", action="store_true", help="ablation: separate AdamW pass over all parameters")
+    ap.add_argument("--no-fused-swiglu-bwd", action="store_true",
+                    help="ablation: SwiGLU backward as a kernel of its own instead of the data-gradient GEMM's epilogue")
     ap.add_argument("--streaming-ce", action="store_true", help="cross-entropy inside the logits GEMM's epilogues (GEMM runs twice)")
     args = ap.parse_args()
     if args.impl == "reference":
