@@ -234,10 +234,10 @@ def test_head_loss_and_weight_gradients_on_sampled_entries(run):
 
 @pytest.mark.parametrize("name", ["c3_1b", "c4_8b_slice"])
 def test_bench_launch_configuration_equals_the_plain_step_bit_for_bit(name):
-    """bench.py times the step as a replayed CUDA graph with AdamW inside the weight-gradient epilogues and the weight
-    gradients on a second stream.  At full size (16 layers at c3; recomputation at c4, where all layers share one
+    """bench.py times the step as a replayed CUDA graph with AdamW inside the weight-gradient epilogues, the SwiGLU
+    backward inside the down projection's data-gradient epilogue and the weight gradients on a second stream.  At full size (16 layers at c3; recomputation at c4, where all layers share one
     activation slot) that configuration must leave the same bits as the plain step (one stream, separate optimizer
-    pass, launch by launch), whose kernels the sampled-parity tests above tie to the oracle."""
+    and SwiGLU-backward passes, launch by launch), whose kernels the sampled-parity tests above tie to the oracle."""
     import gc
     from paper_2609_13645_b200 import binding as B
     w = SI.WORKLOADS[name]
@@ -262,6 +262,7 @@ def test_bench_launch_configuration_equals_the_plain_step_bit_for_bit(name):
     plain = B.Model(cfg, seed=SI.WEIGHT_SEED)
     plain.set_fused_update(False)
     plain.set_overlap(False)
+    plain.set_fused_swiglu_bwd(False)  # the separate SwiGLU-backward pass, as the tap runs above have it
     l_plain = [plain.train_step(to_dev(t), to_dev(l))[0] for t, l in batches]
     s_plain = state(plain)
     plain.close()
