@@ -232,7 +232,7 @@ def test_head_loss_and_weight_gradients_on_sampled_entries(run):
     assert rel_l2(gH[vv], dzc.T @ hF_all) < 1e-3
 
 
-@pytest.mark.parametrize("name", ["c3_1b", "c4_8b_slice"])
+@pytest.mark.parametrize("name", ["c2_124m", "c3_1b", "c4_8b_slice", "c5_1b_long"])
 def test_bench_launch_configuration_equals_the_plain_step_bit_for_bit(name):
     """bench.py times the step as a replayed CUDA graph with AdamW inside the weight-gradient epilogues, the SwiGLU
     backward inside the down projection's data-gradient epilogue and the weight gradients on a second stream.  At full size (16 layers at c3; recomputation at c4, where all layers share one
