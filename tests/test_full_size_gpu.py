@@ -232,7 +232,16 @@ def test_head_loss_and_weight_gradients_on_sampled_entries(run):
     assert rel_l2(gH[vv], dzc.T @ hF_all) < 1e-3
 
 
-@pytest.mark.parametrize("name", ["c2_124m", "c3_1b", "c4_8b_slice", "c5_1b_long"])
+# the variants bench.py offers on the c3_1b shape (same factors as its --variant switch)
+_C3_VARIANTS = {
+    "mup_mtp": dict(emb_scale=12.0, resid_scale=1.4 / 16 ** 0.5, logit_scale=256.0 / 2048, mtp=True, mtp_weight=1.0),
+    "qknorm_tied": dict(qk_norm=True, tie_embeddings=True),
+    "mup_tied": dict(emb_scale=12.0, resid_scale=1.4 / 16 ** 0.5, logit_scale=256.0 / 2048, tie_embeddings=True),
+}
+
+
+@pytest.mark.parametrize("name", ["c2_124m", "c3_1b", "c4_8b_slice", "c5_1b_long", "c3_1b+mup_mtp", "c3_1b+qknorm_tied",
+                                  "c3_1b+mup_tied"])
 def test_bench_launch_configuration_equals_the_plain_step_bit_for_bit(name):
     """bench.py times the step as a replayed CUDA graph with AdamW inside the weight-gradient epilogues, the SwiGLU
     backward inside the down projection's data-gradient epilogue and the weight gradients on a second stream.  At full size (16 layers at c3; recomputation at c4, where all layers share one
@@ -240,16 +249,23 @@ def test_bench_launch_configuration_equals_the_plain_step_bit_for_bit(name):
     and SwiGLU-backward passes, launch by launch), whose kernels the sampled-parity tests above tie to the oracle."""
     import gc
     from paper_2609_13645_b200 import binding as B
+    name, _, variant = name.partition("+")
     w = SI.WORKLOADS[name]
-    ocfg = oracle_config(**{k: w[k] for k in SI.MODEL_KEYS})
+    ocfg = oracle_config(**{k: w[k] for k in SI.MODEL_KEYS}, **_C3_VARIANTS.get(variant, {}))
     cfg = lib_config(B, ocfg, w["batch"], w["seq"], recompute=w["recompute"])
     gc.collect()
     torch.cuda.empty_cache()
     if torch.cuda.mem_get_info()[0] < B.workspace_bytes(cfg) + (4 << 30):
         pytest.skip("not enough free device memory")
     L = ocfg.n_layers
-    names = ["embed", "lm_head", "norm_f"] + [f"layers.{l}.{t}" for l in (0, L // 2, L - 1)
-                                              for t in ("wqkv", "wo", "wgu", "wd", "norm1", "norm2")]
+    names = ["embed", "norm_f"] + [f"layers.{l}.{t}" for l in (0, L // 2, L - 1)
+                                   for t in ("wqkv", "wo", "wgu", "wd", "norm1", "norm2")]
+    if not ocfg.tie_embeddings:
+        names.append("lm_head")
+    if ocfg.qk_norm:
+        names += ["layers.0.q_norm", f"layers.{L - 1}.k_norm"]
+    if ocfg.mtp:
+        names += ["mtp.proj_h", "mtp.proj_e", "mtp.norm_e", "mtp.layer.wgu", "mtp.layer.wqkv", "mtp.norm_f"]
     batches = [SI.batch(ocfg.vocab, w["batch"], w["seq"], w["dist"], step=s) for s in range(3)]
 
     def state(model):
