@@ -240,6 +240,25 @@ _C3_VARIANTS = {
 }
 
 
+@pytest.mark.parametrize("variant", sorted(_C3_VARIANTS))
+def test_variant_loss_at_initialisation_at_full_size(variant):
+    """A property that holds at any size: at initialisation hF has RMS 1 and the head's rows are N(0, 0.02^2), so every
+    logit is N(0, (logit_scale 0.02)^2 h) and each cross-entropy is ln V + sigma^2 / 2 up to the sample offset of the
+    label term (a few tenths at logit_scale 1, an eighth of that with the muP factor); with the MTP head the loss is
+    the sum of two such terms."""
+    from paper_2609_13645_b200 import binding as B
+    w = SI.WORKLOADS["c3_1b"]
+    ocfg = oracle_config(**{k: w[k] for k in SI.MODEL_KEYS}, **_C3_VARIANTS[variant])
+    model = B.Model(lib_config(B, ocfg, w["batch"], w["seq"]), seed=SI.WEIGHT_SEED)
+    tok, lab = SI.workload_batch("c3_1b")
+    loss = model.forward_loss(to_dev(tok), to_dev(lab))
+    model.close()
+    model.workspace = None
+    one = math.log(ocfg.vocab) + 0.5 * (float(ocfg.logit_scale or 1.0) * 0.02) ** 2 * ocfg.d_model
+    expect = one * (1.0 + (float(ocfg.mtp_weight) if ocfg.mtp else 0.0))
+    assert abs(loss - expect) < (0.1 if ocfg.logit_scale not in (0.0, 1.0) else 0.4), (loss, expect)
+
+
 @pytest.mark.parametrize("name", ["c2_124m", "c3_1b", "c4_8b_slice", "c5_1b_long", "c3_1b+mup_mtp", "c3_1b+qknorm_tied",
                                   "c3_1b+mup_tied"])
 def test_bench_launch_configuration_equals_the_plain_step_bit_for_bit(name):
