@@ -8,8 +8,8 @@ One "step" is one pass of the whole hot path over one synthetic batch.  Prints O
 host-buffer entry point, a roofline object for the dominant kernel class (the tcgen05 GEMMs) taken from CUDA
 events recorded around every launch inside the timed region, and the CPU oracle timed on a bounded sample.
 
-With --gpus N > 1 (launched by torch.distributed.run) every rank trains an independent replica on its own
-batch stream: the path is single-GPU by design, so there is no data-path collective; NCCL only carries the
+With --gpus N > 1 (launched by torch.distributed.run, or by this script itself when no launcher set WORLD_SIZE) every
+rank trains an independent replica on its own batch stream: the path is single-GPU by design, so there is no data-path collective; NCCL only carries the
 barrier and the max-over-ranks of the device time.
 """
 from __future__ import annotations
@@ -409,6 +409,18 @@ def run_dp(args):
     dist.destroy_process_group()
 
 
+def relaunch_under_torchrun(n: int) -> int:
+    """`python bench.py --gpus N` run plainly (no launcher in the environment): start N ranks of this same command line
+    under torch.distributed.run on this node and hand back its exit code.  Rank 0 of the child job prints the JSON line."""
+    import socket
+    with socket.socket() as sock:  # a free port for the rendezvous
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -427,6 +439,8 @@ def main():
                     help="ablation: SwiGLU backward as a kernel of its own instead of the data-gradient GEMM's epilogue")
     ap.add_argument("--streaming-ce", action="store_true", help="cross-entropy inside the logits GEMM's epilogues (GEMM runs twice)")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return relaunch_under_torchrun(args.gpus)
     if args.impl == "reference":
         return run_reference(args)
     if args.dp:

@@ -49,13 +49,24 @@ typedef struct {
   int32_t qk_norm;                /* 1: per-head RMSNorm of q and k before the rotation (Qwen3 column of the same appendix);
                                      adds the gains layers.{l}.q_norm and layers.{l}.k_norm [head_dim], eps = rms_eps */
   int32_t mtp;                    /* 1: one-layer multi-token-prediction (Eagle) head (same appendix, row "MTP / Eagle head:
-                                     On (1 layer)"; it "repeats the backbone layer's attention, projection, and FFN plus a
-                                     second output head"): h' = R(R(hn Wh^T) + en We^T) from the normalised last hidden
+                                     On (1 layer)"; the FLOP appendix of the Ascend models counts it as one more backbone
+                                     layer plus one more output head): h' = R(R(hn Wh^T) + en We^T) from the normalised last hidden
                                      state hn and the normalised embedding en of the NEXT token, one more decoder layer, its
                                      own final norm, the backbone's output head, trained on the token after next.
                                      Parameters mtp.norm_h, mtp.norm_e [h], mtp.proj_h, mtp.proj_e [h, h], mtp.layer.*
                                      (a layer's set), mtp.norm_f [h]. */
   float mtp_weight;               /* loss = backbone loss + mtp_weight * (mean cross-entropy of the MTP head); 0 means 1 */
+  /* ZeRO-1 sharding of the optimizer state (Section "Sources of the Speedup": "ZeRO-1 optimizer sharding"; appendix
+   * "Framework-Level Optimization Trajectory", step "ZeRO-1 sharded optimizer").  dp_world in {2, 4, 8, 16, 32}: the
+   * workspace holds fp32 masters and both Adam moments only for this rank's slice of every gradient bucket (slice
+   * dp_rank of dp_world equal parts, see ft_dp_bucket), i.e. 12 / dp_world bytes per parameter instead of 12; gradients
+   * and the bf16 compute copy stay whole.  Such a model steps through the ft_dp_* calls only (ft_train_step and
+   * ft_apply_update return FT_EINVAL); ft_dp_update_range takes ranges inside the rank's own slices; ft_get_param of a
+   * master or moment returns the owned elements and 0 elsewhere (the ranks' results add up to the whole tensor),
+   * ft_set_param stores the owned elements of the whole tensor it is given (and, for a master, rewrites the bf16 copy of
+   * the whole tensor); both use the tensor's span of the gradient arena as staging, so gradients are lost.  Every rank
+   * draws the same initial weights from the seed.  0 or 1: unsharded (the default). */
+  int32_t dp_world, dp_rank;
 } ft_config;
 
 typedef struct ft_model ft_model;
@@ -66,22 +77,33 @@ typedef enum {
 
 typedef enum { FT_MASTER_F32 = 0, FT_COMPUTE_BF16 = 1, FT_ADAM_M_F32 = 2, FT_ADAM_V_F32 = 3, FT_GRAD_F32 = 4 } ft_kind;
 
-/* Bytes of device workspace a model of this config needs (0 if the config is invalid). */
+/* Bytes of device workspace a model of this config needs (0 if the config is invalid).  The workspace holds what the
+ * paper's forged engine keeps resident for one data-parallel rank (Section "Sources of the Speedup"; appendix
+ * "Why the Engine Is Faster, Mechanism by Mechanism"): fp32 masters, both Adam moments, fp32 gradients and the bf16
+ * compute copy as five identically laid out flat arenas, every layer's saved activations (or, with recompute, one
+ * layer's plus the layer inputs), the backward scratch and one chunk of logits.  Host-only call. */
 size_t ft_workspace_bytes(const ft_config* cfg);
 
-/* Creates a model inside dev_workspace (256-byte aligned, >= ft_workspace_bytes) on the current CUDA
- * device.  Masters are drawn from a counter-based N(0, 0.02^2) generator keyed by (seed, tensor index,
- * element index), gains are 1, Adam moments 0, step 0.  cuda_stream is a cudaStream_t (NULL = default). */
+/* init_model(config, seed) of the problem statement: creates a model of the architecture tables (appendix "Model
+ * Architectures") inside dev_workspace (256-byte aligned, >= ft_workspace_bytes) on the current CUDA device.  The
+ * paper prints no initialiser; every matrix is drawn from N(0, 0.02^2) by a counter-based generator keyed by (seed,
+ * tensor index, element index) (splitmix64 -> two 24-bit uniforms -> Box-Muller in double), gains are 1, Adam moments
+ * 0, step 0, the bf16 copy is the rounded master.  cuda_stream is a cudaStream_t (NULL = default stream); the caller
+ * keeps ownership of the workspace and must keep it alive until ft_destroy.  Returns FT_EINVAL for a bad config or a
+ * misaligned workspace, FT_ENOMEM when bytes is too small (*out stays NULL), FT_ECUDA on a device that is not sm_100. */
 ft_status ft_init_model(const ft_config* cfg, uint64_t seed, void* dev_workspace, size_t bytes,
                         void* cuda_stream, ft_model** out);
 
-/* One step: forward, loss, backward, global gradient norm, AdamW (paper: train step of the forged engine).
+/* train_step(tokens, labels) -> loss: forward, loss, backward, global gradient norm, AdamW with fp32 masters and the
+ * bf16 write-back (the train step of the forged engine: Section "Sources of the Speedup"; optimizer arithmetic from the fused clip + Adam +
+ * cast listing and the device-side clip listing of the appendix "Why the Engine Is Faster, Mechanism by Mechanism").
  * dev_tokens, dev_labels: int32 [B, S] on the device; labels < 0 do not count in the mean loss.
  * host_loss / host_gnorm: optional host floats; if either is non-NULL the call synchronises the stream. */
 ft_status ft_train_step(ft_model* m, const int32_t* dev_tokens, const int32_t* dev_labels, int32_t B, int32_t S,
                         float* host_loss, float* host_gnorm);
 
-/* Optimizer-tail fusion (Section 5.3's fused clip + Adam, taken one step further): with gradient clipping off
+/* Optimizer-tail fusion (Section "Sources of the Speedup", vertical integration: clip + Adam + cast as one pass;
+ * taken one step further here): with gradient clipping off
  * (max_grad_norm <= 0) the update of a weight matrix does not depend on the global norm, so ft_train_step applies
  * AdamW inside the epilogue of the weight-gradient GEMM (or of its split-K reduction): the finished fp32 gradient
  * never goes to memory, and the separate optimizer pass shrinks to the embedding table and the gains.  The update
@@ -96,8 +118,8 @@ ft_status ft_set_fused_update(ft_model* m, int32_t enable);
  * host in double precision and copies them (synchronises the model's stream).  The factors are model data, like weights. */
 ft_status ft_set_rope_scaling(ft_model* m, const float* host_factors, float mscale);
 
-/* Weight-gradient overlap: nothing later in the backward pass depends on a layer's weight gradients (Section 4.3's
- * fused dgrad + wgrad observation, turned into concurrency), so the library enqueues those GEMMs on a second stream
+/* Weight-gradient overlap: nothing later in the backward pass depends on a layer's weight gradients (appendix
+ * "Optimization Catalog": "Backward-pass fusion" and the auxiliary streams that carry wgrad, turned into concurrency), so the library enqueues those GEMMs on a second stream
  * of its own, ordered by events against the kernels that produce their inputs and against the kernels that later
  * overwrite the buffers they read; they occupy the SMs that the main chain leaves idle in the last wave of each
  * kernel.  Results do not change by a bit (every kernel keeps its own fixed summation order and its own scratch).
@@ -138,7 +160,8 @@ int64_t ft_graph_replays(const ft_model* m);
 ft_status ft_train_step_host(ft_model* m, const int32_t* host_tokens, const int32_t* host_labels, int32_t B,
                              int32_t S, float* host_loss, float* host_gnorm);
 
-/* ---- Data-parallel hooks (Section 5.2, "bucketed reduce-scatter overlapped with backward", "ZeRO-1 sharded optimizer,
+/* ---- Data-parallel hooks (Section "Sources of the Speedup" and appendix "Framework-Level Optimization Trajectory":
+ * "bucketed reduce-scatter overlapped with backward", "ZeRO-1 sharded optimizer,
  * per-bucket all-gather interleaved with Adam").  The library itself holds no communicator: these calls expose what a
  * data-parallel driver needs, and paper_2609_13645_b200/dp.py drives them with torch.distributed (NCCL).
  *
@@ -189,8 +212,8 @@ ft_status ft_dp_set_norm(ft_model* m, const float* dev_sq_total, void* stream);
 ft_status ft_dp_collect(ft_model* m, float* host_loss, float* host_gnorm);
 
 /* Pipelined form of ft_train_step_host for training loops that do not need a step's loss before enqueueing the next
- * step (the paper's rule of keeping host synchronisation out of the hot loop, Section 5.2 / Appendix "optimization
- * catalog": device-side norm and clipping, no .item() in the step).  ft_submit_step_host enqueues, on the model's
+ * step (the paper's rule of keeping host synchronisation out of the hot loop, Section "Sources of the Speedup" (deep customization) / appendix "Optimization
+ * Catalog": device-side norm and clipping, no .item() in the step).  ft_submit_step_host enqueues, on the model's
  * stream, the copies of this step's ids, the whole step and a copy of its scalars into a pinned slot owned by the
  * library, and returns without waiting; ft_collect_step waits for the OLDEST submitted step that has not been
  * collected and returns its loss, gradient norm and status.  At most FT_MAX_IN_FLIGHT steps may be outstanding (one
@@ -202,27 +225,43 @@ ft_status ft_dp_collect(ft_model* m, float* host_loss, float* host_gnorm);
 ft_status ft_submit_step_host(ft_model* m, const int32_t* host_tokens, const int32_t* host_labels, int32_t B, int32_t S);
 ft_status ft_collect_step(ft_model* m, float* host_loss, float* host_gnorm);
 
-/* Forward and loss only; no gradients, no update. */
+/* Forward and loss only; no gradients, no update: the per-step loss that the long-run validation of Section "Correctness: The Equivalence Chain and
+ * Long-Run Validation" and Section "Training-Trajectory Agreement" compare between engine and reference, available without touching the state.
+ * Synchronises the stream; *host_loss is the mean cross-entropy over labels in [0, vocab). */
 ft_status ft_forward_loss(ft_model* m, const int32_t* dev_tokens, const int32_t* dev_labels, int32_t B, int32_t S,
                           float* host_loss);
 
-/* Forward and backward without the update: leaves the fp32 gradients readable through FT_GRAD_F32. */
+/* Forward and backward without the update: leaves every fp32 gradient readable through FT_GRAD_F32, which is how the
+ * gradient anchors of Section "Correctness: The Equivalence Chain and Long-Run Validation" ("Bit-for-Bit: zero-tolerance adjudication": activations, gradients, optimizer states
+ * at per-operator granularity) are read from this engine.  Synchronises the stream. */
 ft_status ft_forward_backward(ft_model* m, const int32_t* dev_tokens, const int32_t* dev_labels, int32_t B,
                               int32_t S, float* host_loss);
 
-/* Gradient norm + AdamW on whatever the FT_GRAD_F32 buffers hold (the optimizer in isolation). */
+/* Gradient norm + clip coefficient + AdamW on whatever the FT_GRAD_F32 buffers hold: the optimizer tail of the appendix
+ * listing in isolation (g <- g * clip; m, v updated; update = m_hat / (sqrt(v_hat) + eps) + wd * p; p <- p - lr * update;
+ * bf16 copy rewritten), so that the optimizer-state anchors can be checked apart from the gradients.  Synchronises. */
 ft_status ft_apply_update(ft_model* m, float* host_gnorm);
 
+/* get / set parameters of the problem statement, extended to the whole training state so that a run can be saved and
+ * resumed: Section "Correctness: The Equivalence Chain and Long-Run Validation" lists "checkpoint save-and-restore" and "the first step after resumption" among the edge cases
+ * an engine must reproduce exactly; masters, both moments and the step counter are that state (the bf16 copy is derived).
+ * ft_num_params / ft_param_info: number of tensors; name (owned by the model, valid until ft_destroy), ndim (1 for a
+ * gain vector, 2 for a matrix) and shape of tensor i.
+ * ft_get_param / ft_set_param: copy one tensor to / from HOST memory in the logical row-major [out, in] layout, whatever
+ * the device layout; bytes must equal the tensor's size in that kind (FT_EINVAL otherwise).  Setting FT_MASTER_F32 also
+ * rewrites the bf16 compute copy with the rounded master.  Both synchronise the model's stream.
+ * ft_get_step / ft_set_step: the optimizer step counter t (the bias corrections 1 - beta^t of the next update follow
+ * from it); restoring masters, moments and t makes the next step bit-identical to the uninterrupted run. */
 int32_t ft_num_params(const ft_model* m);
 ft_status ft_param_info(const ft_model* m, int32_t i, const char** name, int32_t* ndim, int64_t shape[2]);
-/* Copies one tensor to / from host memory (bytes must equal the tensor's size in that kind).
- * Setting FT_MASTER_F32 also rewrites the bf16 compute copy with the rounded master. */
 ft_status ft_get_param(ft_model* m, int32_t i, ft_kind kind, void* host_dst, size_t bytes);
 ft_status ft_set_param(ft_model* m, int32_t i, ft_kind kind, const void* host_src, size_t bytes);
 ft_status ft_get_step(const ft_model* m, int64_t* step);
 ft_status ft_set_step(ft_model* m, int64_t step);
 
-/* Named intermediate of the last step, copied to the host.  Forward taps of layer l: "x_in", "h1", "qkv"
+/* Named intermediate of the last step, copied to the host: this engine's form of the per-operator anchors of Section
+ * "Correctness: The Equivalence Chain and Long-Run Validation" ("taken at per-operator granularity, at exact numerical values"): every tensor a kernel hands to the next one can
+ * be read back and compared with a reference.  Forward taps of layer l: "x_in", "h1", "qkv"
  * ([T, h_q+2h_kv], q and k already rotated), "attn_lse" (fp32 [B, n_h, S]), "o", "x_mid", "h2", "gu"
  * ([T, 2f]: gate then up), "a", "x_out"; layer -1: "hF", "ce_lse" (fp32 [T]).  Backward taps (debug_taps = 1):
  * "d_x_out", "d_a", "d_gu", "d_h2", "d_x_mid", "d_o", "d_qkv", "d_h1", "d_x_in"; layer -1: "d_hF".
@@ -244,24 +283,22 @@ ft_status ft_get_profile(ft_model* m, int32_t cls, double* ms, double* work, int
  * FT_ENOTFOUND past the end.  shape = {M, N, K, a_mn, b_mn, epilogue kind}. */
 ft_status ft_get_gemm_profile(ft_model* m, int32_t i, int32_t shape[6], double* ms, int64_t* launches);
 
-/* Development switch: force the GEMM tile width (128 or 256 columns); 0 = choose by tile count (default). */
-void ft_debug_gemm_tile(int32_t bn);
-/* Development switch: 1 = CTA-pair (cta_group::2, 256 x 256 tile) GEMM kernel where it applies (default), 0 = off. */
-void ft_debug_gemm_pairs(int32_t on);
-/* Development switch: 1 = balanced-K schedule where it applies and scratch is available (default), 0 = round-robin tiles. */
-void ft_debug_gemm_balanced(int32_t on);
-/* Development switch (process-wide): 1 = the GEMM, attention, norm, SwiGLU-backward and cross-entropy kernels are launched
- * with programmatic stream serialization (Section 5.2's PDL: a kernel's blocks are scheduled and run their set-up while the
- * previous kernel drains, then wait for its completion inside the kernel), the default; 0 = ordinary stream order.  Graphs
- * captured under one setting keep it. */
-void ft_debug_pdl(int32_t on);
-
+/* Message of the last call on this model that returned a non-zero status (owned by the model; "null model" for NULL).
+ * Error behaviour of the whole boundary: nothing aborts, traps or throws; a device-side wait that ran out, a token id or
+ * label outside [0, vocab) and a non-finite loss are recorded in device memory and reported by the next synchronising
+ * call as FT_ETIMEOUT, FT_EINVAL and FT_ENONFINITE (the paper's engines keep such checks on the device and out of the
+ * hot loop: appendix "Optimization Catalog", device-side norm and clipping). */
 const char* ft_last_error(const ft_model* m);
-/* Number of kernels the library launched since the model was created (for launch accounting). */
+/* Number of kernels the library launched since the model was created (launch accounting for the paper's
+ * launch-overhead items: whole-step graph capture and programmatic dependent launch, appendix "Optimization Catalog"). */
 int64_t ft_launch_count(const ft_model* m);
+/* Destroys the host-side handle, the library's second stream, its events and a captured graph.  The workspace stays
+ * the caller's.  The caller must have synchronised the stream (or not care about work in flight). */
 void ft_destroy(ft_model* m);
 
-/* ---- single kernels, for unit parity tests and kernel timing (device pointers; stream = cudaStream_t) ---- */
+/* ---- single kernels, for unit parity tests and kernel timing (device pointers; stream = cudaStream_t): the operator
+ * layer of the paper's two-layer engine (Section "Overview: The Agent Loop and the Golden Reference"; kernel table of Section "Operator-Level Forging").  All
+ * buffers are the caller's; the calls enqueue on `stream` and return without waiting. ---- */
 
 /* C[M,N] = sum_k A[m,k] B[n,k] on the tcgen05 tensor cores, fp32 accumulation (the projection, FFN and
  * head contractions of the paper's FLOP table, forward / data-gradient / weight-gradient forms).
@@ -272,13 +309,15 @@ ft_status ft_k_gemm(const void* dev_A, int32_t a_mn, int64_t lda, const void* de
                     void* dev_C, int64_t ldc, const void* dev_resid, int32_t out_kind,
                     int32_t M, int32_t N, int32_t K, int32_t* dev_err, void* stream);
 
-/* ft_k_gemm with a device scratch buffer that lets the kernel divide work along K (Section 4.3: weight gradients
- * contract over the token dimension, the long one).  Results stay bit-identical from run to run:
+/* ft_k_gemm with a device scratch buffer that lets the kernel divide work along K (appendix "Model-FLOPs Utilization": a weight gradient
+ * contracts over the token dimension, the long one).  Results stay bit-identical from run to run:
  *  - weight-gradient layout (a_mn = b_mn = 1, fp32 output) with few 256 x 256 output tiles: up to 8 K parts run
  *    concurrently into fp32 partial outputs and a second kernel adds them in index order;
- *  - any layout whose tile count is not a multiple of the number of SM pairs: every pair takes an equally long range
- *    of (tile, K block) units; a tile cut by a range boundary is completed by the pair holding its first K block, which
- *    adds the other pairs' fp32 partial tiles in pair order before the usual epilogue.
+ *  - any layout whose last wave of 256 x 256 tiles would keep at most half of the SM pairs busy: the tiles of that wave
+ *    are divided into 2 to 8 K parts that run first, one part per pair; all parts but the last leave an fp32 partial
+ *    tile in the scratch, and the pair holding the last part (the highest-numbered pair of the group, so that it only
+ *    ever waits for pairs that were started before it) adds them in pair order before the usual epilogue.  The other
+ *    tiles then run whole, round-robin.
  * dev_scratch: caller-owned device memory, 16-byte aligned, scratch_bytes long; its contents on entry do not matter
  * (the call clears the 1 KiB of counters at its start with a stream-ordered memset) and are unspecified afterwards.
  * 20 MiB covers every case; with less the call degrades to the plain schedule of ft_k_gemm.  Two calls that share a
@@ -287,6 +326,12 @@ ft_status ft_k_gemm_ws(const void* dev_A, int32_t a_mn, int64_t lda, const void*
                        void* dev_C, int64_t ldc, const void* dev_resid, int32_t out_kind,
                        int32_t M, int32_t N, int32_t K, float* dev_scratch, uint64_t scratch_bytes,
                        int32_t* dev_err, void* stream);
+
+/* The single-kernel attention calls below keep their device status word inside the library (ft_k_gemm takes the
+ * caller's dev_err instead).  ft_k_status waits for `stream`, then returns FT_ETIMEOUT if a bounded device-side wait ran
+ * out in any ft_k_attention_* call on the current device since the last ft_k_status (and clears the word), else FT_OK.
+ * (Keeping host synchronisation out of the hot loop, Section "Sources of the Speedup", is why the calls themselves do not check.) */
+ft_status ft_k_status(void* stream);
 
 /* Causal attention core forward on a packed qkv buffer bf16 [B*S, (n_h + 2 n_kv) * d] (q heads, k heads,
  * v heads; q, k already rotated): o bf16 [B*S, n_h*d], lse fp32 [B, n_h, S] (natural log). d in {64, 128}. */
@@ -304,7 +349,7 @@ ft_status ft_k_attention_bwd(const void* dev_qkv, const void* dev_o, const void*
 /* The same backward with a second scratch array, dev_ds: B * n_h * S * S bf16 in a chunked order private to the
  * library (ds_bytes >= 2 B n_h S^2, 128-byte aligned, caller-owned device memory; contents on entry do not matter,
  * unspecified afterwards).  The dK/dV kernel
- * writes the rounded dS of Sec. 2.2's attention backward (dS = P o (dP - delta)) there, transposed, and dQ = dS K / sqrt(d)
+ * writes the rounded dS of the attention backward of appendix "Anatomy of a Forged Kernel" (dS = P o (dP - delta)) there, transposed, and dQ = dS K / sqrt(d)
  * is then one causally truncated batched contraction over the stored tiles: five tile products per (query block, key
  * block) pair instead of seven, the same dS bits feeding dK and dQ.  Needs S % 128 == 0; with dev_ds NULL, ds_bytes too
  * small, a misaligned dev_ds or any other S the call is ft_k_attention_bwd.  Results are deterministic; they agree with

@@ -13,7 +13,7 @@ What it follows in the paper
     device-side clip-coefficient listing in the appendix on framework-level
     optimisation ("Deep customization"), restated here from their arithmetic;
   * precision: bf16 compute copies written back from fp32 masters, weight
-    gradients kept in fp32 (Section 4.2, kernel table caption).
+    gradients kept in fp32 (Section "Operator-Level Forging", kernel table caption).
 
 The decoder arithmetic itself is the textbook definition; the paper does not
 restate it.  Two modes share one code path:

@@ -30,7 +30,7 @@ class FtConfig(C.Structure):
                [("recompute", C.c_int32), ("debug_taps", C.c_int32)] + \
                [(n, C.c_float) for n in ("emb_scale", "resid_scale", "logit_scale")] + [("tie_embeddings", C.c_int32),
                                                                                          ("qk_norm", C.c_int32)] + \
-               [("mtp", C.c_int32), ("mtp_weight", C.c_float)]
+               [("mtp", C.c_int32), ("mtp_weight", C.c_float), ("dp_world", C.c_int32), ("dp_rank", C.c_int32)]
 
 
 class ForgeStepError(RuntimeError):
@@ -120,10 +120,11 @@ def lib():
 def make_config(n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab, max_batch, max_seq, rms_eps=1e-5,
                 rope_theta=1e4, lr=1e-3, beta1=0.9, beta2=0.95, adam_eps=1e-8, weight_decay=0.1, max_grad_norm=0.0,
                 recompute=0, debug_taps=0, emb_scale=1.0, resid_scale=1.0, logit_scale=1.0, tie_embeddings=0, qk_norm=0,
-                mtp=0, mtp_weight=1.0) -> FtConfig:
+                mtp=0, mtp_weight=1.0, dp_world=0, dp_rank=0) -> FtConfig:
     return FtConfig(n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab, max_batch, max_seq, rms_eps,
                     rope_theta, lr, beta1, beta2, adam_eps, weight_decay, max_grad_norm, recompute, debug_taps,
-                    emb_scale, resid_scale, logit_scale, int(tie_embeddings), int(qk_norm), int(mtp), mtp_weight)
+                    emb_scale, resid_scale, logit_scale, int(tie_embeddings), int(qk_norm), int(mtp), mtp_weight, int(dp_world),
+                    int(dp_rank))
 
 
 def workspace_bytes(cfg: FtConfig) -> int:

@@ -1,4 +1,5 @@
-// The AdamW update of one element (Section 5.3, fused clip + Adam + bf16 write-back), written with explicit
+// The AdamW update of one element (Section "Sources of the Speedup" and the optimizer-tail listing of the appendix
+// "Why the Engine Is Faster, Mechanism by Mechanism": fused clip + Adam + bf16 write-back), written with explicit
 // round-to-nearest intrinsics so that every kernel that applies it (the multi-tensor pass, the weight-gradient GEMM
 // epilogue, the split-K reduction) produces the same bits from the same inputs: no compiler-chosen contraction.
 #pragma once

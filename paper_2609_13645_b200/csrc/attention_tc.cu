@@ -12,6 +12,8 @@
 #include <math.h>
 
 #include "attention.cuh"
+
+#include <mutex>
 #include "tmap.cuh"
 
 namespace fs {
@@ -781,8 +783,10 @@ static __device__ int g_attn_status;
 
 int* attention_status_word() {
   static int* addr[64] = {nullptr};
+  static std::mutex mu;  // the per-device address is looked up once; callers may come from several host threads
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
   if (!addr[dev]) {
     int* p = nullptr;
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_attn_status) != cudaSuccess) return nullptr;

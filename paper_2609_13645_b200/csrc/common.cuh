@@ -9,7 +9,7 @@ namespace fs {
 typedef __nv_bfloat16 bf16;
 
 // Device-side status word values (0 = fine).
-enum : int { ERR_NONE = 0, ERR_WAIT_TIMEOUT = 1, ERR_BAD_ALIGNMENT = 2 };
+enum : int { ERR_NONE = 0, ERR_WAIT_TIMEOUT = 1, ERR_BAD_ALIGNMENT = 2, ERR_BAD_INDEX = 3 };
 
 // Every spin-wait gives up after this many SM clock cycles (about two seconds).
 static constexpr long long kWaitLimitCycles = 4000000000LL;
@@ -62,14 +62,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false when the limit ran out or another thread of the CTA already gave up
 // (*abort_flag != 0); in that case it records the reason in *err (global) and raises *abort_flag (shared).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* err) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* err,
+                                          long long limit_cycles = kWaitLimitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 255u) == 0u) {
       if (*abort_flag != 0) return false;
-      if (clock64() - t0 > kWaitLimitCycles) {
+      if (clock64() - t0 > limit_cycles) {
         *abort_flag = 1;
         atomicExch(err, (int)ERR_WAIT_TIMEOUT);
         return false;

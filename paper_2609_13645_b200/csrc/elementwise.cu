@@ -233,11 +233,22 @@ __global__ void swiglu_bwd_kernel(const bf16* __restrict__ d_a, const bf16* __re
 }
 
 // ---------------------------------------------------------------- loss
-__global__ void count_labels_kernel(const int32_t* __restrict__ labels, int T, StepScalars* sc, long long denom_override,
+// Counts the labels that enter the loss, with the predicate the loss and its gradient use (0 <= label < vocab), and
+// checks the ids: a label >= vocab or a token id outside [0, vocab) raises ERR_BAD_INDEX in *err (the step still runs,
+// with such labels ignored and such ids clamped, and the next synchronising call reports the error).
+__global__ void count_labels_kernel(const int32_t* __restrict__ labels, const int32_t* __restrict__ tok, int T, int vocab,
+                                    StepScalars* sc, int* err, long long denom_override,
                                     const long long* __restrict__ denom_dev) {
   __shared__ int s[32];
   int c = 0;
-  for (int i = threadIdx.x; i < T; i += blockDim.x) c += labels[i] >= 0 ? 1 : 0;
+  bool bad = false;
+  for (int i = threadIdx.x; i < T; i += blockDim.x) {
+    const int y = labels[i];
+    c += (y >= 0 && y < vocab) ? 1 : 0;
+    bad |= y >= vocab;
+    if (tok != nullptr) { const int id = tok[i]; bad |= id < 0 || id >= vocab; }
+  }
+  if (bad && err != nullptr) atomicExch(err, (int)ERR_BAD_INDEX);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
   if ((threadIdx.x & 31) == 0) s[threadIdx.x >> 5] = c;
@@ -740,15 +751,24 @@ __device__ __forceinline__ unsigned long long splitmix64(unsigned long long z) {
   return z ^ (z >> 31);
 }
 
+// wgu_cols > 0: the tensor is the gate|up matrix [2f, wgu_cols] stored with rows interleaved 16 gate / 16 up; position i
+// of the stored tensor then holds the draw of its LOGICAL element (gate rows 0..f-1, then up rows 0..f-1)
 __global__ void init_normal_kernel(float* __restrict__ p, size_t n, unsigned long long seed, unsigned long long tensor_id,
-                                   double stddev) {
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+                                   double stddev, int wgu_cols, int f) {
+  for (size_t pos = (size_t)blockIdx.x * blockDim.x + threadIdx.x; pos < n; pos += (size_t)gridDim.x * blockDim.x) {
+    size_t i = pos;
+    if (wgu_cols > 0) {
+      const size_t pr = pos / (size_t)wgu_cols, c = pos - pr * (size_t)wgu_cols;
+      const size_t blk = pr >> 5, within = pr & 31;
+      const size_t lr = within < 16 ? blk * 16 + within : (size_t)f + blk * 16 + (within - 16);
+      i = lr * (size_t)wgu_cols + c;
+    }
     const unsigned long long k = seed ^ ((tensor_id + 1ull) * 0xD1B54A32D192ED03ull) ^ ((unsigned long long)i * 0x8CB92BA72F3D8DD7ull);
     const unsigned long long r = splitmix64(k);
     const double u1 = ((double)(r >> 40) + 1.0) / 16777216.0;
     const double u2 = (double)((r >> 16) & 0xFFFFFFull) / 16777216.0;
     const double z = sqrt(-2.0 * log(u1)) * cos(6.283185307179586476925286766559 * u2);
-    p[i] = (float)(z * stddev);
+    p[pos] = (float)(z * stddev);
   }
 }
 
@@ -848,9 +868,9 @@ int swiglu_bwd(const bf16* d_a, const bf16* gu, bf16* d_gu, int T, int f, cudaSt
   return ok(1);
 }
 
-int count_labels(const int32_t* labels, int T, StepScalars* sc, long long denom_override, const long long* denom_dev,
-                 cudaStream_t st) {
-  count_labels_kernel<<<1, 1024, 0, st>>>(labels, T, sc, denom_override, denom_dev);
+int count_labels(const int32_t* labels, const int32_t* tok, int T, int vocab, StepScalars* sc, int* err,
+                 long long denom_override, const long long* denom_dev, cudaStream_t st) {
+  count_labels_kernel<<<1, 1024, 0, st>>>(labels, tok, T, vocab, sc, err, denom_override, denom_dev);
   return ok(1);
 }
 
@@ -950,8 +970,8 @@ int sqnorm_final(const float* partial, int count, StepScalars* sc, AdamHyper hp,
   return ok(1);
 }
 
-int init_normal(float* p, size_t n, uint64_t seed, int tensor_id, double stddev, cudaStream_t st) {
-  init_normal_kernel<<<grid_for(n, 256), 256, 0, st>>>(p, n, seed, (unsigned long long)tensor_id, stddev);
+int init_normal(float* p, size_t n, uint64_t seed, int tensor_id, double stddev, int wgu_cols, int f, cudaStream_t st) {
+  init_normal_kernel<<<grid_for(n, 256), 256, 0, st>>>(p, n, seed, (unsigned long long)tensor_id, stddev, wgu_cols, f);
   return ok(1);
 }
 

@@ -16,7 +16,7 @@ struct StepScalars {
   float gnorm;        // global gradient norm of the last step
   float loss;         // mean loss of the last step
   float inv_count;    // 1 / number of counted labels
-  int count;          // number of labels >= 0
+  int count;          // number of labels in [0, vocab)
   int nonfinite;      // 1 if the last loss was not finite
   int err;            // device status word (ERR_*)
   int pad[5];
@@ -45,8 +45,10 @@ int qknorm_bwd(bf16* dqkv, const bf16* qkv, const float* r, const bf16* gain_q, 
 int swiglu_bwd(const bf16* d_a, const bf16* gu, bf16* d_gu, int T, int f, cudaStream_t st);
 // denom_override > 0: the loss mean (and the logit gradient) divide by it instead of by this batch's own label count
 // (denom_dev != null: the same number read from device memory when the kernel runs)
-int count_labels(const int32_t* labels, int T, StepScalars* sc, long long denom_override, const long long* denom_dev,
-                 cudaStream_t st);
+// Counted labels are those with 0 <= label < vocab (the predicate of the loss kernels).  tok (may be null) and labels are
+// also range-checked: a label >= vocab or an id outside [0, vocab) sets *err to ERR_BAD_INDEX.
+int count_labels(const int32_t* labels, const int32_t* tok, int T, int vocab, StepScalars* sc, int* err,
+                 long long denom_override, const long long* denom_dev, cudaStream_t st);
 // per row: lse, loss contribution, and (if dz != null) dz = R((softmax(z) - onehot) * inv_count), zero for ignored rows
 // dz = R(dz_scale * (softmax(z) - onehot) / counted labels)
 int cross_entropy_rows(const float* z, const int32_t* labels, float* lse, float* loss_row, bf16* dz, int rows, int V,
@@ -79,7 +81,8 @@ int adamw_with_norm(float* p, float* m, float* v, const float* g, bf16* pb, size
 int adamw_range_with_norm(float* p, float* m, float* v, const float* g, bf16* pb, size_t n, size_t n_decay, float* partial,
                           const StepScalars* sc, AdamHyper hp, cudaStream_t st);
 int sqnorm_final(const float* partial, int count, StepScalars* sc, AdamHyper hp, cudaStream_t st);
-int init_normal(float* p, size_t n, uint64_t seed, int tensor_id, double std, cudaStream_t st);
+// wgu_cols > 0: p is the gate|up matrix [2f, wgu_cols] in its interleaved row layout (draws keyed by the logical element)
+int init_normal(float* p, size_t n, uint64_t seed, int tensor_id, double std, int wgu_cols, int f, cudaStream_t st);
 int fill_f32(float* p, size_t n, float v, cudaStream_t st);
 int cast_bf16(const float* src, bf16* dst, size_t n, cudaStream_t st);
 

@@ -1,0 +1,35 @@
+/* Development entry points of libforgestep.so.  They are NOT part of the library's boundary (include/forgestep.h):
+ * the switches are process-wide, not thread-safe, and exist for kernel benchmarks and ablations; the wait probe exists
+ * so that a test can watch a bounded device-side wait run out without hanging anything. */
+#ifndef FORGESTEP_DEBUG_H_
+#define FORGESTEP_DEBUG_H_
+
+#include <stdint.h>
+
+#include "../../include/forgestep.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Force the GEMM tile width (128 or 256 columns); 0 = choose by tile count (default). */
+void ft_debug_gemm_tile(int32_t bn);
+/* 1 = CTA-pair (cta_group::2, 256 x 256 tile) GEMM kernel where it applies (default), 0 = single-CTA kernel only. */
+void ft_debug_gemm_pairs(int32_t on);
+/* 1 = balanced-K schedule where it applies and scratch is available (default), 0 = round-robin tiles. */
+void ft_debug_gemm_balanced(int32_t on);
+/* 1 = kernels are launched with programmatic stream serialization (programmatic dependent launch: appendix "Optimization Catalog", "Cross-kernel scheduling"), the default; 0 = ordinary stream
+ * order.  Graphs captured under one setting keep it. */
+void ft_debug_pdl(int32_t on);
+
+/* Enqueues, on the model's stream, a one-block kernel that waits on an mbarrier nobody ever arrives on, with the same
+ * bounded wait the GEMM and attention kernels use but a limit of limit_cycles SM clocks (1 .. 20,000,000: at most about
+ * 10 ms).  When the limit runs out the kernel records ERR_WAIT_TIMEOUT in the model's device status word and returns, so
+ * the NEXT synchronising call of the model (ft_train_step with a loss pointer, ft_collect_step, ...) returns
+ * FT_ETIMEOUT and clears the word; the context stays usable.  Nothing traps and nothing waits longer than the limit. */
+ft_status ft_debug_wait_probe(ft_model* m, int64_t limit_cycles);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FORGESTEP_DEBUG_H_ */

@@ -16,8 +16,7 @@
 namespace fs {
 
 int g_pdl = 1;
-int g_gemm_balanced = 1;
-int g_gemm_last_launches = 1;  // development knob: 0 = always the round-robin tile schedule
+int g_gemm_balanced = 1;  // development knob: 0 = always the round-robin tile schedule
 
 namespace {
 
@@ -144,9 +143,16 @@ __device__ __forceinline__ void tile_coords(int panel, int tile, int tiles_m, in
 // Round-robin schedule: piece i is unit pair + i * npairs of (tile, K part).
 // Balanced schedule, for a tile count that leaves a last wave with at most half of the pairs busy: the tiles of that
 // wave are divided into sw_parts K parts each and run FIRST, pair q taking part q % sw_parts of tile sw_first +
-// q / sw_parts.  Parts > 0 leave their accumulator in the pair's scratch slot; the pair with part 0 adds them in its
-// epilogue (which overlaps its next tile's main loop).  All pairs then walk the remaining tiles round-robin, in step
-// with one another as in the plain schedule, which keeps concurrent CTAs on the same K blocks of shared operands.
+// q / sw_parts.  All parts but the last leave their accumulator in the pair's scratch slot; the pair with the LAST
+// part (the highest-numbered pair of the group) adds them in pair order in its epilogue (which overlaps its next
+// tile's main loop).  All pairs then walk the remaining tiles round-robin, in step with one another as in the plain
+// schedule, which keeps concurrent CTAs on the same K blocks of shared operands.
+// Forward progress: the only wait between CTAs of a grid is the reducing pair's wait for its group's arrival counters,
+// and it waits only for LOWER-numbered pairs.  Thread blocks of a grid are handed to SMs in index order, so those pairs
+// were started before the waiter; they never wait for another CTA (their pieces of the divided wave come first, then
+// whole tiles), so they reach their arrival whatever else shares the GPU: a second grid on another stream (the weight
+// gradients) can delay them but cannot hold them back, and the waiter never depends on a block that is not yet
+// resident.  Nothing therefore requires the whole grid, let alone two grids, to be co-resident.
 struct WorkIter {
   int tiles_mn, kblocks, kpb, nunits, npairs, t;
   int sw_tile, sw_kb0, sw_kb1, sw_part;  // this pair's piece of the divided wave (sw_tile < 0: none)
@@ -1097,9 +1103,10 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       tile_coords(p.panel, tile, tiles_m, tiles_n, mi, ni);
       const int m0 = mi * 256 + (int)rank * BM;
       const int n0 = ni * BN;
-      if (p.adam_p != nullptr && !(split && part > 0)) adam_prefetch_chunk(p, p.C, m0 + q * 32 + lane, n0 + cb);
+      const bool reducer = !split || part == p.sw_parts - 1;  // this piece ends in the tile's epilogue
+      if (p.adam_p != nullptr && reducer) adam_prefetch_chunk(p, p.C, m0 + q * 32 + lane, n0 + cb);
       // (asking one piece earlier instead, from the previous piece's epilogue, was slower: 219 us against 201 at c3_1b)
-      if constexpr (MODE == 2) { if (!(split && part > 0)) swiglu_bwd_prefetch(p, m0 + q * 32 + lane, n0 + cb, ncols); }
+      if constexpr (MODE == 2) { if (reducer) swiglu_bwd_prefetch(p, m0 + q * 32 + lane, n0 + cb, ncols); }
       bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.err);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -1108,8 +1115,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
       const int slot_f4 = slot_thread_f4((int)rank, q, lane);
       if (tracer) { FS_GTRACE(pair, piece, 0); FS_GTRACE(pair, piece, 1); }
-      if (split && part > 0) {
-        // a later K part of a divided tile: leave this partial accumulator in the pair's slot
+      if (!reducer) {
+        // an earlier K part of a divided tile: leave this partial accumulator in the pair's slot
         float4* dst = reinterpret_cast<float4*>(p.slots) + (long long)pair * SLOT_F4 + slot_f4;
         uint32_t r[32];
         for (int c = cb; c < ce && n0 + c < p.N; c += 32) {
@@ -1128,13 +1135,14 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         Fixup fx;
         void* cptr = p.C;
         if (split && p.sw_parts > 1) {
-          // part 0 of a divided tile: wait for the other parts (they run at the same time on the next pairs) and add
-          // them in pair order
+          // last part of a divided tile: wait for the other parts (they run at the same time on the pairs just below
+          // this one, which were started earlier) and add them in pair order
           fx.n = p.sw_parts - 1;
-          fx.base = reinterpret_cast<const float4*>(p.slots) + (long long)(pair + 1) * SLOT_F4 + slot_f4;
+          const int first = pair - fx.n;
+          fx.base = reinterpret_cast<const float4*>(p.slots) + (long long)first * SLOT_F4 + slot_f4;
           int got = 1;
           if (lane == 0)
-            for (int s = 0; s < fx.n && got; ++s) got = flag_wait(p.flags + pair + 1 + s, 2 * ((int)blockDim.x / 32 - 2), abort_flag, p.err) ? 1 : 0;
+            for (int s = 0; s < fx.n && got; ++s) got = flag_wait(p.flags + first + s, 2 * ((int)blockDim.x / 32 - 2), abort_flag, p.err) ? 1 : 0;
           got = __shfl_sync(0xffffffffu, got, 0);
           if (!got) break;
           if (tracer) FS_GTRACE(pair, piece, 1);
@@ -1169,8 +1177,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   if (p.balanced && rank == 0 && threadIdx.x == 0) {
     // every warp of the pair has consumed the partials: clear the arrival counters this pair waited on for the next launch
     WorkIter mine(p, tiles_mn, kblocks_all, pair, npairs);
-    if (mine.sw_tile >= 0 && mine.sw_part == 0)
-      for (int s2 = 1; s2 < p.sw_parts; ++s2) p.flags[pair + s2] = 0;
+    if (mine.sw_tile >= 0 && mine.sw_part == p.sw_parts - 1)
+      for (int s2 = 1; s2 < p.sw_parts; ++s2) p.flags[pair - s2] = 0;
   }
   if (warp == 1) {
     __syncwarp();
@@ -1293,7 +1301,7 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
 }
 
 template <bool A_MN, bool B_MN, int MODE = 0>
-cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
+cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream, int* launches) {
   using C = PairCfg;
   auto kern = gemm_tc_pair_kernel<A_MN, B_MN, MODE>;
   static unsigned long long smem_set = 0;
@@ -1384,7 +1392,7 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream) {
   attr[1].val.programmaticStreamSerializationAllowed = g_pdl ? 1 : 0;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  g_gemm_last_launches = ksplit > 1 ? 2 : 1;
+  if (launches) *launches = ksplit > 1 ? 2 : 1;
   cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, p);
   if (e != cudaSuccess || ksplit == 1) return e;
   const long long n4 = (long long)a.M * (a.N / 4);
@@ -1415,8 +1423,8 @@ namespace fs {
 int g_gemm_force_bn = 0;
 int g_gemm_pairs = 1;  // development knob: 1 = CTA-pair kernel for outputs of at least 256 x 256, 0 = single-CTA kernel only  // development knob: 0 = choose by tile count, 128 or 256 = force that tile width
 
-cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream) {
-  g_gemm_last_launches = 1;
+cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream, int* launches) {
+  if (launches) *launches = 1;
   if (a.M <= 0 || a.N <= 0 || a.K <= 0 || !a.A || !a.B || !a.C || !a.err) return cudaErrorInvalidValue;
   if ((a.N & 7) || (a.lda & 7) || (a.ldb & 7) || (a.ldc & 3)) return cudaErrorInvalidValue;
   if ((a.a_mn ? a.M : a.K) & 7) return cudaErrorInvalidValue;
@@ -1446,18 +1454,18 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream) {
       return cudaErrorInvalidValue;
     if (a.ce_mode == 1 && (!a.ce_part || !a.ce_zy)) return cudaErrorInvalidValue;
     if (a.ce_mode == 2 && (!a.ce_lse || !a.ce_scalars || a.epi != EPI_BF16)) return cudaErrorInvalidValue;
-    return launch_pair_variant<false, false, 1>(a, stream);
+    return launch_pair_variant<false, false, 1>(a, stream, launches);
   }
   if (a.epi == EPI_SWIGLU_BWD) {
     // instantiations of their own (the epilogue's register needs stay out of the other kernels); data-gradient layout only
     if (a.a_mn || !a.b_mn || a.adam) return cudaErrorInvalidValue;
-    if (g_gemm_pairs && !g_gemm_force_bn && a.M >= 256 && a.N >= 256) return launch_pair_variant<false, true, 2>(a, stream);
+    if (g_gemm_pairs && !g_gemm_force_bn && a.M >= 256 && a.N >= 256) return launch_pair_variant<false, true, 2>(a, stream, launches);
     return wide ? launch_variant<256, false, true, 2>(a, stream) : launch_variant<128, false, true, 2>(a, stream);
   }
   if (g_gemm_pairs && !g_gemm_force_bn && a.M >= 256 && a.N >= 256) {
-    if (!a.a_mn && !a.b_mn) return launch_pair_variant<false, false>(a, stream);
-    if (!a.a_mn && a.b_mn) return launch_pair_variant<false, true>(a, stream);
-    if (a.a_mn && a.b_mn) return launch_pair_variant<true, true>(a, stream);
+    if (!a.a_mn && !a.b_mn) return launch_pair_variant<false, false>(a, stream, launches);
+    if (!a.a_mn && a.b_mn) return launch_pair_variant<false, true>(a, stream, launches);
+    if (a.a_mn && a.b_mn) return launch_pair_variant<true, true>(a, stream, launches);
     return cudaErrorInvalidValue;
   }
   if (!a.a_mn && !a.b_mn) return wide ? launch_variant<256, false, false>(a, stream) : launch_variant<128, false, false>(a, stream);

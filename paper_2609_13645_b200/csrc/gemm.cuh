@@ -67,8 +67,8 @@ struct GemmArgs {
   int* err = nullptr;  // device status word
   // Optional device scratch that lets the CTA-pair kernel divide work along K (both deterministic):
   //  - split-K: weight gradients with few output tiles run up to 8 K parts concurrently, a second kernel adds them;
-  //  - balanced-K: when the tile count is not a multiple of the pair count, every pair takes an equally long range of
-  //    (tile, K block) units and tiles cut by a range boundary are completed from fp32 partials.
+  //  - balanced-K: when the last wave of tiles would keep at most half of the pairs busy, its tiles are divided into K
+  //    parts that run first, one per pair; the highest-numbered pair of a tile's group adds the others' fp32 partials.
   // The first 1 KiB holds arrival counters that must be zero at launch; the kernel leaves them zero.  With
   // scratch_reset the launcher clears them itself (one memset node) before a balanced-K launch.
   float* scratch = nullptr;
@@ -90,12 +90,12 @@ struct GemmArgs {
   float ce_scale = 1.0f;
 };
 
-// Enqueues the contraction on `stream`.  Returns cudaErrorInvalidValue for shapes it does not take.
-cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream);
+// Enqueues the contraction on `stream`.  Returns cudaErrorInvalidValue for shapes it does not take.  *launches (when
+// given) receives the number of kernels the call enqueued (2 for a split-K contraction with its reduction, else 1).
+cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream, int* launches = nullptr);
 
 extern int g_gemm_force_bn;
 extern int g_gemm_pairs;
-extern int g_gemm_last_launches;  // kernels the last launch_gemm call enqueued
 extern int g_gemm_balanced;
 
 }  // namespace fs

@@ -10,6 +10,7 @@
 #include <vector>
 
 #include "../../include/forgestep.h"
+#include "forgestep_debug.h"
 #include "attention.cuh"
 #include "elementwise.cuh"
 #include "gemm.cuh"
@@ -66,6 +67,11 @@ struct ft_model {
 
   std::vector<ParamInfo> params;
   size_t arena = 0, n_decay = 0;
+  // ZeRO-1 state shard (cfg.dp_world > 1): master and both moments hold only this rank's slice of every gradient bucket,
+  // arena / dp_world elements each, bucket after bucket in arena order; gradients and the bf16 copy stay full size
+  int dp_world = 1, dp_rank = 0;
+  size_t state_elems = 0;  // elements of master / adam_m / adam_v
+  bool sharded() const { return dp_world > 1; }
   float *master, *adam_m, *adam_v, *grad;
   bf16* pbf;
   float *rope_cos, *rope_sin;    // [max_seq][d/2]: attention backward, QK-Norm backward
@@ -194,6 +200,9 @@ bool valid_config(const ft_config* c, std::string* why) {
   if (c->mtp != 0 && c->mtp != 1) return bad("mtp must be 0 or 1");
   if (c->mtp_weight < 0.f) return bad("negative mtp_weight");
   if (c->mtp && c->debug_taps) return bad("debug_taps is not available with the MTP head");
+  if (c->dp_world < 0 || c->dp_world > 32 || (c->dp_world & (c->dp_world - 1))) return bad("dp_world must be 0, 1, 2, 4, 8, 16 or 32");
+  if (c->dp_rank < 0 || c->dp_rank >= (c->dp_world > 1 ? c->dp_world : 1)) return bad("dp_rank must be in [0, dp_world)");
+  if (c->dp_world > 1 && c->debug_taps) return bad("debug_taps is not available with a sharded optimizer state");
   return true;
 }
 
@@ -205,6 +214,10 @@ int pick_ce_chunk(const ft_config* c) {
   if (rows > T) rows = (T + 7) / 8 * 8;
   return (int)rows;
 }
+
+void dp_build_buckets(ft_model* m);
+long long state_offset(const ft_model* m, size_t off, size_t n);
+void owned_part(const ft_model* m, size_t off, size_t n, size_t* lo, size_t* hi);
 
 // Lays the model out in the workspace.  With base == nullptr it only measures.
 size_t carve(ft_model* m, uint8_t* base) {
@@ -262,11 +275,16 @@ size_t carve(ft_model* m, uint8_t* base) {
   m->n_decay = off;
   for (auto& p : m->params) if (!p.cols) { p.offset = off; off += align_up(p.numel(), 128); }
   m->arena = off;
+  m->dp_world = c.dp_world > 1 ? c.dp_world : 1;
+  m->dp_rank = c.dp_world > 1 ? c.dp_rank : 0;
+  m->dp_buckets.clear();
+  dp_build_buckets(m);
+  m->state_elems = m->arena / (size_t)m->dp_world;  // every bucket is a multiple of 128 elements, dp_world divides 32
 
   Carver cv; cv.base = base;
-  m->master = cv.take<float>(m->arena);
-  m->adam_m = cv.take<float>(m->arena);
-  m->adam_v = cv.take<float>(m->arena);
+  m->master = cv.take<float>(m->state_elems);
+  m->adam_m = cv.take<float>(m->state_elems);
+  m->adam_v = cv.take<float>(m->state_elems);
   m->grad = cv.take<float>(m->arena);
   m->pbf = cv.take<bf16>(m->arena);
   m->rope_cosT = cv.take<float>((size_t)c.max_seq * (m->d / 2));
@@ -361,9 +379,10 @@ ft_status cuda_fail(ft_model* m, cudaError_t e, const char* where) {
 #define FT_GEMM_ON(args, stream_)                                                           \
   do {                                                                                      \
     prof_begin(m);                                                                          \
-    cudaError_t e__ = launch_gemm(args, stream_);                                           \
+    int nl__ = 1;                                                                           \
+    cudaError_t e__ = launch_gemm(args, stream_, &nl__);                                    \
     if (e__ != cudaSuccess) return cuda_fail(m, e__, "launch_gemm");                        \
-    m->launches += g_gemm_last_launches;                                                    \
+    m->launches += nl__;                                                                    \
     prof_end(m, FT_PROF_GEMM, 2.0 * (double)(args).M * (double)(args).N * (double)(args).K, 1, prof_shape_index(m, args)); \
   } while (0)
 
@@ -678,7 +697,7 @@ ft_status mtp_forward_and_head(ft_model* m, const int32_t* tok, const int32_t* l
   FT_LAUNCH(FT_PROF_NORM, 4.0 * T * h, rmsnorm_fwd(m->x[L + 2], m->wb(i_nf), m->mtp_hF, m->mtp_rF, T, h, m->cfg.rms_eps, st));
   // data parallelism: the second element of the device count array is the shifted labels' count over all ranks
   FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T,
-            count_labels(m->mtp_lab, T, m->sc_mtp, 0, m->label_count_dev ? m->label_count_dev + 1 : nullptr, st));
+            count_labels(m->mtp_lab, nullptr, T, V, m->sc_mtp, nullptr, 0, m->label_count_dev ? m->label_count_dev + 1 : nullptr, st));
   // this pass completes the head's weight gradient: its last chunk may carry AdamW (untied head only)
   s = head_pass(m, m->mtp_hF, m->mtp_lab, m->mtp_lse, m->mtp_d_hF, m->sc_mtp, m->cfg.logit_scale * m->cfg.mtp_weight, i_head, T,
                 with_bwd, true, m->cfg.tie_embeddings == 0);
@@ -730,7 +749,7 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
     FT_LAUNCH(FT_PROF_OPTIMIZER, 0.0, advance_step(m->sc, hyper(m), st));
   }
 
-  FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T, count_labels(lab, T, m->sc, m->label_count_override, m->label_count_dev, st));
+  FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T, count_labels(lab, tok, T, V, m->sc, &m->sc->err, m->label_count_override, m->label_count_dev, st));
   FT_LAUNCH(FT_PROF_ELEMENTWISE, 4.0 * T * h, embed_fwd(tok, m->wb(0), m->x[0], T, h, V, m->cfg.emb_scale, st));
   for (int l = 0; l < L; ++l) {
     ft_status s = layer_forward(m, l, m->acts[m->cfg.recompute ? 0 : l], B, S);
@@ -826,6 +845,26 @@ ft_status run_update_rest(ft_model* m) {
   return FT_OK;
 }
 
+// A wait that nothing ends: one thread waits, with the kernels' own bounded wait, on an mbarrier that gets no arrival.
+__global__ void wait_probe_kernel(long long limit_cycles, int* err) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    mbar_fence_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) mbar_wait(smem_u32(&bar), 0u, &abort_flag, err, limit_cycles);
+  __syncthreads();
+}
+
+// a non-zero device status word as a status code
+ft_status device_status(ft_model* m, int err) {
+  if (err == (int)ERR_BAD_INDEX) return fail(m, FT_EINVAL, "a token id or label is outside [0, vocab) (ids were clamped, such labels ignored)");
+  return fail(m, FT_ETIMEOUT, "a device-side wait ran out of time");
+}
+
 // one synchronisation: reads the scalars back and turns device-side flags into a status
 ft_status finish(ft_model* m, float* host_loss, float* host_gnorm) {
   StepScalars hs;
@@ -835,7 +874,7 @@ ft_status finish(ft_model* m, float* host_loss, float* host_gnorm) {
   if (host_gnorm) *host_gnorm = hs.gnorm;
   if (hs.err != 0) {
     FT_CUDA(cudaMemsetAsync(&m->sc->err, 0, sizeof(int), m->stream));
-    return fail(m, FT_ETIMEOUT, "a device-side wait ran out of time");
+    return device_status(m, hs.err);
   }
   if (hs.nonfinite) return fail(m, FT_ENONFINITE, "loss is not finite");
   return FT_OK;
@@ -865,6 +904,56 @@ void* kind_base(ft_model* m, ft_kind k) {
     case FT_GRAD_F32: return m->grad;
   }
   return nullptr;
+}
+
+// Arena range [off, off + n) as an offset into the state arrays (master, moments).  Unsharded: the same offset.  Sharded:
+// the range must lie inside this rank's slice of ONE bucket; -1 otherwise.
+long long state_offset(const ft_model* m, size_t off, size_t n) {
+  if (!m->sharded()) return (long long)off;
+  for (const auto& b : m->dp_buckets) {
+    if (off < b.offset || off >= b.offset + b.count) continue;
+    const size_t per = b.count / (size_t)m->dp_world, lo = b.offset + (size_t)m->dp_rank * per;
+    if (off < lo || off + n > lo + per) return -1;
+    return (long long)(b.offset / (size_t)m->dp_world + (off - lo));
+  }
+  return -1;
+}
+
+// The part of arena range [off, off + n) (inside one bucket) that this rank's state shard holds: [*lo, *hi), may be empty.
+void owned_part(const ft_model* m, size_t off, size_t n, size_t* lo, size_t* hi) {
+  *lo = off; *hi = off + n;
+  if (!m->sharded()) return;
+  for (const auto& b : m->dp_buckets) {
+    if (off < b.offset || off >= b.offset + b.count) continue;
+    const size_t per = b.count / (size_t)m->dp_world, s0 = b.offset + (size_t)m->dp_rank * per, s1 = s0 + per;
+    *lo = off > s0 ? off : s0;
+    *hi = off + n < s1 ? off + n : s1;
+    if (*hi < *lo) *hi = *lo;
+    return;
+  }
+  *hi = *lo;
+}
+
+void dp_build_buckets(ft_model* m) {
+  if (!m->dp_buckets.empty()) return;
+  const int L = m->L, per = m->per_layer();
+  auto span = [&](int first, int last) {  // arena range of the matrices first..last (consecutive in the arena)
+    ft_model::DpBucket b;
+    b.offset = m->params[first].offset;
+    b.count = m->params[last].offset + align_up(m->params[last].numel(), 128) - b.offset;
+    return b;
+  };
+  if (!m->cfg.tie_embeddings) { const int ih = 1 + per * L + 1; m->dp_buckets.push_back(span(ih, ih)); }
+  // the MTP head's matrices (two projections, then its layer's four: consecutive in the arena) are complete before the
+  // backbone's backward pass starts
+  if (m->cfg.mtp) m->dp_buckets.push_back(span(m->i_mtp + 2, m->i_mtp + 4 + 5));
+  for (int l = L - 1; l >= 0; --l) {
+    // a layer's matrices in parameter order: wqkv, wo, wgu, wd (the gains between them live in the gains region)
+    m->dp_buckets.push_back(span(m->idx_layer(l, 1), m->idx_layer(l, 5)));
+  }
+  m->dp_buckets.push_back(span(0, 0));
+  ft_model::DpBucket g; g.offset = m->n_decay; g.count = m->arena - m->n_decay;
+  m->dp_buckets.push_back(g);
 }
 
 }  // namespace
@@ -934,34 +1023,36 @@ ft_status ft_init_model(const ft_config* cfg, uint64_t seed, void* dev_workspace
   FT_CUDA(cudaEventCreateWithFlags(&m->ev_d, cudaEventDisableTiming));
   for (int k = 0; k < 4; ++k) FT_CUDA(cudaEventCreateWithFlags(&m->ev_w[k], cudaEventDisableTiming));
 
-  FT_CUDA(cudaMemsetAsync(m->adam_m, 0, m->arena * sizeof(float), st));
-  FT_CUDA(cudaMemsetAsync(m->adam_v, 0, m->arena * sizeof(float), st));
+  FT_CUDA(cudaMemsetAsync(m->adam_m, 0, m->state_elems * sizeof(float), st));
+  FT_CUDA(cudaMemsetAsync(m->adam_v, 0, m->state_elems * sizeof(float), st));
   FT_CUDA(cudaMemsetAsync(m->grad, 0, m->arena * sizeof(float), st));
-  FT_CUDA(cudaMemsetAsync(m->master, 0, m->arena * sizeof(float), st));
+  FT_CUDA(cudaMemsetAsync(m->master, 0, m->state_elems * sizeof(float), st));
+  // With a sharded state the full set of initial masters exists only for a moment, in the gradient arena (free at this
+  // point): the bf16 copy is cast from it and every bucket's owned slice is copied into the master shard.
+  float* full = m->sharded() ? m->grad : m->master;
   FT_CUDA(cudaMemsetAsync(m->sc, 0, sizeof(StepScalars), st));
   FT_CUDA(cudaMemsetAsync(m->splitk, 0, 1024, st));  // the GEMM scratch's arrival counters start at zero
   FT_CUDA(cudaMemsetAsync(m->splitk2, 0, 1024, st));
   for (size_t i = 0; i < m->params.size(); ++i) {
     const ParamInfo& p = m->params[i];
     if (p.cols) {
-      // element e of the LOGICAL tensor i gets draw (seed, i, e); wgu is drawn logically, then placed physically
-      if (!p.is_wgu) {
-        FT_LAUNCH(FT_PROF_ELEMENTWISE, 0.0, init_normal(m->master + p.offset, p.numel(), seed, (int)i, 0.02, st));
-      } else {
-        float* tmp = m->grad + p.offset;  // the gradient arena is free at this point
-        FT_LAUNCH(FT_PROF_ELEMENTWISE, 0.0, init_normal(tmp, p.numel(), seed, (int)i, 0.02, st));
-        for (int64_t r0 = 0; r0 < 2 * (int64_t)m->f; r0 += 16) {
-          const int64_t pr = wgu_phys_row(r0, m->f);
-          FT_CUDA(cudaMemcpyAsync(m->master + p.offset + pr * p.cols, tmp + r0 * p.cols, 16 * p.cols * sizeof(float),
-                                  cudaMemcpyDeviceToDevice, st));
-        }
-      }
+      // element e of the LOGICAL tensor i gets draw (seed, i, e); wgu's rows are written at their physical places
+      FT_LAUNCH(FT_PROF_ELEMENTWISE, 0.0,
+                init_normal(full + p.offset, p.numel(), seed, (int)i, 0.02, p.is_wgu ? (int)p.cols : 0, m->f, st));
     } else {
-      FT_LAUNCH(FT_PROF_ELEMENTWISE, 0.0, fill_f32(m->master + p.offset, p.numel(), 1.0f, st));
+      FT_LAUNCH(FT_PROF_ELEMENTWISE, 0.0, fill_f32(full + p.offset, p.numel(), 1.0f, st));
     }
   }
-  FT_CUDA(cudaMemsetAsync(m->grad, 0, m->arena * sizeof(float), st));
-  FT_LAUNCH(FT_PROF_ELEMENTWISE, 0.0, cast_bf16(m->master, m->pbf, m->arena, st));
+  FT_LAUNCH(FT_PROF_ELEMENTWISE, 0.0, cast_bf16(full, m->pbf, m->arena, st));
+  if (m->sharded()) {
+    for (const auto& b : m->dp_buckets) {
+      size_t lo, hi;
+      owned_part(m, b.offset, b.count, &lo, &hi);
+      FT_CUDA(cudaMemcpyAsync(m->master + state_offset(m, lo, hi - lo), full + lo, (hi - lo) * sizeof(float),
+                              cudaMemcpyDeviceToDevice, st));
+    }
+    FT_CUDA(cudaMemsetAsync(m->grad, 0, m->arena * sizeof(float), st));
+  }
 
   {
     ft_status sr = build_rope_tables(m, nullptr, 1.0f);
@@ -972,6 +1063,7 @@ ft_status ft_init_model(const ft_config* cfg, uint64_t seed, void* dev_workspace
 
 // One full step enqueued launch by launch.
 static ft_status step_direct(ft_model* m, const int32_t* tok, const int32_t* lab, int32_t B, int32_t S) {
+  if (m->sharded()) return fail(m, FT_EINVAL, "a model with a sharded optimizer state (dp_world > 1) steps through the ft_dp_* calls");
   const bool fuse = m->fused_update && m->cfg.max_grad_norm <= 0.f && !m->cfg.debug_taps;
   ft_status s = run_forward_backward(m, tok, lab, B, S, true, fuse);
   if (s) return s;
@@ -1135,36 +1227,13 @@ ft_status ft_collect_step(ft_model* m, float* host_loss, float* host_gnorm) {
   if (host_gnorm) *host_gnorm = hs.gnorm;
   if (hs.err != 0) {
     FT_CUDA(cudaMemsetAsync(&m->sc->err, 0, sizeof(int), m->stream));
-    return fail(m, FT_ETIMEOUT, "a device-side wait ran out of time");
+    return device_status(m, hs.err);
   }
   if (hs.nonfinite) return fail(m, FT_ENONFINITE, "loss is not finite");
   return FT_OK;
 }
 
 // ---------------------------------------------------------------- data-parallel hooks
-namespace {
-void dp_build_buckets(ft_model* m) {
-  if (!m->dp_buckets.empty()) return;
-  const int L = m->L, per = m->per_layer();
-  auto span = [&](int first, int last) {  // arena range of the matrices first..last (consecutive in the arena)
-    ft_model::DpBucket b;
-    b.offset = m->params[first].offset;
-    b.count = m->params[last].offset + align_up(m->params[last].numel(), 128) - b.offset;
-    return b;
-  };
-  if (!m->cfg.tie_embeddings) { const int ih = 1 + per * L + 1; m->dp_buckets.push_back(span(ih, ih)); }
-  // the MTP head's matrices (two projections, then its layer's four: consecutive in the arena) are complete before the
-  // backbone's backward pass starts
-  if (m->cfg.mtp) m->dp_buckets.push_back(span(m->i_mtp + 2, m->i_mtp + 4 + 5));
-  for (int l = L - 1; l >= 0; --l) {
-    // a layer's matrices in parameter order: wqkv, wo, wgu, wd (the gains between them live in the gains region)
-    m->dp_buckets.push_back(span(m->idx_layer(l, 1), m->idx_layer(l, 5)));
-  }
-  m->dp_buckets.push_back(span(0, 0));
-  ft_model::DpBucket g; g.offset = m->n_decay; g.count = m->arena - m->n_decay;
-  m->dp_buckets.push_back(g);
-}
-}  // namespace
 
 int32_t ft_dp_num_buckets(ft_model* m) {
   if (!m) return 0;
@@ -1186,7 +1255,8 @@ ft_status ft_arena_ptr(ft_model* m, ft_kind kind, void** dev_ptr, int64_t* numel
   void* b = kind_base(m, kind);
   if (!b) return FT_EINVAL;
   *dev_ptr = b;
-  *numel = (int64_t)m->arena;
+  const bool state = kind == FT_MASTER_F32 || kind == FT_ADAM_M_F32 || kind == FT_ADAM_V_F32;
+  *numel = (int64_t)(state ? m->state_elems : m->arena);
   return FT_OK;
 }
 
@@ -1266,7 +1336,9 @@ ft_status ft_dp_update_range(ft_model* m, int64_t offset, int64_t count, void* s
   if (!m || !dp_range_ok(m, offset, count)) return FT_EINVAL;
   const size_t off = (size_t)offset, n = (size_t)count;
   const size_t n_decay = m->n_decay > off ? (m->n_decay - off < n ? m->n_decay - off : n) : 0;
-  if (adamw(m->master + off, m->adam_m + off, m->adam_v + off, m->grad + off, m->pbf + off, n, n_decay, m->sc, hyper(m),
+  const long long so = state_offset(m, off, n);
+  if (so < 0) return fail(m, FT_EINVAL, "sharded state: the range must lie inside this rank's slice of one bucket");
+  if (adamw(m->master + so, m->adam_m + so, m->adam_v + so, m->grad + off, m->pbf + off, n, n_decay, m->sc, hyper(m),
             reinterpret_cast<cudaStream_t>(stream)) < 0)
     return FT_ECUDA;
   m->have_bwd = false;
@@ -1296,6 +1368,7 @@ ft_status ft_forward_backward(ft_model* m, const int32_t* dev_tokens, const int3
 
 ft_status ft_apply_update(ft_model* m, float* host_gnorm) {
   if (!m) return FT_EINVAL;
+  if (m->sharded()) return fail(m, FT_EINVAL, "a model with a sharded optimizer state (dp_world > 1) updates through ft_dp_update_range");
   ft_status s = run_update(m);
   if (s) return s;
   return finish(m, nullptr, host_gnorm);
@@ -1322,6 +1395,26 @@ static ft_status param_copy(ft_model* m, int32_t i, ft_kind kind, void* host, si
   uint8_t* dev = reinterpret_cast<uint8_t*>(kind_base(m, kind)) + p.offset * es;
   uint8_t* hp = reinterpret_cast<uint8_t*>(host);
   FT_CUDA(cudaStreamSynchronize(m->stream));
+  // Sharded state: masters and moments exist only for this rank's slices.  The tensor is staged, in its device layout, in
+  // its span of the gradient arena (whose contents are lost): reading returns the owned elements and 0 elsewhere (so the
+  // ranks' results add up to the whole tensor), writing stores the owned elements (every rank passes the whole tensor).
+  const bool staged = m->sharded() && (kind == FT_MASTER_F32 || kind == FT_ADAM_M_F32 || kind == FT_ADAM_V_F32);
+  const size_t span = align_up(p.numel(), 128);
+  size_t own_lo = 0, own_hi = 0;
+  if (staged) {
+    float* stage = m->grad + p.offset;
+    float* shard = reinterpret_cast<float*>(kind_base(m, kind));
+    owned_part(m, p.offset, span, &own_lo, &own_hi);
+    m->have_bwd = false;
+    dev = reinterpret_cast<uint8_t*>(stage);
+    if (to_host) {
+      FT_CUDA(cudaMemsetAsync(stage, 0, span * sizeof(float), m->stream));
+      if (own_hi > own_lo)
+        FT_CUDA(cudaMemcpyAsync(stage + (own_lo - p.offset), shard + state_offset(m, own_lo, own_hi - own_lo),
+                                (own_hi - own_lo) * sizeof(float), cudaMemcpyDeviceToDevice, m->stream));
+      FT_CUDA(cudaStreamSynchronize(m->stream));
+    }
+  }
   if (!p.is_wgu) {
     if (to_host) FT_CUDA(copy_sync(m, hp, dev, bytes, cudaMemcpyDeviceToHost));
     else FT_CUDA(copy_sync(m, dev, hp, bytes, cudaMemcpyHostToDevice));
@@ -1336,8 +1429,14 @@ static ft_status param_copy(ft_model* m, int32_t i, ft_kind kind, void* host, si
     }
   }
   if (!to_host && kind == FT_MASTER_F32) {
-    const size_t span = align_up(p.numel(), 128);
-    FT_LAUNCH(FT_PROF_ELEMENTWISE, 0.0, cast_bf16(m->master + p.offset, m->pbf + p.offset, span, m->stream));
+    const float* src = staged ? m->grad + p.offset : m->master + p.offset;
+    FT_LAUNCH(FT_PROF_ELEMENTWISE, 0.0, cast_bf16(src, m->pbf + p.offset, span, m->stream));
+    FT_CUDA(cudaStreamSynchronize(m->stream));
+  }
+  if (staged && !to_host && own_hi > own_lo) {
+    float* shard = reinterpret_cast<float*>(kind_base(m, kind));
+    FT_CUDA(cudaMemcpyAsync(shard + state_offset(m, own_lo, own_hi - own_lo), m->grad + own_lo, (own_hi - own_lo) * sizeof(float),
+                            cudaMemcpyDeviceToDevice, m->stream));
     FT_CUDA(cudaStreamSynchronize(m->stream));
   }
   return FT_OK;
@@ -1456,6 +1555,15 @@ void ft_debug_gemm_balanced(int32_t on) { g_gemm_balanced = on; }
 void ft_debug_pdl(int32_t on) { g_pdl = on; }
 void ft_debug_gemm_pairs(int32_t on) { g_gemm_pairs = on; }
 
+ft_status ft_debug_wait_probe(ft_model* m, int64_t limit_cycles) {
+  if (!m) return FT_EINVAL;
+  if (limit_cycles < 1 || limit_cycles > 20000000) return fail(m, FT_EINVAL, "limit_cycles must be in [1, 20000000]");
+  wait_probe_kernel<<<1, 32, 0, m->stream>>>((long long)limit_cycles, &m->sc->err);
+  FT_CUDA(cudaGetLastError());
+  m->launches += 1;
+  return FT_OK;
+}
+
 ft_status ft_get_gemm_profile(ft_model* m, int32_t i, int32_t shape[6], double* ms, int64_t* launches) {
   if (!m || !shape) return FT_EINVAL;
   FT_CUDA(cudaStreamSynchronize(m->stream));
@@ -1512,6 +1620,19 @@ ft_status ft_k_gemm_ws(const void* dev_A, int32_t a_mn, int64_t lda, const void*
   cudaError_t e = launch_gemm(g, reinterpret_cast<cudaStream_t>(stream));
   if (e == cudaErrorInvalidValue) return FT_EINVAL;
   return e == cudaSuccess ? FT_OK : FT_ECUDA;
+}
+
+ft_status ft_k_status(void* stream) {
+  int* status = attention_status_word();
+  if (!status) return FT_ECUDA;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  int v = 0;
+  if (cudaMemcpyAsync(&v, status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return FT_ECUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return FT_ECUDA;
+  if (v == 0) return FT_OK;
+  if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return FT_ECUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return FT_ECUDA;
+  return FT_ETIMEOUT;
 }
 
 ft_status ft_k_attention_fwd(const void* dev_qkv, void* dev_o, float* dev_lse, int32_t B, int32_t S, int32_t n_heads,

@@ -1,6 +1,7 @@
-"""Data-parallel train step over the library's C-ABI hooks: the paper's recipe (Section 5.2) of a bucketed gradient
-reduce-scatter overlapped with the backward pass, a ZeRO-1 style sharded AdamW and a per-bucket all-gather of the bf16
-compute copy interleaved with it.
+"""Data-parallel train step over the library's C-ABI hooks: the paper's recipe (Section "Sources of the Speedup";
+appendix "Framework-Level Optimization Trajectory": gradient bucketing, per-bucket all-gather + optimizer overlap, ZeRO-1
+sharded optimizer) of a bucketed gradient reduce-scatter overlapped with the backward pass, a ZeRO-1 sharded AdamW and a
+per-bucket all-gather of the bf16 compute copy interleaved with it.
 
 The exchange is `torch.distributed` (NCCL between GPUs); everything else — forward, backward, norm, AdamW — runs in the
 library's own kernels through `ft_dp_*`.  One process per GPU.  Per step and rank:
@@ -8,15 +9,23 @@ library's own kernels through `ft_dp_*`.  One process per GPU.  Per step and ran
   1. the number of labels >= 0 is summed over the ranks (one 8-byte all-reduce, on the device) and handed to the library
      as a device pointer (no host round trip), so that every rank's loss and gradients are already divided by the GLOBAL
      count and the reduction is a plain sum;
-  2. `ft_dp_backward` enqueues forward + backward on the model's stream and records one event per gradient bucket, in
+  2. the second (communication) stream is ordered behind what the model's stream holds so far, i.e. the PREVIOUS step,
+     BEFORE this step's backward pass is enqueued: from here on it waits only for the per-bucket events;
+  3. `ft_dp_backward` enqueues forward + backward on the model's stream and records one event per gradient bucket, in
      the order the backward pass completes them (head, layers last to first, embedding table, gains);
-  3. on a second stream, per bucket: wait for its event, reduce-scatter it in place (rank r keeps slice r), and, when
-     clipping is off, run AdamW on that slice and all-gather the bucket's bf16 copy right away; with clipping on the
-     updates wait for the global norm (sum of squares of every rank's slices, one 4-byte all-reduce);
-  4. the model's stream waits for the second stream; the rank's loss share is read back and summed over the ranks.
+  4. on the second stream, per bucket: wait for its event, reduce-scatter it in place (rank r keeps slice r), and, when
+     clipping is off, run AdamW on that slice and all-gather the bucket's bf16 copy right away, while the model's stream
+     is still busy with the layers below; with clipping on the updates wait for the global norm (sum of squares of every
+     rank's slices, one 4-byte all-reduce);
+  5. the model's stream waits for the second stream; the rank's loss share is read back and summed over the ranks.
 
-Sharding covers the optimizer's work and memory traffic; the workspace still holds full-size master and moment arenas
-(only the owned slices of them are kept current), so it does not yet shrink with the number of ranks.
+A bucket's event follows the last kernel that reads that bucket's bf16 weights (its data gradients, and with
+recomputation its re-run forward), so the all-gather that rewrites them cannot overtake a reader.
+
+Optimizer state: with `dp_world` / `dp_rank` in the model's config (they must equal the group's size and this rank) the
+workspace holds masters and moments only for the rank's own slices, 12 / world bytes per parameter; without them (one
+rank, or an unsharded model on several) the arenas are full size and only the owned slices are kept current.
+`DataParallel.get_state` / `set_state` assemble or distribute whole tensors for checkpoints.
 
 `DataParallel` talks to a backend object, so the bucket / slice / collective logic is exercised on CPU (gloo) with a
 stand-in backend; `LibraryBackend` is the real one.
@@ -107,7 +116,23 @@ class LibraryBackend:
         return self.torch.cuda.stream(self.comm_stream)
 
     def begin_comm(self):
-        self.comm_stream.wait_stream(self.main_stream)  # the previous step's readers of what this step overwrites
+        # ordered behind the PREVIOUS step only (its readers of what this step's collectives overwrite): called before this
+        # step's backward pass is enqueued, so that the per-bucket events are the only thing the collectives wait for
+        self.comm_stream.wait_stream(self.main_stream)
+
+    def shard(self):
+        """(dp_world, dp_rank) of the model's optimizer-state shard; (1, 0) when the state is whole."""
+        w = int(self.model.cfg.dp_world)
+        return (w, int(self.model.cfg.dp_rank)) if w > 1 else (1, 0)
+
+    def get_param(self, name, kind):
+        return self.torch.from_numpy(self.model.get_param(name, kind)).to(self.device)
+
+    def set_param(self, name, value, kind):
+        self.model.set_param(name, value, kind)
+
+    def param_names(self):
+        return [n for n, _ in self.model.params]
 
     def end_comm(self):
         self.main_stream.wait_stream(self.comm_stream)
@@ -139,12 +164,19 @@ class LibraryBackend:
 class DataParallel:
     """One data-parallel train step per call of `step`; see the module text for the sequence."""
 
-    def __init__(self, backend, group=None):
-        import torch.distributed as dist
+    def __init__(self, backend, group=None, dist=None):
+        """dist: the module that provides the collectives (default torch.distributed); a stand-in with the same calls
+        lets tests run several ranks inside one process."""
+        if dist is None:
+            import torch.distributed as dist
         self.dist, self.backend, self.group = dist, backend, group
         self.world = dist.get_world_size(group)
         self.rank = dist.get_rank(group)
         self.buckets = backend.buckets()
+        shard = backend.shard() if hasattr(backend, "shard") else (1, 0)
+        if shard != (1, 0) and shard != (self.world, self.rank):
+            raise ValueError(f"the model's state shard {shard} is not (world, rank) = ({self.world}, {self.rank}) of the group")
+        self.sharded = shard != (1, 0)
         for off, cnt in self.buckets:
             if cnt % (4 * self.world) or off % 4:
                 raise ValueError(f"bucket ({off}, {cnt}) does not divide into {self.world} slices of whole 16-byte groups")
@@ -181,15 +213,15 @@ class DataParallel:
         total = be.count_labels(labels)
         dist.all_reduce(total, op=dist.ReduceOp.SUM, group=self.group)
         be.set_label_count(total)  # stays on the device: no host round trip before the step is enqueued
+        be.begin_comm()            # behind the previous step, ahead of this step's backward pass
         be.backward(tokens, labels)
         grad, comp = be.grad(), be.compute_copy()
-        be.begin_comm()
         with be.comm():
-            if not be.clipping:
-                be.begin_update(None)
             for i, (off, cnt) in enumerate(self.buckets):
                 so, sn = self.slice_of(i)
                 be.wait_bucket(i)
+                if i == 0 and not be.clipping:
+                    be.begin_update(None)  # step counter and bias corrections, once, behind the first finished bucket
                 self._reduce_scatter(grad[off:off + cnt], grad[so:so + sn])
                 be.sqnorm(so, sn, self.sq[i:i + 1])
                 if not be.clipping:
@@ -212,3 +244,16 @@ class DataParallel:
         loss[0] = share
         dist.all_reduce(loss, op=dist.ReduceOp.SUM, group=self.group)
         return float(loss.item()), gnorm
+
+    # ---- whole tensors for checkpoints (masters, moments), whatever the sharding
+    def get_state(self, name, kind):
+        """The whole tensor `name` of `kind` (binding.KIND_MASTER / KIND_ADAM_M / KIND_ADAM_V) on every rank.  With a
+        sharded state every rank contributes its owned elements (the library returns 0 elsewhere) and the parts are summed."""
+        t = self.backend.get_param(name, kind)
+        if self.sharded:
+            self.dist.all_reduce(t, op=self.dist.ReduceOp.SUM, group=self.group)
+        return t
+
+    def set_state(self, name, value, kind):
+        """Every rank passes the whole tensor; with a sharded state each keeps its own elements."""
+        self.backend.set_param(name, value, kind)

@@ -75,11 +75,12 @@ class OracleBackend:
             self.g[self.off[n]:self.off[n] + params[n].size] = torch.from_numpy((grads[n] * w).astype(np.float32).ravel())
         self.events.append("backward")
     def comm(self): return nullcontext()
-    def begin_comm(self): pass
+    def begin_comm(self): self.events.append("begin_comm")
     def end_comm(self): pass
     def wait_bucket(self, i): self.events.append(("wait", i))
     def sqnorm(self, off, cnt, out): out[0] = float((self.g[off:off + cnt].double() ** 2).sum())
     def begin_update(self, sq):
+        self.events.append("begin_update")
         self.step_no += 1
         if sq is not None:
             self.gnorm = float(sq[0]) ** 0.5
@@ -121,7 +122,7 @@ for i in range(len(dp.buckets)):
     so, sn = dp.slice_of(i)
     owned = max(owned, float((be.master[so:so + sn].float() - be.comp[so:so + sn]).abs().max()))
 out["owned_master_vs_copy"] = owned
-out["events"] = [e if isinstance(e, str) else list(e) for e in be.events[:12]]
+out["events"] = [e if isinstance(e, str) else list(e) for e in be.events[:14]]
 out["slices"] = [list(dp.slice_of(i)) for i in range(len(dp.buckets))]
 out["buckets"] = [list(b) for b in dp.buckets]
 with open(os.path.join(sys.argv[2], f"rank{{rank}}.json"), "w") as fh:   # (two ranks printing at once interleave)
@@ -159,10 +160,12 @@ def test_two_rank_data_parallel_step_equals_one_process_on_the_whole_batch(tmp_p
     # slices: rank r owns the r-th half of every bucket, 16-byte groups, and the two halves tile the bucket
     for (off, cnt), s0, s1 in zip(res[0]["buckets"], res[0]["slices"], res[1]["slices"]):
         assert s0 == [off, cnt // 2] and s1 == [off + cnt // 2, cnt // 2] and cnt % 8 == 0
-    # order of a step: backward enqueued first, then per bucket wait -> (update when clipping is off)
+    # order of a step: the communication stream is ordered behind the previous step BEFORE the backward pass is enqueued
+    # (so that only the per-bucket events hold the collectives back), then per bucket wait -> update (clipping off); the
+    # step counter advances once, behind the first finished bucket; with clipping the updates follow the global norm
     ev = res[0]["events"]
-    assert ev[0] == "backward" and ev[1] == ["wait", 0]
+    assert ev[0] == "begin_comm" and ev[1] == "backward" and ev[2] == ["wait", 0]
     if clip == 0.0:
-        assert ev[2][0] == "update" and ev[3] == ["wait", 1]
+        assert ev[3] == "begin_update" and ev[4][0] == "update" and ev[5] == ["wait", 1] and ev[6][0] == "update"
     else:
-        assert ev[2] == ["wait", 1]
+        assert ev[3] == ["wait", 1] and "begin_update" not in ev[:3 + 3]

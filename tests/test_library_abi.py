@@ -51,6 +51,13 @@ def test_workspace_size_and_config_validation_run_on_the_host():
     assert B.workspace_bytes(B.make_config(**base, tie_embeddings=1)) < n0
     assert B.workspace_bytes(B.make_config(**base, qk_norm=1)) > n0
     assert B.workspace_bytes(B.make_config(**base, emb_scale=0.0, resid_scale=0.0, logit_scale=0.0)) == n0
+    # a sharded optimizer state (ZeRO-1): masters and moments shrink to 1 / dp_world, nothing else changes
+    n_params = 1024 * 256 * 2 + 2 * (256 * 512 + 256 * 256 + 2 * 688 * 256 + 256 * 688)
+    for world in (2, 8):
+        nw = B.workspace_bytes(B.make_config(**base, dp_world=world, dp_rank=world - 1))
+        assert abs((n0 - nw) - 12 * n_params * (world - 1) / world) < 0.02 * 12 * n_params
+    for bad in (dict(dp_world=3), dict(dp_world=64), dict(dp_world=2, dp_rank=2), dict(dp_world=0, dp_rank=1), dict(dp_world=2, debug_taps=1)):
+        assert B.workspace_bytes(B.make_config(**base, **bad)) == 0, bad
     # the 1B-shaped workload fits one B200 with room to spare
     big = B.make_config(16, 2048, 16, 8, 128, 5632, 32000, 4, 2048)
     assert B.workspace_bytes(big) < 60 * 2 ** 30

@@ -1,7 +1,9 @@
 """Whole train step (forward, backward, AdamW) of the CUDA library against the CPU oracle, through the C ABI.
 
-Tolerances are the ones the task states: loss abs 1e-2, per-tensor relative L2 <= 2e-2 on activations and
-gradients, <= 1e-3 on updated fp32 masters; run-to-run results are bit-identical.
+Tolerances: loss abs 1e-2, per-tensor relative L2 <= 2e-2 on activations and gradients, <= 1e-3 on updated fp32
+masters (asserted where Adam's moments are warm; the very first update is g / (|g| + eps) = sign(g), where a gradient
+entry of the wrong sign moves a master by 2 lr, so step 1 is held to the sign-flip bound with a fixed ceiling);
+run-to-run results are bit-identical.
 """
 import numpy as np
 import pytest
@@ -10,10 +12,14 @@ import torch
 import synth_inputs as SI
 from oracle import decoder as D
 from tests.parity_util import (BWD_TAPS, FWD_TAPS, lib_config, lib_tap, load_params, oracle_config, rel_l2, to_dev)
+from tests.parity_util import f32 as parity_f32
 
 pytestmark = pytest.mark.gpu
 
 TOL_LOSS, TOL_ACT, TOL_MASTER = 1e-2, 2e-2, 1e-3
+# step 1 only (cold moments): ceiling on the master error whatever the sign-flip prediction says, so that a regression in
+# the gradients or the update cannot widen its own tolerance (measured worst case over the shapes and variants of this file: 4.5e-3)
+MASTER_CEILING_STEP1 = 6e-3
 
 
 def _c1():
@@ -76,7 +82,7 @@ def _check_step(ocfg, tok, lab, params, debug=True, recompute=0, report=None, st
         rho = worst["grad." + name]
         rms_p = float(np.sqrt(np.mean(st.params[name].astype(np.float64) ** 2)))
         predicted = 2.0 * ocfg.lr / rms_p * np.sqrt(rho / np.pi)
-        assert e < max(TOL_MASTER, 2.5 * predicted), ("master", name, e, predicted)
+        assert e < max(TOL_MASTER, min(2.5 * predicted, MASTER_CEILING_STEP1)), ("master", name, e, predicted)
         # the bf16 compute copy is the rounded new master
         got_b = model.get_param(name, B.KIND_BF16)
         assert np.array_equal(got_b, D.bf16_round(model.get_param(name, B.KIND_MASTER)).astype(np.float32))
@@ -460,9 +466,57 @@ def test_whole_step_graph_replay_is_bit_identical_to_plain_launches():
     plain.close()
 
 
+@pytest.mark.parametrize("shape", ["c1", "gqa", "gqa_clip"])
+def test_masters_after_a_step_with_warm_moments_meet_the_1e_3_bound(shape):
+    """The stated bound on updated masters, rel-L2 <= 1e-3 per tensor, in the regime where it can hold: the state
+    (masters, both moments, step counter) of five oracle steps is loaded into the library, both sides take one more step
+    on the same fresh batch.  With warm moments the update is m_hat / (sqrt(v_hat) + eps), a smooth function of the
+    gradient, so the bf16-level gradient differences (rho ~ 1e-3) move a master by ~ lr * 0.1 * rho, far below the bound.
+    Also: gradients of that step within 2e-2, moments within 1e-3, and the step counter restored and advanced."""
+    from paper_2609_13645_b200 import binding as B
+    if shape == "c1":
+        ocfg, w = _c1()
+        Bsz, S, dist = w["batch"], w["seq"], "uniform"
+    else:
+        ocfg = _small_gqa()
+        if shape == "gqa_clip":
+            ocfg.max_grad_norm = parity_f32(0.5)
+        Bsz, S, dist = 2, 200, "zipf"
+    params = D.init_params(ocfg, 4321)
+    st = D.TrainState(ocfg, params)
+    for k in range(5):
+        tok, lab = SI.batch(ocfg.vocab, Bsz, S, dist, seed=77, step=k)
+        st.train_step(tok, lab)
+    model = B.Model(lib_config(B, ocfg, Bsz, S), seed=1)
+    model.set_fused_update(False)  # the gradients of the step are compared too
+    for name in params:
+        model.set_param(name, st.params[name], B.KIND_MASTER)
+        model.set_param(name, st.m[name], B.KIND_ADAM_M)
+        model.set_param(name, st.v[name], B.KIND_ADAM_V)
+    model.step = st.step
+    assert model.step == 5
+    tok, lab = SI.batch(ocfg.vocab, Bsz, S, dist, seed=77, step=5)
+    loss_o, gn_o, grads_o, _ = st.train_step(tok, lab)
+    loss_g, gn_g = model.train_step(to_dev(tok), to_dev(lab))
+    assert abs(loss_g - loss_o) < TOL_LOSS
+    assert abs(gn_g - gn_o) / gn_o < 5e-3
+    worst = {}
+    for name in params:
+        assert rel_l2(model.get_param(name, B.KIND_GRAD), grads_o[name]) < TOL_ACT, name
+        e = rel_l2(model.get_param(name, B.KIND_MASTER), st.params[name])
+        worst[name] = e
+        assert e < TOL_MASTER, ("master", name, e)
+        assert rel_l2(model.get_param(name, B.KIND_ADAM_M), st.m[name]) < 5e-3, ("m", name)
+        assert rel_l2(model.get_param(name, B.KIND_ADAM_V), st.v[name]) < 5e-3, ("v", name)
+    print("warm-moment master rel-L2, worst:", sorted(worst.items(), key=lambda kv: -kv[1])[:4])
+    assert model.step == 6
+    model.close()
+
+
 def test_ten_step_loss_and_gradient_norm_trajectory_matches_oracle():
     """Ten consecutive steps on fresh batches: per-step loss within 1e-2, gradient norm within 1 %, and the masters
-    after ten steps within the sign-flip bound of one step (the error does not pile up)."""
+    after ten steps within 8e-3 (measured 6.8e-3 on the embedding table, 4e-3 on the projections: the cold first step's
+    sign flips plus the drift of two bf16 trajectories, which Adam's normalisation keeps from piling up)."""
     from paper_2609_13645_b200 import binding as B
     ocfg = oracle_config(n_layers=2, d_model=256, n_heads=4, n_kv_heads=2, head_dim=64, d_ffn=352, vocab=512)
     params = D.init_params(ocfg, 2024)
@@ -476,9 +530,12 @@ def test_ten_step_loss_and_gradient_norm_trajectory_matches_oracle():
         assert abs(loss_g - loss_o) < TOL_LOSS, (step, loss_g, loss_o)
         assert abs(gn_g - gn_o) / gn_o < 1e-2, (step, gn_g, gn_o)
     assert model.step == 10
+    worst = {}
     for name in params:
         e = rel_l2(model.get_param(name), st.params[name])
-        assert e < 1e-2, (name, e)
+        worst[name] = e
+        assert e < 8e-3, (name, e)
+    print("ten-step master rel-L2, worst:", sorted(worst.items(), key=lambda kv: -kv[1])[:4])
     model.close()
 
 
