@@ -168,7 +168,7 @@ def cpu_baseline(workload: str):
     """Oracle on a bounded sample: same shape with 2 layers, 1 x 256 tokens, one step.  The oracle's achieved
     model-FLOP/s on the sample is converted to tokens/s of the full workload with the same FLOP formula."""
     w = SI.WORKLOADS[workload]
-    nl, B, S = min(2, w["n_layers"]), 1, min(256, w["seq"])
+    nl, B, S = oracle_sample_shape(workload)
     times, fl = oracle_sample_run(workload, nl, B, S, steps=1, warmup=0)
     rate = fl / times[0]
     full = model_flops(w, w["seq"])["total"]
@@ -178,12 +178,18 @@ def cpu_baseline(workload: str):
                       f"FLOPs/token"}
 
 
+def oracle_sample_shape(workload: str):
+    """The bounded sample both oracle legs time: the workload's shape with 2 of its layers, batch 1 x 256 tokens."""
+    w = SI.WORKLOADS[workload]
+    return min(2, w["n_layers"]), 1, min(256, w["seq"])
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
     w = SI.WORKLOADS[args.workload]
-    nl, B, S = 1, 1, min(64, w["seq"])
+    nl, B, S = oracle_sample_shape(args.workload)
     times, fl = oracle_sample_run(args.workload, nl, B, S, steps=args.steps, warmup=args.warmup)
     t = sum(times) / len(times)
     rate = fl / t

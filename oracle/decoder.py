@@ -81,8 +81,9 @@ class Config:
     rope_factors: Optional[Tuple[float, ...]] = None
     rope_mscale: float = 1.0
     # One-layer multi-token-prediction (Eagle) head (appendix "Model Architectures", row "MTP / Eagle head: On (1 layer)";
-    # appendix "Ascend Model-FLOPs Utilization": the head "repeats the backbone layer's attention, projection, and FFN
-    # plus a second output head").  The paper fixes that much and no more; reading = the published depth-1 MTP module:
+    # appendix "Ascend Model-FLOPs Utilization": its FLOP count is one more backbone layer, attention core, projections
+    # and feed-forward, plus one more output head).  The paper fixes that much and no more; reading = the published
+    # depth-1 MTP module:
     #   h'_i = R(R(hn_i Wh^T) + en_i We^T),  hn = R(rmsnorm(x_L; g_h)),  en = R(rmsnorm(R(emb_scale E[tok_{i+1}]); g_e)),
     #   x' = one more decoder layer on h' (parameters "mtp.layer.*"), z' = logit_scale * R(rmsnorm(x'; g_f)) W_head^T
     #   with the backbone's output head, trained on the token after next: label'_i = label_{i+1}; the last position of a
@@ -268,6 +269,17 @@ def sigmoid(x: np.ndarray) -> np.ndarray:
     return 1.0 / (1.0 + np.exp(-x))
 
 
+def swiglu_fwd(G: np.ndarray, U: np.ndarray) -> np.ndarray:
+    """a = silu(G) U = G sigmoid(G) U (the SwiGLU feed-forward's gate, appendix "Model Architectures")."""
+    return G * sigmoid(G) * U
+
+
+def swiglu_bwd(d_a: np.ndarray, G: np.ndarray, U: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """(dG, dU) of a = G s U with s = sigmoid(G): dU = d_a G s, dG = d_a U s (1 + G (1 - s)).  Unrounded."""
+    sg = sigmoid(G)
+    return d_a * U * sg * (1.0 + G * (1.0 - sg)), d_a * G * sg
+
+
 def attention_fwd(q, k, v, n_rep: int, R, contract: bool):
     """Causal softmax(q k^T / sqrt(d)) v per batch and head.
 
@@ -398,7 +410,7 @@ def forward_backward(cfg: Config, params: Dict[str, np.ndarray], tokens: np.ndar
         gu = h2 @ W[p + "wgu"].T
         G = R(gu[..., :f])
         U = R(gu[..., f:])
-        a = R(G * sigmoid(G) * U)
+        a = R(swiglu_fwd(G, U))
         x_out = R(x_mid + s_r * (a @ W[p + "wd"].T))
         sv = dict(x_in=x_in, r1=r1, h1=h1, q=q, k=k, v=v, o=o, lse=lse, x_mid=x_mid, r2=r2, h2=h2, G=G, U=U, a=a)
         if cfg.qk_norm:
@@ -473,9 +485,8 @@ def forward_backward(cfg: Config, params: Dict[str, np.ndarray], tokens: np.ndar
         d_a = R((s_r * dx) @ W[p + "wd"])
         grads[p + "wd"] = (s_r * dx).reshape(T, h).T @ sv["a"].reshape(T, f)
         G, U = sv["G"], sv["U"]
-        sg = sigmoid(G)
-        dU = R(d_a * G * sg)
-        dG = R(d_a * U * sg * (1.0 + G * (1.0 - sg)))
+        dG, dU = swiglu_bwd(d_a, G, U)
+        dG, dU = R(dG), R(dU)
         dGU = np.concatenate([dG, dU], axis=-1)
         d_h2 = R(dGU @ W[p + "wgu"])
         grads[p + "wgu"] = dGU.reshape(T, 2 * f).T @ sv["h2"].reshape(T, h)

@@ -51,8 +51,8 @@ struct FwdCfg {
 template <int D>
 __global__ void __launch_bounds__(ATT_THREADS, 2)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKV,
-                   bf16* __restrict__ o, float* __restrict__ lse, int S, int n_heads, int n_kv, float scale_log2,
-                   int* err) {
+                   bf16* __restrict__ o, float* __restrict__ lse, int S, int n_heads, int n_kv, int n_batch, int n_qblocks,
+                   float scale_log2, int* err) {
   using C = FwdCfg<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sbase = smem_u32(smem);
@@ -67,8 +67,13 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     if (threadIdx.x == 0) atomicExch(err, (int)ERR_BAD_ALIGNMENT);
     return;
   }
-  const int qb = gridDim.x - 1 - blockIdx.x;  // heaviest blocks first
-  const int n = blockIdx.y, b = blockIdx.z;
+  // Thread blocks are started in index order, so the index runs over the query blocks from the heaviest (last) to the
+  // lightest across ALL heads and batch rows: the blocks still running at the end of the launch are the short ones.  (With
+  // the query block as the fastest grid dimension the heaviest block of the last head started last and ran alone.)
+  const int groups = n_heads * n_batch;
+  const int qb = n_qblocks - 1 - (int)blockIdx.x / groups;
+  const int grp = (int)blockIdx.x % groups;
+  const int n = grp % n_heads, b = grp / n_heads;
   const int kvh = n / (n_heads / n_kv);
   const int hq = n_heads * D, hkv = n_kv * D;
   const int q0 = qb * C::BQ;
@@ -317,8 +322,9 @@ cudaError_t attention_fwd_tc_t(const bf16* qkv, bf16* o, float* lse, int B, int 
   if (!make_tmap_3d(&tmQ, qkv, nqkv, S, B, nqkv, C::BQ) || !make_tmap_3d(&tmKV, qkv, nqkv, S, B, nqkv, C::BK))
     return cudaErrorInvalidValue;
   const float scale_log2 = (float)((1.0 / sqrt((double)D)) * 1.4426950408889634);
-  dim3 grid((S + C::BQ - 1) / C::BQ, nh, B);
-  cudaError_t el = launch_pdl(attn_fwd_tc_kernel<D>, grid, ATT_THREADS, C::SMEM_BYTES, st, tmQ, tmKV, o, lse, S, nh, nkv, scale_log2, err);
+  const int nqb = (S + C::BQ - 1) / C::BQ;
+  dim3 grid((unsigned)(nqb * nh * B), 1, 1);
+  cudaError_t el = launch_pdl(attn_fwd_tc_kernel<D>, grid, ATT_THREADS, C::SMEM_BYTES, st, tmQ, tmKV, o, lse, S, nh, nkv, B, nqb, scale_log2, err);
   if (el != cudaSuccess) return el;
   return cudaGetLastError();
 }
@@ -397,7 +403,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
                    const __grid_constant__ CUtensorMap tm_do128, const __grid_constant__ CUtensorMap tm_do64,
                    const float* __restrict__ lse, const float* __restrict__ delta, bf16* __restrict__ dqkv,
                    bf16* __restrict__ ds_out, const float* __restrict__ rope_cos, const float* __restrict__ rope_sin, int S,
-                   int n_heads, int n_kv, float scale, float scale_log2, int* err) {
+                   int n_heads, int n_kv, int n_batch, int n_xblocks, float scale, float scale_log2, int* err) {
   using C = BwdCfg<D, MODE>;
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sbase = smem_u32(smem);
@@ -416,16 +422,20 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
   const int n_rep = n_heads / n_kv;
   const int hq = n_heads * D, hkv = n_kv * D;
   const long long ld = hq + 2 * hkv;
-  const int b = blockIdx.z;
+  // one-dimensional grid, heaviest blocks first across all heads and batch rows (see the forward kernel)
+  const int groups = (MODE == MODE_DQ ? n_heads : n_kv) * n_batch;
+  const int xrank = (int)blockIdx.x / groups, grp = (int)blockIdx.x % groups;
+  const int heads_here = MODE == MODE_DQ ? n_heads : n_kv;
+  const int b = grp / heads_here;
   int x0, kvh, n_q = 0, iters, qb0 = 0, per_head = 1;
   if constexpr (MODE == MODE_DQ) {
-    x0 = (gridDim.x - 1 - blockIdx.x) * 128;  // heaviest query blocks first
-    n_q = blockIdx.y;
+    x0 = (n_xblocks - 1 - xrank) * 128;  // the last query blocks see the most keys
+    n_q = grp % heads_here;
     kvh = n_q / n_rep;
     iters = (min(S, x0 + 128) + 63) / 64;
   } else {
-    x0 = blockIdx.x * 128;  // the first key blocks see the most queries
-    kvh = blockIdx.y;
+    x0 = xrank * 128;  // the first key blocks see the most queries
+    kvh = grp % heads_here;
     qb0 = x0 / 64;
     per_head = (S + 63) / 64 - qb0;
     iters = per_head * n_rep;
@@ -761,20 +771,21 @@ cudaError_t attention_bwd_tc_t(const bf16* qkv, const bf16* o, const bf16* d_o, 
   const float scale_log2 = (float)((1.0 / sqrt((double)D)) * 1.4426950408889634);
   cudaError_t e = attention_delta(o, d_o, delta, B, S, nh, D, st);
   if (e != cudaSuccess) return e;
-  dim3 gq((S + 127) / 128, nh, B), gk((S + 127) / 128, nkv, B);
+  const int nxb = (S + 127) / 128;
+  dim3 gq((unsigned)(nxb * nh * B), 1, 1), gk((unsigned)(nxb * nkv * B), 1, 1);
   bf16* none = nullptr;
   if (ds != nullptr) {
     // dK/dV first, leaving dS^T behind; dQ is then one causally truncated batched contraction over it
     e = launch_pdl(attn_bwd_tc_kernel<D, MODE_DKV>, gk, BWD_THREADS, CK::SMEM_BYTES, st, tq128, tq64, td128, td64, lse, delta,
-                   dqkv, ds, cs, sn, S, nh, nkv, scale, scale_log2, err);
+                   dqkv, ds, cs, sn, S, nh, nkv, B, nxb, scale, scale_log2, err);
     if (e != cudaSuccess) return e;
     return attention_dq_from_ds(ds, qkv, dqkv, cs, sn, B, S, nh, nkv, D, err, st);
   }
   e = launch_pdl(attn_bwd_tc_kernel<D, MODE_DQ>, gq, BWD_THREADS, CQ::SMEM_BYTES, st, tq128, tq64, td128, td64, lse, delta,
-                 dqkv, none, cs, sn, S, nh, nkv, scale, scale_log2, err);
+                 dqkv, none, cs, sn, S, nh, nkv, B, nxb, scale, scale_log2, err);
   if (e != cudaSuccess) return e;
   return launch_pdl(attn_bwd_tc_kernel<D, MODE_DKV>, gk, BWD_THREADS, CK::SMEM_BYTES, st, tq128, tq64, td128, td64, lse, delta,
-                    dqkv, none, cs, sn, S, nh, nkv, scale, scale_log2, err);
+                    dqkv, none, cs, sn, S, nh, nkv, B, nxb, scale, scale_log2, err);
 }
 
 static __device__ int g_attn_status;

@@ -168,24 +168,28 @@ rmsnorm_bwd_kernel(const bf16* __restrict__ dy, const bf16* __restrict__ x, cons
   for (int c = threadIdx.x; c < h; c += blockDim.x) partial[(long long)blockIdx.x * h + c] = s_dg[c];
 }
 
-// out[c] = sum over blocks of partial[b][c], in block order: 32 columns x 8 row groups per CTA, the 8 groups
-// (each a fixed strided subset of the blocks) are then added in group order.
-__global__ void colsum_kernel(const float* __restrict__ partial, float* __restrict__ out, int nblk, int h) {
+// Column sums of block partials, in block order: 32 columns x 8 row groups per CTA, the 8 groups (each a fixed strided
+// subset of the blocks) are then added in group order.
+// Many partial buffers at once: blockIdx.y selects slot y ([nblk][h] partials at partial + y * slot_floats) and
+// the gradient tensor out[y] it sums into.  One launch at the end of the backward pass replaces one per norm.
+__global__ void colsum_many_kernel(const float* __restrict__ partial, float* const* __restrict__ out, int nblk, int h,
+                                   long long slot_floats) {
   pdl_trigger();
   pdl_wait();
   __shared__ float s[8][33];
   const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
   const int c = blockIdx.x * 32 + cx;
+  const float* src = partial + (long long)blockIdx.y * slot_floats;
   float a = 0.f;
   if (c < h)
-    for (int b = ry; b < nblk; b += 8) a += partial[(long long)b * h + c];
+    for (int b = ry; b < nblk; b += 8) a += src[(long long)b * h + c];
   s[ry][cx] = a;
   __syncthreads();
   if (ry == 0 && c < h) {
     float tot = 0.f;
 #pragma unroll
     for (int w = 0; w < 8; ++w) tot += s[w][cx];
-    out[c] = tot;
+    out[blockIdx.y][c] = tot;
   }
 }
 
@@ -819,7 +823,7 @@ static void launch_rmsnorm_bwd(int nblk, const bf16* dy, const bf16* x, const fl
   launch_pdl(rmsnorm_bwd_kernel<NCHW, WPR>, nblk, 256, h * sizeof(float), st, dy, x, r, g, resid, dx, partial, T, h);
 }
 
-int rmsnorm_bwd(const bf16* dy, const bf16* x, const float* r, const bf16* g, const bf16* resid, bf16* dx, float* dg,
+int rmsnorm_bwd(const bf16* dy, const bf16* x, const float* r, const bf16* g, const bf16* resid, bf16* dx,
                 float* partial, int T, int h, cudaStream_t st) {
   if ((h & 255) || h > 256 * kNormMaxChunks) return -1;
   const int nblk = elementwise_blocks_for_norm(T);
@@ -837,8 +841,14 @@ int rmsnorm_bwd(const bf16* dy, const bf16* x, const float* r, const bf16* g, co
     }
   }
 #undef FS_NORM_CASE
-  if (launch_pdl(colsum_kernel, (h + 31) / 32, 256, 0, st, partial, dg, nblk, h) != cudaSuccess) return -1;
-  return ok(2);
+  return ok(1);
+}
+
+int colsum_many(const float* partial, float* const* out, int nslots, size_t slot_floats, int T, int h, cudaStream_t st) {
+  if (nslots <= 0) return 0;
+  const int nblk = elementwise_blocks_for_norm(T);
+  if (launch_pdl(colsum_many_kernel, dim3((h + 31) / 32, nslots), 256, 0, st, partial, out, nblk, h, (long long)slot_floats) != cudaSuccess) return -1;
+  return ok(1);
 }
 
 int qknorm_bwd(bf16* dqkv, const bf16* qkv, const float* r, const bf16* gain_q, const bf16* gain_k, const float* cosT,

@@ -33,9 +33,14 @@ size_t sort_pad(size_t n);                         // padded key count of the em
 // each returns the number of kernels it launched, or a negative value after a CUDA launch error
 int embed_fwd(const int32_t* tok, const bf16* E, bf16* x, int T, int h, int vocab, float scale, cudaStream_t st);
 int rmsnorm_fwd(const bf16* x, const bf16* g, bf16* y, float* r, int T, int h, float eps, cudaStream_t st);
-// dx = R(resid + rmsnorm_bwd(dy)) (resid may be null); dg = column sums (fp32, fixed order) via `partial`.
-int rmsnorm_bwd(const bf16* dy, const bf16* x, const float* r, const bf16* g, const bf16* resid, bf16* dx, float* dg,
+// dx = R(resid + rmsnorm_bwd(dy)) (resid may be null).  The gain gradient is left as one partial row per block in
+// `partial` ([elementwise_blocks_for_norm(T)][h] floats, this norm's own slot); colsum_many adds the rows of every slot in
+// block order (fp32, fixed order) into the gradient tensors, once, after the backward pass.
+int rmsnorm_bwd(const bf16* dy, const bf16* x, const float* r, const bf16* g, const bf16* resid, bf16* dx,
                 float* partial, int T, int h, cudaStream_t st);
+// out[y][c] = sum over blocks b < elementwise_blocks_for_norm(T) of partial[y * slot_floats + b * h + c] for every slot
+// y < nslots; out is a DEVICE array of nslots device pointers.  T as in the rmsnorm_bwd calls that filled the slots.
+int colsum_many(const float* partial, float* const* out, int nslots, size_t slot_floats, int T, int h, cudaStream_t st);
 // d_gu (physical 16/16 interleave of gate and up columns) from d_a and the saved gate|up activations.
 // Per-head QK-Norm backward, in place on dqkv's query and key heads (see the kernel); dgain_q, dgain_k [d] fp32 are
 // overwritten; partial: scratch of partial_floats floats (one row of 2 d per block; more room, more blocks, up to 1184).

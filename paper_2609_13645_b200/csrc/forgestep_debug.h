@@ -22,6 +22,11 @@ void ft_debug_gemm_balanced(int32_t on);
  * order.  Graphs captured under one setting keep it. */
 void ft_debug_pdl(int32_t on);
 
+/* Largest bf16 logit-gradient buffer [max_batch * max_seq, vocab] a model created AFTERWARDS will carry (default 4 GiB):
+ * within it the output head's two gradients are single contractions over all rows, above it they are formed per chunk
+ * of rows with the weight gradient accumulating in memory.  0 forces the chunked form (tests cover both). */
+void ft_debug_head_dz_limit(uint64_t bytes);
+
 /* Enqueues, on the model's stream, a one-block kernel that waits on an mbarrier nobody ever arrives on, with the same
  * bounded wait the GEMM and attention kernels use but a limit of limit_cycles SM clocks (1 .. 20,000,000: at most about
  * 10 ms).  When the limit runs out the kernel records ERR_WAIT_TIMEOUT in the model's device status word and returns, so

@@ -21,6 +21,10 @@ namespace {
 
 constexpr size_t kAlign = 256;
 constexpr size_t kAttnDsMaxBytes = 24ull << 30;  // largest dS^T scratch the workspace will carry
+// The logit gradient dz of ALL rows is kept (bf16 [T, V]) when it fits in this many bytes: the output head's data and
+// weight gradients are then one contraction each over all rows; above it they are formed chunk by chunk, the weight
+// gradient accumulating in fp32 memory.  (A variable so that a test can force the chunked form: ft_debug_head_dz_limit.)
+size_t g_head_dz_limit = 4ull << 30;
 constexpr size_t kSplitKFloats = 6u << 20;  // 24 MiB of split-K partial tiles (74 tiles of 256 x 256 fp32 at most)
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -64,6 +68,7 @@ struct ft_model {
   int h, hq, hkv, nqkv, f, V, L, d, maxT;
   int n_slots;
   int ce_chunk;
+  int dz_rows;  // rows of the dz buffer: maxT (gradients of the head in one pass) or ce_chunk (chunk by chunk)
 
   std::vector<ParamInfo> params;
   size_t arena = 0, n_decay = 0;
@@ -86,6 +91,12 @@ struct ft_model {
   bf16 *hF, *d_hF;
   bf16 *dxA, *dxB, *d_h, *d_a, *d_gu, *d_o, *d_qkv;
   float *delta, *norm_partial, *sq_partial, *z, *splitk;
+  // gain gradients of the RMSNorms: every norm's backward leaves block partials in its own slot of norm_partial, and one
+  // kernel after the backward pass sums all slots into the gradient tensors (norm_out: device array of their addresses)
+  std::vector<int> norm_slot_of;  // parameter index -> slot, -1 for everything that is not a [d_model] gain
+  int n_norm_slots = 0;
+  float** norm_out = nullptr;
+  float* qk_partial = nullptr;    // scratch of the per-head QK-Norm backward (one more slot)
   bf16* dz;
   unsigned long long* keys;
   int lastB = 0, lastS = 0;
@@ -227,6 +238,7 @@ size_t carve(ft_model* m, uint8_t* base) {
   m->maxT = c.max_batch * c.max_seq;
   m->n_slots = c.recompute ? 1 : c.n_layers;
   m->ce_chunk = pick_ce_chunk(&c);
+  m->dz_rows = ((size_t)m->maxT * (size_t)c.vocab * sizeof(bf16) <= g_head_dz_limit && m->maxT > m->ce_chunk) ? m->maxT : m->ce_chunk;
   const size_t T = (size_t)m->maxT, h = m->h, f = m->f, hq = m->hq, nqkv = m->nqkv, V = m->V;
 
   // parameter table: matrices first (they get weight decay), gains after
@@ -330,7 +342,14 @@ size_t carve(ft_model* m, uint8_t* base) {
   m->attn_ds_bytes = attention_bwd_ds_bytes(c.max_batch, c.max_seq, c.n_heads);
   if (m->attn_ds_bytes > kAttnDsMaxBytes) m->attn_ds_bytes = 0;
   m->attn_ds = m->attn_ds_bytes ? cv.take<bf16>(m->attn_ds_bytes / sizeof(bf16)) : nullptr;
-  m->norm_partial = cv.take<float>((size_t)elementwise_blocks_for_norm((int)T) * h);
+  m->norm_slot_of.assign(m->params.size(), -1);
+  m->n_norm_slots = 0;
+  for (size_t i = 0; i < m->params.size(); ++i)
+    if (!m->params[i].cols && m->params[i].rows == (int64_t)h) m->norm_slot_of[i] = m->n_norm_slots++;
+  const size_t slot_floats = (size_t)elementwise_blocks_for_norm((int)T) * h;
+  m->norm_partial = cv.take<float>((size_t)(m->n_norm_slots + 1) * slot_floats);
+  m->qk_partial = m->norm_partial ? m->norm_partial + (size_t)m->n_norm_slots * slot_floats : nullptr;
+  m->norm_out = cv.take<float*>((size_t)m->n_norm_slots);
   m->sq_partial = cv.take<float>(kSqnormBlocks);
   m->dp_sq = cv.take<float>(4);
   m->ce_part = cv.take<float2>((size_t)m->ce_chunk * ((V + 255) / 256));
@@ -339,7 +358,7 @@ size_t carve(ft_model* m, uint8_t* base) {
   m->splitk = cv.take<float>(kSplitKFloats);
   m->splitk2 = cv.take<float>(kSplitKFloats);
   m->z = cv.take<float>((size_t)m->ce_chunk * V);
-  m->dz = cv.take<bf16>((size_t)m->ce_chunk * V);
+  m->dz = cv.take<bf16>((size_t)m->dz_rows * V);
   m->keys = cv.take<unsigned long long>(sort_pad(T));
   m->taps.clear();
   if (c.debug_taps) {
@@ -459,6 +478,11 @@ const AdamFuse* fuse_for(ft_model* m, int wi) {
   m->fuse_idx += 1;
   m->fuse_args.push_back(a);
   return &m->fuse_args.back();
+}
+
+// the slot of norm_partial that receives the block partials of gain parameter i's gradient
+float* norm_slot(ft_model* m, int i) {
+  return m->norm_partial + (size_t)m->norm_slot_of[i] * (size_t)elementwise_blocks_for_norm(m->maxT) * m->h;
 }
 
 // forward of layer l from m->x[l] into activation slot `a`, output to m->x[l+1]
@@ -581,7 +605,7 @@ ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
   }
   if ((s = wait_wgrad(m, 2))) return s;  // the previous layer's output-projection weight gradient still reads dxB
   FT_LAUNCH(FT_PROF_NORM, 8.0 * T * h, rmsnorm_bwd(m->d_h, a.x_mid, a.r2, m->wb(m->idx_layer(l, 3)), m->dxA, m->dxB,
-                                                    m->gr(m->idx_layer(l, 3)), m->norm_partial, T, h, st));
+                                                    norm_slot(m, m->idx_layer(l, 3)), T, h, st));
   s = linear_backward(m, m->dxB, a.o, m->idx_layer(l, 2), m->d_o, T, h, hq, 2, m->cfg.resid_scale);
   if (s) return s;
   if ((s = wait_wgrad(m, 3))) return s;  // the previous layer's qkv weight gradient still reads d_qkv
@@ -595,7 +619,7 @@ ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
     // d_q, d_k so far are gradients of the normalised heads: through the per-head norm, in place, and the two gain gradients
     FT_LAUNCH(FT_PROF_NORM, 6.0 * T * (hq + m->hkv),
               qknorm_bwd(m->d_qkv, a.qkv, a.qk_r, m->wb(m->idx_layer(l, 6)), m->wb(m->idx_layer(l, 7)), m->rope_cos,
-                         m->rope_sin, m->gr(m->idx_layer(l, 6)), m->gr(m->idx_layer(l, 7)), m->norm_partial,
+                         m->rope_sin, m->gr(m->idx_layer(l, 6)), m->gr(m->idx_layer(l, 7)), m->qk_partial,
                          (size_t)elementwise_blocks_for_norm(m->maxT) * h, 1.0f / (m->rope_mscale * m->rope_mscale), T, S,
                          m->cfg.n_heads, m->cfg.n_kv_heads, m->d, st));
   }
@@ -609,7 +633,7 @@ ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
   }
   if ((s = wait_wgrad(m, 0))) return s;  // this layer's down-projection weight gradient still reads dxA
   FT_LAUNCH(FT_PROF_NORM, 8.0 * T * h, rmsnorm_bwd(m->d_h, m->x[l], a.r1, m->wb(m->idx_layer(l, 0)), m->dxB, m->dxA,
-                                                    m->gr(m->idx_layer(l, 0)), m->norm_partial, T, h, st));
+                                                    norm_slot(m, m->idx_layer(l, 0)), T, h, st));
   if (tp) { if ((s = copy_tap(m, tp->d_x_in, m->dxA, (size_t)T * h))) return s; }
   return FT_OK;
 }
@@ -622,13 +646,16 @@ ft_status head_pass(ft_model* m, const bf16* hF, const int32_t* lab, float* lse,
                     int i_head, int T, bool with_bwd, bool accumulate, bool fuse_last) {
   const int h = m->h, V = m->V;
   cudaStream_t st = m->stream;
+  // one_pass: dz of every row is kept and both head gradients are single contractions after the chunk loop
+  const bool one_pass = with_bwd && m->dz_rows >= T && T > m->ce_chunk;
   for (int r0 = 0, chunk = 0; r0 < T; r0 += m->ce_chunk, ++chunk) {
     const int rows = (T - r0) < m->ce_chunk ? (T - r0) : m->ce_chunk;
+    bf16* dz = one_pass ? m->dz + (size_t)r0 * V : m->dz;
     if (m->streaming_ce) {
       // no logits in memory: the GEMM's epilogue reduces each 256-column tile of a row to (max, sum), a small kernel
       // combines them, and the same GEMM runs again with an epilogue that turns its accumulators into bf16 dz
       GemmArgs g = gemm_base(m);
-      g.A = hF + (size_t)r0 * h; g.lda = h; g.B = m->wb(i_head); g.ldb = h; g.C = m->dz; g.ldc = V;
+      g.A = hF + (size_t)r0 * h; g.lda = h; g.B = m->wb(i_head); g.ldb = h; g.C = dz; g.ldc = V;
       g.M = rows; g.N = V; g.K = h; g.epi = EPI_BF16; g.alpha = m->cfg.logit_scale;
       g.ce_mode = 1; g.ce_part = m->ce_part; g.ce_tiles = (V + 255) / 256; g.ce_zy = m->ce_zy; g.ce_labels = lab + r0;
       FT_GEMM(g);
@@ -646,24 +673,40 @@ ft_status head_pass(ft_model* m, const bf16* hF, const int32_t* lab, float* lse,
         FT_GEMM(g);
       }
       FT_LAUNCH(FT_PROF_CE, (with_bwd ? 10.0 : 4.0) * rows * V,
-                cross_entropy_rows(m->z, lab + r0, lse + r0, m->loss_row + r0, with_bwd ? m->dz : nullptr, rows, V,
+                cross_entropy_rows(m->z, lab + r0, lse + r0, m->loss_row + r0, with_bwd ? dz : nullptr, rows, V,
                                    sc, dz_scale, st));
     }
-    if (with_bwd) {
+    if (with_bwd && !one_pass) {
       {
         GemmArgs g = gemm_base(m);
-        g.A = m->dz; g.lda = V; g.B = m->wb(i_head); g.b_mn = 1; g.ldb = h; g.C = d_hF + (size_t)r0 * h; g.ldc = h;
+        g.A = dz; g.lda = V; g.B = m->wb(i_head); g.b_mn = 1; g.ldb = h; g.C = d_hF + (size_t)r0 * h; g.ldc = h;
         g.M = rows; g.N = h; g.K = V; g.epi = EPI_BF16;
         FT_GEMM(g);
       }
       {
         GemmArgs g = gemm_base(m);
-        g.A = m->dz; g.a_mn = 1; g.lda = V; g.B = hF + (size_t)r0 * h; g.b_mn = 1; g.ldb = h; g.C = m->gr(i_head);
+        g.A = dz; g.a_mn = 1; g.lda = V; g.B = hF + (size_t)r0 * h; g.b_mn = 1; g.ldb = h; g.C = m->gr(i_head);
         g.ldc = h; g.M = V; g.N = h; g.K = rows; g.epi = (chunk == 0 && !accumulate) ? EPI_F32 : EPI_F32_ACC;
         // the last chunk completes the gradient (with tied embeddings the table's own part is still to come)
         if (m->fusing && fuse_last && r0 + rows >= T) g.adam = fuse_for(m, i_head);
         FT_GEMM(g);
       }
+    }
+  }
+  if (one_pass) {
+    {
+      GemmArgs g = gemm_base(m);
+      g.A = m->dz; g.lda = V; g.B = m->wb(i_head); g.b_mn = 1; g.ldb = h; g.C = d_hF; g.ldc = h;
+      g.M = T; g.N = h; g.K = V; g.epi = EPI_BF16;
+      FT_GEMM(g);
+    }
+    {
+      // the weight gradient in one contraction over all rows: no fp32 read-modify-write passes over a [V, h] tensor
+      GemmArgs g = gemm_base(m);
+      g.A = m->dz; g.a_mn = 1; g.lda = V; g.B = hF; g.b_mn = 1; g.ldb = h; g.C = m->gr(i_head);
+      g.ldc = h; g.M = V; g.N = h; g.K = T; g.epi = accumulate ? EPI_F32_ACC : EPI_F32;
+      if (m->fusing && fuse_last) g.adam = fuse_for(m, i_head);
+      FT_GEMM(g);
     }
   }
   return FT_OK;
@@ -713,20 +756,18 @@ ft_status mtp_forward_and_head(ft_model* m, const int32_t* tok, const int32_t* l
 ft_status mtp_backward(ft_model* m, int B, int S, bool tied) {
   const int T = B * S, h = m->h, V = m->V, L = m->L, i0 = m->i_mtp, i_nf = i0 + 4 + m->per_layer();
   cudaStream_t st = m->stream;
-  FT_LAUNCH(FT_PROF_NORM, 6.0 * T * h, rmsnorm_bwd(m->mtp_d_hF, m->x[L + 2], m->mtp_rF, m->wb(i_nf), nullptr, m->dxA, m->gr(i_nf),
-                                                    m->norm_partial, T, h, st));
+  FT_LAUNCH(FT_PROF_NORM, 6.0 * T * h, rmsnorm_bwd(m->mtp_d_hF, m->x[L + 2], m->mtp_rF, m->wb(i_nf), nullptr, m->dxA, norm_slot(m, i_nf), T, h, st));
   ft_status s = layer_backward(m, L + 1, m->acts_mtp, B, S);
   if (s) return s;
   // h' = R(u1 + en We^T), u1 = R(hn Wh^T): the add hands the same gradient (dxA) to both projections
   if ((s = linear_backward(m, m->dxA, m->mtp_en, i0 + 3, m->mtp_d_en, T, h, h, 0))) return s;
   if ((s = linear_backward(m, m->dxA, m->mtp_hn, i0 + 2, m->mtp_d_hn, T, h, h, 0))) return s;
   FT_LAUNCH(FT_PROF_NORM, 6.0 * T * h, rmsnorm_bwd(m->mtp_d_en, m->mtp_xe, m->mtp_re, m->wb(i0 + 1), nullptr, m->mtp_d_xe,
-                                                    m->gr(i0 + 1), m->norm_partial, T, h, st));
+                                                    norm_slot(m, i0 + 1), T, h, st));
   // with tied embeddings the head passes have already written the table's gradient; otherwise this is its first part
   FT_LAUNCH(FT_PROF_ELEMENTWISE, 2.0 * T * h + 4.0 * V * h,
             embed_bwd(m->mtp_tok, m->mtp_d_xe, m->gr(0), m->keys, T, h, V, m->cfg.emb_scale, tied, st));
-  FT_LAUNCH(FT_PROF_NORM, 6.0 * T * h, rmsnorm_bwd(m->mtp_d_hn, m->x[L], m->mtp_rh, m->wb(i0), nullptr, m->mtp_d_xL, m->gr(i0),
-                                                    m->norm_partial, T, h, st));
+  FT_LAUNCH(FT_PROF_NORM, 6.0 * T * h, rmsnorm_bwd(m->mtp_d_hn, m->x[L], m->mtp_rh, m->wb(i0), nullptr, m->mtp_d_xL, norm_slot(m, i0), T, h, st));
   return FT_OK;
 }
 
@@ -781,8 +822,7 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
     if (m->dp_mode) FT_CUDA(cudaEventRecord(m->dp_ev[dp_base - 1], st));
   }
   FT_LAUNCH(FT_PROF_NORM, 6.0 * T * h,
-            rmsnorm_bwd(m->d_hF, m->x[L], m->rF, m->wb(i_normf), m->cfg.mtp ? m->mtp_d_xL : nullptr, m->dxA, m->gr(i_normf),
-                        m->norm_partial, T, h, st));
+            rmsnorm_bwd(m->d_hF, m->x[L], m->rF, m->wb(i_normf), m->cfg.mtp ? m->mtp_d_xL : nullptr, m->dxA, norm_slot(m, i_normf), T, h, st));
   for (int l = L - 1; l >= 0; --l) {
     LayerActs& a = m->acts[m->cfg.recompute ? 0 : l];
     if (m->cfg.recompute) {
@@ -797,6 +837,9 @@ ft_status run_forward_backward(ft_model* m, const int32_t* tok, const int32_t* l
     if (s) return s;
     if (m->dp_mode) FT_CUDA(cudaEventRecord(m->dp_ev[dp_base + (L - 1 - l)], st));
   }
+  // every RMSNorm gain's gradient: block partials of all norms summed in one launch
+  FT_LAUNCH(FT_PROF_NORM, 4.0 * m->n_norm_slots * (double)elementwise_blocks_for_norm(T) * h,
+            colsum_many(m->norm_partial, m->norm_out, m->n_norm_slots, (size_t)elementwise_blocks_for_norm(m->maxT) * h, T, h, st));
   FT_LAUNCH(FT_PROF_ELEMENTWISE, 2.0 * T * h + 4.0 * V * h, embed_bwd(tok, m->dxA, m->gr(0), m->keys, T, h, V, m->cfg.emb_scale, tied || m->cfg.mtp, st));
   for (int k = 0; k < 4; ++k) { ft_status sw = wait_wgrad(m, k); if (sw) return sw; }  // join the second stream
   if (m->dp_mode) {  // the embedding table and the gains (summed over the whole pass) are complete only now
@@ -1054,6 +1097,13 @@ ft_status ft_init_model(const ft_config* cfg, uint64_t seed, void* dev_workspace
     FT_CUDA(cudaMemsetAsync(m->grad, 0, m->arena * sizeof(float), st));
   }
 
+  {
+    std::vector<float*> outs((size_t)m->n_norm_slots, nullptr);
+    for (size_t i = 0; i < m->params.size(); ++i)
+      if (m->norm_slot_of[i] >= 0) outs[(size_t)m->norm_slot_of[i]] = m->gr((int)i);
+    FT_CUDA(cudaMemcpyAsync(m->norm_out, outs.data(), outs.size() * sizeof(float*), cudaMemcpyHostToDevice, st));
+    FT_CUDA(cudaStreamSynchronize(st));
+  }
   {
     ft_status sr = build_rope_tables(m, nullptr, 1.0f);
     if (sr) return sr;
@@ -1554,6 +1604,7 @@ void ft_debug_gemm_tile(int32_t bn) { g_gemm_force_bn = bn; }
 void ft_debug_gemm_balanced(int32_t on) { g_gemm_balanced = on; }
 void ft_debug_pdl(int32_t on) { g_pdl = on; }
 void ft_debug_gemm_pairs(int32_t on) { g_gemm_pairs = on; }
+void ft_debug_head_dz_limit(uint64_t bytes) { g_head_dz_limit = (size_t)bytes; }
 
 ft_status ft_debug_wait_probe(ft_model* m, int64_t limit_cycles) {
   if (!m) return FT_EINVAL;

@@ -1,10 +1,12 @@
 """Parity at full benchmark size (workloads c2 ... c5 at the sizes and launch configuration bench.py times).
 
-A whole oracle step at this size is hours of fp64 work, so every kernel of the step is checked on SAMPLED outputs
-that the oracle can compute one by one from that kernel's actual inputs (read back through the tap interface):
-row-local operators on sampled token rows, attention on sampled (batch, head, position) triples, weight gradients
-on sampled entries (full contraction over all 8192 tokens), plus properties that hold at any size (loss at
-initialisation, bit-identical repeat).  Tolerance: the stated rel-L2 <= 2e-2 per sampled tensor.
+Whole oracle steps at full size are stored results (tests/test_full_size_golden_gpu.py, c2 and c3).  Here every kernel
+of the step, at all four workloads, is checked on SAMPLED outputs that the oracle's own functions compute from that
+kernel's actual inputs (read back through the tap interface): row-local operators on sampled token rows (D.rmsnorm_fwd /
+_bwd, D.rope_apply, D.swiglu_fwd / _bwd, plain contractions), attention forward and backward on whole (batch, kv group)
+slices through D.attention_fwd / D.attention_bwd, weight gradients on sampled entries (full contraction over all
+tokens), plus properties that hold at any size (loss at initialisation, bit-identical repeat).  Tolerance: the stated
+rel-L2 <= 2e-2 per sampled tensor.
 """
 import math
 
@@ -86,11 +88,8 @@ def test_row_local_forward_and_backward_operators_on_sampled_rows(run, which):
     assert rel_l2(h1, R(y)) < TOL
     acc = h1 @ Wb["wqkv"].T
 
-    def rot(block, nheads):
-        z = block.reshape(len(rows), nheads, d)
-        c, s = cos[posn][:, None, :], sin[posn][:, None, :]
-        z1, z2 = z[..., :d // 2], z[..., d // 2:]
-        return np.concatenate([z1 * c - z2 * s, z2 * c + z1 * s], -1).reshape(len(rows), nheads * d)
+    def rot(block, nheads):  # the oracle's rotation, with the table rows of the sampled positions
+        return D.rope_apply(block.reshape(len(rows), nheads, d), cos[posn], sin[posn]).reshape(len(rows), nheads * d)
 
     want_qkv = np.concatenate([rot(acc[:, :hq], ocfg.n_heads), rot(acc[:, hq:hq + hkv], ocfg.n_kv_heads),
                                acc[:, hq + hkv:]], 1)
@@ -101,15 +100,15 @@ def test_row_local_forward_and_backward_operators_on_sampled_rows(run, which):
     GU = R(h2 @ Wb["wgu"].T)
     assert rel_l2(gu, GU) < TOL
     G, U = gu[:, :f], gu[:, f:]
-    assert rel_l2(a, R(G * D.sigmoid(G) * U)) < TOL
+    assert rel_l2(a, R(D.swiglu_fwd(G, U))) < TOL
     assert rel_l2(x_out, R(x_mid + a @ Wb["wd"].T)) < TOL
 
     # backward, each operator from its own inputs
     d_x_out, d_a, d_gu, d_h2 = tap("d_x_out", h), tap("d_a", f), tap("d_gu", 2 * f), tap("d_h2", h)
     d_x_mid, d_o, d_qkv, d_h1, d_x_in = tap("d_x_mid", h), tap("d_o", hq), tap("d_qkv", nq), tap("d_h1", h), tap("d_x_in", h)
     assert rel_l2(d_a, R(d_x_out @ Wb["wd"])) < TOL
-    sg = D.sigmoid(G)
-    want = np.concatenate([R(d_a * U * sg * (1 + G * (1 - sg))), R(d_a * G * sg)], 1)
+    dG, dU = D.swiglu_bwd(d_a, G, U)
+    want = np.concatenate([R(dG), R(dU)], 1)
     assert rel_l2(d_gu, want) < TOL
     assert rel_l2(d_h2, R(d_gu @ Wb["wgu"])) < TOL
     dxn, _ = D.rmsnorm_bwd(d_h2, x_mid, r2, Wb["norm2"])
@@ -120,66 +119,50 @@ def test_row_local_forward_and_backward_operators_on_sampled_rows(run, which):
     assert rel_l2(d_x_in, R(d_x_mid + dxn)) < TOL
 
 
-def test_attention_forward_and_backward_on_sampled_positions(run):
+def test_attention_forward_and_backward_on_whole_kv_group_slices(run):
+    """The oracle's attention functions on the library's own inputs: for sampled (batch row, kv head) pairs the slice
+    holding that kv head and the query heads that share it goes through D.attention_fwd (o, LSE at every position) and,
+    with the library's o, LSE and d_o, through D.attention_bwd, D.rope_apply_transpose and the rounding (d_q, d_k, d_v
+    at every position)."""
     m, ocfg, w = run["model"], run["ocfg"], run["w"]
     Bsz, S = w["batch"], w["seq"]
-    T, hq, hkv, d, nh, nkv = Bsz * S, ocfg.h_q, ocfg.h_kv, ocfg.head_dim, ocfg.n_heads, ocfg.n_kv_heads
+    hq, hkv, d, nh, nkv = ocfg.h_q, ocfg.h_kv, ocfg.head_dim, ocfg.n_heads, ocfg.n_kv_heads
     nq, n_rep = hq + 2 * hkv, nh // nkv
     R = D.bf16_round
     layer = ocfg.n_layers // 4
-    qkv = m.get_tap("qkv", layer).reshape(Bsz, S, nq).astype(np.float64)
-    o = m.get_tap("o", layer).reshape(Bsz, S, nh, d).astype(np.float64)
-    lse = m.get_tap("attn_lse", layer).reshape(Bsz, nh, S).astype(np.float64)
-    d_o = m.get_tap("d_o", layer).reshape(Bsz, S, nh, d).astype(np.float64)
-    d_qkv = m.get_tap("d_qkv", layer).reshape(Bsz, S, nq).astype(np.float64)
+    qkv = m.get_tap("qkv", layer).reshape(Bsz, S, nq)
+    o = m.get_tap("o", layer).reshape(Bsz, S, nh, d)
+    lse = m.get_tap("attn_lse", layer).reshape(Bsz, nh, S)
+    d_o = m.get_tap("d_o", layer).reshape(Bsz, S, nh, d)
+    d_qkv = m.get_tap("d_qkv", layer).reshape(Bsz, S, nq)
     cos, sin = D.rope_tables(S, d, ocfg.rope_theta)
-    scale = 1.0 / math.sqrt(d)
-    got_o, want_o, got_dq, want_dq, got_l, want_l = [], [], [], [], [], []
-    samples = [(0, 0, 0), (0, 5, 63), (1, 15, 64), (2, 9, 127), (3, 2, 128), (1, 7, S // 2 - 24), (2, 12, S - 1),
-               (3, 0, (3 * S) // 4 - 5)]
-    for b, n, t in [(bb % Bsz, nn % nh, tt) for bb, nn, tt in samples]:
-        g = n // n_rep
-        q = qkv[b, t, n * d:(n + 1) * d]
-        k = qkv[b, :t + 1, hq + g * d:hq + (g + 1) * d]
-        v = qkv[b, :t + 1, hq + hkv + g * d:hq + hkv + (g + 1) * d]
-        s2 = (k @ q) * scale * D.LOG2E
-        c = math.ceil(s2.max())
-        pt = np.exp2(s2 - c)
-        want_o.append(R((R(pt) @ v) / pt.sum()))
-        got_o.append(o[b, t, n])
-        want_l.append((c + math.log2(pt.sum())) * D.LN2)
-        got_l.append(lse[b, n, t])
-        # dq of the same row: P from the stored LSE, dS rounded, rotated back, rounded
-        p = np.exp((k @ q) * scale - lse[b, n, t])
-        dl = float(d_o[b, t, n] @ o[b, t, n])
-        ds = R(p * (v @ d_o[b, t, n] - dl))
-        dq = (ds @ k) * scale
-        dq = D.rope_apply_transpose(dq[None, None, None, :], cos[t:t + 1], sin[t:t + 1])[0, 0, 0]
-        want_dq.append(R(dq))
-        got_dq.append(d_qkv[b, t, n * d:(n + 1) * d])
-    assert rel_l2(np.array(got_o), np.array(want_o)) < TOL
-    assert np.max(np.abs(np.array(got_l) - np.array(want_l))) < 1e-4
-    assert rel_l2(np.array(got_dq), np.array(want_dq)) < TOL
-    # dk, dv of sampled keys: sums over every later query of the two query heads sharing the kv head
-    got, want = [], []
-    for b, g, j in [(bb % Bsz, gg % nkv, jj) for bb, gg, jj in [(0, 0, S - 1), (1, 3, S - 58), (2, 7, S // 2), (3, 5, 17)]]:
-        kj = qkv[b, j, hq + g * d:hq + (g + 1) * d]
-        vj = qkv[b, j, hq + hkv + g * d:hq + hkv + (g + 1) * d]
-        dk = np.zeros(d)
-        dv = np.zeros(d)
-        for n in range(g * n_rep, (g + 1) * n_rep):
-            qs = qkv[b, j:, n * d:(n + 1) * d]
-            p = np.exp((qs @ kj) * scale - lse[b, n, j:])
-            dos = d_o[b, j:, n]
-            dl = np.sum(dos * o[b, j:, n], axis=1)
-            ds = R(p * (dos @ vj - dl))
-            dv += R(p) @ dos
-            dk += (ds @ qs) * scale
-        dk = D.rope_apply_transpose(dk[None, None, None, :], cos[j:j + 1], sin[j:j + 1])[0, 0, 0]
-        want.append(np.concatenate([R(dk), R(dv)]))
-        got.append(np.concatenate([d_qkv[b, j, hq + g * d:hq + (g + 1) * d],
-                                   d_qkv[b, j, hq + hkv + g * d:hq + hkv + (g + 1) * d]]))
-    assert rel_l2(np.array(got), np.array(want)) < TOL
+    for b, g in {(0, 0), ((Bsz - 1), nkv - 1)} if S > 8192 else {(0, 0), (Bsz - 1, nkv - 1), (Bsz // 2, nkv // 2)}:
+        heads = slice(g * n_rep, (g + 1) * n_rep)
+        f64 = lambda x: np.ascontiguousarray(x, dtype=np.float64)
+        q = f64(qkv[b:b + 1, :, :hq].reshape(1, S, nh, d)[:, :, heads])
+        k = f64(qkv[b:b + 1, :, hq:hq + hkv].reshape(1, S, nkv, d)[:, :, g:g + 1])
+        v = f64(qkv[b:b + 1, :, hq + hkv:].reshape(1, S, nkv, d)[:, :, g:g + 1])
+        want_o, want_lse = D.attention_fwd(q, k, v, n_rep, R, True)
+        got_o, got_lse = f64(o[b:b + 1, :, heads]), f64(lse[b:b + 1, heads])
+        assert rel_l2(got_o, want_o) < TOL, (b, g)
+        assert np.max(np.abs(got_lse - want_lse)) < 1e-4, (b, g)
+        dq, dk, dv = D.attention_bwd(q, k, v, got_o, f64(d_o[b:b + 1, :, heads]), got_lse, n_rep, R)
+        dq = R(D.rope_apply_transpose(dq, cos, sin))
+        dk = R(D.rope_apply_transpose(dk, cos, sin))
+        dv = R(dv)
+        got_dq = f64(d_qkv[b:b + 1, :, :hq].reshape(1, S, nh, d)[:, :, heads])
+        got_dk = f64(d_qkv[b:b + 1, :, hq:hq + hkv].reshape(1, S, nkv, d)[:, :, g:g + 1])
+        got_dv = f64(d_qkv[b:b + 1, :, hq + hkv:].reshape(1, S, nkv, d)[:, :, g:g + 1])
+        assert rel_l2(got_dq, dq) < TOL and rel_l2(got_dk, dk) < TOL and rel_l2(got_dv, dv) < TOL, (b, g)
+        # and position by position for the first and the last queries and keys (a tile-boundary slip would hide in a norm)
+        for t in (0, 1, 63, 64, 127, 128, S // 2, S - 129, S - 1):
+            assert rel_l2(got_o[0, t], want_o[0, t]) < TOL, (b, g, t)
+            if t == 0:  # the first query sees one key: o = v, so dS = P (dP - delta) = 0 and d_q vanishes identically;
+                # what the kernel leaves there is the fp32 cancellation noise of dP - delta
+                assert np.max(np.abs(got_dq[0, 0])) < 0.05 * np.max(np.abs(got_dq[0, 1:64])), (b, g)
+            else:
+                assert rel_l2(got_dq[0, t], dq[0, t]) < 2 * TOL, (b, g, t)
+            assert rel_l2(got_dk[0, t], dk[0, t]) < 2 * TOL, (b, g, t)
 
 
 def test_head_loss_and_weight_gradients_on_sampled_entries(run):

@@ -127,6 +127,29 @@ def test_default_path_without_taps_matches_oracle_on_loss_every_gradient_and_mas
     _check_step(ocfg, tok, lab, params, debug=False, recompute=recompute)
 
 
+@pytest.mark.parametrize("one_pass", [True, False])
+def test_output_head_over_several_row_chunks_matches_oracle_in_both_forms(one_pass):
+    """5 x 1024 tokens: the logits are formed in two chunks of rows (4096 + 1024).  By default the logit gradient of all
+    rows is kept and the head's data and weight gradients are one contraction each over all rows; with the buffer limit
+    at 0 they are formed per chunk and the weight gradient accumulates in memory.  Both against the oracle: loss, hF, the
+    log-sum-exp of every row, d_hF, every gradient, masters."""
+    import ctypes as C
+    from paper_2609_13645_b200 import binding as B
+    ocfg, _ = _c1()
+    params = D.init_params(ocfg, SI.WEIGHT_SEED)
+    tok, lab = SI.batch(ocfg.vocab, 5, 1024, "zipf", seed=3)
+    lab = lab.copy()
+    lab[4, 1000:] = -1
+    L = B.lib()
+    L.ft_debug_head_dz_limit.argtypes = [C.c_uint64]
+    L.ft_debug_head_dz_limit.restype = None
+    L.ft_debug_head_dz_limit(C.c_uint64(4 << 30 if one_pass else 0))
+    try:
+        _check_step(ocfg, tok, lab, params)
+    finally:
+        L.ft_debug_head_dz_limit(C.c_uint64(4 << 30))
+
+
 @pytest.mark.parametrize("variant", ["mtp", "mtp+tied+qknorm+mup", "mtp+ragged+streaming"])
 def test_mtp_head_step_matches_oracle_on_loss_every_gradient_and_master(variant):
     """The one-layer MTP (Eagle) head of the paper's 1B configuration: the normalised last hidden state and the normalised
