@@ -645,17 +645,32 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
           rp[i] = __float_as_uint(p * (__uint_as_float(rp[i]) - delta_row));
         }
       } else {
+        if (full) {
 #pragma unroll
-        for (int i = 0; i < 32; i += 4) {
-          const float4 l4 = *reinterpret_cast<const float4*>(st_lse + i);
-          const float4 d4 = *reinterpret_cast<const float4*>(st_dl + i);
-          const float ll[4] = {l4.x, l4.y, l4.z, l4.w}, dd[4] = {d4.x, d4.y, d4.z, d4.w};
+          for (int i = 0; i < 32; i += 4) {
+            const float4 l4 = *reinterpret_cast<const float4*>(st_lse + i);
+            const float4 d4 = *reinterpret_cast<const float4*>(st_dl + i);
+            const float ll[4] = {l4.x, l4.y, l4.z, l4.w}, dd[4] = {d4.x, d4.y, d4.z, d4.w};
 #pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            float p = fast_exp2(fmaf(__uint_as_float(rs[i + u]), scale_log2, -ll[u]));
-            if (!full && (cmin + i + u < row || cmin + i + u >= S)) p = 0.f;
-            rs[i + u] = __float_as_uint(p);
-            rp[i + u] = __float_as_uint(p * (__uint_as_float(rp[i + u]) - dd[u]));
+            for (int u = 0; u < 4; ++u) {
+              const float p = fast_exp2(fmaf(__uint_as_float(rs[i + u]), scale_log2, -ll[u]));
+              rs[i + u] = __float_as_uint(p);
+              rp[i + u] = __float_as_uint(p * (__uint_as_float(rp[i + u]) - dd[u]));
+            }
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; i += 4) {
+            const float4 l4 = *reinterpret_cast<const float4*>(st_lse + i);
+            const float4 d4 = *reinterpret_cast<const float4*>(st_dl + i);
+            const float ll[4] = {l4.x, l4.y, l4.z, l4.w}, dd[4] = {d4.x, d4.y, d4.z, d4.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              float p = fast_exp2(fmaf(__uint_as_float(rs[i + u]), scale_log2, -ll[u]));
+              if (cmin + i + u < row || cmin + i + u >= S) p = 0.f;
+              rs[i + u] = __float_as_uint(p);
+              rp[i + u] = __float_as_uint(p * (__uint_as_float(rp[i + u]) - dd[u]));
+            }
           }
         }
       }
