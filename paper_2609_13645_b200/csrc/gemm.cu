@@ -1354,7 +1354,11 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream, int* lau
   const int left = tiles % max_pairs;
   p.ce_mode = MODE == 1 ? a.ce_mode : 0; p.ce_tiles = a.ce_tiles; p.ce_part = a.ce_part; p.ce_zy = a.ce_zy; p.ce_lse = a.ce_lse;
   p.ce_labels = a.ce_labels; p.ce_sc = a.ce_scalars; p.ce_scale = a.ce_scale;
-  if (MODE != 1 && g_gemm_balanced && ksplit == 1 && data && tiles > max_pairs && left > 0 && max_pairs <= 256 &&
+  // Only for contractions of at least 40 K blocks: a divided tile costs its pairs a pass of the fp32 partial through
+  // scratch (4.6 us written, then read by the reducing pair) before the whole tiles start.  Against a 3 us main loop
+  // (K 768) that makes the launch slower (8192 x 768 x 768: 37 against 29 us), at K 2048 it is a wash to a loss
+  // (8192 x 2048 x 2048: 67.5 against 62.6 us), from K 4096 on it wins (8192 x 2048 x 11264: 230 against 249 us).
+  if (MODE != 1 && g_gemm_balanced && ksplit == 1 && data && tiles > max_pairs && left > 0 && max_pairs <= 256 && kblocks >= 40 &&
       (size_t)max_pairs * SLOT_FLOATS * sizeof(float) <= data_bytes) {
     int parts = max_pairs / left;
     // The pair with part 0 adds the other parts' tiles while its next tile's main loop runs; the longer that loop (K),

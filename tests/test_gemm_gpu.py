@@ -128,10 +128,11 @@ def test_split_k_weight_gradient_matches_the_contraction_and_repeats_bit_for_bit
     assert np.linalg.norm(got1 - ref) / np.linalg.norm(ref) < 1e-5
 
 
-# Shapes with more 256 x 256 tiles than the 74 SM pairs and a last wave of at most 37 tiles: the balanced schedule
-# divides that wave into 2 .. 8 K parts.  Ragged M, N and K (parts of unequal length) included.
-BALANCED = [(2048, 2560, 512), (2048, 2560, 1024), (4096, 4096, 520), (2000, 2568, 1000), (8192, 2048, 704),
-            (2304, 2304, 2048), (2560, 2560, 512)]
+# Shapes with more 256 x 256 tiles than the 74 SM pairs, a last wave of at most 37 tiles and a contraction of at least 40
+# K blocks (K >= 2560): the balanced schedule divides that wave into 2 .. 8 K parts.  Ragged M, N and K (parts of unequal
+# length) included; the last two shapes stay below the K limit and take the plain schedule with the same scratch.
+BALANCED = [(2048, 2560, 2560), (2048, 2560, 4096), (4096, 4096, 2600), (2000, 2568, 3000), (8192, 2048, 2816),
+            (2304, 2304, 6144), (2560, 2560, 8192), (2048, 2560, 1024), (8192, 2048, 704)]
 
 
 @pytest.mark.parametrize("M,N,K", BALANCED)
@@ -149,7 +150,7 @@ def test_balanced_k_schedule_matches_the_contraction(M, N, K, a_mn, b_mn, kind):
 
 def test_balanced_k_schedule_repeats_bit_for_bit_and_leaves_its_counters_clear():
     from paper_2609_13645_b200 import binding as B
-    M, N, K = 2048, 2560, 1024
+    M, N, K = 2048, 2560, 4096
     rng = np.random.default_rng(5)
     _, At = _bf16_tensor(rng, (M, K))
     _, Bt = _bf16_tensor(rng, (N, K))

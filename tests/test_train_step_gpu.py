@@ -579,9 +579,9 @@ def test_adamw_inside_the_weight_gradient_epilogue_equals_the_separate_optimizer
     elif shape == "split_k":   # weight gradients with few tiles and 2048 tokens: K split over 4 parts
         ocfg = oracle_config(n_layers=2, d_model=512, n_heads=4, n_kv_heads=2, head_dim=128, d_ffn=1024, vocab=2048)
         Bsz, S = 2, 1024
-    else:                      # gate/up gradient of 18 x 5 = 90 tiles: the 16 tiles past the 74 pairs are divided
+    else:                      # gate/up gradient of 18 x 5 = 90 tiles over 3072 tokens (48 K blocks): the 16 tiles past the 74 pairs are divided
         ocfg = oracle_config(n_layers=1, d_model=1280, n_heads=10, n_kv_heads=2, head_dim=128, d_ffn=2304, vocab=2048)
-        Bsz, S = 1, 1024
+        Bsz, S = 3, 1024
     runs = []
     for fused in (True, False):
         model = B.Model(lib_config(B, ocfg, Bsz, S), seed=3)
@@ -620,8 +620,8 @@ def test_swiglu_backward_inside_the_data_gradient_epilogue_changes_no_bit(shape)
     elif shape == "one_cta":
         ocfg = oracle_config(n_layers=2, d_model=256, n_heads=4, n_kv_heads=2, head_dim=64, d_ffn=1040, vocab=1024)
         Bsz, S = 1, 136
-    elif shape == "balanced":  # 8 x 10 = 80 tiles of d_a on 74 pairs: the last 6 are divided along K
-        ocfg = oracle_config(n_layers=1, d_model=1280, n_heads=10, n_kv_heads=2, head_dim=128, d_ffn=2560, vocab=2048)
+    elif shape == "balanced":  # 8 x 10 = 80 tiles of d_a on 74 pairs, contraction over d_model = 2560 (40 K blocks): the last 6 are divided along K
+        ocfg = oracle_config(n_layers=1, d_model=2560, n_heads=20, n_kv_heads=4, head_dim=128, d_ffn=2560, vocab=2048)
         Bsz, S = 2, 1024
     else:
         ocfg = oracle_config(n_layers=3, d_model=512, n_heads=4, n_kv_heads=2, head_dim=128, d_ffn=1024, vocab=2048,
