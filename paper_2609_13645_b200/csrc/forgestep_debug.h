@@ -18,6 +18,9 @@ void ft_debug_gemm_tile(int32_t bn);
 void ft_debug_gemm_pairs(int32_t on);
 /* 1 = balanced-K schedule where it applies and scratch is available (default), 0 = round-robin tiles. */
 void ft_debug_gemm_balanced(int32_t on);
+/* 1 = the SwiGLU-backward epilogue of the CTA-pair GEMM moves gate / up and d_gate / d_up as TMA tiles through shared
+ * memory (default), 0 = one row per thread with plain loads and stores.  Both give the same bits. */
+void ft_debug_gemm_swiglu_tma(int32_t on);
 /* 1 = kernels are launched with programmatic stream serialization (programmatic dependent launch: appendix "Optimization Catalog", "Cross-kernel scheduling"), the default; 0 = ordinary stream
  * order.  Graphs captured under one setting keep it. */
 void ft_debug_pdl(int32_t on);

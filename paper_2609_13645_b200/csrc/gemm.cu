@@ -17,6 +17,7 @@ namespace fs {
 
 int g_pdl = 1;
 int g_gemm_balanced = 1;  // development knob: 0 = always the round-robin tile schedule
+int g_gemm_swiglu_tma = 1;  // development knob: 0 = SwiGLU-backward epilogue with per-thread loads and stores
 
 namespace {
 
@@ -60,6 +61,7 @@ struct GemmDev {
   int panel;               // tile numbering (see tile_coords)
   float alpha;             // accumulator scale (1: off)
   int wide_store;          // 1: C, ldc and N allow 32-byte stores (bf16 output)
+  int swiglu_tma;          // SwiGLU-backward epilogue of the pair kernel: gate/up in and d_gate/d_up out as TMA tiles
   float* qk_r;             // per-head QK-Norm in the RoPE epilogue (null: off)
   const bf16* qk_gain_q;
   const bf16* qk_gain_k;
@@ -940,6 +942,92 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
 }
 
+// Tensor maps of an epilogue that moves its tiles through the TMA unit (SwiGLU backward): the forward pass' gate | up
+// [T, 2f] in boxes of 32 rows x 32 columns, and the output d_gate / d_up (interleaved 16 | 16) in boxes of 32 x 64.
+struct EpiMaps {
+  CUtensorMap gu;
+  CUtensorMap dgu;
+};
+
+// One warp's load of the gate and up tiles (32 rows x 32 logical columns from column gc) into its staging buffer
+__device__ __forceinline__ void swiglu_bwd_tma_fetch(const GemmDev& p, const EpiMaps& em, uint32_t buf, uint32_t bar, int gc,
+                                                     int row0) {
+  mbar_expect_tx(bar, 4096);
+  tma_load_2d(buf, &em.gu, bar, gc, row0);
+  tma_load_2d(buf + 2048, &em.gu, bar, p.d_ffn + gc, row0);
+}
+
+// SwiGLU backward with the epilogue's memory traffic on the TMA unit.  The register path above reads gate and up and
+// writes d_gate and d_up with one row per thread, four times the bytes of a plain bf16 epilogue in 32-byte requests that
+// each are a wavefront of their own in the load/store pipe (half of that pipe's peak over the whole kernel).  Here a
+// warp's 32 rows x 32 columns of gate and of up arrive as two TMA boxes (64-byte rows, 64-byte swizzle) on the warp's own
+// mbarrier, the threads read their row from shared memory without bank conflicts, and the 32 x 64 output tile (128-byte
+// rows, 128-byte swizzle) leaves as one TMA store.  The load of chunk c + 1 is issued as soon as chunk c sits in
+// registers; the store of chunk c drains while chunk c + 1 is computed.  Same element function, same roundings:
+// bit-identical to the register path.  Measured at 8192 x 5632 x 2048: 176 -> 168 us alone, 210 -> 199 us inside the c3_1b
+// step; the load/store pipe falls to 13 % of its peak, and what remains over the plain data gradient (124 us) is the
+// epilogue's bytes themselves on the L2-to-SM path that the operand loads already fill.
+// buf: 8 KB, 1024-byte aligned: gate, up, output tile.  Returns false when a bounded wait ran out.
+__device__ __forceinline__ bool epilogue_swiglu_bwd_tma(const GemmDev& p, const EpiMaps& em, uint32_t taddr, int row0, int n0,
+                                                        int cb, int ce, const Fixup& fx, uint32_t buf, uint32_t bar,
+                                                        uint32_t& phase, volatile int* abort_flag) {
+  const int lane = threadIdx.x & 31;
+  const uint32_t in_row = buf + (uint32_t)lane * 64u, sw_in = (uint32_t)((lane >> 1) & 3);
+  const uint32_t out_row = buf + 4096u + (uint32_t)lane * 128u, sw_out = (uint32_t)(lane & 7);
+  uint32_t r[32];
+  for (int c = cb; c < ce; c += 32) {
+    const int gc = n0 + c;
+    if (gc >= p.N) break;
+    bool ok = mbar_wait(bar, phase, abort_flag, p.err);
+    ok = __all_sync(0xffffffffu, ok);
+    if (!ok) return false;
+    phase ^= 1u;
+    uint4 cG[4], cU[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      cG[j] = ld_shared_v4(in_row + (((uint32_t)j ^ sw_in) << 4));
+      cU[j] = ld_shared_v4(in_row + 2048u + (((uint32_t)j ^ sw_in) << 4));
+    }
+    __syncwarp();
+    if (lane == 0 && c + 32 < ce && gc + 32 < p.N) swiglu_bwd_tma_fetch(p, em, buf, bar, gc + 32, row0);
+    ld_acc32(taddr, c, r, fx, p.alpha);
+    uint32_t o[32];  // the thread's 128-byte output row: [16 d_gate | 16 d_up] twice
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+      float dG[16], dU[16];
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        const uint4 g4 = cG[2 * hh + q], u4 = cU[2 * hh + q];
+        const uint32_t gw[4] = {g4.x, g4.y, g4.z, g4.w}, uw[4] = {u4.x, u4.y, u4.z, u4.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int j = 16 * hh + 8 * q + 2 * e;
+          swiglu_bwd_elem(round_bf16(__uint_as_float(r[j])), bf16_lo(gw[e]), bf16_lo(uw[e]), dG[8 * q + 2 * e], dU[8 * q + 2 * e]);
+          swiglu_bwd_elem(round_bf16(__uint_as_float(r[j + 1])), bf16_hi(gw[e]), bf16_hi(uw[e]), dG[8 * q + 2 * e + 1],
+                          dU[8 * q + 2 * e + 1]);
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        o[16 * hh + i] = pack_bf16(dG[2 * i], dG[2 * i + 1]);
+        o[16 * hh + 8 + i] = pack_bf16(dU[2 * i], dU[2 * i + 1]);
+      }
+    }
+    if (lane == 0) bulk_wait_group_read0();  // the previous chunk's store has read the output tile
+    __syncwarp();
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      st_shared_v4(out_row + (((uint32_t)j ^ sw_out) << 4), make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]));
+    fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+      tma_store_2d(&em.dgu, buf + 4096u, 2 * gc, row0);
+      bulk_commit_group();
+    }
+  }
+  return true;
+}
+
 // ---------------------------------------------------------------- CTA-pair variant
 // Two CTAs on neighbouring SMs (a cluster of 2) share one 256 x 256 output tile: each loads its own 128 rows of A and
 // its own 128 of the 256 rows of B, the leader issues tcgen05.mma.cta_group::2 (M = 256), and each CTA's TMEM ends up
@@ -952,8 +1040,9 @@ struct PairCfg {
   static constexpr int B_BYTES = HALF_B * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES_ + B_BYTES;
   static constexpr int STAGES = 6;
+  static constexpr int EPI_BYTES = EPI_STAGE_BYTES;
   static constexpr int TMEM_COLS = 512;
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 256 + EPI_STAGE_BYTES + 1024;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 256 + EPI_BYTES + 1024;
 };
 
 // Warps: TMA producer, MMA issuer, then the epilogue warps.  Launched with 192 threads there are four (one per TMEM lane
@@ -964,12 +1053,15 @@ constexpr int PAIR_THREADS = 320;
 
 template <bool A_MN, bool B_MN, int MODE = 0>
 __global__ void __launch_bounds__(PAIR_THREADS, 1)
-gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmDev p) {
+gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                    const __grid_constant__ EpiMaps em, const GemmDev p) {
   using C = PairCfg;
   constexpr int BN = C::BN;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::STAGES * C::STAGE_BYTES);
+  // operand stages, then the epilogue warps' staging area (1024-byte aligned, as swizzled TMA tiles need), then barriers
+  uint8_t* epi_stage = smem + C::STAGES * C::STAGE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(epi_stage + C::EPI_BYTES);
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (C::STAGES + s); };
@@ -977,6 +1069,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * C::STAGES + 2 + b); };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * C::STAGES + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  auto epi_ld_bar = [&](int w) { return bar0 + 8u * (2 * C::STAGES + 6 + w); };  // one per epilogue warp (TMA epilogue loads)
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -992,10 +1085,15 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       mbar_init(tfull_bar(b), 1);   // one commit, arriving in both CTAs
       mbar_init(tempty_bar(b), 2 * (blockDim.x / 32 - 2));  // the epilogue warps of both CTAs, all arriving at the leader
     }
+    if constexpr (MODE == 2)
+      for (int w = 0; w < 4; ++w) mbar_init(epi_ld_bar(w), 1);
     *abort_flag = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmA);
     tma_prefetch_desc(&tmB);
+    if constexpr (MODE == 2) {
+      if (p.swiglu_tma) { tma_prefetch_desc(&em.gu); tma_prefetch_desc(&em.dgu); }
+    }
   }
   if (warp == 1) {
     tmem_alloc_pair(smem_u32(tmem_slot), C::TMEM_COLS);
@@ -1091,7 +1189,14 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const int ncols = blockDim.x == PAIR_THREADS ? 128 : 256;  // columns of the tile per epilogue warp
     const int cb = ((warp - 2) >> 2) * ncols;
     const int ce = cb + ncols;
-    float* stage = reinterpret_cast<float*>(smem + C::STAGES * C::STAGE_BYTES + 256) + (warp - 2) * EPI_STAGE_FLOATS;
+    float* stage = reinterpret_cast<float*>(epi_stage) + (warp - 2) * EPI_STAGE_FLOATS;
+    // SwiGLU backward through the TMA unit: four epilogue warps, 8 KB of the staging area and one load barrier each.
+    // (Eight warps with 8 KB each, paid for with one of the six operand stages, were no faster: 206 against 199 us per
+    // launch at c3_1b.  What this epilogue costs is its bytes on the L2-to-SM path, which the operand loads fill.)
+    [[maybe_unused]] const bool tma_epi = MODE == 2 && p.swiglu_tma != 0 && blockDim.x == GEMM_THREADS;
+    [[maybe_unused]] const uint32_t tbuf = smem_u32(epi_stage) + (uint32_t)((warp - 2) & 3) * 8192u;
+    [[maybe_unused]] const uint32_t tbar = epi_ld_bar((warp - 2) & 3);
+    [[maybe_unused]] uint32_t tphase = 0;
     int acc = 0;
     uint32_t acc_phase = 0;
     float sq = 0.f;  // fused AdamW: this thread's share of the squared gradient norm
@@ -1106,7 +1211,11 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const bool reducer = !split || part == p.sw_parts - 1;  // this piece ends in the tile's epilogue
       if (p.adam_p != nullptr && reducer) adam_prefetch_chunk(p, p.C, m0 + q * 32 + lane, n0 + cb);
       // (asking one piece earlier instead, from the previous piece's epilogue, was slower: 219 us against 201 at c3_1b)
-      if constexpr (MODE == 2) { if (reducer) swiglu_bwd_prefetch(p, m0 + q * 32 + lane, n0 + cb, ncols); }
+      [[maybe_unused]] const bool tma_tile = tma_epi && reducer && m0 + q * 32 < p.M && n0 + cb < p.N;
+      if constexpr (MODE == 2) {
+        if (reducer) swiglu_bwd_prefetch(p, m0 + q * 32 + lane, n0 + cb, ncols);
+        if (tma_tile && lane == 0) swiglu_bwd_tma_fetch(p, em, tbuf, tbar, n0 + cb, m0 + q * 32);
+      }
       bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.err);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -1149,7 +1258,15 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         } else if (p.ksplit > 1) {
           cptr = reinterpret_cast<float*>(p.C) + (long long)part * p.split_stride;  // this K part's own fp32 partial output
         }
-        epilogue_tile<BN, MODE>(p, cptr, taddr, row, n0, sq, stage, cb, ce, fx);
+        if constexpr (MODE == 2) {
+          if (tma_epi) {
+            if (tma_tile && !epilogue_swiglu_bwd_tma(p, em, taddr, m0 + q * 32, n0, cb, ce, fx, tbuf, tbar, tphase, abort_flag)) break;
+          } else {
+            epilogue_tile<BN, MODE>(p, cptr, taddr, row, n0, sq, stage, cb, ce, fx);
+          }
+        } else {
+          epilogue_tile<BN, MODE>(p, cptr, taddr, row, n0, sq, stage, cb, ce, fx);
+        }
       }
       tc_fence_before();
       __syncwarp();
@@ -1162,6 +1279,9 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (p.adam_p != nullptr) {
       sq = warp_sum(sq);
       if (lane == 0) p.adam_sq[blockIdx.x * 8 + (warp - 2)] = sq;
+    }
+    if constexpr (MODE == 2) {
+      if (tma_epi && lane == 0) bulk_wait_group0();  // this warp's tensor stores have landed before the kernel ends
     }
   }
 
@@ -1293,6 +1413,7 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
   p.qk_r = a.qk_r; p.qk_gain_q = a.qk_gain_q; p.qk_gain_k = a.qk_gain_k; p.n_q_heads = a.n_q_heads; p.qk_eps = a.qk_eps;
   p.panel = (size_t)a.M * a.K * sizeof(bf16) > (48u << 20) ? 1 : 0;
   p.ksplit = 1; p.split_stride = 0; p.balanced = 0; p.sw_first = 0; p.sw_parts = 1; p.sw_kpb = 0; p.flags = nullptr; p.slots = nullptr;
+  p.swiglu_tma = 0;
   p.ce_mode = 0; p.ce_tiles = 0; p.ce_part = nullptr; p.ce_zy = nullptr; p.ce_lse = nullptr; p.ce_labels = nullptr;
   p.ce_sc = nullptr; p.ce_scale = 1.0f;
   const int tiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN);
@@ -1380,6 +1501,16 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream, int* lau
     cudaError_t e0 = cudaMemsetAsync(flags, 0, kScratchFlagFloats * sizeof(float), stream);
     if (e0 != cudaSuccess) return e0;
   }
+  EpiMaps em;
+  memset(&em, 0, sizeof(em));
+  p.swiglu_tma = 0;
+  if (MODE == 2 && a.epi == EPI_SWIGLU_BWD && !a.adam && g_gemm_swiglu_tma && (reinterpret_cast<uintptr_t>(a.gu) & 15) == 0 &&
+      (reinterpret_cast<uintptr_t>(a.C) & 15) == 0 && a.ldc % 8 == 0) {
+    // gate | up of the forward pass [M, 2 f] and the output d_gate / d_up [M, 2 f] (row stride ldc) as TMA tiles
+    if (make_tmap_2d_rows32(&em.gu, a.gu, 2ULL * a.d_ffn, a.M, 2ULL * a.d_ffn, 32) &&
+        make_tmap_2d_rows32(&em.dgu, reinterpret_cast<const bf16*>(a.C), 2ULL * a.d_ffn, a.M, a.ldc, 64))
+      p.swiglu_tma = 1;
+  }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs, 1, 1);
   // eight epilogue warps only for the fused update (for short contractions, whose epilogue is the long pole too, they
@@ -1397,7 +1528,7 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream, int* lau
   cfg.attrs = attr;
   cfg.numAttrs = 2;
   if (launches) *launches = ksplit > 1 ? 2 : 1;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, p);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, em, p);
   if (e != cudaSuccess || ksplit == 1) return e;
   const long long n4 = (long long)a.M * (a.N / 4);
   if (a.adam) {

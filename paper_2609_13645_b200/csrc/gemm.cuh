@@ -97,5 +97,6 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream, int* launches = 
 extern int g_gemm_force_bn;
 extern int g_gemm_pairs;
 extern int g_gemm_balanced;
+extern int g_gemm_swiglu_tma;
 
 }  // namespace fs

@@ -42,6 +42,21 @@ inline bool make_tmap_2d(CUtensorMap* tm, const bf16* base, uint64_t cols, uint6
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 2-D map with a box of 32 rows x box_cols columns (32: 64-byte rows under the 64-byte swizzle; 64: 128-byte rows under
+// the 128-byte swizzle): the tiles a warp of a GEMM epilogue moves between its staging buffer and a row-major matrix.
+inline bool make_tmap_2d_rows32(CUtensorMap* tm, const bf16* base, uint64_t cols, uint64_t rows, uint64_t row_stride,
+                                uint32_t box_cols) {
+  EncodeTiledFn enc = get_encode_fn();
+  if (!enc || (box_cols != 32 && box_cols != 64)) return false;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {row_stride * sizeof(bf16)};
+  cuuint32_t box[2] = {box_cols, 32};
+  cuuint32_t estr[2] = {1, 1};
+  return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<bf16*>(base), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, box_cols == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // 3-D map over [batches][rows][row_stride] (row-major, batches contiguous): box = 64 columns x box_rows rows x 1 batch.
 // Rows past the end of a batch read as zero instead of running into the next batch.
 inline bool make_tmap_3d(CUtensorMap* tm, const bf16* base, uint64_t cols, uint64_t rows, uint64_t batches,

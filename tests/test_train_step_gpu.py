@@ -608,7 +608,9 @@ def test_swiglu_backward_inside_the_data_gradient_epilogue_changes_no_bit(shape)
     reads gate and up, and writes d_gate | d_up.  Same element function on the same rounded value as the separate
     elementwise pass, so losses, norms and the whole optimizer state must equal that path bit for bit.  Shapes: the
     CTA-pair kernel; an ffn width whose last 32-column chunk is half empty; few tokens (single-CTA kernel); a tile count
-    that divides the last wave along K (partials completed before the epilogue); muP factors with recomputation."""
+    that divides the last wave along K (partials completed before the epilogue); muP factors with recomputation.  The
+    fused epilogue has two forms (gate / up and the result moved as TMA tiles through shared memory, or one row per thread
+    with plain loads and stores): both are run."""
     from paper_2609_13645_b200 import binding as B
     kw, recompute = {}, 0
     if shape == "c1":
@@ -628,19 +630,25 @@ def test_swiglu_backward_inside_the_data_gradient_epilogue_changes_no_bit(shape)
                              emb_scale=12.0, resid_scale=0.7, logit_scale=0.5, max_grad_norm=1.0)
         Bsz, S, recompute = 2, 512, 1
     runs = []
-    for fused in (True, False):
-        model = B.Model(lib_config(B, ocfg, Bsz, S, recompute=recompute), seed=9)
-        model.set_fused_swiglu_bwd(fused)
-        out = []
-        for s in range(3):
-            tok, lab = SI.batch(ocfg.vocab, Bsz, S, "zipf", step=s)
-            out.append(model.train_step(to_dev(tok), to_dev(lab)))
+    # fused with the epilogue's tiles moved by TMA (the default), fused with one row per thread, separate pass
+    for fused, tma in ((True, 1), (True, 0), (False, 1)):
+        B.lib().ft_debug_gemm_swiglu_tma(tma)
+        try:
+            model = B.Model(lib_config(B, ocfg, Bsz, S, recompute=recompute), seed=9)
+            model.set_fused_swiglu_bwd(fused)
+            out = []
+            for s in range(3):
+                tok, lab = SI.batch(ocfg.vocab, Bsz, S, "zipf", step=s)
+                out.append(model.train_step(to_dev(tok), to_dev(lab)))
+        finally:
+            B.lib().ft_debug_gemm_swiglu_tma(1)
         runs.append((model, out))
-    (mf, lf), (mu, lu) = runs
-    assert lf == lu
-    for a, b in zip(_state_bits(mf), _state_bits(mu)):
-        assert np.array_equal(a, b)
+    (mf, lf), (mr, lr), (mu, lu) = runs
+    assert lf == lu and lr == lu
+    for a, b, c in zip(_state_bits(mf), _state_bits(mr), _state_bits(mu)):
+        assert np.array_equal(a, c) and np.array_equal(b, c)
     mf.close()
+    mr.close()
     mu.close()
 
 
