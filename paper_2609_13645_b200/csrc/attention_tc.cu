@@ -22,13 +22,6 @@ namespace {
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRefSlack = 8.0f;
 
-#ifdef FS_ATTN_TRACE
-__device__ long long g_trace[8192];
-#define FS_TRACE(slot) do { if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) g_trace[(slot)] = clock64(); } while (0)
-#else
-#define FS_TRACE(slot) do { } while (0)
-#endif
-
 // barrier slots of the forward kernel
 enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 4, B_VFULL = 7, B_VEMPTY = 9, B_SFULL = 11, B_PFULL = 13, B_ODONE = 15,
        B_COUNT = 16 };
@@ -490,7 +483,6 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
       bool ok = mbar_wait(bar(BB_YEMPTY + st), (((uint32_t)(it / C::NST)) & 1u) ^ 1u, abort_flag, err);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
-      if (lane == 0 && it < 100) FS_TRACE(it * 16 + 10);
       const uint32_t ydst = sbase + C::OFF_Y + st * 2 * C::Y_BYTES;
       if constexpr (MODE == MODE_DQ) {
         if (lane == 0) {
@@ -561,14 +553,11 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
           if (!mbar_wait(bar(BB_YFULL + y1s), ((uint32_t)((it + 1) / C::NST)) & 1u, abort_flag, err)) { ok = false; break; }
           // the TMEM columns this writes were last read by this same thread's accumulating MMAs of block it-1: in order
           tc_fence_after();
-          if (side == 0 && it < 100) FS_TRACE(it * 16 + 0);
           issue_sdp(it + 1);
-          if (side == 0 && it < 100) FS_TRACE(it * 16 + 1);
         }
         const int bf = it & 1;
         if (!mbar_wait(bar(BB_TFULL + bf), ((uint32_t)it >> 1) & 1u, abort_flag, err)) { ok = false; break; }
         tc_fence_after();
-        if (side == 0 && it < 100) FS_TRACE(it * 16 + 2);
         const int yst = it % C::NST;
         const uint32_t y1 = sbase + C::OFF_Y + yst * 2 * C::Y_BYTES, y2 = y1 + C::Y_BYTES;
         // A operands (bf16 P^T / dS^T) sit in TMEM where S / dP were: 16 queries (K = 16) = 8 columns; the two
@@ -586,7 +575,6 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
           }
         }
         umma_commit(bar(BB_YEMPTY + yst));
-        if (side == 0 && it < 100) FS_TRACE(it * 16 + 3);
       }
       if (ok) umma_commit(bar(BB_ACCDONE));
     }
@@ -611,12 +599,10 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      if (threadIdx.x == 64 && it < 100) FS_TRACE(it * 16 + 4);
       uint32_t rs[32], rp[32];
       tmem_ld32(tlane + (uint32_t)(bf * 128 + ch * 32), rs);
       tmem_ld32(tlane + (uint32_t)(bf * 128 + 64 + ch * 32), rp);
       tmem_ld_wait();
-      if (threadIdx.x == 64 && it < 100) FS_TRACE(it * 16 + 5);
 
       int y0;
       const int yst = it % C::NST;
@@ -674,7 +660,6 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
           }
         }
       }
-      if (threadIdx.x == 64 && it < 100) FS_TRACE(it * 16 + 6);
       // bf16 pairs back into TMEM, over this warp's own (already loaded) fp32 columns
       uint32_t wp[16], wd[16];
 #pragma unroll
@@ -685,11 +670,9 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
       if constexpr (MODE == MODE_DKV) tmem_st16(tlane + (uint32_t)(bf * 128 + ch * 32), wp);
       tmem_st16(tlane + (uint32_t)(bf * 128 + 64 + ch * 32), wd);
       tmem_st_wait();
-      if (threadIdx.x == 64 && it < 100) FS_TRACE(it * 16 + 8);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(BB_TFULL + bf));
-      if (threadIdx.x == 64 && it < 100) FS_TRACE(it * 16 + 9);
       if constexpr (MODE == MODE_DKV) {
         // after the arrival, off the MMA chain's critical path: the same rounded dS also goes to the dS^T scratch
         // of the dQ contraction that follows (S % 128 == 0 there)
@@ -850,13 +833,5 @@ cudaError_t attention_bwd(const bf16* qkv, const bf16* o, const bf16* d_o, const
                           const float* cs, const float* sn, int B, int S, int nh, int nkv, int d, int* err, cudaStream_t st) {
   return attention_bwd_ws(qkv, o, d_o, lse, delta, dqkv, cs, sn, nullptr, 0, B, S, nh, nkv, d, err, st);
 }
-
-#ifdef FS_ATTN_TRACE
-}  // namespace fs
-extern "C" int ft_debug_attn_trace(long long* host_dst, int n) {
-  return (int)cudaMemcpyFromSymbol(host_dst, fs::g_trace, sizeof(long long) * n);
-}
-namespace fs {
-#endif
 
 }  // namespace fs

@@ -241,19 +241,6 @@ __device__ __forceinline__ void store8_bf16(bf16* dst, const float* v) {
   *reinterpret_cast<uint4*>(dst) = o;
 }
 
-#ifdef FS_GEMM_TRACE
-// development trace: per CTA pair and piece, globaltimer at (accumulator ready, partials ready, epilogue done)
-__device__ unsigned long long g_gemm_trace[148 * 32 * 4];
-__device__ __forceinline__ unsigned long long gtimer() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-#define FS_GTRACE(pair, piece, k) do { if ((piece) < 32) g_gemm_trace[((pair) * 32 + (piece)) * 4 + (k)] = gtimer(); } while (0)
-#else
-#define FS_GTRACE(pair, piece, k) do { } while (0)
-#endif
-
 constexpr int SLOT_FLOATS = 256 * 256;  // one fp32 partial tile of a CTA pair
 
 // Partial accumulators of the same output tile that other CTA pairs left in scratch.  A slot holds a pair's 256 x 256
@@ -1200,9 +1187,6 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     int acc = 0;
     uint32_t acc_phase = 0;
     float sq = 0.f;  // fused AdamW: this thread's share of the squared gradient norm
-    [[maybe_unused]] int piece = 0;
-    [[maybe_unused]] const bool tracer = (warp == 2 && lane == 0 && rank == 0);
-    if (tracer) FS_GTRACE(pair, 31, 0);
     while (work.next(tile, kb0, kb1, part, split)) {
       int mi, ni;
       tile_coords(p.panel, tile, tiles_m, tiles_n, mi, ni);
@@ -1223,7 +1207,6 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int row = m0 + q * 32 + lane;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
       const int slot_f4 = slot_thread_f4((int)rank, q, lane);
-      if (tracer) { FS_GTRACE(pair, piece, 0); FS_GTRACE(pair, piece, 1); }
       if (!reducer) {
         // an earlier K part of a divided tile: leave this partial accumulator in the pair's slot
         float4* dst = reinterpret_cast<float4*>(p.slots) + (long long)pair * SLOT_F4 + slot_f4;
@@ -1254,7 +1237,6 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             for (int s = 0; s < fx.n && got; ++s) got = flag_wait(p.flags + first + s, 2 * ((int)blockDim.x / 32 - 2), abort_flag, p.err) ? 1 : 0;
           got = __shfl_sync(0xffffffffu, got, 0);
           if (!got) break;
-          if (tracer) FS_GTRACE(pair, piece, 1);
         } else if (p.ksplit > 1) {
           cptr = reinterpret_cast<float*>(p.C) + (long long)part * p.split_stride;  // this K part's own fp32 partial output
         }
@@ -1271,8 +1253,6 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_leader(tempty_bar(acc));
-      if (tracer) FS_GTRACE(pair, piece, 2);
-      ++piece;
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
     }
@@ -1546,14 +1526,6 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream, int* lau
 }
 
 }  // namespace
-
-#ifdef FS_GEMM_TRACE
-}  // namespace fs
-extern "C" int ft_debug_gemm_trace(unsigned long long* host_dst, int n) {
-  return (int)cudaMemcpyFromSymbol(host_dst, fs::g_gemm_trace, sizeof(unsigned long long) * n);
-}
-namespace fs {
-#endif
 
 int g_gemm_force_bn = 0;
 int g_gemm_pairs = 1;  // development knob: 1 = CTA-pair kernel for outputs of at least 256 x 256, 0 = single-CTA kernel only  // development knob: 0 = choose by tile count, 128 or 256 = force that tile width
