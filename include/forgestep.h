@@ -280,8 +280,9 @@ typedef enum {
 ft_status ft_set_profiling(ft_model* m, int32_t enable);
 ft_status ft_get_profile(ft_model* m, int32_t cls, double* ms, double* work, int64_t* launches);
 /* The GEMM class broken down by (M, N, K, a_mn, b_mn, epilogue): entry i of the table built while profiling was on;
- * FT_ENOTFOUND past the end.  shape = {M, N, K, a_mn, b_mn, epilogue kind}. */
-ft_status ft_get_gemm_profile(ft_model* m, int32_t i, int32_t shape[6], double* ms, int64_t* launches);
+ * FT_ENOTFOUND past the end.  shape = {M, N, K, a_mn, b_mn, epilogue kind, M2, N2}: M2 x N2 is the second output of a
+ * launch that computed two weight gradients over the same K at once (0, 0 otherwise); its work is 2 K (M N + M2 N2). */
+ft_status ft_get_gemm_profile(ft_model* m, int32_t i, int32_t shape[8], double* ms, int64_t* launches);
 
 /* Message of the last call on this model that returned a non-zero status (owned by the model; "null model" for NULL).
  * Error behaviour of the whole boundary: nothing aborts, traps or throws; a device-side wait that ran out, a token id or

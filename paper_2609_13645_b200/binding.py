@@ -78,6 +78,8 @@ def lib():
         L.ft_debug_gemm_pairs.restype = None
         L.ft_debug_gemm_swiglu_tma.argtypes = [i32]
         L.ft_debug_gemm_swiglu_tma.restype = None
+        L.ft_debug_gemm_group.argtypes = [i32]
+        L.ft_debug_gemm_group.restype = None
         L.ft_get_gemm_profile.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(C.c_double), C.POINTER(i64)]
         L.ft_get_gemm_profile.restype = C.c_int
         L.ft_set_fused_update.argtypes = [vp, i32]
@@ -174,6 +176,10 @@ class Model:
 
     def close(self):
         if self._h:
+            # the library also works on streams of its own (weight gradients): nothing of this model may still be running
+            # when its workspace goes back to the allocator
+            import torch
+            torch.cuda.synchronize()
             lib().ft_destroy(self._h)
             self._h = C.c_void_p()
 
@@ -321,17 +327,18 @@ class Model:
         return out
 
     def get_gemm_profile(self):
-        """List of dicts (M, N, K, a_mn, b_mn, epi, ms, launches, tflops) for every GEMM shape seen while profiling."""
+        """List of dicts (M, N, K, a_mn, b_mn, epi, M2, N2, ms, launches, tflops) for every GEMM shape seen while profiling;
+        M2 x N2: the second output of a launch that computed two weight gradients at once (0 otherwise)."""
         out, i = [], 0
         while True:
-            shp, ms, n = (C.c_int32 * 6)(), C.c_double(), C.c_int64()
+            shp, ms, n = (C.c_int32 * 8)(), C.c_double(), C.c_int64()
             st = lib().ft_get_gemm_profile(self._h, i, shp, C.byref(ms), C.byref(n))
             if st == FT_ENOTFOUND:
                 break
             self._check(st)
-            M, N, K = shp[0], shp[1], shp[2]
-            out.append(dict(M=M, N=N, K=K, a_mn=shp[3], b_mn=shp[4], epi=shp[5], ms=ms.value, launches=int(n.value),
-                            tflops=2.0 * M * N * K * n.value / (ms.value * 1e-3) / 1e12 if ms.value > 0 else 0.0))
+            M, N, K, M2, N2 = shp[0], shp[1], shp[2], shp[6], shp[7]
+            out.append(dict(M=M, N=N, K=K, a_mn=shp[3], b_mn=shp[4], epi=shp[5], M2=M2, N2=N2, ms=ms.value, launches=int(n.value),
+                            tflops=2.0 * (M * N + M2 * N2) * K * n.value / (ms.value * 1e-3) / 1e12 if ms.value > 0 else 0.0))
             i += 1
         return out
 

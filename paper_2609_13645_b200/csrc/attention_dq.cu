@@ -110,7 +110,7 @@ attn_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_ds, const __grid_cons
         const int b = z / n_heads, h = z % n_heads, kvh = h / n_rep;
         const int q0 = qt * DQ_BM, kblocks = (q0 + DQ_BM) / DQ_BK;
         for (int kb = 0; kb < kblocks; ++kb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, err)) { ok = false; break; }
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, err, kWaitLimitCycles, 0x51)) { ok = false; break; }
           const uint32_t fb = full_bar(stage);
           mbar_expect_tx(fb, C::STAGE_BYTES);
           const uint32_t a_dst = sbase + stage * C::STAGE_BYTES;
@@ -136,11 +136,11 @@ attn_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_ds, const __grid_cons
         int qt, z;
         tile_of(t, qt, z);
         const int kblocks = (qt * DQ_BM + DQ_BM) / DQ_BK;
-        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, err)) break;
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, err, kWaitLimitCycles, 0x52)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * D);
         for (int kb = 0; kb < kblocks; ++kb) {
-          if (!mbar_wait(full_bar(stage), phase, abort_flag, err)) { ok = false; break; }
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, err, kWaitLimitCycles, 0x53)) { ok = false; break; }
           tc_fence_after();
           const uint32_t a_addr = sbase + stage * C::STAGE_BYTES;
           const uint32_t b_addr = a_addr + C::A_BYTES;
@@ -168,7 +168,7 @@ attn_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_ds, const __grid_cons
       int qt, z;
       tile_of(t, qt, z);
       const int b = z / n_heads, h = z % n_heads;
-      bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, err);
+      bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, err, kWaitLimitCycles, 0x54);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();

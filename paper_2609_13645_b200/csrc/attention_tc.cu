@@ -115,7 +115,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         tma_load_3d(sbase + kc * (C::BQ * 128), &tmQ, bar(B_QFULL), n * D + kc * 64, q0, b);
       for (int j = 0; j < nb; ++j) {
         const int st = j % C::NK;
-        if (!mbar_wait(bar(B_KEMPTY + st), ((uint32_t)(j / C::NK) & 1u) ^ 1u, abort_flag, err)) break;
+        if (!mbar_wait(bar(B_KEMPTY + st), ((uint32_t)(j / C::NK) & 1u) ^ 1u, abort_flag, err, kWaitLimitCycles, 0x31)) break;
         mbar_expect_tx(bar(B_KFULL + st), C::KV_BYTES);
 #pragma unroll
         for (int kc = 0; kc < C::KC; ++kc)
@@ -128,7 +128,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     if (lane == 0) {
       for (int j = 0; j < nb; ++j) {
         const int st = j % C::NV;
-        if (!mbar_wait(bar(B_VEMPTY + st), ((uint32_t)(j / C::NV) & 1u) ^ 1u, abort_flag, err)) break;
+        if (!mbar_wait(bar(B_VEMPTY + st), ((uint32_t)(j / C::NV) & 1u) ^ 1u, abort_flag, err, kWaitLimitCycles, 0x32)) break;
         mbar_expect_tx(bar(B_VFULL + st), C::KV_BYTES);
 #pragma unroll
         for (int kc = 0; kc < C::KC; ++kc)
@@ -146,7 +146,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       // S_j overwrites the TMEM buffer that held P_{j-2}; PV_{j-2} was issued earlier by this thread, so it is ordered
       auto issue_s = [&](int j) -> bool {
         const int st = j % C::NK;
-        if (!mbar_wait(bar(B_KFULL + st), (uint32_t)(j / C::NK) & 1u, abort_flag, err)) return false;
+        if (!mbar_wait(bar(B_KFULL + st), (uint32_t)(j / C::NK) & 1u, abort_flag, err, kWaitLimitCycles, 0x33)) return false;
         tc_fence_after();
         const uint64_t dk = umma_desc_sw128(sbase + C::OFF_K + st * C::KV_BYTES, 0, 1024);
         const uint32_t d_tmem = tmem_base + (uint32_t)((j & 1) * C::BK);
@@ -160,13 +160,13 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         umma_commit(bar(B_KEMPTY + st));  // K_j is free as soon as S_j is done
         return true;
       };
-      bool ok = mbar_wait(bar(B_QFULL), 0, abort_flag, err);
+      bool ok = mbar_wait(bar(B_QFULL), 0, abort_flag, err, kWaitLimitCycles, 0x34);
       if (ok) ok = issue_s(0);
       for (int j = 0; j < nb && ok; ++j) {
         if (j + 1 < nb && !issue_s(j + 1)) { ok = false; break; }
         const int st = j % C::NV;
-        if (!mbar_wait(bar(B_VFULL + st), (uint32_t)(j / C::NV) & 1u, abort_flag, err)) { ok = false; break; }
-        if (!mbar_wait(bar(B_PFULL + (j & 1)), ((uint32_t)j >> 1) & 1u, abort_flag, err)) { ok = false; break; }
+        if (!mbar_wait(bar(B_VFULL + st), (uint32_t)(j / C::NV) & 1u, abort_flag, err, kWaitLimitCycles, 0x35)) { ok = false; break; }
+        if (!mbar_wait(bar(B_PFULL + (j & 1)), ((uint32_t)j >> 1) & 1u, abort_flag, err, kWaitLimitCycles, 0x36)) { ok = false; break; }
         tc_fence_after();
         const uint64_t dv = umma_desc_sw128(sbase + C::OFF_V + st * C::KV_BYTES, C::BK * 128, 1024);
         const uint32_t tp = tmem_base + (uint32_t)((j & 1) * C::BK);  // bf16 P: 16 keys = 8 columns per K step
@@ -187,7 +187,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     float mref = -INFINITY, lsum = 0.f;
     bool ok = true;
     for (int j = 0; j < nb; ++j) {
-      ok = mbar_wait(bar(B_SFULL + (j & 1)), ((uint32_t)j >> 1) & 1u, abort_flag, err);
+      ok = mbar_wait(bar(B_SFULL + (j & 1)), ((uint32_t)j >> 1) & 1u, abort_flag, err, kWaitLimitCycles, 0x37);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -233,7 +233,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       // O has to be rescaled only when this row's integer reference moved (rare after the first blocks); only then
       // does the softmax wait for the previous P V product
       if (j > 0 && __any_sync(0xffffffffu, alpha != 1.0f)) {
-        ok = mbar_wait(bar(B_ODONE), (uint32_t)(j - 1) & 1u, abort_flag, err);
+        ok = mbar_wait(bar(B_ODONE), (uint32_t)(j - 1) & 1u, abort_flag, err, kWaitLimitCycles, 0x38);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
@@ -257,11 +257,11 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     // A parity wait can only tell two consecutive phases apart.  Seeing S_j guarantees P V products up to block j-2
     // (they were issued before S_j), so after the last block the products nb-2 and nb-1 are waited for in turn.
     if (ok && nb >= 2) {
-      ok = mbar_wait(bar(B_ODONE), (uint32_t)(nb - 2) & 1u, abort_flag, err);
+      ok = mbar_wait(bar(B_ODONE), (uint32_t)(nb - 2) & 1u, abort_flag, err, kWaitLimitCycles, 0x39);
       ok = __all_sync(0xffffffffu, ok);
     }
     if (ok) {
-      ok = mbar_wait(bar(B_ODONE), (uint32_t)(nb - 1) & 1u, abort_flag, err);
+      ok = mbar_wait(bar(B_ODONE), (uint32_t)(nb - 1) & 1u, abort_flag, err, kWaitLimitCycles, 0x3a);
       ok = __all_sync(0xffffffffu, ok);
     }
     if (ok) {
@@ -480,7 +480,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
     }
     for (int it = 0; it < iters; ++it) {
       const int st = it % C::NST;
-      bool ok = mbar_wait(bar(BB_YEMPTY + st), (((uint32_t)(it / C::NST)) & 1u) ^ 1u, abort_flag, err);
+      bool ok = mbar_wait(bar(BB_YEMPTY + st), (((uint32_t)(it / C::NST)) & 1u) ^ 1u, abort_flag, err, kWaitLimitCycles, 0x41);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       const uint32_t ydst = sbase + C::OFF_Y + st * 2 * C::Y_BYTES;
@@ -542,7 +542,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
         }
         umma_commit(bar(BB_SDPFULL + (it & 1)));
       };
-      bool ok = mbar_wait(bar(BB_XFULL), 0, abort_flag, err) && mbar_wait(bar(BB_YFULL), 0, abort_flag, err);
+      bool ok = mbar_wait(bar(BB_XFULL), 0, abort_flag, err, kWaitLimitCycles, 0x42) && mbar_wait(bar(BB_YFULL), 0, abort_flag, err, kWaitLimitCycles, 0x43);
       if (ok) {
         tc_fence_after();
         issue_sdp(0);
@@ -550,13 +550,13 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
       for (int it = 0; it < iters && ok; ++it) {
         if (it + 1 < iters) {
           const int y1s = (it + 1) % C::NST;
-          if (!mbar_wait(bar(BB_YFULL + y1s), ((uint32_t)((it + 1) / C::NST)) & 1u, abort_flag, err)) { ok = false; break; }
+          if (!mbar_wait(bar(BB_YFULL + y1s), ((uint32_t)((it + 1) / C::NST)) & 1u, abort_flag, err, kWaitLimitCycles, 0x44)) { ok = false; break; }
           // the TMEM columns this writes were last read by this same thread's accumulating MMAs of block it-1: in order
           tc_fence_after();
           issue_sdp(it + 1);
         }
         const int bf = it & 1;
-        if (!mbar_wait(bar(BB_TFULL + bf), ((uint32_t)it >> 1) & 1u, abort_flag, err)) { ok = false; break; }
+        if (!mbar_wait(bar(BB_TFULL + bf), ((uint32_t)it >> 1) & 1u, abort_flag, err, kWaitLimitCycles, 0x45)) { ok = false; break; }
         tc_fence_after();
         const int yst = it % C::NST;
         const uint32_t y1 = sbase + C::OFF_Y + yst * 2 * C::Y_BYTES, y2 = y1 + C::Y_BYTES;
@@ -595,7 +595,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
     bool ok = true;
     for (int it = 0; it < iters; ++it) {
       const int bf = it & 1;
-      ok = mbar_wait(bar(BB_SDPFULL + bf), ((uint32_t)it >> 1) & 1u, abort_flag, err);
+      ok = mbar_wait(bar(BB_SDPFULL + bf), ((uint32_t)it >> 1) & 1u, abort_flag, err, kWaitLimitCycles, 0x46);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -612,7 +612,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
         y0 = it * 64;
       } else {
         y0 = (qb0 + it % per_head) * 64;
-        ok = mbar_wait(bar(BB_YFULL + yst), ((uint32_t)(it / C::NST)) & 1u, abort_flag, err);  // acquire the staged statistics
+        ok = mbar_wait(bar(BB_YFULL + yst), ((uint32_t)(it / C::NST)) & 1u, abort_flag, err, kWaitLimitCycles, 0x47);  // acquire the staged statistics
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
       }
@@ -686,7 +686,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_qkv128, const __grid_c
       }
     }
     if (ok) {
-      ok = mbar_wait(bar(BB_ACCDONE), 0, abort_flag, err);
+      ok = mbar_wait(bar(BB_ACCDONE), 0, abort_flag, err, kWaitLimitCycles, 0x48);
       ok = __all_sync(0xffffffffu, ok);
     }
     if (ok) {

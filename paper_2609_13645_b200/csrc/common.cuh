@@ -62,8 +62,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false when the limit ran out or another thread of the CTA already gave up
 // (*abort_flag != 0); in that case it records the reason in *err (global) and raises *abort_flag (shared).
+// site: a small code of the waiting place, kept in the status word above its low byte (the error kind) for diagnosis.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* err,
-                                          long long limit_cycles = kWaitLimitCycles) {
+                                          long long limit_cycles = kWaitLimitCycles, int site = 0) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t it = 1;; ++it) {
@@ -72,7 +73,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (*abort_flag != 0) return false;
       if (clock64() - t0 > limit_cycles) {
         *abort_flag = 1;
-        atomicExch(err, (int)ERR_WAIT_TIMEOUT);
+        atomicExch(err, (int)ERR_WAIT_TIMEOUT | (site << 8));
         return false;
       }
     }

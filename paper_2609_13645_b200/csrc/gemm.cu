@@ -18,6 +18,7 @@ namespace fs {
 int g_pdl = 1;
 int g_gemm_balanced = 1;  // development knob: 0 = always the round-robin tile schedule
 int g_gemm_swiglu_tma = 1;  // development knob: 0 = SwiGLU-backward epilogue with per-thread loads and stores
+int g_gemm_group = 1;       // development knob: 0 = never two weight gradients in one launch
 
 namespace {
 
@@ -62,6 +63,18 @@ struct GemmDev {
   float alpha;             // accumulator scale (1: off)
   int wide_store;          // 1: C, ldc and N allow 32-byte stores (bf16 output)
   int swiglu_tma;          // SwiGLU-backward epilogue of the pair kernel: gate/up in and d_gate/d_up out as TMA tiles
+  // grouped launch (pair kernel, weight gradients): tiles [0, g_tiles0) are this problem's, the tiles after them belong to
+  // a second output with the same K whose operand maps travel in AuxMaps and whose fields below replace C, ldc, M, N,
+  // panel, alpha and the AdamW pointers in its tiles' loads and epilogues (g_tiles0 = 0: one problem)
+  int g_tiles0;
+  int g_M, g_N, g_panel;
+  long long g_ldc;
+  void* g_C;
+  float g_alpha;
+  float* g_adam_p;
+  float* g_adam_m;
+  float* g_adam_v;
+  bf16* g_adam_pb;
   float* qk_r;             // per-head QK-Norm in the RoPE epilogue (null: off)
   const bf16* qk_gain_q;
   const bf16* qk_gain_k;
@@ -201,7 +214,7 @@ __device__ __forceinline__ bool flag_wait(const int* flag, int target, volatile 
       if (*abort_flag != 0) return false;
       if (clock64() - t0 > kWaitLimitCycles) {
         *abort_flag = 1;
-        atomicExch(err, (int)ERR_WAIT_TIMEOUT);
+        atomicExch(err, (int)ERR_WAIT_TIMEOUT | (0x25 << 8));
         return false;
       }
     }
@@ -826,7 +839,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tile_coords(p.panel, t, tiles_m, tiles_n, mi, ni);
         const int m0 = mi * BM, n0 = ni * BN;
         for (int kb = 0; kb < kblocks; ++kb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.err)) { ok = false; break; }
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.err, kWaitLimitCycles, 0x11)) { ok = false; break; }
           const uint32_t fb = full_bar(stage);
           mbar_expect_tx(fb, C::STAGE_BYTES);
           const uint32_t a_dst = smem_u32(smem + stage * C::STAGE_BYTES);
@@ -858,11 +871,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t acc_phase = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
-        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.err)) break;
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.err, kWaitLimitCycles, 0x12)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
         for (int kb = 0; kb < kblocks; ++kb) {
-          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.err)) { ok = false; break; }
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.err, kWaitLimitCycles, 0x13)) { ok = false; break; }
           tc_fence_after();
           const uint32_t a_addr = smem_u32(smem + stage * C::STAGE_BYTES);
           const uint32_t b_addr = a_addr + A_BYTES;
@@ -894,7 +907,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int m0 = mi * BM, n0 = ni * BN;
       if (p.adam_p != nullptr) adam_prefetch_chunk(p, p.C, m0 + q * 32 + lane, n0);
       if constexpr (MODE == 2) swiglu_bwd_prefetch(p, m0 + q * 32 + lane, n0, BN);
-      bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.err);
+      bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.err, kWaitLimitCycles, 0x14);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -929,19 +942,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
 }
 
-// Tensor maps of an epilogue that moves its tiles through the TMA unit (SwiGLU backward): the forward pass' gate | up
-// [T, 2f] in boxes of 32 rows x 32 columns, and the output d_gate / d_up (interleaved 16 | 16) in boxes of 32 x 64.
-struct EpiMaps {
-  CUtensorMap gu;
-  CUtensorMap dgu;
+// Two more tensor maps of a launch.  SwiGLU backward (its epilogue moves tiles through the TMA unit): m0 = the forward
+// pass' gate | up [T, 2f] in boxes of 32 rows x 32 columns, m1 = the output d_gate / d_up (interleaved 16 | 16) in boxes
+// of 32 x 64.  Grouped weight gradients: m0, m1 = operands A and B of the second problem.
+struct AuxMaps {
+  CUtensorMap m0;
+  CUtensorMap m1;
 };
 
 // One warp's load of the gate and up tiles (32 rows x 32 logical columns from column gc) into its staging buffer
-__device__ __forceinline__ void swiglu_bwd_tma_fetch(const GemmDev& p, const EpiMaps& em, uint32_t buf, uint32_t bar, int gc,
+__device__ __forceinline__ void swiglu_bwd_tma_fetch(const GemmDev& p, const AuxMaps& em, uint32_t buf, uint32_t bar, int gc,
                                                      int row0) {
   mbar_expect_tx(bar, 4096);
-  tma_load_2d(buf, &em.gu, bar, gc, row0);
-  tma_load_2d(buf + 2048, &em.gu, bar, p.d_ffn + gc, row0);
+  tma_load_2d(buf, &em.m0, bar, gc, row0);
+  tma_load_2d(buf + 2048, &em.m0, bar, p.d_ffn + gc, row0);
 }
 
 // SwiGLU backward with the epilogue's memory traffic on the TMA unit.  The register path above reads gate and up and
@@ -955,7 +969,7 @@ __device__ __forceinline__ void swiglu_bwd_tma_fetch(const GemmDev& p, const Epi
 // step; the load/store pipe falls to 13 % of its peak, and what remains over the plain data gradient (124 us) is the
 // epilogue's bytes themselves on the L2-to-SM path that the operand loads already fill.
 // buf: 8 KB, 1024-byte aligned: gate, up, output tile.  Returns false when a bounded wait ran out.
-__device__ __forceinline__ bool epilogue_swiglu_bwd_tma(const GemmDev& p, const EpiMaps& em, uint32_t taddr, int row0, int n0,
+__device__ __forceinline__ bool epilogue_swiglu_bwd_tma(const GemmDev& p, const AuxMaps& em, uint32_t taddr, int row0, int n0,
                                                         int cb, int ce, const Fixup& fx, uint32_t buf, uint32_t bar,
                                                         uint32_t& phase, volatile int* abort_flag) {
   const int lane = threadIdx.x & 31;
@@ -965,7 +979,7 @@ __device__ __forceinline__ bool epilogue_swiglu_bwd_tma(const GemmDev& p, const 
   for (int c = cb; c < ce; c += 32) {
     const int gc = n0 + c;
     if (gc >= p.N) break;
-    bool ok = mbar_wait(bar, phase, abort_flag, p.err);
+    bool ok = mbar_wait(bar, phase, abort_flag, p.err, kWaitLimitCycles, 0x26);
     ok = __all_sync(0xffffffffu, ok);
     if (!ok) return false;
     phase ^= 1u;
@@ -1008,7 +1022,7 @@ __device__ __forceinline__ bool epilogue_swiglu_bwd_tma(const GemmDev& p, const 
     fence_proxy_async_smem();
     __syncwarp();
     if (lane == 0) {
-      tma_store_2d(&em.dgu, buf + 4096u, 2 * gc, row0);
+      tma_store_2d(&em.m1, buf + 4096u, 2 * gc, row0);
       bulk_commit_group();
     }
   }
@@ -1041,7 +1055,10 @@ constexpr int PAIR_THREADS = 320;
 template <bool A_MN, bool B_MN, int MODE = 0>
 __global__ void __launch_bounds__(PAIR_THREADS, 1)
 gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                    const __grid_constant__ EpiMaps em, const GemmDev p) {
+                    const __grid_constant__ AuxMaps em, const __grid_constant__ GemmDev p,
+                    const __grid_constant__ GemmDev p2) {
+  // p2 (grouped launch, MODE 3): p with C, ldc, M, N, panel, alpha and the AdamW pointers of the second problem; a copy
+  // of p otherwise.  Both live in parameter space, so the epilogue's reads of either cost what they cost in the other modes.
   using C = PairCfg;
   constexpr int BN = C::BN;
   extern __shared__ uint8_t smem_raw[];
@@ -1074,12 +1091,16 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
     if constexpr (MODE == 2)
       for (int w = 0; w < 4; ++w) mbar_init(epi_ld_bar(w), 1);
+    if constexpr (MODE == 3) {
+      tma_prefetch_desc(&em.m0);
+      tma_prefetch_desc(&em.m1);
+    }
     *abort_flag = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmA);
     tma_prefetch_desc(&tmB);
     if constexpr (MODE == 2) {
-      if (p.swiglu_tma) { tma_prefetch_desc(&em.gu); tma_prefetch_desc(&em.dgu); }
+      if (p.swiglu_tma) { tma_prefetch_desc(&em.m0); tma_prefetch_desc(&em.m1); }
     }
   }
   if (warp == 1) {
@@ -1096,7 +1117,11 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
   const int tiles_m = (p.M + 255) / 256;
   const int tiles_n = (p.N + BN - 1) / BN;
-  const int tiles_mn = tiles_m * tiles_n;
+  const int tiles0 = tiles_m * tiles_n;
+  constexpr bool grouped = MODE == 3;  // tiles from tiles0 on belong to the second problem
+  const int g_tiles_m = grouped ? (p.g_M + 255) / 256 : 0;
+  const int g_tiles_n = grouped ? (p.g_N + BN - 1) / BN : 0;
+  const int tiles_mn = tiles0 + g_tiles_m * g_tiles_n;
   const int kblocks_all = (p.K + BK - 1) / BK;
   WorkIter work(p, tiles_mn, kblocks_all, pair, npairs);
   int tile, kb0, kb1, part;
@@ -1109,27 +1134,31 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       bool ok = true;
       while (ok && work.next(tile, kb0, kb1, part, split)) {
         int mi, ni;
-        tile_coords(p.panel, tile, tiles_m, tiles_n, mi, ni);
+        const bool second = grouped && tile >= tiles0;
+        if (second) tile_coords(p.g_panel, tile - tiles0, g_tiles_m, g_tiles_n, mi, ni);
+        else tile_coords(p.panel, tile, tiles_m, tiles_n, mi, ni);
+        const CUtensorMap* mapA = second ? &em.m0 : &tmA;
+        const CUtensorMap* mapB = second ? &em.m1 : &tmB;
         const int m0 = mi * 256 + (int)rank * BM;        // this CTA's rows of A / of the output
         const int nb0 = ni * BN + (int)rank * C::HALF_B;  // this CTA's rows of B
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.err)) { ok = false; break; }
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.err, kWaitLimitCycles, 0x21 | (MODE << 8))) { ok = false; break; }
           const uint32_t fb = full_bar(stage);
           if (rank == 0) mbar_expect_tx(fb, 2 * C::STAGE_BYTES);
           const uint32_t a_dst = smem_u32(smem + stage * C::STAGE_BYTES);
           const uint32_t b_dst = a_dst + C::A_BYTES_;
           if constexpr (!A_MN) {
-            tma_load_2d_pair(a_dst, &tmA, fb, kb * BK, m0);
+            tma_load_2d_pair(a_dst, mapA, fb, kb * BK, m0);
           } else {
 #pragma unroll
-            for (int j = 0; j < BM / 64; ++j) tma_load_2d_pair(a_dst + j * CHUNK_BYTES, &tmA, fb, m0 + 64 * j, kb * BK);
+            for (int j = 0; j < BM / 64; ++j) tma_load_2d_pair(a_dst + j * CHUNK_BYTES, mapA, fb, m0 + 64 * j, kb * BK);
           }
           if constexpr (!B_MN) {
-            tma_load_2d_pair(b_dst, &tmB, fb, kb * BK, nb0);
+            tma_load_2d_pair(b_dst, mapB, fb, kb * BK, nb0);
           } else {
 #pragma unroll
             for (int j = 0; j < C::HALF_B / 64; ++j)
-              tma_load_2d_pair(b_dst + j * CHUNK_BYTES, &tmB, fb, nb0 + 64 * j, kb * BK);
+              tma_load_2d_pair(b_dst + j * CHUNK_BYTES, mapB, fb, nb0 + 64 * j, kb * BK);
           }
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -1146,11 +1175,11 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       uint32_t acc_phase = 0;
       bool ok = true;
       while (ok && work.next(tile, kb0, kb1, part, split)) {
-        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.err)) break;
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.err, kWaitLimitCycles, 0x22 | (MODE << 8))) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.err)) { ok = false; break; }
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.err, kWaitLimitCycles, 0x23 | (MODE << 8))) { ok = false; break; }
           tc_fence_after();
           const uint32_t a_addr = smem_u32(smem + stage * C::STAGE_BYTES);
           const uint32_t b_addr = a_addr + C::A_BYTES_;
@@ -1189,18 +1218,25 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     float sq = 0.f;  // fused AdamW: this thread's share of the squared gradient norm
     while (work.next(tile, kb0, kb1, part, split)) {
       int mi, ni;
-      tile_coords(p.panel, tile, tiles_m, tiles_n, mi, ni);
+      const bool second = grouped && tile >= tiles0;
+      if (second) tile_coords(p.g_panel, tile - tiles0, g_tiles_m, g_tiles_n, mi, ni);
+      else tile_coords(p.panel, tile, tiles_m, tiles_n, mi, ni);
+      const int pe_N = second ? p2.N : p.N;   // of the problem this tile belongs to
+      void* const pe_C = second ? p2.C : p.C;
       const int m0 = mi * 256 + (int)rank * BM;
       const int n0 = ni * BN;
       const bool reducer = !split || part == p.sw_parts - 1;  // this piece ends in the tile's epilogue
-      if (p.adam_p != nullptr && reducer) adam_prefetch_chunk(p, p.C, m0 + q * 32 + lane, n0 + cb);
+      if (p.adam_p != nullptr && reducer) {
+        if (second) adam_prefetch_chunk(p2, p2.C, m0 + q * 32 + lane, n0 + cb);
+        else adam_prefetch_chunk(p, p.C, m0 + q * 32 + lane, n0 + cb);
+      }
       // (asking one piece earlier instead, from the previous piece's epilogue, was slower: 219 us against 201 at c3_1b)
       [[maybe_unused]] const bool tma_tile = tma_epi && reducer && m0 + q * 32 < p.M && n0 + cb < p.N;
       if constexpr (MODE == 2) {
         if (reducer) swiglu_bwd_prefetch(p, m0 + q * 32 + lane, n0 + cb, ncols);
         if (tma_tile && lane == 0) swiglu_bwd_tma_fetch(p, em, tbuf, tbar, n0 + cb, m0 + q * 32);
       }
-      bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.err);
+      bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.err, kWaitLimitCycles, 0x24 | (MODE << 8));
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -1211,7 +1247,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         // an earlier K part of a divided tile: leave this partial accumulator in the pair's slot
         float4* dst = reinterpret_cast<float4*>(p.slots) + (long long)pair * SLOT_F4 + slot_f4;
         uint32_t r[32];
-        for (int c = cb; c < ce && n0 + c < p.N; c += 32) {
+        for (int c = cb; c < ce && n0 + c < pe_N; c += 32) {
           tmem_ld32(taddr + c, r);
           tmem_ld_wait();
 #pragma unroll
@@ -1225,7 +1261,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (lane == 0) atomicAdd(p.flags + pair, 1);
       } else {
         Fixup fx;
-        void* cptr = p.C;
+        void* cptr = pe_C;
         if (split && p.sw_parts > 1) {
           // last part of a divided tile: wait for the other parts (they run at the same time on the pairs just below
           // this one, which were started earlier) and add them in pair order
@@ -1246,6 +1282,9 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           } else {
             epilogue_tile<BN, MODE>(p, cptr, taddr, row, n0, sq, stage, cb, ce, fx);
           }
+        } else if constexpr (MODE == 3) {
+          if (second) epilogue_tile<BN, 0>(p2, cptr, taddr, row, n0, sq, stage, cb, ce, fx);
+          else epilogue_tile<BN, 0>(p, cptr, taddr, row, n0, sq, stage, cb, ce, fx);
         } else {
           epilogue_tile<BN, MODE>(p, cptr, taddr, row, n0, sq, stage, cb, ce, fx);
         }
@@ -1394,6 +1433,8 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
   p.panel = (size_t)a.M * a.K * sizeof(bf16) > (48u << 20) ? 1 : 0;
   p.ksplit = 1; p.split_stride = 0; p.balanced = 0; p.sw_first = 0; p.sw_parts = 1; p.sw_kpb = 0; p.flags = nullptr; p.slots = nullptr;
   p.swiglu_tma = 0;
+  p.g_tiles0 = 0; p.g_M = 0; p.g_N = 0; p.g_panel = 0; p.g_ldc = 0; p.g_C = nullptr; p.g_alpha = 1.0f;
+  p.g_adam_p = nullptr; p.g_adam_m = nullptr; p.g_adam_v = nullptr; p.g_adam_pb = nullptr;
   p.ce_mode = 0; p.ce_tiles = 0; p.ce_part = nullptr; p.ce_zy = nullptr; p.ce_lse = nullptr; p.ce_labels = nullptr;
   p.ce_sc = nullptr; p.ce_scale = 1.0f;
   const int tiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN);
@@ -1401,9 +1442,11 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
   return launch_pdl(kern, grid, GEMM_THREADS, C::SMEM_BYTES, stream, tmA, tmB, p);
 }
 
+// b2: the second problem of a grouped launch (MODE 3 only; validated by gemm_group2_ok)
 template <bool A_MN, bool B_MN, int MODE = 0>
-cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream, int* launches) {
+cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream, int* launches, const GemmArgs* b2 = nullptr) {
   using C = PairCfg;
+  if ((MODE == 3) != (b2 != nullptr)) return cudaErrorInvalidValue;
   auto kern = gemm_tc_pair_kernel<A_MN, B_MN, MODE>;
   static unsigned long long smem_set = 0;
   cudaError_t e0 = ensure_dynamic_smem(kern, C::SMEM_BYTES, smem_set);
@@ -1428,7 +1471,23 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream, int* lau
   }
   p.qk_r = a.qk_r; p.qk_gain_q = a.qk_gain_q; p.qk_gain_k = a.qk_gain_k; p.n_q_heads = a.n_q_heads; p.qk_eps = a.qk_eps;
   p.panel = (size_t)a.M * a.K * sizeof(bf16) > (48u << 20) ? 1 : 0;
-  const int tiles = ((a.M + 255) / 256) * ((a.N + 255) / 256);
+  int tiles = ((a.M + 255) / 256) * ((a.N + 255) / 256);
+  AuxMaps em;
+  memset(&em, 0, sizeof(em));
+  p.g_tiles0 = 0; p.g_M = 0; p.g_N = 0; p.g_panel = 0; p.g_ldc = 0; p.g_C = nullptr; p.g_alpha = 1.0f;
+  p.g_adam_p = nullptr; p.g_adam_m = nullptr; p.g_adam_v = nullptr; p.g_adam_pb = nullptr;
+  if (b2) {
+    const GemmArgs& b = *b2;
+    ok = A_MN ? make_tmap_2d(&em.m0, b.A, b.M, b.K, b.lda, 64) : make_tmap_2d(&em.m0, b.A, b.K, b.M, b.lda, BM);
+    ok = ok && (B_MN ? make_tmap_2d(&em.m1, b.B, b.N, b.K, b.ldb, 64) : make_tmap_2d(&em.m1, b.B, b.K, b.N, b.ldb, C::HALF_B));
+    if (!ok) return cudaErrorInvalidValue;
+    p.g_tiles0 = tiles;
+    p.g_M = b.M; p.g_N = b.N; p.g_ldc = b.ldc; p.g_C = b.C; p.g_alpha = b.alpha;
+    p.g_panel = (size_t)b.M * b.K * sizeof(bf16) > (48u << 20) ? 1 : 0;
+    if (b.adam) { p.g_adam_p = b.adam->p; p.g_adam_m = b.adam->m; p.g_adam_v = b.adam->v; p.g_adam_pb = b.adam->pb; }
+    if ((reinterpret_cast<uintptr_t>(b.C) & 31) != 0 || (b.ldc & 7) != 0 || (b.N & 7) != 0) p.wide_store = 0;
+    tiles += ((b.M + 255) / 256) * ((b.N + 255) / 256);
+  }
   const int max_pairs = sm_count() / 2;
   // scratch layout: 256 arrival counters (kept zero between launches), then fp32 partial tiles
   int* flags = reinterpret_cast<int*>(a.scratch);
@@ -1437,7 +1496,7 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream, int* lau
   const int kblocks = (a.K + BK - 1) / BK;
   // split-K for weight gradients whose output has too few tiles to occupy the machine
   int ksplit = 1;
-  if (A_MN && B_MN && (a.epi == EPI_F32 || a.epi == EPI_F32_ACC) && data && tiles * 2 <= max_pairs) {
+  if (A_MN && B_MN && !b2 && (a.epi == EPI_F32 || a.epi == EPI_F32_ACC) && data && tiles * 2 <= max_pairs) {
     int want = max_pairs / tiles;
     if (want > 8) want = 8;
     if (want > kblocks / 8) want = kblocks / 8;  // at least 8 K blocks per part
@@ -1481,14 +1540,12 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream, int* lau
     cudaError_t e0 = cudaMemsetAsync(flags, 0, kScratchFlagFloats * sizeof(float), stream);
     if (e0 != cudaSuccess) return e0;
   }
-  EpiMaps em;
-  memset(&em, 0, sizeof(em));
   p.swiglu_tma = 0;
   if (MODE == 2 && a.epi == EPI_SWIGLU_BWD && !a.adam && g_gemm_swiglu_tma && (reinterpret_cast<uintptr_t>(a.gu) & 15) == 0 &&
       (reinterpret_cast<uintptr_t>(a.C) & 15) == 0 && a.ldc % 8 == 0) {
     // gate | up of the forward pass [M, 2 f] and the output d_gate / d_up [M, 2 f] (row stride ldc) as TMA tiles
-    if (make_tmap_2d_rows32(&em.gu, a.gu, 2ULL * a.d_ffn, a.M, 2ULL * a.d_ffn, 32) &&
-        make_tmap_2d_rows32(&em.dgu, reinterpret_cast<const bf16*>(a.C), 2ULL * a.d_ffn, a.M, a.ldc, 64))
+    if (make_tmap_2d_rows32(&em.m0, a.gu, 2ULL * a.d_ffn, a.M, 2ULL * a.d_ffn, 32) &&
+        make_tmap_2d_rows32(&em.m1, reinterpret_cast<const bf16*>(a.C), 2ULL * a.d_ffn, a.M, a.ldc, 64))
       p.swiglu_tma = 1;
   }
   cudaLaunchConfig_t cfg = {};
@@ -1508,7 +1565,12 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream, int* lau
   cfg.attrs = attr;
   cfg.numAttrs = 2;
   if (launches) *launches = ksplit > 1 ? 2 : 1;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, em, p);
+  GemmDev p2 = p;
+  if (b2) {
+    p2.M = p.g_M; p2.N = p.g_N; p2.ldc = p.g_ldc; p2.C = p.g_C; p2.panel = p.g_panel; p2.alpha = p.g_alpha;
+    p2.adam_p = p.g_adam_p; p2.adam_m = p.g_adam_m; p2.adam_v = p.g_adam_v; p2.adam_pb = p.g_adam_pb;
+  }
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, em, p, p2);
   if (e != cudaSuccess || ksplit == 1) return e;
   const long long n4 = (long long)a.M * (a.N / 4);
   if (a.adam) {
@@ -1579,6 +1641,39 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream, int* launches) {
   if (!a.a_mn && a.b_mn) return wide ? launch_variant<256, false, true>(a, stream) : launch_variant<128, false, true>(a, stream);
   if (a.a_mn && a.b_mn) return wide ? launch_variant<256, true, true>(a, stream) : launch_variant<128, true, true>(a, stream);
   return cudaErrorInvalidValue;  // (mn-major A with k-major B) is not needed by the train step
+}
+
+bool gemm_group2_ok(const GemmArgs& a, const GemmArgs& b) {
+  if (!g_gemm_group || !g_gemm_pairs || g_gemm_force_bn) return false;
+  if (!a.a_mn || !a.b_mn || !b.a_mn || !b.b_mn) return false;  // weight gradients only
+  if (a.K != b.K || a.K <= 0 || a.M < 256 || a.N < 256 || b.M < 256 || b.N < 256) return false;
+  if (a.epi != b.epi || (a.epi != EPI_F32 && a.epi != EPI_F32_ACC)) return false;
+  if (a.ce_mode || b.ce_mode || a.err != b.err || !a.err) return false;
+  if (a.scratch != b.scratch || a.scratch_bytes != b.scratch_bytes) return false;
+  if ((a.adam == nullptr) != (b.adam == nullptr)) return false;
+  if (a.adam) {
+    const AdamFuse &x = *a.adam, &y = *b.adam;
+    if (x.scalars != y.scalars || x.lr != y.lr || x.beta1 != y.beta1 || x.beta2 != y.beta2 || x.eps != y.eps || x.wd != y.wd)
+      return false;
+    if (!y.p || !y.m || !y.v || !y.pb) return false;
+  }
+  // the second problem's operands and output must pass the checks launch_gemm makes for the first
+  if ((b.N & 7) || (b.lda & 7) || (b.ldb & 7) || (b.ldc & 3) || (b.M & 7)) return false;
+  if (!b.A || !b.B || !b.C) return false;
+  if ((reinterpret_cast<uintptr_t>(b.A) | reinterpret_cast<uintptr_t>(b.B) | reinterpret_cast<uintptr_t>(b.C)) & 15) return false;
+  return true;
+}
+
+cudaError_t launch_gemm_group2(const GemmArgs& a, const GemmArgs& b, cudaStream_t stream, int* launches) {
+  if (launches) *launches = 1;
+  if (!gemm_group2_ok(a, b)) return cudaErrorInvalidValue;
+  if (a.M <= 0 || a.N <= 0 || !a.A || !a.B || !a.C) return cudaErrorInvalidValue;
+  if ((a.N & 7) || (a.lda & 7) || (a.ldb & 7) || (a.ldc & 3) || (a.M & 7)) return cudaErrorInvalidValue;
+  if ((reinterpret_cast<uintptr_t>(a.A) | reinterpret_cast<uintptr_t>(a.B) | reinterpret_cast<uintptr_t>(a.C)) & 15)
+    return cudaErrorInvalidValue;
+  if (a.adam && (!a.adam->p || !a.adam->m || !a.adam->v || !a.adam->pb || !a.adam->scalars || !a.adam->sq_slots))
+    return cudaErrorInvalidValue;
+  return launch_pair_variant<true, true, 3>(a, stream, launches, &b);
 }
 
 }  // namespace fs

@@ -94,6 +94,15 @@ struct GemmArgs {
 // given) receives the number of kernels the call enqueued (2 for a split-K contraction with its reduction, else 1).
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream, int* launches = nullptr);
 
+// Two weight gradients (both operands mn-major, the same contraction length K, the same fp32 / AdamW epilogue kind) as
+// ONE launch of the CTA-pair kernel: the tiles of `b` follow the tiles of `a` in the persistent schedule, so the last,
+// partly filled wave of `a` and its exposed optimizer epilogue run beside the first tiles of `b`.  Every tile is computed
+// exactly as a launch of its own would compute a whole tile; which tiles the balanced schedule divides along K depends on
+// the combined tile count.  gemm_group2_ok says whether the pair qualifies (otherwise: two launch_gemm calls).
+bool gemm_group2_ok(const GemmArgs& a, const GemmArgs& b);
+cudaError_t launch_gemm_group2(const GemmArgs& a, const GemmArgs& b, cudaStream_t stream, int* launches = nullptr);
+
+extern int g_gemm_group;
 extern int g_gemm_force_bn;
 extern int g_gemm_pairs;
 extern int g_gemm_balanced;

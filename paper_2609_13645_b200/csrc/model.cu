@@ -161,7 +161,7 @@ struct ft_model {
 
   // optional per-class timing with CUDA events on the model's stream
   struct ProfRec { cudaEvent_t a, b; int cls; double work; int shape; };
-  struct GemmShape { int M, N, K, a_mn, b_mn, epi; double ms; long long launches; };
+  struct GemmShape { int M, N, K, a_mn, b_mn, epi, M2, N2; double ms; long long launches; };  // M2, N2: second output of a grouped launch
   std::vector<GemmShape> prof_shapes;
   bool prof = false;
   std::vector<ProfRec> prof_pending;
@@ -404,6 +404,18 @@ ft_status cuda_fail(ft_model* m, cudaError_t e, const char* where) {
     m->launches += nl__;                                                                    \
     prof_end(m, FT_PROF_GEMM, 2.0 * (double)(args).M * (double)(args).N * (double)(args).K, 1, prof_shape_index(m, args)); \
   } while (0)
+// two weight gradients as one launch (gemm_group2_ok(a0, a1) holds)
+#define FT_GEMM_GROUP_ON(a0, a1, stream_)                                                   \
+  do {                                                                                      \
+    prof_begin(m);                                                                          \
+    int nl__ = 1;                                                                           \
+    cudaError_t e__ = launch_gemm_group2(a0, a1, stream_, &nl__);                           \
+    if (e__ != cudaSuccess) return cuda_fail(m, e__, "launch_gemm_group2");                 \
+    m->launches += nl__;                                                                    \
+    prof_end(m, FT_PROF_GEMM,                                                               \
+             2.0 * (double)(a0).K * ((double)(a0).M * (double)(a0).N + (double)(a1).M * (double)(a1).N), 1, \
+             prof_shape_index(m, a0, &(a1)));                                               \
+  } while (0)
 
 cudaEvent_t prof_event(ft_model* m) {
   if (!m->prof_pool.empty()) { cudaEvent_t e = m->prof_pool.back(); m->prof_pool.pop_back(); return e; }
@@ -441,13 +453,15 @@ void prof_collect(ft_model* m) {
 }
 
 // index of this GEMM's (shape, layout, epilogue) in the per-shape profile table
-int prof_shape_index(ft_model* m, const GemmArgs& g) {
+int prof_shape_index(ft_model* m, const GemmArgs& g, const GemmArgs* second = nullptr) {
   if (!m->prof) return -1;
+  const int M2 = second ? second->M : 0, N2 = second ? second->N : 0;
   for (size_t i = 0; i < m->prof_shapes.size(); ++i) {
     const auto& s = m->prof_shapes[i];
-    if (s.M == g.M && s.N == g.N && s.K == g.K && s.a_mn == g.a_mn && s.b_mn == g.b_mn && s.epi == g.epi) return (int)i;
+    if (s.M == g.M && s.N == g.N && s.K == g.K && s.a_mn == g.a_mn && s.b_mn == g.b_mn && s.epi == g.epi && s.M2 == M2 && s.N2 == N2)
+      return (int)i;
   }
-  ft_model::GemmShape s = {g.M, g.N, g.K, g.a_mn, g.b_mn, g.epi, 0.0, 0};
+  ft_model::GemmShape s = {g.M, g.N, g.K, g.a_mn, g.b_mn, g.epi, M2, N2, 0.0, 0};
   m->prof_shapes.push_back(s);
   return (int)m->prof_shapes.size() - 1;
 }
@@ -542,12 +556,56 @@ ft_status wait_wgrad(ft_model* m, int k) {
   return FT_OK;
 }
 
+// A weight gradient whose launch is put off until the next one of the layer is ready, so that both run as one launch
+struct WgradHold {
+  GemmArgs g;
+  int k = -1;
+  bool valid = false;
+};
+
+// Enqueues the weight gradient g (slot k of the layer's four) and, when `held` holds one, that one with it: as ONE grouped
+// launch when the two qualify (the partly filled last wave and the exposed optimizer epilogue of the first then run
+// beside the second's tiles), else as two launches.  On the second stream when the step overlaps, after every data
+// gradient enqueued so far (they still read the bf16 weights the fused update overwrites).
+ft_status wgrad_launch(ft_model* m, GemmArgs g, int k, WgradHold* held) {
+  const bool have = held != nullptr && held->valid;
+  cudaStream_t on = m->stream;
+  if (m->overlapping) {
+    ft_status s = wait_wgrad(m, k);  // one weight gradient per slot in flight
+    if (s) return s;
+    if (have && (s = wait_wgrad(m, held->k))) return s;
+    FT_CUDA(cudaEventRecord(m->ev_d, m->stream));
+    FT_CUDA(cudaStreamWaitEvent(m->side, m->ev_d, 0));
+    g.scratch = m->splitk2;
+    if (have) held->g.scratch = m->splitk2;
+    on = m->side;
+  }
+  if (have && gemm_group2_ok(held->g, g)) {
+    FT_GEMM_GROUP_ON(held->g, g, on);
+  } else {
+    if (have) FT_GEMM_ON(held->g, on);
+    FT_GEMM_ON(g, on);
+  }
+  if (m->overlapping) {
+    FT_CUDA(cudaEventRecord(m->ev_w[k], m->side));
+    m->w_pending[k] = true;
+    if (have) {
+      FT_CUDA(cudaEventRecord(m->ev_w[held->k], m->side));
+      m->w_pending[held->k] = true;
+    }
+  }
+  if (held) held->valid = false;
+  return FT_OK;
+}
+
 // dX = dY W (data gradient) and dW = dY^T X (weight gradient, slot k of the layer's four)
 // alpha: factor the branch output carried into the residual stream (its gradient is alpha * dY, never rounded)
 // swiglu_gu: when given, X is the SwiGLU output a = silu(G) U of the gate|up tensor swiglu_gu [T, 2 n_in], dX is not
 // stored, and the data-gradient epilogue writes d_gate, d_up to swiglu_dgu [T, 2 n_in] (alternating 16 / 16 columns)
+// hold: the weight gradient is not enqueued but left there for a later call; join: a held one to enqueue with this one
 ft_status linear_backward(ft_model* m, const bf16* dY, const bf16* X, int wi, bf16* dX, int T, int n_out, int n_in, int k,
-                          float alpha = 1.0f, const bf16* swiglu_gu = nullptr, bf16* swiglu_dgu = nullptr) {
+                          float alpha = 1.0f, const bf16* swiglu_gu = nullptr, bf16* swiglu_dgu = nullptr,
+                          WgradHold* hold = nullptr, WgradHold* join = nullptr) {
   {
     GemmArgs g = gemm_base(m);
     g.A = dY; g.lda = n_out; g.B = m->wb(wi); g.b_mn = 1; g.ldb = n_in; g.C = dX; g.ldc = n_in;
@@ -562,20 +620,12 @@ ft_status linear_backward(ft_model* m, const bf16* dY, const bf16* X, int wi, bf
     g.A = dY; g.a_mn = 1; g.lda = n_out; g.B = X; g.b_mn = 1; g.ldb = n_in; g.C = m->gr(wi); g.ldc = n_in;
     g.M = n_out; g.N = n_in; g.K = T; g.epi = EPI_F32; g.alpha = alpha;
     if (m->fusing) g.adam = fuse_for(m, wi);
-    if (!m->overlapping) {
-      FT_GEMM(g);
-    } else {
-      ft_status s = wait_wgrad(m, k);  // one weight gradient per slot in flight
-      if (s) return s;
-      FT_CUDA(cudaEventRecord(m->ev_d, m->stream));
-      FT_CUDA(cudaStreamWaitEvent(m->side, m->ev_d, 0));
-      g.scratch = m->splitk2;
-      FT_GEMM_ON(g, m->side);
-      FT_CUDA(cudaEventRecord(m->ev_w[k], m->side));
-      m->w_pending[k] = true;
+    if (hold != nullptr) {
+      hold->g = g; hold->k = k; hold->valid = true;
+      return FT_OK;
     }
+    return wgrad_launch(m, g, k, join);
   }
-  return FT_OK;
 }
 
 ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
@@ -585,18 +635,20 @@ ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
   // m->dxA holds d_x_out
   if (tp) { ft_status s = copy_tap(m, tp->d_x_out, m->dxA, (size_t)T * h); if (s) return s; }
   ft_status s;
+  WgradHold held;
   if (m->fused_swiglu_bwd && !tp) {
     // d_a stays in the data-gradient GEMM's accumulators: its epilogue reads gate | up and writes d_gate | d_up
     if ((s = wait_wgrad(m, 1))) return s;  // the previous layer's gate/up weight gradient still reads d_gu
-    s = linear_backward(m, m->dxA, a.a, m->idx_layer(l, 5), nullptr, T, h, f, 0, m->cfg.resid_scale, a.gu, m->d_gu);
+    s = linear_backward(m, m->dxA, a.a, m->idx_layer(l, 5), nullptr, T, h, f, 0, m->cfg.resid_scale, a.gu, m->d_gu, &held);
     if (s) return s;
   } else {
-    s = linear_backward(m, m->dxA, a.a, m->idx_layer(l, 5), m->d_a, T, h, f, 0, m->cfg.resid_scale);
+    s = linear_backward(m, m->dxA, a.a, m->idx_layer(l, 5), m->d_a, T, h, f, 0, m->cfg.resid_scale, nullptr, nullptr, &held);
     if (s) return s;
     if ((s = wait_wgrad(m, 1))) return s;  // the previous layer's gate/up weight gradient still reads d_gu
     FT_LAUNCH(FT_PROF_ELEMENTWISE, 10.0 * T * f, swiglu_bwd(m->d_a, a.gu, m->d_gu, T, f, st));
   }
-  s = linear_backward(m, m->d_gu, a.h2, m->idx_layer(l, 4), m->d_h, T, 2 * f, h, 1);
+  // the down projection's weight gradient (held) and the gate/up one: one launch
+  s = linear_backward(m, m->d_gu, a.h2, m->idx_layer(l, 4), m->d_h, T, 2 * f, h, 1, 1.0f, nullptr, nullptr, nullptr, &held);
   if (s) return s;
   if (tp) {
     if ((s = copy_tap(m, tp->d_a, m->d_a, (size_t)T * f))) return s;
@@ -606,7 +658,7 @@ ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
   if ((s = wait_wgrad(m, 2))) return s;  // the previous layer's output-projection weight gradient still reads dxB
   FT_LAUNCH(FT_PROF_NORM, 8.0 * T * h, rmsnorm_bwd(m->d_h, a.x_mid, a.r2, m->wb(m->idx_layer(l, 3)), m->dxA, m->dxB,
                                                     norm_slot(m, m->idx_layer(l, 3)), T, h, st));
-  s = linear_backward(m, m->dxB, a.o, m->idx_layer(l, 2), m->d_o, T, h, hq, 2, m->cfg.resid_scale);
+  s = linear_backward(m, m->dxB, a.o, m->idx_layer(l, 2), m->d_o, T, h, hq, 2, m->cfg.resid_scale, nullptr, nullptr, &held);
   if (s) return s;
   if ((s = wait_wgrad(m, 3))) return s;  // the previous layer's qkv weight gradient still reads d_qkv
   prof_begin(m);
@@ -623,7 +675,8 @@ ft_status layer_backward(ft_model* m, int l, LayerActs& a, int B, int S) {
                          (size_t)elementwise_blocks_for_norm(m->maxT) * h, 1.0f / (m->rope_mscale * m->rope_mscale), T, S,
                          m->cfg.n_heads, m->cfg.n_kv_heads, m->d, st));
   }
-  s = linear_backward(m, m->d_qkv, a.h1, m->idx_layer(l, 1), m->d_h, T, nqkv, h, 3);
+  // the output projection's weight gradient (held) and the qkv one: one launch
+  s = linear_backward(m, m->d_qkv, a.h1, m->idx_layer(l, 1), m->d_h, T, nqkv, h, 3, 1.0f, nullptr, nullptr, nullptr, &held);
   if (s) return s;
   if (tp) {
     if ((s = copy_tap(m, tp->d_x_mid, m->dxB, (size_t)T * h))) return s;
@@ -898,14 +951,16 @@ __global__ void wait_probe_kernel(long long limit_cycles, int* err) {
     mbar_fence_init();
   }
   __syncthreads();
-  if (threadIdx.x == 0) mbar_wait(smem_u32(&bar), 0u, &abort_flag, err, limit_cycles);
+  if (threadIdx.x == 0) mbar_wait(smem_u32(&bar), 0u, &abort_flag, err, limit_cycles, 0x61);
   __syncthreads();
 }
 
 // a non-zero device status word as a status code
 ft_status device_status(ft_model* m, int err) {
-  if (err == (int)ERR_BAD_INDEX) return fail(m, FT_EINVAL, "a token id or label is outside [0, vocab) (ids were clamped, such labels ignored)");
-  return fail(m, FT_ETIMEOUT, "a device-side wait ran out of time");
+  if ((err & 0xff) == (int)ERR_BAD_INDEX) return fail(m, FT_EINVAL, "a token id or label is outside [0, vocab) (ids were clamped, such labels ignored)");
+  char msg[96];
+  snprintf(msg, sizeof(msg), "a device-side wait ran out of time (status word 0x%x: wait site 0x%x)", (unsigned)err, (unsigned)err >> 8);
+  return fail(m, FT_ETIMEOUT, msg);
 }
 
 // one synchronisation: reads the scalars back and turns device-side flags into a status
@@ -1602,6 +1657,7 @@ ft_status ft_get_profile(ft_model* m, int32_t cls, double* ms, double* work, int
 
 void ft_debug_gemm_tile(int32_t bn) { g_gemm_force_bn = bn; }
 void ft_debug_gemm_balanced(int32_t on) { g_gemm_balanced = on; }
+void ft_debug_gemm_group(int32_t on) { g_gemm_group = on; }
 void ft_debug_gemm_swiglu_tma(int32_t on) { g_gemm_swiglu_tma = on; }
 void ft_debug_pdl(int32_t on) { g_pdl = on; }
 void ft_debug_gemm_pairs(int32_t on) { g_gemm_pairs = on; }
@@ -1616,13 +1672,14 @@ ft_status ft_debug_wait_probe(ft_model* m, int64_t limit_cycles) {
   return FT_OK;
 }
 
-ft_status ft_get_gemm_profile(ft_model* m, int32_t i, int32_t shape[6], double* ms, int64_t* launches) {
+ft_status ft_get_gemm_profile(ft_model* m, int32_t i, int32_t shape[8], double* ms, int64_t* launches) {
   if (!m || !shape) return FT_EINVAL;
   FT_CUDA(cudaStreamSynchronize(m->stream));
   prof_collect(m);
   if (i < 0 || i >= (int32_t)m->prof_shapes.size()) return FT_ENOTFOUND;
   const auto& s = m->prof_shapes[i];
   shape[0] = s.M; shape[1] = s.N; shape[2] = s.K; shape[3] = s.a_mn; shape[4] = s.b_mn; shape[5] = s.epi;
+  shape[6] = s.M2; shape[7] = s.N2;
   if (ms) *ms = s.ms;
   if (launches) *launches = s.launches;
   return FT_OK;
