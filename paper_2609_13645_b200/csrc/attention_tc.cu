@@ -24,7 +24,7 @@ constexpr float kRefSlack = 8.0f;
 
 // barrier slots of the forward kernel
 enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 4, B_VFULL = 7, B_VEMPTY = 9, B_SFULL = 11, B_PFULL = 13, B_ODONE = 15,
-       B_COUNT = 16 };
+       B_OFINAL = 16, B_COUNT = 17 };
 constexpr int ATT_THREADS = 224;  // K producer, MMA issuer, 4 softmax warps, V producer
 
 template <int D>
@@ -90,6 +90,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       mbar_init(bar(B_PFULL + i), 4);
     }
     mbar_init(bar(B_ODONE), 1);
+    mbar_init(bar(B_OFINAL), 1);
     *abort_flag = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmQ);
@@ -177,6 +178,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         umma_commit(bar(B_VEMPTY + st));
         umma_commit(bar(B_ODONE));
       }
+      if (ok) umma_commit(bar(B_OFINAL));  // every product of this tile is done: a barrier of its own, one phase
     }
   } else {
     // ------------------------------------------------------------------ softmax warps (2..5)
@@ -254,14 +256,12 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(B_PFULL + (j & 1)));
     }
-    // A parity wait can only tell two consecutive phases apart.  Seeing S_j guarantees P V products up to block j-2
-    // (they were issued before S_j), so after the last block the products nb-2 and nb-1 are waited for in turn.
-    if (ok && nb >= 2) {
-      ok = mbar_wait(bar(B_ODONE), (uint32_t)(nb - 2) & 1u, abort_flag, err, kWaitLimitCycles, 0x39);
-      ok = __all_sync(0xffffffffu, ok);
-    }
+    // The end of the last P V product is signalled on a barrier of its own.  (B_ODONE cannot serve: a parity wait only
+    // tells two consecutive phases apart, and a warp that is slow to get here after its last arrival can find that
+    // barrier two phases on, products nb-2 AND nb-1 both done, which reads like "nb-2 still running": waiting for the
+    // two in turn ran into its time limit about once in 10^7 thread blocks.)
     if (ok) {
-      ok = mbar_wait(bar(B_ODONE), (uint32_t)(nb - 1) & 1u, abort_flag, err, kWaitLimitCycles, 0x3a);
+      ok = mbar_wait(bar(B_OFINAL), 0, abort_flag, err, kWaitLimitCycles, 0x39);
       ok = __all_sync(0xffffffffu, ok);
     }
     if (ok) {
