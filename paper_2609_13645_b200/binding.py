@@ -80,6 +80,8 @@ def lib():
         L.ft_debug_gemm_swiglu_tma.restype = None
         L.ft_debug_gemm_group.argtypes = [i32]
         L.ft_debug_gemm_group.restype = None
+        L.ft_debug_gemm_tma_out.argtypes = [i32]
+        L.ft_debug_gemm_tma_out.restype = None
         L.ft_get_gemm_profile.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(C.c_double), C.POINTER(i64)]
         L.ft_get_gemm_profile.restype = C.c_int
         L.ft_set_fused_update.argtypes = [vp, i32]

@@ -21,6 +21,9 @@ void ft_debug_gemm_balanced(int32_t on);
 /* 1 = the two pairs of weight gradients of a layer (down + gate/up, output + qkv projection) run as one launch each
  * (default), 0 = one launch per weight gradient. */
 void ft_debug_gemm_group(int32_t on);
+/* 1 = plain bf16 outputs of the CTA-pair GEMM leave as TMA tensor stores (default), 0 = one row per thread with 32-byte
+ * stores.  Both give the same bits. */
+void ft_debug_gemm_tma_out(int32_t on);
 /* 1 = the SwiGLU-backward epilogue of the CTA-pair GEMM moves gate / up and d_gate / d_up as TMA tiles through shared
  * memory (default), 0 = one row per thread with plain loads and stores.  Both give the same bits. */
 void ft_debug_gemm_swiglu_tma(int32_t on);

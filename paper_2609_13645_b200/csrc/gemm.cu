@@ -19,6 +19,7 @@ int g_pdl = 1;
 int g_gemm_balanced = 1;  // development knob: 0 = always the round-robin tile schedule
 int g_gemm_swiglu_tma = 1;  // development knob: 0 = SwiGLU-backward epilogue with per-thread loads and stores
 int g_gemm_group = 1;       // development knob: 0 = never two weight gradients in one launch
+int g_gemm_tma_out = 1;     // development knob: 0 = plain bf16 epilogue with per-thread stores
 
 namespace {
 
@@ -63,6 +64,7 @@ struct GemmDev {
   float alpha;             // accumulator scale (1: off)
   int wide_store;          // 1: C, ldc and N allow 32-byte stores (bf16 output)
   int swiglu_tma;          // SwiGLU-backward epilogue of the pair kernel: gate/up in and d_gate/d_up out as TMA tiles
+  int tma_out;             // plain bf16 epilogue of the pair kernel: output tiles leave as TMA stores (AuxMaps::m1 = C)
   // grouped launch (pair kernel, weight gradients): tiles [0, g_tiles0) are this problem's, the tiles after them belong to
   // a second output with the same K whose operand maps travel in AuxMaps and whose fields below replace C, ldc, M, N,
   // panel, alpha and the AdamW pointers in its tiles' loads and epilogues (g_tiles0 = 0: one problem)
@@ -1029,6 +1031,49 @@ __device__ __forceinline__ bool epilogue_swiglu_bwd_tma(const GemmDev& p, const 
   return true;
 }
 
+// Plain bf16 output through the TMA unit: a warp packs 32 rows x 64 columns of its accumulator into a 4 KB tile
+// (128-byte rows, 128-byte swizzle: no bank conflicts with one row per thread) and one lane sends it off as a tensor
+// store of full 128-byte lines, alternating between two tiles so that the store of one drains while the next is packed.
+// One row per thread with 32-byte global stores is bound by L2 store requests, which shows wherever the epilogue is not
+// hidden behind a main loop (short contractions, the last wave of any launch).  Same values, same rounding.
+// buf: 8 KB, 1024-byte aligned.
+__device__ __forceinline__ void epilogue_bf16_tma(const GemmDev& p, const AuxMaps& em, uint32_t taddr, int row0, int n0,
+                                                  int cb, int ce, const Fixup& fx, uint32_t buf) {
+  const int lane = threadIdx.x & 31;
+  const uint32_t sw = (uint32_t)(lane & 7);
+  uint32_t r[32];
+  int b = 0;
+  for (int c = cb; c < ce; c += 64) {
+    const int gc = n0 + c;
+    if (gc >= p.N) break;
+    uint32_t o[32];
+    ld_acc32(taddr, c, r, fx, p.alpha);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) o[i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+    if (gc + 32 < p.N) {
+      ld_acc32(taddr, c + 32, r, fx, p.alpha);
+#pragma unroll
+      for (int i = 0; i < 16; ++i) o[16 + i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+    } else {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) o[16 + i] = 0u;  // columns past N: dropped by the store
+    }
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");  // the store that last read this tile
+    __syncwarp();
+    const uint32_t tile = buf + (uint32_t)b * 4096u, trow = tile + (uint32_t)lane * 128u;
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      st_shared_v4(trow + (((uint32_t)j ^ sw) << 4), make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]));
+    fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+      tma_store_2d(&em.m1, tile, gc, row0);
+      bulk_commit_group();
+    }
+    b ^= 1;
+  }
+}
+
 // ---------------------------------------------------------------- CTA-pair variant
 // Two CTAs on neighbouring SMs (a cluster of 2) share one 256 x 256 output tile: each loads its own 128 rows of A and
 // its own 128 of the 256 rows of B, the leader issues tcgen05.mma.cta_group::2 (M = 256), and each CTA's TMEM ends up
@@ -1101,6 +1146,9 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     tma_prefetch_desc(&tmB);
     if constexpr (MODE == 2) {
       if (p.swiglu_tma) { tma_prefetch_desc(&em.m0); tma_prefetch_desc(&em.m1); }
+    }
+    if constexpr (MODE == 0) {
+      if (p.tma_out) tma_prefetch_desc(&em.m1);
     }
   }
   if (warp == 1) {
@@ -1285,6 +1333,12 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         } else if constexpr (MODE == 3) {
           if (second) epilogue_tile<BN, 0>(p2, cptr, taddr, row, n0, sq, stage, cb, ce, fx);
           else epilogue_tile<BN, 0>(p, cptr, taddr, row, n0, sq, stage, cb, ce, fx);
+        } else if constexpr (MODE == 0) {
+          if (p.tma_out) {
+            if (m0 + q * 32 < p.M) epilogue_bf16_tma(p, em, taddr, m0 + q * 32, n0, cb, ce, fx, tbuf);
+          } else {
+            epilogue_tile<BN, MODE>(p, cptr, taddr, row, n0, sq, stage, cb, ce, fx);
+          }
         } else {
           epilogue_tile<BN, MODE>(p, cptr, taddr, row, n0, sq, stage, cb, ce, fx);
         }
@@ -1301,6 +1355,9 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
     if constexpr (MODE == 2) {
       if (tma_epi && lane == 0) bulk_wait_group0();  // this warp's tensor stores have landed before the kernel ends
+    }
+    if constexpr (MODE == 0) {
+      if (p.tma_out && lane == 0) bulk_wait_group0();
     }
   }
 
@@ -1432,7 +1489,7 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t stream) {
   p.qk_r = a.qk_r; p.qk_gain_q = a.qk_gain_q; p.qk_gain_k = a.qk_gain_k; p.n_q_heads = a.n_q_heads; p.qk_eps = a.qk_eps;
   p.panel = (size_t)a.M * a.K * sizeof(bf16) > (48u << 20) ? 1 : 0;
   p.ksplit = 1; p.split_stride = 0; p.balanced = 0; p.sw_first = 0; p.sw_parts = 1; p.sw_kpb = 0; p.flags = nullptr; p.slots = nullptr;
-  p.swiglu_tma = 0;
+  p.swiglu_tma = 0; p.tma_out = 0;
   p.g_tiles0 = 0; p.g_M = 0; p.g_N = 0; p.g_panel = 0; p.g_ldc = 0; p.g_C = nullptr; p.g_alpha = 1.0f;
   p.g_adam_p = nullptr; p.g_adam_m = nullptr; p.g_adam_v = nullptr; p.g_adam_pb = nullptr;
   p.ce_mode = 0; p.ce_tiles = 0; p.ce_part = nullptr; p.ce_zy = nullptr; p.ce_lse = nullptr; p.ce_labels = nullptr;
@@ -1539,6 +1596,11 @@ cudaError_t launch_pair_variant(const GemmArgs& a, cudaStream_t stream, int* lau
   if (p.balanced && a.scratch_reset) {
     cudaError_t e0 = cudaMemsetAsync(flags, 0, kScratchFlagFloats * sizeof(float), stream);
     if (e0 != cudaSuccess) return e0;
+  }
+  p.tma_out = 0;
+  if (MODE == 0 && a.epi == EPI_BF16 && !a.adam && ksplit == 1 && g_gemm_tma_out && (reinterpret_cast<uintptr_t>(a.C) & 15) == 0 &&
+      a.ldc % 8 == 0) {
+    if (make_tmap_2d_rows32(&em.m1, reinterpret_cast<const bf16*>(a.C), a.N, a.M, a.ldc, 64)) p.tma_out = 1;
   }
   p.swiglu_tma = 0;
   if (MODE == 2 && a.epi == EPI_SWIGLU_BWD && !a.adam && g_gemm_swiglu_tma && (reinterpret_cast<uintptr_t>(a.gu) & 15) == 0 &&

@@ -103,6 +103,7 @@ bool gemm_group2_ok(const GemmArgs& a, const GemmArgs& b);
 cudaError_t launch_gemm_group2(const GemmArgs& a, const GemmArgs& b, cudaStream_t stream, int* launches = nullptr);
 
 extern int g_gemm_group;
+extern int g_gemm_tma_out;
 extern int g_gemm_force_bn;
 extern int g_gemm_pairs;
 extern int g_gemm_balanced;

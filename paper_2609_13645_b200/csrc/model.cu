@@ -1658,6 +1658,7 @@ ft_status ft_get_profile(ft_model* m, int32_t cls, double* ms, double* work, int
 void ft_debug_gemm_tile(int32_t bn) { g_gemm_force_bn = bn; }
 void ft_debug_gemm_balanced(int32_t on) { g_gemm_balanced = on; }
 void ft_debug_gemm_group(int32_t on) { g_gemm_group = on; }
+void ft_debug_gemm_tma_out(int32_t on) { g_gemm_tma_out = on; }
 void ft_debug_gemm_swiglu_tma(int32_t on) { g_gemm_swiglu_tma = on; }
 void ft_debug_pdl(int32_t on) { g_pdl = on; }
 void ft_debug_gemm_pairs(int32_t on) { g_gemm_pairs = on; }

@@ -165,3 +165,24 @@ def test_balanced_k_schedule_repeats_bit_for_bit_and_leaves_its_counters_clear()
         assert int(scratch[:256].view(torch.int32).abs().sum().item()) == 0
         outs.append(out.view(torch.int16).cpu().numpy())
     assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])
+
+
+@pytest.mark.parametrize("M,N,K,a_mn,b_mn,ws", [(1000, 1376, 256, 0, 0, False), (300, 328, 128, 0, 0, False),
+                                                 (2048, 4096, 512, 0, 0, False), (512, 688, 256, 0, 1, False),
+                                                 (8192, 2560, 2560, 0, 1, True), (4096, 768, 768, 0, 1, False)])
+def test_bf16_output_through_tensor_stores_changes_no_bit(M, N, K, a_mn, b_mn, ws):
+    """The plain bf16 epilogue of the CTA-pair kernel has two forms: tiles of 32 rows x 64 columns packed in shared memory
+    and sent off as TMA tensor stores (default), or one row per thread with 32-byte stores.  Same accumulators, same
+    rounding: the outputs must be equal bit for bit, ragged rows and columns, a balanced (K-divided) last wave and a
+    short contraction included."""
+    from paper_2609_13645_b200 import binding as B
+    outs = []
+    for on in (1, 0):
+        B.lib().ft_debug_gemm_tma_out(on)
+        try:
+            rel, got, _ = _run(M, N, K, a_mn, b_mn, 0, seed=5, ws=ws)
+        finally:
+            B.lib().ft_debug_gemm_tma_out(1)
+        assert rel < 2e-3, rel
+        outs.append(got)
+    assert np.array_equal(outs[0], outs[1])
