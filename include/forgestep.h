@@ -314,7 +314,8 @@ ft_status ft_k_gemm(const void* dev_A, int32_t a_mn, int64_t lda, const void* de
  * contracts over the token dimension, the long one).  Results stay bit-identical from run to run:
  *  - weight-gradient layout (a_mn = b_mn = 1, fp32 output) with few 256 x 256 output tiles: up to 8 K parts run
  *    concurrently into fp32 partial outputs and a second kernel adds them in index order;
- *  - any layout whose last wave of 256 x 256 tiles would keep at most half of the SM pairs busy: the tiles of that wave
+ *  - any layout with a contraction of at least 2560 (40 blocks of 64; below that the division costs more than it saves)
+ *    whose last wave of 256 x 256 tiles would keep at most half of the SM pairs busy: the tiles of that wave
  *    are divided into 2 to 8 K parts that run first, one part per pair; all parts but the last leave an fp32 partial
  *    tile in the scratch, and the pair holding the last part (the highest-numbered pair of the group, so that it only
  *    ever waits for pairs that were started before it) adds them in pair order before the usual epilogue.  The other
