@@ -273,25 +273,12 @@ def run_cuda(args):
     launches = model.launch_count - launches0
     graph_replays = model.graph_replays
 
-    # ---- (2) the same K steps launch by launch with CUDA events around every kernel: per-class times and roofline
-    model.set_profiling(True)
-    ev4, ev5 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    ev4.record()
-    for i in range(args.steps):
-        model.train_step(*dev_batches[args.warmup + i], want_loss=False)
-    ev5.record()
-    barrier()
-    ms_prof = ev4.elapsed_time(ev5)
-    prof = model.get_profile()
-    gemm_shapes = model.get_gemm_profile()
-    model.set_profiling(False)
-    loss_check = model.forward_loss(*dev_batches[0])
-
-    # ---- (3) end to end: host buffers in, loss out, every step
+    # ---- (2) end to end: host buffers in, loss out, every step (directly after the headline pass, so that both see
+    # the GPU in the same thermal state)
     pinned = [(torch.from_numpy(t).pin_memory(), torch.from_numpy(l).pin_memory()) for t, l in host_batches]
-    for i in range(min(2, args.warmup)):
-        model.train_step_host(pinned[i][0].numpy(), pinned[i][1].numpy())
+    for i in range(min(2, args.warmup)):  # through the same calls as the timed loop: their one-time set-up (the pinned
+        model.submit_step_host(pinned[i][0].numpy(), pinned[i][1].numpy())  # result ring, its events) happens here
+        model.collect_step()
     barrier()
     ev2, ev3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev2.record()
@@ -308,6 +295,22 @@ def run_cuda(args):
     ev3.record()
     barrier()
     ms_e2e = ev2.elapsed_time(ev3)
+
+
+    # ---- (3) the same K steps launch by launch with CUDA events around every kernel: per-class times and roofline
+    model.set_profiling(True)
+    ev4, ev5 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev4.record()
+    for i in range(args.steps):
+        model.train_step(*dev_batches[args.warmup + i], want_loss=False)
+    ev5.record()
+    barrier()
+    ms_prof = ev4.elapsed_time(ev5)
+    prof = model.get_profile()
+    gemm_shapes = model.get_gemm_profile()
+    model.set_profiling(False)
+    loss_check = model.forward_loss(*dev_batches[0])
 
     ms_total, ms_e2e, ms_prof = max_over_ranks([ms_total, ms_e2e, ms_prof], world, device="cuda")
 
