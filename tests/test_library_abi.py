@@ -30,6 +30,19 @@ def test_library_builds_loads_and_exports_every_declared_symbol():
         assert hasattr(lib, s), s
 
 
+def test_development_header_is_private_and_its_switches_are_exported():
+    """The development switches live in a header of their own inside the package, none of them in the boundary, and the
+    library exports each one (the kernel benchmarks and the ablation tests call them)."""
+    text = open(os.path.join(ROOT, "paper_2609_13645_b200", "csrc", "forgestep_debug.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    dbg = sorted(set(re.findall(r"\b(ft_debug_[a-z_0-9]+)\s*\(", text)))
+    assert len(dbg) >= 8 and not [s for s in declared_symbols() if s.startswith("ft_debug_")]
+    from paper_2609_13645_b200 import build
+    lib = ctypes.CDLL(build.build())
+    for s in dbg:
+        assert hasattr(lib, s), s
+
+
 def test_workspace_size_and_config_validation_run_on_the_host():
     from paper_2609_13645_b200 import binding as B
     ok = B.make_config(1, 256, 4, 4, 64, 688, 1024, 2, 128)
